@@ -1,0 +1,477 @@
+#!/usr/bin/env python
+"""Benchmark of the im2win hot path on B200.
+
+A step is one pass of the whole hot path over one batch of the headline layer
+(ResNet-style 3x3 layer, N=128 C=64 56x56 -> 64): im2win transform, filter
+pack and convolution, once in fp32 (CUDA cores) and once in fp16-in /
+fp32-accumulate (tensor cores).  The metric is convolution TFLOPS,
+2*N*Co*Ho*Wo*C*Kh*Kw per precision, over the device time of the whole step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--report FILE]
+
+prints one JSON line (rank 0).  `--report FILE` additionally times every layer
+of the workload table kernel by kernel and writes one JSON object per layer.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2608_20725_b200 import workloads  # noqa: E402
+
+METRIC = "conv TFLOPS (fp32 + fp16 passes of the layer, transform and filter pack included)"
+UNIT = "TFLOP/s"
+SM_COUNT = 148
+FP32_LANES_PER_SM = 128
+SM_MAX_GHZ = 1.965
+# fp32 FFMA peak from unit counts and the maximum SM clock: 148 * 128 lanes * 2 flop * 1.965 GHz
+FP32_PEAK_TFLOPS = SM_COUNT * FP32_LANES_PER_SM * 2 * SM_MAX_GHZ / 1e3
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            d = json.load(fh)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+def layer_flops(layer, ho, wo):
+    return 2.0 * layer.N * layer.Co * ho * wo * layer.C * layer.Kh * layer.Kw
+
+
+# --------------------------------------------------------------------- clocks ----
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm), "power_w_max": max(power) if power else None}
+
+
+# -------------------------------------------------------------- the GPU arm ----
+class LayerRunner:
+    """Device-resident buffers of one layer and the four calls of a step."""
+
+    def __init__(self, layer, precisions=("f32", "f16")):
+        from paper_2608_20725_b200 import binding
+        self.b = binding
+        self.layer = layer
+        self.dims = layer.dims()
+        x, f = workloads.make_inputs(layer)
+        self.host = {}
+        self.dev = {}
+        for prec in precisions:
+            tdt = torch.float32 if prec == "f32" else torch.float16
+            xh, fh = x.to(tdt).contiguous(), f.to(tdt).contiguous()
+            window, scratch, y = binding.alloc_layer_buffers(self.dims, tdt)
+            self.dev[prec] = dict(x=xh.cuda(), f=fh.cuda(), window=window, scratch=scratch, y=y)
+            self.host[prec] = (xh, fh)
+        code = binding.F32 if "f32" in precisions else binding.F16
+        _, _, self.ho, self.wo = binding.im2win_workspace_size(self.dims, code)
+        self.flops = layer_flops(layer, self.ho, self.wo)
+        self.precisions = precisions
+
+    def transform(self, prec):
+        d = self.dev[prec]
+        self.b.im2win_transform(d["x"], d["window"], self.dims)
+
+    def conv(self, prec):
+        d = self.dev[prec]
+        if prec == "f32":
+            self.b.im2win_conv_f32(d["window"], d["f"], d["y"], d["scratch"], self.dims)
+        else:
+            self.b.im2win_conv_f16(d["window"], d["f"], d["y"], d["scratch"], self.dims)
+
+    def step(self, events=None):
+        """One pass of the hot path; with `events` (list) records an event before/after each call."""
+        for prec in self.precisions:
+            for name, fn in (("transform", self.transform), ("conv", self.conv)):
+                if events is not None:
+                    e0 = torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                fn(prec)
+                if events is not None:
+                    e1 = torch.cuda.Event(enable_timing=True)
+                    e1.record()
+                    events.append((f"{name}_{prec}", e0, e1))
+
+    def algorithmic_bytes(self, kernel):
+        """Bytes each kernel must move once (stated per kernel in the design doc)."""
+        l, es = self.layer, (4 if kernel.endswith("f32") else 2)
+        x_el = l.N * l.C * l.H * l.W
+        win_el = l.N * l.C * self.ho * l.Kh * (l.W + 2 * l.pad)
+        out_el = l.N * l.Co * self.ho * self.wo
+        f_el = l.Co * l.C * l.Kh * l.Kw
+        if kernel.startswith("transform"):
+            return (x_el + win_el) * es
+        return win_el * es + f_el * es + out_el * 4
+
+    def memory_report(self):
+        l = self.layer
+        rep = {}
+        for prec in self.precisions:
+            es = 4 if prec == "f32" else 2
+            win = l.N * l.C * self.ho * l.Kh * (l.W + 2 * l.pad) * es
+            out = l.N * l.Co * self.ho * self.wo * 4
+            rep[prec] = {"window_bytes": win, "output_bytes": out, "window_plus_output_bytes": win + out,
+                         "scratch_bytes": self.dev[prec]["scratch"].numel(),
+                         "im2col_bytes": l.N * l.C * l.Kh * l.Kw * self.ho * self.wo * es}
+        return rep
+
+
+def kernel_rooflines(runner, avg_ms, peaks, peak_kind):
+    """Roofline entry of every call of the step from its average device time."""
+    out = {}
+    for name, ms in avg_ms.items():
+        sec = ms * 1e-3
+        nbytes = runner.algorithmic_bytes(name)
+        if name.startswith("transform"):
+            a = nbytes / sec / 1e9
+            out[name] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": a / peaks["hbm_gbs"], "peak_kind": peak_kind, "ms": ms}
+        elif name == "conv_f32":
+            a = runner.flops / sec / 1e12
+            out[name] = {"bound": "alu", "achieved": a, "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s",
+                         "frac": a / FP32_PEAK_TFLOPS, "peak_kind": "148 SM x 128 lanes x 2 x 1.965 GHz", "ms": ms}
+        else:
+            tf = runner.flops / sec / 1e12
+            # fp16 dense peak: measured bf16 GEMM peak (same tensor rate for fp16 and bf16)
+            tensor_peak = peaks["bf16_tflops"]
+            t_tensor = runner.flops / (tensor_peak * 1e12)
+            t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+            if t_hbm > t_tensor:
+                a = nbytes / sec / 1e9
+                out[name] = {"bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                             "frac": a / peaks["hbm_gbs"], "peak_kind": peak_kind, "ms": ms, "tflops": tf}
+            else:
+                out[name] = {"bound": "tensor", "achieved": tf, "peak": tensor_peak, "unit": "TFLOP/s",
+                             "frac": tf / tensor_peak, "peak_kind": peak_kind, "ms": ms, "tflops": tf}
+    return out
+
+
+def load_traffic():
+    """Per-launch DRAM traffic of each kernel from the committed ncu summary, if present."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as fh:
+            return json.load(fh)
+    except Exception:
+        return {}
+
+
+def time_cpu_oracle(layer, target_seconds=12.0):
+    """Times the oracle's im2win route (fp64, OpenMP) on a bounded slice of the batch."""
+    import numpy as np
+    import oracle
+    x, f = workloads.make_inputs(layer)
+    xn, fn = x.numpy(), f.numpy()
+    dims = layer.dims()
+    ho, wo = oracle.out_dims(dims)
+    per_image = layer_flops(layer, ho, wo) / layer.N
+    t0 = time.perf_counter()
+    oracle.conv_im2win_range(xn, fn, dims, 0, 1)
+    t1 = time.perf_counter() - t0
+    n = int(max(1, min(layer.N - 1, target_seconds / max(t1, 1e-6))))
+    t0 = time.perf_counter()
+    oracle.conv_im2win_range(xn, fn, dims, 1, 1 + n)
+    dt = time.perf_counter() - t0
+    return {"value": per_image * n / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"fp64 im2win route on {n} of {layer.N} images of {layer.name} ({dt:.1f} s)"}
+
+
+def run_gpu_arm(args):
+    from paper_2608_20725_b200 import binding
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    layer = workloads.LAYERS[workloads.BENCH_LAYER]
+    runner = LayerRunner(layer)
+    peaks, peak_kind = load_peaks()
+    torch.cuda.reset_peak_memory_stats()
+
+    for _ in range(args.warmup):
+        runner.step()
+    for prec in runner.precisions:
+        binding.im2win_check_status(runner.dev[prec]["scratch"])
+
+    # ---- timed region: K steps, device time, max over ranks --------------------
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    events = []
+    start = torch.cuda.Event(enable_timing=True)
+    stop = torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        runner.step(events)
+    stop.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = start.elapsed_time(stop)
+    for prec in runner.precisions:
+        binding.im2win_check_status(runner.dev[prec]["scratch"])
+    peak_alloc = torch.cuda.max_memory_allocated()
+
+    per_call = {}
+    for name, e0, e1 in events:
+        per_call.setdefault(name, []).append(e0.elapsed_time(e1))
+    avg_ms = {k: sum(v) / len(v) for k, v in per_call.items()}
+
+    # ---- end to end: host buffers, copies inside the timed region ---------------
+    e2e_sets = {}
+    for prec in runner.precisions:
+        xh, fh = runner.host[prec]
+        code = binding.F32 if prec == "f32" else binding.F16
+        nbytes = binding.im2win_layer_workspace_size(runner.dims, code)
+        e2e_sets[prec] = dict(x=xh.pin_memory(), f=fh.pin_memory(),
+                              y=torch.empty((layer.N, layer.Co, runner.ho, runner.wo), dtype=torch.float32).pin_memory(),
+                              ws=torch.empty(nbytes, dtype=torch.uint8, device="cuda"))
+
+    def e2e_step():
+        for prec in runner.precisions:
+            s = e2e_sets[prec]
+            binding.im2win_layer_forward_host(s["x"], s["f"], s["y"], s["ws"], runner.dims)
+
+    e2e_steps = max(1, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    es, ee = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    es.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    ee.record()
+    barrier()
+    e2e_ms = es.elapsed_time(ee)
+    h2d = sum(e2e_sets[p]["x"].numel() * e2e_sets[p]["x"].element_size()
+              + e2e_sets[p]["f"].numel() * e2e_sets[p]["f"].element_size() for p in runner.precisions)
+    d2h = sum(e2e_sets[p]["y"].numel() * 4 for p in runner.precisions)
+
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = times.tolist()
+
+    step_flops = runner.flops * len(runner.precisions)
+    value = world * step_flops * args.steps / (total_ms * 1e-3) / 1e12
+    e2e_value = world * step_flops * e2e_steps / (e2e_ms * 1e-3) / 1e12
+
+    rooflines = kernel_rooflines(runner, avg_ms, peaks, peak_kind)
+    traffic = load_traffic()
+    dominant = max(avg_ms, key=avg_ms.get)
+    roof = dict(rooflines[dominant])
+    roof["kernel"] = dominant
+    roof["traffic"] = traffic.get(f"{layer.name}:{dominant}")
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32+f16", "data": "synthetic",
+        "config": {"workload": f"{layer.name}: N={layer.N} C={layer.C} H=W={layer.H} Co={layer.Co} "
+                               f"K={layer.Kh}x{layer.Kw} stride={layer.stride} pad={layer.pad}, fp32 and fp16 passes",
+                   "l2": "working set per pass (input+window+output >= 360 MB) exceeds the 126 MB L2",
+                   "parallelism": f"batch replicas x{world}, no collective"},
+        "tflops": {p: runner.flops / (avg_ms[f"conv_{p}"] * 1e-3) / 1e12 for p in runner.precisions},
+        "tflops_with_transform": {p: runner.flops / ((avg_ms[f"conv_{p}"] + avg_ms[f"transform_{p}"]) * 1e-3) / 1e12
+                                  for p in runner.precisions},
+        "roofline": roof,
+        "kernels": rooflines,
+        "memory": dict(runner.memory_report(), torch_peak_allocated_bytes=peak_alloc),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": 6 * args.steps,
+        "clocks": clocks,
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = time_cpu_oracle(layer)
+        print(json.dumps(out))
+    if args.report and rank == 0:
+        write_report(args.report, peaks, peak_kind)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------- per-layer report ----
+def time_call(fn, iters, flush):
+    """Average device time (ms) of fn over `iters` launches, each preceded by an L2 flush."""
+    total = 0.0
+    best = float("inf")
+    for _ in range(iters):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        e1.synchronize()
+        ms = e0.elapsed_time(e1)
+        total += ms
+        best = min(best, ms)
+    return total / iters, best
+
+
+def write_report(path, peaks, peak_kind, names=None, iters=10):
+    from paper_2608_20725_b200 import binding
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
+    rows = []
+    table = dict(workloads.LAYERS)
+    table.update(workloads.TABLE1_LAYERS)
+    for name in (names or list(workloads.LAYERS)):
+        layer = table[name]
+        runner = LayerRunner(layer, layer.precisions)
+        for _ in range(3):
+            runner.step()
+        avg, best = {}, {}
+        for prec in layer.precisions:
+            for kind, fn in (("transform", runner.transform), ("conv", runner.conv)):
+                avg[f"{kind}_{prec}"], best[f"{kind}_{prec}"] = time_call(lambda: fn(prec), iters, flush)
+            binding.im2win_check_status(runner.dev[prec]["scratch"])
+        row = {"layer": name, "dims": layer.dims(), "gflop": runner.flops / 1e9, "avg_ms": avg, "best_ms": best,
+               "kernels": kernel_rooflines(runner, avg, peaks, peak_kind), "memory": runner.memory_report()}
+        rows.append(row)
+        del runner
+        torch.cuda.empty_cache()
+    os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+    with open(path, "w") as fh:
+        for row in rows:
+            fh.write(json.dumps(row) + "\n")
+
+
+# ------------------------------------------------------ the reference arm ----
+def run_reference_arm(args):
+    """Times the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    layer = workloads.LAYERS[workloads.BENCH_LAYER]
+    x, f = workloads.make_inputs(layer)
+    _, x16 = oracle.round_to_f16(x.numpy())
+    _, f16 = oracle.round_to_f16(f.numpy())
+    sets = {"f32": (x.numpy(), f.numpy()), "f16": (x16, f16)}
+    dims = layer.dims()
+    ho, wo = oracle.out_dims(dims)
+    n_img = 2                                   # images per precision per step: a bounded sample of the batch
+    flops_step = 2 * n_img * layer_flops(layer, ho, wo) / layer.N
+
+    def step(i):
+        for prec in ("f32", "f16"):
+            xs, fs = sets[prec]
+            b = (i * n_img) % (layer.N - n_img + 1)
+            oracle.conv_im2win_range(xs, fs, dims, b, b + n_img)
+
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    dt = time.perf_counter() - t0
+    value = flops_step * args.steps / dt / 1e12
+    sample = (f"fp64 im2win route (transform + convolution) on {n_img} of {layer.N} images of {layer.name} "
+              f"per precision per step")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{layer.name}: N={layer.N} C={layer.C} H=W={layer.H} Co={layer.Co} "
+                               f"K={layer.Kh}x{layer.Kw} stride={layer.stride} pad={layer.pad}, fp32 and fp16 passes",
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--report", default=None, help="also write a per-layer, per-kernel report (JSON lines)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference_arm(args)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    run_gpu_arm(args)
+
+
+if __name__ == "__main__":
+    main()

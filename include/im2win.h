@@ -1,0 +1,157 @@
+/*
+ * im2win.h -- C ABI of the B200 (sm_100a) im2win convolution library.
+ *
+ * The library implements the hot path of the im2win convolution: the im2win
+ * data transformation (paper Eq. 2) and the forward convolution over the
+ * im2win tensor (paper Eq. 3, GEMM view of Algorithm 1) in two precisions:
+ * fp32 on CUDA cores and fp16-input / fp32-accumulate on tensor cores.
+ *
+ * Problem statement (paper, Section "Notation"): input I[N][C][H][W], filter
+ * F[Co][C][Kh][Kw] (OIHW), output O[N][Co][Ho][Wo], all row-major with the
+ * last index fastest; one stride s for both axes; a symmetric zero padding p
+ * (the paper's layers have p = 0).  Ho = floor((H + 2p - Kh) / s) + 1 and
+ * likewise Wo.  The operation is a cross-correlation (Eq. 1, no kernel flip).
+ *
+ * General conventions
+ *   - Every data pointer is a DEVICE pointer unless its name ends in _host.
+ *     The caller owns all memory; the library allocates no device memory and
+ *     keeps no per-call state.  Buffers must stay valid until the work queued
+ *     on `cuda_stream` has completed.
+ *   - All calls are asynchronous on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL is the default stream), except where stated.
+ *   - Inputs are never written.  Output, window, scratch and input buffers
+ *     must not overlap one another.
+ *   - Device pointers must be 16-byte aligned, else IM2WIN_ERR_MISALIGNED.
+ *   - Arguments are validated before anything is launched; on any error no
+ *     device work has been queued by that call.
+ *   - There is no CPU fallback: without a CUDA device the compute entry points
+ *     return IM2WIN_ERR_CUDA.
+ */
+#ifndef IM2WIN_H_
+#define IM2WIN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct {
+  int32_t N, C, H, W;   /* input  [N][C][H][W]                          */
+  int32_t Co, Kh, Kw;   /* filter [Co][C][Kh][Kw]                       */
+  int32_t stride;       /* >= 1, same for both axes                     */
+  int32_t pad;          /* >= 0, zero rows/columns added on every side  */
+} im2win_shape;
+
+typedef enum {
+  IM2WIN_F32 = 0,       /* 4-byte elements, IEEE binary32 */
+  IM2WIN_F16 = 1        /* 2-byte elements, IEEE binary16 */
+} im2win_dtype;
+
+typedef enum {
+  IM2WIN_OK = 0,
+  IM2WIN_ERR_INVALID_ARG = 1,         /* non-positive size, negative pad, Ho or Wo < 1, bad dtype */
+  IM2WIN_ERR_NULL_POINTER = 2,
+  IM2WIN_ERR_MISALIGNED = 3,          /* a device pointer is not 16-byte aligned */
+  IM2WIN_ERR_WORKSPACE_TOO_SMALL = 4,
+  IM2WIN_ERR_UNSUPPORTED = 5,         /* sizes beyond the kernels' index ranges */
+  IM2WIN_ERR_CUDA = 6,                /* a CUDA call failed (no device, launch error) */
+  IM2WIN_ERR_TIMEOUT = 7              /* a bounded device-side wait gave up (see im2win_check_status) */
+} im2win_status;
+
+/* Static, NUL-terminated description of a status code. */
+const char* im2win_status_string(im2win_status status);
+
+/*
+ * Sizes, in bytes, of the buffers a layer needs (host-only, launches nothing).
+ *   window_bytes  = N*C*Ho*Kh*(W+2p) * sizeof(element): the closed-form size
+ *                   of the im2win tensor (paper Eq. 2; Section "Im2win Data
+ *                   Transformation"), with no hidden padding.
+ *   scratch_bytes = what im2win_conv_f32 / im2win_conv_f16 need in `scratch`
+ *                   (a status block, the repacked filter and an offset table).
+ *   Ho, Wo        = output height and width.
+ * Any of the four output pointers may be NULL.
+ */
+im2win_status im2win_workspace_size(const im2win_shape* shape, im2win_dtype dtype,
+                                    size_t* window_bytes, size_t* scratch_bytes,
+                                    int32_t* Ho, int32_t* Wo);
+
+/*
+ * im2win data transformation (paper Eq. 2, 0-based):
+ *     window[n][c][ho][k*Kh + u] = Xpad[n][c][ho*s + u][k],
+ *     k in [0, W+2p), u in [0, Kh),
+ * where Xpad is x with p zero rows/columns on every side.  The result is
+ * [N][C][Ho][Kh*(W+2p)]; every Kh x Kw sliding window of output row ho is the
+ * contiguous run of Kh*Kw elements starting at (wo*s)*Kh.  Elements are moved
+ * as bit patterns (NaN payloads and -0 are preserved); padding positions are
+ * written as +0.  `x_nchw` holds N*C*H*W elements and `window` window_bytes
+ * bytes, both of `dtype`.
+ */
+im2win_status im2win_transform(const void* x_nchw, void* window, const im2win_shape* shape,
+                               im2win_dtype dtype, void* cuda_stream);
+
+/*
+ * Forward convolution over the im2win tensor, fp32 on CUDA cores
+ * (paper Eq. 3; Section "im2win convolutions", the "CC" variant):
+ *     y[n][co][ho][wo] = sum_c sum_{t < Kh*Kw} window[n][c][ho][(wo*s)*Kh + t] * Fp[co][c][t],
+ *     Fp[co][c][v*Kh + u] = filter_oihw[co][c][u][v]   (height before width).
+ * The filter is repacked into `scratch` on every call (part of the timed
+ * operation).  `y_nchw` is [N][Co][Ho][Wo] fp32.  `scratch` must hold at least
+ * the scratch_bytes reported by im2win_workspace_size(shape, IM2WIN_F32, ...).
+ * Products and sums are fp32; the summation order is unspecified.
+ */
+im2win_status im2win_conv_f32(const float* window, const float* filter_oihw, float* y_nchw,
+                              void* scratch, size_t scratch_bytes, const im2win_shape* shape,
+                              void* cuda_stream);
+
+/*
+ * Forward convolution over the im2win tensor, fp16 inputs on tensor cores with
+ * fp32 accumulation and fp32 output (paper Algorithm 1; Section "Im2win
+ * Convolution on Tensor Cores", the "TC" variant; GEMM view M x N x K =
+ * positions x Co x C*Kh*Kw).  `window` and `filter_oihw` hold IEEE binary16
+ * bit patterns; `y_nchw` is [N][Co][Ho][Wo] fp32.  `scratch` as above with
+ * IM2WIN_F16.  Device-side waits in this kernel are bounded; if one gives up
+ * the kernel records it in the status block at the start of `scratch` and
+ * returns early (see im2win_check_status).
+ */
+im2win_status im2win_conv_f16(const uint16_t* window, const uint16_t* filter_oihw, float* y_nchw,
+                              void* scratch, size_t scratch_bytes, const im2win_shape* shape,
+                              void* cuda_stream);
+
+/*
+ * Synchronises `cuda_stream`, reads the status block at the start of `scratch`
+ * (written by the last convolution call that used it) and returns
+ * IM2WIN_ERR_TIMEOUT if a bounded device wait gave up, IM2WIN_ERR_CUDA if the
+ * stream reports an error, else IM2WIN_OK.  Blocking.
+ */
+im2win_status im2win_check_status(const void* scratch, void* cuda_stream);
+
+/*
+ * Size in bytes of the device workspace im2win_layer_forward_host needs for
+ * one layer: input copy + window tensor + scratch + output, each rounded up
+ * to 256 bytes (host-only, launches nothing).
+ */
+im2win_status im2win_layer_workspace_size(const im2win_shape* shape, im2win_dtype dtype,
+                                          size_t* device_bytes);
+
+/*
+ * Whole layer from HOST buffers: copies x and the filter to the device
+ * workspace, runs im2win_transform and the convolution of `dtype`, and copies
+ * y back, all queued on `cuda_stream` (paper Sections "Im2win Data
+ * Transformation" and "Im2win Convolution" back to back).  x_host and
+ * filter_host hold elements of `dtype` (binary16 bit patterns for F16);
+ * y_host receives N*Co*Ho*Wo floats.  Host buffers should be page-locked for
+ * the copies to overlap nothing else; they must stay valid until the stream
+ * has been synchronised by the caller.  `device_workspace` is a 256-byte
+ * aligned device buffer of at least im2win_layer_workspace_size bytes.
+ */
+im2win_status im2win_layer_forward_host(const void* x_host, const void* filter_host, float* y_host,
+                                        void* device_workspace, size_t device_workspace_bytes,
+                                        const im2win_shape* shape, im2win_dtype dtype,
+                                        void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IM2WIN_H_ */

@@ -1,0 +1,229 @@
+// C ABI of the im2win library: argument validation, buffer-size queries and
+// dispatch to the kernels.  Declarations and the contract of every entry
+// point are in include/im2win.h.
+#include "common.cuh"
+
+namespace im2win {
+
+static inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+
+im2win_status derive_geometry(const im2win_shape* s, Geometry* g) {
+  if (!s) return IM2WIN_ERR_NULL_POINTER;
+  if (s->N < 1 || s->C < 1 || s->H < 1 || s->W < 1 || s->Co < 1 || s->Kh < 1 || s->Kw < 1 ||
+      s->stride < 1 || s->pad < 0)
+    return IM2WIN_ERR_INVALID_ARG;
+  const int64_t hspan = (int64_t)s->H + 2 * (int64_t)s->pad - s->Kh;
+  const int64_t wspan = (int64_t)s->W + 2 * (int64_t)s->pad - s->Kw;
+  if (hspan < 0 || wspan < 0) return IM2WIN_ERR_INVALID_ARG;
+  g->N = s->N; g->C = s->C; g->H = s->H; g->W = s->W; g->Co = s->Co;
+  g->Kh = s->Kh; g->Kw = s->Kw; g->s = s->stride; g->p = s->pad;
+  g->Ho = (int32_t)(hspan / s->stride) + 1;
+  g->Wo = (int32_t)(wspan / s->stride) + 1;
+  const int64_t Wp = (int64_t)s->W + 2 * (int64_t)s->pad;
+  const int64_t T = (int64_t)s->Kh * s->Kw;
+  // Index ranges of the kernels: 32-bit per-image offsets and counts, 64-bit bases.
+  const int64_t lim = (int64_t)1 << 31;
+  if (Wp >= lim || T >= lim) return IM2WIN_ERR_UNSUPPORTED;
+  g->Wp = (int32_t)Wp;
+  g->T = (int32_t)T;
+  g->strip = (int64_t)s->Kh * Wp;
+  if (g->strip >= lim) return IM2WIN_ERR_UNSUPPORTED;
+  g->chan_stride = (int64_t)g->Ho * g->strip;
+  if (g->chan_stride >= lim) return IM2WIN_ERR_UNSUPPORTED;
+  g->img_stride = (int64_t)s->C * g->chan_stride;
+  if (g->img_stride >= lim) return IM2WIN_ERR_UNSUPPORTED;    // k -> offset table is int32
+  g->K = (int64_t)s->C * T;
+  if (g->K >= lim - 64) return IM2WIN_ERR_UNSUPPORTED;
+  if ((int64_t)g->Ho * g->Wo >= lim) return IM2WIN_ERR_UNSUPPORTED;
+  g->P = (int64_t)s->N * g->Ho * g->Wo;
+  if (g->P >= lim * 64) return IM2WIN_ERR_UNSUPPORTED;        // grid.x of 128-row tiles
+  if ((int64_t)s->N * s->C * g->Ho * Wp >= lim * 4) return IM2WIN_ERR_UNSUPPORTED;      // transform grid
+  if ((int64_t)s->H * s->W >= lim) return IM2WIN_ERR_UNSUPPORTED;
+  if ((int64_t)s->Kh * 8 * 4 > 200 * 1024) return IM2WIN_ERR_UNSUPPORTED;  // transform staging
+  if ((int64_t)s->Co * g->K >= lim * 16) return IM2WIN_ERR_UNSUPPORTED;
+  g->window_elems = (int64_t)s->N * g->img_stride;
+  g->out_elems = (int64_t)s->N * s->Co * g->Ho * g->Wo;
+  return IM2WIN_OK;
+}
+
+im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayout* l) {
+  if (dtype == IM2WIN_F32) {
+    l->Kp = round_up(g.K, kF32KBlock);
+    l->Co_pad = g.Co > 64 ? round_up(g.Co, 128) : 64;
+  } else if (dtype == IM2WIN_F16) {
+    l->Kp = round_up(g.K, kF16KBlock);
+    l->Co_pad = g.Co;
+  } else {
+    return IM2WIN_ERR_INVALID_ARG;
+  }
+  l->koff_off = kStatusBytes;
+  l->filter_off = (size_t)round_up((int64_t)l->koff_off + 4 * l->Kp, 256);
+  const int64_t fbytes = l->Kp * l->Co_pad * (dtype == IM2WIN_F32 ? 4 : 2);
+  l->total = (size_t)round_up((int64_t)l->filter_off + fbytes, 256);
+  return IM2WIN_OK;
+}
+
+static inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+static im2win_status conv_common(const void* window, const void* filter, float* y, void* scratch,
+                                 size_t scratch_bytes, const im2win_shape* shape, im2win_dtype dtype,
+                                 void* cuda_stream) {
+  if (!window || !filter || !y || !scratch || !shape) return IM2WIN_ERR_NULL_POINTER;
+  Geometry g;
+  im2win_status st = derive_geometry(shape, &g);
+  if (st != IM2WIN_OK) return st;
+  ScratchLayout l;
+  st = scratch_layout(g, dtype, &l);
+  if (st != IM2WIN_OK) return st;
+  if (misaligned(window) || misaligned(filter) || misaligned(y) || misaligned(scratch))
+    return IM2WIN_ERR_MISALIGNED;
+  if (scratch_bytes < l.total) return IM2WIN_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e;
+  if (dtype == IM2WIN_F32) {
+    e = launch_pack_f32(static_cast<const float*>(filter), scratch, g, l, stream);
+    if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
+    e = launch_conv_f32(static_cast<const float*>(window), y, scratch, g, l, stream);
+  } else {
+    e = launch_pack_f16(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
+    if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
+    e = launch_conv_f16(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
+  }
+  return e == cudaSuccess ? IM2WIN_OK : IM2WIN_ERR_CUDA;
+}
+
+}  // namespace im2win
+
+using namespace im2win;
+
+extern "C" {
+
+const char* im2win_status_string(im2win_status status) {
+  switch (status) {
+    case IM2WIN_OK: return "ok";
+    case IM2WIN_ERR_INVALID_ARG: return "invalid argument";
+    case IM2WIN_ERR_NULL_POINTER: return "null pointer";
+    case IM2WIN_ERR_MISALIGNED: return "device pointer not 16-byte aligned";
+    case IM2WIN_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case IM2WIN_ERR_UNSUPPORTED: return "shape beyond the kernels' index ranges";
+    case IM2WIN_ERR_CUDA: return "CUDA error";
+    case IM2WIN_ERR_TIMEOUT: return "bounded device wait gave up";
+  }
+  return "unknown status";
+}
+
+im2win_status im2win_workspace_size(const im2win_shape* shape, im2win_dtype dtype, size_t* window_bytes,
+                                    size_t* scratch_bytes, int32_t* Ho, int32_t* Wo) {
+  Geometry g;
+  im2win_status st = derive_geometry(shape, &g);
+  if (st != IM2WIN_OK) return st;
+  ScratchLayout l;
+  st = scratch_layout(g, dtype, &l);
+  if (st != IM2WIN_OK) return st;
+  if (window_bytes) *window_bytes = (size_t)g.window_elems * (dtype == IM2WIN_F32 ? 4 : 2);
+  if (scratch_bytes) *scratch_bytes = l.total;
+  if (Ho) *Ho = g.Ho;
+  if (Wo) *Wo = g.Wo;
+  return IM2WIN_OK;
+}
+
+im2win_status im2win_transform(const void* x_nchw, void* window, const im2win_shape* shape,
+                               im2win_dtype dtype, void* cuda_stream) {
+  if (!x_nchw || !window || !shape) return IM2WIN_ERR_NULL_POINTER;
+  if (dtype != IM2WIN_F32 && dtype != IM2WIN_F16) return IM2WIN_ERR_INVALID_ARG;
+  Geometry g;
+  im2win_status st = derive_geometry(shape, &g);
+  if (st != IM2WIN_OK) return st;
+  if (misaligned(x_nchw) || misaligned(window)) return IM2WIN_ERR_MISALIGNED;
+  cudaError_t e = launch_transform(x_nchw, window, g, dtype == IM2WIN_F32 ? 4 : 2,
+                                   static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? IM2WIN_OK : IM2WIN_ERR_CUDA;
+}
+
+im2win_status im2win_conv_f32(const float* window, const float* filter_oihw, float* y_nchw, void* scratch,
+                              size_t scratch_bytes, const im2win_shape* shape, void* cuda_stream) {
+  return conv_common(window, filter_oihw, y_nchw, scratch, scratch_bytes, shape, IM2WIN_F32, cuda_stream);
+}
+
+im2win_status im2win_conv_f16(const uint16_t* window, const uint16_t* filter_oihw, float* y_nchw,
+                              void* scratch, size_t scratch_bytes, const im2win_shape* shape,
+                              void* cuda_stream) {
+  return conv_common(window, filter_oihw, y_nchw, scratch, scratch_bytes, shape, IM2WIN_F16, cuda_stream);
+}
+
+im2win_status im2win_check_status(const void* scratch, void* cuda_stream) {
+  if (!scratch) return IM2WIN_ERR_NULL_POINTER;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0;
+  if (cudaMemcpyAsync(&word, scratch, sizeof(word), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return IM2WIN_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return IM2WIN_ERR_CUDA;
+  return word ? IM2WIN_ERR_TIMEOUT : IM2WIN_OK;
+}
+
+namespace {
+struct LayerLayout {
+  size_t x_off, f_off, win_off, scratch_off, y_off, total;
+  size_t x_bytes, f_bytes, win_bytes, scratch_bytes, y_bytes;
+};
+im2win_status layer_layout(const Geometry& g, im2win_dtype dtype, LayerLayout* L) {
+  ScratchLayout l;
+  im2win_status st = scratch_layout(g, dtype, &l);
+  if (st != IM2WIN_OK) return st;
+  const size_t es = dtype == IM2WIN_F32 ? 4 : 2;
+  L->x_bytes = (size_t)g.N * g.C * g.H * g.W * es;
+  L->f_bytes = (size_t)g.Co * g.K * es;
+  L->win_bytes = (size_t)g.window_elems * es;
+  L->scratch_bytes = l.total;
+  L->y_bytes = (size_t)g.out_elems * 4;
+  auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+  L->x_off = 0;
+  L->f_off = L->x_off + up(L->x_bytes);
+  L->win_off = L->f_off + up(L->f_bytes);
+  L->scratch_off = L->win_off + up(L->win_bytes);
+  L->y_off = L->scratch_off + up(L->scratch_bytes);
+  L->total = L->y_off + up(L->y_bytes);
+  return IM2WIN_OK;
+}
+}  // namespace
+
+im2win_status im2win_layer_workspace_size(const im2win_shape* shape, im2win_dtype dtype, size_t* device_bytes) {
+  Geometry g;
+  im2win_status st = derive_geometry(shape, &g);
+  if (st != IM2WIN_OK) return st;
+  LayerLayout L;
+  st = layer_layout(g, dtype, &L);
+  if (st != IM2WIN_OK) return st;
+  if (device_bytes) *device_bytes = L.total;
+  return IM2WIN_OK;
+}
+
+im2win_status im2win_layer_forward_host(const void* x_host, const void* filter_host, float* y_host,
+                                        void* device_workspace, size_t device_workspace_bytes,
+                                        const im2win_shape* shape, im2win_dtype dtype, void* cuda_stream) {
+  if (!x_host || !filter_host || !y_host || !device_workspace || !shape) return IM2WIN_ERR_NULL_POINTER;
+  Geometry g;
+  im2win_status st = derive_geometry(shape, &g);
+  if (st != IM2WIN_OK) return st;
+  LayerLayout L;
+  st = layer_layout(g, dtype, &L);
+  if (st != IM2WIN_OK) return st;
+  if ((reinterpret_cast<uintptr_t>(device_workspace) & 255u) != 0) return IM2WIN_ERR_MISALIGNED;
+  if (device_workspace_bytes < L.total) return IM2WIN_ERR_WORKSPACE_TOO_SMALL;
+  unsigned char* ws = static_cast<unsigned char*>(device_workspace);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(ws + L.x_off, x_host, L.x_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return IM2WIN_ERR_CUDA;
+  if (cudaMemcpyAsync(ws + L.f_off, filter_host, L.f_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return IM2WIN_ERR_CUDA;
+  st = im2win_transform(ws + L.x_off, ws + L.win_off, shape, dtype, cuda_stream);
+  if (st != IM2WIN_OK) return st;
+  st = conv_common(ws + L.win_off, ws + L.f_off, reinterpret_cast<float*>(ws + L.y_off), ws + L.scratch_off,
+                   L.scratch_bytes, shape, dtype, cuda_stream);
+  if (st != IM2WIN_OK) return st;
+  if (cudaMemcpyAsync(y_host, ws + L.y_off, L.y_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return IM2WIN_ERR_CUDA;
+  return IM2WIN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,58 @@
+// Shared host-side definitions of the im2win library: derived geometry,
+// scratch layout and launch prototypes.  Device code lives in the .cu files.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/im2win.h"
+
+namespace im2win {
+
+// Quantities derived from an im2win_shape (notation of the paper's Section
+// "Notation" and Eq. 2/3): Wp = W + 2p, strip = Kh*Wp elements per (n,c,ho),
+// T = Kh*Kw window elements per channel, K = C*T reduction length,
+// P = N*Ho*Wo output positions.
+struct Geometry {
+  int32_t N, C, H, W, Co, Kh, Kw, s, p;
+  int32_t Ho, Wo, Wp, T;
+  int64_t strip;         // Kh*Wp
+  int64_t chan_stride;   // Ho*strip: distance between channels of one image in the window tensor
+  int64_t img_stride;    // C*chan_stride
+  int64_t K;             // C*T
+  int64_t P;             // N*Ho*Wo
+  int64_t window_elems;  // N*img_stride
+  int64_t out_elems;     // N*Co*Ho*Wo
+};
+
+// Scratch layout shared by both precisions (offsets in bytes from `scratch`):
+//   [0, 256)            status block (uint32 words; word 0 = timeout flag)
+//   [256, 256 + 4*Kp)   k -> element offset table (int32), -1 for padded k
+//   [filter_off, ...)   repacked filter
+struct ScratchLayout {
+  int64_t Kp;            // K rounded up to the k-block of the kernel
+  int64_t Co_pad;        // Co rounded up to the filter tile of the kernel
+  size_t koff_off, filter_off, total;
+};
+
+constexpr int kStatusBytes = 256;
+constexpr int kF32KBlock = 16;     // k-block of the fp32 kernel
+constexpr int kF16KBlock = 64;     // k-block of the fp16 kernel (64 halves = one 128-byte swizzle row)
+
+im2win_status derive_geometry(const im2win_shape* s, Geometry* g);
+im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayout* l);
+
+// Kernel launchers (each queues work on `stream` and returns the launch status).
+cudaError_t launch_transform(const void* x, void* window, const Geometry& g, int elem_bytes,
+                             cudaStream_t stream);
+cudaError_t launch_pack_f32(const float* filter, void* scratch, const Geometry& g,
+                            const ScratchLayout& l, cudaStream_t stream);
+cudaError_t launch_pack_f16(const uint16_t* filter, void* scratch, const Geometry& g,
+                            const ScratchLayout& l, cudaStream_t stream);
+cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, const Geometry& g,
+                            const ScratchLayout& l, cudaStream_t stream);
+cudaError_t launch_conv_f16(const uint16_t* window, float* y, void* scratch, const Geometry& g,
+                            const ScratchLayout& l, cudaStream_t stream);
+
+}  // namespace im2win

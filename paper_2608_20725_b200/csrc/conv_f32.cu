@@ -1,0 +1,181 @@
+// fp32 im2win convolution on CUDA cores (paper Eq. 3, "CC" variant) for sm_100a.
+//
+// GEMM view (Algorithm 1's dimensions with positions as rows):
+//     y[p][co] = sum_k A[p][k] * Fk[k][co],  p = (n, ho, wo),  k = (c, v, u),
+//     A[p][k]  = window[n][c][ho][(wo*s)*Kh + v*Kh + u].
+// A CTA computes a BM x BN tile of y.  Per k-block of 16 it gathers the A tile
+// from the window tensor (lanes walk consecutive positions, i.e. addresses
+// s*Kh elements apart inside one strip; the k -> offset table is precomputed)
+// and the Fk tile (contiguous) into shared memory, double buffered with the
+// global loads of the next k-block held in registers while the current block
+// is multiplied.  Each thread accumulates an 8 x 8 register tile with 128-bit
+// shared-memory loads (2 x 4 positions by 2 x 4 output channels).  Positions
+// run along the lanes, so stores to the NCHW output are contiguous per output
+// channel.
+#include "common.cuh"
+
+namespace im2win {
+namespace {
+
+struct ConvF32Params {
+  const float* __restrict__ win;
+  const float* __restrict__ fk;      // [Kp][Co_pad]
+  const int32_t* __restrict__ koff;  // [Kp]
+  float* __restrict__ y;
+  int64_t P, img_stride, strip;
+  int32_t HoWo, Wo, sKh, Co, Co_pad, Kp;
+};
+
+constexpr int BM = 128;
+constexpr int BK = kF32KBlock;
+
+template <int BN>
+__global__ void __launch_bounds__((BM / 8) * (BN / 8))
+conv_f32_kernel(ConvF32Params q) {
+  constexpr int THREADS = (BM / 8) * (BN / 8);
+  constexpr int A_PER_THREAD = BK * BM / THREADS;         // scalar gathers per k-block
+  constexpr int A_KK_STEP = THREADS / BM;                 // 2 (256 threads) or 1 (128 threads)
+  constexpr int B_VEC_PER_THREAD = BK * BN / 4 / THREADS; // float4 loads per k-block
+  static_assert(THREADS % BM == 0 && A_PER_THREAD * A_KK_STEP == BK, "loader mapping");
+
+  __shared__ __align__(16) float As[2][BK][BM];
+  __shared__ __align__(16) float Bs[2][BK][BN];
+
+  const int tid = threadIdx.x;
+  const int tm = tid % (BM / 8);     // position direction: fastest across lanes
+  const int tn = tid / (BM / 8);
+  const int64_t m0 = (int64_t)blockIdx.x * BM;
+  const int n0 = blockIdx.y * BN;
+
+  // Loader role: one fixed position (row of A) per thread.
+  const int lm = tid % BM;
+  const int lkk0 = tid / BM;
+  const int64_t lp = m0 + lm;
+  const bool lvalid = lp < q.P;
+  const float* abase = q.win;
+  if (lvalid) {
+    const int64_t n = lp / q.HoWo;
+    const int r = (int)(lp - n * q.HoWo);
+    const int ho = r / q.Wo;
+    const int wo = r - ho * q.Wo;
+    abase += n * q.img_stride + ho * q.strip + (int64_t)wo * q.sKh;
+  }
+
+  float areg[A_PER_THREAD];
+  float4 breg[B_VEC_PER_THREAD];
+
+  auto load_global = [&](int kb) {
+    const int k0 = kb * BK;
+#pragma unroll
+    for (int i = 0; i < A_PER_THREAD; ++i) {
+      const int off = __ldg(q.koff + k0 + lkk0 + i * A_KK_STEP);
+      areg[i] = (lvalid && off >= 0) ? __ldg(abase + off) : 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < B_VEC_PER_THREAD; ++i) {
+      const int e = tid + i * THREADS;       // float4 index inside the BK x BN tile
+      const int kk = e / (BN / 4);
+      const int nn = (e - kk * (BN / 4)) * 4;
+      breg[i] = __ldg(reinterpret_cast<const float4*>(q.fk + (int64_t)(k0 + kk) * q.Co_pad + n0 + nn));
+    }
+  };
+  auto store_shared = [&](int buf) {
+#pragma unroll
+    for (int i = 0; i < A_PER_THREAD; ++i) As[buf][lkk0 + i * A_KK_STEP][lm] = areg[i];
+#pragma unroll
+    for (int i = 0; i < B_VEC_PER_THREAD; ++i) {
+      const int e = tid + i * THREADS;
+      const int kk = e / (BN / 4);
+      const int nn = (e - kk * (BN / 4)) * 4;
+      *reinterpret_cast<float4*>(&Bs[buf][kk][nn]) = breg[i];
+    }
+  };
+
+  float acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+
+  const int nkb = q.Kp / BK;
+  load_global(0);
+  store_shared(0);
+  __syncthreads();
+
+  for (int kb = 0; kb < nkb; ++kb) {
+    const int buf = kb & 1;
+    if (kb + 1 < nkb) load_global(kb + 1);
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][kk][tm * 4]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[buf][kk][BM / 2 + tm * 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][kk][tn * 4]);
+      const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][kk][BN / 2 + tn * 4]);
+      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    if (kb + 1 < nkb) {
+      store_shared(buf ^ 1);
+      __syncthreads();
+    }
+  }
+
+  // Epilogue: positions of one half-tile are 4 consecutive p; NCHW output is
+  // contiguous in p within an image for a fixed output channel.
+  const bool vec_ok = (q.HoWo % 4) == 0;
+#pragma unroll
+  for (int hm = 0; hm < 2; ++hm) {
+    const int64_t p = m0 + hm * (BM / 2) + tm * 4;
+    if (p >= q.P) continue;
+    const int64_t n = p / q.HoWo;
+    const int r = (int)(p - n * q.HoWo);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int co = n0 + (j / 4) * (BN / 2) + tn * 4 + (j % 4);
+      if (co >= q.Co) continue;
+      if (vec_ok) {
+        float4 v = make_float4(acc[hm * 4 + 0][j], acc[hm * 4 + 1][j], acc[hm * 4 + 2][j], acc[hm * 4 + 3][j]);
+        *reinterpret_cast<float4*>(q.y + (n * q.Co + co) * q.HoWo + r) = v;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int64_t pi = p + i;
+          if (pi >= q.P) break;
+          const int64_t ni = pi / q.HoWo;
+          const int ri = (int)(pi - ni * q.HoWo);
+          q.y[(ni * q.Co + co) * q.HoWo + ri] = acc[hm * 4 + i][j];
+        }
+      }
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, const Geometry& g,
+                            const ScratchLayout& l, cudaStream_t stream) {
+  const unsigned char* base = static_cast<const unsigned char*>(scratch);
+  ConvF32Params q;
+  q.win = window;
+  q.fk = reinterpret_cast<const float*>(base + l.filter_off);
+  q.koff = reinterpret_cast<const int32_t*>(base + l.koff_off);
+  q.y = y;
+  q.P = g.P; q.img_stride = g.img_stride; q.strip = g.strip;
+  q.HoWo = g.Ho * g.Wo; q.Wo = g.Wo; q.sKh = g.s * g.Kh;
+  q.Co = g.Co; q.Co_pad = (int32_t)l.Co_pad; q.Kp = (int32_t)l.Kp;
+  const unsigned mt = (unsigned)((g.P + BM - 1) / BM);
+  if (g.Co > 64) {
+    dim3 grid(mt, (unsigned)(l.Co_pad / 128));
+    conv_f32_kernel<128><<<grid, (BM / 8) * (128 / 8), 0, stream>>>(q);
+  } else {
+    dim3 grid(mt, (unsigned)(l.Co_pad / 64));
+    conv_f32_kernel<64><<<grid, (BM / 8) * (64 / 8), 0, stream>>>(q);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace im2win

@@ -1,0 +1,116 @@
+// Filter repacking for the im2win convolution kernels (sm_100a).
+//
+// The im2win window of one channel is stored height-fastest (offset v*Kh + u),
+// so the filter is repacked to the same order (paper, Section "Im2win
+// Convolution": the filter layout puts height before width):
+//     k = c*T + v*Kh + u,   T = Kh*Kw,   Fp[co][k] = F[co][c][u][v].
+// The same pass writes the table k -> element offset of window element k
+// relative to the window of channel 0 (c*chan_stride + v*Kh + u); entries of
+// the zero-padded tail k >= K hold -1.  It also clears the status block at the
+// start of the scratch buffer.
+//   fp32 kernel layout: Fk[k][Co_pad]  (co contiguous), zero padded in k and co
+//   fp16 kernel layout: Fp[co][Kp]     (k contiguous),  zero padded in k
+#include "common.cuh"
+
+namespace im2win {
+namespace {
+
+struct PackParams {
+  int32_t C, Co, Kh, Kw, T;
+  int64_t K, Kp, Co_pad, chan_stride;
+};
+
+__device__ __forceinline__ void split_k(const PackParams& q, int64_t k, int& c, int& u, int& v) {
+  c = (int)(k / q.T);
+  const int t = (int)(k - (int64_t)c * q.T);
+  v = t / q.Kh;
+  u = t - v * q.Kh;
+}
+
+__global__ void pack_f32_kernel(const float* __restrict__ f, float* __restrict__ fk,
+                                int32_t* __restrict__ koff, uint32_t* __restrict__ status,
+                                PackParams q) {
+  if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
+  const int64_t total = q.Kp * q.Co_pad;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int64_t k = i / q.Co_pad;
+    const int co = (int)(i - k * q.Co_pad);
+    float val = 0.f;
+    if (k < q.K && co < q.Co) {
+      int c, u, v;
+      split_k(q, k, c, u, v);
+      val = f[(((int64_t)co * q.C + c) * q.Kh + u) * q.Kw + v];
+    }
+    fk[i] = val;
+    if (co == 0) {
+      int32_t off = -1;
+      if (k < q.K) {
+        int c, u, v;
+        split_k(q, k, c, u, v);
+        off = (int32_t)(c * q.chan_stride + v * q.Kh + u);
+      }
+      koff[k] = off;
+    }
+  }
+}
+
+__global__ void pack_f16_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp,
+                                int32_t* __restrict__ koff, uint32_t* __restrict__ status,
+                                PackParams q) {
+  if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
+  const int64_t total = q.Kp * q.Co;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int64_t co = i / q.Kp;
+    const int64_t k = i - co * q.Kp;
+    uint16_t val = 0;
+    int32_t off = -1;
+    if (k < q.K) {
+      int c, u, v;
+      split_k(q, k, c, u, v);
+      val = f[((co * q.C + c) * q.Kh + u) * q.Kw + v];
+      off = (int32_t)(c * q.chan_stride + v * q.Kh + u);
+    }
+    fp[i] = val;
+    if (co == 0) koff[k] = off;
+  }
+}
+
+PackParams make_params(const Geometry& g, const ScratchLayout& l) {
+  PackParams q;
+  q.C = g.C; q.Co = g.Co; q.Kh = g.Kh; q.Kw = g.Kw; q.T = g.T;
+  q.K = g.K; q.Kp = l.Kp; q.Co_pad = l.Co_pad; q.chan_stride = g.chan_stride;
+  return q;
+}
+
+int grid_for(int64_t total) {
+  int64_t b = (total + 255) / 256;
+  if (b > 148 * 8) b = 148 * 8;
+  if (b < 1) b = 1;
+  return (int)b;
+}
+
+}  // namespace
+
+cudaError_t launch_pack_f32(const float* filter, void* scratch, const Geometry& g,
+                            const ScratchLayout& l, cudaStream_t stream) {
+  unsigned char* base = static_cast<unsigned char*>(scratch);
+  PackParams q = make_params(g, l);
+  pack_f32_kernel<<<grid_for(q.Kp * q.Co_pad), 256, 0, stream>>>(
+      filter, reinterpret_cast<float*>(base + l.filter_off),
+      reinterpret_cast<int32_t*>(base + l.koff_off), reinterpret_cast<uint32_t*>(base), q);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pack_f16(const uint16_t* filter, void* scratch, const Geometry& g,
+                            const ScratchLayout& l, cudaStream_t stream) {
+  unsigned char* base = static_cast<unsigned char*>(scratch);
+  PackParams q = make_params(g, l);
+  pack_f16_kernel<<<grid_for(q.Kp * q.Co), 256, 0, stream>>>(
+      filter, reinterpret_cast<uint16_t*>(base + l.filter_off),
+      reinterpret_cast<int32_t*>(base + l.koff_off), reinterpret_cast<uint32_t*>(base), q);
+  return cudaGetLastError();
+}
+
+}  // namespace im2win

@@ -1,0 +1,95 @@
+"""Helpers of the GPU parity tests: run the CUDA path through the C ABI with guard bands
+around every output buffer, and compare with the CPU oracle."""
+import numpy as np
+import torch
+
+import oracle
+from paper_2608_20725_b200 import binding
+
+TOL_F32 = 1e-5     # |gpu - oracle| <= TOL * sum |x||w|   (fp32 path)
+TOL_F16 = 2e-3     # same, fp16 inputs with fp32 accumulation, oracle on fp16-rounded inputs
+
+GUARD = 64         # guard elements before and after each output buffer
+
+
+def guarded(numel, dtype, fill):
+    """A device buffer with GUARD canary elements on both sides; returns (whole, view)."""
+    whole = torch.full((numel + 2 * GUARD,), fill, dtype=dtype, device="cuda")
+    return whole, whole[GUARD:GUARD + numel]
+
+
+def assert_guards_intact(whole, numel, fill):
+    head = whole[:GUARD].cpu()
+    tail = whole[GUARD + numel:].cpu()
+    ref = torch.full((GUARD,), fill, dtype=whole.dtype)
+    assert torch.equal(head.view(torch.uint8), ref.view(torch.uint8)), "write before the buffer"
+    assert torch.equal(tail.view(torch.uint8), ref.view(torch.uint8)), "write past the buffer"
+
+
+def gpu_transform(x_cpu: torch.Tensor, dims: dict) -> np.ndarray:
+    """x (float32/float16/int32/int16 CPU tensor) -> window tensor as a numpy array of the same dtype."""
+    code = binding.F32 if x_cpu.element_size() == 4 else binding.F16
+    tdt = torch.float32 if code == binding.F32 else torch.float16
+    wb, _, ho, _ = binding.im2win_workspace_size(dims, code)
+    n = wb // x_cpu.element_size()
+    whole, win = guarded(n, tdt, 7.0)
+    xd = x_cpu.contiguous().view(tdt).cuda()
+    binding.im2win_transform(xd, win, dims)
+    torch.cuda.synchronize()
+    assert_guards_intact(whole, n, 7.0)
+    out = win.cpu().view(x_cpu.dtype).numpy()
+    return out.reshape(dims["N"], dims["C"], ho, dims["Kh"] * (dims["W"] + 2 * dims["pad"]))
+
+
+def gpu_conv(x_cpu: torch.Tensor, f_cpu: torch.Tensor, dims: dict, precision: str):
+    """Transform + convolution on the GPU.  precision 'f32' or 'f16' (inputs are cast with
+    torch's round-to-nearest-even conversion).  Returns (y float32 numpy, x_used, f_used as float32 numpy)."""
+    tdt = torch.float32 if precision == "f32" else torch.float16
+    code = binding.F32 if precision == "f32" else binding.F16
+    xd = x_cpu.to(tdt).cuda().contiguous()
+    fd = f_cpu.to(tdt).cuda().contiguous()
+    wb, sb, ho, wo = binding.im2win_workspace_size(dims, code)
+    nwin = wb // xd.element_size()
+    nout = dims["N"] * dims["Co"] * ho * wo
+    wwhole, win = guarded(nwin, tdt, 3.0)
+    ywhole, y = guarded(nout, torch.float32, -123.0)
+    swhole, scratch = guarded(sb, torch.uint8, 0x5a)
+    assert scratch.data_ptr() % 16 == 0 and y.data_ptr() % 16 == 0 and win.data_ptr() % 16 == 0
+    binding.im2win_transform(xd, win, dims)
+    if precision == "f32":
+        binding.im2win_conv_f32(win, fd, y, scratch, dims)
+    else:
+        binding.im2win_conv_f16(win, fd, y, scratch, dims)
+    binding.im2win_check_status(scratch)
+    assert_guards_intact(wwhole, nwin, 3.0)
+    assert_guards_intact(ywhole, nout, -123.0)
+    assert_guards_intact(swhole, sb, 0x5a)
+    yh = y.cpu().numpy().reshape(dims["N"], dims["Co"], ho, wo)
+    return yh, xd.float().cpu().numpy(), fd.float().cpu().numpy()
+
+
+def oracle_inputs(x_cpu: torch.Tensor, f_cpu: torch.Tensor, precision: str):
+    """The values the oracle computes on: fp32 inputs as they are, or rounded to binary16 by the
+    oracle's own routine for the fp16 path."""
+    x = x_cpu.numpy().astype(np.float32)
+    f = f_cpu.numpy().astype(np.float32)
+    if precision == "f16":
+        _, x = oracle.round_to_f16(x)
+        _, f = oracle.round_to_f16(f)
+    return x, f
+
+
+def check_conv(y_gpu, y_ref, a_ref, precision, what=""):
+    tol = TOL_F32 if precision == "f32" else TOL_F16
+    err = np.abs(y_gpu.astype(np.float64) - y_ref)
+    bound = tol * a_ref
+    bad = err > bound
+    if bad.any():
+        i = np.unravel_index(np.argmax(err - bound), err.shape)
+        raise AssertionError(f"{what} {precision}: {bad.sum()} of {bad.size} outputs out of tolerance; worst at {i}: "
+                             f"gpu={y_gpu[i]!r} oracle={y_ref[i]!r} err={err[i]:.3e} bound={bound[i]:.3e}")
+    zero = a_ref == 0
+    assert np.all(y_gpu[zero] == 0), f"{what}: outputs with no non-zero term must be exactly 0"
+    with np.errstate(divide="ignore", invalid="ignore"):
+        rel = np.where(a_ref > 0, err / a_ref, 0.0)
+    return float(rel.max())

@@ -1,0 +1,176 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+
+Transform: bit-exact.  Convolution: |gpu - oracle| <= 1e-5 * sum|x||w| (fp32) and
+<= 2e-3 * sum|x||w| (fp16 inputs, oracle on binary16-rounded inputs), per output element.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_20725_b200 import binding, workloads
+from paper_2608_20725_b200.workloads import Layer
+from gpu_helpers import (assert_guards_intact, check_conv, gpu_conv, gpu_transform, guarded,
+                         oracle_inputs)
+
+pytestmark = pytest.mark.gpu
+
+
+def L(name, N, C, H, W, Co, Kh, Kw, s, p, seed=0, xd="normal01", fd="he_normal"):
+    return Layer(name, N, C, H, W, Co, Kh, Kw, s, p, seed, xd, fd)
+
+
+# Small layers that still span several tiles (128 positions, 64/128/256 channels, 16/64-wide
+# k-blocks) and leave ragged tails in every dimension.
+SMALL = [
+    workloads.LAYERS["cfg1"],
+    L("tail_pos", 3, 5, 13, 11, 7, 3, 3, 1, 1, 11),            # P = 429: 3 full tiles + a ragged one
+    L("k147", 2, 3, 37, 37, 64, 7, 7, 2, 3, 12),                # K = 147 (pads to 160 / 192)
+    L("co_tail", 2, 16, 12, 12, 72, 3, 3, 1, 1, 13),            # Co = 72: two fp32 channel tiles, one masked
+    L("co_300", 1, 8, 10, 10, 300, 3, 3, 1, 1, 14),             # Co = 300: 256 + 44 for the tensor-core tile
+    L("rect", 2, 4, 9, 14, 10, 2, 5, 1, 2, 15),                 # Kh != Kw
+    L("rect2", 2, 4, 14, 9, 10, 5, 2, 2, 0, 16),
+    L("stride3", 2, 6, 17, 19, 12, 3, 3, 3, 1, 17),
+    L("one_by_one", 3, 40, 7, 7, 33, 1, 1, 1, 0, 18),
+    L("k11", 1, 6, 30, 30, 20, 11, 11, 1, 5, 19),
+    L("k5s2", 2, 10, 21, 21, 24, 5, 5, 2, 2, 20),
+    L("single_out", 1, 3, 3, 3, 2, 3, 3, 1, 0, 21),             # Ho = Wo = 1
+    L("deep", 2, 130, 7, 7, 140, 3, 3, 1, 1, 22),               # K = 1170: many k-blocks, odd strips (54 B)
+    L("wide_row", 1, 2, 4, 300, 5, 3, 3, 1, 1, 23),             # one output row longer than a tile
+    L("uncovered_cols", 1, 3, 10, 12, 4, 3, 4, 3, 0, 24),       # (Wp - Kw) % s != 0: trailing columns never read
+]
+
+
+@pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
+@pytest.mark.parametrize("es", [4, 2])
+def test_transform_bit_exact_small(layer, es):
+    dims = layer.dims()
+    x, _ = workloads.make_inputs(layer)
+    xb = x if es == 4 else x.half()
+    raw = xb.view(torch.int32 if es == 4 else torch.int16)
+    got = gpu_transform(raw, dims)
+    want = oracle.transform(raw.numpy(), dims)
+    assert got.shape == want.shape and np.array_equal(got, want)
+
+
+def test_transform_preserves_special_bit_patterns():
+    layer = L("bits", 2, 3, 9, 10, 1, 3, 3, 2, 2, 30)
+    dims = layer.dims()
+    g = torch.Generator().manual_seed(31)
+    n = 2 * 3 * 9 * 10
+    raw32 = torch.randint(-2 ** 31, 2 ** 31 - 1, (n,), generator=g, dtype=torch.int64).to(torch.int32).reshape(2, 3, 9, 10)
+    raw32.view(-1)[:4] = torch.tensor([0x7fc01234, -2 ** 31, -1, 0x7f800001], dtype=torch.int64).to(torch.int32)
+    assert np.array_equal(gpu_transform(raw32, dims), oracle.transform(raw32.numpy(), dims))
+    raw16 = torch.randint(-2 ** 15, 2 ** 15 - 1, (n,), generator=g, dtype=torch.int64).to(torch.int16).reshape(2, 3, 9, 10)
+    raw16.view(-1)[:3] = torch.tensor([0x7e01, -2 ** 15, -1], dtype=torch.int64).to(torch.int16)
+    assert np.array_equal(gpu_transform(raw16, dims), oracle.transform(raw16.numpy(), dims))
+
+
+@pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
+@pytest.mark.parametrize("precision", ["f32", "f16"])
+def test_conv_parity_small(layer, precision):
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    y, _, _ = gpu_conv(x, f, dims, precision)
+    xo, fo = oracle_inputs(x, f, precision)
+    yr, ar = oracle.conv_direct(xo, fo, dims)
+    check_conv(y, yr, ar, precision, layer.name)
+
+
+@pytest.mark.parametrize("layer", [SMALL[1], SMALL[2], SMALL[4], SMALL[12]], ids=lambda l: l.name)
+@pytest.mark.parametrize("precision", ["f32", "f16"])
+def test_conv_exact_on_integer_inputs(layer, precision):
+    """x in {-2..2}, filter in {-1,0,1}: every partial sum is a small integer, so any summation
+    order gives the oracle's value exactly.  Separates indexing errors from rounding."""
+    dims = layer.dims()
+    x, f = workloads.make_small_integer_inputs(layer)
+    y, _, _ = gpu_conv(x, f, dims, precision)
+    yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+    assert np.array_equal(y.astype(np.float64), yr)
+
+
+def test_f16_inputs_are_the_oracles_rounding():
+    """The cast that feeds the fp16 path (torch .half()) and the oracle's rounding agree bit for bit."""
+    layer = workloads.LAYERS["cfg5k11"].with_batch(1)
+    x, f = workloads.make_inputs(layer)
+    for t in (x, f):
+        bits, _ = oracle.round_to_f16(t.numpy())
+        assert np.array_equal(bits, t.half().view(torch.int16).numpy().view(np.uint16))
+
+
+def test_delta_filter_reproduces_input_on_gpu():
+    C = 24
+    x = torch.randn((2, C, 10, 12), generator=torch.Generator().manual_seed(40))
+    f = torch.zeros((C, C, 3, 3))
+    for c in range(C):
+        f[c, c, 1, 1] = 1.0
+    dims = dict(N=2, C=C, H=10, W=12, Co=C, Kh=3, Kw=3, stride=1, pad=1)
+    y, _, _ = gpu_conv(x, f, dims, "f32")
+    assert np.array_equal(y, x.numpy())
+    y16, x16, _ = gpu_conv(x, f, dims, "f16")
+    assert np.array_equal(y16, x16)
+
+
+def test_layer_forward_host_matches_device_path():
+    layer = L("host", 3, 6, 15, 13, 20, 3, 3, 2, 1, 50)
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    for precision, tdt, code in (("f32", torch.float32, binding.F32), ("f16", torch.float16, binding.F16)):
+        y_dev, _, _ = gpu_conv(x, f, dims, precision)
+        xh = x.to(tdt).pin_memory()
+        fh = f.to(tdt).pin_memory()
+        _, _, ho, wo = binding.im2win_workspace_size(dims, code)
+        yh = torch.empty((layer.N, layer.Co, ho, wo), dtype=torch.float32).pin_memory()
+        nbytes = binding.im2win_layer_workspace_size(dims, code)
+        whole, ws = guarded(nbytes + 192, torch.uint8, 0x33)   # +192 keeps the view 256-byte aligned
+        ws = ws[192:]
+        assert ws.data_ptr() % 256 == 0
+        binding.im2win_layer_forward_host(xh, fh, yh, ws, dims)
+        torch.cuda.synchronize()
+        assert_guards_intact(whole, nbytes + 192, 0x33)
+        assert np.array_equal(yh.numpy(), y_dev)
+
+
+def test_repeated_calls_are_deterministic_and_do_not_depend_on_stale_scratch():
+    layer = SMALL[3]
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    for precision in ("f32", "f16"):
+        y1, _, _ = gpu_conv(x, f, dims, precision)
+        y2, _, _ = gpu_conv(x, f, dims, precision)
+        assert np.array_equal(y1, y2)
+
+
+# ------------------------------------------------------------ full-size layers ----
+FULL = [workloads.LAYERS[k] for k in ("cfg2", "cfg3", "cfg4a", "cfg4b", "cfg4c", "cfg5k1", "cfg5k3", "cfg5k5")]
+
+
+@pytest.mark.parametrize("layer", FULL, ids=lambda l: l.name)
+def test_full_size_sampled_outputs(layer):
+    """At the benchmark's sizes: the transform is compared bit for bit on whole images, the
+    convolution on 4096 sampled outputs (plus the corners of the output tensor) that the
+    oracle computes one by one from Eq. 1."""
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    ho, wo = oracle.out_dims(dims)
+    total = layer.N * layer.Co * ho * wo
+    rng = np.random.default_rng(layer.seed)
+    idx = np.concatenate([rng.integers(0, total, 4096), [0, total - 1, wo - 1, ho * wo - 1, total - ho * wo]])
+    for precision in layer.precisions:
+        # transform: first and last image, bit for bit
+        tdt = torch.float32 if precision == "f32" else torch.float16
+        raw = x.to(tdt).view(torch.int32 if precision == "f32" else torch.int16)
+        got = gpu_transform(raw, dims)
+        for n in (0, layer.N - 1):
+            one = dict(dims, N=1)
+            want = oracle.transform(raw[n:n + 1].numpy(), one)
+            assert np.array_equal(got[n:n + 1], want), (layer.name, precision, n)
+        del got
+        y, _, _ = gpu_conv(x, f, dims, precision)
+        xo, fo = oracle_inputs(x, f, precision)
+        yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
+        check_conv(y.reshape(-1)[idx], yr, ar, precision, layer.name)
+        # a whole image through the im2win route as well
+        one = dict(dims, N=1)
+        yi, ai = oracle.conv_im2win(xo[-1:], fo, one)
+        check_conv(y[-1:], yi, ai, precision, layer.name + " last image")
