@@ -1,6 +1,9 @@
 // C ABI of the im2win library: argument validation, buffer-size queries and
 // dispatch to the kernels.  Declarations and the contract of every entry
 // point are in include/im2win.h.
+#include <stdlib.h>
+#include <string.h>
+
 #include "common.cuh"
 
 namespace im2win {
@@ -56,10 +59,28 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
   } else {
     return IM2WIN_ERR_INVALID_ARG;
   }
+  l->f16_shift = false;
   l->koff_off = kStatusBytes;
   l->filter_off = (size_t)round_up((int64_t)l->koff_off + 4 * l->Kp, 256);
-  const int64_t fbytes = l->Kp * l->Co_pad * (dtype == IM2WIN_F32 ? 4 : 2);
+  int64_t fbytes = l->Kp * l->Co_pad * (dtype == IM2WIN_F32 ? 4 : 2);
   l->total = (size_t)round_up((int64_t)l->filter_off + fbytes, 256);
+  if (dtype == IM2WIN_F16) {
+    // The shifted-view kernel is used whenever the layer is eligible; IM2WIN_F16_KERNEL=gather
+    // forces the general gather kernel (a testing aid).  The scratch size covers both layouts.
+    const ShiftPlan plan = plan_f16_shift(g);
+    if (plan.eligible) {
+      const size_t shift_filter_off = (size_t)round_up((int64_t)kStatusBytes + 4 * plan.K2p, 256);
+      const size_t shift_total = (size_t)round_up((int64_t)shift_filter_off + plan.K2p * g.Co * g.Kw * 2, 256);
+      const char* force = getenv("IM2WIN_F16_KERNEL");
+      const bool use_shift = !(force && strcmp(force, "gather") == 0);
+      if (use_shift) {
+        l->f16_shift = true;
+        l->Kp = plan.K2p;
+        l->filter_off = shift_filter_off;
+      }
+      if (shift_total > l->total) l->total = shift_total;
+    }
+  }
   return IM2WIN_OK;
 }
 
@@ -85,9 +106,15 @@ static im2win_status conv_common(const void* window, const void* filter, float* 
     if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
     e = launch_conv_f32(static_cast<const float*>(window), y, scratch, g, l, stream);
   } else {
-    e = launch_pack_f16(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
-    if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
-    e = launch_conv_f16(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
+    if (l.f16_shift) {
+      e = launch_pack_f16_shift(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
+      if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
+      e = launch_conv_f16_shift(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
+    } else {
+      e = launch_pack_f16(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
+      if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
+      e = launch_conv_f16_gather(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
+    }
   }
   return e == cudaSuccess ? IM2WIN_OK : IM2WIN_ERR_CUDA;
 }

@@ -31,10 +31,23 @@ struct Geometry {
 //   [256, 256 + 4*Kp)   k -> element offset table (int32), -1 for padded k
 //   [filter_off, ...)   repacked filter
 struct ScratchLayout {
-  int64_t Kp;            // K rounded up to the k-block of the kernel
+  int64_t Kp;            // reduction length rounded up to the k-block of the kernel
   int64_t Co_pad;        // Co rounded up to the filter tile of the kernel
   size_t koff_off, filter_off, total;
+  bool f16_shift;        // fp16 only: the shifted-view kernel (and its filter layout) is used
 };
+
+// Tile geometry of the fp16 shifted-view kernel for one layer (see conv_f16_shift.cu).
+struct ShiftPlan {
+  bool eligible;
+  int32_t Wq;            // virtual positions per strip = Wp / s
+  int32_t rows;          // rows of one shared-memory sub-tile: 128 + halo, multiple of 8
+  int32_t total_rows;    // s * rows
+  int32_t items;         // 16-byte chunks each producer thread fills per stage
+  int64_t K2, K2p;       // C*Kh and its round-up to 64
+  int64_t VQ;            // N*Ho*Wq virtual positions
+};
+ShiftPlan plan_f16_shift(const Geometry& g);
 
 constexpr int kStatusBytes = 256;
 constexpr int kF32KBlock = 16;     // k-block of the fp32 kernel
@@ -52,7 +65,11 @@ cudaError_t launch_pack_f16(const uint16_t* filter, void* scratch, const Geometr
                             const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, const Geometry& g,
                             const ScratchLayout& l, cudaStream_t stream);
-cudaError_t launch_conv_f16(const uint16_t* window, float* y, void* scratch, const Geometry& g,
-                            const ScratchLayout& l, cudaStream_t stream);
+cudaError_t launch_pack_f16_shift(const uint16_t* filter, void* scratch, const Geometry& g,
+                                  const ScratchLayout& l, cudaStream_t stream);
+cudaError_t launch_conv_f16_gather(const uint16_t* window, float* y, void* scratch, const Geometry& g,
+                                   const ScratchLayout& l, cudaStream_t stream);
+cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratch, const Geometry& g,
+                                  const ScratchLayout& l, cudaStream_t stream);
 
 }  // namespace im2win

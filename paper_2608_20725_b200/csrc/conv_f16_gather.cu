@@ -24,16 +24,18 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "ptx_sm100.cuh"
 
 namespace im2win {
 namespace {
+
+using namespace ptx;
 
 constexpr int TILE_M = 128;               // positions per CTA (= MMA M)
 constexpr int KB = kF16KBlock;            // halves per k-block (one 128-byte row)
 constexpr int STAGES = 4;
 constexpr int A_STAGE_BYTES = TILE_M * KB * 2;
 constexpr int NUM_THREADS = 192;          // warps 0-3 producers/epilogue, 4 TMA, 5 MMA
-constexpr uint32_t SPIN_LIMIT = 1u << 24;
 
 struct ConvF16Params {
   const uint16_t* __restrict__ win;
@@ -43,112 +45,10 @@ struct ConvF16Params {
   int32_t HoWo, Wo, sKh, Co, T, num_kb;
 };
 
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok;
-}
-// Bounded wait.  Returns false (and raises the flags) when the limit is hit or
-// another thread of the CTA has already given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* status) {
-  for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 1023u) == 1023u && *abort_flag) return false;
-  }
-  *abort_flag = 1u;
-  atomicExch(status, 1u);
-  return false;
-}
-__device__ __forceinline__ void fence_proxy_async_smem() {
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_before() {
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_after() {
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
-               : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                         uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor of a k-major tile whose rows are 128 bytes
-// (64 halves) with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3ffffu) >> 4);   // start address / 16
-  d |= (uint64_t)1 << 16;                     // leading byte offset (unused with swizzle) = 16 B
-  d |= (uint64_t)(1024 >> 4) << 32;           // stride byte offset between 8-row groups
-  d |= (uint64_t)1 << 46;                     // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                     // 128-byte swizzle
-  return d;
-}
-// Instruction descriptor: fp16 A and B, both k-major, fp32 accumulator, M x N tile.
-__host__ __device__ constexpr uint32_t instr_desc_f16(int M, int N) {
-  return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
 // ---------------------------------------------------------------------- kernel
 template <int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-conv_f16_kernel(const __grid_constant__ CUtensorMap fmap, ConvF16Params q) {
+conv_f16_gather_kernel(const __grid_constant__ CUtensorMap fmap, ConvF16Params q) {
   constexpr int B_STAGE_BYTES = BN * KB * 2;
   constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 
@@ -358,16 +258,16 @@ cudaError_t launch_bn(const uint16_t* window, float* y, void* scratch, const Geo
   q.num_kb = (int32_t)(l.Kp / KB);
 
   constexpr int smem_bytes = STAGES * (A_STAGE_BYTES + BN * KB * 2) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(conv_f16_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  cudaError_t e = cudaFuncSetAttribute(conv_f16_gather_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
   dim3 grid((unsigned)((g.P + TILE_M - 1) / TILE_M), (unsigned)((g.Co + BN - 1) / BN));
-  conv_f16_kernel<BN><<<grid, NUM_THREADS, smem_bytes, stream>>>(fmap, q);
+  conv_f16_gather_kernel<BN><<<grid, NUM_THREADS, smem_bytes, stream>>>(fmap, q);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_conv_f16(const uint16_t* window, float* y, void* scratch, const Geometry& g,
+cudaError_t launch_conv_f16_gather(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                             const ScratchLayout& l, cudaStream_t stream) {
   if (g.Co <= 64) return launch_bn<64>(window, y, scratch, g, l, stream);
   if (g.Co <= 128) return launch_bn<128>(window, y, scratch, g, l, stream);

@@ -1,0 +1,408 @@
+// fp16-input / fp32-accumulate im2win convolution on the sm_100a tensor cores:
+// the "shifted-view" kernel (paper Algorithm 1's GEMM, "TC" variant, with the
+// operand staging redesigned around the im2win layout).
+//
+// In the im2win tensor a strip (n, c, ho) is a row of Wp "columns", column k'
+// being the Kh contiguous elements {u}.  The window of output wo is columns
+// wo*s .. wo*s + Kw - 1, so for a fixed kernel column v the operand of output
+// wo is column wo*s + v: the SAME data as for v = 0, shifted by v columns.
+// The kernel therefore stages each column ONCE per channel block,
+//     S[row = virtual column][k2 = c*Kh + u]     (64 halves = 128 bytes per row),
+// in the k-major 128-byte-swizzled layout, and issues the MMAs of the Kw kernel
+// columns against row-shifted views of the same tile: the shared-memory
+// descriptor of kernel column v starts (v div s) rows further, inside sub-tile
+// (v mod s).  (With stride s the columns are de-interleaved into s sub-tiles,
+// sub-tile j holding columns k' = j mod s, which turns the column stride s of
+// consecutive outputs into a row stride of 1.)  Every element of the window
+// tensor is read from L2/HBM once per output-channel tile and written to shared
+// memory once, instead of Kw times as in an im2col-style expansion.
+//
+// The MMA rows are "virtual positions" q = (n*Ho + ho)*Wq + kq with Wq = Wp/s:
+// q runs over ALL columns of a strip, also the (Wq - Wo) trailing ones that are
+// no output; their accumulator rows are computed and dropped.  Tiles are 128
+// consecutive q and may span strips and images.  Useful work is Wo/Wq of the
+// MMA work (0.97 for 56-wide rows, 0.78 for 7-wide rows).
+//
+//   GEMM:  acc[q][co] += sum_{k2} S_v[q][k2] * Fp2[v][co][k2]   for v = 0..Kw-1
+//
+// Roles: 8 producer warps gather S (one 16-byte chunk = 8 k2 per work item, lanes
+// on consecutive rows so that global reads are contiguous Kh-element records),
+// one warp streams the filter tiles Fp2[v][n0:n0+BN][kb*64:+64] by TMA, one
+// thread issues tcgen05.mma and commits to the "empty" mbarriers; afterwards the
+// producer warps read the accumulator from tensor memory and store the real
+// outputs.  Two rings of stages: S tiles (each used by Kw MMA groups) and
+// filter tiles (each used by one).  All mbarrier waits are bounded.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ptx_sm100.cuh"
+
+namespace im2win {
+namespace {
+
+using namespace ptx;
+
+constexpr int TILE_M = 128;
+constexpr int KB = kF16KBlock;
+constexpr int PRODUCER_WARPS = 8;
+constexpr int PRODUCER_THREADS = PRODUCER_WARPS * 32;
+constexpr int NUM_THREADS = PRODUCER_THREADS + 64;   // + TMA warp + MMA warp
+constexpr int MAX_STAGES = 8;
+constexpr int ITEM_GROUP = 5;                        // work items whose loads are issued together
+
+struct ShiftParams {
+  const uint16_t* __restrict__ win;
+  const int32_t* __restrict__ koff2;   // k2 -> c*chan_stride + u, -1 for padded k2
+  float* __restrict__ y;
+  uint32_t* status;
+  int64_t VQ, img_stride, strip;
+  int32_t Wq, Ho, Wo, HoWo, Co, Kh, Kw, s, num_kb;
+  int32_t rows, total_rows, sub_bytes, a_stage_bytes, sa, sb;
+};
+
+template <int BN, int ITEMS>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
+  constexpr int B_STAGE_BYTES = BN * KB * 2;
+
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+  __shared__ __align__(8) uint64_t bars[4 * MAX_STAGES + 1];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ volatile uint32_t abort_flag;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t a_ring = smem_u32(smem);
+  const uint32_t b_ring = a_ring + q.sa * q.a_stage_bytes;
+  const uint32_t a_full0 = smem_u32(&bars[0]);
+  const uint32_t a_empty0 = smem_u32(&bars[MAX_STAGES]);
+  const uint32_t b_full0 = smem_u32(&bars[2 * MAX_STAGES]);
+  const uint32_t b_empty0 = smem_u32(&bars[3 * MAX_STAGES]);
+  const uint32_t acc_bar = smem_u32(&bars[4 * MAX_STAGES]);
+
+  const int64_t q0 = (int64_t)blockIdx.x * TILE_M;
+  const int n0 = blockIdx.y * BN;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0u;
+    for (int i = 0; i < MAX_STAGES; ++i) {
+      mbar_init(a_full0 + 8 * i, PRODUCER_WARPS);
+      mbar_init(a_empty0 + 8 * i, 1);
+      mbar_init(b_full0 + 8 * i, 1);
+      mbar_init(b_empty0 + 8 * i, 1);
+    }
+    mbar_init(acc_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == PRODUCER_WARPS + 1) tmem_alloc(smem_u32(&tmem_base_slot), BN);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_acc = tmem_base_slot;
+
+  if (warp < PRODUCER_WARPS) {
+    // ---------------- producers of the S tile ---------------------------------
+    // Work item = (row, 16-byte chunk); item = chunk * total_rows + row so that the
+    // lanes of a warp walk consecutive rows (contiguous records in the window tensor).
+    int64_t base[ITEMS];      // element offset of (row, channel 0, u = 0); -1: row is beyond the tensor
+    uint32_t soff[ITEMS];     // byte offset of the chunk inside a stage (swizzled)
+    int32_t kch[ITEMS];       // first k2 of the chunk inside a k-block; -1: no such item
+    const int n_items = q.total_rows * 8;
+#pragma unroll
+    for (int it = 0; it < ITEMS; ++it) {
+      const int item = threadIdx.x + it * PRODUCER_THREADS;
+      base[it] = -1;
+      soff[it] = 0;
+      kch[it] = -1;
+      if (item < n_items) {
+        const int ch = item / q.total_rows;
+        const int ri = item - ch * q.total_rows;
+        const int sub = ri / q.rows;
+        const int i = ri - sub * q.rows;
+        kch[it] = ch * 8;
+        soff[it] = (uint32_t)(sub * q.sub_bytes + i * 128 + ((ch ^ (i & 7)) << 4));
+        const int64_t vq = q0 + i;
+        if (vq < q.VQ) {
+          const int64_t sg = vq / q.Wq;
+          const int kq = (int)(vq - sg * q.Wq);
+          const int64_t n = sg / q.Ho;
+          const int ho = (int)(sg - n * q.Ho);
+          base[it] = n * q.img_stride + ho * q.strip + (int64_t)(kq * q.s + sub) * q.Kh;
+        }
+      }
+    }
+
+    bool ok = true;
+    for (int kb = 0; kb < q.num_kb; ++kb) {
+      const int st = kb % q.sa;
+      const uint32_t round = (uint32_t)(kb / q.sa);
+      if (lane == 0) ok = mbar_wait(a_empty0 + 8 * st, (round & 1u) ^ 1u, &abort_flag, q.status);
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      if (!ok) break;
+      const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
+      const int32_t* kt = q.koff2 + kb * KB;
+#pragma unroll
+      for (int g0 = 0; g0 < ITEMS; g0 += ITEM_GROUP) {
+        constexpr int G = ITEM_GROUP;
+        int4 o[G][2];
+        uint32_t h[G][8];
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) {
+          const int it = g0 + gi;
+          if (it < ITEMS && kch[it] >= 0) {
+            o[gi][0] = __ldg(reinterpret_cast<const int4*>(kt + kch[it]));
+            o[gi][1] = __ldg(reinterpret_cast<const int4*>(kt + kch[it] + 4));
+          } else {
+            o[gi][0] = o[gi][1] = make_int4(-1, -1, -1, -1);
+          }
+        }
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) {
+          const int it = g0 + gi;
+          if (it < ITEMS) {
+            const int32_t off[8] = {o[gi][0].x, o[gi][0].y, o[gi][0].z, o[gi][0].w,
+                                    o[gi][1].x, o[gi][1].y, o[gi][1].z, o[gi][1].w};
+            const bool row_ok = base[it] >= 0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              uint32_t v = 0;
+              if (row_ok && off[e] >= 0) v = (uint32_t)__ldg(q.win + base[it] + off[e]);
+              h[gi][e] = v;
+            }
+          }
+        }
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) {
+          const int it = g0 + gi;
+          if (it < ITEMS && kch[it] >= 0) {
+            const uint32_t w0 = h[gi][0] | (h[gi][1] << 16), w1 = h[gi][2] | (h[gi][3] << 16);
+            const uint32_t w2 = h[gi][4] | (h[gi][5] << 16), w3 = h[gi][6] | (h[gi][7] << 16);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_stage + soff[it]), "r"(w0), "r"(w1),
+                         "r"(w2), "r"(w3)
+                         : "memory");
+          }
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(a_full0 + 8 * st);
+    }
+
+    // ---------------- epilogue --------------------------------------------------
+    if (ok && lane == 0) ok = mbar_wait(acc_bar, 0u, &abort_flag, q.status);
+    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+    if (ok) {
+      tc_fence_after();
+      const int lq = warp & 3;                 // tensor-memory lane quadrant this warp may read
+      const int chalf = warp >> 2;             // which half of the channel tile
+      const int64_t vq = q0 + lq * 32 + lane;  // accumulator row = virtual position
+      bool valid = false;
+      float* yrow = q.y;
+      if (vq < q.VQ) {
+        const int64_t sg = vq / q.Wq;
+        const int kq = (int)(vq - sg * q.Wq);
+        const int64_t n = sg / q.Ho;
+        const int ho = (int)(sg - n * q.Ho);
+        valid = kq < q.Wo;                     // trailing columns of a strip are no output
+        yrow += (n * q.Co) * q.HoWo + ho * q.Wo + kq;
+      }
+      const uint32_t lane_base = tmem_acc + ((uint32_t)(lq * 32) << 16);
+#pragma unroll 1
+      for (int c0 = chalf * (BN / 2); c0 < (chalf + 1) * (BN / 2); c0 += 32) {
+        if (n0 + c0 >= q.Co) break;
+        uint32_t v[32];
+        tmem_ld32(lane_base + (uint32_t)c0, v);
+        if (valid) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int co = n0 + c0 + j;
+            if (co < q.Co) yrow[(int64_t)co * q.HoWo] = __uint_as_float(v[j]);
+          }
+        }
+      }
+    }
+  } else if (warp == PRODUCER_WARPS) {
+    // ---------------- TMA producer of the filter tiles -------------------------
+    if (lane == 0) {
+      int g = 0;
+      for (int kb = 0; kb < q.num_kb; ++kb) {
+        for (int v = 0; v < q.Kw; ++v, ++g) {
+          const int st = g % q.sb;
+          const uint32_t round = (uint32_t)(g / q.sb);
+          if (!mbar_wait(b_empty0 + 8 * st, (round & 1u) ^ 1u, &abort_flag, q.status)) goto tma_done;
+          const uint32_t bar = b_full0 + 8 * st;
+          mbar_arrive_expect_tx(bar, B_STAGE_BYTES);
+          tma_load_3d(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0, v, bar);
+        }
+      }
+    tma_done:;
+    }
+  } else {
+    // ---------------- MMA issuer ------------------------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc_f16(TILE_M, BN);
+      bool ok = true;
+      int g = 0;
+      for (int kb = 0; kb < q.num_kb && ok; ++kb) {
+        const int sta = kb % q.sa;
+        ok = mbar_wait(a_full0 + 8 * sta, (uint32_t)(kb / q.sa) & 1u, &abort_flag, q.status);
+        if (!ok) break;
+        const uint32_t a_stage = a_ring + sta * q.a_stage_bytes;
+        for (int v = 0; v < q.Kw; ++v, ++g) {
+          const int stb = g % q.sb;
+          ok = mbar_wait(b_full0 + 8 * stb, (uint32_t)(g / q.sb) & 1u, &abort_flag, q.status);
+          if (!ok) break;
+          tc_fence_after();
+          const int sub = v % q.s;
+          const int shift = v / q.s;
+          const uint32_t a_addr = a_stage + sub * q.sub_bytes + shift * 128;
+          const uint32_t b_addr = b_ring + stb * B_STAGE_BYTES;
+#pragma unroll
+          for (int j = 0; j < KB / 16; ++j) {
+            const uint64_t ad = smem_desc_k_major_sw128(a_addr + j * 32);
+            const uint64_t bd = smem_desc_k_major_sw128(b_addr + j * 32);
+            umma_f16(tmem_acc, ad, bd, idesc, (g > 0 || j > 0) ? 1u : 0u);
+          }
+          umma_commit(b_empty0 + 8 * stb);
+        }
+        if (ok) umma_commit(a_empty0 + 8 * sta);
+      }
+      if (ok) umma_commit(acc_bar);
+    }
+  }
+
+  // ---------------- teardown ---------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == PRODUCER_WARPS + 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_acc, BN);
+  }
+}
+
+// ------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+constexpr int kSmemBudget = 220 * 1024;
+
+template <int BN>
+void choose_stages(const ShiftPlan& plan, int* sa, int* sb) {
+  const int a_bytes = plan.total_rows * 128;
+  const int b_bytes = BN * KB * 2;
+  int a = 2, b = 2;
+  // Grow the rings alternately while they fit: filter stages turn over Kw times faster.
+  for (;;) {
+    bool grew = false;
+    if (b < MAX_STAGES && (a * a_bytes + (b + 1) * b_bytes) <= kSmemBudget - 2048 && b < 6) { ++b; grew = true; }
+    if (a < 4 && ((a + 1) * a_bytes + b * b_bytes) <= kSmemBudget - 2048) { ++a; grew = true; }
+    if (!grew) break;
+  }
+  *sa = a;
+  *sb = b;
+}
+
+template <int BN, int ITEMS>
+cudaError_t launch_variant(const CUtensorMap& fmap, const ShiftParams& q0, const ShiftPlan& plan, int co,
+                           cudaStream_t stream) {
+  ShiftParams q = q0;
+  int sa, sb;
+  choose_stages<BN>(plan, &sa, &sb);
+  q.sa = sa;
+  q.sb = sb;
+  const int smem_bytes = sa * q.a_stage_bytes + sb * BN * KB * 2 + 1024;
+  cudaError_t e = cudaFuncSetAttribute(conv_f16_shift_kernel<BN, ITEMS>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  if (e != cudaSuccess) return e;
+  dim3 grid((unsigned)((plan.VQ + TILE_M - 1) / TILE_M), (unsigned)((co + BN - 1) / BN));
+  conv_f16_shift_kernel<BN, ITEMS><<<grid, NUM_THREADS, smem_bytes, stream>>>(fmap, q);
+  return cudaGetLastError();
+}
+
+template <int BN>
+cudaError_t launch_bn(const CUtensorMap& fmap, const ShiftParams& q, const ShiftPlan& plan, int co,
+                      cudaStream_t stream) {
+  if (plan.items <= 5) return launch_variant<BN, 5>(fmap, q, plan, co, stream);
+  if (plan.items <= 10) return launch_variant<BN, 10>(fmap, q, plan, co, stream);
+  return launch_variant<BN, 15>(fmap, q, plan, co, stream);
+}
+
+}  // namespace
+
+ShiftPlan plan_f16_shift(const Geometry& g) {
+  ShiftPlan p{};
+  p.eligible = false;
+  if (g.Wp % g.s != 0) return p;
+  p.Wq = g.Wp / g.s;
+  const int halo = (g.Kw - 1 + g.s - 1) / g.s;
+  p.rows = TILE_M + (halo + 7) / 8 * 8;
+  p.total_rows = g.s * p.rows;
+  p.items = (p.total_rows * 8 + PRODUCER_THREADS - 1) / PRODUCER_THREADS;
+  p.K2 = (int64_t)g.C * g.Kh;
+  p.K2p = (p.K2 + KB - 1) / KB * KB;
+  p.VQ = (int64_t)g.N * g.Ho * p.Wq;
+  if (p.items > 15) return p;
+  // two stages of each ring must fit even for the widest channel tile
+  if (2 * p.total_rows * 128 + 2 * 256 * KB * 2 > kSmemBudget - 2048) return p;
+  if ((p.VQ + TILE_M - 1) / TILE_M >= ((int64_t)1 << 31)) return p;
+  p.eligible = true;
+  return p;
+}
+
+cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratch, const Geometry& g,
+                                  const ScratchLayout& l, cudaStream_t stream) {
+  const ShiftPlan plan = plan_f16_shift(g);
+  if (!plan.eligible) return cudaErrorInvalidValue;
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return cudaErrorNotSupported;
+  unsigned char* base = static_cast<unsigned char*>(scratch);
+  const int bn = g.Co <= 64 ? 64 : (g.Co <= 128 ? 128 : 256);
+
+  // Filter as Fp2[v][co][k2p] halves: a 3-D tensor (k2 fastest), one box = 64 k2 x BN channels of one v.
+  CUtensorMap fmap;
+  const cuuint64_t dims[3] = {(cuuint64_t)plan.K2p, (cuuint64_t)g.Co, (cuuint64_t)g.Kw};
+  const cuuint64_t strides[2] = {(cuuint64_t)plan.K2p * 2, (cuuint64_t)plan.K2p * 2 * (cuuint64_t)g.Co};
+  const cuuint32_t box[3] = {(cuuint32_t)KB, (cuuint32_t)bn, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult cr = encode(&fmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base + l.filter_off, dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+
+  ShiftParams q;
+  q.win = window;
+  q.koff2 = reinterpret_cast<const int32_t*>(base + l.koff_off);
+  q.y = y;
+  q.status = reinterpret_cast<uint32_t*>(base);
+  q.VQ = plan.VQ; q.img_stride = g.img_stride; q.strip = g.strip;
+  q.Wq = plan.Wq; q.Ho = g.Ho; q.Wo = g.Wo; q.HoWo = g.Ho * g.Wo; q.Co = g.Co;
+  q.Kh = g.Kh; q.Kw = g.Kw; q.s = g.s; q.num_kb = (int32_t)(plan.K2p / KB);
+  q.rows = plan.rows; q.total_rows = plan.total_rows;
+  q.sub_bytes = plan.rows * 128; q.a_stage_bytes = plan.total_rows * 128;
+  q.sa = q.sb = 2;
+  if (bn == 64) return launch_bn<64>(fmap, q, plan, g.Co, stream);
+  if (bn == 128) return launch_bn<128>(fmap, q, plan, g.Co, stream);
+  return launch_bn<256>(fmap, q, plan, g.Co, stream);
+}
+
+}  // namespace im2win

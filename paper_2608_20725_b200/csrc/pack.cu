@@ -9,7 +9,8 @@
 // the zero-padded tail k >= K hold -1.  It also clears the status block at the
 // start of the scratch buffer.
 //   fp32 kernel layout: Fk[k][Co_pad]  (co contiguous), zero padded in k and co
-//   fp16 kernel layout: Fp[co][Kp]     (k contiguous),  zero padded in k
+//   fp16 gather kernel: Fp[co][Kp]     (k contiguous),  zero padded in k
+//   fp16 shifted-view kernel: Fp2[v][co][K2p] with k2 = c*Kh + u (see pack_f16_shift_kernel)
 #include "common.cuh"
 
 namespace im2win {
@@ -77,6 +78,34 @@ __global__ void pack_f16_kernel(const uint16_t* __restrict__ f, uint16_t* __rest
   }
 }
 
+// Layout of the shifted-view fp16 kernel: Fp2[v][co][k2], k2 = c*Kh + u (zero padded to K2p),
+// and the table k2 -> c*chan_stride + u.
+__global__ void pack_f16_shift_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp,
+                                      int32_t* __restrict__ koff, uint32_t* __restrict__ status,
+                                      PackParams q) {
+  if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
+  const int64_t K2 = (int64_t)q.C * q.Kh;
+  const int64_t per_v = q.Kp * q.Co;
+  const int64_t total = per_v * q.Kw;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int64_t v = i / per_v;
+    const int64_t r = i - v * per_v;
+    const int64_t co = r / q.Kp;
+    const int64_t k2 = r - co * q.Kp;
+    uint16_t val = 0;
+    int32_t off = -1;
+    if (k2 < K2) {
+      const int64_t c = k2 / q.Kh;
+      const int64_t u = k2 - c * q.Kh;
+      val = f[((co * q.C + c) * q.Kh + u) * q.Kw + v];
+      off = (int32_t)(c * q.chan_stride + u);
+    }
+    fp[i] = val;
+    if (v == 0 && co == 0) koff[k2] = off;
+  }
+}
+
 PackParams make_params(const Geometry& g, const ScratchLayout& l) {
   PackParams q;
   q.C = g.C; q.Co = g.Co; q.Kh = g.Kh; q.Kw = g.Kw; q.T = g.T;
@@ -108,6 +137,16 @@ cudaError_t launch_pack_f16(const uint16_t* filter, void* scratch, const Geometr
   unsigned char* base = static_cast<unsigned char*>(scratch);
   PackParams q = make_params(g, l);
   pack_f16_kernel<<<grid_for(q.Kp * q.Co), 256, 0, stream>>>(
+      filter, reinterpret_cast<uint16_t*>(base + l.filter_off),
+      reinterpret_cast<int32_t*>(base + l.koff_off), reinterpret_cast<uint32_t*>(base), q);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pack_f16_shift(const uint16_t* filter, void* scratch, const Geometry& g,
+                                  const ScratchLayout& l, cudaStream_t stream) {
+  unsigned char* base = static_cast<unsigned char*>(scratch);
+  PackParams q = make_params(g, l);
+  pack_f16_shift_kernel<<<grid_for(q.Kp * q.Co * q.Kw), 256, 0, stream>>>(
       filter, reinterpret_cast<uint16_t*>(base + l.filter_off),
       reinterpret_cast<int32_t*>(base + l.koff_off), reinterpret_cast<uint32_t*>(base), q);
   return cudaGetLastError();

@@ -1,5 +1,7 @@
 """Helpers of the GPU parity tests: run the CUDA path through the C ABI with guard bands
 around every output buffer, and compare with the CPU oracle."""
+import os
+
 import numpy as np
 import torch
 
@@ -42,8 +44,15 @@ def gpu_transform(x_cpu: torch.Tensor, dims: dict) -> np.ndarray:
 
 
 def gpu_conv(x_cpu: torch.Tensor, f_cpu: torch.Tensor, dims: dict, precision: str):
-    """Transform + convolution on the GPU.  precision 'f32' or 'f16' (inputs are cast with
-    torch's round-to-nearest-even conversion).  Returns (y float32 numpy, x_used, f_used as float32 numpy)."""
+    """Transform + convolution on the GPU.  precision 'f32', 'f16' (the kernel the library picks)
+    or 'f16-gather' (the general fp16 kernel forced); inputs are cast with torch's
+    round-to-nearest-even conversion.  Returns (y float32 numpy, x_used, f_used as float32 numpy)."""
+    if precision == "f16-gather":
+        os.environ["IM2WIN_F16_KERNEL"] = "gather"
+        try:
+            return gpu_conv(x_cpu, f_cpu, dims, "f16")
+        finally:
+            del os.environ["IM2WIN_F16_KERNEL"]
     tdt = torch.float32 if precision == "f32" else torch.float16
     code = binding.F32 if precision == "f32" else binding.F16
     xd = x_cpu.to(tdt).cuda().contiguous()
@@ -73,7 +82,7 @@ def oracle_inputs(x_cpu: torch.Tensor, f_cpu: torch.Tensor, precision: str):
     oracle's own routine for the fp16 path."""
     x = x_cpu.numpy().astype(np.float32)
     f = f_cpu.numpy().astype(np.float32)
-    if precision == "f16":
+    if precision.startswith("f16"):
         _, x = oracle.round_to_f16(x)
         _, f = oracle.round_to_f16(f)
     return x, f
