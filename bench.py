@@ -17,7 +17,6 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
 import threading
 import time
@@ -56,59 +55,71 @@ def layer_flops(layer, ho, wo):
 
 # --------------------------------------------------------------------- clocks ----
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and throttle reasons of one GPU through NVML (read-only queries)
+    from a background thread while the timed region runs."""
 
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20,
+               "hw_thermal_slowdown": 0x40}
 
-    def __init__(self, index: int):
+    def __init__(self, index: int, period_s: float = 0.002):
         self.index = index
-        self.proc = None
-        self.lines = []
+        self.period = period_s
+        self.samples = []
+        self.stop_flag = threading.Event()
         self.thread = None
+        self.handle = None
+        self.nvml = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if visible:
+                ids = [v.strip() for v in visible.split(",") if v.strip()]
+                if index < len(ids) and ids[index].isdigit():
+                    phys = int(ids[index])
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.nvml = pynvml
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nvml = None
+
+    def _sample(self):
+        n = self.nvml
+        try:
+            mhz = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+            reasons = int(n.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+            power = n.nvmlDeviceGetPowerUsage(self.handle) / 1000.0
+            self.samples.append((mhz, reasons, power))
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self.stop_flag.is_set():
+            self._sample()
+            time.sleep(self.period)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
-                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except Exception:
-            self.proc = None
+        if self.nvml is None:
             return
-        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self._sample()
+        self.thread = threading.Thread(target=self._run, daemon=True)
         self.thread.start()
 
-    def _pump(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
-
     def stop(self):
-        if self.proc is None:
+        if self.nvml is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons, power = [], [], set(), []
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.lines:
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 7:
-                continue
-            try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
-                power.append(float(parts[2]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm), "power_w_max": max(power) if power else None}
+        self._sample()
+        self.stop_flag.set()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        mhz = sorted(s[0] for s in self.samples)
+        seen = 0
+        for s in self.samples:
+            seen |= s[1]
+        reasons = sorted(k for k, bit in self.REASONS.items() if seen & bit)
+        return {"sm_mhz": mhz[len(mhz) // 2] if mhz else None, "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(mhz), "power_w_max": max((s[2] for s in self.samples), default=None)}
 
 
 # -------------------------------------------------------------- the GPU arm ----
@@ -234,12 +245,15 @@ def time_cpu_oracle(layer, target_seconds=12.0):
     t0 = time.perf_counter()
     oracle.conv_im2win_range(xn, fn, dims, 0, 1)
     t1 = time.perf_counter() - t0
-    n = int(max(1, min(layer.N - 1, target_seconds / max(t1, 1e-6))))
+    n = int(max(1, min(layer.N, target_seconds / max(t1, 1e-6))))
+    reps = int(max(1, min(50, round(target_seconds / max(t1 * n, 1e-6)))))
     t0 = time.perf_counter()
-    oracle.conv_im2win_range(xn, fn, dims, 1, 1 + n)
+    for _ in range(reps):
+        oracle.conv_im2win_range(xn, fn, dims, 0, n)
     dt = time.perf_counter() - t0
-    return {"value": per_image * n / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"fp64 im2win route on {n} of {layer.N} images of {layer.name} ({dt:.1f} s)"}
+    return {"value": per_image * n * reps / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"fp64 im2win route (transform + convolution) on {n} of {layer.N} images of {layer.name}, "
+                      f"{reps} passes ({dt:.1f} s)"}
 
 
 def run_gpu_arm(args):
@@ -360,7 +374,8 @@ def run_gpu_arm(args):
             out["cpu_baseline"] = time_cpu_oracle(layer)
         print(json.dumps(out))
     if args.report and rank == 0:
-        write_report(args.report, peaks, peak_kind)
+        write_report(args.report, peaks, peak_kind,
+                     names=args.report_layers.split(",") if args.report_layers else None)
     if dist is not None:
         dist.destroy_process_group()
 
@@ -372,6 +387,9 @@ def time_call(fn, iters, flush):
     best = float("inf")
     for _ in range(iters):
         flush.zero_()
+        # keep the GPU busy (~0.3 ms) while the host queues the events and the call, so that the
+        # bracket measures device time, not launch latency
+        torch.cuda._sleep(600_000)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         fn()
@@ -408,6 +426,24 @@ def write_report(path, peaks, peak_kind, names=None, iters=10):
     with open(path, "w") as fh:
         for row in rows:
             fh.write(json.dumps(row) + "\n")
+
+
+def run_kernel_loop(spec, launches=3):
+    """`LAYER:KERNEL[:BATCH]` -- a few launches of one kernel of one layer (for profilers)."""
+    parts = spec.split(":")
+    table = dict(workloads.LAYERS)
+    table.update(workloads.TABLE1_LAYERS)
+    layer = table[parts[0]]
+    kind, prec = parts[1].rsplit("_", 1)
+    if len(parts) > 2:
+        layer = layer.with_batch(int(parts[2]))
+    runner = LayerRunner(layer, (prec,))
+    runner.transform(prec)
+    fn = runner.transform if kind == "transform" else runner.conv
+    for _ in range(launches):
+        fn(prec)
+    runner.b.im2win_check_status(runner.dev[prec]["scratch"]) if kind == "conv" else torch.cuda.synchronize()
+    print(f"kernel-loop {spec}: {launches} launches done")
 
 
 # ------------------------------------------------------ the reference arm ----
@@ -462,7 +498,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--report", default=None, help="also write a per-layer, per-kernel report (JSON lines)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-loop", default=None, metavar="LAYER:KERNEL[:BATCH]",
+                    help="run a few launches of one kernel (e.g. cfg2:conv_f32) and exit; for profilers")
+    ap.add_argument("--report-layers", default=None, help="comma-separated layer names for --report")
     args = ap.parse_args()
+    if args.kernel_loop:
+        run_kernel_loop(args.kernel_loop)
+        return
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

@@ -99,9 +99,22 @@ def _dtype_code(t: torch.dtype) -> int:
     raise TypeError(f"unsupported dtype {t}")
 
 
+_size_cache: dict = {}
+
+
 def im2win_workspace_size(shape, dtype: int) -> Tuple[int, int, int, int]:
     """Returns (window_bytes, scratch_bytes, Ho, Wo)."""
     s = as_shape(shape)
+    key = (s.N, s.C, s.H, s.W, s.Co, s.Kh, s.Kw, s.stride, s.pad, dtype)
+    hit = _size_cache.get(key)
+    if hit is not None:
+        return hit
+    out = _workspace_size_uncached(s, dtype)
+    _size_cache[key] = out
+    return out
+
+
+def _workspace_size_uncached(s: Shape, dtype: int) -> Tuple[int, int, int, int]:
     wb, sb = ctypes.c_size_t(), ctypes.c_size_t()
     ho, wo = ctypes.c_int32(), ctypes.c_int32()
     _check(lib().im2win_workspace_size(ctypes.byref(s), dtype, ctypes.byref(wb), ctypes.byref(sb),

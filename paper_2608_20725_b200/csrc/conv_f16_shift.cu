@@ -33,6 +33,7 @@
 // outputs.  Two rings of stages: S tiles (each used by Kw MMA groups) and
 // filter tiles (each used by one).  All mbarrier waits are bounded.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
@@ -57,11 +58,13 @@ struct ShiftParams {
   uint32_t* status;
   int64_t VQ, img_stride, strip;
   int32_t Wq, Ho, Wo, HoWo, Co, Kh, Kw, s, num_kb;
-  int32_t rows, total_rows, sub_bytes, a_stage_bytes, sa, sb;
+  int32_t halo8;          // halo rows of a sub-tile, rounded up to 8
+  int32_t nbig;           // the first nbig tiles are 256 positions tall (two MMA halves), the rest 128
+  int32_t a_stage_bytes, sa, sb;
 };
 
 template <int BN, int ITEMS>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(NUM_THREADS, (BN <= 128 ? 2 : 1))
 conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
   constexpr int B_STAGE_BYTES = BN * KB * 2;
 
@@ -81,8 +84,15 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
   const uint32_t b_empty0 = smem_u32(&bars[3 * MAX_STAGES]);
   const uint32_t acc_bar = smem_u32(&bars[4 * MAX_STAGES]);
 
-  const int64_t q0 = (int64_t)blockIdx.x * TILE_M;
+  // Tall tiles (two 128-row MMA halves sharing every filter stage) come first in the grid.
+  const bool big = (int)blockIdx.x < q.nbig;
+  const int mt = big ? 2 : 1;
+  const int64_t q0 = big ? (int64_t)blockIdx.x * (2 * TILE_M)
+                         : (int64_t)q.nbig * (2 * TILE_M) + (int64_t)((int)blockIdx.x - q.nbig) * TILE_M;
   const int n0 = blockIdx.y * BN;
+  const int rows = TILE_M * mt + q.halo8;          // rows of one sub-tile
+  const int total_rows = q.s * rows;
+  const int sub_bytes = rows * 128;
 
   if (threadIdx.x == 0) {
     abort_flag = 0u;
@@ -95,7 +105,10 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
     mbar_init(acc_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == PRODUCER_WARPS + 1) tmem_alloc(smem_u32(&tmem_base_slot), BN);
+  if (warp == PRODUCER_WARPS + 1) tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
+  // k2 -> element offset table of the whole reduction, kept in shared memory
+  int32_t* koff_s = reinterpret_cast<int32_t*>(smem + q.sa * q.a_stage_bytes + q.sb * B_STAGE_BYTES);
+  for (int i = threadIdx.x; i < q.num_kb * KB; i += NUM_THREADS) koff_s[i] = __ldg(q.koff2 + i);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -105,30 +118,36 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
     // ---------------- producers of the S tile ---------------------------------
     // Work item = (row, 16-byte chunk); item = chunk * total_rows + row so that the
     // lanes of a warp walk consecutive rows (contiguous records in the window tensor).
-    int64_t base[ITEMS];      // element offset of (row, channel 0, u = 0); -1: row is beyond the tensor
-    uint32_t soff[ITEMS];     // byte offset of the chunk inside a stage (swizzled)
-    int32_t kch[ITEMS];       // first k2 of the chunk inside a k-block; -1: no such item
-    const int n_items = q.total_rows * 8;
+    // Per item: rel = element offset of (row, channel 0, u 0) from the tile's first image,
+    // meta = swizzled byte offset of the chunk in a stage | chunk index (bits 0-2) |
+    // row-inside-tensor flag (bit 3); 0xffffffff marks "no such item".
+    // Loads are unconditional (a dead row or a padded k2 reads element 0 of the tile's
+    // image and is masked afterwards) so that the compiler can issue all of a group's
+    // loads back to back.
+    uint32_t rel[ITEMS], meta[ITEMS];
+    const int n_items = total_rows * 8;
+    const int64_t img_rows = (int64_t)q.Ho * q.Wq;          // virtual positions per image
+    const int64_t n_first = q0 / img_rows;
+    const uint16_t* __restrict__ tile_win = q.win + n_first * q.img_stride;
 #pragma unroll
     for (int it = 0; it < ITEMS; ++it) {
       const int item = threadIdx.x + it * PRODUCER_THREADS;
-      base[it] = -1;
-      soff[it] = 0;
-      kch[it] = -1;
+      rel[it] = 0;
+      meta[it] = 0xffffffffu;
       if (item < n_items) {
-        const int ch = item / q.total_rows;
-        const int ri = item - ch * q.total_rows;
-        const int sub = ri / q.rows;
-        const int i = ri - sub * q.rows;
-        kch[it] = ch * 8;
-        soff[it] = (uint32_t)(sub * q.sub_bytes + i * 128 + ((ch ^ (i & 7)) << 4));
+        const int ch = item / total_rows;
+        const int ri = item - ch * total_rows;
+        const int sub = ri / rows;
+        const int i = ri - sub * rows;
+        meta[it] = (uint32_t)(sub * sub_bytes + i * 128 + ((ch ^ (i & 7)) << 4)) | (uint32_t)ch;
         const int64_t vq = q0 + i;
         if (vq < q.VQ) {
           const int64_t sg = vq / q.Wq;
           const int kq = (int)(vq - sg * q.Wq);
           const int64_t n = sg / q.Ho;
           const int ho = (int)(sg - n * q.Ho);
-          base[it] = n * q.img_stride + ho * q.strip + (int64_t)(kq * q.s + sub) * q.Kh;
+          rel[it] = (uint32_t)((n - n_first) * q.img_stride + ho * q.strip + (int64_t)(kq * q.s + sub) * q.Kh);
+          meta[it] |= 8u;
         }
       }
     }
@@ -141,45 +160,32 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
       if (!ok) break;
       const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
-      const int32_t* kt = q.koff2 + kb * KB;
+      const int4* kt = reinterpret_cast<const int4*>(koff_s + kb * KB);   // this k-block's offsets (shared memory)
 #pragma unroll
       for (int g0 = 0; g0 < ITEMS; g0 += ITEM_GROUP) {
         constexpr int G = ITEM_GROUP;
-        int4 o[G][2];
         uint32_t h[G][8];
 #pragma unroll
         for (int gi = 0; gi < G; ++gi) {
           const int it = g0 + gi;
-          if (it < ITEMS && kch[it] >= 0) {
-            o[gi][0] = __ldg(reinterpret_cast<const int4*>(kt + kch[it]));
-            o[gi][1] = __ldg(reinterpret_cast<const int4*>(kt + kch[it] + 4));
-          } else {
-            o[gi][0] = o[gi][1] = make_int4(-1, -1, -1, -1);
-          }
+          const int ch = (int)(meta[it] & 7u);
+          const int4 o0 = kt[ch * 2], o1 = kt[ch * 2 + 1];
+          const int32_t off[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
+          const uint16_t* src = tile_win + rel[it];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) h[gi][e] = (uint32_t)__ldg(src + max(off[e], 0));
+          const bool row_ok = (meta[it] & 8u) != 0;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) h[gi][e] = (row_ok && off[e] >= 0) ? h[gi][e] : 0u;
         }
 #pragma unroll
         for (int gi = 0; gi < G; ++gi) {
           const int it = g0 + gi;
-          if (it < ITEMS) {
-            const int32_t off[8] = {o[gi][0].x, o[gi][0].y, o[gi][0].z, o[gi][0].w,
-                                    o[gi][1].x, o[gi][1].y, o[gi][1].z, o[gi][1].w};
-            const bool row_ok = base[it] >= 0;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              uint32_t v = 0;
-              if (row_ok && off[e] >= 0) v = (uint32_t)__ldg(q.win + base[it] + off[e]);
-              h[gi][e] = v;
-            }
-          }
-        }
-#pragma unroll
-        for (int gi = 0; gi < G; ++gi) {
-          const int it = g0 + gi;
-          if (it < ITEMS && kch[it] >= 0) {
+          if (meta[it] != 0xffffffffu) {
             const uint32_t w0 = h[gi][0] | (h[gi][1] << 16), w1 = h[gi][2] | (h[gi][3] << 16);
             const uint32_t w2 = h[gi][4] | (h[gi][5] << 16), w3 = h[gi][6] | (h[gi][7] << 16);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_stage + soff[it]), "r"(w0), "r"(w1),
-                         "r"(w2), "r"(w3)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_stage + (meta[it] & ~15u)), "r"(w0),
+                         "r"(w1), "r"(w2), "r"(w3)
                          : "memory");
           }
         }
@@ -196,28 +202,30 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
       tc_fence_after();
       const int lq = warp & 3;                 // tensor-memory lane quadrant this warp may read
       const int chalf = warp >> 2;             // which half of the channel tile
-      const int64_t vq = q0 + lq * 32 + lane;  // accumulator row = virtual position
-      bool valid = false;
-      float* yrow = q.y;
-      if (vq < q.VQ) {
-        const int64_t sg = vq / q.Wq;
-        const int kq = (int)(vq - sg * q.Wq);
-        const int64_t n = sg / q.Ho;
-        const int ho = (int)(sg - n * q.Ho);
-        valid = kq < q.Wo;                     // trailing columns of a strip are no output
-        yrow += (n * q.Co) * q.HoWo + ho * q.Wo + kq;
-      }
-      const uint32_t lane_base = tmem_acc + ((uint32_t)(lq * 32) << 16);
+      for (int half = 0; half < mt; ++half) {
+        const int64_t vq = q0 + half * TILE_M + lq * 32 + lane;   // accumulator row = virtual position
+        bool valid = false;
+        float* yrow = q.y;
+        if (vq < q.VQ) {
+          const int64_t sg = vq / q.Wq;
+          const int kq = (int)(vq - sg * q.Wq);
+          const int64_t n = sg / q.Ho;
+          const int ho = (int)(sg - n * q.Ho);
+          valid = kq < q.Wo;                   // trailing columns of a strip are no output
+          yrow += (n * q.Co) * q.HoWo + ho * q.Wo + kq;
+        }
+        const uint32_t lane_base = tmem_acc + ((uint32_t)(lq * 32) << 16) + (uint32_t)(half * BN);
 #pragma unroll 1
-      for (int c0 = chalf * (BN / 2); c0 < (chalf + 1) * (BN / 2); c0 += 32) {
-        if (n0 + c0 >= q.Co) break;
-        uint32_t v[32];
-        tmem_ld32(lane_base + (uint32_t)c0, v);
-        if (valid) {
+        for (int c0 = chalf * (BN / 2); c0 < (chalf + 1) * (BN / 2); c0 += 32) {
+          if (n0 + c0 >= q.Co) break;
+          uint32_t v[32];
+          tmem_ld32(lane_base + (uint32_t)c0, v);
+          if (valid) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int co = n0 + c0 + j;
-            if (co < q.Co) yrow[(int64_t)co * q.HoWo] = __uint_as_float(v[j]);
+            for (int j = 0; j < 32; ++j) {
+              const int co = n0 + c0 + j;
+              if (co < q.Co) yrow[(int64_t)co * q.HoWo] = __uint_as_float(v[j]);
+            }
           }
         }
       }
@@ -256,13 +264,15 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
           tc_fence_after();
           const int sub = v % q.s;
           const int shift = v / q.s;
-          const uint32_t a_addr = a_stage + sub * q.sub_bytes + shift * 128;
           const uint32_t b_addr = b_ring + stb * B_STAGE_BYTES;
+          for (int half = 0; half < mt; ++half) {
+            const uint32_t a_addr = a_stage + sub * sub_bytes + (half * TILE_M + shift) * 128;
 #pragma unroll
-          for (int j = 0; j < KB / 16; ++j) {
-            const uint64_t ad = smem_desc_k_major_sw128(a_addr + j * 32);
-            const uint64_t bd = smem_desc_k_major_sw128(b_addr + j * 32);
-            umma_f16(tmem_acc, ad, bd, idesc, (g > 0 || j > 0) ? 1u : 0u);
+            for (int j = 0; j < KB / 16; ++j) {
+              const uint64_t ad = smem_desc_k_major_sw128(a_addr + j * 32);
+              const uint64_t bd = smem_desc_k_major_sw128(b_addr + j * 32);
+              umma_f16(tmem_acc + (uint32_t)(half * BN), ad, bd, idesc, (g > 0 || j > 0) ? 1u : 0u);
+            }
           }
           umma_commit(b_empty0 + 8 * stb);
         }
@@ -282,7 +292,7 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
   if (warp == PRODUCER_WARPS + 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_acc, BN);
+    tmem_dealloc(tmem_acc, 2 * BN);
   }
 }
 
@@ -307,17 +317,18 @@ EncodeTiledFn get_encode_fn() {
 constexpr int kSmemBudget = 220 * 1024;
 
 template <int BN>
-void choose_stages(const ShiftPlan& plan, int* sa, int* sb) {
-  const int a_bytes = plan.total_rows * 128;
+void choose_stages(const ShiftPlan& plan, int a_bytes, int* sa, int* sb) {
   const int b_bytes = BN * KB * 2;
+  // Narrow channel tiles leave room for two CTAs per SM: give each half of the budget.
+  const int budget = (BN <= 128 ? kSmemBudget / 2 : kSmemBudget) - 2048 - (int)plan.K2p * 4;
   int a = 2, b = 2;
-  // Grow the rings alternately while they fit: filter stages turn over Kw times faster.
-  for (;;) {
-    bool grew = false;
-    if (b < MAX_STAGES && (a * a_bytes + (b + 1) * b_bytes) <= kSmemBudget - 2048 && b < 6) { ++b; grew = true; }
-    if (a < 4 && ((a + 1) * a_bytes + b * b_bytes) <= kSmemBudget - 2048) { ++a; grew = true; }
-    if (!grew) break;
-  }
+  // Filter stages turn over Kw (x2 for tall tiles) times faster than S stages and hide the
+  // L2 latency of the TMA loads: grow them to 4 first, then S to 3, then both further.
+  auto fits = [&](int aa, int bb) { return aa * a_bytes + bb * b_bytes <= budget; };
+  while (b < 4 && fits(a, b + 1)) ++b;
+  if (fits(a + 1, b)) ++a;
+  while (b < 6 && fits(a, b + 1)) ++b;
+  if (a < 4 && fits(a + 1, b)) ++a;
   *sa = a;
   *sb = b;
 }
@@ -327,23 +338,57 @@ cudaError_t launch_variant(const CUtensorMap& fmap, const ShiftParams& q0, const
                            cudaStream_t stream) {
   ShiftParams q = q0;
   int sa, sb;
-  choose_stages<BN>(plan, &sa, &sb);
+  choose_stages<BN>(plan, q.a_stage_bytes, &sa, &sb);
   q.sa = sa;
   q.sb = sb;
-  const int smem_bytes = sa * q.a_stage_bytes + sb * BN * KB * 2 + 1024;
+  const int smem_bytes = sa * q.a_stage_bytes + sb * BN * KB * 2 + (int)plan.K2p * 4 + 1024;
   cudaError_t e = cudaFuncSetAttribute(conv_f16_shift_kernel<BN, ITEMS>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
-  dim3 grid((unsigned)((plan.VQ + TILE_M - 1) / TILE_M), (unsigned)((co + BN - 1) / BN));
+  const int64_t units = (plan.VQ + TILE_M - 1) / TILE_M;
+  dim3 grid((unsigned)(units - q.nbig), (unsigned)((co + BN - 1) / BN));   // a tall tile covers two units
   conv_f16_shift_kernel<BN, ITEMS><<<grid, NUM_THREADS, smem_bytes, stream>>>(fmap, q);
   return cudaGetLastError();
 }
 
+// Number of 256-position tiles: whole waves of tall tiles while two units per slot remain, and
+// in the last round as many tall tiles as it takes for the rest to fit in one wave.
+int choose_nbig(int64_t units, int cotiles, int ctas_per_sm, int kw) {
+  const char* force = getenv("IM2WIN_F16_TALL");     // testing aid: 1 = all tall, 0 = none
+  if (force) return atoi(force) ? (int)(units / 2) : 0;
+  // Tall tiles halve the filter traffic per flop, which is what bounds wide kernels (measured:
+  // +40 % at 11x11, +25 % at 5x5); with three kernel columns the S producers are the bound and
+  // a tall tile only doubles their per-stage latency (measured: -30 % on 3x3 stride 2).
+  if (kw < 5) return 0;
+  int64_t slots = (int64_t)148 * ctas_per_sm / cotiles;
+  if (slots < 1) slots = 1;
+  const int64_t full = units / (2 * slots) * slots;
+  const int64_t rest = units - 2 * full;
+  const int64_t extra = rest > slots ? rest - slots : 0;
+  return (int)(full + extra);
+}
+
 template <int BN>
-cudaError_t launch_bn(const CUtensorMap& fmap, const ShiftParams& q, const ShiftPlan& plan, int co,
-                      cudaStream_t stream) {
-  if (plan.items <= 5) return launch_variant<BN, 5>(fmap, q, plan, co, stream);
-  if (plan.items <= 10) return launch_variant<BN, 10>(fmap, q, plan, co, stream);
+cudaError_t launch_bn(const CUtensorMap& fmap, const ShiftParams& q0, const ShiftPlan& plan, int co,
+                      int s, cudaStream_t stream) {
+  ShiftParams q = q0;
+  const int64_t units = (plan.VQ + TILE_M - 1) / TILE_M;
+  q.nbig = choose_nbig(units, (co + BN - 1) / BN, BN <= 128 ? 2 : 1, q.Kw);
+  const int mt = q.nbig > 0 ? 2 : 1;
+  const int total_rows = s * (TILE_M * mt + q.halo8);
+  q.a_stage_bytes = total_rows * 128;
+  if (2 * q.a_stage_bytes + 2 * BN * KB * 2 + (int)plan.K2p * 4 > (BN <= 128 ? kSmemBudget / 2 : kSmemBudget) - 2048) {
+    q.nbig = 0;                                   // tall tiles do not fit: fall back to 128-row tiles
+    q.a_stage_bytes = s * (TILE_M + q.halo8) * 128;
+  }
+  const int rows_all = q.a_stage_bytes / 128;
+  const int items = (rows_all * 8 + PRODUCER_THREADS - 1) / PRODUCER_THREADS;
+  if (items <= 5) return launch_variant<BN, 5>(fmap, q, plan, co, stream);
+  if (items <= 10) return launch_variant<BN, 10>(fmap, q, plan, co, stream);
+  if (items <= 15) return launch_variant<BN, 15>(fmap, q, plan, co, stream);
+  if (items <= 20) return launch_variant<BN, 20>(fmap, q, plan, co, stream);
+  q.nbig = 0;
+  q.a_stage_bytes = s * (TILE_M + q.halo8) * 128;
   return launch_variant<BN, 15>(fmap, q, plan, co, stream);
 }
 
@@ -362,8 +407,10 @@ ShiftPlan plan_f16_shift(const Geometry& g) {
   p.K2p = (p.K2 + KB - 1) / KB * KB;
   p.VQ = (int64_t)g.N * g.Ho * p.Wq;
   if (p.items > 15) return p;
+  if (p.K2p * 4 > 24 * 1024) return p;                    // offset table lives in shared memory
+  if (g.img_stride >= ((int64_t)1 << 30)) return p;       // 32-bit offsets relative to the tile's first image
   // two stages of each ring must fit even for the widest channel tile
-  if (2 * p.total_rows * 128 + 2 * 256 * KB * 2 > kSmemBudget - 2048) return p;
+  if (2 * p.total_rows * 128 + 2 * 256 * KB * 2 + p.K2p * 4 > kSmemBudget - 2048) return p;
   if ((p.VQ + TILE_M - 1) / TILE_M >= ((int64_t)1 << 31)) return p;
   p.eligible = true;
   return p;
@@ -397,12 +444,13 @@ cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratc
   q.VQ = plan.VQ; q.img_stride = g.img_stride; q.strip = g.strip;
   q.Wq = plan.Wq; q.Ho = g.Ho; q.Wo = g.Wo; q.HoWo = g.Ho * g.Wo; q.Co = g.Co;
   q.Kh = g.Kh; q.Kw = g.Kw; q.s = g.s; q.num_kb = (int32_t)(plan.K2p / KB);
-  q.rows = plan.rows; q.total_rows = plan.total_rows;
-  q.sub_bytes = plan.rows * 128; q.a_stage_bytes = plan.total_rows * 128;
+  q.halo8 = plan.rows - TILE_M;
+  q.nbig = 0;
+  q.a_stage_bytes = plan.total_rows * 128;
   q.sa = q.sb = 2;
-  if (bn == 64) return launch_bn<64>(fmap, q, plan, g.Co, stream);
-  if (bn == 128) return launch_bn<128>(fmap, q, plan, g.Co, stream);
-  return launch_bn<256>(fmap, q, plan, g.Co, stream);
+  if (bn == 64) return launch_bn<64>(fmap, q, plan, g.Co, g.s, stream);
+  if (bn == 128) return launch_bn<128>(fmap, q, plan, g.Co, g.s, stream);
+  return launch_bn<256>(fmap, q, plan, g.Co, g.s, stream);
 }
 
 }  // namespace im2win
