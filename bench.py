@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
-from paper_2608_20725_b200 import workloads  # noqa: E402
+from paper_2608_20725_b200 import replicas, workloads  # noqa: E402
 
 METRIC = "conv TFLOPS (fp32 + fp16 passes of the layer, transform and filter pack included)"
 UNIT = "TFLOP/s"
@@ -334,14 +334,11 @@ def run_gpu_arm(args):
               + e2e_sets[p]["f"].numel() * e2e_sets[p]["f"].element_size() for p in runner.precisions)
     d2h = sum(e2e_sets[p]["y"].numel() * 4 for p in runner.precisions)
 
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = times.tolist()
+    total_ms, e2e_ms = replicas.max_over_ranks([total_ms, e2e_ms], device="cuda")
 
     step_flops = runner.flops * len(runner.precisions)
-    value = world * step_flops * args.steps / (total_ms * 1e-3) / 1e12
-    e2e_value = world * step_flops * e2e_steps / (e2e_ms * 1e-3) / 1e12
+    value = replicas.whole_job_rate(step_flops * args.steps, world, total_ms) / 1e12
+    e2e_value = replicas.whole_job_rate(step_flops * e2e_steps, world, e2e_ms) / 1e12
 
     rooflines = kernel_rooflines(runner, avg_ms, peaks, peak_kind)
     traffic = load_traffic()
