@@ -151,6 +151,38 @@ im2win_status im2win_layer_forward_host(const void* x_host, const void* filter_h
                                         const im2win_shape* shape, im2win_dtype dtype,
                                         void* cuda_stream);
 
+/*
+ * fp32 convolution without a scratch argument, for callers that cannot allocate
+ * device memory (the paper has no counterpart; this is a convenience of this
+ * library).  Think of code running where cudaMalloc is off limits: a real-time
+ * loop with a frozen memory map, a plug-in that receives input and output
+ * buffers but no allocator, a process whose device memory is managed by another
+ * runtime.  Such a caller cannot produce the `scratch` buffer im2win_conv_f32
+ * wants, so the library keeps one itself: a fixed array of
+ * IM2WIN_STATIC_SCRATCH_BYTES that every GPU which loads the library holds until
+ * the process exits.
+ *
+ * Same operation, arguments and results as im2win_conv_f32 (window, filter and
+ * y are the caller's device buffers).  Differences:
+ *   - A layer whose scratch_bytes (im2win_workspace_size, IM2WIN_F32) exceed
+ *     IM2WIN_STATIC_SCRATCH_BYTES is rejected with IM2WIN_ERR_WORKSPACE_TOO_SMALL
+ *     before anything is launched (roughly: Co*C*Kh*Kw above one million filter
+ *     elements does not fit).
+ *   - The call allocates nothing: no cudaMalloc, no cudaFree, no allocating
+ *     library routine.
+ *   - The first call on each device looks up the device address of the array
+ *     (with that device current) and caches it; make that first call outside any
+ *     stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the last
+ *     call left in it.  Each call rewrites every byte it later reads, so
+ *     back-to-back calls on one stream are safe; two calls whose kernels may
+ *     overlap on the GPU (different streams, no ordering between them) race on
+ *     the array and must be serialised by the caller.
+ */
+#define IM2WIN_STATIC_SCRATCH_BYTES (4u << 20)
+im2win_status im2win_conv_f32_static(const float* window, const float* filter_oihw, float* y_nchw,
+                                     const im2win_shape* shape, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

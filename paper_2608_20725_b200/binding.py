@@ -25,7 +25,10 @@ STATUS_NAMES = {
 EXPORTS = (
     "im2win_status_string", "im2win_workspace_size", "im2win_transform", "im2win_conv_f32", "im2win_conv_f16",
     "im2win_check_status", "im2win_layer_workspace_size", "im2win_layer_forward_host",
+    "im2win_conv_f32_static",
 )
+
+STATIC_SCRATCH_BYTES = 4 << 20
 
 
 class Shape(ctypes.Structure):
@@ -60,6 +63,7 @@ def lib() -> ctypes.CDLL:
     L.im2win_check_status.argtypes = [vp, vp]
     L.im2win_layer_workspace_size.argtypes = [P(Shape), ctypes.c_int, P(sz)]
     L.im2win_layer_forward_host.argtypes = [vp, vp, vp, vp, sz, P(Shape), ctypes.c_int, vp]
+    L.im2win_conv_f32_static.argtypes = [vp, vp, vp, P(Shape), vp]
     for name in EXPORTS[1:]:
         getattr(L, name).restype = ctypes.c_int
     _lib = L
@@ -153,6 +157,17 @@ def im2win_conv_f32(window, filter_oihw, y, scratch, shape, stream=None) -> None
 
 def im2win_conv_f16(window, filter_oihw, y, scratch, shape, stream=None) -> None:
     _conv("im2win_conv_f16", torch.float16, F16, window, filter_oihw, y, scratch, shape, stream)
+
+
+def im2win_conv_f32_static(window, filter_oihw, y, shape, stream=None) -> None:
+    """fp32 convolution for callers that cannot allocate device memory: same as im2win_conv_f32
+    but the scratch lives in a fixed array inside the library (layers needing more than
+    STATIC_SCRATCH_BYTES are rejected).  Calls that may overlap on the GPU must be serialised."""
+    s = as_shape(shape)
+    for t in (window, filter_oihw, y):
+        assert t.is_cuda and t.is_contiguous() and t.dtype == torch.float32
+    _check(lib().im2win_conv_f32_static(window.data_ptr(), filter_oihw.data_ptr(), y.data_ptr(),
+                                        ctypes.byref(s), _stream(stream)), "im2win_conv_f32_static")
 
 
 def im2win_check_status(scratch: torch.Tensor, stream=None) -> None:
