@@ -46,7 +46,7 @@ __device__ __forceinline__ float2 unpack2(unsigned long long v) {
 }
 
 template <int BM, int BN>
-__global__ void __launch_bounds__((BM / 8) * (BN / 8))
+__global__ void __launch_bounds__((BM / 8) * (BN / 8), ((BM / 8) * (BN / 8) == 256 ? 2 : 1))
 conv_f32_kernel(ConvF32Params q) {
   constexpr int THREADS = (BM / 8) * (BN / 8);
   constexpr int A_PER_THREAD = BK * BM / THREADS;         // scalar gathers per k-block
@@ -79,14 +79,23 @@ conv_f32_kernel(ConvF32Params q) {
 
   float areg[A_PER_THREAD];
   float4 breg[B_VEC_PER_THREAD];
+  int offreg[A_PER_THREAD];          // offsets of the k-block after the one being loaded
 
-  auto load_global = [&](int kb) {
+  // The offset table is read one k-block ahead of the data it addresses, so that the
+  // dependent window loads never wait for it.
+  auto load_offsets = [&](int kb) {
+    const int k0 = kb * BK;
+#pragma unroll
+    for (int i = 0; i < A_PER_THREAD; ++i) offreg[i] = __ldg(q.koff + k0 + lkk0 + i * A_KK_STEP);
+  };
+  auto load_global = [&](int kb, bool more) {
     const int k0 = kb * BK;
 #pragma unroll
     for (int i = 0; i < A_PER_THREAD; ++i) {
-      const int off = __ldg(q.koff + k0 + lkk0 + i * A_KK_STEP);
+      const int off = offreg[i];
       areg[i] = (lvalid && off >= 0) ? __ldg(abase + off) : 0.f;
     }
+    if (more) load_offsets(kb + 1);
 #pragma unroll
     for (int i = 0; i < B_VEC_PER_THREAD; ++i) {
       const int e = tid + i * THREADS;       // float4 index inside the BK x BN tile
@@ -114,13 +123,14 @@ conv_f32_kernel(ConvF32Params q) {
     for (int jp = 0; jp < 4; ++jp) acc2[i][jp] = 0ull;
 
   const int nkb = q.Kp / BK;
-  load_global(0);
+  load_offsets(0);
+  load_global(0, nkb > 1);
   store_shared(0);
   __syncthreads();
 
   for (int kb = 0; kb < nkb; ++kb) {
     const int buf = kb & 1;
-    if (kb + 1 < nkb) load_global(kb + 1);
+    if (kb + 1 < nkb) load_global(kb + 1, kb + 2 < nkb);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
       const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][kk][tm * 4]);
