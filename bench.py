@@ -406,12 +406,15 @@ def write_report(path, peaks, peak_kind, names=None, iters=10):
     table.update(workloads.TABLE1_LAYERS)
     for name in (names or list(workloads.LAYERS)):
         layer = table[name]
+        print(f"[report] {name}", file=sys.stderr, flush=True)
         runner = LayerRunner(layer, layer.precisions)
         for _ in range(3):
             runner.step()
+        torch.cuda.synchronize()
         avg, best = {}, {}
         for prec in layer.precisions:
             for kind, fn in (("transform", runner.transform), ("conv", runner.conv)):
+                print(f"[report]   {kind}_{prec}", file=sys.stderr, flush=True)
                 avg[f"{kind}_{prec}"], best[f"{kind}_{prec}"] = time_call(lambda: fn(prec), iters, flush)
             binding.im2win_check_status(runner.dev[prec]["scratch"])
         row = {"layer": name, "dims": layer.dims(), "gflop": runner.flops / 1e9, "avg_ms": avg, "best_ms": best,

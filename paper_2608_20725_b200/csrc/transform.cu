@@ -2,6 +2,19 @@
 //
 //   window[n][c][ho][k*Kh + u] = Xpad[n][c][ho*s + u][k]
 //
+// Two kernels.  The strip kernel (default) gives every CTA a run of whole strips
+// (n, c, ho): sub-warps walk the columns of a strip (lanes = consecutive k, so
+// each input row is read as coalesced runs; the Kh rows of a column come from
+// L1/L2 when neighbouring strips re-read them; four items per thread are loaded
+// before the first is stored), pack the Kh (fp32) or 2*Kh (fp16, two columns)
+// elements of an item into 32-bit words and store them into a
+// shared-memory staging buffer laid out exactly like the output range -- same
+// 16-byte phase as the global address.  The 16-byte-aligned body of the range
+// then leaves with ONE bulk asynchronous copy (cp.async.bulk shared -> global)
+// issued by one thread; only the ragged head and tail (< 16 bytes each) are
+// stored by hand.  The column kernel below serves kernel heights other than
+// 1, 3, 5 and strips too long to stage.
+//
 // The window tensor is one flat array of "columns": column g = (strip, k) with
 // strip = (n*C + c)*Ho + ho holds the Kh elements {u = 0..Kh-1} at flat offset
 // g*Kh.  A CTA owns a contiguous range of columns, hence a contiguous range of
@@ -11,6 +24,9 @@
 // HBM with 16-byte stores.  The kernel is HBM-bound: the input is read once
 // from DRAM (re-reads by overlapping strips hit L1/L2) and the window tensor
 // is written once.
+#include <stdlib.h>
+#include <string.h>
+
 #include "common.cuh"
 
 namespace im2win {
@@ -95,6 +111,173 @@ transform_kernel(const E* __restrict__ x, E* __restrict__ win, TransformParams q
   for (int e = tail0 + threadIdx.x; e < nelem; e += step) oe[e] = stage[e];
 }
 
+
+// ------------------------------------------------------------------ strip kernel
+struct StripParams {
+  int32_t H, W, Wp, Kh, s, p, Ho;
+  int32_t L;                 // Kh*Wp elements per strip
+  int32_t strips_per_cta;
+  int32_t group;             // threads that walk one strip together: a power of two <= 256
+  int64_t total_strips;      // N*C*Ho
+};
+
+constexpr int kStripThreads = 256;
+constexpr int kStripUnroll = 4;      // items per thread whose loads are issued before the first store
+
+template <typename E, int KH>
+__global__ void __launch_bounds__(kStripThreads)
+transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParams q) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  constexpr int ES = (int)sizeof(E);
+  constexpr int CPL = 4 / ES;                     // columns per item: one 32-bit word per kernel row
+  constexpr int U = kStripUnroll;
+
+  const int64_t s0 = (int64_t)blockIdx.x * q.strips_per_cta;
+  const int64_t left = q.total_strips - s0;
+  const int ns = left < q.strips_per_cta ? (int)left : q.strips_per_cta;
+  const int64_t out_byte0 = s0 * q.L * ES;        // first output byte of this CTA
+  const int mis = (int)(out_byte0 & 15);          // staging mirrors the 16-byte phase of the output
+  unsigned char* stage = smem_raw + mis;
+
+  // A group of G threads walks one strip, U items per thread and pass; 256/G strips are in
+  // flight per pass.  Strip index -> (plane, ho) by one 32-bit division relative to the CTA's first strip.
+  const int G = q.group;
+  const int grp = threadIdx.x / G, gl = threadIdx.x - grp * G;
+  const int ngrp = kStripThreads / G;
+  const int64_t plane0 = s0 / q.Ho;
+  const int ho0 = (int)(s0 - plane0 * q.Ho);
+  const int64_t plane_elems = (int64_t)q.H * q.W;
+
+  for (int ls = grp; ls < ns; ls += ngrp) {
+    const int t = ho0 + ls;
+    const int dpl = t / q.Ho;
+    const int ho = t - dpl * q.Ho;
+    const int h0 = ho * q.s - q.p;
+    const E* __restrict__ src = x + (plane0 + dpl) * plane_elems;
+    const int sbyte = ls * q.L * ES;              // byte offset of the strip inside the staging
+    unsigned char* dst_strip = stage + sbyte;
+    const bool word_ok = ((mis + sbyte) & 3) == 0;
+    for (int kbase = gl * CPL; kbase < q.Wp; kbase += G * CPL * U) {
+      E v[U][CPL][KH];
+#pragma unroll
+      for (int j = 0; j < U; ++j) {
+        const int k = kbase + j * G * CPL;
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) {
+          const int w = k + c - q.p;
+          const bool w_ok = (unsigned)w < (unsigned)q.W;     // also false beyond the strip
+#pragma unroll
+          for (int u = 0; u < KH; ++u) {
+            const int h = h0 + u;
+            v[j][c][u] = 0;
+            if (w_ok && (unsigned)h < (unsigned)q.H) v[j][c][u] = __ldg(src + h * q.W + w);
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < U; ++j) {
+        const int k = kbase + j * G * CPL;
+        if (k >= q.Wp) break;
+        unsigned char* d = dst_strip + (size_t)k * KH * ES;
+        if constexpr (ES == 4) {
+#pragma unroll
+          for (int u = 0; u < KH; ++u) reinterpret_cast<uint32_t*>(d)[u] = (uint32_t)v[j][0][u];
+        } else {
+          if (word_ok && k + 1 < q.Wp) {
+#pragma unroll
+            for (int jj = 0; jj < KH; ++jj) {        // word jj holds elements 2jj, 2jj+1 of the 2*KH run
+              const int e0 = 2 * jj, e1 = 2 * jj + 1;
+              const uint32_t lo = (uint32_t)(e0 < KH ? v[j][0][e0] : v[j][1][e0 - KH]);
+              const uint32_t hi = (uint32_t)(e1 < KH ? v[j][0][e1] : v[j][1][e1 - KH]);
+              reinterpret_cast<uint32_t*>(d)[jj] = lo | (hi << 16);
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < CPL; ++c)
+              if (k + c < q.Wp) {
+#pragma unroll
+                for (int u = 0; u < KH; ++u) reinterpret_cast<E*>(d)[c * KH + u] = v[j][c][u];
+              }
+          }
+        }
+      }
+    }
+  }
+  // Make the generic-proxy writes visible to the bulk-copy engine, then meet.
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+
+  // The 16-byte-aligned body leaves with one bulk copy.
+  const int total = ns * q.L * ES;
+  int head = (16 - mis) & 15;
+  if (head > total) head = total;
+  const int body = (total - head) & ~15;
+  const int tail = total - head - body;
+  unsigned char* gout = reinterpret_cast<unsigned char*>(win) + out_byte0;
+  if (threadIdx.x == 0 && body > 0) {
+    const uint32_t saddr = (uint32_t)__cvta_generic_to_shared(stage + head);
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gout + head), "r"(saddr),
+                 "r"(body)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  }
+  // ragged ends, element by element (never more than 15 bytes each)
+  if ((int)threadIdx.x * ES < head)
+    reinterpret_cast<E*>(gout)[threadIdx.x] = reinterpret_cast<const E*>(stage)[threadIdx.x];
+  if ((int)threadIdx.x * ES < tail) {
+    const int o = head + body;
+    reinterpret_cast<E*>(gout + o)[threadIdx.x] = reinterpret_cast<const E*>(stage + o)[threadIdx.x];
+  }
+  // the staging buffer must outlive the bulk copy's reads
+  if (threadIdx.x == 0 && body > 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+
+// The strip kernel is used for the kernel heights it is instantiated for, when a strip can be
+// staged; measured faster than the column kernel for Kh <= 5 and slower beyond (register
+// pressure of the unrolled gathers), so taller kernels keep the column kernel.
+template <typename E>
+bool plan_strips(const Geometry& g, StripParams* q, size_t* smem_bytes) {
+  constexpr int ES = (int)sizeof(E);
+  if (!(g.Kh == 1 || g.Kh == 3 || g.Kh == 5)) return false;
+  const int64_t strip_bytes = g.strip * ES;
+  const int64_t total_strips = (int64_t)g.N * g.C * g.Ho;
+  if (strip_bytes > 64 * 1024 || total_strips >= ((int64_t)1 << 31)) return false;
+  int r = (int)(16384 / strip_bytes);
+  if (r < 1) r = 1;
+  q->H = g.H; q->W = g.W; q->Wp = g.Wp; q->Kh = g.Kh; q->s = g.s; q->p = g.p; q->Ho = g.Ho;
+  q->L = (int32_t)g.strip;
+  q->total_strips = total_strips;
+  q->strips_per_cta = r;
+  const int items = (g.Wp + (4 / ES) - 1) / (4 / ES);
+  const int per_group = (items + kStripUnroll - 1) / kStripUnroll;
+  int grp = 1;
+  while (grp < kStripThreads && grp < per_group) grp *= 2;
+  q->group = grp;
+  *smem_bytes = (size_t)(r * strip_bytes + 16);
+  return true;
+}
+
+template <typename E>
+cudaError_t launch_strips(const void* x, void* window, const StripParams& q, size_t smem, int Kh,
+                          cudaStream_t stream) {
+  const int64_t blocks = (q.total_strips + q.strips_per_cta - 1) / q.strips_per_cta;
+  const E* xi = static_cast<const E*>(x);
+  E* wo = static_cast<E*>(window);
+  auto run = [&](auto kernel) -> cudaError_t {
+    if (smem > 48 * 1024) {
+      cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
+    kernel<<<(unsigned)blocks, kStripThreads, smem, stream>>>(xi, wo, q);
+    return cudaGetLastError();
+  };
+  switch (Kh) {
+    case 1: return run(transform_strips_kernel<E, 1>);
+    case 3: return run(transform_strips_kernel<E, 3>);
+    default: return run(transform_strips_kernel<E, 5>);
+  }
+}
+
 template <typename E>
 cudaError_t launch_typed(const void* x, void* window, const Geometry& g, cudaStream_t stream) {
   TransformParams q;
@@ -131,7 +314,17 @@ cudaError_t launch_typed(const void* x, void* window, const Geometry& g, cudaStr
 
 cudaError_t launch_transform(const void* x, void* window, const Geometry& g, int elem_bytes,
                              cudaStream_t stream) {
-  if (elem_bytes == 4) return launch_typed<uint32_t>(x, window, g, stream);
+  // Strips that fit a staging buffer go to the strip kernel; IM2WIN_TRANSFORM_KERNEL=columns
+  // forces the fallback (a testing aid).
+  const char* force = getenv("IM2WIN_TRANSFORM_KERNEL");
+  const bool columns = force && strcmp(force, "columns") == 0;
+  StripParams q;
+  size_t smem = 0;
+  if (elem_bytes == 4) {
+    if (!columns && plan_strips<uint32_t>(g, &q, &smem)) return launch_strips<uint32_t>(x, window, q, smem, g.Kh, stream);
+    return launch_typed<uint32_t>(x, window, g, stream);
+  }
+  if (!columns && plan_strips<uint16_t>(g, &q, &smem)) return launch_strips<uint16_t>(x, window, q, smem, g.Kh, stream);
   return launch_typed<uint16_t>(x, window, g, stream);
 }
 

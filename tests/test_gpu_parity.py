@@ -43,7 +43,12 @@ SMALL = [
 
 @pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
 @pytest.mark.parametrize("es", [4, 2])
-def test_transform_bit_exact_small(layer, es):
+@pytest.mark.parametrize("kernel", ["strips", "columns"])
+def test_transform_bit_exact_small(layer, es, kernel, monkeypatch):
+    """Both transform kernels (the strip kernel the library picks, and the column kernel it
+    falls back to for very long strips) against the oracle, bit for bit."""
+    if kernel == "columns":
+        monkeypatch.setenv("IM2WIN_TRANSFORM_KERNEL", "columns")
     dims = layer.dims()
     x, _ = workloads.make_inputs(layer)
     xb = x if es == 4 else x.half()
@@ -51,6 +56,15 @@ def test_transform_bit_exact_small(layer, es):
     got = gpu_transform(raw, dims)
     want = oracle.transform(raw.numpy(), dims)
     assert got.shape == want.shape and np.array_equal(got, want)
+
+
+def test_transform_long_strips_use_the_column_kernel():
+    """A strip longer than the staging limit (Kh*Wp*4 bytes > 96 KB) takes the fallback path."""
+    layer = L("long", 1, 2, 5, 9000, 1, 3, 3, 1, 1, 33)
+    dims = layer.dims()
+    x, _ = workloads.make_inputs(layer)
+    raw = x.view(torch.int32)
+    assert np.array_equal(gpu_transform(raw, dims), oracle.transform(raw.numpy(), dims))
 
 
 def test_transform_preserves_special_bit_patterns():
