@@ -56,17 +56,41 @@ struct ShiftParams {
   const int32_t* __restrict__ koff2;   // k2 -> c*chan_stride + u, -1 for padded k2
   float* __restrict__ y;
   uint32_t* status;
-  int64_t VQ, img_stride, strip;
+  int64_t VQ, img_stride, strip, chan_stride, window_elems;
+  int32_t C, N;
   int32_t Wq, Ho, Wo, HoWo, Co, Kh, Kw, s, num_kb;
   int32_t halo8;          // halo rows of a sub-tile, rounded up to 8
   int32_t nbig;           // the first nbig tiles are 256 positions tall (two MMA halves), the rest 128
   int32_t a_stage_bytes, sa, sb;
 };
 
+#ifdef IM2WIN_F16_TIMERS
+// Debug build only: per-thread cycle counters, flushed once into the 64-bit words 4.. of the status block.
+#define TIMER_DECL long long t_prev = clock64(), t_now, t_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
+#define TIMER_LAP(slot)                 \
+  do {                                  \
+    t_now = clock64();                  \
+    t_acc[slot] += t_now - t_prev;      \
+    t_prev = t_now;                     \
+  } while (0)
+#define TIMER_FLUSH()                                                                                              \
+  do {                                                                                                             \
+    for (int ti = 0; ti < 12; ++ti)                                                                                \
+      if (t_acc[ti]) atomicAdd(reinterpret_cast<unsigned long long*>(q.status) + 4 + ti, (unsigned long long)t_acc[ti]); \
+  } while (0)
+#else
+#define TIMER_DECL
+#define TIMER_LAP(slot)
+#define TIMER_FLUSH()
+#endif
+
 template <int BN, int ITEMS>
 __global__ void __launch_bounds__(NUM_THREADS, (BN <= 128 ? 2 : 1))
 conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
   constexpr int B_STAGE_BYTES = BN * KB * 2;
+  // Register double-buffering of the producers' loads needs ~40 more registers per thread:
+  // affordable with one CTA per SM (256-channel tiles), not with two.
+  constexpr bool PREFETCH = BN > 128;
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
@@ -153,51 +177,94 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
     }
 
     bool ok = true;
-    for (int kb = 0; kb < q.num_kb; ++kb) {
-      const int st = kb % q.sa;
-      const uint32_t round = (uint32_t)(kb / q.sa);
-      if (lane == 0) ok = mbar_wait(a_empty0 + 8 * st, (round & 1u) ^ 1u, &abort_flag, q.status);
-      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-      if (!ok) break;
-      const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
+    TIMER_DECL;
+    if (threadIdx.x == 0) TIMER_LAP(0);   // setup
+    // The stage is produced in units of ITEM_GROUP items.  With PREFETCH the loads of the next
+    // unit are issued before the current one is packed and stored, so that one DRAM/L2 round
+    // trip overlaps the pack/store/handshake of the previous unit.  Dead rows and padded k2 read
+    // a word of the status block that is always zero, so nothing needs masking afterwards.
+    constexpr int G = ITEM_GROUP;
+    constexpr int NG = ITEMS / G;
+    const uint16_t* __restrict__ zero16 = reinterpret_cast<const uint16_t*>(q.status + 2);
+    auto issue = [&](int kb, int gidx, uint32_t (&h)[G][8]) {
       const int4* kt = reinterpret_cast<const int4*>(koff_s + kb * KB);   // this k-block's offsets (shared memory)
 #pragma unroll
-      for (int g0 = 0; g0 < ITEMS; g0 += ITEM_GROUP) {
-        constexpr int G = ITEM_GROUP;
-        uint32_t h[G][8];
+      for (int gi = 0; gi < G; ++gi) {
+        const int it = gidx * G + gi;
+        const int ch = (int)(meta[it] & 7u);
+        const int4 o0 = kt[ch * 2], o1 = kt[ch * 2 + 1];
+        const int32_t off[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
+        const uint16_t* src = tile_win + rel[it];
+        const bool row_ok = (meta[it] & 8u) != 0;
 #pragma unroll
-        for (int gi = 0; gi < G; ++gi) {
-          const int it = g0 + gi;
-          const int ch = (int)(meta[it] & 7u);
-          const int4 o0 = kt[ch * 2], o1 = kt[ch * 2 + 1];
-          const int32_t off[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
-          const uint16_t* src = tile_win + rel[it];
+        for (int e = 0; e < 8; ++e) h[gi][e] = (uint32_t)__ldg((row_ok && off[e] >= 0) ? src + off[e] : zero16);
+      }
+    };
+    auto store = [&](uint32_t a_stage, int gidx, const uint32_t (&h)[G][8]) {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) h[gi][e] = (uint32_t)__ldg(src + max(off[e], 0));
-          const bool row_ok = (meta[it] & 8u) != 0;
-#pragma unroll
-          for (int e = 0; e < 8; ++e) h[gi][e] = (row_ok && off[e] >= 0) ? h[gi][e] : 0u;
-        }
-#pragma unroll
-        for (int gi = 0; gi < G; ++gi) {
-          const int it = g0 + gi;
-          if (meta[it] != 0xffffffffu) {
-            const uint32_t w0 = h[gi][0] | (h[gi][1] << 16), w1 = h[gi][2] | (h[gi][3] << 16);
-            const uint32_t w2 = h[gi][4] | (h[gi][5] << 16), w3 = h[gi][6] | (h[gi][7] << 16);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_stage + (meta[it] & ~15u)), "r"(w0),
-                         "r"(w1), "r"(w2), "r"(w3)
-                         : "memory");
-          }
+      for (int gi = 0; gi < G; ++gi) {
+        const int it = gidx * G + gi;
+        if (meta[it] != 0xffffffffu) {
+          const uint32_t w0 = h[gi][0] | (h[gi][1] << 16), w1 = h[gi][2] | (h[gi][3] << 16);
+          const uint32_t w2 = h[gi][4] | (h[gi][5] << 16), w3 = h[gi][6] | (h[gi][7] << 16);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_stage + (meta[it] & ~15u)), "r"(w0),
+                       "r"(w1), "r"(w2), "r"(w3)
+                       : "memory");
         }
       }
+    };
+
+    int st = 0;                 // ring slot and its phase bit, advanced without divisions
+    uint32_t ph = 0;
+    uint32_t bufA[G][8], bufB[G][8];
+    // One k-block: unit gidx lives in `first` when gidx is even, in `second` when odd; the loads
+    // of the following unit go to the other buffer (no register copies, so nothing waits for
+    // loads before they are needed).
+    auto do_stage = [&](int kb, uint32_t (&first)[G][8], uint32_t (&second)[G][8]) {
+      const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
+#pragma unroll
+      for (int gidx = 0; gidx < NG; ++gidx) {
+        uint32_t (&cur)[G][8] = (gidx & 1) ? second : first;
+        uint32_t (&nxt)[G][8] = (gidx & 1) ? first : second;
+        if (PREFETCH) {
+          if (gidx + 1 < NG) issue(kb, gidx + 1, nxt);
+          else if (kb + 1 < q.num_kb) issue(kb + 1, 0, nxt);
+        } else {
+          issue(kb, gidx, cur);
+        }
+        if (gidx == 0) {
+          if (threadIdx.x == 0) TIMER_LAP(2);   // issuing loads
+          if (lane == 0) ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+          ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+          if (threadIdx.x == 0) TIMER_LAP(1);   // wait for a free stage
+        }
+        if (ok) store(a_stage, gidx, cur);
+      }
+      if (!ok) return;
+      if (threadIdx.x == 0) TIMER_LAP(3);   // waiting for the loads, pack + store
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(a_full0 + 8 * st);
+      if (threadIdx.x == 0) TIMER_LAP(4);   // fence + arrive
+      if (++st == q.sa) {
+        st = 0;
+        ph ^= 1u;
+      }
+    };
+    if (PREFETCH) issue(0, 0, bufA);
+    for (int kb = 0; kb < q.num_kb && ok; kb += 2) {
+      do_stage(kb, bufA, bufB);
+      if (kb + 1 < q.num_kb && ok) {
+        // with an odd number of units per k-block the roles of the buffers swap every k-block
+        if (NG & 1) do_stage(kb + 1, bufB, bufA);
+        else do_stage(kb + 1, bufA, bufB);
+      }
     }
 
     // ---------------- epilogue --------------------------------------------------
     if (ok && lane == 0) ok = mbar_wait(acc_bar, 0u, &abort_flag, q.status);
     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+    if (threadIdx.x == 0) TIMER_LAP(5);     // wait for the accumulator
     if (ok) {
       tc_fence_after();
       const int lq = warp & 3;                 // tensor-memory lane quadrant this warp may read
@@ -230,55 +297,132 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
         }
       }
     }
+    if (threadIdx.x == 0) { TIMER_LAP(6); TIMER_FLUSH(); }     // epilogue
   } else if (warp == PRODUCER_WARPS) {
     // ---------------- TMA producer of the filter tiles -------------------------
-    if (lane == 0) {
-      int g = 0;
-      for (int kb = 0; kb < q.num_kb; ++kb) {
-        for (int v = 0; v < q.Kw; ++v, ++g) {
-          const int st = g % q.sb;
-          const uint32_t round = (uint32_t)(g / q.sb);
-          if (!mbar_wait(b_empty0 + 8 * st, (round & 1u) ^ 1u, &abort_flag, q.status)) goto tma_done;
-          const uint32_t bar = b_full0 + 8 * st;
+    // The whole warp walks the loop (warp-uniform values can stay in uniform registers, which
+    // the TMA and MMA instructions take their operands from); one elected lane issues.
+    const bool leader = elect_one();
+    bool ok = true;
+    int st = 0;
+    uint32_t ph = 0;
+    // L2 prefetch of the window data the producers will gather a few k-blocks later: lane l asks
+    // for the contiguous run of channel (first channel of the k-block + l), one bulk prefetch per
+    // image the tile touches.  It turns the producers' DRAM round trips into L2 hits.
+    constexpr int PREFETCH_AHEAD = 3;
+    const int64_t img_rows_t = (int64_t)q.Ho * q.Wq;
+    const int64_t n_first_t = q0 / img_rows_t;
+    const int64_t a_first = q0 - n_first_t * img_rows_t;       // first virtual row inside its image
+    const int64_t win_bytes16 = (q.window_elems * 2) & ~(int64_t)15;
+    auto prefetch_block = [&](int kbp) {
+      const int c = (kbp * KB) / q.Kh + lane;
+      const int c_hi = (kbp * KB + KB - 1) / q.Kh;
+      if (c > c_hi || c >= q.C) return;
+      int64_t n = n_first_t, a = a_first;
+      int remaining = rows;
+      for (int seg = 0; seg < 8 && remaining > 0 && n < q.N; ++seg) {
+        const int64_t cnt = remaining < img_rows_t - a ? remaining : img_rows_t - a;
+        const int64_t byte0 = (n * q.img_stride + (int64_t)c * q.chan_stride + a * q.s * q.Kh) * 2;
+        const int64_t beg = byte0 & ~(int64_t)15;
+        int64_t end = (byte0 + cnt * q.s * q.Kh * 2 + 15) & ~(int64_t)15;
+        if (end > win_bytes16) end = win_bytes16;
+        if (end > beg)
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const char*>(q.win) + beg),
+                       "r"((uint32_t)(end - beg))
+                       : "memory");
+        remaining -= (int)cnt;
+        a = 0;
+        ++n;
+      }
+    };
+    for (int kbp = 1; kbp < PREFETCH_AHEAD && kbp < q.num_kb; ++kbp) prefetch_block(kbp);
+    for (int kb = 0; kb < q.num_kb && ok; ++kb) {
+      if (kb + PREFETCH_AHEAD < q.num_kb) prefetch_block(kb + PREFETCH_AHEAD);
+      __syncwarp();
+      for (int v = 0; v < q.Kw; ++v) {
+        ok = mbar_wait(b_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint32_t bar = b_full0 + 8 * st;
+        if (leader) {
           mbar_arrive_expect_tx(bar, B_STAGE_BYTES);
           tma_load_3d(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0, v, bar);
         }
+        __syncwarp();
+        if (++st == q.sb) {
+          st = 0;
+          ph ^= 1u;
+        }
       }
-    tma_done:;
     }
   } else {
     // ---------------- MMA issuer ------------------------------------------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc_f16(TILE_M, BN);
-      bool ok = true;
-      int g = 0;
-      for (int kb = 0; kb < q.num_kb && ok; ++kb) {
-        const int sta = kb % q.sa;
-        ok = mbar_wait(a_full0 + 8 * sta, (uint32_t)(kb / q.sa) & 1u, &abort_flag, q.status);
+    constexpr uint32_t idesc = instr_desc_f16(TILE_M, BN);
+    const bool leader = elect_one();
+    bool ok = true;
+    int sta = 0, stb = 0;                 // ring slots and phase bits, advanced without divisions
+    uint32_t pha = 0, phb = 0, first = 0;
+    // Descriptor low words (16-byte units) of the ring bases; kernel column v reads sub-tile
+    // v mod s shifted down v div s rows (128 bytes each).
+    const uint32_t a_lo0 = smem_desc_lo(a_ring), b_lo0 = smem_desc_lo(b_ring);
+    const uint32_t sub_lo = (uint32_t)sub_bytes >> 4;
+    TIMER_DECL;
+    for (int kb = 0; kb < q.num_kb && ok; ++kb) {
+      TIMER_LAP(8);
+      ok = mbar_wait(a_full0 + 8 * sta, pha, &abort_flag, q.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      TIMER_LAP(9);                         // MMA warp: wait for an S stage
+      const uint32_t a_lo_stage = a_lo0 + (uint32_t)(sta * (q.a_stage_bytes >> 4));
+      uint32_t a_view = 0;                  // offset of kernel column v's view inside the stage
+      int sub = 0;
+      for (int v = 0; v < q.Kw; ++v) {
+        TIMER_LAP(8);
+        ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
+        ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        const uint32_t a_stage = a_ring + sta * q.a_stage_bytes;
-        for (int v = 0; v < q.Kw; ++v, ++g) {
-          const int stb = g % q.sb;
-          ok = mbar_wait(b_full0 + 8 * stb, (uint32_t)(g / q.sb) & 1u, &abort_flag, q.status);
-          if (!ok) break;
-          tc_fence_after();
-          const int sub = v % q.s;
-          const int shift = v / q.s;
-          const uint32_t b_addr = b_ring + stb * B_STAGE_BYTES;
+        TIMER_LAP(10);                      // MMA warp: wait for a filter stage
+        tc_fence_after();
+        const uint32_t b_lo = b_lo0 + (uint32_t)(stb * (B_STAGE_BYTES >> 4));
+        uint32_t a_lo = a_lo_stage + a_view;
+        // next kernel column: next sub-tile, or back to sub-tile 0 one row (128 bytes) further down
+        if (++sub == q.s) {
+          sub = 0;
+          a_view += 8u - (uint32_t)(q.s - 1) * sub_lo;
+        } else {
+          a_view += sub_lo;
+        }
+        if (leader) {
+          uint32_t acc_col = tmem_acc;
           for (int half = 0; half < mt; ++half) {
-            const uint32_t a_addr = a_stage + sub * sub_bytes + (half * TILE_M + shift) * 128;
 #pragma unroll
-            for (int j = 0; j < KB / 16; ++j) {
-              const uint64_t ad = smem_desc_k_major_sw128(a_addr + j * 32);
-              const uint64_t bd = smem_desc_k_major_sw128(b_addr + j * 32);
-              umma_f16(tmem_acc + (uint32_t)(half * BN), ad, bd, idesc, (g > 0 || j > 0) ? 1u : 0u);
-            }
+            for (int j = 0; j < KB / 16; ++j)
+              umma_f16_lohi(acc_col, a_lo + 2 * j, b_lo + 2 * j, idesc, first | (uint32_t)j);
+            a_lo += (uint32_t)(TILE_M * 128) >> 4;
+            acc_col += (uint32_t)BN;
           }
           umma_commit(b_empty0 + 8 * stb);
         }
-        if (ok) umma_commit(a_empty0 + 8 * sta);
+        __syncwarp();
+        TIMER_LAP(11);                      // MMA warp: issue + commit
+        first = 1u;                         // every later MMA accumulates
+        if (++stb == q.sb) {
+          stb = 0;
+          phb ^= 1u;
+        }
       }
-      if (ok) umma_commit(acc_bar);
+      if (ok && leader) umma_commit(a_empty0 + 8 * sta);
+      __syncwarp();
+      if (++sta == q.sa) {
+        sta = 0;
+        pha ^= 1u;
+      }
+    }
+    if (ok && leader) umma_commit(acc_bar);
+    __syncwarp();
+    if (leader) {
+      TIMER_LAP(8);
+      TIMER_FLUSH();
     }
   }
 
@@ -442,6 +586,7 @@ cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratc
   q.y = y;
   q.status = reinterpret_cast<uint32_t*>(base);
   q.VQ = plan.VQ; q.img_stride = g.img_stride; q.strip = g.strip;
+  q.chan_stride = g.chan_stride; q.window_elems = g.window_elems; q.C = g.C; q.N = g.N;
   q.Wq = plan.Wq; q.Ho = g.Ho; q.Wo = g.Wo; q.HoWo = g.Ho * g.Wo; q.Co = g.Co;
   q.Kh = g.Kh; q.Kw = g.Kw; q.s = g.s; q.num_kb = (int32_t)(plan.K2p / KB);
   q.halo8 = plan.rows - TILE_M;

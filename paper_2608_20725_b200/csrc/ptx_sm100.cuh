@@ -47,6 +47,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   atomicExch(status, 1u);
   return false;
 }
+// True in exactly one lane of the (converged) warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -119,6 +129,25 @@ __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                     // 128-byte swizzle
   return d;
 }
+// The same descriptor split into its two 32-bit halves: the high half is the same for every
+// k-major 128-byte-swizzled tile, and moving a view by 16 bytes adds 1 to the low half, so an
+// MMA issue loop only does 32-bit adds.
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr) {
+  return ((saddr & 0x3ffffu) >> 4) | (1u << 16);
+}
+constexpr uint32_t kSmemDescHiSw128 = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ void umma_f16_lohi(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                              uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %5};\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kSmemDescHiSw128)
+      : "memory");
+}
+
 // Instruction descriptor: fp16 A and B, both k-major, fp32 accumulator, M x N tile.
 __host__ __device__ constexpr uint32_t instr_desc_f16(int M, int N) {
   return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
