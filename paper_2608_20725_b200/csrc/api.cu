@@ -60,6 +60,7 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
     return IM2WIN_ERR_INVALID_ARG;
   }
   l->f16_shift = false;
+  l->f16_raw = false;
   l->koff_off = kStatusBytes;
   l->filter_off = (size_t)round_up((int64_t)l->koff_off + 4 * l->Kp, 256);
   int64_t fbytes = l->Kp * l->Co_pad * (dtype == IM2WIN_F32 ? 4 : 2);
@@ -77,6 +78,8 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
         l->f16_shift = true;
         l->Kp = plan.K2p;
         l->filter_off = shift_filter_off;
+        // the bulk-copy variant shares the filter layout; IM2WIN_F16_KERNEL=shift keeps the gathering one
+        l->f16_raw = plan_f16_raw(g).eligible && !(force && strcmp(force, "shift") == 0);
       }
       if (shift_total > l->total) l->total = shift_total;
     }
@@ -106,7 +109,11 @@ static im2win_status conv_common(const void* window, const void* filter, float* 
     if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
     e = launch_conv_f32(static_cast<const float*>(window), y, scratch, g, l, stream);
   } else {
-    if (l.f16_shift) {
+    if (l.f16_raw) {
+      e = launch_pack_f16_raw(static_cast<const uint16_t*>(filter), scratch, g, l, plan_f16_raw(g), stream);
+      if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
+      e = launch_conv_f16_raw(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
+    } else if (l.f16_shift) {
       e = launch_pack_f16_shift(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
       if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
       e = launch_conv_f16_shift(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);

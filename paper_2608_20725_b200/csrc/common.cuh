@@ -34,7 +34,8 @@ struct ScratchLayout {
   int64_t Kp;            // reduction length rounded up to the k-block of the kernel
   int64_t Co_pad;        // Co rounded up to the filter tile of the kernel
   size_t koff_off, filter_off, total;
-  bool f16_shift;        // fp16 only: the shifted-view kernel (and its filter layout) is used
+  bool f16_shift;        // fp16 only: a shifted-view kernel (and its filter layout) is used
+  bool f16_raw;          // fp16 only: the bulk-copy variant of the shifted-view kernel is used
 };
 
 // Tile geometry of the fp16 shifted-view kernel for one layer (see conv_f16_shift.cu).
@@ -48,6 +49,15 @@ struct ShiftPlan {
   int64_t VQ;            // N*Ho*Wq virtual positions
 };
 ShiftPlan plan_f16_shift(const Geometry& g);
+
+// Tile geometry of the bulk-copy shifted-view kernel (see conv_f16_raw.cu).
+struct RawPlan {
+  bool eligible;
+  int32_t Wq, rows;
+  int32_t nslot, pitch, raw_stage_bytes, a_stage_bytes;
+  int64_t K2, K2p, VQ;
+};
+RawPlan plan_f16_raw(const Geometry& g);
 
 constexpr int kStatusBytes = 256;
 constexpr int kF32KBlock = 16;     // k-block of the fp32 kernel
@@ -67,6 +77,10 @@ cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, 
                             const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_pack_f16_shift(const uint16_t* filter, void* scratch, const Geometry& g,
                                   const ScratchLayout& l, cudaStream_t stream);
+cudaError_t launch_pack_f16_raw(const uint16_t* filter, void* scratch, const Geometry& g,
+                                const ScratchLayout& l, const RawPlan& plan, cudaStream_t stream);
+cudaError_t launch_conv_f16_raw(const uint16_t* window, float* y, void* scratch, const Geometry& g,
+                                const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_conv_f16_gather(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                    const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratch, const Geometry& g,

@@ -64,25 +64,6 @@ struct ShiftParams {
   int32_t a_stage_bytes, sa, sb;
 };
 
-#ifdef IM2WIN_F16_TIMERS
-// Debug build only: per-thread cycle counters, flushed once into the 64-bit words 4.. of the status block.
-#define TIMER_DECL long long t_prev = clock64(), t_now, t_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
-#define TIMER_LAP(slot)                 \
-  do {                                  \
-    t_now = clock64();                  \
-    t_acc[slot] += t_now - t_prev;      \
-    t_prev = t_now;                     \
-  } while (0)
-#define TIMER_FLUSH()                                                                                              \
-  do {                                                                                                             \
-    for (int ti = 0; ti < 12; ++ti)                                                                                \
-      if (t_acc[ti]) atomicAdd(reinterpret_cast<unsigned long long*>(q.status) + 4 + ti, (unsigned long long)t_acc[ti]); \
-  } while (0)
-#else
-#define TIMER_DECL
-#define TIMER_LAP(slot)
-#define TIMER_FLUSH()
-#endif
 
 template <int BN, int ITEMS>
 __global__ void __launch_bounds__(NUM_THREADS, (BN <= 128 ? 2 : 1))

@@ -106,6 +106,25 @@ __global__ void pack_f16_shift_kernel(const uint16_t* __restrict__ f, uint16_t* 
   }
 }
 
+// Table of the bulk-copy fp16 kernel: k2 -> byte offset of element (c, u) inside a raw stage,
+// slot (c - first channel of the k-block) * pitch + u*2, with (c * cs16) & 15 in bits 20..23
+// (how far the 16-byte phase of channel c's run is from channel 0's); padded k2 point at the
+// all-zero slot `nslot`.
+__global__ void rawtab_kernel(uint32_t* __restrict__ tab, int64_t K2, int64_t K2p, int Kh, int pitch, int nslot,
+                              int cs16) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t k2 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k2 < K2p; k2 += stride) {
+    uint32_t e = (uint32_t)(nslot * pitch);
+    if (k2 < K2) {
+      const int64_t c = k2 / Kh;
+      const int u = (int)(k2 - c * Kh);
+      const int64_t c_lo = (k2 / kF16KBlock) * kF16KBlock / Kh;
+      e = (uint32_t)((c - c_lo) * pitch + u * 2) | ((uint32_t)((c * cs16) & 15) << 20);
+    }
+    tab[k2] = e;
+  }
+}
+
 PackParams make_params(const Geometry& g, const ScratchLayout& l) {
   PackParams q;
   q.C = g.C; q.Co = g.Co; q.Kh = g.Kh; q.Kw = g.Kw; q.T = g.T;
@@ -149,6 +168,18 @@ cudaError_t launch_pack_f16_shift(const uint16_t* filter, void* scratch, const G
   pack_f16_shift_kernel<<<grid_for(q.Kp * q.Co * q.Kw), 256, 0, stream>>>(
       filter, reinterpret_cast<uint16_t*>(base + l.filter_off),
       reinterpret_cast<int32_t*>(base + l.koff_off), reinterpret_cast<uint32_t*>(base), q);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pack_f16_raw(const uint16_t* filter, void* scratch, const Geometry& g,
+                                const ScratchLayout& l, const RawPlan& plan, cudaStream_t stream) {
+  // same filter layout as the shifted-view kernel; its offset table is then replaced by the raw table
+  cudaError_t e = launch_pack_f16_shift(filter, scratch, g, l, stream);
+  if (e != cudaSuccess) return e;
+  unsigned char* base = static_cast<unsigned char*>(scratch);
+  rawtab_kernel<<<grid_for(plan.K2p), 256, 0, stream>>>(reinterpret_cast<uint32_t*>(base + l.koff_off), plan.K2,
+                                                        plan.K2p, g.Kh, plan.pitch, plan.nslot,
+                                                        (int)((g.chan_stride * 2) & 15));
   return cudaGetLastError();
 }
 

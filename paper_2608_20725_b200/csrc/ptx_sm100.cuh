@@ -7,6 +7,26 @@
 #include <cuda.h>
 #include <stdint.h>
 
+#ifdef IM2WIN_F16_TIMERS
+// Debug build only: per-thread cycle counters, flushed once into the 64-bit words 4.. of the status block.
+#define TIMER_DECL long long t_prev = clock64(), t_now, t_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
+#define TIMER_LAP(slot)                 \
+  do {                                  \
+    t_now = clock64();                  \
+    t_acc[slot] += t_now - t_prev;      \
+    t_prev = t_now;                     \
+  } while (0)
+#define TIMER_FLUSH()                                                                                              \
+  do {                                                                                                             \
+    for (int ti = 0; ti < 12; ++ti)                                                                                \
+      if (t_acc[ti]) atomicAdd(reinterpret_cast<unsigned long long*>(q.status) + 4 + ti, (unsigned long long)t_acc[ti]); \
+  } while (0)
+#else
+#define TIMER_DECL
+#define TIMER_LAP(slot)
+#define TIMER_FLUSH()
+#endif
+
 namespace im2win {
 namespace ptx {
 
@@ -23,6 +43,18 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Adds `bytes` to the barrier's pending transaction count without arriving.
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Untiled bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completion
+// counted on an mbarrier.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
