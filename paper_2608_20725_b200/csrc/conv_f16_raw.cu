@@ -5,21 +5,26 @@
 // of im2win columns and Kw row-shifted views of it), but the S tile is no longer
 // gathered from global memory with 2-byte loads.  For one channel the columns a
 // tile needs are ONE contiguous run of the window tensor (rows x Kh halves, per
-// image the tile touches).  A loader warp therefore brings the runs of the ~22
-// channels of a k-block into a "raw" shared-memory stage with untiled bulk copies
-// (cp.async.bulk, 16-byte-aligned supersets of the runs, completion on an
-// mbarrier), several stages ahead; HBM/L2 latency is hidden by the copy engine
-// and no load/store-unit request is spent on global memory.  The producer warps
-// only re-lay a raw stage into the k-major swizzled S stage (2-byte shared loads,
+// image the tile touches).  The window tensor is a 2-D array [N*C channel planes]
+// [Ho*Kh*Wp halves] to TMA (the plane pitch must be a multiple of 16 bytes), so a
+// loader warp brings the runs of the ~22 channels of a k-block into a "raw"
+// shared-memory stage with a handful of tiled TMA loads (boxes of 128 halves x
+// nslot planes, starting on 8-element boundaries and overlapping by 8 so that
+// every Kh-element record lies inside one box), several stages ahead: HBM/L2
+// latency is hidden by the copy engine and no load/store-unit request is spent on
+// global memory.  (One untiled bulk copy per channel was tried first: ~120 cycles
+// of issue per copy made the loader the bottleneck.)  The producer warps only
+// re-lay a raw stage into the k-major swizzled S stage (2-byte shared loads,
 // 16-byte shared stores), which is latency-free work.
 //
-//   raw stage:  [slot = channel - first channel of the k-block][PITCH bytes]
-//               slot layout: segment g (one per image) at soff_g, data starting
-//               at its 16-byte phase;  a last all-zero slot serves padded k2.
+//   raw stage:  [box][slot = channel - first channel of the k-block][128 halves];
+//               one more, all-zero slot per box serves padded k2.
 //   S stage:    [row][64 halves], 128-byte swizzle            (as in conv_f16_shift.cu)
 //
-// Roles (11 warps): 8 repack/epilogue warps, filter-TMA warp, MMA warp, raw-loader
-// warp.  Rings: raw stages, S stages, filter stages.  All mbarrier waits are bounded.
+// Roles (16 warps): 8 repack warps, filter-TMA warp, MMA warp, raw-loader warp, 4 epilogue
+// warps.  The kernel is persistent with a double-buffered accumulator in tensor memory, so
+// that the epilogue of one tile overlaps the main loop of the next.  Rings: raw stages, S
+// stages, filter stages.  All mbarrier waits are bounded.
 #include <cuda.h>
 #include <stdlib.h>
 
@@ -35,44 +40,84 @@ constexpr int TILE_M = 128;
 constexpr int KB = kF16KBlock;
 constexpr int PRODUCER_WARPS = 8;
 constexpr int PRODUCER_THREADS = PRODUCER_WARPS * 32;
-constexpr int NUM_THREADS = PRODUCER_THREADS + 96;   // + filter-TMA warp + MMA warp + raw-loader warp
+constexpr int WARP_TMA = 8, WARP_MMA = 9, WARP_RAW = 10, WARP_EPI0 = 12;   // warp 11 idles
+constexpr int NUM_WARPS = 16;
+constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr int MAX_STAGES = 6;
 constexpr int SEG_MAX = 4;                           // images one tile may touch
 constexpr int ITEMS = 5;                             // 16-byte chunks per producer thread and stage (<= 160 rows)
 
 struct RawParams {
   const uint16_t* __restrict__ win;
-  const uint32_t* __restrict__ rawtab;   // k2 -> (slot*pitch + u*2) | ((c*cs16)&15) << 20 ; padded k2 -> zero slot
+  const uint32_t* __restrict__ rawtab;   // k2 -> slot*256 + u*2 ; padded k2 -> the zero slot
   float* __restrict__ y;
   uint32_t* status;
   int64_t VQ, img_stride, chan_stride, window_elems;
   int32_t C, N, Wq, Ho, Wo, HoWo, Co, Kh, Kw, num_kb;
   int32_t rows;             // rows of the S tile: 128 + halo, multiple of 8
-  int32_t pitch, nslot;     // raw slot pitch in bytes; slots per stage (without the zero slot)
-  int32_t raw_stage_bytes;  // (nslot + 1) * pitch
+  int32_t nslot;            // channel planes per box (without the zero slot)
+  int32_t box_bytes;        // (nslot + 1) * 256
+  int32_t raw_stage_bytes;  // maxbox * box_bytes
   int32_t a_stage_bytes;    // rows * 128
-  int32_t cs16;             // (chan_stride * 2) & 15: how the 16-byte phase moves from channel to channel
   int32_t rs, sa, sb;       // ring depths
+  int32_t ntm, nwork;       // position tiles; work items = position tiles x channel tiles
+  int32_t dbg_skip_b;       // experiment switch: do not load filter tiles (timing only, wrong results)
 };
+
+constexpr int BOXW = 128;   // halves per box row
+constexpr int BOXSTEP = 120;  // boxes of one segment start 120 halves apart (overlap 8 >= Kh - 1)
 
 struct Segment {            // the part of a tile that lies in one image
-  int64_t elem0;            // element offset of (image, channel 0, first row of the segment)
+  int32_t plane0;           // first channel plane of the image: n * C
+  int32_t x0;               // first box column: the segment's first element rounded down to 8
+  int32_t o0;               // offset of the segment's first element from x0 (0..7)
   int32_t row0, cnt;        // tile rows [row0, row0 + cnt)
-  int32_t soff;             // byte offset of the segment inside a raw slot (multiple of 16)
+  int32_t box0, nbox;       // boxes [box0, box0 + nbox) of the raw stage belong to this segment
+  int32_t pad_;
 };
 
+// Splits the rows of the tile starting at virtual position q0 by image: within an image the
+// columns of one channel are contiguous in the window tensor.
+__device__ __forceinline__ int split_by_image(const RawParams& q, int64_t q0, Segment* segs) {
+  const int64_t img_rows = (int64_t)q.Ho * q.Wq;
+  int64_t n = q0 / img_rows, a = q0 - n * img_rows;
+  int remaining = q.rows, row0 = 0, box0 = 0, g = 0;
+  while (remaining > 0 && n < q.N && g < SEG_MAX) {
+    const int cnt = (int)(remaining < img_rows - a ? remaining : img_rows - a);
+    const int f0 = (int)(a * q.Kh);                      // element offset inside the channel plane
+    const int span = (f0 & 7) + cnt * q.Kh;
+    segs[g].plane0 = (int)(n * q.C);
+    segs[g].x0 = f0 & ~7;
+    segs[g].o0 = f0 & 7;
+    segs[g].row0 = row0;
+    segs[g].cnt = cnt;
+    segs[g].box0 = box0;
+    segs[g].nbox = span <= BOXW ? 1 : (span - (BOXW - BOXSTEP) + BOXSTEP - 1) / BOXSTEP;
+    box0 += segs[g].nbox;
+    row0 += cnt;
+    remaining -= cnt;
+    a = 0;
+    ++n;
+    ++g;
+  }
+  return g;
+}
+
+// Persistent kernel: every CTA walks work items w = blockIdx.x, blockIdx.x + gridDim.x, ...
+// (w -> position tile w mod ntm, channel tile w div ntm).  The rings and their phases run on
+// across work items; the accumulator is double buffered in tensor memory so that the epilogue
+// warps drain one tile while the MMA warp already fills the next.
 template <int BN>
 __global__ void __launch_bounds__(NUM_THREADS, (BN <= 128 ? 2 : 1))
-conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, RawParams q) {
+conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_constant__ CUtensorMap wmap, RawParams q) {
   constexpr int B_STAGE_BYTES = BN * KB * 2;
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-  __shared__ __align__(8) uint64_t bars[6 * MAX_STAGES + 1];
+  __shared__ __align__(8) uint64_t bars[6 * MAX_STAGES + 4];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile uint32_t abort_flag;
-  __shared__ Segment segs[SEG_MAX];
-  __shared__ int nseg_s;
+  __shared__ Segment seg_s[NUM_WARPS][SEG_MAX];     // each warp keeps its own copy of the tile's segments
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -88,11 +133,8 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, RawParams q) {
   const uint32_t b_empty0 = smem_u32(&bars[3 * MAX_STAGES]);
   const uint32_t r_full0 = smem_u32(&bars[4 * MAX_STAGES]);
   const uint32_t r_empty0 = smem_u32(&bars[5 * MAX_STAGES]);
-  const uint32_t acc_bar = smem_u32(&bars[6 * MAX_STAGES]);
-
-  const int64_t q0 = (int64_t)blockIdx.x * TILE_M;   // first virtual position of the tile
-  const int n0 = blockIdx.y * BN;
-  const int64_t img_rows = (int64_t)q.Ho * q.Wq;     // virtual positions per image
+  const uint32_t acc_full0 = smem_u32(&bars[6 * MAX_STAGES]);
+  const uint32_t acc_empty0 = smem_u32(&bars[6 * MAX_STAGES + 2]);
 
   if (threadIdx.x == 0) {
     abort_flag = 0u;
@@ -104,137 +146,243 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, RawParams q) {
       mbar_init(r_full0 + 8 * i, 1);
       mbar_init(r_empty0 + 8 * i, PRODUCER_WARPS);
     }
-    mbar_init(acc_bar, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    // Split the tile's rows by image: within an image the columns of one channel are contiguous.
-    int64_t n = q0 / img_rows, a = q0 - n * img_rows;
-    int remaining = q.rows, row0 = 0, soff = 0, g = 0;
-    while (remaining > 0 && n < q.N && g < SEG_MAX) {
-      const int cnt = (int)(remaining < img_rows - a ? remaining : img_rows - a);
-      segs[g].elem0 = n * q.img_stride + a * q.Kh;
-      segs[g].row0 = row0;
-      segs[g].cnt = cnt;
-      segs[g].soff = soff;
-      soff += (cnt * q.Kh * 2 + 16 + 15) & ~15;
-      row0 += cnt;
-      remaining -= cnt;
-      a = 0;
-      ++n;
-      ++g;
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(acc_full0 + 8 * i, 1);
+      mbar_init(acc_empty0 + 8 * i, 4);      // the four epilogue warps
     }
-    nseg_s = g;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == PRODUCER_WARPS + 1) tmem_alloc(smem_u32(&tmem_base_slot), BN);
+  if (warp == WARP_MMA) tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
   // k2 table into shared memory; zero slot of every raw stage
   for (int i = threadIdx.x; i < q.num_kb * KB; i += NUM_THREADS) tab_s[i] = __ldg(q.rawtab + i);
-  for (int r = 0; r < q.rs; ++r) {
-    uint32_t* z = reinterpret_cast<uint32_t*>(raw_ptr + r * q.raw_stage_bytes + q.nslot * q.pitch);
-    for (int i = threadIdx.x; i < q.pitch / 4; i += NUM_THREADS) z[i] = 0u;
+  for (int r = 0; r < q.rs * (q.raw_stage_bytes / q.box_bytes); ++r) {
+    uint32_t* z = reinterpret_cast<uint32_t*>(raw_ptr + r * q.box_bytes + q.nslot * 256);
+    for (int i = threadIdx.x; i < 64; i += NUM_THREADS) z[i] = 0u;
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_acc = tmem_base_slot;
-  const int nseg = nseg_s;
+  Segment* segs = seg_s[warp];
 
   if (warp < PRODUCER_WARPS) {
     // ---------------- repack: raw stage -> S stage ------------------------------
-    // item = (row, 16-byte chunk), item = chunk * rows + row (lanes on consecutive rows).
-    // rbase = byte offset of the row's data inside a raw slot (segment offset + rows before it
-    // + the segment's 16-byte phase for channel 0); meta = swizzled S offset | chunk | valid << 3.
+    // item = (row, 16-byte chunk), item = chunk * rows + row (lanes on consecutive rows): fixed
+    // per thread.  Per tile: rbase = byte offset of the row's data inside a raw slot (segment
+    // offset + rows before it) | the segment's 16-byte phase for channel 0 << 24; bit 3 of meta
+    // marks rows inside the tensor.
     uint32_t rbase[ITEMS], meta[ITEMS];
+    int irow[ITEMS];
     const int n_items = q.rows * 8;
 #pragma unroll
     for (int it = 0; it < ITEMS; ++it) {
       const int item = threadIdx.x + it * PRODUCER_THREADS;
-      rbase[it] = 0;
       meta[it] = 0xffffffffu;
+      irow[it] = 0;
       if (item < n_items) {
         const int ch = item / q.rows;
         const int i = item - ch * q.rows;
+        irow[it] = i;
         meta[it] = (uint32_t)(i * 128 + ((ch ^ (i & 7)) << 4)) | (uint32_t)ch;
-        for (int g = 0; g < nseg; ++g) {
-          if (i >= segs[g].row0 && i < segs[g].row0 + segs[g].cnt) {
-            const uint32_t m0 = (uint32_t)((segs[g].elem0 * 2) & 15);
-            rbase[it] = (uint32_t)(segs[g].soff + (i - segs[g].row0) * q.Kh * 2) | (m0 << 24);
-            meta[it] |= 8u;
-          }
-        }
       }
     }
-    const bool phase_moves = q.cs16 != 0;   // channel stride not a multiple of 16 bytes
-
     bool ok = true;
     int st = 0, rst = 0;
     uint32_t ph = 0, rph = 0;
     TIMER_DECL;
-    if (threadIdx.x == 0) TIMER_LAP(0);
-    for (int kb = 0; kb < q.num_kb; ++kb) {
-      if (lane == 0) {
-        ok = mbar_wait(r_full0 + 8 * rst, rph, &abort_flag, q.status);
-        if (threadIdx.x == 0) TIMER_LAP(1);   // wait for the raw stage
-        if (ok) ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
-        if (threadIdx.x == 0) TIMER_LAP(2);   // wait for a free S stage
-      }
-      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-      if (!ok) break;
-      const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
-      const uint32_t raw_stage = raw_ring + rst * q.raw_stage_bytes;
-      const uint4* kt = reinterpret_cast<const uint4*>(tab_s + kb * KB);
+    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
+      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+      int nseg = 0;
+      if (lane == 0) nseg = split_by_image(q, q0, segs);
+      nseg = __shfl_sync(0xffffffffu, nseg, 0);
 #pragma unroll
       for (int it = 0; it < ITEMS; ++it) {
-        if (meta[it] == 0xffffffffu) continue;
-        const int ch = (int)(meta[it] & 7u);
-        const uint4 t0 = kt[ch * 2], t1 = kt[ch * 2 + 1];
-        const uint32_t t[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
-        uint32_t h[8];
-        if (!phase_moves) {
-          const uint32_t base = raw_stage + (rbase[it] & 0xffffffu) + (rbase[it] >> 24);
+        rbase[it] = 0;
+        meta[it] &= ~8u;
+        if (meta[it] == 0xfffffff7u) meta[it] = 0xffffffffu;   // "no such item" stays
+        for (int g = 0; g < nseg; ++g) {
+          const int i = irow[it];
+          if (meta[it] != 0xffffffffu && i >= segs[g].row0 && i < segs[g].row0 + segs[g].cnt) {
+            const int o = segs[g].o0 + (i - segs[g].row0) * q.Kh;   // offset of the row's record from x0
+            int j = o / BOXSTEP;                                    // the box that holds the whole record
+            if (j > segs[g].nbox - 1) j = segs[g].nbox - 1;
+            rbase[it] = (uint32_t)((segs[g].box0 + j) * q.box_bytes + (o - j * BOXSTEP) * 2);
+            meta[it] |= 8u;
+          }
+        }
+      }
+      if (threadIdx.x == 0) TIMER_LAP(0);       // per-tile setup
+      for (int kb = 0; kb < q.num_kb; ++kb) {
+        if (lane == 0) {
+          ok = mbar_wait(r_full0 + 8 * rst, rph, &abort_flag, q.status);
+          if (threadIdx.x == 0) TIMER_LAP(1);   // wait for the raw stage
+          if (ok) ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+          if (threadIdx.x == 0) TIMER_LAP(2);   // wait for a free S stage
+        }
+        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        if (!ok) break;
+        const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
+        const uint32_t raw_stage = raw_ring + rst * q.raw_stage_bytes;
+        const uint4* kt = reinterpret_cast<const uint4*>(tab_s + kb * KB);
+#pragma unroll
+        for (int it = 0; it < ITEMS; ++it) {
+          if (meta[it] == 0xffffffffu) continue;
+          const int ch = (int)(meta[it] & 7u);
+          const uint4 t0 = kt[ch * 2], t1 = kt[ch * 2 + 1];
+          const uint32_t t[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+          uint32_t h[8];
+          const uint32_t base = raw_stage + rbase[it];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             uint16_t v;
             asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(base + t[e]));
             h[e] = v;
           }
-        } else {
-          const uint32_t base = raw_stage + (rbase[it] & 0xffffffu);
-          const uint32_t m0 = rbase[it] >> 24;
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            uint16_t v;
-            const uint32_t mis = (m0 + (t[e] >> 20)) & 15u;
-            asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(base + (t[e] & 0xfffffu) + mis));
-            h[e] = v;
-          }
+          const bool live = (meta[it] & 8u) != 0;   // rows beyond the tensor contribute zeros
+          const uint32_t w0 = live ? (h[0] | (h[1] << 16)) : 0u, w1 = live ? (h[2] | (h[3] << 16)) : 0u;
+          const uint32_t w2 = live ? (h[4] | (h[5] << 16)) : 0u, w3 = live ? (h[6] | (h[7] << 16)) : 0u;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_stage + (meta[it] & ~15u)), "r"(w0),
+                       "r"(w1), "r"(w2), "r"(w3)
+                       : "memory");
         }
-        const bool live = (meta[it] & 8u) != 0;   // rows beyond the tensor contribute zeros
-        const uint32_t w0 = live ? (h[0] | (h[1] << 16)) : 0u, w1 = live ? (h[2] | (h[3] << 16)) : 0u;
-        const uint32_t w2 = live ? (h[4] | (h[5] << 16)) : 0u, w3 = live ? (h[6] | (h[7] << 16)) : 0u;
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_stage + (meta[it] & ~15u)), "r"(w0),
-                     "r"(w1), "r"(w2), "r"(w3)
-                     : "memory");
+        if (threadIdx.x == 0) TIMER_LAP(3);     // repack
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(a_full0 + 8 * st);
+          mbar_arrive(r_empty0 + 8 * rst);
+        }
+        if (threadIdx.x == 0) TIMER_LAP(4);     // fence + arrive
+        if (++st == q.sa) { st = 0; ph ^= 1u; }
+        if (++rst == q.rs) { rst = 0; rph ^= 1u; }
       }
-      if (threadIdx.x == 0) TIMER_LAP(3);     // repack
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(a_full0 + 8 * st);
-        mbar_arrive(r_empty0 + 8 * rst);
-      }
-      if (threadIdx.x == 0) TIMER_LAP(4);     // fence + arrive
-      if (++st == q.sa) { st = 0; ph ^= 1u; }
-      if (++rst == q.rs) { rst = 0; rph ^= 1u; }
     }
-
-    // ---------------- epilogue --------------------------------------------------
-    if (ok && lane == 0) ok = mbar_wait(acc_bar, 0u, &abort_flag, q.status);
-    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-    if (threadIdx.x == 0) TIMER_LAP(5);        // wait for the accumulator
-    if (ok) {
+    if (threadIdx.x == 0) TIMER_FLUSH();
+  } else if (warp == WARP_TMA) {
+    // ---------------- TMA loader of the filter tiles ---------------------------
+    const bool leader = elect_one();
+    bool ok = true;
+    int st = 0;
+    uint32_t ph = 0;
+    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
+      const int n0 = (w / q.ntm) * BN;
+      for (int kb = 0; kb < q.num_kb && ok; ++kb) {
+        for (int v = 0; v < q.Kw; ++v) {
+          ok = mbar_wait(b_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          const uint32_t bar = b_full0 + 8 * st;
+          if (leader) {
+            if (q.dbg_skip_b) {
+              mbar_arrive(bar);
+            } else {
+              mbar_arrive_expect_tx(bar, B_STAGE_BYTES);
+              tma_load_3d(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0, v, bar);
+            }
+          }
+          __syncwarp();
+          if (++st == q.sb) { st = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == WARP_MMA) {
+    // ---------------- MMA issuer ------------------------------------------------
+    constexpr uint32_t idesc = instr_desc_f16(TILE_M, BN);
+    const bool leader = elect_one();
+    bool ok = true;
+    int sta = 0, stb = 0;
+    uint32_t pha = 0, phb = 0;
+    uint32_t it = 0;                             // work items done by this CTA: accumulator buffer = it & 1
+    const uint32_t a_lo0 = smem_desc_lo(a_ring), b_lo0 = smem_desc_lo(b_ring);
+    TIMER_DECL;
+    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
+      const uint32_t buf = it & 1u;
+      TIMER_LAP(8);
+      ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      TIMER_LAP(11);                             // MMA warp: wait for a free accumulator
       tc_fence_after();
-      const int lq = warp & 3;                 // tensor-memory lane quadrant this warp may read
-      const int chalf = warp >> 2;             // which half of the channel tile
-      const int64_t vq = q0 + lq * 32 + lane;  // accumulator row = virtual position
+      const uint32_t acc = tmem_acc + buf * (uint32_t)BN;
+      uint32_t first = 0;
+      for (int kb = 0; kb < q.num_kb && ok; ++kb) {
+        TIMER_LAP(8);
+        ok = mbar_wait(a_full0 + 8 * sta, pha, &abort_flag, q.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        TIMER_LAP(9);                            // MMA warp: wait for an S stage
+        const uint32_t a_lo_stage = a_lo0 + (uint32_t)(sta * (q.a_stage_bytes >> 4));
+        for (int v = 0; v < q.Kw; ++v) {
+          TIMER_LAP(8);
+          ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          TIMER_LAP(10);                         // MMA warp: wait for a filter stage
+          tc_fence_after();
+          const uint32_t b_lo = b_lo0 + (uint32_t)(stb * (B_STAGE_BYTES >> 4));
+          const uint32_t a_lo = a_lo_stage + (uint32_t)v * 8u;   // kernel column v: the view starts v rows further down
+          if (leader) {
+#pragma unroll
+            for (int j = 0; j < KB / 16; ++j) umma_f16_lohi(acc, a_lo + 2 * j, b_lo + 2 * j, idesc, first | (uint32_t)j);
+            umma_commit(b_empty0 + 8 * stb);
+          }
+          __syncwarp();
+          first = 1u;
+          if (++stb == q.sb) { stb = 0; phb ^= 1u; }
+        }
+        if (ok && leader) umma_commit(a_empty0 + 8 * sta);
+        __syncwarp();
+        if (++sta == q.sa) { sta = 0; pha ^= 1u; }
+      }
+      if (ok && leader) umma_commit(acc_full0 + 8 * buf);
+      __syncwarp();
+    }
+    if (leader) { TIMER_LAP(8); TIMER_FLUSH(); }
+  } else if (warp == WARP_RAW) {
+    // ---------------- raw loader: tiled TMA loads of the channel runs -----------
+    const bool leader = elect_one();
+    bool ok = true;
+    int rst = 0;
+    uint32_t rph = 0;
+    TIMER_DECL;
+    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
+      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+      int nseg = 0;
+      if (lane == 0) nseg = split_by_image(q, q0, segs);
+      nseg = __shfl_sync(0xffffffffu, nseg, 0);
+      for (int kb = 0; kb < q.num_kb && ok; ++kb) {
+        if (leader) TIMER_LAP(6);              // raw loader: issuing copies
+        ok = mbar_wait(r_empty0 + 8 * rst, rph ^ 1u, &abort_flag, q.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (leader) TIMER_LAP(5);              // raw loader: wait for a free raw stage
+        const uint32_t bar = r_full0 + 8 * rst;
+        const int c_lo = (kb * KB) / q.Kh;
+        const uint32_t stage = raw_ring + rst * q.raw_stage_bytes;
+        if (leader) {
+          int nbox = 0;
+          for (int g = 0; g < nseg; ++g) nbox += segs[g].nbox;
+          mbar_arrive_expect_tx(bar, (uint32_t)(nbox * q.nslot * 256));
+          for (int g = 0; g < nseg; ++g)
+            for (int j = 0; j < segs[g].nbox; ++j)
+              tma_load_2d(stage + (segs[g].box0 + j) * q.box_bytes, &wmap, segs[g].x0 + j * BOXSTEP,
+                          segs[g].plane0 + c_lo, bar);
+        }
+        __syncwarp();
+        if (++rst == q.rs) { rst = 0; rph ^= 1u; }
+      }
+    }
+    if (leader) { TIMER_LAP(6); TIMER_FLUSH(); }
+  } else if (warp >= WARP_EPI0) {
+    // ---------------- epilogue: tensor memory -> NCHW output --------------------
+    const int lq = warp & 3;                     // tensor-memory lane quadrant this warp may read
+    bool ok = true;
+    uint32_t it = 0;
+    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
+      const uint32_t buf = it & 1u;
+      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+      const int n0 = (w / q.ntm) * BN;
+      const int64_t vq = q0 + lq * 32 + lane;    // accumulator row = virtual position
       bool valid = false;
       float* yrow = q.y;
       if (vq < q.VQ) {
@@ -242,12 +390,16 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, RawParams q) {
         const int kq = (int)(vq - sg * q.Wq);
         const int64_t n = sg / q.Ho;
         const int ho = (int)(sg - n * q.Ho);
-        valid = kq < q.Wo;                     // trailing columns of a strip are no output
+        valid = kq < q.Wo;                       // trailing columns of a strip are no output
         yrow += (n * q.Co) * q.HoWo + ho * q.Wo + kq;
       }
-      const uint32_t lane_base = tmem_acc + ((uint32_t)(lq * 32) << 16);
+      if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
 #pragma unroll 1
-      for (int c0 = chalf * (BN / 2); c0 < (chalf + 1) * (BN / 2); c0 += 32) {
+      for (int c0 = 0; c0 < BN; c0 += 32) {
         if (n0 + c0 >= q.Co) break;
         uint32_t v[32];
         tmem_ld32(lane_base + (uint32_t)c0, v);
@@ -259,109 +411,10 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, RawParams q) {
           }
         }
       }
-    }
-    if (threadIdx.x == 0) { TIMER_LAP(6); TIMER_FLUSH(); }   // epilogue
-  } else if (warp == PRODUCER_WARPS) {
-    // ---------------- TMA loader of the filter tiles ---------------------------
-    const bool leader = elect_one();
-    bool ok = true;
-    int st = 0;
-    uint32_t ph = 0;
-    for (int kb = 0; kb < q.num_kb && ok; ++kb) {
-      for (int v = 0; v < q.Kw; ++v) {
-        ok = mbar_wait(b_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        const uint32_t bar = b_full0 + 8 * st;
-        if (leader) {
-          mbar_arrive_expect_tx(bar, B_STAGE_BYTES);
-          tma_load_3d(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0, v, bar);
-        }
-        __syncwarp();
-        if (++st == q.sb) { st = 0; ph ^= 1u; }
-      }
-    }
-  } else if (warp == PRODUCER_WARPS + 1) {
-    // ---------------- MMA issuer ------------------------------------------------
-    constexpr uint32_t idesc = instr_desc_f16(TILE_M, BN);
-    const bool leader = elect_one();
-    bool ok = true;
-    int sta = 0, stb = 0;
-    uint32_t pha = 0, phb = 0, first = 0;
-    const uint32_t a_lo0 = smem_desc_lo(a_ring), b_lo0 = smem_desc_lo(b_ring);
-    TIMER_DECL;
-    for (int kb = 0; kb < q.num_kb && ok; ++kb) {
-      TIMER_LAP(8);
-      ok = mbar_wait(a_full0 + 8 * sta, pha, &abort_flag, q.status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      TIMER_LAP(9);                            // MMA warp: wait for an S stage
-      const uint32_t a_lo_stage = a_lo0 + (uint32_t)(sta * (q.a_stage_bytes >> 4));
-      for (int v = 0; v < q.Kw; ++v) {
-        TIMER_LAP(8);
-        ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        TIMER_LAP(10);                         // MMA warp: wait for a filter stage
-        tc_fence_after();
-        const uint32_t b_lo = b_lo0 + (uint32_t)(stb * (B_STAGE_BYTES >> 4));
-        const uint32_t a_lo = a_lo_stage + (uint32_t)v * 8u;   // kernel column v: the view starts v rows further down
-        if (leader) {
-#pragma unroll
-          for (int j = 0; j < KB / 16; ++j) umma_f16_lohi(tmem_acc, a_lo + 2 * j, b_lo + 2 * j, idesc, first | (uint32_t)j);
-          umma_commit(b_empty0 + 8 * stb);
-        }
-        __syncwarp();
-        first = 1u;
-        if (++stb == q.sb) { stb = 0; phb ^= 1u; }
-      }
-      if (ok && leader) umma_commit(a_empty0 + 8 * sta);
+      // the buffer may be overwritten once all four warps have read it
+      tc_fence_before();
       __syncwarp();
-      if (++sta == q.sa) { sta = 0; pha ^= 1u; }
-    }
-    if (ok && leader) umma_commit(acc_bar);
-    __syncwarp();
-    if (leader) { TIMER_LAP(8); TIMER_FLUSH(); }
-  } else {
-    // ---------------- raw loader: bulk copies of the channel runs ---------------
-    // Lane l serves slots l, l + 32, ... of a stage: for every image the tile touches, one
-    // bulk copy of the 16-byte-aligned superset of (rows x Kh) halves of that channel.
-    bool ok = true;
-    int rst = 0;
-    uint32_t rph = 0;
-    const int64_t win_bytes = q.window_elems * 2;
-    const int64_t win_bytes16 = win_bytes & ~(int64_t)15;
-    for (int kb = 0; kb < q.num_kb && ok; ++kb) {
-      ok = mbar_wait(r_empty0 + 8 * rst, rph ^ 1u, &abort_flag, q.status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      const uint32_t bar = r_full0 + 8 * rst;
-      const int c_lo = (kb * KB) / q.Kh;
-      int c_hi = (kb * KB + KB - 1) / q.Kh;
-      if (c_hi >= q.C) c_hi = q.C - 1;
-      unsigned char* stage_ptr = raw_ptr + rst * q.raw_stage_bytes;
-      for (int c = c_lo + lane; c <= c_hi; c += 32) {
-        const int slot = c - c_lo;
-        for (int g = 0; g < nseg; ++g) {
-          const int64_t byte0 = (segs[g].elem0 + (int64_t)c * q.chan_stride) * 2;
-          const int64_t beg = byte0 & ~(int64_t)15;
-          const int64_t want_end = byte0 + (int64_t)segs[g].cnt * q.Kh * 2;
-          int64_t end = (want_end + 15) & ~(int64_t)15;
-          if (end > win_bytes16) end = win_bytes16;       // never read past the tensor
-          unsigned char* dst = stage_ptr + slot * q.pitch + segs[g].soff;
-          if (end > beg) {
-            mbar_expect_tx(bar, (uint32_t)(end - beg));
-            bulk_load(smem_u32(dst), reinterpret_cast<const unsigned char*>(q.win) + beg, (uint32_t)(end - beg), bar);
-          }
-          // the last (< 16) bytes of the whole tensor, if this run needs them, by plain loads
-          for (int64_t b = (end > beg ? end : beg); b < want_end && b < win_bytes; b += 2)
-            *reinterpret_cast<uint16_t*>(dst + (b - beg)) = __ldg(reinterpret_cast<const uint16_t*>(
-                reinterpret_cast<const unsigned char*>(q.win) + b));
-        }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar);   // the one pending arrival: the phase completes when the bytes have landed
-      if (++rst == q.rs) { rst = 0; rph ^= 1u; }
+      if (lane == 0) mbar_arrive(acc_empty0 + 8 * buf);
     }
   }
 
@@ -372,10 +425,10 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, RawParams q) {
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
   }
-  if (warp == PRODUCER_WARPS + 1) {
+  if (warp == WARP_MMA) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_acc, BN);
+    tmem_dealloc(tmem_acc, 2 * BN);
   }
 }
 
@@ -401,10 +454,14 @@ constexpr int kSmemMax = 227 * 1024;
 
 // Ring depths that fit: S ring 2, raw ring 3 (2 if tight), filter ring as deep as fits (<= 4).
 bool choose_rings(int bn, const RawPlan& plan, int* rs, int* sa, int* sb, int* smem_bytes) {
-  const int budget = (bn <= 128 ? kSmemMax / 2 : kSmemMax) - 1024 - 512;
+  // dynamic shared memory left after the alignment slack, the static part (barriers, segment
+  // copies) and, for two CTAs per SM, the 1 KB the runtime reserves per CTA
+  const int budget = (bn <= 128 ? kSmemMax / 2 : kSmemMax) - 1024 - 4096;
   const int fixed = (int)plan.K2p * 4;
   const int a = plan.a_stage_bytes, r = plan.raw_stage_bytes, b = bn * KB * 2;
-  for (int rr = 3; rr >= 2; --rr)
+  const char* fr = getenv("IM2WIN_DBG_RS");
+  const int rr0 = fr ? atoi(fr) : 3;
+  for (int rr = rr0; rr >= 2; --rr)
     for (int bb = 4; bb >= 2; --bb)
       if (2 * a + rr * r + bb * b + fixed <= budget && (bb >= 3 || rr == 2)) {
         *rs = rr; *sa = 2; *sb = bb;
@@ -415,13 +472,20 @@ bool choose_rings(int bn, const RawPlan& plan, int* rs, int* sa, int* sb, int* s
 }
 
 template <int BN>
-cudaError_t launch_bn(const CUtensorMap& fmap, RawParams q, const RawPlan& plan, int co, cudaStream_t stream) {
+cudaError_t launch_bn(const CUtensorMap& fmap, const CUtensorMap& wmap, RawParams q, const RawPlan& plan, int co,
+                      cudaStream_t stream) {
   int smem_bytes = 0;
   if (!choose_rings(BN, plan, &q.rs, &q.sa, &q.sb, &smem_bytes)) return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(conv_f16_raw_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
-  dim3 grid((unsigned)((plan.VQ + TILE_M - 1) / TILE_M), (unsigned)((co + BN - 1) / BN));
-  conv_f16_raw_kernel<BN><<<grid, NUM_THREADS, smem_bytes, stream>>>(fmap, q);
+  const int64_t ntm = (plan.VQ + TILE_M - 1) / TILE_M;
+  const int64_t nwork = ntm * ((co + BN - 1) / BN);
+  if (nwork >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
+  q.ntm = (int32_t)ntm;
+  q.nwork = (int32_t)nwork;
+  const int slots = 148 * (BN <= 128 ? 2 : 1);        // persistent CTAs: one (two for narrow tiles) per SM
+  const unsigned grid = (unsigned)(nwork < slots ? nwork : slots);
+  conv_f16_raw_kernel<BN><<<grid, NUM_THREADS, smem_bytes, stream>>>(fmap, wmap, q);
   return cudaGetLastError();
 }
 
@@ -442,14 +506,36 @@ RawPlan plan_f16_raw(const Geometry& g) {
   const int64_t img_rows = (int64_t)g.Ho * p.Wq;
   const int64_t segmax = (p.rows - 2) / img_rows + 2;     // images a tile can touch
   if (segmax > SEG_MAX) return p;
+  if (g.Kh > 8) return p;                                 // a record must fit the 8-element box overlap
+  if ((g.chan_stride * 2) % 16 != 0) return p;            // TMA needs a plane pitch that is a multiple of 16 bytes
+  if ((int64_t)g.N * g.C >= ((int64_t)1 << 31)) return p;
   p.nslot = (KB - 1 + g.Kh - 1) / g.Kh + 1;               // channels a 64-wide k2 block can touch
   if (p.nslot > g.C) p.nslot = g.C;
-  p.pitch = ((p.rows * g.Kh * 2 + 15) & ~15) + 32 * (int)segmax;
-  if ((int64_t)(p.nslot + 1) * p.pitch >= (1 << 20)) return p;   // table entries keep 20 bits of offset
-  p.raw_stage_bytes = (p.nslot + 1) * p.pitch;
+  if (p.nslot > 256) return p;
+  p.pitch = 256;
+  // boxes one stage can need: the exact maximum over the tile start positions (period <= img_rows tiles)
+  int maxbox = 1;
+  {
+    const int64_t ntiles = (p.VQ + TILE_M - 1) / TILE_M;
+    const int64_t probe = ntiles < img_rows ? ntiles : img_rows;
+    for (int64_t t = 0; t < probe && t < 65536; ++t) {
+      int64_t a = (t * TILE_M) % img_rows;
+      int remaining = p.rows, boxes = 0;
+      while (remaining > 0) {
+        const int cnt = (int)(remaining < img_rows - a ? remaining : img_rows - a);
+        const int span = (int)((a * g.Kh) & 7) + cnt * g.Kh;
+        boxes += span <= BOXW ? 1 : (span - (BOXW - BOXSTEP) + BOXSTEP - 1) / BOXSTEP;
+        remaining -= cnt;
+        a = 0;
+      }
+      if (boxes > maxbox) maxbox = boxes;
+    }
+    if (probe > 65536) maxbox += (int)segmax;   // unprobed phases: leave room for one more box per image
+  }
+  p.raw_stage_bytes = maxbox * (p.nslot + 1) * 256;
   p.a_stage_bytes = p.rows * 128;
   if (p.K2p * 4 > 24 * 1024) return p;
-  if ((p.VQ + TILE_M - 1) / TILE_M >= ((int64_t)1 << 31)) return p;
+  if ((p.VQ + TILE_M - 1) / TILE_M * ((g.Co + 63) / 64) >= ((int64_t)1 << 31)) return p;
   int rs, sa, sb, smem;
   const int bn = g.Co <= 64 ? 64 : (g.Co <= 128 ? 128 : 256);
   if (!choose_rings(bn, p, &rs, &sa, &sb, &smem)) return p;
@@ -477,6 +563,19 @@ cudaError_t launch_conv_f16_raw(const uint16_t* window, float* y, void* scratch,
                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
 
+  // Window tensor as [N*C planes][chan_stride halves]; one box = 128 halves of nslot planes.
+  CUtensorMap wmap;
+  {
+    const cuuint64_t wd[2] = {(cuuint64_t)g.chan_stride, (cuuint64_t)g.N * (cuuint64_t)g.C};
+    const cuuint64_t ws[1] = {(cuuint64_t)g.chan_stride * 2};
+    const cuuint32_t wb[2] = {(cuuint32_t)BOXW, (cuuint32_t)plan.nslot};
+    const cuuint32_t we[2] = {1, 1};
+    cr = encode(&wmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<uint16_t*>(window), wd, ws, wb, we,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
+
   RawParams q;
   q.win = window;
   q.rawtab = reinterpret_cast<const uint32_t*>(base + l.koff_off);
@@ -485,13 +584,13 @@ cudaError_t launch_conv_f16_raw(const uint16_t* window, float* y, void* scratch,
   q.VQ = plan.VQ; q.img_stride = g.img_stride; q.chan_stride = g.chan_stride; q.window_elems = g.window_elems;
   q.C = g.C; q.N = g.N; q.Wq = plan.Wq; q.Ho = g.Ho; q.Wo = g.Wo; q.HoWo = g.Ho * g.Wo; q.Co = g.Co;
   q.Kh = g.Kh; q.Kw = g.Kw; q.num_kb = (int32_t)(plan.K2p / KB);
-  q.rows = plan.rows; q.pitch = plan.pitch; q.nslot = plan.nslot;
+  q.rows = plan.rows; q.nslot = plan.nslot; q.box_bytes = (plan.nslot + 1) * 256;
   q.raw_stage_bytes = plan.raw_stage_bytes; q.a_stage_bytes = plan.a_stage_bytes;
-  q.cs16 = (int32_t)((g.chan_stride * 2) & 15);
   q.rs = q.sa = q.sb = 2;
-  if (bn == 64) return launch_bn<64>(fmap, q, plan, g.Co, stream);
-  if (bn == 128) return launch_bn<128>(fmap, q, plan, g.Co, stream);
-  return launch_bn<256>(fmap, q, plan, g.Co, stream);
+  q.dbg_skip_b = getenv("IM2WIN_DBG_SKIP_B") ? 1 : 0;
+  if (bn == 64) return launch_bn<64>(fmap, wmap, q, plan, g.Co, stream);
+  if (bn == 128) return launch_bn<128>(fmap, wmap, q, plan, g.Co, stream);
+  return launch_bn<256>(fmap, wmap, q, plan, g.Co, stream);
 }
 
 }  // namespace im2win

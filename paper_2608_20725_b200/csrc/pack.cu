@@ -106,10 +106,9 @@ __global__ void pack_f16_shift_kernel(const uint16_t* __restrict__ f, uint16_t* 
   }
 }
 
-// Table of the bulk-copy fp16 kernel: k2 -> byte offset of element (c, u) inside a raw stage,
-// slot (c - first channel of the k-block) * pitch + u*2, with (c * cs16) & 15 in bits 20..23
-// (how far the 16-byte phase of channel c's run is from channel 0's); padded k2 point at the
-// all-zero slot `nslot`.
+// Table of the TMA-staged fp16 kernel: k2 -> byte offset of element (c, u) inside a raw box,
+// slot (c - first channel of the k-block) * pitch + u*2; padded k2 point at the all-zero slot
+// `nslot`.
 __global__ void rawtab_kernel(uint32_t* __restrict__ tab, int64_t K2, int64_t K2p, int Kh, int pitch, int nslot,
                               int cs16) {
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -119,7 +118,7 @@ __global__ void rawtab_kernel(uint32_t* __restrict__ tab, int64_t K2, int64_t K2
       const int64_t c = k2 / Kh;
       const int u = (int)(k2 - c * Kh);
       const int64_t c_lo = (k2 / kF16KBlock) * kF16KBlock / Kh;
-      e = (uint32_t)((c - c_lo) * pitch + u * 2) | ((uint32_t)((c * cs16) & 15) << 20);
+      e = (uint32_t)((c - c_lo) * pitch + u * 2);
     }
     tab[k2] = e;
   }
