@@ -69,9 +69,6 @@ template <int BN, int ITEMS>
 __global__ void __launch_bounds__(NUM_THREADS, (BN <= 128 ? 2 : 1))
 conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
   constexpr int B_STAGE_BYTES = BN * KB * 2;
-  // Register double-buffering of the producers' loads needs ~40 more registers per thread:
-  // affordable with one CTA per SM (256-channel tiles), not with two.
-  constexpr bool PREFETCH = BN > 128;
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
@@ -160,10 +157,10 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
     bool ok = true;
     TIMER_DECL;
     if (threadIdx.x == 0) TIMER_LAP(0);   // setup
-    // The stage is produced in units of ITEM_GROUP items.  With PREFETCH the loads of the next
-    // unit are issued before the current one is packed and stored, so that one DRAM/L2 round
-    // trip overlaps the pack/store/handshake of the previous unit.  Dead rows and padded k2 read
-    // a word of the status block that is always zero, so nothing needs masking afterwards.
+    // The stage is produced in units of ITEM_GROUP items whose loads are issued back to back.
+    // Dead rows and padded k2 read a word of the status block that is always zero, so nothing
+    // needs masking afterwards.  (Holding the next unit's loads in a second register buffer,
+    // and L2 prefetches of the next k-blocks' runs, were measured and did not pay.)
     constexpr int G = ITEM_GROUP;
     constexpr int NG = ITEMS / G;
     const uint16_t* __restrict__ zero16 = reinterpret_cast<const uint16_t*>(q.status + 2);
@@ -197,31 +194,21 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
 
     int st = 0;                 // ring slot and its phase bit, advanced without divisions
     uint32_t ph = 0;
-    uint32_t bufA[G][8], bufB[G][8];
-    // One k-block: unit gidx lives in `first` when gidx is even, in `second` when odd; the loads
-    // of the following unit go to the other buffer (no register copies, so nothing waits for
-    // loads before they are needed).
-    auto do_stage = [&](int kb, uint32_t (&first)[G][8], uint32_t (&second)[G][8]) {
+    uint32_t buf[G][8];
+    for (int kb = 0; kb < q.num_kb && ok; ++kb) {
       const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
 #pragma unroll
       for (int gidx = 0; gidx < NG; ++gidx) {
-        uint32_t (&cur)[G][8] = (gidx & 1) ? second : first;
-        uint32_t (&nxt)[G][8] = (gidx & 1) ? first : second;
-        if (PREFETCH) {
-          if (gidx + 1 < NG) issue(kb, gidx + 1, nxt);
-          else if (kb + 1 < q.num_kb) issue(kb + 1, 0, nxt);
-        } else {
-          issue(kb, gidx, cur);
-        }
+        issue(kb, gidx, buf);
         if (gidx == 0) {
           if (threadIdx.x == 0) TIMER_LAP(2);   // issuing loads
           if (lane == 0) ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
           ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
           if (threadIdx.x == 0) TIMER_LAP(1);   // wait for a free stage
         }
-        if (ok) store(a_stage, gidx, cur);
+        if (ok) store(a_stage, gidx, buf);
       }
-      if (!ok) return;
+      if (!ok) break;
       if (threadIdx.x == 0) TIMER_LAP(3);   // waiting for the loads, pack + store
       fence_proxy_async_smem();
       __syncwarp();
@@ -230,15 +217,6 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
       if (++st == q.sa) {
         st = 0;
         ph ^= 1u;
-      }
-    };
-    if (PREFETCH) issue(0, 0, bufA);
-    for (int kb = 0; kb < q.num_kb && ok; kb += 2) {
-      do_stage(kb, bufA, bufB);
-      if (kb + 1 < q.num_kb && ok) {
-        // with an odd number of units per k-block the roles of the buffers swap every k-block
-        if (NG & 1) do_stage(kb + 1, bufB, bufA);
-        else do_stage(kb + 1, bufA, bufB);
       }
     }
 
@@ -287,39 +265,7 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
     bool ok = true;
     int st = 0;
     uint32_t ph = 0;
-    // L2 prefetch of the window data the producers will gather a few k-blocks later: lane l asks
-    // for the contiguous run of channel (first channel of the k-block + l), one bulk prefetch per
-    // image the tile touches.  It turns the producers' DRAM round trips into L2 hits.
-    constexpr int PREFETCH_AHEAD = 3;
-    const int64_t img_rows_t = (int64_t)q.Ho * q.Wq;
-    const int64_t n_first_t = q0 / img_rows_t;
-    const int64_t a_first = q0 - n_first_t * img_rows_t;       // first virtual row inside its image
-    const int64_t win_bytes16 = (q.window_elems * 2) & ~(int64_t)15;
-    auto prefetch_block = [&](int kbp) {
-      const int c = (kbp * KB) / q.Kh + lane;
-      const int c_hi = (kbp * KB + KB - 1) / q.Kh;
-      if (c > c_hi || c >= q.C) return;
-      int64_t n = n_first_t, a = a_first;
-      int remaining = rows;
-      for (int seg = 0; seg < 8 && remaining > 0 && n < q.N; ++seg) {
-        const int64_t cnt = remaining < img_rows_t - a ? remaining : img_rows_t - a;
-        const int64_t byte0 = (n * q.img_stride + (int64_t)c * q.chan_stride + a * q.s * q.Kh) * 2;
-        const int64_t beg = byte0 & ~(int64_t)15;
-        int64_t end = (byte0 + cnt * q.s * q.Kh * 2 + 15) & ~(int64_t)15;
-        if (end > win_bytes16) end = win_bytes16;
-        if (end > beg)
-          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const char*>(q.win) + beg),
-                       "r"((uint32_t)(end - beg))
-                       : "memory");
-        remaining -= (int)cnt;
-        a = 0;
-        ++n;
-      }
-    };
-    for (int kbp = 1; kbp < PREFETCH_AHEAD && kbp < q.num_kb; ++kbp) prefetch_block(kbp);
     for (int kb = 0; kb < q.num_kb && ok; ++kb) {
-      if (kb + PREFETCH_AHEAD < q.num_kb) prefetch_block(kb + PREFETCH_AHEAD);
-      __syncwarp();
       for (int v = 0; v < q.Kw; ++v) {
         ok = mbar_wait(b_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
         ok = __all_sync(0xffffffffu, ok);
