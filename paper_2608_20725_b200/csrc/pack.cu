@@ -78,49 +78,38 @@ __global__ void pack_f16_kernel(const uint16_t* __restrict__ f, uint16_t* __rest
   }
 }
 
-// Layout of the shifted-view fp16 kernel: Fp2[v][co][k2], k2 = c*Kh + u (zero padded to K2p),
-// and the table k2 -> c*chan_stride + u.
+// Layout of the shifted-view fp16 kernels: Fp2[v][co][k2], k2 = c*Kh + u (zero padded to K2p),
+// and one of two tables: k2 -> c*chan_stride + u (gathering kernel, raw_pitch = 0; -1 for padded
+// k2), or k2 -> byte offset of element (c, u) inside a raw box, slot (c - first channel of the
+// k-block) * raw_pitch + u*2, padded k2 pointing at the all-zero slot `nslot` (TMA-staged kernel).
+// Grid: x over k2, y over output channels, z over kernel columns: no per-element divisions
+// beyond k2 / Kh.
 __global__ void pack_f16_shift_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp,
-                                      int32_t* __restrict__ koff, uint32_t* __restrict__ status,
-                                      PackParams q) {
-  if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
-  const int64_t K2 = (int64_t)q.C * q.Kh;
-  const int64_t per_v = q.Kp * q.Co;
-  const int64_t total = per_v * q.Kw;
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-    const int64_t v = i / per_v;
-    const int64_t r = i - v * per_v;
-    const int64_t co = r / q.Kp;
-    const int64_t k2 = r - co * q.Kp;
-    uint16_t val = 0;
-    int32_t off = -1;
-    if (k2 < K2) {
-      const int64_t c = k2 / q.Kh;
-      const int64_t u = k2 - c * q.Kh;
-      val = f[((co * q.C + c) * q.Kh + u) * q.Kw + v];
-      off = (int32_t)(c * q.chan_stride + u);
+                                      uint32_t* __restrict__ table, uint32_t* __restrict__ status,
+                                      PackParams q, int raw_pitch, int nslot) {
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x < kStatusBytes / 4)
+    status[threadIdx.x] = 0u;
+  const int K2 = q.C * q.Kh;
+  const int K2p = (int)q.Kp;
+  const int v = blockIdx.z;
+  for (int co = blockIdx.y; co < q.Co; co += gridDim.y) {
+    for (int k2 = blockIdx.x * blockDim.x + threadIdx.x; k2 < K2p; k2 += gridDim.x * blockDim.x) {
+      uint16_t val = 0;
+      uint32_t entry = raw_pitch > 0 ? (uint32_t)(nslot * raw_pitch) : 0xffffffffu;
+      if (k2 < K2) {
+        const int c = k2 / q.Kh;
+        const int u = k2 - c * q.Kh;
+        val = f[(((size_t)co * q.C + c) * q.Kh + u) * q.Kw + v];
+        if (raw_pitch > 0) {
+          const int c_lo = (k2 / kF16KBlock) * kF16KBlock / q.Kh;
+          entry = (uint32_t)((c - c_lo) * raw_pitch + u * 2);
+        } else {
+          entry = (uint32_t)(c * q.chan_stride + u);
+        }
+      }
+      fp[((size_t)v * q.Co + co) * K2p + k2] = val;
+      if (v == 0 && co == 0) table[k2] = entry;
     }
-    fp[i] = val;
-    if (v == 0 && co == 0) koff[k2] = off;
-  }
-}
-
-// Table of the TMA-staged fp16 kernel: k2 -> byte offset of element (c, u) inside a raw box,
-// slot (c - first channel of the k-block) * pitch + u*2; padded k2 point at the all-zero slot
-// `nslot`.
-__global__ void rawtab_kernel(uint32_t* __restrict__ tab, int64_t K2, int64_t K2p, int Kh, int pitch, int nslot,
-                              int cs16) {
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t k2 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k2 < K2p; k2 += stride) {
-    uint32_t e = (uint32_t)(nslot * pitch);
-    if (k2 < K2) {
-      const int64_t c = k2 / Kh;
-      const int u = (int)(k2 - c * Kh);
-      const int64_t c_lo = (k2 / kF16KBlock) * kF16KBlock / Kh;
-      e = (uint32_t)((c - c_lo) * pitch + u * 2);
-    }
-    tab[k2] = e;
   }
 }
 
@@ -160,26 +149,26 @@ cudaError_t launch_pack_f16(const uint16_t* filter, void* scratch, const Geometr
   return cudaGetLastError();
 }
 
-cudaError_t launch_pack_f16_shift(const uint16_t* filter, void* scratch, const Geometry& g,
-                                  const ScratchLayout& l, cudaStream_t stream) {
+static cudaError_t pack_shift_common(const uint16_t* filter, void* scratch, const Geometry& g,
+                                     const ScratchLayout& l, int raw_pitch, int nslot, cudaStream_t stream) {
   unsigned char* base = static_cast<unsigned char*>(scratch);
   PackParams q = make_params(g, l);
-  pack_f16_shift_kernel<<<grid_for(q.Kp * q.Co * q.Kw), 256, 0, stream>>>(
-      filter, reinterpret_cast<uint16_t*>(base + l.filter_off),
-      reinterpret_cast<int32_t*>(base + l.koff_off), reinterpret_cast<uint32_t*>(base), q);
+  const unsigned gx = (unsigned)((q.Kp + 255) / 256);
+  dim3 grid(gx > 64 ? 64 : gx, (unsigned)(g.Co < 32768 ? g.Co : 32768), (unsigned)(g.Kw < 65535 ? g.Kw : 65535));
+  pack_f16_shift_kernel<<<grid, 256, 0, stream>>>(filter, reinterpret_cast<uint16_t*>(base + l.filter_off),
+                                                  reinterpret_cast<uint32_t*>(base + l.koff_off),
+                                                  reinterpret_cast<uint32_t*>(base), q, raw_pitch, nslot);
   return cudaGetLastError();
+}
+
+cudaError_t launch_pack_f16_shift(const uint16_t* filter, void* scratch, const Geometry& g,
+                                  const ScratchLayout& l, cudaStream_t stream) {
+  return pack_shift_common(filter, scratch, g, l, 0, 0, stream);
 }
 
 cudaError_t launch_pack_f16_raw(const uint16_t* filter, void* scratch, const Geometry& g,
                                 const ScratchLayout& l, const RawPlan& plan, cudaStream_t stream) {
-  // same filter layout as the shifted-view kernel; its offset table is then replaced by the raw table
-  cudaError_t e = launch_pack_f16_shift(filter, scratch, g, l, stream);
-  if (e != cudaSuccess) return e;
-  unsigned char* base = static_cast<unsigned char*>(scratch);
-  rawtab_kernel<<<grid_for(plan.K2p), 256, 0, stream>>>(reinterpret_cast<uint32_t*>(base + l.koff_off), plan.K2,
-                                                        plan.K2p, g.Kh, plan.pitch, plan.nslot,
-                                                        (int)((g.chan_stride * 2) & 15));
-  return cudaGetLastError();
+  return pack_shift_common(filter, scratch, g, l, plan.pitch, plan.nslot, stream);
 }
 
 }  // namespace im2win
