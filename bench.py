@@ -246,11 +246,14 @@ def time_cpu_oracle(layer, target_seconds=12.0):
     oracle.conv_im2win_range(xn, fn, dims, 0, 1)
     t1 = time.perf_counter() - t0
     n = int(max(1, min(layer.N, target_seconds / max(t1, 1e-6))))
-    reps = int(max(1, min(50, round(target_seconds / max(t1 * n, 1e-6)))))
+    reps = 0
     t0 = time.perf_counter()
-    for _ in range(reps):
+    while True:                                   # whole passes over the sample until ~target_seconds
         oracle.conv_im2win_range(xn, fn, dims, 0, n)
-    dt = time.perf_counter() - t0
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt >= target_seconds or reps >= 200:
+            break
     return {"value": per_image * n * reps / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"fp64 im2win route (transform + convolution) on {n} of {layer.N} images of {layer.name}, "
                       f"{reps} passes ({dt:.1f} s)"}
