@@ -6,9 +6,9 @@
 // A CTA computes a BM x BN tile of y.  Per k-block of 16 it gathers the A tile
 // from the window tensor (lanes walk consecutive positions, i.e. addresses
 // s*Kh elements apart inside one strip; the k -> offset table is precomputed)
-// and the Fk tile (contiguous) into shared memory, double buffered with the
-// global loads of the next k-block held in registers while the current block
-// is multiplied.  Each thread accumulates an 8 x 8 register tile with 128-bit
+// and the Fk tile (contiguous) into a three-slot shared-memory ring with
+// asynchronous copies (cp.async: no registers, two k-blocks in flight while the
+// current one is multiplied).  Each thread accumulates an 8 x 8 register tile with 128-bit
 // shared-memory loads (2 x 4 positions by 2 x 4 output channels).  The tile is
 // held as 8 x 4 pairs of adjacent output channels and updated with the packed
 // fma.rn.f32x2 instruction: one issue slot per two FMAs (the FMA pipe rate is
@@ -54,8 +54,9 @@ conv_f32_kernel(ConvF32Params q) {
   constexpr int B_VEC_PER_THREAD = BK * BN / 4 / THREADS; // float4 loads per k-block
   static_assert(THREADS % BM == 0 && A_PER_THREAD * A_KK_STEP == BK, "loader mapping");
 
-  __shared__ __align__(16) float As[2][BK][BM];
-  __shared__ __align__(16) float Bs[2][BK][BN];
+  constexpr int STAGES = 3;          // shared-memory ring filled by asynchronous copies
+  __shared__ __align__(16) float As[STAGES][BK][BM];
+  __shared__ __align__(16) float Bs[STAGES][BK][BN];
 
   const int tid = threadIdx.x;
   const int tm = tid % (BM / 8);     // position direction: fastest across lanes
@@ -77,43 +78,38 @@ conv_f32_kernel(ConvF32Params q) {
     abase += n * q.img_stride + ho * q.strip + (int64_t)wo * q.sKh;
   }
 
-  float areg[A_PER_THREAD];
-  float4 breg[B_VEC_PER_THREAD];
-  int offreg[A_PER_THREAD];          // offsets of the k-block after the one being loaded
+  int offreg[A_PER_THREAD];          // offsets of the next k-block to be issued
 
-  // The offset table is read one k-block ahead of the data it addresses, so that the
-  // dependent window loads never wait for it.
+  // The offset table is read one k-block ahead of the copies it addresses, so that issuing
+  // the copies never waits for it.
   auto load_offsets = [&](int kb) {
     const int k0 = kb * BK;
 #pragma unroll
     for (int i = 0; i < A_PER_THREAD; ++i) offreg[i] = __ldg(q.koff + k0 + lkk0 + i * A_KK_STEP);
   };
-  auto load_global = [&](int kb, bool more) {
+  // Asynchronous copies (global -> shared, no registers) of k-block kb into ring slot `buf`:
+  // 4-byte gathers of the window operand (zero-filled outside the tensor and in the padded
+  // tail of k), 16-byte copies of the filter rows.
+  auto issue_copies = [&](int kb, int buf, bool more) {
     const int k0 = kb * BK;
 #pragma unroll
     for (int i = 0; i < A_PER_THREAD; ++i) {
       const int off = offreg[i];
-      areg[i] = (lvalid && off >= 0) ? __ldg(abase + off) : 0.f;
+      const bool ok = lvalid && off >= 0;
+      const float* src = ok ? abase + off : q.win;
+      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&As[buf][lkk0 + i * A_KK_STEP][lm]);
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(ok ? 4 : 0) : "memory");
     }
-    if (more) load_offsets(kb + 1);
 #pragma unroll
     for (int i = 0; i < B_VEC_PER_THREAD; ++i) {
       const int e = tid + i * THREADS;       // float4 index inside the BK x BN tile
       const int kk = e / (BN / 4);
       const int nn = (e - kk * (BN / 4)) * 4;
-      breg[i] = __ldg(reinterpret_cast<const float4*>(q.fk + (int64_t)(k0 + kk) * q.Co_pad + n0 + nn));
+      const float* src = q.fk + (int64_t)(k0 + kk) * q.Co_pad + n0 + nn;
+      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&Bs[buf][kk][nn]);
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
     }
-  };
-  auto store_shared = [&](int buf) {
-#pragma unroll
-    for (int i = 0; i < A_PER_THREAD; ++i) As[buf][lkk0 + i * A_KK_STEP][lm] = areg[i];
-#pragma unroll
-    for (int i = 0; i < B_VEC_PER_THREAD; ++i) {
-      const int e = tid + i * THREADS;
-      const int kk = e / (BN / 4);
-      const int nn = (e - kk * (BN / 4)) * 4;
-      *reinterpret_cast<float4*>(&Bs[buf][kk][nn]) = breg[i];
-    }
+    if (more) load_offsets(kb + 1);
   };
 
   unsigned long long acc2[8][4];     // acc2[i][jp] = (acc[i][2jp], acc[i][2jp+1])
@@ -124,13 +120,23 @@ conv_f32_kernel(ConvF32Params q) {
 
   const int nkb = q.Kp / BK;
   load_offsets(0);
-  load_global(0, nkb > 1);
-  store_shared(0);
-  __syncthreads();
+#pragma unroll
+  for (int s = 0; s < STAGES - 1; ++s) {
+    if (s < nkb) issue_copies(s, s, s + 1 < nkb);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
 
+  int buf = 0;                        // ring slot of k-block kb
   for (int kb = 0; kb < nkb; ++kb) {
-    const int buf = kb & 1;
-    if (kb + 1 < nkb) load_global(kb + 1, kb + 2 < nkb);
+    asm volatile("cp.async.wait_group %0;" ::"n"(STAGES - 2) : "memory");
+    __syncthreads();                  // k-block kb has landed for everyone; slot (kb-1) is free
+    {
+      const int nk = kb + STAGES - 1;
+      int nbuf = buf + STAGES - 1;
+      if (nbuf >= STAGES) nbuf -= STAGES;
+      if (nk < nkb) issue_copies(nk, nbuf, nk + 1 < nkb);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
       const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][kk][tm * 4]);
@@ -146,10 +152,7 @@ conv_f32_kernel(ConvF32Params q) {
         for (int jp = 0; jp < 4; ++jp) ffma2(acc2[i][jp], ad, b[jp]);
       }
     }
-    if (kb + 1 < nkb) {
-      store_shared(buf ^ 1);
-      __syncthreads();
-    }
+    if (++buf == STAGES) buf = 0;
   }
 
   float acc[8][8];
