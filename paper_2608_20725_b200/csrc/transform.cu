@@ -32,6 +32,23 @@
 namespace im2win {
 namespace {
 
+// Predicated read-only load: the element if `ok`, else 0.  One predicated instruction instead
+// of a branch around the load, and no memory request at all when the predicate is off.
+__device__ __forceinline__ uint32_t ld_if(const uint32_t* p, bool ok) {
+  uint32_t v = 0;
+  asm("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p ld.global.nc.b32 %0, [%1];\n\t}"
+      : "+r"(v)
+      : "l"(p), "r"((int)ok));
+  return v;
+}
+__device__ __forceinline__ uint16_t ld_if(const uint16_t* p, bool ok) {
+  uint16_t v = 0;
+  asm("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %2, 0;\n\t@p ld.global.nc.u16 %0, [%1];\n\t}"
+      : "+h"(v)
+      : "l"(p), "r"((int)ok));
+  return v;
+}
+
 struct TransformParams {
   int32_t H, W, Wp, Kh, s, p, Ho;
   int32_t cols_per_cta;   // multiple of 8, so every CTA's output range starts 16-byte aligned
@@ -75,8 +92,7 @@ transform_kernel(const E* __restrict__ x, E* __restrict__ win, TransformParams q
 #pragma unroll
       for (int u = 0; u < KH; ++u) {
         const int h = h0 + u;
-        v[u] = 0;
-        if (w_ok && (unsigned)h < (unsigned)q.H) v[u] = __ldg(src + (size_t)h * q.W);
+        v[u] = ld_if(src + (size_t)h * q.W, w_ok && (unsigned)h < (unsigned)q.H);
       }
 #pragma unroll
       for (int u = 0; u < KH; ++u) dst[u] = v[u];
@@ -122,7 +138,8 @@ struct StripParams {
 };
 
 constexpr int kStripThreads = 256;
-constexpr int kStripUnroll = 4;      // items per thread whose loads are issued before the first store
+// items per thread whose loads are issued before the first store: fewer for tall kernels (registers)
+__host__ __device__ constexpr int strip_unroll(int kh, int es) { return (4 / es) * kh > 10 ? 2 : 4; }
 
 template <typename E, int KH>
 __global__ void __launch_bounds__(kStripThreads)
@@ -130,7 +147,7 @@ transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParam
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int ES = (int)sizeof(E);
   constexpr int CPL = 4 / ES;                     // columns per item: one 32-bit word per kernel row
-  constexpr int U = kStripUnroll;
+  constexpr int U = strip_unroll(KH, ES);
 
   const int64_t s0 = (int64_t)blockIdx.x * q.strips_per_cta;
   const int64_t left = q.total_strips - s0;
@@ -169,8 +186,7 @@ transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParam
 #pragma unroll
           for (int u = 0; u < KH; ++u) {
             const int h = h0 + u;
-            v[j][c][u] = 0;
-            if (w_ok && (unsigned)h < (unsigned)q.H) v[j][c][u] = __ldg(src + h * q.W + w);
+            v[j][c][u] = ld_if(src + h * q.W + w, w_ok && (unsigned)h < (unsigned)q.H);
           }
         }
       }
@@ -249,7 +265,8 @@ bool plan_strips(const Geometry& g, StripParams* q, size_t* smem_bytes) {
   q->total_strips = total_strips;
   q->strips_per_cta = r;
   const int items = (g.Wp + (4 / ES) - 1) / (4 / ES);
-  const int per_group = (items + kStripUnroll - 1) / kStripUnroll;
+  const int unroll = strip_unroll(g.Kh, ES);
+  const int per_group = (items + unroll - 1) / unroll;
   int grp = 1;
   while (grp < kStripThreads && grp < per_group) grp *= 2;
   q->group = grp;
@@ -274,7 +291,9 @@ cudaError_t launch_strips(const void* x, void* window, const StripParams& q, siz
   switch (Kh) {
     case 1: return run(transform_strips_kernel<E, 1>);
     case 3: return run(transform_strips_kernel<E, 3>);
-    default: return run(transform_strips_kernel<E, 5>);
+    case 5: return run(transform_strips_kernel<E, 5>);
+    case 7: return run(transform_strips_kernel<E, 7>);
+    default: return run(transform_strips_kernel<E, 11>);
   }
 }
 
