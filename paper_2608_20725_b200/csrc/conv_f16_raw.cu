@@ -61,7 +61,6 @@ struct RawParams {
   int32_t a_stage_bytes;    // rows * 128
   int32_t rs, sa, sb;       // ring depths
   int32_t ntm, nwork;       // position tiles; work items = position tiles x channel tiles
-  int32_t dbg_skip_b;       // experiment switch: do not load filter tiles (timing only, wrong results)
 };
 
 constexpr int BOXW = 128;   // halves per box row
@@ -273,12 +272,8 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
           if (!ok) break;
           const uint32_t bar = b_full0 + 8 * st;
           if (leader) {
-            if (q.dbg_skip_b) {
-              mbar_arrive(bar);
-            } else {
-              mbar_arrive_expect_tx(bar, B_STAGE_BYTES);
-              tma_load_3d(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0, v, bar);
-            }
+            mbar_arrive_expect_tx(bar, B_STAGE_BYTES);
+            tma_load_3d(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0, v, bar);
           }
           __syncwarp();
           if (++st == q.sb) { st = 0; ph ^= 1u; }
@@ -459,9 +454,7 @@ bool choose_rings(int bn, const RawPlan& plan, int* rs, int* sa, int* sb, int* s
   const int budget = (bn <= 128 ? kSmemMax / 2 : kSmemMax) - 1024 - 4096;
   const int fixed = (int)plan.K2p * 4;
   const int a = plan.a_stage_bytes, r = plan.raw_stage_bytes, b = bn * KB * 2;
-  const char* fr = getenv("IM2WIN_DBG_RS");
-  const int rr0 = fr ? atoi(fr) : 3;
-  for (int rr = rr0; rr >= 2; --rr)
+  for (int rr = 3; rr >= 2; --rr)
     for (int bb = 4; bb >= 2; --bb)
       if (2 * a + rr * r + bb * b + fixed <= budget && (bb >= 3 || rr == 2)) {
         *rs = rr; *sa = 2; *sb = bb;
@@ -587,7 +580,6 @@ cudaError_t launch_conv_f16_raw(const uint16_t* window, float* y, void* scratch,
   q.rows = plan.rows; q.nslot = plan.nslot; q.box_bytes = (plan.nslot + 1) * 256;
   q.raw_stage_bytes = plan.raw_stage_bytes; q.a_stage_bytes = plan.a_stage_bytes;
   q.rs = q.sa = q.sb = 2;
-  q.dbg_skip_b = getenv("IM2WIN_DBG_SKIP_B") ? 1 : 0;
   if (bn == 64) return launch_bn<64>(fmap, wmap, q, plan, g.Co, stream);
   if (bn == 128) return launch_bn<128>(fmap, wmap, q, plan, g.Co, stream);
   return launch_bn<256>(fmap, wmap, q, plan, g.Co, stream);
