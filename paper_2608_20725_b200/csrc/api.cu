@@ -61,6 +61,7 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
   }
   l->f16_shift = false;
   l->f16_raw = false;
+  l->f16_mat = false;
   l->koff_off = kStatusBytes;
   l->filter_off = (size_t)round_up((int64_t)l->koff_off + 4 * l->Kp, 256);
   int64_t fbytes = l->Kp * l->Co_pad * (dtype == IM2WIN_F32 ? 4 : 2);
@@ -82,6 +83,15 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
         l->f16_raw = plan_f16_raw(g).eligible && !(force && strcmp(force, "shift") == 0);
       }
       if (shift_total > l->total) l->total = shift_total;
+    }
+    const MatPlan mat = plan_f16_mat(g);
+    if (mat.eligible) {
+      const char* force = getenv("IM2WIN_F16_KERNEL");
+      // measured: the matrix-transpose kernel wins for strided layers (the others stage such
+      // layers with 2-byte gathers); IM2WIN_F16_KERNEL=mat forces it everywhere (a testing aid)
+      l->f16_mat = force ? strcmp(force, "mat") == 0 : g.s > 1;
+      const size_t mat_total = (size_t)round_up((int64_t)mat.scratch_bytes, 256);
+      if (mat_total > l->total) l->total = mat_total;
     }
   }
   return IM2WIN_OK;
@@ -109,7 +119,10 @@ static im2win_status conv_common(const void* window, const void* filter, float* 
     if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
     e = launch_conv_f32(static_cast<const float*>(window), y, scratch, g, l, stream);
   } else {
-    if (l.f16_raw) {
+    if (l.f16_mat) {
+      e = launch_conv_f16_mat(static_cast<const uint16_t*>(window), static_cast<const uint16_t*>(filter), y, scratch,
+                              g, stream);
+    } else if (l.f16_raw) {
       e = launch_pack_f16_raw(static_cast<const uint16_t*>(filter), scratch, g, l, plan_f16_raw(g), stream);
       if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
       e = launch_conv_f16_raw(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);

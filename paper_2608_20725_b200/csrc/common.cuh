@@ -36,6 +36,7 @@ struct ScratchLayout {
   size_t koff_off, filter_off, total;
   bool f16_shift;        // fp16 only: a shifted-view kernel (and its filter layout) is used
   bool f16_raw;          // fp16 only: the bulk-copy variant of the shifted-view kernel is used
+  bool f16_mat;          // fp16 only: the matrix-transpose variant is used (own scratch layout)
 };
 
 // Tile geometry of the fp16 shifted-view kernel for one layer (see conv_f16_shift.cu).
@@ -59,6 +60,15 @@ struct RawPlan {
 };
 RawPlan plan_f16_raw(const Geometry& g);
 
+// Tile geometry of the matrix-transpose shifted-view kernel (see conv_f16_mat.cu).
+struct MatPlan {
+  bool eligible;
+  int32_t Wq, rows, R, Cp8, nch_last, nplanes, box_bytes, raw_stage_bytes, a_stage_bytes, num_kb;
+  int64_t K2p, VQ;
+  size_t scratch_bytes;  // status block + packed filter
+};
+MatPlan plan_f16_mat(const Geometry& g);
+
 constexpr int kStatusBytes = 256;
 constexpr int kF32KBlock = 16;     // k-block of the fp32 kernel
 constexpr int kF16KBlock = 64;     // k-block of the fp16 kernel (64 halves = one 128-byte swizzle row)
@@ -81,6 +91,9 @@ cudaError_t launch_pack_f16_raw(const uint16_t* filter, void* scratch, const Geo
                                 const ScratchLayout& l, const RawPlan& plan, cudaStream_t stream);
 cudaError_t launch_conv_f16_raw(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                 const ScratchLayout& l, cudaStream_t stream);
+// Packs the filter into `scratch` and runs the matrix-transpose kernel.
+cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, float* y, void* scratch,
+                                const Geometry& g, cudaStream_t stream);
 cudaError_t launch_conv_f16_gather(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                    const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratch, const Geometry& g,

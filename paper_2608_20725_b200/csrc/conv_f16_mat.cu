@@ -1,0 +1,660 @@
+// fp16-input / fp32-accumulate im2win convolution on the sm_100a tensor cores:
+// shifted-view kernel whose S tile is built by 8x8 matrix transposes.
+//
+// GEMM formulation (paper Algorithm 1, M x N x K = positions x Co x C*Kh*Kw): as in
+// conv_f16_shift.cu every im2win column is staged once, S[row = virtual column][k2 = (c, u)],
+// and the Kw kernel columns are Kw MMA groups against row-shifted views of that tile.
+//
+// What is new here is how S is built.  The shared-memory data pipe is the bottleneck of this
+// kernel family (tensor-core operand reads, TMA writes and the producers' own loads/stores all
+// go through it), so the re-layout from "channel planes of the window tensor" to "rows of S"
+// must cost as few shared-memory wavefronts as possible:
+//
+//   * k order: k2 = (oct*Kh + u)*8 + e with channel c = 8*oct + e.  One 16-byte unit of an S
+//     row then holds the 8 channels of an octet at one (column, u): an 8-vector ACROSS channel
+//     planes, i.e. one row of a transposed 8x8 block of the raw data.
+//   * raw stage: tiled TMA boxes [8*noct planes][136 halves] of the window tensor viewed as
+//     [N][C][Ho*Kh*Wp]; boxes of a segment start 128 halves apart (the last 8 halves of a box
+//     row only make the row pitch 272 bytes, which spreads the 8 planes of an octet over all
+//     bank groups).  Channels beyond C are filled with zeros by the copy engine.
+//   * re-layout: ONE ldmatrix.x4.trans (8 planes x 32 halves) and ONE stmatrix.x4 per 512
+//     bytes: every lane computes one source address and one destination address, no data
+//     shuffling in registers.
+//   * S stage without swizzle: S[sub-tile][unit 0..7][row] 16 bytes each, so the address is
+//     linear in the row and a view shifted by r rows starts 16*r bytes further (the MMA's
+//     "no swizzle" K-major layout with 128 bytes between 8-row groups).  The rows per unit
+//     plane, R, are chosen with R*Kh = 1 (mod 8) when Kh is odd, which makes the 8 destination
+//     rows of one stmatrix matrix fall into 8 different bank groups.
+//
+// Any stride s with Wp mod s = 0 (columns are de-interleaved into s sub-tiles as in
+// conv_f16_shift.cu); the plane pitch of the window tensor must be a multiple of 16 bytes.
+// Persistent CTAs, double-buffered accumulator in tensor memory, bounded mbarrier waits.
+#include <cuda.h>
+#include <stdlib.h>
+
+#include "common.cuh"
+#include "ptx_sm100.cuh"
+
+namespace im2win {
+namespace {
+
+using namespace ptx;
+
+constexpr int TILE_M = 128;
+constexpr int KB = kF16KBlock;                       // 64 halves = 8 units per k-block
+constexpr int REPACK_WARPS = 8;
+constexpr int WARP_TMA = 8, WARP_MMA = 9, WARP_RAW = 10, WARP_EPI0 = 12;   // warp 11 idles
+constexpr int NUM_WARPS = 16;
+constexpr int NUM_THREADS = NUM_WARPS * 32;
+constexpr int MAX_STAGES = 6;
+constexpr int SEG_MAX = 4;                           // images one tile may touch
+constexpr int BOXW = 136;                            // halves per box row (272-byte pitch)
+constexpr int BOXSTEP = 128;                         // halves of a box row that are used
+constexpr int BATCH = 4;                             // re-layout tasks in flight per warp
+constexpr int MAX_KB = 1024;                         // k-blocks (table in shared memory)
+
+struct MatParams {
+  float* __restrict__ y;
+  uint32_t* status;
+  int64_t VQ;
+  int32_t C, N, Wq, Ho, Wo, HoWo, Co, Kh, Kw, s, num_kb;
+  int32_t rows;             // virtual positions staged per tile: 128 + (Kw-1)/s
+  int32_t R;                // rows per unit plane of an S sub-tile
+  int32_t Cp8;              // channel octets
+  int32_t nch_last;         // units of the last k-block (1..8)
+  int32_t nplanes;          // planes per box
+  int32_t box_bytes;        // nplanes * 272
+  int32_t raw_stage_bytes;  // maxbox * box_bytes
+  int32_t a_stage_bytes;    // s * 8 * R * 16, rounded up to 128
+  uint32_t magic_kh, magic_s;   // floor(e / d) = (e * magic) >> 16 for e < 8192
+  int32_t rs, sa, sb;       // ring depths
+  int32_t ntm, nwork;       // position tiles; work items = position tiles x channel tiles
+};
+
+struct Segment {            // the part of a tile that lies in one image
+  int32_t n;                // image
+  int32_t x0;               // first box column: the segment's first element rounded down to 8
+  int32_t o0;               // offset of the segment's first element from x0 (0..7)
+  int32_t row0;             // first S row of the segment
+  int32_t elems;            // elements of one channel the segment covers: cnt * s * Kh
+  int32_t box0, nbox;       // boxes [box0, box0 + nbox) of the raw stage belong to this segment
+  int32_t pad_;
+};
+
+// Splits the rows of the tile starting at virtual position q0 by image: within an image the
+// columns of one channel are contiguous in the window tensor.  Returns the number of segments
+// and, in *total_boxes, the boxes of one raw stage.
+__device__ __forceinline__ int split_by_image(const MatParams& q, int64_t q0, Segment* segs, int* total_boxes) {
+  const int64_t img_rows = (int64_t)q.Ho * q.Wq;
+  int64_t n = q0 / img_rows, a = q0 - n * img_rows;
+  int remaining = q.rows, row0 = 0, box0 = 0, g = 0;
+  const int per_row = q.s * q.Kh;
+  while (remaining > 0 && n < q.N && g < SEG_MAX) {
+    const int cnt = (int)(remaining < img_rows - a ? remaining : img_rows - a);
+    const int f0 = (int)(a * per_row);                     // element offset inside the channel plane
+    const int span = (f0 & 7) + cnt * per_row;
+    segs[g].n = (int)n;
+    segs[g].x0 = f0 & ~7;
+    segs[g].o0 = f0 & 7;
+    segs[g].row0 = row0;
+    segs[g].elems = cnt * per_row;
+    segs[g].box0 = box0;
+    segs[g].nbox = (span + BOXSTEP - 1) / BOXSTEP;
+    box0 += segs[g].nbox;
+    row0 += cnt;
+    remaining -= cnt;
+    a = 0;
+    ++n;
+    ++g;
+  }
+  *total_boxes = box0;
+  return g;
+}
+
+template <int BN>
+__global__ void __launch_bounds__(NUM_THREADS, (BN <= 128 ? 2 : 1))
+conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_constant__ CUtensorMap wmap, MatParams q) {
+  constexpr int B_STAGE_BYTES = BN * KB * 2;
+
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+  __shared__ __align__(8) uint64_t bars[6 * MAX_STAGES + 4];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ volatile uint32_t abort_flag;
+  __shared__ Segment seg_s[NUM_WARPS][SEG_MAX];     // each warp keeps its own copy of the tile's segments
+  __shared__ __align__(16) unsigned char trash[512];   // destination of matrix rows that belong to no S unit
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  // shared-memory map: filter ring (1024-byte aligned stages) | S ring | raw ring | k-block table
+  const uint32_t b_ring = smem_u32(smem);
+  const uint32_t a_ring = b_ring + q.sb * B_STAGE_BYTES;
+  const uint32_t raw_ring = a_ring + q.sa * q.a_stage_bytes;
+  uint32_t* kbinfo = reinterpret_cast<uint32_t*>(smem + q.sb * B_STAGE_BYTES + q.sa * q.a_stage_bytes +
+                                                 q.rs * q.raw_stage_bytes);
+  const uint32_t a_full0 = smem_u32(&bars[0]);
+  const uint32_t a_empty0 = smem_u32(&bars[MAX_STAGES]);
+  const uint32_t b_full0 = smem_u32(&bars[2 * MAX_STAGES]);
+  const uint32_t b_empty0 = smem_u32(&bars[3 * MAX_STAGES]);
+  const uint32_t r_full0 = smem_u32(&bars[4 * MAX_STAGES]);
+  const uint32_t r_empty0 = smem_u32(&bars[5 * MAX_STAGES]);
+  const uint32_t acc_full0 = smem_u32(&bars[6 * MAX_STAGES]);
+  const uint32_t acc_empty0 = smem_u32(&bars[6 * MAX_STAGES + 2]);
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0u;
+    for (int i = 0; i < MAX_STAGES; ++i) {
+      mbar_init(a_full0 + 8 * i, REPACK_WARPS);
+      mbar_init(a_empty0 + 8 * i, 1);
+      mbar_init(b_full0 + 8 * i, 1);
+      mbar_init(b_empty0 + 8 * i, 1);
+      mbar_init(r_full0 + 8 * i, 1);
+      mbar_init(r_empty0 + 8 * i, REPACK_WARPS);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(acc_full0 + 8 * i, 1);
+      mbar_init(acc_empty0 + 8 * i, 4);      // the four epilogue warps
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == WARP_MMA) tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
+  // per k-block: first channel octet | octets << 16
+  for (int kb = threadIdx.x; kb < q.num_kb; kb += NUM_THREADS) {
+    const int oct_lo = (8 * kb) / q.Kh;
+    int oct_hi = (8 * kb + 7) / q.Kh;
+    if (oct_hi > q.Cp8 - 1) oct_hi = q.Cp8 - 1;
+    kbinfo[kb] = (uint32_t)oct_lo | ((uint32_t)(oct_hi - oct_lo + 1) << 16);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_acc = tmem_base_slot;
+  Segment* segs = seg_s[warp];
+
+  if (warp < REPACK_WARPS) {
+    // ---------------- re-layout: raw stage -> S stage ---------------------------
+    // task = (box, octet of the k-block, group of 32 halves); warp w takes tasks w, w + 8, ...
+    bool ok = true;
+    int st = 0, rst = 0;
+    uint32_t ph = 0, rph = 0;
+    const uint32_t trash_l = smem_u32(trash) + (lane >> 3) * 128;
+    const uint32_t src_l = (uint32_t)(((lane & 7) * BOXW + (warp & 3) * 32 + (lane >> 3) * 8) * 2);
+    const int m_l = (warp & 3) * 32 + lane;       // lane's matrix row = element m of the box row
+    TIMER_DECL;
+    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
+      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+      int nseg = 0, total_boxes = 0;
+      if (lane == 0) nseg = split_by_image(q, q0, segs, &total_boxes);
+      nseg = __shfl_sync(0xffffffffu, nseg, 0);
+      total_boxes = __shfl_sync(0xffffffffu, total_boxes, 0);
+      __syncwarp();
+      const int s0_o0 = segs[0].o0, s0_elems = segs[0].elems, s0_nbox = segs[0].nbox;
+      if (threadIdx.x == 0) TIMER_LAP(0);       // per-tile setup
+      for (int kb = 0; kb < q.num_kb; ++kb) {
+        if (lane == 0) {
+          ok = mbar_wait(r_full0 + 8 * rst, rph, &abort_flag, q.status);
+          if (threadIdx.x == 0) TIMER_LAP(1);   // wait for the raw stage
+          if (ok) ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+          if (threadIdx.x == 0) TIMER_LAP(2);   // wait for a free S stage
+        }
+        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        if (!ok) break;
+        const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
+        const uint32_t raw_stage = raw_ring + rst * q.raw_stage_bytes;
+        const uint32_t info = kbinfo[kb];
+        const int oct_lo = (int)(info & 0xffffu), noct = (int)(info >> 16);
+        const int nch = kb == q.num_kb - 1 ? q.nch_last : 8;
+        const int unit0 = oct_lo * q.Kh - kb * 8;       // S unit of (first octet, u = 0); may be negative
+        int o = warp >> 2, b = 0;
+        while (o >= noct) { o -= noct; ++b; }
+        // the current segment lives in registers; it changes at most SEG_MAX - 1 times per stage
+        int g = 0, seg_o0 = s0_o0, seg_row0 = 0, seg_elems = s0_elems, seg_box0 = 0, seg_end = s0_nbox;
+        while (b < total_boxes) {
+          // BATCH tasks at a time: all matrix loads first, then the stores, so that the loads'
+          // latencies overlap
+          uint32_t r[BATCH][4], dst[BATCH];
+          int cnt = 0;
+#pragma unroll
+          for (int k = 0; k < BATCH; ++k) {
+            if (b < total_boxes) {
+              while (b >= seg_end) {
+                ++g;
+                seg_o0 = segs[g].o0; seg_row0 = segs[g].row0; seg_elems = segs[g].elems;
+                seg_box0 = segs[g].box0; seg_end = seg_box0 + segs[g].nbox;
+              }
+              ldmatrix_x4_trans(raw_stage + (uint32_t)(b * q.box_bytes + o * (8 * BOXW * 2)) + src_l, r[k]);
+              const int e = (b - seg_box0) * BOXSTEP + m_l - seg_o0;      // element of the segment
+              const int ubase = unit0 + o * q.Kh;
+              // rows that belong to no S unit go to a scratch line, into the bank group the real
+              // destination would have had (R*e + const mod 8 when R*Kh = 1 mod 8), so that the 8
+              // rows of a matrix never collide
+              dst[k] = trash_l + (uint32_t)(((q.R * e + ubase * q.R + seg_row0) & 7) << 4);
+              if ((unsigned)e < (unsigned)seg_elems) {
+                const int col = (int)(((uint32_t)e * q.magic_kh) >> 16);
+                const int u = e - col * q.Kh;
+                const int unit = ubase + u;
+                if ((unsigned)unit < (unsigned)nch) {
+                  const int vr = (int)(((uint32_t)col * q.magic_s) >> 16);
+                  const int sub = col - vr * q.s;
+                  dst[k] = a_stage + (uint32_t)((((sub << 3) + unit) * q.R + seg_row0 + vr) << 4);
+                }
+              }
+              o += 2;
+              while (o >= noct) { o -= noct; ++b; }
+              cnt = k + 1;
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < BATCH; ++k)
+            if (k < cnt) stmatrix_x4(dst[k], r[k]);
+        }
+        if ((nch & 1) && kb == q.num_kb - 1) {
+          // odd number of units: the last k step reads one more unit; make it zeros
+          for (int sub = 0; sub < q.s; ++sub)
+            for (int i = threadIdx.x; i < q.R; i += REPACK_WARPS * 32)
+              asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(
+                               a_stage + (uint32_t)((((sub << 3) + nch) * q.R + i) << 4)),
+                           "r"(0u)
+                           : "memory");
+        }
+        if (threadIdx.x == 0) TIMER_LAP(3);     // re-layout
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(a_full0 + 8 * st);
+          mbar_arrive(r_empty0 + 8 * rst);
+        }
+        if (threadIdx.x == 0) TIMER_LAP(4);     // fence + arrive
+        if (++st == q.sa) { st = 0; ph ^= 1u; }
+        if (++rst == q.rs) { rst = 0; rph ^= 1u; }
+      }
+    }
+    if (threadIdx.x == 0) TIMER_FLUSH();
+  } else if (warp == WARP_TMA) {
+    // ---------------- TMA loader of the filter tiles ---------------------------
+    const bool leader = elect_one();
+    bool ok = true;
+    int st = 0;
+    uint32_t ph = 0;
+    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
+      const int n0 = (w / q.ntm) * BN;
+      for (int kb = 0; kb < q.num_kb && ok; ++kb) {
+        for (int v = 0; v < q.Kw; ++v) {
+          ok = mbar_wait(b_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          const uint32_t bar = b_full0 + 8 * st;
+          if (leader) {
+            mbar_arrive_expect_tx(bar, B_STAGE_BYTES);
+            tma_load_3d(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0, v, bar);
+          }
+          __syncwarp();
+          if (++st == q.sb) { st = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == WARP_MMA) {
+    // ---------------- MMA issuer ------------------------------------------------
+    constexpr uint32_t idesc = instr_desc_f16(TILE_M, BN);
+    const bool leader = elect_one();
+    bool ok = true;
+    int sta = 0, stb = 0;
+    uint32_t pha = 0, phb = 0;
+    uint32_t it = 0;                             // work items done by this CTA: accumulator buffer = it & 1
+    const uint32_t a_lo0 = smem_desc_lo_noswz(a_ring, (uint32_t)q.R * 16u), b_lo0 = smem_desc_lo(b_ring);
+    const uint32_t sub_units = 8u * (uint32_t)q.R;       // 16-byte units per sub-tile
+    const uint32_t kstep_units = 2u * (uint32_t)q.R;     // 16-byte units per 16-element k step
+    const int ks_last = (q.nch_last + 1) >> 1;
+    TIMER_DECL;
+    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
+      const uint32_t buf = it & 1u;
+      TIMER_LAP(8);
+      ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      TIMER_LAP(11);                             // MMA warp: wait for a free accumulator
+      tc_fence_after();
+      const uint32_t acc = tmem_acc + buf * (uint32_t)BN;
+      uint32_t first = 0;
+      for (int kb = 0; kb < q.num_kb && ok; ++kb) {
+        TIMER_LAP(8);
+        ok = mbar_wait(a_full0 + 8 * sta, pha, &abort_flag, q.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        TIMER_LAP(9);                            // MMA warp: wait for an S stage
+        const uint32_t a_lo_stage = a_lo0 + (uint32_t)(sta * (q.a_stage_bytes >> 4));
+        const int nks = kb == q.num_kb - 1 ? ks_last : KB / 16;
+        uint32_t sub = 0, shift = 0;             // kernel column v reads sub-tile v mod s from row v div s on
+        for (int v = 0; v < q.Kw; ++v) {
+          TIMER_LAP(8);
+          ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          TIMER_LAP(10);                         // MMA warp: wait for a filter stage
+          tc_fence_after();
+          const uint32_t b_lo = b_lo0 + (uint32_t)(stb * (B_STAGE_BYTES >> 4));
+          const uint32_t a_lo = a_lo_stage + sub * sub_units + shift;
+          if (leader) {
+#pragma unroll 1
+            for (int j = 0; j < nks; ++j)
+              umma_f16_ab(acc, a_lo + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j, kSmemDescHiSw128,
+                          idesc, first | (uint32_t)j);
+            umma_commit(b_empty0 + 8 * stb);
+          }
+          __syncwarp();
+          first = 1u;
+          if (++sub == (uint32_t)q.s) { sub = 0; ++shift; }
+          if (++stb == q.sb) { stb = 0; phb ^= 1u; }
+        }
+        if (ok && leader) umma_commit(a_empty0 + 8 * sta);
+        __syncwarp();
+        if (++sta == q.sa) { sta = 0; pha ^= 1u; }
+      }
+      if (ok && leader) umma_commit(acc_full0 + 8 * buf);
+      __syncwarp();
+    }
+    if (leader) { TIMER_LAP(8); TIMER_FLUSH(); }
+  } else if (warp == WARP_RAW) {
+    // ---------------- raw loader: tiled TMA loads of the channel planes ----------
+    const bool leader = elect_one();
+    bool ok = true;
+    int rst = 0;
+    uint32_t rph = 0;
+    TIMER_DECL;
+    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
+      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+      int nseg = 0, total_boxes = 0;
+      if (lane == 0) nseg = split_by_image(q, q0, segs, &total_boxes);
+      nseg = __shfl_sync(0xffffffffu, nseg, 0);
+      total_boxes = __shfl_sync(0xffffffffu, total_boxes, 0);
+      __syncwarp();
+      for (int kb = 0; kb < q.num_kb && ok; ++kb) {
+        if (leader) TIMER_LAP(6);              // raw loader: issuing copies
+        ok = mbar_wait(r_empty0 + 8 * rst, rph ^ 1u, &abort_flag, q.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (leader) TIMER_LAP(5);              // raw loader: wait for a free raw stage
+        const uint32_t bar = r_full0 + 8 * rst;
+        const int c_lo = (int)(kbinfo[kb] & 0xffffu) * 8;
+        const uint32_t stage = raw_ring + rst * q.raw_stage_bytes;
+        if (leader) {
+          mbar_arrive_expect_tx(bar, (uint32_t)(total_boxes * q.box_bytes));
+          for (int g = 0; g < nseg; ++g)
+            for (int j = 0; j < segs[g].nbox; ++j)
+              tma_load_3d(stage + (segs[g].box0 + j) * q.box_bytes, &wmap, segs[g].x0 + j * BOXSTEP, c_lo, segs[g].n,
+                          bar);
+        }
+        __syncwarp();
+        if (++rst == q.rs) { rst = 0; rph ^= 1u; }
+      }
+    }
+    if (leader) { TIMER_LAP(6); TIMER_FLUSH(); }
+  } else if (warp >= WARP_EPI0) {
+    // ---------------- epilogue: tensor memory -> NCHW output --------------------
+    const int lq = warp & 3;                     // tensor-memory lane quadrant this warp may read
+    bool ok = true;
+    uint32_t it = 0;
+    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
+      const uint32_t buf = it & 1u;
+      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+      const int n0 = (w / q.ntm) * BN;
+      const int64_t vq = q0 + lq * 32 + lane;    // accumulator row = virtual position
+      bool valid = false;
+      float* yrow = q.y;
+      if (vq < q.VQ) {
+        const int64_t sg = vq / q.Wq;
+        const int kq = (int)(vq - sg * q.Wq);
+        const int64_t n = sg / q.Ho;
+        const int ho = (int)(sg - n * q.Ho);
+        valid = kq < q.Wo;                       // trailing columns of a strip are no output
+        yrow += (n * q.Co) * q.HoWo + ho * q.Wo + kq;
+      }
+      if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        if (n0 + c0 >= q.Co) break;
+        uint32_t v[32];
+        tmem_ld32(lane_base + (uint32_t)c0, v);
+        if (valid) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int co = n0 + c0 + j;
+            if (co < q.Co) yrow[(int64_t)co * q.HoWo] = __uint_as_float(v[j]);
+          }
+        }
+      }
+      // the buffer may be overwritten once all four warps have read it
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty0 + 8 * buf);
+    }
+  }
+
+  // ---------------- teardown ---------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == WARP_MMA) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_acc, 2 * BN);
+  }
+}
+
+// Filter pack for this kernel: Fp3[v][co][k2p], k2 = (oct*Kh + u)*8 + e, c = 8*oct + e
+// (paper Section "Im2win Convolution": height before width; here additionally grouped by
+// channel octets).  Padded k2 (c >= C or beyond the last unit) hold zeros.  Block (0,0,0)
+// also clears the status block.
+__global__ void pack_f16_mat_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, uint32_t* status,
+                                    int C, int Co, int Kh, int Kw, int K2p) {
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
+  for (int v = blockIdx.z; v < Kw; v += gridDim.z)
+    for (int co = blockIdx.y; co < Co; co += gridDim.y)
+      for (int k2 = blockIdx.x * blockDim.x + threadIdx.x; k2 < K2p; k2 += gridDim.x * blockDim.x) {
+        const int unit = k2 >> 3, e = k2 & 7;
+        const int oct = unit / Kh, u = unit - oct * Kh;
+        const int c = oct * 8 + e;
+        uint16_t val = 0;
+        if (c < C) val = f[(((size_t)co * C + c) * Kh + u) * Kw + v];
+        fp[((size_t)v * Co + co) * K2p + k2] = val;
+      }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+constexpr int kSmemMax = 227 * 1024;
+
+int tile_bn(const Geometry& g) { return g.Co <= 64 ? 64 : (g.Co <= 128 ? 128 : 256); }
+
+// Ring depths that fit: S ring 2, raw ring 3 (2 if tight), filter ring as deep as fits (<= 4).
+// Narrow tiles try to fit two CTAs on an SM first.
+bool choose_rings(int bn, const MatPlan& plan, int* rs, int* sa, int* sb, int* smem_bytes) {
+  const int fixed = plan.num_kb * 4;
+  const int a = plan.a_stage_bytes, r = plan.raw_stage_bytes, b = bn * KB * 2;
+  for (int half = (bn <= 128 ? 1 : 0); half >= 0; --half) {
+    // dynamic shared memory left after the alignment slack, the static part (barriers, segment
+    // copies) and, for two CTAs per SM, the 1 KB the runtime reserves per CTA
+    const int budget = (half ? kSmemMax / 2 : kSmemMax) - 1024 - 4096;
+    for (int rr = 3; rr >= 2; --rr)
+      for (int bb = 4; bb >= 2; --bb)
+        if (2 * a + rr * r + bb * b + fixed <= budget && (bb >= 3 || rr == 2)) {
+          *rs = rr; *sa = 2; *sb = bb;
+          *smem_bytes = 2 * a + rr * r + bb * b + fixed + 1024;
+          return true;
+        }
+  }
+  return false;
+}
+
+template <int BN>
+cudaError_t launch_bn(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParams q, const MatPlan& plan, int co,
+                      cudaStream_t stream) {
+  int smem_bytes = 0;
+  if (!choose_rings(BN, plan, &q.rs, &q.sa, &q.sb, &smem_bytes)) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(conv_f16_mat_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  if (e != cudaSuccess) return e;
+  const int64_t ntm = (plan.VQ + TILE_M - 1) / TILE_M;
+  const int64_t nwork = ntm * ((co + BN - 1) / BN);
+  if (nwork >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
+  q.ntm = (int32_t)ntm;
+  q.nwork = (int32_t)nwork;
+  const int per_sm = (BN <= 128 && smem_bytes + 1024 <= kSmemMax / 2) ? 2 : 1;
+  const int slots = 148 * per_sm;                      // persistent CTAs
+  const unsigned grid = (unsigned)(nwork < slots ? nwork : slots);
+  conv_f16_mat_kernel<BN><<<grid, NUM_THREADS, smem_bytes, stream>>>(fmap, wmap, q);
+  return cudaGetLastError();
+}
+
+uint32_t magic16(int d) { return (uint32_t)(65536 / d + 1); }
+
+}  // namespace
+
+MatPlan plan_f16_mat(const Geometry& g) {
+  MatPlan p{};
+  p.eligible = false;
+  if (g.Wp % g.s != 0) return p;
+  if ((g.chan_stride * 2) % 16 != 0) return p;            // TMA needs a plane pitch that is a multiple of 16 bytes
+  if (g.Kh > 16 || g.s > 8) return p;
+  p.Wq = g.Wp / g.s;
+  p.rows = TILE_M + (g.Kw - 1) / g.s;
+  // rows per unit plane: R*Kh = 1 (mod 8) for odd Kh (conflict-free matrix stores), odd otherwise
+  p.R = p.rows;
+  while ((g.Kh & 1) ? ((p.R * g.Kh) & 7) != 1 : (p.R & 1) == 0) ++p.R;
+  // the kernel divides by Kh and s with 16-bit reciprocals: check them over the ranges it uses
+  for (int e = 0; e < p.rows * g.s * g.Kh + 8; ++e)
+    if ((int)(((uint32_t)e * magic16(g.Kh)) >> 16) != e / g.Kh) return p;
+  for (int c = 0; c < p.rows * g.s + 8; ++c)
+    if ((int)(((uint32_t)c * magic16(g.s)) >> 16) != c / g.s) return p;
+  p.Cp8 = (g.C + 7) / 8;
+  const int64_t units = (int64_t)p.Cp8 * g.Kh;
+  p.K2p = (units * 8 + KB - 1) / KB * KB;
+  p.num_kb = (int32_t)(p.K2p / KB);
+  if (p.num_kb > MAX_KB) return p;
+  p.nch_last = (int32_t)(units - 8 * (int64_t)(p.num_kb - 1));
+  p.VQ = (int64_t)g.N * g.Ho * p.Wq;
+  const int64_t img_rows = (int64_t)g.Ho * p.Wq;
+  const int64_t segmax = (p.rows - 2) / img_rows + 2;     // images a tile can touch
+  if (segmax > SEG_MAX) return p;
+  if (g.chan_stride >= ((int64_t)1 << 31)) return p;
+  int noct = 1;
+  for (int kb = 0; kb < p.num_kb && kb < 64; ++kb) {      // the pattern repeats after Kh k-blocks
+    int hi = (8 * kb + 7) / g.Kh;
+    if (hi > p.Cp8 - 1) hi = p.Cp8 - 1;
+    const int n = hi - (8 * kb) / g.Kh + 1;
+    if (n > noct) noct = n;
+  }
+  p.nplanes = 8 * noct;
+  p.box_bytes = p.nplanes * BOXW * 2;
+  // boxes one stage can need: the exact maximum over the tile start positions (period <= img_rows tiles)
+  int maxbox = 1;
+  {
+    const int per_row = g.s * g.Kh;
+    const int64_t ntiles = (p.VQ + TILE_M - 1) / TILE_M;
+    const int64_t probe = ntiles < img_rows ? ntiles : img_rows;
+    for (int64_t t = 0; t < probe && t < 65536; ++t) {
+      int64_t a = (t * TILE_M) % img_rows;
+      int remaining = p.rows, boxes = 0;
+      while (remaining > 0) {
+        const int cnt = (int)(remaining < img_rows - a ? remaining : img_rows - a);
+        const int span = (int)((a * per_row) & 7) + cnt * per_row;
+        boxes += (span + BOXSTEP - 1) / BOXSTEP;
+        remaining -= cnt;
+        a = 0;
+      }
+      if (boxes > maxbox) maxbox = boxes;
+    }
+    if (probe > 65536) maxbox += (int)segmax;   // unprobed phases: leave room for one more box per image
+  }
+  p.raw_stage_bytes = maxbox * p.box_bytes;
+  p.a_stage_bytes = (g.s * 8 * p.R * 16 + 127) / 128 * 128;
+  if ((p.VQ + TILE_M - 1) / TILE_M * ((g.Co + 63) / 64) >= ((int64_t)1 << 31)) return p;
+  p.scratch_bytes = (size_t)kStatusBytes + (size_t)p.K2p * g.Co * g.Kw * 2;
+  int rs, sa, sb, smem;
+  if (!choose_rings(tile_bn(g), p, &rs, &sa, &sb, &smem)) return p;
+  p.eligible = true;
+  return p;
+}
+
+cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, float* y, void* scratch,
+                                const Geometry& g, cudaStream_t stream) {
+  const MatPlan plan = plan_f16_mat(g);
+  if (!plan.eligible) return cudaErrorInvalidValue;
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return cudaErrorNotSupported;
+  unsigned char* base = static_cast<unsigned char*>(scratch);
+  uint16_t* fp = reinterpret_cast<uint16_t*>(base + kStatusBytes);
+  const int bn = tile_bn(g);
+
+  {
+    const unsigned gx = (unsigned)((plan.K2p + 255) / 256);
+    dim3 grid(gx > 64 ? 64 : gx, (unsigned)(g.Co < 32768 ? g.Co : 32768), (unsigned)(g.Kw < 65535 ? g.Kw : 65535));
+    pack_f16_mat_kernel<<<grid, 256, 0, stream>>>(filter, fp, reinterpret_cast<uint32_t*>(base), g.C, g.Co, g.Kh, g.Kw,
+                                                  (int)plan.K2p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+
+  // Filter as Fp3[v][co][k2p] halves: a 3-D tensor (k2 fastest), one box = 64 k2 x BN channels of one v.
+  CUtensorMap fmap;
+  const cuuint64_t dims[3] = {(cuuint64_t)plan.K2p, (cuuint64_t)g.Co, (cuuint64_t)g.Kw};
+  const cuuint64_t strides[2] = {(cuuint64_t)plan.K2p * 2, (cuuint64_t)plan.K2p * 2 * (cuuint64_t)g.Co};
+  const cuuint32_t box[3] = {(cuuint32_t)KB, (cuuint32_t)bn, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult cr = encode(&fmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, fp, dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+
+  // Window tensor as [N][C][chan_stride halves]; one box = 136 halves of nplanes channel planes of one image.
+  CUtensorMap wmap;
+  {
+    const cuuint64_t wd[3] = {(cuuint64_t)g.chan_stride, (cuuint64_t)g.C, (cuuint64_t)g.N};
+    const cuuint64_t ws[2] = {(cuuint64_t)g.chan_stride * 2, (cuuint64_t)g.img_stride * 2};
+    const cuuint32_t wb[3] = {(cuuint32_t)BOXW, (cuuint32_t)plan.nplanes, 1};
+    const cuuint32_t we[3] = {1, 1, 1};
+    cr = encode(&wmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<uint16_t*>(window), wd, ws, wb, we,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
+
+  MatParams q;
+  q.y = y;
+  q.status = reinterpret_cast<uint32_t*>(base);
+  q.VQ = plan.VQ;
+  q.C = g.C; q.N = g.N; q.Wq = plan.Wq; q.Ho = g.Ho; q.Wo = g.Wo; q.HoWo = g.Ho * g.Wo; q.Co = g.Co;
+  q.Kh = g.Kh; q.Kw = g.Kw; q.s = g.s; q.num_kb = plan.num_kb;
+  q.rows = plan.rows; q.R = plan.R; q.Cp8 = plan.Cp8; q.nch_last = plan.nch_last;
+  q.nplanes = plan.nplanes; q.box_bytes = plan.box_bytes;
+  q.raw_stage_bytes = plan.raw_stage_bytes; q.a_stage_bytes = plan.a_stage_bytes;
+  q.magic_kh = magic16(g.Kh); q.magic_s = magic16(g.s);
+  q.rs = q.sa = q.sb = 2;
+  q.ntm = q.nwork = 0;
+  if (bn == 64) return launch_bn<64>(fmap, wmap, q, plan, g.Co, stream);
+  if (bn == 128) return launch_bn<128>(fmap, wmap, q, plan, g.Co, stream);
+  return launch_bn<256>(fmap, wmap, q, plan, g.Co, stream);
+}
+
+}  // namespace im2win

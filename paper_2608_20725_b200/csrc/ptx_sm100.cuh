@@ -180,6 +180,44 @@ __device__ __forceinline__ void umma_f16_lohi(uint32_t tmem_d, uint32_t a_lo, ui
       : "memory");
 }
 
+// K-major tile WITHOUT swizzle: 16-byte units (8 halves of one row) are the atoms; the 8 rows of
+// a group lie 16 bytes apart, groups of 8 rows `sbo` bytes apart and the two 8-element halves of
+// a 16-element k step `lbo` bytes apart.  With sbo = 128 the address is linear in the row, so a
+// view may start at any row (16 bytes per row).  Low half: start address and lbo; high half: sbo.
+__device__ __forceinline__ uint32_t smem_desc_lo_noswz(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr & 0x3ffffu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+constexpr uint32_t kSmemDescHiNoSwz128 = (uint32_t)(128 >> 4) | (1u << 14);
+// MMA with separately described operands (A without swizzle, B with the 128-byte swizzle).
+__device__ __forceinline__ void umma_f16_ab(uint32_t tmem_d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                            uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(tmem_d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// Four 8x8 matrices of 16-bit elements, shared memory -> registers, transposed on the way: lane l
+// gives the address of row l%8 (16 bytes) of matrix l/8; afterwards lane i holds in r[t] the
+// elements (row 2*(i%4), column i/4) and (row 2*(i%4)+1, column i/4) of matrix t.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
+// Four 8x8 matrices registers -> shared memory: lane i holds in r[t] the elements (row i/4,
+// columns 2*(i%4), 2*(i%4)+1) of matrix t; lane l gives the address of row l%8 of matrix l/8.
+__device__ __forceinline__ void stmatrix_x4(uint32_t addr, const uint32_t (&r)[4]) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(r[0]), "r"(r[1]),
+               "r"(r[2]), "r"(r[3])
+               : "memory");
+}
+
 // Instruction descriptor: fp16 A and B, both k-major, fp32 accumulator, M x N tile.
 __host__ __device__ constexpr uint32_t instr_desc_f16(int M, int N) {
   return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);

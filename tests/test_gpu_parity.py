@@ -81,7 +81,7 @@ def test_transform_preserves_special_bit_patterns():
 
 
 @pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
-@pytest.mark.parametrize("precision", ["f32", "f16", "f16-shift", "f16-gather"])
+@pytest.mark.parametrize("precision", ["f32", "f16", "f16-shift", "f16-mat", "f16-gather"])
 def test_conv_parity_small(layer, precision):
     dims = layer.dims()
     x, f = workloads.make_inputs(layer)
@@ -92,7 +92,7 @@ def test_conv_parity_small(layer, precision):
 
 
 @pytest.mark.parametrize("layer", [SMALL[1], SMALL[2], SMALL[4], SMALL[8], SMALL[10], SMALL[12]], ids=lambda l: l.name)
-@pytest.mark.parametrize("precision", ["f32", "f16", "f16-shift", "f16-gather"])
+@pytest.mark.parametrize("precision", ["f32", "f16", "f16-shift", "f16-mat", "f16-gather"])
 def test_conv_exact_on_integer_inputs(layer, precision):
     """x in {-2..2}, filter in {-1,0,1}: every partial sum is a small integer, so any summation
     order gives the oracle's value exactly.  Separates indexing errors from rounding."""
