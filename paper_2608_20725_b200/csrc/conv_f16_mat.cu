@@ -43,14 +43,15 @@ using namespace ptx;
 constexpr int TILE_M = 128;
 constexpr int KB = kF16KBlock;                       // 64 halves = 8 units per k-block
 constexpr int REPACK_WARPS = 8;
-constexpr int WARP_TMA = 8, WARP_MMA = 9, WARP_RAW = 10, WARP_EPI0 = 12;   // warp 11 idles
+constexpr int WARP_TMA = 8, WARP_MMA = 9, WARP_RAW = 10, WARP_EPI0 = 12;   // warps 10 and 11 load raw boxes
 constexpr int NUM_WARPS = 16;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr int MAX_STAGES = 6;
 constexpr int SEG_MAX = 4;                           // images one tile may touch
 constexpr int BOXW = 136;                            // halves per box row (272-byte pitch)
 constexpr int BOXSTEP = 128;                         // halves of a box row that are used
-constexpr int BATCH = 4;                             // re-layout tasks in flight per warp
+constexpr int BATCH = 4;                             // direct path: re-layout tasks in flight per warp
+constexpr int MAXBOX = 16;                           // boxes of one raw stage (per-lane table in registers)
 constexpr int MAX_KB = 1024;                         // k-blocks (table in shared memory)
 
 struct MatParams {
@@ -84,16 +85,16 @@ struct Segment {            // the part of a tile that lies in one image
 // Splits the rows of the tile starting at virtual position q0 by image: within an image the
 // columns of one channel are contiguous in the window tensor.  Returns the number of segments
 // and, in *total_boxes, the boxes of one raw stage.
-__device__ __forceinline__ int split_by_image(const MatParams& q, int64_t q0, Segment* segs, int* total_boxes) {
-  const int64_t img_rows = (int64_t)q.Ho * q.Wq;
-  int64_t n = q0 / img_rows, a = q0 - n * img_rows;
+__device__ __forceinline__ int split_by_image(const MatParams& q, int q0, Segment* segs, int* total_boxes) {
+  const int img_rows = q.Ho * q.Wq;              // VQ < 2^31 is a condition of this kernel
+  int n = q0 / img_rows, a = q0 - n * img_rows;
   int remaining = q.rows, row0 = 0, box0 = 0, g = 0;
   const int per_row = q.s * q.Kh;
   while (remaining > 0 && n < q.N && g < SEG_MAX) {
-    const int cnt = (int)(remaining < img_rows - a ? remaining : img_rows - a);
-    const int f0 = (int)(a * per_row);                     // element offset inside the channel plane
+    const int cnt = remaining < img_rows - a ? remaining : img_rows - a;
+    const int f0 = a * per_row;                            // element offset inside the channel plane
     const int span = (f0 & 7) + cnt * per_row;
-    segs[g].n = (int)n;
+    segs[g].n = n;
     segs[g].x0 = f0 & ~7;
     segs[g].o0 = f0 & 7;
     segs[g].row0 = row0;
@@ -111,10 +112,20 @@ __device__ __forceinline__ int split_by_image(const MatParams& q, int64_t q0, Se
   return g;
 }
 
-template <int BN>
-__global__ void __launch_bounds__(NUM_THREADS, (BN <= 128 ? 2 : 1))
-conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_constant__ CUtensorMap wmap, MatParams q) {
-  constexpr int B_STAGE_BYTES = BN * KB * 2;
+// Kernel body.  PAIR = false: one CTA per work item (128 positions x BN channels).  PAIR = true:
+// two CTAs of a cluster share every MMA (M = 256: 128 positions from each CTA, N = BN): each CTA
+// stages its own S tile and HALF of the filter tile, the leader CTA (rank 0) issues the MMAs,
+// the accumulator rows of a CTA's positions land in its own tensor memory.  Per CTA that halves
+// the filter bytes written to and read from shared memory, which is what bounds the 1-CTA form.
+// Barriers the leader's MMA warp waits on live in the leader CTA and collect arrivals from both
+// CTAs; barriers signalled by MMA completion exist in both CTAs and are signalled together.
+template <int BN, bool PAIR>
+__device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const CUtensorMap& wmap, const MatParams& q) {
+  constexpr int B_ROWS = PAIR ? BN / 2 : BN;            // filter rows (output channels) this CTA stages
+  constexpr int B_STAGE_BYTES = B_ROWS * KB * 2;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const int w_first = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int w_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
@@ -144,7 +155,7 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
   if (threadIdx.x == 0) {
     abort_flag = 0u;
     for (int i = 0; i < MAX_STAGES; ++i) {
-      mbar_init(a_full0 + 8 * i, REPACK_WARPS);
+      mbar_init(a_full0 + 8 * i, PAIR ? 2 * REPACK_WARPS : REPACK_WARPS);
       mbar_init(a_empty0 + 8 * i, 1);
       mbar_init(b_full0 + 8 * i, 1);
       mbar_init(b_empty0 + 8 * i, 1);
@@ -153,11 +164,14 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(acc_full0 + 8 * i, 1);
-      mbar_init(acc_empty0 + 8 * i, 4);      // the four epilogue warps
+      mbar_init(acc_empty0 + 8 * i, PAIR ? 8 : 4);      // the four epilogue warps (of each CTA)
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == WARP_MMA) tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
+  if (warp == WARP_MMA) {
+    if (PAIR) tmem_alloc_pair(smem_u32(&tmem_base_slot), 2 * BN);
+    else tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
+  }
   // per k-block: first channel octet | octets << 16
   for (int kb = threadIdx.x; kb < q.num_kb; kb += NUM_THREADS) {
     const int oct_lo = (8 * kb) / q.Kh;
@@ -167,28 +181,65 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();               // the peer's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_acc = tmem_base_slot;
+  // where this CTA's arrivals for the MMA issuer go: the leader's barriers
+  const uint32_t a_full_dst = PAIR ? mapa_shared(a_full0, 0) : a_full0;
+  const uint32_t b_full_dst = PAIR ? mapa_shared(b_full0, 0) : b_full0;
+  const uint32_t acc_empty_dst = PAIR ? mapa_shared(acc_empty0, 0) : acc_empty0;
   Segment* segs = seg_s[warp];
 
   if (warp < REPACK_WARPS) {
     // ---------------- re-layout: raw stage -> S stage ---------------------------
-    // task = (box, octet of the k-block, group of 32 halves); warp w takes tasks w, w + 8, ...
+    // task = (box, octet of the k-block, group of 32 halves).  A warp owns one group of 32 halves
+    // of every box and every second octet.  Where a lane's matrix row goes depends on the tile and
+    // the box only, so it is worked out once per tile (boxinfo); per task only the unit of the
+    // (octet, u) pair is added.
     bool ok = true;
     int st = 0, rst = 0;
     uint32_t ph = 0, rph = 0;
     const uint32_t trash_l = smem_u32(trash) + (lane >> 3) * 128;
     const uint32_t src_l = (uint32_t)(((lane & 7) * BOXW + (warp & 3) * 32 + (lane >> 3) * 8) * 2);
     const int m_l = (warp & 3) * 32 + lane;       // lane's matrix row = element m of the box row
+    const int par = warp >> 2;                    // octets par, par + 2, ... (alternating with the box)
+    const uint32_t r16 = (uint32_t)q.R * 16u;
+    const bool use_table = q.num_kb > 2;
     TIMER_DECL;
-    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
-      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+    for (int w = w_first; w < q.nwork && ok; w += w_step) {
+      const int q0 = (PAIR ? 2 * (w % q.ntm) + (int)rank : w % q.ntm) * TILE_M;
       int nseg = 0, total_boxes = 0;
       if (lane == 0) nseg = split_by_image(q, q0, segs, &total_boxes);
       nseg = __shfl_sync(0xffffffffu, nseg, 0);
       total_boxes = __shfl_sync(0xffffffffu, total_boxes, 0);
       __syncwarp();
-      const int s0_o0 = segs[0].o0, s0_elems = segs[0].elems, s0_nbox = segs[0].nbox;
+      // boxinfo[b]: byte offset of (sub-tile, unit 0, this lane's S row) | u in the low 4 bits, or
+      // bit 31 | bank group << 4 when the lane's element lies outside the segment
+      uint32_t boxinfo[MAXBOX];
+      if (use_table) {
+        int g = 0, row0 = 0, seg_elems = segs[0].elems, seg_end = segs[0].nbox;
+        int e0 = m_l - segs[0].o0;               // this lane's element in box 0 of the segment
+#pragma unroll
+        for (int b = 0; b < MAXBOX; ++b) {
+          boxinfo[b] = 0x80000000u;
+          if (b < total_boxes) {
+            while (b >= seg_end) {
+              ++g;
+              row0 = segs[g].row0; seg_elems = segs[g].elems; seg_end = segs[g].box0 + segs[g].nbox;
+              e0 = m_l - segs[g].o0 - segs[g].box0 * BOXSTEP;
+            }
+            const int e = b * BOXSTEP + e0;                                     // element of the segment
+            boxinfo[b] = 0x80000000u | (uint32_t)(((q.R * e + row0) & 7) << 4);
+            if ((unsigned)e < (unsigned)seg_elems) {
+              const int col = (int)(((uint32_t)e * q.magic_kh) >> 16);
+              const int u = e - col * q.Kh;
+              const int vr = (int)(((uint32_t)col * q.magic_s) >> 16);
+              const int sub = col - vr * q.s;
+              boxinfo[b] = (uint32_t)((((sub << 3) * q.R + row0 + vr) << 4) | u);
+            }
+          }
+        }
+      }
       if (threadIdx.x == 0) TIMER_LAP(0);       // per-tile setup
       for (int kb = 0; kb < q.num_kb; ++kb) {
         if (lane == 0) {
@@ -200,53 +251,104 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
         if (!ok) break;
         const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
-        const uint32_t raw_stage = raw_ring + rst * q.raw_stage_bytes;
+        const uint32_t raw_stage = raw_ring + rst * q.raw_stage_bytes + src_l;
         const uint32_t info = kbinfo[kb];
         const int oct_lo = (int)(info & 0xffffu), noct = (int)(info >> 16);
         const int nch = kb == q.num_kb - 1 ? q.nch_last : 8;
         const int unit0 = oct_lo * q.Kh - kb * 8;       // S unit of (first octet, u = 0); may be negative
-        int o = warp >> 2, b = 0;
-        while (o >= noct) { o -= noct; ++b; }
-        // the current segment lives in registers; it changes at most SEG_MAX - 1 times per stage
-        int g = 0, seg_o0 = s0_o0, seg_row0 = 0, seg_elems = s0_elems, seg_box0 = 0, seg_end = s0_nbox;
-        while (b < total_boxes) {
-          // BATCH tasks at a time: all matrix loads first, then the stores, so that the loads'
-          // latencies overlap
-          uint32_t r[BATCH][4], dst[BATCH];
-          int cnt = 0;
-#pragma unroll
-          for (int k = 0; k < BATCH; ++k) {
-            if (b < total_boxes) {
-              while (b >= seg_end) {
-                ++g;
-                seg_o0 = segs[g].o0; seg_row0 = segs[g].row0; seg_elems = segs[g].elems;
-                seg_box0 = segs[g].box0; seg_end = seg_box0 + segs[g].nbox;
-              }
-              ldmatrix_x4_trans(raw_stage + (uint32_t)(b * q.box_bytes + o * (8 * BOXW * 2)) + src_l, r[k]);
-              const int e = (b - seg_box0) * BOXSTEP + m_l - seg_o0;      // element of the segment
-              const int ubase = unit0 + o * q.Kh;
-              // rows that belong to no S unit go to a scratch line, into the bank group the real
-              // destination would have had (R*e + const mod 8 when R*Kh = 1 mod 8), so that the 8
-              // rows of a matrix never collide
-              dst[k] = trash_l + (uint32_t)(((q.R * e + ubase * q.R + seg_row0) & 7) << 4);
-              if ((unsigned)e < (unsigned)seg_elems) {
-                const int col = (int)(((uint32_t)e * q.magic_kh) >> 16);
-                const int u = e - col * q.Kh;
-                const int unit = ubase + u;
-                if ((unsigned)unit < (unsigned)nch) {
-                  const int vr = (int)(((uint32_t)col * q.magic_s) >> 16);
-                  const int sub = col - vr * q.s;
-                  dst[k] = a_stage + (uint32_t)((((sub << 3) + unit) * q.R + seg_row0 + vr) << 4);
+        if (use_table) {
+          // Four boxes (up to eight tasks) at a time: all matrix loads first, then the stores, so that
+          // the loads' latencies overlap.  Within a box this warp takes octets o and o + 2.
+          for (int oc = 0; oc < noct; oc += 4) {
+  #pragma unroll
+            for (int bg = 0; bg < MAXBOX; bg += 4) {
+              if (bg < total_boxes) {
+                uint32_t r[4][2][4];
+  #pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const int b = bg + i;
+                  if (b < total_boxes) {
+                    const int o = oc + ((par + b) & 1);
+                    const uint32_t src = raw_stage + (uint32_t)(b * q.box_bytes + o * (8 * BOXW * 2));
+                    if (o < noct) ldmatrix_x4_trans(src, r[i][0]);
+                    if (o + 2 < noct) ldmatrix_x4_trans(src + 2 * (8 * BOXW * 2), r[i][1]);
+                  }
+                }
+  #pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const int b = bg + i;
+                  if (b < total_boxes) {
+                    const int o = oc + ((par + b) & 1);
+                    const uint32_t bi = boxinfo[b];
+                    const uint32_t base = bi & 0x7ffffff0u;
+                    const bool in_seg = (bi >> 31) == 0u;
+                    const int unit_a = unit0 + o * q.Kh + (int)(bi & 15u);
+                    // rows that belong to no S unit go to a scratch line, into the bank group the real
+                    // destination would have had, so that the 8 rows of a matrix never collide
+                    if (o < noct) {
+                      const uint32_t ta = base + (uint32_t)unit_a * r16;
+                      const uint32_t da =
+                          (in_seg && (unsigned)unit_a < (unsigned)nch) ? a_stage + ta : trash_l + (ta & 0x70u);
+                      stmatrix_x4(da, r[i][0]);
+                    }
+                    if (o + 2 < noct) {
+                      const int unit_b = unit_a + 2 * q.Kh;
+                      const uint32_t tb = base + (uint32_t)unit_b * r16;
+                      const uint32_t db =
+                          (in_seg && (unsigned)unit_b < (unsigned)nch) ? a_stage + tb : trash_l + (tb & 0x70u);
+                      stmatrix_x4(db, r[i][1]);
+                    }
+                  }
                 }
               }
-              o += 2;
-              while (o >= noct) { o -= noct; ++b; }
-              cnt = k + 1;
             }
           }
-#pragma unroll
-          for (int k = 0; k < BATCH; ++k)
-            if (k < cnt) stmatrix_x4(dst[k], r[k]);
+        } else {
+          // tiles with one or two k-blocks: the per-tile table would cost more than it saves;
+          // warp w takes tasks w, w + 8, ... and works out each destination on the spot
+          int o = warp >> 2, b = 0;
+          while (o >= noct) { o -= noct; ++b; }
+          // the current segment lives in registers; it changes at most SEG_MAX - 1 times per stage
+          int g = 0, seg_o0 = segs[0].o0, seg_row0 = 0, seg_elems = segs[0].elems, seg_box0 = 0, seg_end = segs[0].nbox;
+          while (b < total_boxes) {
+            // BATCH tasks at a time: all matrix loads first, then the stores, so that the loads'
+            // latencies overlap
+            uint32_t r[BATCH][4], dst[BATCH];
+            int cnt = 0;
+  #pragma unroll
+            for (int k = 0; k < BATCH; ++k) {
+              if (b < total_boxes) {
+                while (b >= seg_end) {
+                  ++g;
+                  seg_o0 = segs[g].o0; seg_row0 = segs[g].row0; seg_elems = segs[g].elems;
+                  seg_box0 = segs[g].box0; seg_end = seg_box0 + segs[g].nbox;
+                }
+                ldmatrix_x4_trans(raw_stage + (uint32_t)(b * q.box_bytes + o * (8 * BOXW * 2)), r[k]);
+                const int e = (b - seg_box0) * BOXSTEP + m_l - seg_o0;      // element of the segment
+                const int ubase = unit0 + o * q.Kh;
+                // rows that belong to no S unit go to a scratch line, into the bank group the real
+                // destination would have had (R*e + const mod 8 when R*Kh = 1 mod 8), so that the 8
+                // rows of a matrix never collide
+                dst[k] = trash_l + (uint32_t)(((q.R * e + ubase * q.R + seg_row0) & 7) << 4);
+                if ((unsigned)e < (unsigned)seg_elems) {
+                  const int col = (int)(((uint32_t)e * q.magic_kh) >> 16);
+                  const int u = e - col * q.Kh;
+                  const int unit = ubase + u;
+                  if ((unsigned)unit < (unsigned)nch) {
+                    const int vr = (int)(((uint32_t)col * q.magic_s) >> 16);
+                    const int sub = col - vr * q.s;
+                    dst[k] = a_stage + (uint32_t)((((sub << 3) + unit) * q.R + seg_row0 + vr) << 4);
+                  }
+                }
+                o += 2;
+                while (o >= noct) { o -= noct; ++b; }
+                cnt = k + 1;
+              }
+            }
+  #pragma unroll
+            for (int k = 0; k < BATCH; ++k)
+              if (k < cnt) stmatrix_x4(dst[k], r[k]);
+          }
         }
         if ((nch & 1) && kb == q.num_kb - 1) {
           // odd number of units: the last k step reads one more unit; make it zeros
@@ -261,7 +363,8 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          mbar_arrive(a_full0 + 8 * st);
+          if (PAIR) mbar_arrive_cluster(a_full_dst + 8 * st);
+          else mbar_arrive(a_full0 + 8 * st);
           mbar_arrive(r_empty0 + 8 * rst);
         }
         if (threadIdx.x == 0) TIMER_LAP(4);     // fence + arrive
@@ -276,26 +379,32 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
     bool ok = true;
     int st = 0;
     uint32_t ph = 0;
-    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
+    for (int w = w_first; w < q.nwork && ok; w += w_step) {
       const int n0 = (w / q.ntm) * BN;
       for (int kb = 0; kb < q.num_kb && ok; ++kb) {
         for (int v = 0; v < q.Kw; ++v) {
           ok = mbar_wait(b_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          const uint32_t bar = b_full0 + 8 * st;
           if (leader) {
-            mbar_arrive_expect_tx(bar, B_STAGE_BYTES);
-            tma_load_3d(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0, v, bar);
+            if (PAIR) {
+              // the leader CTA announces both halves; each CTA's copy reports to the leader's barrier
+              if (rank == 0) mbar_arrive_expect_tx(b_full0 + 8 * st, 2 * B_STAGE_BYTES);
+              tma_load_3d_pair(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0 + (int)rank * B_ROWS, v,
+                               b_full_dst + 8 * st);
+            } else {
+              mbar_arrive_expect_tx(b_full0 + 8 * st, B_STAGE_BYTES);
+              tma_load_3d(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0, v, b_full0 + 8 * st);
+            }
           }
           __syncwarp();
           if (++st == q.sb) { st = 0; ph ^= 1u; }
         }
       }
     }
-  } else if (warp == WARP_MMA) {
-    // ---------------- MMA issuer ------------------------------------------------
-    constexpr uint32_t idesc = instr_desc_f16(TILE_M, BN);
+  } else if (warp == WARP_MMA && rank == 0) {
+    // ---------------- MMA issuer (leader CTA of a pair) -------------------------
+    constexpr uint32_t idesc = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN);
     const bool leader = elect_one();
     bool ok = true;
     int sta = 0, stb = 0;
@@ -306,10 +415,11 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
     const uint32_t kstep_units = 2u * (uint32_t)q.R;     // 16-byte units per 16-element k step
     const int ks_last = (q.nch_last + 1) >> 1;
     TIMER_DECL;
-    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
+    for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
       const uint32_t buf = it & 1u;
       TIMER_LAP(8);
-      ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
+      ok = PAIR ? mbar_wait_cluster(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status)
+                : mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       TIMER_LAP(11);                             // MMA warp: wait for a free accumulator
@@ -318,7 +428,8 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
       uint32_t first = 0;
       for (int kb = 0; kb < q.num_kb && ok; ++kb) {
         TIMER_LAP(8);
-        ok = mbar_wait(a_full0 + 8 * sta, pha, &abort_flag, q.status);
+        ok = PAIR ? mbar_wait_cluster(a_full0 + 8 * sta, pha, &abort_flag, q.status)
+                  : mbar_wait(a_full0 + 8 * sta, pha, &abort_flag, q.status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         TIMER_LAP(9);                            // MMA warp: wait for an S stage
@@ -327,7 +438,8 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
         uint32_t sub = 0, shift = 0;             // kernel column v reads sub-tile v mod s from row v div s on
         for (int v = 0; v < q.Kw; ++v) {
           TIMER_LAP(8);
-          ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
+          ok = PAIR ? mbar_wait_cluster(b_full0 + 8 * stb, phb, &abort_flag, q.status)
+                    : mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           TIMER_LAP(10);                         // MMA warp: wait for a filter stage
@@ -336,33 +448,48 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
           const uint32_t a_lo = a_lo_stage + sub * sub_units + shift;
           if (leader) {
 #pragma unroll 1
-            for (int j = 0; j < nks; ++j)
-              umma_f16_ab(acc, a_lo + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j, kSmemDescHiSw128,
-                          idesc, first | (uint32_t)j);
-            umma_commit(b_empty0 + 8 * stb);
+            for (int j = 0; j < nks; ++j) {
+              if (PAIR)
+                umma_f16_ab_pair(acc, a_lo + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j,
+                                 kSmemDescHiSw128, idesc, first | (uint32_t)j);
+              else
+                umma_f16_ab(acc, a_lo + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j, kSmemDescHiSw128,
+                            idesc, first | (uint32_t)j);
+            }
+            if (PAIR) umma_commit_pair(b_empty0 + 8 * stb);
+            else umma_commit(b_empty0 + 8 * stb);
           }
           __syncwarp();
           first = 1u;
           if (++sub == (uint32_t)q.s) { sub = 0; ++shift; }
           if (++stb == q.sb) { stb = 0; phb ^= 1u; }
         }
-        if (ok && leader) umma_commit(a_empty0 + 8 * sta);
+        if (ok && leader) {
+          if (PAIR) umma_commit_pair(a_empty0 + 8 * sta);
+          else umma_commit(a_empty0 + 8 * sta);
+        }
         __syncwarp();
         if (++sta == q.sa) { sta = 0; pha ^= 1u; }
       }
-      if (ok && leader) umma_commit(acc_full0 + 8 * buf);
+      if (ok && leader) {
+        if (PAIR) umma_commit_pair(acc_full0 + 8 * buf);
+        else umma_commit(acc_full0 + 8 * buf);
+      }
       __syncwarp();
     }
     if (leader) { TIMER_LAP(8); TIMER_FLUSH(); }
-  } else if (warp == WARP_RAW) {
-    // ---------------- raw loader: tiled TMA loads of the channel planes ----------
+  } else if (warp == WARP_RAW || warp == WARP_RAW + 1) {
+    // ---------------- raw loaders: tiled TMA loads of the channel planes ---------
+    // two warps share the boxes of a stage (even / odd): issuing a copy costs a few hundred
+    // cycles and the stage is only complete when its last box has been requested
+    const int half = warp - WARP_RAW;
     const bool leader = elect_one();
     bool ok = true;
     int rst = 0;
     uint32_t rph = 0;
     TIMER_DECL;
-    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
-      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+    for (int w = w_first; w < q.nwork && ok; w += w_step) {
+      const int q0 = (PAIR ? 2 * (w % q.ntm) + (int)rank : w % q.ntm) * TILE_M;
       int nseg = 0, total_boxes = 0;
       if (lane == 0) nseg = split_by_image(q, q0, segs, &total_boxes);
       nseg = __shfl_sync(0xffffffffu, nseg, 0);
@@ -378,11 +505,12 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
         const int c_lo = (int)(kbinfo[kb] & 0xffffu) * 8;
         const uint32_t stage = raw_ring + rst * q.raw_stage_bytes;
         if (leader) {
-          mbar_arrive_expect_tx(bar, (uint32_t)(total_boxes * q.box_bytes));
+          if (half == 0) mbar_arrive_expect_tx(bar, (uint32_t)(total_boxes * q.box_bytes));
           for (int g = 0; g < nseg; ++g)
             for (int j = 0; j < segs[g].nbox; ++j)
-              tma_load_3d(stage + (segs[g].box0 + j) * q.box_bytes, &wmap, segs[g].x0 + j * BOXSTEP, c_lo, segs[g].n,
-                          bar);
+              if (((segs[g].box0 + j) & 1) == half)
+                tma_load_3d(stage + (segs[g].box0 + j) * q.box_bytes, &wmap, segs[g].x0 + j * BOXSTEP, c_lo,
+                            segs[g].n, bar);
         }
         __syncwarp();
         if (++rst == q.rs) { rst = 0; rph ^= 1u; }
@@ -394,20 +522,20 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
     const int lq = warp & 3;                     // tensor-memory lane quadrant this warp may read
     bool ok = true;
     uint32_t it = 0;
-    for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
+    for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
       const uint32_t buf = it & 1u;
-      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+      const int q0 = (PAIR ? 2 * (w % q.ntm) + (int)rank : w % q.ntm) * TILE_M;
       const int n0 = (w / q.ntm) * BN;
-      const int64_t vq = q0 + lq * 32 + lane;    // accumulator row = virtual position
+      const int vq = q0 + lq * 32 + lane;        // accumulator row = virtual position
       bool valid = false;
       float* yrow = q.y;
-      if (vq < q.VQ) {
-        const int64_t sg = vq / q.Wq;
-        const int kq = (int)(vq - sg * q.Wq);
-        const int64_t n = sg / q.Ho;
-        const int ho = (int)(sg - n * q.Ho);
+      if (vq < (int)q.VQ) {
+        const int sg = vq / q.Wq;
+        const int kq = vq - sg * q.Wq;
+        const int n = sg / q.Ho;
+        const int ho = sg - n * q.Ho;
         valid = kq < q.Wo;                       // trailing columns of a strip are no output
-        yrow += (n * q.Co) * q.HoWo + ho * q.Wo + kq;
+        yrow += ((int64_t)n * q.Co) * q.HoWo + ho * q.Wo + kq;
       }
       if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -430,7 +558,10 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
       // the buffer may be overwritten once all four warps have read it
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty0 + 8 * buf);
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_cluster(acc_empty_dst + 8 * buf);
+        else mbar_arrive(acc_empty0 + 8 * buf);
+      }
     }
   }
 
@@ -441,11 +572,25 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
   }
+  if (PAIR) cluster_sync_all();               // no CTA leaves while its peer may still signal or read it
   if (warp == WARP_MMA) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_acc, 2 * BN);
+    if (PAIR) tmem_dealloc_pair(tmem_acc, 2 * BN);
+    else tmem_dealloc(tmem_acc, 2 * BN);
   }
+}
+
+template <int BN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_constant__ CUtensorMap wmap, MatParams q) {
+  conv_f16_mat_body<BN, false>(fmap, wmap, q);
+}
+
+// CTA-pair form for wide channel tiles (Co > 128): clusters of two CTAs.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+conv_f16_mat_pair_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_constant__ CUtensorMap wmap, MatParams q) {
+  conv_f16_mat_body<256, true>(fmap, wmap, q);
 }
 
 // Filter pack for this kernel: Fp3[v][co][k2p], k2 = (oct*Kh + u)*8 + e, c = 8*oct + e
@@ -488,22 +633,22 @@ constexpr int kSmemMax = 227 * 1024;
 
 int tile_bn(const Geometry& g) { return g.Co <= 64 ? 64 : (g.Co <= 128 ? 128 : 256); }
 
-// Ring depths that fit: S ring 2, raw ring 3 (2 if tight), filter ring as deep as fits (<= 4).
-// Narrow tiles try to fit two CTAs on an SM first.
-bool choose_rings(int bn, const MatPlan& plan, int* rs, int* sa, int* sb, int* smem_bytes) {
+// Ring depths that fit: S ring 2, raw ring 2, filter ring as deep as fits (<= 6), then a third raw
+// stage if there is room.  Narrow tiles try to fit two CTAs on an SM first.
+bool choose_rings(int bn, int b_rows, const MatPlan& plan, int* rs, int* sa, int* sb, int* smem_bytes) {
   const int fixed = plan.num_kb * 4;
-  const int a = plan.a_stage_bytes, r = plan.raw_stage_bytes, b = bn * KB * 2;
+  const int a = plan.a_stage_bytes, r = plan.raw_stage_bytes, b = b_rows * KB * 2;
   for (int half = (bn <= 128 ? 1 : 0); half >= 0; --half) {
     // dynamic shared memory left after the alignment slack, the static part (barriers, segment
     // copies) and, for two CTAs per SM, the 1 KB the runtime reserves per CTA
     const int budget = (half ? kSmemMax / 2 : kSmemMax) - 1024 - 4096;
-    for (int rr = 3; rr >= 2; --rr)
-      for (int bb = 4; bb >= 2; --bb)
-        if (2 * a + rr * r + bb * b + fixed <= budget && (bb >= 3 || rr == 2)) {
-          *rs = rr; *sa = 2; *sb = bb;
-          *smem_bytes = 2 * a + rr * r + bb * b + fixed + 1024;
-          return true;
-        }
+    for (int bb = MAX_STAGES; bb >= 2; --bb)
+      if (2 * a + 2 * r + bb * b + fixed <= budget) {
+        const int rr = (bb >= 4 && 2 * a + 3 * r + bb * b + fixed <= budget) ? 3 : 2;
+        *rs = rr; *sa = 2; *sb = bb;
+        *smem_bytes = 2 * a + rr * r + bb * b + fixed + 1024;
+        return true;
+      }
   }
   return false;
 }
@@ -512,7 +657,7 @@ template <int BN>
 cudaError_t launch_bn(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParams q, const MatPlan& plan, int co,
                       cudaStream_t stream) {
   int smem_bytes = 0;
-  if (!choose_rings(BN, plan, &q.rs, &q.sa, &q.sb, &smem_bytes)) return cudaErrorInvalidValue;
+  if (!choose_rings(BN, BN, plan, &q.rs, &q.sa, &q.sb, &smem_bytes)) return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(conv_f16_mat_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
   const int64_t ntm = (plan.VQ + TILE_M - 1) / TILE_M;
@@ -524,6 +669,40 @@ cudaError_t launch_bn(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParam
   const int slots = 148 * per_sm;                      // persistent CTAs
   const unsigned grid = (unsigned)(nwork < slots ? nwork : slots);
   conv_f16_mat_kernel<BN><<<grid, NUM_THREADS, smem_bytes, stream>>>(fmap, wmap, q);
+  return cudaGetLastError();
+}
+
+// CTA-pair launch (Co > 128): clusters of two CTAs, as many as can be resident at once.
+cudaError_t launch_pair(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParams q, const MatPlan& plan, int co,
+                        cudaStream_t stream) {
+  int smem_bytes = 0;
+  if (!choose_rings(256, 128, plan, &q.rs, &q.sa, &q.sb, &smem_bytes)) return cudaErrorInvalidValue;
+  cudaError_t e =
+      cudaFuncSetAttribute(conv_f16_mat_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  if (e != cudaSuccess) return e;
+  const int64_t ntm = (plan.VQ + TILE_M - 1) / TILE_M;
+  const int64_t ntp = (ntm + 1) / 2;                   // pairs of position tiles
+  const int64_t nwork = ntp * ((co + 255) / 256);
+  if (nwork >= ((int64_t)1 << 30)) return cudaErrorInvalidValue;
+  q.ntm = (int32_t)ntp;
+  q.nwork = (int32_t)nwork;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.gridDim = dim3(148, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem_bytes;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int clusters = 0;
+  e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_mat_pair_kernel, &cfg);
+  if (e != cudaSuccess) return e;
+  if (clusters < 1) return cudaErrorInvalidValue;
+  if (clusters > 74) clusters = 74;
+  if ((int64_t)clusters > nwork) clusters = (int)nwork;
+  conv_f16_mat_pair_kernel<<<2 * clusters, NUM_THREADS, smem_bytes, stream>>>(fmap, wmap, q);
   return cudaGetLastError();
 }
 
@@ -554,6 +733,7 @@ MatPlan plan_f16_mat(const Geometry& g) {
   if (p.num_kb > MAX_KB) return p;
   p.nch_last = (int32_t)(units - 8 * (int64_t)(p.num_kb - 1));
   p.VQ = (int64_t)g.N * g.Ho * p.Wq;
+  if (p.VQ >= ((int64_t)1 << 31) - 4 * TILE_M) return p;    // the kernel indexes virtual positions with 32 bits
   const int64_t img_rows = (int64_t)g.Ho * p.Wq;
   const int64_t segmax = (p.rows - 2) / img_rows + 2;     // images a tile can touch
   if (segmax > SEG_MAX) return p;
@@ -587,12 +767,13 @@ MatPlan plan_f16_mat(const Geometry& g) {
     }
     if (probe > 65536) maxbox += (int)segmax;   // unprobed phases: leave room for one more box per image
   }
+  if (maxbox > MAXBOX) return p;
   p.raw_stage_bytes = maxbox * p.box_bytes;
   p.a_stage_bytes = (g.s * 8 * p.R * 16 + 127) / 128 * 128;
   if ((p.VQ + TILE_M - 1) / TILE_M * ((g.Co + 63) / 64) >= ((int64_t)1 << 31)) return p;
   p.scratch_bytes = (size_t)kStatusBytes + (size_t)p.K2p * g.Co * g.Kw * 2;
   int rs, sa, sb, smem;
-  if (!choose_rings(tile_bn(g), p, &rs, &sa, &sb, &smem)) return p;
+  if (!choose_rings(tile_bn(g), tile_bn(g), p, &rs, &sa, &sb, &smem)) return p;
   p.eligible = true;
   return p;
 }
@@ -606,6 +787,8 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, 
   unsigned char* base = static_cast<unsigned char*>(scratch);
   uint16_t* fp = reinterpret_cast<uint16_t*>(base + kStatusBytes);
   const int bn = tile_bn(g);
+  const char* pair_env = getenv("IM2WIN_F16_PAIR");     // testing aid: 0 = never pair CTAs
+  const bool pair = bn == 256 && !(pair_env && pair_env[0] == '0');
 
   {
     const unsigned gx = (unsigned)((plan.K2p + 255) / 256);
@@ -620,7 +803,7 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, 
   CUtensorMap fmap;
   const cuuint64_t dims[3] = {(cuuint64_t)plan.K2p, (cuuint64_t)g.Co, (cuuint64_t)g.Kw};
   const cuuint64_t strides[2] = {(cuuint64_t)plan.K2p * 2, (cuuint64_t)plan.K2p * 2 * (cuuint64_t)g.Co};
-  const cuuint32_t box[3] = {(cuuint32_t)KB, (cuuint32_t)bn, 1};
+  const cuuint32_t box[3] = {(cuuint32_t)KB, (cuuint32_t)(pair ? bn / 2 : bn), 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   CUresult cr = encode(&fmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, fp, dims, strides, box, estr,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -652,6 +835,7 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, 
   q.magic_kh = magic16(g.Kh); q.magic_s = magic16(g.s);
   q.rs = q.sa = q.sb = 2;
   q.ntm = q.nwork = 0;
+  if (pair) return launch_pair(fmap, wmap, q, plan, g.Co, stream);
   if (bn == 64) return launch_bn<64>(fmap, wmap, q, plan, g.Co, stream);
   if (bn == 128) return launch_bn<128>(fmap, wmap, q, plan, g.Co, stream);
   return launch_bn<256>(fmap, wmap, q, plan, g.Co, stream);

@@ -38,6 +38,8 @@ SMALL = [
     L("deep", 2, 130, 7, 7, 140, 3, 3, 1, 1, 22),               # K = 1170: many k-blocks, odd strips (54 B)
     L("wide_row", 1, 2, 4, 300, 5, 3, 3, 1, 1, 23),             # one output row longer than a tile
     L("uncovered_cols", 1, 3, 10, 12, 4, 3, 4, 3, 0, 24),       # (Wp - Kw) % s != 0: trailing columns never read
+    L("pair_odd", 3, 16, 18, 22, 260, 3, 3, 1, 1, 25),          # Co > 256 and an odd number of position tiles (CTA pairs)
+    L("pair_s2", 2, 24, 16, 14, 200, 3, 3, 2, 1, 26),           # CTA pairs with stride 2
 ]
 
 
@@ -153,6 +155,37 @@ def test_repeated_calls_are_deterministic_and_do_not_depend_on_stale_scratch():
         y1, _, _ = gpu_conv(x, f, dims, precision)
         y2, _, _ = gpu_conv(x, f, dims, precision)
         assert np.array_equal(y1, y2)
+
+
+@pytest.mark.parametrize("pair", ["0", "1"])
+def test_mat_kernel_with_and_without_cta_pairs(pair, monkeypatch):
+    """The matrix-transpose fp16 kernel in its one-CTA and CTA-pair forms on a wide layer."""
+    monkeypatch.setenv("IM2WIN_F16_PAIR", pair)
+    for layer in (SMALL[15], SMALL[16], SMALL[4]):
+        dims = layer.dims()
+        x, f = workloads.make_small_integer_inputs(layer)
+        y, _, _ = gpu_conv(x, f, dims, "f16-mat")
+        yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+        assert np.array_equal(y.astype(np.float64), yr), layer.name
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg4a", "cfg5k3"])
+def test_full_size_mat_kernel_sampled(name):
+    """The matrix-transpose fp16 kernel forced at benchmark sizes, on sampled outputs."""
+    layer = workloads.LAYERS[name]
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    ho, wo = oracle.out_dims(dims)
+    total = layer.N * layer.Co * ho * wo
+    rng = np.random.default_rng(layer.seed + 7)
+    idx = np.concatenate([rng.integers(0, total, 4096), [0, total - 1, wo - 1, ho * wo - 1, total - ho * wo]])
+    y, _, _ = gpu_conv(x, f, dims, "f16-mat")
+    xo, fo = oracle_inputs(x, f, "f16-mat")
+    yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
+    check_conv(y.reshape(-1)[idx], yr, ar, "f16-mat", layer.name)
+    one = dict(dims, N=1)
+    yi, ai = oracle.conv_im2win(xo[-1:], fo, one)
+    check_conv(y[-1:], yi, ai, "f16-mat", layer.name + " last image")
 
 
 # ------------------------------------------------------------ full-size layers ----
