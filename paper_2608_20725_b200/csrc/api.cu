@@ -88,9 +88,9 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
     if (mat.eligible) {
       const char* force = getenv("IM2WIN_F16_KERNEL");
       // measured: the matrix-transpose kernel wins for strided layers (the others stage such
-      // layers with 2-byte gathers) and, in its CTA-pair form, for narrow kernels with more than
-      // 128 output channels; IM2WIN_F16_KERNEL=mat forces it everywhere (a testing aid)
-      l->f16_mat = force ? strcmp(force, "mat") == 0 : (g.s > 1 || (g.Co > 128 && g.Kw < 5));
+      // layers with 2-byte gathers) and, in its CTA-pair form, for kernels up to 5 wide with more
+      // than 128 output channels; IM2WIN_F16_KERNEL=mat forces it everywhere (a testing aid)
+      l->f16_mat = force ? strcmp(force, "mat") == 0 : (g.s > 1 || (g.Co > 128 && g.Kw <= 5));
       const size_t mat_total = (size_t)round_up((int64_t)mat.scratch_bytes, 256);
       if (mat_total > l->total) l->total = mat_total;
     }

@@ -69,7 +69,9 @@ struct MatParams {
   int32_t a_stage_bytes;    // s * 8 * R * 16, rounded up to 128
   uint32_t magic_kh, magic_s;   // floor(e / d) = (e * magic) >> 16 for e < 8192
   int32_t rs, sa, sb;       // ring depths
+  int32_t vg;               // kernel columns per filter stage
   int32_t ntm, nwork;       // position tiles; work items = position tiles x channel tiles
+  int32_t frows;            // 2 KB rows of the packed filter per (kernel column, k-block): 4 per 64 channels
 };
 
 struct Segment {            // the part of a tile that lies in one image
@@ -122,7 +124,8 @@ __device__ __forceinline__ int split_by_image(const MatParams& q, int q0, Segmen
 template <int BN, bool PAIR>
 __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const CUtensorMap& wmap, const MatParams& q) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;            // filter rows (output channels) this CTA stages
-  constexpr int B_STAGE_BYTES = B_ROWS * KB * 2;
+  constexpr int B_TILE_BYTES = B_ROWS * KB * 2;         // one kernel column of one k-block
+  const int B_STAGE_BYTES = q.vg * B_TILE_BYTES;        // a filter stage holds vg kernel columns
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
   const int w_first = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int w_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
@@ -380,21 +383,27 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
     int st = 0;
     uint32_t ph = 0;
     for (int w = w_first; w < q.nwork && ok; w += w_step) {
-      const int n0 = (w / q.ntm) * BN;
+      // first 2 KB row of this CTA's part of the channel tile in the packed filter (4 rows per 64 channels)
+      const int row0 = ((w / q.ntm) * BN + (int)rank * B_ROWS) / 16;
       for (int kb = 0; kb < q.num_kb && ok; ++kb) {
-        for (int v = 0; v < q.Kw; ++v) {
+        for (int v0 = 0; v0 < q.Kw; v0 += q.vg) {
+          const int nv = q.Kw - v0 < q.vg ? q.Kw - v0 : q.vg;      // kernel columns in this stage
           ok = mbar_wait(b_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           if (leader) {
+            const uint32_t dst = b_ring + st * B_STAGE_BYTES;
             if (PAIR) {
-              // the leader CTA announces both halves; each CTA's copy reports to the leader's barrier
-              if (rank == 0) mbar_arrive_expect_tx(b_full0 + 8 * st, 2 * B_STAGE_BYTES);
-              tma_load_3d_pair(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0 + (int)rank * B_ROWS, v,
-                               b_full_dst + 8 * st);
+              // the leader CTA announces both halves; each CTA's copies report to the leader's barrier
+              if (rank == 0) mbar_arrive_expect_tx(b_full0 + 8 * st, (uint32_t)(2 * nv * B_TILE_BYTES));
+              for (int i = 0; i < nv; ++i)
+                tma_load_2d_pair(dst + i * B_TILE_BYTES, &fmap, 0, ((v0 + i) * q.num_kb + kb) * q.frows + row0,
+                                 b_full_dst + 8 * st);
             } else {
-              mbar_arrive_expect_tx(b_full0 + 8 * st, B_STAGE_BYTES);
-              tma_load_3d(b_ring + st * B_STAGE_BYTES, &fmap, kb * KB, n0, v, b_full0 + 8 * st);
+              mbar_arrive_expect_tx(b_full0 + 8 * st, (uint32_t)(nv * B_TILE_BYTES));
+              for (int i = 0; i < nv; ++i)
+                tma_load_2d(dst + i * B_TILE_BYTES, &fmap, 0, ((v0 + i) * q.num_kb + kb) * q.frows + row0,
+                            b_full0 + 8 * st);
             }
           }
           __syncwarp();
@@ -436,7 +445,8 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
         const uint32_t a_lo_stage = a_lo0 + (uint32_t)(sta * (q.a_stage_bytes >> 4));
         const int nks = kb == q.num_kb - 1 ? ks_last : KB / 16;
         uint32_t sub = 0, shift = 0;             // kernel column v reads sub-tile v mod s from row v div s on
-        for (int v = 0; v < q.Kw; ++v) {
+        for (int v0 = 0; v0 < q.Kw; v0 += q.vg) {
+          const int nv = q.Kw - v0 < q.vg ? q.Kw - v0 : q.vg;
           TIMER_LAP(8);
           ok = PAIR ? mbar_wait_cluster(b_full0 + 8 * stb, phb, &abort_flag, q.status)
                     : mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
@@ -444,24 +454,27 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
           if (!ok) break;
           TIMER_LAP(10);                         // MMA warp: wait for a filter stage
           tc_fence_after();
-          const uint32_t b_lo = b_lo0 + (uint32_t)(stb * (B_STAGE_BYTES >> 4));
-          const uint32_t a_lo = a_lo_stage + sub * sub_units + shift;
+          uint32_t b_lo = b_lo0 + (uint32_t)(stb * (B_STAGE_BYTES >> 4));
           if (leader) {
+            for (int i = 0; i < nv; ++i) {
+              const uint32_t a_lo = a_lo_stage + sub * sub_units + shift;
 #pragma unroll 1
-            for (int j = 0; j < nks; ++j) {
-              if (PAIR)
-                umma_f16_ab_pair(acc, a_lo + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j,
-                                 kSmemDescHiSw128, idesc, first | (uint32_t)j);
-              else
-                umma_f16_ab(acc, a_lo + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j, kSmemDescHiSw128,
-                            idesc, first | (uint32_t)j);
+              for (int j = 0; j < nks; ++j) {
+                if (PAIR)
+                  umma_f16_ab_pair(acc, a_lo + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j,
+                                   kSmemDescHiSw128, idesc, first | (uint32_t)j);
+                else
+                  umma_f16_ab(acc, a_lo + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j,
+                              kSmemDescHiSw128, idesc, first | (uint32_t)j);
+              }
+              first = 1u;
+              b_lo += (uint32_t)(B_TILE_BYTES >> 4);
+              if (++sub == (uint32_t)q.s) { sub = 0; ++shift; }
             }
             if (PAIR) umma_commit_pair(b_empty0 + 8 * stb);
             else umma_commit(b_empty0 + 8 * stb);
           }
           __syncwarp();
-          first = 1u;
-          if (++sub == (uint32_t)q.s) { sub = 0; ++shift; }
           if (++stb == q.sb) { stb = 0; phb ^= 1u; }
         }
         if (ok && leader) {
@@ -593,22 +606,29 @@ conv_f16_mat_pair_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_
   conv_f16_mat_body<256, true>(fmap, wmap, q);
 }
 
-// Filter pack for this kernel: Fp3[v][co][k2p], k2 = (oct*Kh + u)*8 + e, c = 8*oct + e
-// (paper Section "Im2win Convolution": height before width; here additionally grouped by
-// channel octets).  Padded k2 (c >= C or beyond the last unit) hold zeros.  Block (0,0,0)
+// Filter pack for this kernel (paper Section "Im2win Convolution": height before width; here
+// additionally grouped by channel octets): k2 = (oct*Kh + u)*8 + e, c = 8*oct + e.  The packed
+// filter is a sequence of 8 KB images, one per (kernel column v, k-block kb, group of 64 output
+// channels), each laid out exactly as the MMA wants a k-major tile with the 128-byte swizzle in
+// shared memory (row = channel, 128 bytes; 16-byte chunk index XOR row mod 8), so that a filter
+// tile is ONE contiguous run and can be copied with 2 KB rows (the copy engine spends about a
+// cycle per row on top of the bytes).  Padded k2 and channels >= Co hold zeros.  Block (0,0,0)
 // also clears the status block.
 __global__ void pack_f16_mat_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, uint32_t* status,
-                                    int C, int Co, int Kh, int Kw, int K2p) {
+                                    int C, int Co, int Kh, int Kw, int K2p, int ncog) {
   if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
+  const int num_kb = K2p / KB;
   for (int v = blockIdx.z; v < Kw; v += gridDim.z)
-    for (int co = blockIdx.y; co < Co; co += gridDim.y)
+    for (int co = blockIdx.y; co < ncog * 64; co += gridDim.y)
       for (int k2 = blockIdx.x * blockDim.x + threadIdx.x; k2 < K2p; k2 += gridDim.x * blockDim.x) {
         const int unit = k2 >> 3, e = k2 & 7;
         const int oct = unit / Kh, u = unit - oct * Kh;
         const int c = oct * 8 + e;
         uint16_t val = 0;
-        if (c < C) val = f[(((size_t)co * C + c) * Kh + u) * Kw + v];
-        fp[((size_t)v * Co + co) * K2p + k2] = val;
+        if (c < C && co < Co) val = f[(((size_t)co * C + c) * Kh + u) * Kw + v];
+        const int kb = k2 >> 6, chunk = (k2 & 63) >> 3, r = co & 63;
+        const size_t image = ((size_t)v * num_kb + kb) * ncog + (co >> 6);
+        fp[image * 4096 + (size_t)r * 64 + (size_t)(((chunk ^ (r & 7)) << 3) + e)] = val;
       }
 }
 
@@ -633,22 +653,28 @@ constexpr int kSmemMax = 227 * 1024;
 
 int tile_bn(const Geometry& g) { return g.Co <= 64 ? 64 : (g.Co <= 128 ? 128 : 256); }
 
-// Ring depths that fit: S ring 2, raw ring 2, filter ring as deep as fits (<= 6), then a third raw
-// stage if there is room.  Narrow tiles try to fit two CTAs on an SM first.
-bool choose_rings(int bn, int b_rows, const MatPlan& plan, int* rs, int* sa, int* sb, int* smem_bytes) {
+// Ring depths that fit: S ring 2, raw ring 2, a filter stage of as many kernel columns as fit
+// twice (every barrier round trip and commit costs the MMA issuer time, so fewer, larger filter
+// stages are better), filter ring as deep as fits (<= 6), then a third raw stage if there is room.
+// Narrow tiles try to fit two CTAs on an SM first.
+bool choose_rings(int bn, int b_rows, int kw, const MatPlan& plan, int* rs, int* sa, int* sb, int* vg,
+                  int* smem_bytes) {
   const int fixed = plan.num_kb * 4;
-  const int a = plan.a_stage_bytes, r = plan.raw_stage_bytes, b = b_rows * KB * 2;
+  const int a = plan.a_stage_bytes, r = plan.raw_stage_bytes, tile = b_rows * KB * 2;
   for (int half = (bn <= 128 ? 1 : 0); half >= 0; --half) {
     // dynamic shared memory left after the alignment slack, the static part (barriers, segment
     // copies) and, for two CTAs per SM, the 1 KB the runtime reserves per CTA
     const int budget = (half ? kSmemMax / 2 : kSmemMax) - 1024 - 4096;
-    for (int bb = MAX_STAGES; bb >= 2; --bb)
-      if (2 * a + 2 * r + bb * b + fixed <= budget) {
-        const int rr = (bb >= 4 && 2 * a + 3 * r + bb * b + fixed <= budget) ? 3 : 2;
-        *rs = rr; *sa = 2; *sb = bb;
-        *smem_bytes = 2 * a + rr * r + bb * b + fixed + 1024;
-        return true;
-      }
+    for (int g = kw; g >= 1; --g) {
+      const int b = g * tile;
+      if (2 * a + 2 * r + 2 * b + fixed > budget) continue;
+      int bb = 2;
+      while (bb < MAX_STAGES && (bb + 1) * g <= 12 && 2 * a + 2 * r + (bb + 1) * b + fixed <= budget) ++bb;
+      const int rr = (2 * a + 3 * r + bb * b + fixed <= budget) ? 3 : 2;
+      *rs = rr; *sa = 2; *sb = bb; *vg = g;
+      *smem_bytes = 2 * a + rr * r + bb * b + fixed + 1024;
+      return true;
+    }
   }
   return false;
 }
@@ -657,7 +683,7 @@ template <int BN>
 cudaError_t launch_bn(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParams q, const MatPlan& plan, int co,
                       cudaStream_t stream) {
   int smem_bytes = 0;
-  if (!choose_rings(BN, BN, plan, &q.rs, &q.sa, &q.sb, &smem_bytes)) return cudaErrorInvalidValue;
+  if (!choose_rings(BN, BN, q.Kw, plan, &q.rs, &q.sa, &q.sb, &q.vg, &smem_bytes)) return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(conv_f16_mat_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
   const int64_t ntm = (plan.VQ + TILE_M - 1) / TILE_M;
@@ -676,7 +702,7 @@ cudaError_t launch_bn(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParam
 cudaError_t launch_pair(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParams q, const MatPlan& plan, int co,
                         cudaStream_t stream) {
   int smem_bytes = 0;
-  if (!choose_rings(256, 128, plan, &q.rs, &q.sa, &q.sb, &smem_bytes)) return cudaErrorInvalidValue;
+  if (!choose_rings(256, 128, q.Kw, plan, &q.rs, &q.sa, &q.sb, &q.vg, &smem_bytes)) return cudaErrorInvalidValue;
   cudaError_t e =
       cudaFuncSetAttribute(conv_f16_mat_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
@@ -771,9 +797,9 @@ MatPlan plan_f16_mat(const Geometry& g) {
   p.raw_stage_bytes = maxbox * p.box_bytes;
   p.a_stage_bytes = (g.s * 8 * p.R * 16 + 127) / 128 * 128;
   if ((p.VQ + TILE_M - 1) / TILE_M * ((g.Co + 63) / 64) >= ((int64_t)1 << 31)) return p;
-  p.scratch_bytes = (size_t)kStatusBytes + (size_t)p.K2p * g.Co * g.Kw * 2;
-  int rs, sa, sb, smem;
-  if (!choose_rings(tile_bn(g), tile_bn(g), p, &rs, &sa, &sb, &smem)) return p;
+  p.scratch_bytes = (size_t)kStatusBytes + (size_t)p.K2p * ((g.Co + 63) / 64 * 64) * g.Kw * 2;
+  int rs, sa, sb, vg, smem;
+  if (!choose_rings(tile_bn(g), tile_bn(g), g.Kw, p, &rs, &sa, &sb, &vg, &smem)) return p;
   p.eligible = true;
   return p;
 }
@@ -790,23 +816,28 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, 
   const char* pair_env = getenv("IM2WIN_F16_PAIR");     // testing aid: 0 = never pair CTAs
   const bool pair = bn == 256 && !(pair_env && pair_env[0] == '0');
 
+  const int ncog = (g.Co + 63) / 64;                    // groups of 64 output channels
   {
     const unsigned gx = (unsigned)((plan.K2p + 255) / 256);
-    dim3 grid(gx > 64 ? 64 : gx, (unsigned)(g.Co < 32768 ? g.Co : 32768), (unsigned)(g.Kw < 65535 ? g.Kw : 65535));
+    dim3 grid(gx > 64 ? 64 : gx, (unsigned)(ncog * 64 < 32768 ? ncog * 64 : 32768),
+              (unsigned)(g.Kw < 65535 ? g.Kw : 65535));
     pack_f16_mat_kernel<<<grid, 256, 0, stream>>>(filter, fp, reinterpret_cast<uint32_t*>(base), g.C, g.Co, g.Kh, g.Kw,
-                                                  (int)plan.K2p);
+                                                  (int)plan.K2p, ncog);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
 
-  // Filter as Fp3[v][co][k2p] halves: a 3-D tensor (k2 fastest), one box = 64 k2 x BN channels of one v.
+  // Packed filter as a 2-D array of 2 KB rows (256 eight-byte elements); one box = this CTA's
+  // rows of one (v, k-block): 128 bytes per output channel.
   CUtensorMap fmap;
-  const cuuint64_t dims[3] = {(cuuint64_t)plan.K2p, (cuuint64_t)g.Co, (cuuint64_t)g.Kw};
-  const cuuint64_t strides[2] = {(cuuint64_t)plan.K2p * 2, (cuuint64_t)plan.K2p * 2 * (cuuint64_t)g.Co};
-  const cuuint32_t box[3] = {(cuuint32_t)KB, (cuuint32_t)(pair ? bn / 2 : bn), 1};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  CUresult cr = encode(&fmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, fp, dims, strides, box, estr,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+  const int b_rows = pair ? bn / 2 : bn;
+  const cuuint64_t frows_total = (cuuint64_t)g.Kw * plan.num_kb * ncog * 4;
+  const cuuint64_t dims[2] = {256, frows_total};
+  const cuuint64_t strides[1] = {2048};
+  const cuuint32_t box[2] = {256, (cuuint32_t)(b_rows / 16)};
+  const cuuint32_t estr[2] = {1, 1};
+  CUresult cr = encode(&fmap, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, fp, dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
 
@@ -834,7 +865,9 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, 
   q.raw_stage_bytes = plan.raw_stage_bytes; q.a_stage_bytes = plan.a_stage_bytes;
   q.magic_kh = magic16(g.Kh); q.magic_s = magic16(g.s);
   q.rs = q.sa = q.sb = 2;
+  q.vg = 1;
   q.ntm = q.nwork = 0;
+  q.frows = ncog * 4;
   if (pair) return launch_pair(fmap, wmap, q, plan, g.Co, stream);
   if (bn == 64) return launch_bn<64>(fmap, wmap, q, plan, g.Co, stream);
   if (bn == 128) return launch_bn<128>(fmap, wmap, q, plan, g.Co, stream);

@@ -294,6 +294,12 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 }
 // TMA tile load inside a CTA pair: the destination is this CTA's shared memory, the mbarrier may
 // be the peer's (a shared::cluster address).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster)
+      : "memory");
+}
 __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
                                                  uint32_t bar_cluster) {
   asm volatile(
