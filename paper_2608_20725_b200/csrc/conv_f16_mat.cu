@@ -600,10 +600,12 @@ conv_f16_mat_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
   conv_f16_mat_body<BN, false>(fmap, wmap, q);
 }
 
-// CTA-pair form for wide channel tiles (Co > 128): clusters of two CTAs.
+// CTA-pair form: clusters of two CTAs share every MMA (half as many MMA instructions per tile,
+// half the filter tile per CTA).
+template <int BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 conv_f16_mat_pair_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_constant__ CUtensorMap wmap, MatParams q) {
-  conv_f16_mat_body<256, true>(fmap, wmap, q);
+  conv_f16_mat_body<BN, true>(fmap, wmap, q);
 }
 
 // Filter pack for this kernel (paper Section "Im2win Convolution": height before width; here
@@ -668,9 +670,9 @@ bool choose_rings(int bn, int b_rows, int kw, const MatPlan& plan, int* rs, int*
     for (int g = kw; g >= 1; --g) {
       const int b = g * tile;
       if (2 * a + 2 * r + 2 * b + fixed > budget) continue;
+      const int rr = (2 * a + 3 * r + 2 * b + fixed <= budget) ? 3 : 2;
       int bb = 2;
-      while (bb < MAX_STAGES && (bb + 1) * g <= 12 && 2 * a + 2 * r + (bb + 1) * b + fixed <= budget) ++bb;
-      const int rr = (2 * a + 3 * r + bb * b + fixed <= budget) ? 3 : 2;
+      while (bb < MAX_STAGES && (bb + 1) * g <= 12 && 2 * a + rr * r + (bb + 1) * b + fixed <= budget) ++bb;
       *rs = rr; *sa = 2; *sb = bb; *vg = g;
       *smem_bytes = 2 * a + rr * r + bb * b + fixed + 1024;
       return true;
@@ -698,17 +700,18 @@ cudaError_t launch_bn(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParam
   return cudaGetLastError();
 }
 
-// CTA-pair launch (Co > 128): clusters of two CTAs, as many as can be resident at once.
+// CTA-pair launch: clusters of two CTAs, as many as can be resident at once.
+template <int BN>
 cudaError_t launch_pair(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParams q, const MatPlan& plan, int co,
                         cudaStream_t stream) {
   int smem_bytes = 0;
-  if (!choose_rings(256, 128, q.Kw, plan, &q.rs, &q.sa, &q.sb, &q.vg, &smem_bytes)) return cudaErrorInvalidValue;
+  if (!choose_rings(256, BN / 2, q.Kw, plan, &q.rs, &q.sa, &q.sb, &q.vg, &smem_bytes)) return cudaErrorInvalidValue;
   cudaError_t e =
-      cudaFuncSetAttribute(conv_f16_mat_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+      cudaFuncSetAttribute(conv_f16_mat_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
   const int64_t ntm = (plan.VQ + TILE_M - 1) / TILE_M;
   const int64_t ntp = (ntm + 1) / 2;                   // pairs of position tiles
-  const int64_t nwork = ntp * ((co + 255) / 256);
+  const int64_t nwork = ntp * ((co + BN - 1) / BN);
   if (nwork >= ((int64_t)1 << 30)) return cudaErrorInvalidValue;
   q.ntm = (int32_t)ntp;
   q.nwork = (int32_t)nwork;
@@ -723,12 +726,12 @@ cudaError_t launch_pair(const CUtensorMap& fmap, const CUtensorMap& wmap, MatPar
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int clusters = 0;
-  e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_mat_pair_kernel, &cfg);
+  e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_mat_pair_kernel<BN>, &cfg);
   if (e != cudaSuccess) return e;
   if (clusters < 1) return cudaErrorInvalidValue;
   if (clusters > 74) clusters = 74;
   if ((int64_t)clusters > nwork) clusters = (int)nwork;
-  conv_f16_mat_pair_kernel<<<2 * clusters, NUM_THREADS, smem_bytes, stream>>>(fmap, wmap, q);
+  conv_f16_mat_pair_kernel<BN><<<2 * clusters, NUM_THREADS, smem_bytes, stream>>>(fmap, wmap, q);
   return cudaGetLastError();
 }
 
@@ -814,6 +817,7 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, 
   uint16_t* fp = reinterpret_cast<uint16_t*>(base + kStatusBytes);
   const int bn = tile_bn(g);
   const char* pair_env = getenv("IM2WIN_F16_PAIR");     // testing aid: 0 = never pair CTAs
+  // measured: pairing pays for 256-channel tiles (the filter tile halves); narrow tiles gain nothing
   const bool pair = bn == 256 && !(pair_env && pair_env[0] == '0');
 
   const int ncog = (g.Co + 63) / 64;                    // groups of 64 output channels
@@ -868,7 +872,7 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, 
   q.vg = 1;
   q.ntm = q.nwork = 0;
   q.frows = ncog * 4;
-  if (pair) return launch_pair(fmap, wmap, q, plan, g.Co, stream);
+  if (pair) return launch_pair<256>(fmap, wmap, q, plan, g.Co, stream);
   if (bn == 64) return launch_bn<64>(fmap, wmap, q, plan, g.Co, stream);
   if (bn == 128) return launch_bn<128>(fmap, wmap, q, plan, g.Co, stream);
   return launch_bn<256>(fmap, wmap, q, plan, g.Co, stream);
