@@ -40,17 +40,23 @@ SMALL = [
     L("uncovered_cols", 1, 3, 10, 12, 4, 3, 4, 3, 0, 24),       # (Wp - Kw) % s != 0: trailing columns never read
     L("pair_odd", 3, 16, 18, 22, 260, 3, 3, 1, 1, 25),          # Co > 256 and an odd number of position tiles (CTA pairs)
     L("pair_s2", 2, 24, 16, 14, 200, 3, 3, 2, 1, 26),           # CTA pairs with stride 2
+    L("vec_w16", 2, 5, 11, 16, 6, 3, 3, 1, 1, 27),              # W a multiple of 8: vector-load transform, odd pad
+    L("vec_w24_p2", 3, 3, 9, 24, 4, 5, 5, 1, 2, 28),            # ... even pad, Kh = 5
+    L("vec_w32_k1", 2, 7, 6, 32, 9, 1, 1, 1, 0, 29),            # ... Kh = 1, no pad
 ]
 
 
 @pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
 @pytest.mark.parametrize("es", [4, 2])
-@pytest.mark.parametrize("kernel", ["strips", "columns"])
+@pytest.mark.parametrize("kernel", ["strips", "strips-scalar", "columns"])
 def test_transform_bit_exact_small(layer, es, kernel, monkeypatch):
-    """Both transform kernels (the strip kernel the library picks, and the column kernel it
-    falls back to for very long strips) against the oracle, bit for bit."""
+    """All transform kernels (the strip kernel the library picks, with vector loads where the
+    row length allows and element-wise otherwise, and the column kernel it falls back to for
+    very long strips) against the oracle, bit for bit."""
     if kernel == "columns":
         monkeypatch.setenv("IM2WIN_TRANSFORM_KERNEL", "columns")
+    if kernel == "strips-scalar":
+        monkeypatch.setenv("IM2WIN_TRANSFORM_SCALAR", "1")
     dims = layer.dims()
     x, _ = workloads.make_inputs(layer)
     xb = x if es == 4 else x.half()
