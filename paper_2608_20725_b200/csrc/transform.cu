@@ -57,6 +57,14 @@ __device__ __forceinline__ uint4 ld_if128(const void* p, bool ok) {
   return v;
 }
 
+__device__ __forceinline__ uint2 ld_if64(const void* p, bool ok) {
+  uint2 v = make_uint2(0u, 0u);
+  asm("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %3, 0;\n\t@p ld.global.nc.v2.b32 {%0, %1}, [%2];\n\t}"
+      : "+r"(v.x), "+r"(v.y)
+      : "l"(p), "r"((int)ok));
+  return v;
+}
+
 struct TransformParams {
   int32_t H, W, Wp, Kh, s, p, Ho;
   int32_t cols_per_cta;   // multiple of 8, so every CTA's output range starts 16-byte aligned
@@ -149,33 +157,26 @@ constexpr int kStripThreads = 256;
 // items per thread whose loads are issued before the first store: fewer for tall kernels (registers)
 __host__ __device__ constexpr int strip_unroll(int kh, int es) { return (4 / es) * kh > 10 ? 2 : 4; }
 
-// Element n (in output order) of a run of 16/ES columns whose KH rows were loaded as one 16-byte
-// vector each: row n % KH, column n / KH.
-template <int KH>
-__device__ __forceinline__ uint32_t run_word32(const uint4 (&r)[KH], int n) {
-  const uint4& v = r[n % KH];
-  const int i = n / KH;
-  return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
+// Output order of a run of columns whose KH rows were loaded as one vector of NW 32-bit words
+// each (r[row][word]): element n of the run is row n % KH, column n / KH.
+template <int KH, int NW>
+__device__ __forceinline__ uint32_t run_word32(const uint32_t (&r)[KH][NW], int n) {
+  return r[n % KH][n / KH];
 }
-template <int KH>
-__device__ __forceinline__ uint32_t run_half_word(const uint4 (&r)[KH], int n) {   // the word holding half n
-  const uint4& v = r[n % KH];
-  const int i = (n / KH) >> 1;
-  return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
-}
-// 32-bit word made of halves n0 (low) and n1 (high) of the run.
-template <int KH>
-__device__ __forceinline__ uint32_t run_pair16(const uint4 (&r)[KH], int n0, int n1) {
-  const uint32_t a = run_half_word<KH>(r, n0), b = run_half_word<KH>(r, n1);
+// 32-bit word made of halves n0 (low) and n1 (high) of a run of 2-byte elements.
+template <int KH, int NW>
+__device__ __forceinline__ uint32_t run_pair16(const uint32_t (&r)[KH][NW], int n0, int n1) {
+  const uint32_t a = r[n0 % KH][(n0 / KH) >> 1], b = r[n1 % KH][(n1 / KH) >> 1];
   const uint32_t sel = (((n0 / KH) & 1) ? 0x32u : 0x10u) | (((n1 / KH) & 1) ? 0x7600u : 0x5400u);
   return __byte_perm(a, b, sel);
 }
 
-// VEC: the input rows are read as aligned 16-byte vectors (W a multiple of 16/ES elements, so that
-// every row starts 16-byte aligned): one load per kernel row brings 16/ES columns, which leave as a
-// contiguous run of KH*16/ES output elements.  Per element that is well under half the
-// instructions of the element-wise form, which is what bounds this kernel.
-template <typename E, int KH, bool VEC>
+// VB > 0: the input rows are read as aligned VB-byte vectors (16 or 8; the row length must be a
+// multiple of VB bytes so that every row starts aligned): one load per kernel row brings VB/ES
+// columns, which leave as a contiguous run of KH*VB/ES output elements.  Per element that is
+// well under half the instructions of the element-wise form (VB = 0), which is what bounds
+// this kernel.
+template <typename E, int KH, int VB>
 __global__ void __launch_bounds__(kStripThreads)
 transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParams q) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -208,9 +209,10 @@ transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParam
     const int sbyte = ls * q.L * ES;              // byte offset of the strip inside the staging
     unsigned char* dst_strip = stage + sbyte;
     const bool word_ok = ((mis + sbyte) & 3) == 0;
-    if constexpr (VEC) {
-      constexpr int VL = 16 / ES;                 // columns per vector
-      constexpr int VU = 2;                       // vectors per thread whose loads precede the first store
+    if constexpr (VB > 0) {
+      constexpr int VL = VB / ES;                 // columns per vector
+      constexpr int NW = VB / 4;                  // 32-bit words per vector
+      constexpr int VU = 32 / VB;                 // vectors per thread whose loads precede the first store
       constexpr int RUN = VL * KH;                // output elements per vector
       const int nvec = q.W / VL;
       // padded columns on both sides of the strip: p*KH zeros each
@@ -221,14 +223,21 @@ transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParam
       }
       const bool aligned4 = ES == 4 || ((mis + sbyte + padel * ES) & 3) == 0;
       for (int vb = gl; vb < nvec; vb += G * VU) {
-        uint4 r[VU][KH];
+        uint32_t r[VU][KH][NW];
 #pragma unroll
         for (int j = 0; j < VU; ++j) {
           const int vi = vb + j * G;
 #pragma unroll
           for (int u = 0; u < KH; ++u) {
             const int h = h0 + u;
-            r[j][u] = ld_if128(src + (int64_t)h * q.W + vi * VL, vi < nvec && (unsigned)h < (unsigned)q.H);
+            const bool ok = vi < nvec && (unsigned)h < (unsigned)q.H;
+            if constexpr (VB == 16) {
+              const uint4 t = ld_if128(src + (int64_t)h * q.W + vi * VL, ok);
+              r[j][u][0] = t.x; r[j][u][1] = t.y; r[j][u][2] = t.z; r[j][u][3] = t.w;
+            } else {
+              const uint2 t = ld_if64(src + (int64_t)h * q.W + vi * VL, ok);
+              r[j][u][0] = t.x; r[j][u][1] = t.y;
+            }
           }
         }
 #pragma unroll
@@ -238,18 +247,19 @@ transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParam
           unsigned char* d = dst_strip + (size_t)(vi * VL + q.p) * KH * ES;
           if constexpr (ES == 4) {
 #pragma unroll
-            for (int n = 0; n < RUN; ++n) reinterpret_cast<uint32_t*>(d)[n] = run_word32<KH>(r[j], n);
+            for (int n = 0; n < RUN; ++n) reinterpret_cast<uint32_t*>(d)[n] = run_word32<KH, NW>(r[j], n);
           } else {
             if (aligned4) {
 #pragma unroll
-              for (int w = 0; w < RUN / 2; ++w) reinterpret_cast<uint32_t*>(d)[w] = run_pair16<KH>(r[j], 2 * w, 2 * w + 1);
+              for (int w = 0; w < RUN / 2; ++w)
+                reinterpret_cast<uint32_t*>(d)[w] = run_pair16<KH, NW>(r[j], 2 * w, 2 * w + 1);
             } else {
               // the run starts on an odd half: one half, RUN/2 - 1 words, one half
-              reinterpret_cast<uint16_t*>(d)[0] = (uint16_t)(run_pair16<KH>(r[j], 0, 0) & 0xffffu);
+              reinterpret_cast<uint16_t*>(d)[0] = (uint16_t)(run_pair16<KH, NW>(r[j], 0, 0) & 0xffffu);
 #pragma unroll
               for (int w = 0; w < RUN / 2 - 1; ++w)
-                reinterpret_cast<uint32_t*>(d + 2)[w] = run_pair16<KH>(r[j], 2 * w + 1, 2 * w + 2);
-              reinterpret_cast<uint16_t*>(d)[RUN - 1] = (uint16_t)(run_pair16<KH>(r[j], RUN - 1, RUN - 1) & 0xffffu);
+                reinterpret_cast<uint32_t*>(d + 2)[w] = run_pair16<KH, NW>(r[j], 2 * w + 1, 2 * w + 2);
+              reinterpret_cast<uint16_t*>(d)[RUN - 1] = (uint16_t)(run_pair16<KH, NW>(r[j], RUN - 1, RUN - 1) & 0xffffu);
             }
           }
         }
@@ -334,7 +344,7 @@ transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParam
 // staged; measured faster than the column kernel for Kh <= 5 and slower beyond (register
 // pressure of the unrolled gathers), so taller kernels keep the column kernel.
 template <typename E>
-bool plan_strips(const Geometry& g, StripParams* q, size_t* smem_bytes, bool* vec) {
+bool plan_strips(const Geometry& g, StripParams* q, size_t* smem_bytes, int* vec) {
   constexpr int ES = (int)sizeof(E);
   if (!(g.Kh == 1 || g.Kh == 3 || g.Kh == 5)) return false;
   const int64_t strip_bytes = g.strip * ES;
@@ -346,11 +356,15 @@ bool plan_strips(const Geometry& g, StripParams* q, size_t* smem_bytes, bool* ve
   q->L = (int32_t)g.strip;
   q->total_strips = total_strips;
   q->strips_per_cta = r;
-  // vector loads: rows must start 16-byte aligned; measured faster for Kh <= 3, slower for Kh = 5
+  // vector loads: rows must start 16- (or 8-) byte aligned; measured faster for Kh <= 3, slower for Kh = 5
   // (registers); IM2WIN_TRANSFORM_SCALAR forces the element-wise form (a testing aid)
-  *vec = (g.W % (16 / ES)) == 0 && g.Kh <= 3 && getenv("IM2WIN_TRANSFORM_SCALAR") == nullptr;
-  const int items = *vec ? g.W / (16 / ES) : (g.Wp + (4 / ES) - 1) / (4 / ES);
-  const int unroll = *vec ? 2 : strip_unroll(g.Kh, ES);
+  *vec = 0;
+  if (g.Kh <= 3 && getenv("IM2WIN_TRANSFORM_SCALAR") == nullptr) {
+    if ((g.W * ES) % 16 == 0) *vec = 16;
+    else if (ES == 2 && (g.W * ES) % 8 == 0) *vec = 8;      // 8-byte vectors of 4-byte elements measured slower
+  }
+  const int items = *vec ? g.W * ES / *vec : (g.Wp + (4 / ES) - 1) / (4 / ES);
+  const int unroll = *vec ? 32 / *vec : strip_unroll(g.Kh, ES);
   const int per_group = (items + unroll - 1) / unroll;
   int grp = 1;
   while (grp < kStripThreads && grp < per_group) grp *= 2;
@@ -360,7 +374,7 @@ bool plan_strips(const Geometry& g, StripParams* q, size_t* smem_bytes, bool* ve
 }
 
 template <typename E>
-cudaError_t launch_strips(const void* x, void* window, const StripParams& q, size_t smem, int Kh, bool vec,
+cudaError_t launch_strips(const void* x, void* window, const StripParams& q, size_t smem, int Kh, int vec,
                           cudaStream_t stream) {
   const int64_t blocks = (q.total_strips + q.strips_per_cta - 1) / q.strips_per_cta;
   const E* xi = static_cast<const E*>(x);
@@ -373,16 +387,12 @@ cudaError_t launch_strips(const void* x, void* window, const StripParams& q, siz
     kernel<<<(unsigned)blocks, kStripThreads, smem, stream>>>(xi, wo, q);
     return cudaGetLastError();
   };
-  if (vec) {
-    switch (Kh) {
-      case 1: return run(transform_strips_kernel<E, 1, true>);
-      default: return run(transform_strips_kernel<E, 3, true>);
-    }
-  }
+  if (vec == 16) return Kh == 1 ? run(transform_strips_kernel<E, 1, 16>) : run(transform_strips_kernel<E, 3, 16>);
+  if (vec == 8) return Kh == 1 ? run(transform_strips_kernel<E, 1, 8>) : run(transform_strips_kernel<E, 3, 8>);
   switch (Kh) {
-    case 1: return run(transform_strips_kernel<E, 1, false>);
-    case 3: return run(transform_strips_kernel<E, 3, false>);
-    default: return run(transform_strips_kernel<E, 5, false>);
+    case 1: return run(transform_strips_kernel<E, 1, 0>);
+    case 3: return run(transform_strips_kernel<E, 3, 0>);
+    default: return run(transform_strips_kernel<E, 5, 0>);
   }
 }
 
@@ -428,7 +438,7 @@ cudaError_t launch_transform(const void* x, void* window, const Geometry& g, int
   const bool columns = force && strcmp(force, "columns") == 0;
   StripParams q;
   size_t smem = 0;
-  bool vec = false;
+  int vec = 0;
   if (elem_bytes == 4) {
     if (!columns && plan_strips<uint32_t>(g, &q, &smem, &vec))
       return launch_strips<uint32_t>(x, window, q, smem, g.Kh, vec, stream);

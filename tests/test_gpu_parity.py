@@ -43,6 +43,8 @@ SMALL = [
     L("vec_w16", 2, 5, 11, 16, 6, 3, 3, 1, 1, 27),              # W a multiple of 8: vector-load transform, odd pad
     L("vec_w24_p2", 3, 3, 9, 24, 4, 5, 5, 1, 2, 28),            # ... even pad, Kh = 5
     L("vec_w32_k1", 2, 7, 6, 32, 9, 1, 1, 1, 0, 29),            # ... Kh = 1, no pad
+    L("vec_w12", 2, 4, 10, 12, 5, 3, 3, 1, 1, 30),              # W = 12: 8-byte vectors for fp16, 16-byte for fp32
+    L("vec_w6_s2", 2, 3, 9, 6, 4, 3, 3, 2, 1, 31),              # W = 6: 8-byte vectors for fp32 only, stride 2
 ]
 
 
