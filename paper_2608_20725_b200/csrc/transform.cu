@@ -212,7 +212,7 @@ transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParam
     if constexpr (VB > 0) {
       constexpr int VL = VB / ES;                 // columns per vector
       constexpr int NW = VB / 4;                  // 32-bit words per vector
-      constexpr int VU = 32 / VB;                 // vectors per thread whose loads precede the first store
+      constexpr int VU = KH <= 3 ? 32 / VB : 1;   // vectors per thread whose loads precede the first store
       constexpr int RUN = VL * KH;                // output elements per vector
       const int nvec = q.W / VL;
       // padded columns on both sides of the strip: p*KH zeros each
@@ -346,7 +346,7 @@ transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParam
 template <typename E>
 bool plan_strips(const Geometry& g, StripParams* q, size_t* smem_bytes, int* vec) {
   constexpr int ES = (int)sizeof(E);
-  if (!(g.Kh == 1 || g.Kh == 3 || g.Kh == 5)) return false;
+  if (!(g.Kh == 1 || g.Kh == 3 || g.Kh == 5 || g.Kh == 7 || g.Kh == 11)) return false;
   const int64_t strip_bytes = g.strip * ES;
   const int64_t total_strips = (int64_t)g.N * g.C * g.Ho;
   if (strip_bytes > 64 * 1024 || total_strips >= ((int64_t)1 << 31)) return false;
@@ -356,15 +356,16 @@ bool plan_strips(const Geometry& g, StripParams* q, size_t* smem_bytes, int* vec
   q->L = (int32_t)g.strip;
   q->total_strips = total_strips;
   q->strips_per_cta = r;
-  // vector loads: rows must start 16- (or 8-) byte aligned; measured faster for Kh <= 3, slower for Kh = 5
-  // (registers); IM2WIN_TRANSFORM_SCALAR forces the element-wise form (a testing aid)
+  // vector loads: rows must start 16- (or 8-) byte aligned; IM2WIN_TRANSFORM_SCALAR forces the
+  // element-wise form (a testing aid)
   *vec = 0;
-  if (g.Kh <= 3 && getenv("IM2WIN_TRANSFORM_SCALAR") == nullptr) {
+  if (getenv("IM2WIN_TRANSFORM_SCALAR") == nullptr && (ES == 2 || g.Kh <= 3)) {   // fp32, Kh > 3: measured slower
     if ((g.W * ES) % 16 == 0) *vec = 16;
     else if (ES == 2 && (g.W * ES) % 8 == 0) *vec = 8;      // 8-byte vectors of 4-byte elements measured slower
   }
   const int items = *vec ? g.W * ES / *vec : (g.Wp + (4 / ES) - 1) / (4 / ES);
-  const int unroll = *vec ? 32 / *vec : strip_unroll(g.Kh, ES);
+  const int unroll = *vec ? (g.Kh <= 3 ? 32 / *vec : 1) : strip_unroll(g.Kh, ES);
+  if (!*vec && g.Kh > 5) return false;          // element-wise strips are slower than columns for tall kernels
   const int per_group = (items + unroll - 1) / unroll;
   int grp = 1;
   while (grp < kStripThreads && grp < per_group) grp *= 2;
@@ -387,8 +388,24 @@ cudaError_t launch_strips(const void* x, void* window, const StripParams& q, siz
     kernel<<<(unsigned)blocks, kStripThreads, smem, stream>>>(xi, wo, q);
     return cudaGetLastError();
   };
-  if (vec == 16) return Kh == 1 ? run(transform_strips_kernel<E, 1, 16>) : run(transform_strips_kernel<E, 3, 16>);
-  if (vec == 8) return Kh == 1 ? run(transform_strips_kernel<E, 1, 8>) : run(transform_strips_kernel<E, 3, 8>);
+  if (vec == 16) {
+    switch (Kh) {
+      case 1: return run(transform_strips_kernel<E, 1, 16>);
+      case 3: return run(transform_strips_kernel<E, 3, 16>);
+      case 5: return run(transform_strips_kernel<E, 5, 16>);
+      case 7: return run(transform_strips_kernel<E, 7, 16>);
+      default: return run(transform_strips_kernel<E, 11, 16>);
+    }
+  }
+  if (vec == 8) {
+    switch (Kh) {
+      case 1: return run(transform_strips_kernel<E, 1, 8>);
+      case 3: return run(transform_strips_kernel<E, 3, 8>);
+      case 5: return run(transform_strips_kernel<E, 5, 8>);
+      case 7: return run(transform_strips_kernel<E, 7, 8>);
+      default: return run(transform_strips_kernel<E, 11, 8>);
+    }
+  }
   switch (Kh) {
     case 1: return run(transform_strips_kernel<E, 1, 0>);
     case 3: return run(transform_strips_kernel<E, 3, 0>);

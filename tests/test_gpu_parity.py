@@ -44,7 +44,9 @@ SMALL = [
     L("vec_w24_p2", 3, 3, 9, 24, 4, 5, 5, 1, 2, 28),            # ... even pad, Kh = 5
     L("vec_w32_k1", 2, 7, 6, 32, 9, 1, 1, 1, 0, 29),            # ... Kh = 1, no pad
     L("vec_w12", 2, 4, 10, 12, 5, 3, 3, 1, 1, 30),              # W = 12: 8-byte vectors for fp16, 16-byte for fp32
-    L("vec_w6_s2", 2, 3, 9, 6, 4, 3, 3, 2, 1, 31),              # W = 6: 8-byte vectors for fp32 only, stride 2
+    L("vec_w6_s2", 2, 3, 9, 6, 4, 3, 3, 2, 1, 31),              # W = 6: no vectors (12- / 24-byte rows), stride 2
+    L("vec_w16_k7", 2, 3, 20, 16, 4, 7, 7, 2, 3, 32),           # tall kernel with vector loads (fp16), stride 2
+    L("vec_w24_k11", 1, 2, 26, 24, 3, 11, 11, 1, 5, 33),        # Kh = 11 with vector loads (fp16)
 ]
 
 
