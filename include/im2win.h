@@ -15,7 +15,8 @@
  * General conventions
  *   - Every data pointer is a DEVICE pointer unless its name ends in _host.
  *     The caller owns all memory; the library allocates no device memory and
- *     keeps no per-call state.  Buffers must stay valid until the work queued
+ *     keeps no per-call state (per device it keeps two auxiliary streams, see
+ *     im2win_layer_forward_host, and the array of im2win_conv_f32_static).  Buffers must stay valid until the work queued
  *     on `cuda_stream` has completed.
  *   - All calls are asynchronous on `cuda_stream` (a cudaStream_t passed as
  *     void*; NULL is the default stream), except where stated.
@@ -145,6 +146,13 @@ im2win_status im2win_layer_workspace_size(const im2win_shape* shape, im2win_dtyp
  * the copies to overlap nothing else; they must stay valid until the stream
  * has been synchronised by the caller.  `device_workspace` is a 256-byte
  * aligned device buffer of at least im2win_layer_workspace_size bytes.
+ * Layers that move more than 8 MB are processed in four batch chunks: the
+ * upload of a chunk, the kernels of the previous one and the download of the
+ * one before overlap.  The copies of such a call run on two auxiliary streams
+ * that the library creates once per device and keeps; they are ordered after
+ * everything queued on `cuda_stream` before the call, and `cuda_stream` waits
+ * for the last of them, so synchronising `cuda_stream` still completes the
+ * call.  The result does not depend on the chunking.
  */
 im2win_status im2win_layer_forward_host(const void* x_host, const void* filter_host, float* y_host,
                                         void* device_workspace, size_t device_workspace_bytes,

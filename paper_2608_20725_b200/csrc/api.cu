@@ -4,6 +4,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace im2win {
@@ -210,6 +212,30 @@ im2win_status im2win_check_status(const void* scratch, void* cuda_stream) {
 }
 
 namespace {
+// Two auxiliary streams per device for the chunked host-to-host path (created on first use and kept
+// for the life of the process; the only state the library keeps besides the static scratch array).
+struct AuxStreams {
+  cudaStream_t in, out;
+};
+bool get_aux_streams(AuxStreams* a) {
+  static std::mutex mu;
+  static AuxStreams cache[64];
+  static bool have[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!have[dev]) {
+    if (cudaStreamCreateWithFlags(&cache[dev].in, cudaStreamNonBlocking) != cudaSuccess) return false;
+    if (cudaStreamCreateWithFlags(&cache[dev].out, cudaStreamNonBlocking) != cudaSuccess) {
+      cudaStreamDestroy(cache[dev].in);
+      return false;
+    }
+    have[dev] = true;
+  }
+  *a = cache[dev];
+  return true;
+}
+
 struct LayerLayout {
   size_t x_off, f_off, win_off, scratch_off, y_off, total;
   size_t x_bytes, f_bytes, win_bytes, scratch_bytes, y_bytes;
@@ -260,17 +286,68 @@ im2win_status im2win_layer_forward_host(const void* x_host, const void* filter_h
   if (device_workspace_bytes < L.total) return IM2WIN_ERR_WORKSPACE_TOO_SMALL;
   unsigned char* ws = static_cast<unsigned char*>(device_workspace);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (cudaMemcpyAsync(ws + L.x_off, x_host, L.x_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+  const size_t es = dtype == IM2WIN_F32 ? 4 : 2;
+
+  // Large layers are cut into batch chunks so that the upload of chunk i+1, the kernels of chunk
+  // i and the download of chunk i-1 overlap (the two copy directions run concurrently on the
+  // link).  Chunks start at images whose slices of x, window and y are 16-byte aligned.
+  const size_t x_img = (size_t)g.C * g.H * g.W * es, w_img = (size_t)g.img_stride * es,
+               y_img = (size_t)g.Co * g.Ho * g.Wo * 4;
+  int unit = 1;                                   // images per alignment unit
+  while (unit <= 8 && ((unit * x_img) % 16 || (unit * w_img) % 16 || (unit * y_img) % 16)) unit *= 2;
+  int nchunk = 1;
+  AuxStreams aux{};
+  if (unit <= 8 && g.N >= 4 * unit && L.x_bytes + L.y_bytes >= ((size_t)8 << 20) && get_aux_streams(&aux)) nchunk = 4;
+  if (nchunk == 1) {
+    if (cudaMemcpyAsync(ws + L.x_off, x_host, L.x_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      return IM2WIN_ERR_CUDA;
+    if (cudaMemcpyAsync(ws + L.f_off, filter_host, L.f_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      return IM2WIN_ERR_CUDA;
+    st = im2win_transform(ws + L.x_off, ws + L.win_off, shape, dtype, cuda_stream);
+    if (st != IM2WIN_OK) return st;
+    st = conv_common(ws + L.win_off, ws + L.f_off, reinterpret_cast<float*>(ws + L.y_off), ws + L.scratch_off,
+                     L.scratch_bytes, shape, dtype, cuda_stream);
+    if (st != IM2WIN_OK) return st;
+    if (cudaMemcpyAsync(y_host, ws + L.y_off, L.y_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+      return IM2WIN_ERR_CUDA;
+    return IM2WIN_OK;
+  }
+
+  // Everything the auxiliary streams do is ordered after the work already queued on `stream`, and
+  // `stream` ends up waiting for the last download, so the caller still only synchronises `stream`.
+  cudaEvent_t ev;
+  auto fence = [&](cudaStream_t from, cudaStream_t to) -> bool {      // `to` waits for what `from` has queued
+    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return false;
+    const bool ok = cudaEventRecord(ev, from) == cudaSuccess && cudaStreamWaitEvent(to, ev, 0) == cudaSuccess;
+    cudaEventDestroy(ev);                                              // released once it has completed
+    return ok;
+  };
+  if (!fence(stream, aux.in) || !fence(stream, aux.out)) return IM2WIN_ERR_CUDA;
+  if (cudaMemcpyAsync(ws + L.f_off, filter_host, L.f_bytes, cudaMemcpyHostToDevice, aux.in) != cudaSuccess)
     return IM2WIN_ERR_CUDA;
-  if (cudaMemcpyAsync(ws + L.f_off, filter_host, L.f_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
-    return IM2WIN_ERR_CUDA;
-  st = im2win_transform(ws + L.x_off, ws + L.win_off, shape, dtype, cuda_stream);
-  if (st != IM2WIN_OK) return st;
-  st = conv_common(ws + L.win_off, ws + L.f_off, reinterpret_cast<float*>(ws + L.y_off), ws + L.scratch_off,
-                   L.scratch_bytes, shape, dtype, cuda_stream);
-  if (st != IM2WIN_OK) return st;
-  if (cudaMemcpyAsync(y_host, ws + L.y_off, L.y_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
-    return IM2WIN_ERR_CUDA;
+  const int per = ((g.N + nchunk - 1) / nchunk + unit - 1) / unit * unit;
+  for (int n0 = 0; n0 < g.N; n0 += per) {
+    const int n1 = n0 + per < g.N ? n0 + per : g.N;
+    im2win_shape part = *shape;
+    part.N = n1 - n0;
+    unsigned char* xd = ws + L.x_off + (size_t)n0 * x_img;
+    unsigned char* wd = ws + L.win_off + (size_t)n0 * w_img;
+    unsigned char* yd = ws + L.y_off + (size_t)n0 * y_img;
+    if (cudaMemcpyAsync(xd, static_cast<const unsigned char*>(x_host) + (size_t)n0 * x_img, (size_t)part.N * x_img,
+                        cudaMemcpyHostToDevice, aux.in) != cudaSuccess)
+      return IM2WIN_ERR_CUDA;
+    if (!fence(aux.in, stream)) return IM2WIN_ERR_CUDA;
+    st = im2win_transform(xd, wd, &part, dtype, cuda_stream);
+    if (st != IM2WIN_OK) return st;
+    st = conv_common(wd, ws + L.f_off, reinterpret_cast<float*>(yd), ws + L.scratch_off, L.scratch_bytes, &part, dtype,
+                     cuda_stream);
+    if (st != IM2WIN_OK) return st;
+    if (!fence(stream, aux.out)) return IM2WIN_ERR_CUDA;
+    if (cudaMemcpyAsync(reinterpret_cast<unsigned char*>(y_host) + (size_t)n0 * y_img, yd, (size_t)part.N * y_img,
+                        cudaMemcpyDeviceToHost, aux.out) != cudaSuccess)
+      return IM2WIN_ERR_CUDA;
+  }
+  if (!fence(aux.out, stream) || !fence(aux.in, stream)) return IM2WIN_ERR_CUDA;
   return IM2WIN_OK;
 }
 

@@ -157,6 +157,30 @@ def test_layer_forward_host_matches_device_path():
         assert np.array_equal(yh.numpy(), y_dev)
 
 
+@pytest.mark.parametrize("n", [9, 16])
+def test_layer_forward_host_in_batch_chunks(n):
+    """Layers above 8 MB go through the host path in batch chunks on auxiliary streams; the
+    result must not depend on the chunking (ragged last chunk for N = 9), also when the call is
+    repeated back to back on the same buffers."""
+    layer = L("host_chunks", n, 32, 64, 64, 64, 3, 3, 1, 1, 51)
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    for precision, tdt, code in (("f32", torch.float32, binding.F32), ("f16", torch.float16, binding.F16)):
+        y_dev, _, _ = gpu_conv(x, f, dims, precision)
+        xh = x.to(tdt).pin_memory()
+        fh = f.to(tdt).pin_memory()
+        _, _, ho, wo = binding.im2win_workspace_size(dims, code)
+        yh = torch.full((layer.N, layer.Co, ho, wo), float("nan"), dtype=torch.float32).pin_memory()
+        nbytes = binding.im2win_layer_workspace_size(dims, code)
+        whole, ws = guarded(nbytes + 192, torch.uint8, 0x33)
+        ws = ws[192:]
+        for _ in range(2):
+            binding.im2win_layer_forward_host(xh, fh, yh, ws, dims)
+        torch.cuda.synchronize()
+        assert_guards_intact(whole, nbytes + 192, 0x33)
+        assert np.array_equal(yh.numpy(), y_dev), precision
+
+
 def test_repeated_calls_are_deterministic_and_do_not_depend_on_stale_scratch():
     layer = SMALL[3]
     dims = layer.dims()
