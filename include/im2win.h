@@ -16,8 +16,9 @@
  *   - Every data pointer is a DEVICE pointer unless its name ends in _host.
  *     The caller owns all memory; the library allocates no device memory and
  *     keeps no per-call state (per device it keeps two auxiliary streams, see
- *     im2win_layer_forward_host, and the array of im2win_conv_f32_static).  Buffers must stay valid until the work queued
- *     on `cuda_stream` has completed.
+ *     im2win_layer_forward_host, and the array of im2win_conv_f32_static).
+ *     Buffers must stay valid until the work queued on `cuda_stream` has
+ *     completed.
  *   - All calls are asynchronous on `cuda_stream` (a cudaStream_t passed as
  *     void*; NULL is the default stream), except where stated.
  *   - Inputs are never written.  Output, window, scratch and input buffers
