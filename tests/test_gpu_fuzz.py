@@ -1,0 +1,60 @@
+"""Seeded random small layers through every convolution path, against the fp64 oracle (Eq. 1).
+
+The fixed cases of test_gpu_parity.py pin known tile/tail situations; this sweep looks for the
+ones nobody thought of: odd combinations of kernel size, stride, padding, channel counts and
+image sizes (tiles that cross several images, strips shorter than the kernel's boxes, one-channel
+layers, wide output-channel tails)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_20725_b200 import workloads
+from gpu_helpers import check_conv, gpu_conv, gpu_transform, oracle, oracle_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def random_layers(seed, count):
+    rng = np.random.default_rng(seed)
+    layers = []
+    while len(layers) < count:
+        kh = int(rng.choice([1, 2, 3, 3, 3, 4, 5, 7]))
+        kw = int(rng.choice([1, 2, 3, 3, 3, 4, 5, 7]))
+        s = int(rng.choice([1, 1, 1, 2, 2, 3]))
+        p = int(rng.integers(0, 3))
+        h = int(rng.integers(kh, 26))
+        w = int(rng.integers(kw, 40))
+        if rng.random() < 0.6:                 # plane pitches that are 16-byte multiples: the TMA-staged kernels
+            w = max(kw, (w + 2 * p + 7) // 8 * 8 - 2 * p)
+        if h + 2 * p < kh or w + 2 * p < kw:
+            continue
+        n = int(rng.integers(1, 5))
+        c = int(rng.choice([1, 2, 3, 5, 8, 9, 16, 17, 24, 40]))
+        co = int(rng.choice([1, 3, 8, 20, 64, 65, 130, 260]))
+        ho = (h + 2 * p - kh) // s + 1
+        wo = (w + 2 * p - kw) // s + 1
+        if n * co * ho * wo * c * kh * kw > 60_000_000:      # keep the oracle in the seconds range
+            continue
+        layers.append(workloads.Layer(f"fuzz{len(layers)}_{n}x{c}x{h}x{w}_co{co}_k{kh}x{kw}_s{s}_p{p}", n, c, h, w, co,
+                                      kh, kw, s, p, 9000 + len(layers), "normal01", "he_normal"))
+    return layers
+
+
+FUZZ = random_layers(20260725, 64)
+
+
+@pytest.mark.parametrize("layer", FUZZ, ids=lambda l: l.name)
+def test_random_layer_all_paths(layer):
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    for es, tdt in ((4, torch.float32), (2, torch.float16)):
+        raw = x.to(tdt).view(torch.int32 if es == 4 else torch.int16)
+        assert np.array_equal(gpu_transform(raw, dims), oracle.transform(raw.numpy(), dims)), (layer.name, es)
+    yr32, ar32 = oracle.conv_direct(*oracle_inputs(x, f, "f32"), dims)
+    y, _, _ = gpu_conv(x, f, dims, "f32")
+    check_conv(y, yr32, ar32, "f32", layer.name)
+    xo, fo = oracle_inputs(x, f, "f16")
+    yr16, ar16 = oracle.conv_direct(xo, fo, dims)
+    for precision in ("f16", "f16-mat", "f16-shift", "f16-gather"):
+        y, _, _ = gpu_conv(x, f, dims, precision)
+        check_conv(y, yr16, ar16, precision, layer.name)
