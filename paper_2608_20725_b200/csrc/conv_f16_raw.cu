@@ -77,15 +77,15 @@ struct Segment {            // the part of a tile that lies in one image
 
 // Splits the rows of the tile starting at virtual position q0 by image: within an image the
 // columns of one channel are contiguous in the window tensor.
-__device__ __forceinline__ int split_by_image(const RawParams& q, int64_t q0, Segment* segs) {
-  const int64_t img_rows = (int64_t)q.Ho * q.Wq;
-  int64_t n = q0 / img_rows, a = q0 - n * img_rows;
+__device__ __forceinline__ int split_by_image(const RawParams& q, int q0, Segment* segs) {
+  const int img_rows = q.Ho * q.Wq;               // VQ < 2^31 is a condition of this kernel
+  int n = q0 / img_rows, a = q0 - n * img_rows;
   int remaining = q.rows, row0 = 0, box0 = 0, g = 0;
   while (remaining > 0 && n < q.N && g < SEG_MAX) {
-    const int cnt = (int)(remaining < img_rows - a ? remaining : img_rows - a);
-    const int f0 = (int)(a * q.Kh);                      // element offset inside the channel plane
+    const int cnt = remaining < img_rows - a ? remaining : img_rows - a;
+    const int f0 = a * q.Kh;                             // element offset inside the channel plane
     const int span = (f0 & 7) + cnt * q.Kh;
-    segs[g].plane0 = (int)(n * q.C);
+    segs[g].plane0 = n * q.C;
     segs[g].x0 = f0 & ~7;
     segs[g].o0 = f0 & 7;
     segs[g].row0 = row0;
@@ -190,7 +190,7 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
     uint32_t ph = 0, rph = 0;
     TIMER_DECL;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
-      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+      const int q0 = (w % q.ntm) * TILE_M;
       int nseg = 0;
       if (lane == 0) nseg = split_by_image(q, q0, segs);
       nseg = __shfl_sync(0xffffffffu, nseg, 0);
@@ -341,7 +341,7 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
     uint32_t rph = 0;
     TIMER_DECL;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
-      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+      const int q0 = (w % q.ntm) * TILE_M;
       int nseg = 0;
       if (lane == 0) nseg = split_by_image(q, q0, segs);
       nseg = __shfl_sync(0xffffffffu, nseg, 0);
@@ -375,18 +375,18 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
     uint32_t it = 0;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
       const uint32_t buf = it & 1u;
-      const int64_t q0 = (int64_t)(w % q.ntm) * TILE_M;
+      const int q0 = (w % q.ntm) * TILE_M;
       const int n0 = (w / q.ntm) * BN;
-      const int64_t vq = q0 + lq * 32 + lane;    // accumulator row = virtual position
+      const int vq = q0 + lq * 32 + lane;        // accumulator row = virtual position
       bool valid = false;
       float* yrow = q.y;
-      if (vq < q.VQ) {
-        const int64_t sg = vq / q.Wq;
-        const int kq = (int)(vq - sg * q.Wq);
-        const int64_t n = sg / q.Ho;
-        const int ho = (int)(sg - n * q.Ho);
+      if (vq < (int)q.VQ) {
+        const int sg = vq / q.Wq;
+        const int kq = vq - sg * q.Wq;
+        const int n = sg / q.Ho;
+        const int ho = sg - n * q.Ho;
         valid = kq < q.Wo;                       // trailing columns of a strip are no output
-        yrow += (n * q.Co) * q.HoWo + ho * q.Wo + kq;
+        yrow += ((int64_t)n * q.Co) * q.HoWo + ho * q.Wo + kq;
       }
       if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -496,6 +496,7 @@ RawPlan plan_f16_raw(const Geometry& g) {
   p.K2 = (int64_t)g.C * g.Kh;
   p.K2p = (p.K2 + KB - 1) / KB * KB;
   p.VQ = (int64_t)g.N * g.Ho * p.Wq;
+  if (p.VQ >= ((int64_t)1 << 31) - 4 * TILE_M) return p;    // the kernel indexes virtual positions with 32 bits
   const int64_t img_rows = (int64_t)g.Ho * p.Wq;
   const int64_t segmax = (p.rows - 2) / img_rows + 2;     // images a tile can touch
   if (segmax > SEG_MAX) return p;
