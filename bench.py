@@ -382,9 +382,11 @@ def run_gpu_arm(args):
 
 # ------------------------------------------------------- per-layer report ----
 def time_call(fn, iters, flush):
-    """Average device time (ms) of fn over `iters` launches, each preceded by an L2 flush."""
+    """Average, best and median device time (ms) of fn over `iters` launches, each preceded by an
+    L2 flush (the paper reports the best of 50 runs; the average is what the rooflines use)."""
     total = 0.0
     best = float("inf")
+    samples = []
     for _ in range(iters):
         flush.zero_()
         # keep the GPU busy (~0.3 ms) while the host queues the events and the call, so that the
@@ -398,10 +400,12 @@ def time_call(fn, iters, flush):
         ms = e0.elapsed_time(e1)
         total += ms
         best = min(best, ms)
-    return total / iters, best
+        samples.append(ms)
+    samples.sort()
+    return total / iters, best, samples[len(samples) // 2]
 
 
-def write_report(path, peaks, peak_kind, names=None, iters=10):
+def write_report(path, peaks, peak_kind, names=None, iters=20):
     from paper_2608_20725_b200 import binding
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
     rows = []
@@ -414,13 +418,14 @@ def write_report(path, peaks, peak_kind, names=None, iters=10):
         for _ in range(3):
             runner.step()
         torch.cuda.synchronize()
-        avg, best = {}, {}
+        avg, best, median = {}, {}, {}
         for prec in layer.precisions:
             for kind, fn in (("transform", runner.transform), ("conv", runner.conv)):
                 print(f"[report]   {kind}_{prec}", file=sys.stderr, flush=True)
-                avg[f"{kind}_{prec}"], best[f"{kind}_{prec}"] = time_call(lambda: fn(prec), iters, flush)
+                key = f"{kind}_{prec}"
+                avg[key], best[key], median[key] = time_call(lambda: fn(prec), iters, flush)
             binding.im2win_check_status(runner.dev[prec]["scratch"])
-        row = {"layer": name, "dims": layer.dims(), "gflop": runner.flops / 1e9, "avg_ms": avg, "best_ms": best,
+        row = {"layer": name, "dims": layer.dims(), "gflop": runner.flops / 1e9, "avg_ms": avg, "best_ms": best, "median_ms": median,
                "kernels": kernel_rooflines(runner, avg, peaks, peak_kind), "memory": runner.memory_report()}
         rows.append(row)
         del runner
