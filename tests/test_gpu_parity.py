@@ -222,6 +222,25 @@ def test_full_size_mat_kernel_sampled(name):
     check_conv(y[-1:], yi, ai, "f16-mat", layer.name + " last image")
 
 
+@pytest.mark.parametrize("name", ["cfg5k7", "cfg5k11"])
+def test_full_size_wide_kernels_sampled(name):
+    """The two largest sweep layers at benchmark size (K = 12 544 and 30 976): sampled outputs
+    only, the oracle needs minutes for a whole image of these."""
+    layer = workloads.LAYERS[name]
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    ho, wo = oracle.out_dims(dims)
+    total = layer.N * layer.Co * ho * wo
+    rng = np.random.default_rng(layer.seed + 11)
+    idx = np.concatenate([rng.integers(0, total, 2048), [0, total - 1, wo - 1, ho * wo - 1, total - ho * wo]])
+    for precision in layer.precisions:
+        y, _, _ = gpu_conv(x, f, dims, precision)
+        xo, fo = oracle_inputs(x, f, precision)
+        yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
+        check_conv(y.reshape(-1)[idx], yr, ar, precision, layer.name)
+        del y
+
+
 # ------------------------------------------------------------ full-size layers ----
 FULL = [workloads.LAYERS[k] for k in ("cfg2", "cfg3", "cfg4a", "cfg4b", "cfg4c", "cfg5k1", "cfg5k3", "cfg5k5")]
 
