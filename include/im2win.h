@@ -122,6 +122,23 @@ im2win_status im2win_conv_f16(const uint16_t* window, const uint16_t* filter_oih
                               void* cuda_stream);
 
 /*
+ * The two halves of im2win_conv_f32 / im2win_conv_f16 for static weights (the
+ * paper repacks the filter "height before width" once, Section "Im2win
+ * Convolution"): im2win_pack_filter writes the packed filter (and clears the
+ * status block) into `scratch`; im2win_conv_packed runs the convolution of
+ * `dtype` on a filter packed earlier into the same `scratch` for the same
+ * shape and dtype, any number of times.  `filter_oihw` and `window` hold
+ * elements of `dtype` (binary16 bit patterns for IM2WIN_F16); arguments,
+ * scratch size and errors as for the one-call forms.  The packed layout depends
+ * on the kernel the library selects for the shape; both calls must come from
+ * the same process with an unchanged environment.
+ */
+im2win_status im2win_pack_filter(const void* filter_oihw, void* scratch, size_t scratch_bytes,
+                                 const im2win_shape* shape, im2win_dtype dtype, void* cuda_stream);
+im2win_status im2win_conv_packed(const void* window, float* y_nchw, void* scratch, size_t scratch_bytes,
+                                 const im2win_shape* shape, im2win_dtype dtype, void* cuda_stream);
+
+/*
  * Synchronises `cuda_stream`, reads the status block at the start of `scratch`
  * (written by the last convolution call that used it) and returns
  * IM2WIN_ERR_TIMEOUT if a bounded device wait gave up, IM2WIN_ERR_CUDA if the

@@ -25,7 +25,7 @@ STATUS_NAMES = {
 EXPORTS = (
     "im2win_status_string", "im2win_workspace_size", "im2win_transform", "im2win_conv_f32", "im2win_conv_f16",
     "im2win_check_status", "im2win_layer_workspace_size", "im2win_layer_forward_host",
-    "im2win_conv_f32_static",
+    "im2win_conv_f32_static", "im2win_pack_filter", "im2win_conv_packed",
 )
 
 STATIC_SCRATCH_BYTES = 4 << 20
@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
     L.im2win_layer_workspace_size.argtypes = [P(Shape), ctypes.c_int, P(sz)]
     L.im2win_layer_forward_host.argtypes = [vp, vp, vp, vp, sz, P(Shape), ctypes.c_int, vp]
     L.im2win_conv_f32_static.argtypes = [vp, vp, vp, P(Shape), vp]
+    L.im2win_pack_filter.argtypes = [vp, vp, sz, P(Shape), ctypes.c_int, vp]
+    L.im2win_conv_packed.argtypes = [vp, vp, vp, sz, P(Shape), ctypes.c_int, vp]
     for name in EXPORTS[1:]:
         getattr(L, name).restype = ctypes.c_int
     _lib = L
@@ -168,6 +170,25 @@ def im2win_conv_f32_static(window, filter_oihw, y, shape, stream=None) -> None:
         assert t.is_cuda and t.is_contiguous() and t.dtype == torch.float32
     _check(lib().im2win_conv_f32_static(window.data_ptr(), filter_oihw.data_ptr(), y.data_ptr(),
                                         ctypes.byref(s), _stream(stream)), "im2win_conv_f32_static")
+
+
+def im2win_pack_filter(filter_oihw, scratch, shape, stream=None) -> None:
+    """Packs the filter into `scratch` once (static weights); im2win_conv_packed then reuses it."""
+    s = as_shape(shape)
+    assert filter_oihw.is_cuda and filter_oihw.is_contiguous() and scratch.is_cuda
+    _check(lib().im2win_pack_filter(filter_oihw.data_ptr(), scratch.data_ptr(), scratch.numel() * scratch.element_size(),
+                                    ctypes.byref(s), _dtype_code(filter_oihw.dtype), _stream(stream)),
+           "im2win_pack_filter")
+
+
+def im2win_conv_packed(window, y, scratch, shape, stream=None) -> None:
+    """Convolution with the filter that im2win_pack_filter left in `scratch` (same shape and dtype)."""
+    s = as_shape(shape)
+    assert window.is_cuda and window.is_contiguous() and y.is_cuda and y.dtype == torch.float32 and scratch.is_cuda
+    _check(lib().im2win_conv_packed(window.data_ptr(), y.data_ptr(), scratch.data_ptr(),
+                                    scratch.numel() * scratch.element_size(), ctypes.byref(s),
+                                    _dtype_code(window.dtype), _stream(stream)),
+           "im2win_conv_packed")
 
 
 def im2win_check_status(scratch: torch.Tensor, stream=None) -> None:

@@ -102,42 +102,41 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
 
 static inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
+// mode bit 0: pack the filter into scratch; bit 1: run the convolution on the packed filter.
+enum { kDoPack = 1, kDoConv = 2 };
 static im2win_status conv_common(const void* window, const void* filter, float* y, void* scratch,
                                  size_t scratch_bytes, const im2win_shape* shape, im2win_dtype dtype,
-                                 void* cuda_stream) {
-  if (!window || !filter || !y || !scratch || !shape) return IM2WIN_ERR_NULL_POINTER;
+                                 void* cuda_stream, int mode = kDoPack | kDoConv) {
+  if (!scratch || !shape) return IM2WIN_ERR_NULL_POINTER;
+  if ((mode & kDoPack) && !filter) return IM2WIN_ERR_NULL_POINTER;
+  if ((mode & kDoConv) && (!window || !y)) return IM2WIN_ERR_NULL_POINTER;
   Geometry g;
   im2win_status st = derive_geometry(shape, &g);
   if (st != IM2WIN_OK) return st;
   ScratchLayout l;
   st = scratch_layout(g, dtype, &l);
   if (st != IM2WIN_OK) return st;
-  if (misaligned(window) || misaligned(filter) || misaligned(y) || misaligned(scratch))
+  if (misaligned(scratch) || ((mode & kDoPack) && misaligned(filter)) ||
+      ((mode & kDoConv) && (misaligned(window) || misaligned(y))))
     return IM2WIN_ERR_MISALIGNED;
   if (scratch_bytes < l.total) return IM2WIN_ERR_WORKSPACE_TOO_SMALL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  cudaError_t e;
-  if (dtype == IM2WIN_F32) {
-    e = launch_pack_f32(static_cast<const float*>(filter), scratch, g, l, stream);
-    if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
-    e = launch_conv_f32(static_cast<const float*>(window), y, scratch, g, l, stream);
-  } else {
-    if (l.f16_mat) {
-      e = launch_conv_f16_mat(static_cast<const uint16_t*>(window), static_cast<const uint16_t*>(filter), y, scratch,
-                              g, stream);
-    } else if (l.f16_raw) {
+  cudaError_t e = cudaSuccess;
+  if (mode & kDoPack) {
+    if (dtype == IM2WIN_F32) e = launch_pack_f32(static_cast<const float*>(filter), scratch, g, l, stream);
+    else if (l.f16_mat) e = launch_pack_f16_mat(static_cast<const uint16_t*>(filter), scratch, g, stream);
+    else if (l.f16_raw)
       e = launch_pack_f16_raw(static_cast<const uint16_t*>(filter), scratch, g, l, plan_f16_raw(g), stream);
-      if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
-      e = launch_conv_f16_raw(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
-    } else if (l.f16_shift) {
-      e = launch_pack_f16_shift(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
-      if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
-      e = launch_conv_f16_shift(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
-    } else {
-      e = launch_pack_f16(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
-      if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
-      e = launch_conv_f16_gather(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
-    }
+    else if (l.f16_shift) e = launch_pack_f16_shift(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
+    else e = launch_pack_f16(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
+    if (e != cudaSuccess) return IM2WIN_ERR_CUDA;
+  }
+  if (mode & kDoConv) {
+    if (dtype == IM2WIN_F32) e = launch_conv_f32(static_cast<const float*>(window), y, scratch, g, l, stream);
+    else if (l.f16_mat) e = launch_conv_f16_mat(static_cast<const uint16_t*>(window), y, scratch, g, stream);
+    else if (l.f16_raw) e = launch_conv_f16_raw(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
+    else if (l.f16_shift) e = launch_conv_f16_shift(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
+    else e = launch_conv_f16_gather(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
   }
   return e == cudaSuccess ? IM2WIN_OK : IM2WIN_ERR_CUDA;
 }
@@ -199,6 +198,16 @@ im2win_status im2win_conv_f16(const uint16_t* window, const uint16_t* filter_oih
                               void* scratch, size_t scratch_bytes, const im2win_shape* shape,
                               void* cuda_stream) {
   return conv_common(window, filter_oihw, y_nchw, scratch, scratch_bytes, shape, IM2WIN_F16, cuda_stream);
+}
+
+im2win_status im2win_pack_filter(const void* filter_oihw, void* scratch, size_t scratch_bytes,
+                                 const im2win_shape* shape, im2win_dtype dtype, void* cuda_stream) {
+  return conv_common(nullptr, filter_oihw, nullptr, scratch, scratch_bytes, shape, dtype, cuda_stream, kDoPack);
+}
+
+im2win_status im2win_conv_packed(const void* window, float* y_nchw, void* scratch, size_t scratch_bytes,
+                                 const im2win_shape* shape, im2win_dtype dtype, void* cuda_stream) {
+  return conv_common(window, nullptr, y_nchw, scratch, scratch_bytes, shape, dtype, cuda_stream, kDoConv);
 }
 
 im2win_status im2win_check_status(const void* scratch, void* cuda_stream) {

@@ -91,9 +91,10 @@ cudaError_t launch_pack_f16_raw(const uint16_t* filter, void* scratch, const Geo
                                 const ScratchLayout& l, const RawPlan& plan, cudaStream_t stream);
 cudaError_t launch_conv_f16_raw(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                 const ScratchLayout& l, cudaStream_t stream);
-// Packs the filter into `scratch` and runs the matrix-transpose kernel.
-cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, float* y, void* scratch,
-                                const Geometry& g, cudaStream_t stream);
+// Matrix-transpose kernel: filter pack into `scratch` (own layout) and the convolution on it.
+cudaError_t launch_pack_f16_mat(const uint16_t* filter, void* scratch, const Geometry& g, cudaStream_t stream);
+cudaError_t launch_conv_f16_mat(const uint16_t* window, float* y, void* scratch, const Geometry& g,
+                                cudaStream_t stream);
 cudaError_t launch_conv_f16_gather(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                    const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratch, const Geometry& g,

@@ -807,8 +807,22 @@ MatPlan plan_f16_mat(const Geometry& g) {
   return p;
 }
 
-cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, float* y, void* scratch,
-                                const Geometry& g, cudaStream_t stream) {
+cudaError_t launch_pack_f16_mat(const uint16_t* filter, void* scratch, const Geometry& g, cudaStream_t stream) {
+  const MatPlan plan = plan_f16_mat(g);
+  if (!plan.eligible) return cudaErrorInvalidValue;
+  unsigned char* base = static_cast<unsigned char*>(scratch);
+  uint16_t* fp = reinterpret_cast<uint16_t*>(base + kStatusBytes);
+  const int ncog = (g.Co + 63) / 64;                    // groups of 64 output channels
+  const unsigned gx = (unsigned)((plan.K2p + 255) / 256);
+  dim3 grid(gx > 64 ? 64 : gx, (unsigned)(ncog * 64 < 32768 ? ncog * 64 : 32768),
+            (unsigned)(g.Kw < 65535 ? g.Kw : 65535));
+  pack_f16_mat_kernel<<<grid, 256, 0, stream>>>(filter, fp, reinterpret_cast<uint32_t*>(base), g.C, g.Co, g.Kh, g.Kw,
+                                                (int)plan.K2p, ncog);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_conv_f16_mat(const uint16_t* window, float* y, void* scratch, const Geometry& g,
+                                cudaStream_t stream) {
   const MatPlan plan = plan_f16_mat(g);
   if (!plan.eligible) return cudaErrorInvalidValue;
   EncodeTiledFn encode = get_encode_fn();
@@ -819,17 +833,7 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, const uint16_t* filter, 
   const char* pair_env = getenv("IM2WIN_F16_PAIR");     // testing aid: 0 = never pair CTAs
   // measured: pairing pays for 256-channel tiles (the filter tile halves); narrow tiles gain nothing
   const bool pair = bn == 256 && !(pair_env && pair_env[0] == '0');
-
   const int ncog = (g.Co + 63) / 64;                    // groups of 64 output channels
-  {
-    const unsigned gx = (unsigned)((plan.K2p + 255) / 256);
-    dim3 grid(gx > 64 ? 64 : gx, (unsigned)(ncog * 64 < 32768 ? ncog * 64 : 32768),
-              (unsigned)(g.Kw < 65535 ? g.Kw : 65535));
-    pack_f16_mat_kernel<<<grid, 256, 0, stream>>>(filter, fp, reinterpret_cast<uint32_t*>(base), g.C, g.Co, g.Kh, g.Kw,
-                                                  (int)plan.K2p, ncog);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-  }
 
   // Packed filter as a 2-D array of 2 KB rows (256 eight-byte elements); one box = this CTA's
   // rows of one (v, k-block): 128 bytes per output channel.

@@ -101,6 +101,14 @@ def test_null_and_misaligned_pointers_rejected_before_launch():
     assert lib.im2win_conv_f16(ctypes.c_void_p(256), ctypes.c_void_p(1024), ctypes.c_void_p(512), ctypes.c_void_p(768),
                                16, sp, None) == 4
     assert lib.im2win_check_status(None, None) == 2
+    vp = ctypes.c_void_p
+    assert lib.im2win_pack_filter(None, vp(768), 1 << 20, sp, 0, None) == 2
+    assert lib.im2win_pack_filter(vp(1024), vp(776), 1 << 20, sp, 0, None) == 3
+    assert lib.im2win_pack_filter(vp(1024), vp(768), 16, sp, 1, None) == 4
+    assert lib.im2win_pack_filter(vp(1024), vp(768), 1 << 20, sp, 7, None) == 1
+    assert lib.im2win_conv_packed(None, vp(512), vp(768), 1 << 20, sp, 0, None) == 2
+    assert lib.im2win_conv_packed(vp(256), vp(520), vp(768), 1 << 20, sp, 1, None) == 3
+    assert lib.im2win_conv_packed(vp(256), vp(512), vp(768), 16, sp, 0, None) == 4
     assert lib.im2win_layer_forward_host(ctypes.c_void_p(256), ctypes.c_void_p(256), ctypes.c_void_p(256),
                                          ctypes.c_void_p(128), 1 << 30, sp, 0, None) == 3
     assert lib.im2win_layer_forward_host(ctypes.c_void_p(256), ctypes.c_void_p(256), ctypes.c_void_p(256),

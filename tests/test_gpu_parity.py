@@ -181,6 +181,26 @@ def test_layer_forward_host_in_batch_chunks(n):
         assert np.array_equal(yh.numpy(), y_dev), precision
 
 
+@pytest.mark.parametrize("layer", [SMALL[1], SMALL[4], SMALL[12], SMALL[15], SMALL[16]], ids=lambda l: l.name)
+def test_pack_once_then_convolve_twice(layer):
+    """im2win_pack_filter + im2win_conv_packed (twice, on different inputs) give what the one-call
+    forms give, bit for bit, in both precisions."""
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    x2 = torch.flip(x, dims=[0, 3]).contiguous()
+    for precision, tdt in (("f32", torch.float32), ("f16", torch.float16)):
+        fd = f.to(tdt).cuda().contiguous()
+        window, scratch, y = binding.alloc_layer_buffers(dims, tdt)
+        binding.im2win_pack_filter(fd, scratch, dims)
+        for xin in (x, x2):
+            want, _, _ = gpu_conv(xin, f, dims, precision)
+            binding.im2win_transform(xin.to(tdt).cuda().contiguous(), window, dims)
+            y.fill_(float("nan"))
+            binding.im2win_conv_packed(window, y, scratch, dims)
+            binding.im2win_check_status(scratch)
+            assert np.array_equal(y.cpu().numpy(), want), (layer.name, precision)
+
+
 def test_repeated_calls_are_deterministic_and_do_not_depend_on_stale_scratch():
     layer = SMALL[3]
     dims = layer.dims()
