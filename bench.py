@@ -156,6 +156,11 @@ class LayerRunner:
         else:
             self.b.im2win_conv_f16(d["window"], d["f"], d["y"], d["scratch"], self.dims)
 
+    def conv_packed(self, prec):
+        """The convolution alone, on the filter the last conv() call left packed in scratch."""
+        d = self.dev[prec]
+        self.b.im2win_conv_packed(d["window"], d["y"], d["scratch"], self.dims)
+
     def step(self, events=None):
         """One pass of the hot path; with `events` (list) records an event before/after each call."""
         for prec in self.precisions:
@@ -425,7 +430,13 @@ def write_report(path, peaks, peak_kind, names=None, iters=20):
                 key = f"{kind}_{prec}"
                 avg[key], best[key], median[key] = time_call(lambda: fn(prec), iters, flush)
             binding.im2win_check_status(runner.dev[prec]["scratch"])
-        row = {"layer": name, "dims": layer.dims(), "gflop": runner.flops / 1e9, "avg_ms": avg, "best_ms": best, "median_ms": median,
+        # the convolution kernel without the filter pack (static weights), for reference
+        packed = {}
+        for prec in layer.precisions:
+            a, b_, m = time_call(lambda: runner.conv_packed(prec), iters, flush)
+            packed[f"conv_{prec}"] = {"avg_ms": a, "best_ms": b_, "median_ms": m}
+        row = {"layer": name, "dims": layer.dims(), "gflop": runner.flops / 1e9, "avg_ms": avg, "best_ms": best,
+               "median_ms": median, "conv_without_pack": packed,
                "kernels": kernel_rooflines(runner, avg, peaks, peak_kind), "memory": runner.memory_report()}
         rows.append(row)
         del runner

@@ -84,6 +84,13 @@ struct Segment {            // the part of a tile that lies in one image
   int32_t pad_;
 };
 
+// Programmatic dependent launch: the convolution kernel is launched so that it may start while
+// the filter pack (the kernel before it in the stream) is still running; its barrier setup, tensor
+// memory allocation and descriptor fetches overlap the pack.  Every role that touches global memory
+// first waits for the preceding kernel to have completed (and its writes to be visible).
+__device__ __forceinline__ void wait_for_previous_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void let_next_kernel_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Splits the rows of the tile starting at virtual position q0 by image: within an image the
 // columns of one channel are contiguous in the window tensor.  Returns the number of segments
 // and, in *total_boxes, the boxes of one raw stage.
@@ -378,6 +385,7 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
     if (threadIdx.x == 0) TIMER_FLUSH();
   } else if (warp == WARP_TMA) {
     // ---------------- TMA loader of the filter tiles ---------------------------
+    wait_for_previous_kernel();
     const bool leader = elect_one();
     bool ok = true;
     int st = 0;
@@ -496,6 +504,7 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
     // two warps share the boxes of a stage (even / odd): issuing a copy costs a few hundred
     // cycles and the stage is only complete when its last box has been requested
     const int half = warp - WARP_RAW;
+    wait_for_previous_kernel();
     const bool leader = elect_one();
     bool ok = true;
     int rst = 0;
@@ -533,6 +542,7 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
   } else if (warp >= WARP_EPI0) {
     // ---------------- epilogue: tensor memory -> NCHW output --------------------
     const int lq = warp & 3;                     // tensor-memory lane quadrant this warp may read
+    wait_for_previous_kernel();                  // before the first store to y
     bool ok = true;
     uint32_t it = 0;
     for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
@@ -616,22 +626,57 @@ conv_f16_mat_pair_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_
 // tile is ONE contiguous run and can be copied with 2 KB rows (the copy engine spends about a
 // cycle per row on top of the bytes).  Padded k2 and channels >= Co hold zeros.  Block (0,0,0)
 // also clears the status block.
+// One block handles one output channel and `noct` consecutive channel octets: their source halves
+// ((co*C + c)*Kh + u)*Kw + v are one contiguous run of the OIHW filter, read coalesced into shared
+// memory; every thread then assembles 16-byte units (8 channels of one (octet, u, v)) and stores
+// them at their place in the tile images.
 __global__ void pack_f16_mat_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, uint32_t* status,
-                                    int C, int Co, int Kh, int Kw, int K2p, int ncog) {
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
+                                    int C, int Co, int Kh, int Kw, int K2p, int ncog, int noct) {
+  extern __shared__ uint16_t pack_s[];
+  let_next_kernel_start();
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
   const int num_kb = K2p / KB;
-  for (int v = blockIdx.z; v < Kw; v += gridDim.z)
-    for (int co = blockIdx.y; co < ncog * 64; co += gridDim.y)
-      for (int k2 = blockIdx.x * blockDim.x + threadIdx.x; k2 < K2p; k2 += gridDim.x * blockDim.x) {
-        const int unit = k2 >> 3, e = k2 & 7;
-        const int oct = unit / Kh, u = unit - oct * Kh;
-        const int c = oct * 8 + e;
-        uint16_t val = 0;
-        if (c < C && co < Co) val = f[(((size_t)co * C + c) * Kh + u) * Kw + v];
-        const int kb = k2 >> 6, chunk = (k2 & 63) >> 3, r = co & 63;
-        const size_t image = ((size_t)v * num_kb + kb) * ncog + (co >> 6);
-        fp[image * 4096 + (size_t)r * 64 + (size_t)(((chunk ^ (r & 7)) << 3) + e)] = val;
+  const int T = Kh * Kw;
+  const int oct_a = blockIdx.x * noct;
+  const int units_total = K2p / 8;                       // units per (co, v), padding included
+  const int unit_a = oct_a * Kh;
+  // the last block also covers the padded units beyond the last octet
+  const int unit_b = (blockIdx.x == gridDim.x - 1) ? units_total : (oct_a + noct) * Kh;
+  const int c_a = oct_a * 8;
+  int nsrc = (C - c_a < noct * 8 ? C - c_a : noct * 8) * T;    // source halves that exist
+  if (nsrc < 0) nsrc = 0;
+  for (int co = blockIdx.y; co < ncog * 64; co += gridDim.y) {
+    __syncthreads();
+    if (co < Co) {
+      const uint16_t* src = f + ((size_t)co * C + c_a) * T;
+      for (int i = threadIdx.x; i < nsrc; i += blockDim.x) pack_s[i] = src[i];
+    }
+    __syncthreads();
+    const int r = co & 63;
+    const int nunits = unit_b - unit_a;
+    for (int i = threadIdx.x; i < nunits * Kw; i += blockDim.x) {
+      const int v = i / nunits;
+      const int unit = unit_a + (i - v * nunits);
+      const int oct = unit / Kh, u = unit - oct * Kh;
+      uint32_t w[4];
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        uint32_t pair = 0;
+#pragma unroll
+        for (int lo = 0; lo < 2; ++lo) {
+          const int e = 2 * h + lo;
+          const int idx = ((oct - oct_a) * 8 + e) * T + u * Kw + v;     // (c - c_a)*T + u*Kw + v
+          const uint32_t val = (co < Co && idx < nsrc && oct < oct_a + noct) ? pack_s[idx] : 0u;
+          pair |= val << (16 * lo);
+        }
+        w[h] = pair;
       }
+      const int kb = unit >> 3, chunk = unit & 7;
+      const size_t image = ((size_t)v * num_kb + kb) * ncog + (co >> 6);
+      *reinterpret_cast<uint4*>(fp + image * 4096 + (size_t)r * 64 + (size_t)((chunk ^ (r & 7)) << 3)) =
+          make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -696,8 +741,17 @@ cudaError_t launch_bn(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParam
   const int per_sm = (BN <= 128 && smem_bytes + 1024 <= kSmemMax / 2) ? 2 : 1;
   const int slots = 148 * per_sm;                      // persistent CTAs
   const unsigned grid = (unsigned)(nwork < slots ? nwork : slots);
-  conv_f16_mat_kernel<BN><<<grid, NUM_THREADS, smem_bytes, stream>>>(fmap, wmap, q);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem_bytes;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, conv_f16_mat_kernel<BN>, fmap, wmap, q);
 }
 
 // CTA-pair launch: clusters of two CTAs, as many as can be resident at once.
@@ -731,8 +785,14 @@ cudaError_t launch_pair(const CUtensorMap& fmap, const CUtensorMap& wmap, MatPar
   if (clusters < 1) return cudaErrorInvalidValue;
   if (clusters > 74) clusters = 74;
   if ((int64_t)clusters > nwork) clusters = (int)nwork;
-  conv_f16_mat_pair_kernel<BN><<<2 * clusters, NUM_THREADS, smem_bytes, stream>>>(fmap, wmap, q);
-  return cudaGetLastError();
+  cudaLaunchAttribute lattr[2];
+  lattr[0] = attr[0];
+  lattr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  lattr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.gridDim = dim3(2 * clusters, 1, 1);
+  cfg.attrs = lattr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, conv_f16_mat_pair_kernel<BN>, fmap, wmap, q);
 }
 
 uint32_t magic16(int d) { return (uint32_t)(65536 / d + 1); }
@@ -813,11 +873,14 @@ cudaError_t launch_pack_f16_mat(const uint16_t* filter, void* scratch, const Geo
   unsigned char* base = static_cast<unsigned char*>(scratch);
   uint16_t* fp = reinterpret_cast<uint16_t*>(base + kStatusBytes);
   const int ncog = (g.Co + 63) / 64;                    // groups of 64 output channels
-  const unsigned gx = (unsigned)((plan.K2p + 255) / 256);
-  dim3 grid(gx > 64 ? 64 : gx, (unsigned)(ncog * 64 < 32768 ? ncog * 64 : 32768),
-            (unsigned)(g.Kw < 65535 ? g.Kw : 65535));
-  pack_f16_mat_kernel<<<grid, 256, 0, stream>>>(filter, fp, reinterpret_cast<uint32_t*>(base), g.C, g.Co, g.Kh, g.Kw,
-                                                (int)plan.K2p, ncog);
+  int noct = 4096 / (8 * g.T);                          // octets per block: staging of <= 4096 halves
+  if (noct < 1) noct = 1;
+  if (noct > plan.Cp8) noct = plan.Cp8;
+  const size_t smem = (size_t)noct * 8 * g.T * sizeof(uint16_t);
+  if (smem > 48 * 1024) return cudaErrorInvalidValue;
+  dim3 grid((unsigned)((plan.Cp8 + noct - 1) / noct), (unsigned)(ncog * 64 < 32768 ? ncog * 64 : 32768));
+  pack_f16_mat_kernel<<<grid, 256, smem, stream>>>(filter, fp, reinterpret_cast<uint32_t*>(base), g.C, g.Co, g.Kh, g.Kw,
+                                                   (int)plan.K2p, ncog, noct);
   return cudaGetLastError();
 }
 

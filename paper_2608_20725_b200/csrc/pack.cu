@@ -82,24 +82,40 @@ __global__ void pack_f16_kernel(const uint16_t* __restrict__ f, uint16_t* __rest
 // and one of two tables: k2 -> c*chan_stride + u (gathering kernel, raw_pitch = 0; -1 for padded
 // k2), or k2 -> byte offset of element (c, u) inside a raw box, slot (c - first channel of the
 // k-block) * raw_pitch + u*2, padded k2 pointing at the all-zero slot `nslot` (TMA-staged kernel).
-// Grid: x over k2, y over output channels, z over kernel columns: no per-element divisions
-// beyond k2 / Kh.
+// One block handles one output channel and `chunk` (even, <= 512) consecutive k2: its Kw*chunk source halves
+// are one contiguous run of the OIHW filter ((co*K2 + k2)*Kw + v), which is read coalesced into
+// shared memory and written back out as Kw coalesced rows of the packed layout.
 __global__ void pack_f16_shift_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp,
                                       uint32_t* __restrict__ table, uint32_t* __restrict__ status,
-                                      PackParams q, int raw_pitch, int nslot) {
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x < kStatusBytes / 4)
-    status[threadIdx.x] = 0u;
+                                      PackParams q, int raw_pitch, int nslot, int chunk) {
+  extern __shared__ uint16_t pack_s[];
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
   const int K2 = q.C * q.Kh;
   const int K2p = (int)q.Kp;
-  const int v = blockIdx.z;
+  const int k2a = blockIdx.x * chunk;
+  const int k2b = k2a + chunk < K2p ? k2a + chunk : K2p;
+  const int nreal = (k2b < K2 ? k2b : K2) - k2a;          // k2 of this chunk that exist in the filter (may be <= 0)
   for (int co = blockIdx.y; co < q.Co; co += gridDim.y) {
-    for (int k2 = blockIdx.x * blockDim.x + threadIdx.x; k2 < K2p; k2 += gridDim.x * blockDim.x) {
-      uint16_t val = 0;
+    const uint16_t* src = f + ((size_t)co * K2 + k2a) * q.Kw;
+    __syncthreads();
+    for (int i = threadIdx.x; i < nreal * q.Kw; i += blockDim.x) pack_s[i] = src[i];
+    __syncthreads();
+    for (int v = 0; v < q.Kw; ++v) {
+      uint16_t* dst = fp + ((size_t)v * q.Co + co) * K2p + k2a;
+      // two k2 per thread: one 32-bit store (k2a and K2p are even)
+      for (int j = 2 * threadIdx.x; j < k2b - k2a; j += 2 * blockDim.x) {
+        const uint32_t lo = j < nreal ? pack_s[j * q.Kw + v] : 0u;
+        const uint32_t hi = j + 1 < nreal ? pack_s[(j + 1) * q.Kw + v] : 0u;
+        *reinterpret_cast<uint32_t*>(dst + j) = lo | (hi << 16);
+      }
+    }
+  }
+  if (blockIdx.y == 0) {
+    for (int k2 = k2a + threadIdx.x; k2 < k2b; k2 += blockDim.x) {
       uint32_t entry = raw_pitch > 0 ? (uint32_t)(nslot * raw_pitch) : 0xffffffffu;
       if (k2 < K2) {
         const int c = k2 / q.Kh;
         const int u = k2 - c * q.Kh;
-        val = f[(((size_t)co * q.C + c) * q.Kh + u) * q.Kw + v];
         if (raw_pitch > 0) {
           const int c_lo = (k2 / kF16KBlock) * kF16KBlock / q.Kh;
           entry = (uint32_t)((c - c_lo) * raw_pitch + u * 2);
@@ -107,8 +123,7 @@ __global__ void pack_f16_shift_kernel(const uint16_t* __restrict__ f, uint16_t* 
           entry = (uint32_t)(c * q.chan_stride + u);
         }
       }
-      fp[((size_t)v * q.Co + co) * K2p + k2] = val;
-      if (v == 0 && co == 0) table[k2] = entry;
+      table[k2] = entry;
     }
   }
 }
@@ -153,11 +168,14 @@ static cudaError_t pack_shift_common(const uint16_t* filter, void* scratch, cons
                                      const ScratchLayout& l, int raw_pitch, int nslot, cudaStream_t stream) {
   unsigned char* base = static_cast<unsigned char*>(scratch);
   PackParams q = make_params(g, l);
-  const unsigned gx = (unsigned)((q.Kp + 255) / 256);
-  dim3 grid(gx > 64 ? 64 : gx, (unsigned)(g.Co < 32768 ? g.Co : 32768), (unsigned)(g.Kw < 65535 ? g.Kw : 65535));
-  pack_f16_shift_kernel<<<grid, 256, 0, stream>>>(filter, reinterpret_cast<uint16_t*>(base + l.filter_off),
-                                                  reinterpret_cast<uint32_t*>(base + l.koff_off),
-                                                  reinterpret_cast<uint32_t*>(base), q, raw_pitch, nslot);
+  int chunk = 512;                                          // k2 per block: staging of chunk*Kw halves within 40 KB
+  while (chunk > 2 && (size_t)chunk * g.Kw * sizeof(uint16_t) > 40 * 1024) chunk /= 2;
+  const size_t smem = (size_t)chunk * g.Kw * sizeof(uint16_t);
+  if (smem > 48 * 1024) return cudaErrorInvalidValue;
+  dim3 grid((unsigned)((q.Kp + chunk - 1) / chunk), (unsigned)(g.Co < 32768 ? g.Co : 32768));
+  pack_f16_shift_kernel<<<grid, 256, smem, stream>>>(filter, reinterpret_cast<uint16_t*>(base + l.filter_off),
+                                                     reinterpret_cast<uint32_t*>(base + l.koff_off),
+                                                     reinterpret_cast<uint32_t*>(base), q, raw_pitch, nslot, chunk);
   return cudaGetLastError();
 }
 
