@@ -26,9 +26,18 @@
 //     plane, R, are chosen with R*Kh = 1 (mod 8) when Kh is odd, which makes the 8 destination
 //     rows of one stmatrix matrix fall into 8 different bank groups.
 //
+//   * filter: packed as 8 KB images (64 output channels x 64 k2, already in the 128-byte-swizzled
+//     order of a k-major MMA tile), so a filter tile is one contiguous run copied with 2 KB rows;
+//     a filter stage holds all kernel columns of a k-block that fit, which keeps the MMA issuer's
+//     barrier round trips at two waits and two commits per k-block.
+//   * CTA pairs (tiles of 256 output channels): the two CTAs of a cluster share every MMA
+//     (cta_group::2, M = 256), each staging its own 128 positions and half of the filter tile.
+//
 // Any stride s with Wp mod s = 0 (columns are de-interleaved into s sub-tiles as in
 // conv_f16_shift.cu); the plane pitch of the window tensor must be a multiple of 16 bytes.
 // Persistent CTAs, double-buffered accumulator in tensor memory, bounded mbarrier waits.
+// Warp roles: 0-7 re-layout, 8 filter copies, 9 MMA issue (and tensor-memory allocation),
+// 10-11 raw box copies, 12-15 epilogue.
 #include <cuda.h>
 #include <stdlib.h>
 
