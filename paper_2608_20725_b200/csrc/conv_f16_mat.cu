@@ -79,6 +79,7 @@ struct MatParams {
   uint32_t magic_kh, magic_s;   // floor(e / d) = (e * magic) >> 16 for e < 8192
   int32_t rs, sa, sb;       // ring depths
   int32_t vg;               // kernel columns per filter stage
+  int32_t resident;         // 1: the filter ring holds the whole filter of the (only) channel tile: loaded once
   int32_t ntm, nwork;       // position tiles; work items = position tiles x channel tiles
   int32_t frows;            // 2 KB rows of the packed filter per (kernel column, k-block): 4 per 64 channels
 };
@@ -427,6 +428,7 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
           if (++st == q.sb) { st = 0; ph ^= 1u; }
         }
       }
+      if (q.resident) break;          // every stage now holds its k-block for good
     }
   } else if (warp == WARP_MMA && rank == 0) {
     // ---------------- MMA issuer (leader CTA of a pair) -------------------------
@@ -465,10 +467,12 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
         for (int v0 = 0; v0 < q.Kw; v0 += q.vg) {
           const int nv = q.Kw - v0 < q.vg ? q.Kw - v0 : q.vg;
           TIMER_LAP(8);
-          ok = PAIR ? mbar_wait_cluster(b_full0 + 8 * stb, phb, &abort_flag, q.status)
-                    : mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
+          if (!(q.resident && it > 0)) {       // a resident filter is complete after the first work item
+            ok = PAIR ? mbar_wait_cluster(b_full0 + 8 * stb, phb, &abort_flag, q.status)
+                      : mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
           TIMER_LAP(10);                         // MMA warp: wait for a filter stage
           tc_fence_after();
           uint32_t b_lo = b_lo0 + (uint32_t)(stb * (B_STAGE_BYTES >> 4));
@@ -488,8 +492,10 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
               b_lo += (uint32_t)(B_TILE_BYTES >> 4);
               if (++sub == (uint32_t)q.s) { sub = 0; ++shift; }
             }
-            if (PAIR) umma_commit_pair(b_empty0 + 8 * stb);
-            else umma_commit(b_empty0 + 8 * stb);
+            if (!q.resident) {
+              if (PAIR) umma_commit_pair(b_empty0 + 8 * stb);
+              else umma_commit(b_empty0 + 8 * stb);
+            }
           }
           __syncwarp();
           if (++stb == q.sb) { stb = 0; phb ^= 1u; }
@@ -713,14 +719,27 @@ int tile_bn(const Geometry& g) { return g.Co <= 64 ? 64 : (g.Co <= 128 ? 128 : 2
 // twice (every barrier round trip and commit costs the MMA issuer time, so fewer, larger filter
 // stages are better), filter ring as deep as fits (<= 6), then a third raw stage if there is room.
 // Narrow tiles try to fit two CTAs on an SM first.
-bool choose_rings(int bn, int b_rows, int kw, const MatPlan& plan, int* rs, int* sa, int* sb, int* vg,
-                  int* smem_bytes) {
+bool choose_rings(int bn, int b_rows, int kw, int nct, const MatPlan& plan, int* rs, int* sa, int* sb, int* vg,
+                  int* resident, int* smem_bytes) {
   const int fixed = plan.num_kb * 4;
   const int a = plan.a_stage_bytes, r = plan.raw_stage_bytes, tile = b_rows * KB * 2;
+  *resident = 0;
   for (int half = (bn <= 128 ? 1 : 0); half >= 0; --half) {
     // dynamic shared memory left after the alignment slack, the static part (barriers, segment
     // copies) and, for two CTAs per SM, the 1 KB the runtime reserves per CTA
     const int budget = (half ? kSmemMax / 2 : kSmemMax) - 1024 - 4096;
+    // One channel tile and a filter small enough: keep all of it in shared memory (loaded once per
+    // CTA instead of once per work item).
+    if (nct == 1 && plan.num_kb <= MAX_STAGES) {
+      const int b = kw * tile;
+      if (2 * a + 2 * r + plan.num_kb * b + fixed <= budget) {
+        const int rr = (2 * a + 3 * r + plan.num_kb * b + fixed <= budget) ? 3 : 2;
+        const int aa = (3 * a + rr * r + plan.num_kb * b + fixed <= budget) ? 3 : 2;
+        *rs = rr; *sa = aa; *sb = plan.num_kb; *vg = kw; *resident = 1;
+        *smem_bytes = aa * a + rr * r + plan.num_kb * b + fixed + 1024;
+        return true;
+      }
+    }
     for (int g = kw; g >= 1; --g) {
       const int b = g * tile;
       if (2 * a + 2 * r + 2 * b + fixed > budget) continue;
@@ -739,7 +758,8 @@ template <int BN>
 cudaError_t launch_bn(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParams q, const MatPlan& plan, int co,
                       cudaStream_t stream) {
   int smem_bytes = 0;
-  if (!choose_rings(BN, BN, q.Kw, plan, &q.rs, &q.sa, &q.sb, &q.vg, &smem_bytes)) return cudaErrorInvalidValue;
+  if (!choose_rings(BN, BN, q.Kw, (co + BN - 1) / BN, plan, &q.rs, &q.sa, &q.sb, &q.vg, &q.resident, &smem_bytes))
+    return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(conv_f16_mat_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
   const int64_t ntm = (plan.VQ + TILE_M - 1) / TILE_M;
@@ -768,7 +788,8 @@ template <int BN>
 cudaError_t launch_pair(const CUtensorMap& fmap, const CUtensorMap& wmap, MatParams q, const MatPlan& plan, int co,
                         cudaStream_t stream) {
   int smem_bytes = 0;
-  if (!choose_rings(256, BN / 2, q.Kw, plan, &q.rs, &q.sa, &q.sb, &q.vg, &smem_bytes)) return cudaErrorInvalidValue;
+  if (!choose_rings(256, BN / 2, q.Kw, (co + BN - 1) / BN, plan, &q.rs, &q.sa, &q.sb, &q.vg, &q.resident, &smem_bytes))
+    return cudaErrorInvalidValue;
   cudaError_t e =
       cudaFuncSetAttribute(conv_f16_mat_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
@@ -870,8 +891,8 @@ MatPlan plan_f16_mat(const Geometry& g) {
   p.a_stage_bytes = (g.s * 8 * p.R * 16 + 127) / 128 * 128;
   if ((p.VQ + TILE_M - 1) / TILE_M * ((g.Co + 63) / 64) >= ((int64_t)1 << 31)) return p;
   p.scratch_bytes = (size_t)kStatusBytes + (size_t)p.K2p * ((g.Co + 63) / 64 * 64) * g.Kw * 2;
-  int rs, sa, sb, vg, smem;
-  if (!choose_rings(tile_bn(g), tile_bn(g), g.Kw, p, &rs, &sa, &sb, &vg, &smem)) return p;
+  int rs, sa, sb, vg, resident, smem;
+  if (!choose_rings(tile_bn(g), tile_bn(g), g.Kw, 2, p, &rs, &sa, &sb, &vg, &resident, &smem)) return p;
   p.eligible = true;
   return p;
 }
@@ -946,6 +967,7 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, float* y, void* scratch,
   q.magic_kh = magic16(g.Kh); q.magic_s = magic16(g.s);
   q.rs = q.sa = q.sb = 2;
   q.vg = 1;
+  q.resident = 0;
   q.ntm = q.nwork = 0;
   q.frows = ncog * 4;
   if (pair) return launch_pair<256>(fmap, wmap, q, plan, g.Co, stream);
