@@ -64,6 +64,7 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
   l->f16_shift = false;
   l->f16_raw = false;
   l->f16_mat = false;
+  l->f16_matc = false;
   l->koff_off = kStatusBytes;
   l->filter_off = (size_t)round_up((int64_t)l->koff_off + 4 * l->Kp, 256);
   int64_t fbytes = l->Kp * l->Co_pad * (dtype == IM2WIN_F32 ? 4 : 2);
@@ -87,14 +88,20 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
       if (shift_total > l->total) l->total = shift_total;
     }
     const MatPlan mat = plan_f16_mat(g);
+    const MatcPlan matc = mat.eligible ? MatcPlan{} : plan_f16_matc(g);
+    const char* force = getenv("IM2WIN_F16_KERNEL");
+    // measured: the matrix-transpose kernels win for strided layers (the others stage such layers
+    // with 2-byte gathers) and, in their CTA-pair form, for kernels up to 5 wide with more than 128
+    // output channels; IM2WIN_F16_KERNEL=mat forces them wherever they can run (a testing aid)
+    const bool want = force ? strcmp(force, "mat") == 0 : (g.s > 1 || (g.Co > 128 && g.Kw <= 5));
     if (mat.eligible) {
-      const char* force = getenv("IM2WIN_F16_KERNEL");
-      // measured: the matrix-transpose kernel wins for strided layers (the others stage such
-      // layers with 2-byte gathers) and, in its CTA-pair form, for kernels up to 5 wide with more
-      // than 128 output channels; IM2WIN_F16_KERNEL=mat forces it everywhere (a testing aid)
-      l->f16_mat = force ? strcmp(force, "mat") == 0 : (g.s > 1 || (g.Co > 128 && g.Kw <= 5));
+      l->f16_mat = want;
       const size_t mat_total = (size_t)round_up((int64_t)mat.scratch_bytes, 256);
       if (mat_total > l->total) l->total = mat_total;
+    } else if (matc.eligible) {
+      l->f16_matc = want;
+      const size_t matc_total = (size_t)round_up((int64_t)matc.scratch_bytes, 256);
+      if (matc_total > l->total) l->total = matc_total;
     }
   }
   return IM2WIN_OK;
@@ -125,6 +132,7 @@ static im2win_status conv_common(const void* window, const void* filter, float* 
   if (mode & kDoPack) {
     if (dtype == IM2WIN_F32) e = launch_pack_f32(static_cast<const float*>(filter), scratch, g, l, stream);
     else if (l.f16_mat) e = launch_pack_f16_mat(static_cast<const uint16_t*>(filter), scratch, g, stream);
+    else if (l.f16_matc) e = launch_pack_f16_matc(static_cast<const uint16_t*>(filter), scratch, g, stream);
     else if (l.f16_raw)
       e = launch_pack_f16_raw(static_cast<const uint16_t*>(filter), scratch, g, l, plan_f16_raw(g), stream);
     else if (l.f16_shift) e = launch_pack_f16_shift(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
@@ -134,6 +142,7 @@ static im2win_status conv_common(const void* window, const void* filter, float* 
   if (mode & kDoConv) {
     if (dtype == IM2WIN_F32) e = launch_conv_f32(static_cast<const float*>(window), y, scratch, g, l, stream);
     else if (l.f16_mat) e = launch_conv_f16_mat(static_cast<const uint16_t*>(window), y, scratch, g, stream);
+    else if (l.f16_matc) e = launch_conv_f16_matc(static_cast<const uint16_t*>(window), y, scratch, g, stream);
     else if (l.f16_raw) e = launch_conv_f16_raw(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
     else if (l.f16_shift) e = launch_conv_f16_shift(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
     else e = launch_conv_f16_gather(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);

@@ -37,6 +37,7 @@ struct ScratchLayout {
   bool f16_shift;        // fp16 only: a shifted-view kernel (and its filter layout) is used
   bool f16_raw;          // fp16 only: the bulk-copy variant of the shifted-view kernel is used
   bool f16_mat;          // fp16 only: the matrix-transpose variant is used (own scratch layout)
+  bool f16_matc;         // fp16 only: its general form (channel classes / batched raw stages) is used
 };
 
 // Tile geometry of the fp16 shifted-view kernel for one layer (see conv_f16_shift.cu).
@@ -69,6 +70,17 @@ struct MatPlan {
 };
 MatPlan plan_f16_mat(const Geometry& g);
 
+// Tile geometry of the general matrix-transpose kernel (channel classes, batched raw stages; see
+// conv_f16_matc.cu).
+struct MatcPlan {
+  bool eligible;
+  int32_t Wq, rows, R, nplanes, rawbox, box_bytes, raw_stage_bytes, a_stage_bytes, num_kb;
+  int32_t P, shift1, kbpc, units0, units1;   // channel classes (conv_f16_matc.cu, WinMaps)
+  int64_t K2p, VQ;
+  size_t scratch_bytes;  // status block + packed filter
+};
+MatcPlan plan_f16_matc(const Geometry& g);
+
 constexpr int kStatusBytes = 256;
 constexpr int kF32KBlock = 16;     // k-block of the fp32 kernel
 constexpr int kF16KBlock = 64;     // k-block of the fp16 kernel (64 halves = one 128-byte swizzle row)
@@ -95,6 +107,9 @@ cudaError_t launch_conv_f16_raw(const uint16_t* window, float* y, void* scratch,
 cudaError_t launch_pack_f16_mat(const uint16_t* filter, void* scratch, const Geometry& g, cudaStream_t stream);
 cudaError_t launch_conv_f16_mat(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                 cudaStream_t stream);
+cudaError_t launch_pack_f16_matc(const uint16_t* filter, void* scratch, const Geometry& g, cudaStream_t stream);
+cudaError_t launch_conv_f16_matc(const uint16_t* window, float* y, void* scratch, const Geometry& g,
+                                 cudaStream_t stream);
 cudaError_t launch_conv_f16_gather(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                    const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratch, const Geometry& g,

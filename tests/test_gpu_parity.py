@@ -47,6 +47,10 @@ SMALL = [
     L("vec_w6_s2", 2, 3, 9, 6, 4, 3, 3, 2, 1, 31),              # W = 6: no vectors (12- / 24-byte rows), stride 2
     L("vec_w16_k7", 2, 3, 20, 16, 4, 7, 7, 2, 3, 32),           # tall kernel with vector loads (fp16), stride 2
     L("vec_w24_k11", 1, 2, 26, 24, 3, 11, 11, 1, 5, 33),        # Kh = 11 with vector loads (fp16)
+    L("cls2_s2", 2, 12, 12, 12, 20, 3, 3, 2, 1, 34),            # fp16 plane pitch 8 (mod 16): two channel classes, stride 2
+    L("cls2_wide", 3, 10, 9, 10, 260, 3, 3, 1, 1, 35),          # ... with CTA pairs
+    L("cls2_deep", 2, 40, 9, 10, 24, 3, 3, 1, 1, 36),           # ... several k-blocks per class (lane tables per class)
+    L("cls2_odd", 2, 22, 9, 10, 24, 3, 3, 1, 1, 37),            # ... 11 channels per class: ragged last octet
 ]
 
 
