@@ -730,8 +730,9 @@ conv_f16_mat_pair_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_
 // them at their place in the tile images.
 __global__ void pack_f16_mat_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, uint32_t* status,
                                     int C, int Co, int Kh, int Kw, int K2p, int ncog, int noct) {
-  extern __shared__ uint16_t pack_s[];
+  extern __shared__ __align__(16) uint16_t pack_s[];
   let_next_kernel_start();
+  const size_t f_total = (size_t)Co * C * Kh * Kw;
   if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
   const int num_kb = K2p / KB;
   const int T = Kh * Kw;
@@ -744,12 +745,23 @@ __global__ void pack_f16_mat_kernel(const uint16_t* __restrict__ f, uint16_t* __
   int nsrc = (C - c_a < noct * 8 ? C - c_a : noct * 8) * T;    // source halves that exist
   if (nsrc < 0) nsrc = 0;
   for (int co = blockIdx.y; co < ncog * 64; co += gridDim.y) {
+    // The run is read with 16-byte loads from the 16-byte boundary at or before its start; run
+    // element i then sits at run[i] = pack_s[i + mis].
+    const size_t start = ((size_t)co * C + c_a) * T;
+    const int mis = (int)(start & 7);
     __syncthreads();
     if (co < Co) {
-      const uint16_t* src = f + ((size_t)co * C + c_a) * T;
-      for (int i = threadIdx.x; i < nsrc; i += blockDim.x) pack_s[i] = src[i];
+      for (int vec = threadIdx.x; vec * 8 < mis + nsrc; vec += blockDim.x) {
+        const size_t i0 = start - mis + (size_t)vec * 8;
+        if (i0 + 8 <= f_total) {
+          reinterpret_cast<uint4*>(pack_s)[vec] = __ldg(reinterpret_cast<const uint4*>(f + i0));
+        } else {
+          for (int h = 0; h < 8; ++h) pack_s[vec * 8 + h] = i0 + h < f_total ? f[i0 + h] : (uint16_t)0;
+        }
+      }
     }
     __syncthreads();
+    const uint16_t* run = pack_s + mis;
     const int r = co & 63;
     const int nunits = unit_b - unit_a;
     for (int i = threadIdx.x; i < nunits * Kw; i += blockDim.x) {
@@ -764,7 +776,7 @@ __global__ void pack_f16_mat_kernel(const uint16_t* __restrict__ f, uint16_t* __
         for (int lo = 0; lo < 2; ++lo) {
           const int e = 2 * h + lo;
           const int idx = ((oct - oct_a) * 8 + e) * T + u * Kw + v;     // (c - c_a)*T + u*Kw + v
-          const uint32_t val = (co < Co && idx < nsrc && oct < oct_a + noct) ? pack_s[idx] : 0u;
+          const uint32_t val = (co < Co && idx < nsrc && oct < oct_a + noct) ? run[idx] : 0u;
           pair |= val << (16 * lo);
         }
         w[h] = pair;
@@ -1055,7 +1067,7 @@ cudaError_t launch_pack_f16_matc(const uint16_t* filter, void* scratch, const Ge
   int noct = 4096 / (8 * g.T);                          // octets per block: staging of <= 4096 halves
   if (noct < 1) noct = 1;
   if (noct > Cp8) noct = Cp8;
-  const size_t smem = (size_t)noct * 8 * g.T * sizeof(uint16_t);
+  const size_t smem = ((size_t)noct * 8 * g.T + 16) * sizeof(uint16_t);
   if (smem > 48 * 1024) return cudaErrorInvalidValue;
   dim3 grid((unsigned)((Cp8 + noct - 1) / noct), (unsigned)(ncog * 64 < 32768 ? ncog * 64 : 32768));
   pack_f16_mat_kernel<<<grid, 256, smem, stream>>>(filter, fp, reinterpret_cast<uint32_t*>(base), g.C, g.Co, g.Kh, g.Kw,

@@ -88,25 +88,43 @@ __global__ void pack_f16_kernel(const uint16_t* __restrict__ f, uint16_t* __rest
 __global__ void pack_f16_shift_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp,
                                       uint32_t* __restrict__ table, uint32_t* __restrict__ status,
                                       PackParams q, int raw_pitch, int nslot, int chunk) {
-  extern __shared__ uint16_t pack_s[];
+  extern __shared__ __align__(16) uint16_t pack_s[];
   if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
   const int K2 = q.C * q.Kh;
   const int K2p = (int)q.Kp;
   const int k2a = blockIdx.x * chunk;
   const int k2b = k2a + chunk < K2p ? k2a + chunk : K2p;
   const int nreal = (k2b < K2 ? k2b : K2) - k2a;          // k2 of this chunk that exist in the filter (may be <= 0)
+  const size_t f_total = (size_t)q.Co * K2 * q.Kw;
   for (int co = blockIdx.y; co < q.Co; co += gridDim.y) {
-    const uint16_t* src = f + ((size_t)co * K2 + k2a) * q.Kw;
+    // The run is read with 16-byte loads from the 16-byte boundary at or before its start; run
+    // element i then sits at pack_s[i + mis].
+    const size_t start = ((size_t)co * K2 + k2a) * q.Kw;
+    const int mis = (int)(start & 7);
+    const int n = nreal > 0 ? nreal * q.Kw : 0;
     __syncthreads();
-    for (int i = threadIdx.x; i < nreal * q.Kw; i += blockDim.x) pack_s[i] = src[i];
+    for (int vec = threadIdx.x; vec * 8 < mis + n; vec += blockDim.x) {
+      const size_t i0 = start - mis + (size_t)vec * 8;
+      if (i0 + 8 <= f_total) {
+        reinterpret_cast<uint4*>(pack_s)[vec] = __ldg(reinterpret_cast<const uint4*>(f + i0));
+      } else {
+        for (int h = 0; h < 8; ++h) pack_s[vec * 8 + h] = i0 + h < f_total ? f[i0 + h] : (uint16_t)0;
+      }
+    }
     __syncthreads();
+    const uint16_t* run = pack_s + mis;
     for (int v = 0; v < q.Kw; ++v) {
       uint16_t* dst = fp + ((size_t)v * q.Co + co) * K2p + k2a;
-      // two k2 per thread: one 32-bit store (k2a and K2p are even)
-      for (int j = 2 * threadIdx.x; j < k2b - k2a; j += 2 * blockDim.x) {
-        const uint32_t lo = j < nreal ? pack_s[j * q.Kw + v] : 0u;
-        const uint32_t hi = j + 1 < nreal ? pack_s[(j + 1) * q.Kw + v] : 0u;
-        *reinterpret_cast<uint32_t*>(dst + j) = lo | (hi << 16);
+      // eight k2 per thread: one 16-byte store (k2a and K2p are multiples of 8)
+      for (int j = 8 * threadIdx.x; j < k2b - k2a; j += 8 * blockDim.x) {
+        uint32_t w[4];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+          const uint32_t lo = j + 2 * h < nreal ? run[(j + 2 * h) * q.Kw + v] : 0u;
+          const uint32_t hi = j + 2 * h + 1 < nreal ? run[(j + 2 * h + 1) * q.Kw + v] : 0u;
+          w[h] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
       }
     }
   }
@@ -169,8 +187,8 @@ static cudaError_t pack_shift_common(const uint16_t* filter, void* scratch, cons
   unsigned char* base = static_cast<unsigned char*>(scratch);
   PackParams q = make_params(g, l);
   int chunk = 512;                                          // k2 per block: staging of chunk*Kw halves within 40 KB
-  while (chunk > 2 && (size_t)chunk * g.Kw * sizeof(uint16_t) > 40 * 1024) chunk /= 2;
-  const size_t smem = (size_t)chunk * g.Kw * sizeof(uint16_t);
+  while (chunk > 8 && (size_t)chunk * g.Kw * sizeof(uint16_t) > 40 * 1024) chunk /= 2;
+  const size_t smem = ((size_t)chunk * g.Kw + 16) * sizeof(uint16_t);
   if (smem > 48 * 1024) return cudaErrorInvalidValue;
   dim3 grid((unsigned)((q.Kp + chunk - 1) / chunk), (unsigned)(g.Co < 32768 ? g.Co : 32768));
   pack_f16_shift_kernel<<<grid, 256, smem, stream>>>(filter, reinterpret_cast<uint16_t*>(base + l.filter_off),
