@@ -65,6 +65,7 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
   l->f16_raw = false;
   l->f16_mat = false;
   l->f16_matc = false;
+  l->f16_stem = false;
   l->koff_off = kStatusBytes;
   l->filter_off = (size_t)round_up((int64_t)l->koff_off + 4 * l->Kp, 256);
   int64_t fbytes = l->Kp * l->Co_pad * (dtype == IM2WIN_F32 ? 4 : 2);
@@ -73,17 +74,21 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
     // The shifted-view kernel is used whenever the layer is eligible; IM2WIN_F16_KERNEL=gather
     // forces the general gather kernel (a testing aid).  The scratch size covers both layouts.
     const ShiftPlan plan = plan_f16_shift(g);
-    if (plan.eligible) {
-      const size_t shift_filter_off = (size_t)round_up((int64_t)kStatusBytes + 4 * plan.K2p, 256);
-      const size_t shift_total = (size_t)round_up((int64_t)shift_filter_off + plan.K2p * g.Co * g.Kw * 2, 256);
+    const bool stem_ok = plan_f16_stem(g).eligible;       // shares the filter layout of the shifted-view kernel
+    if (plan.eligible || stem_ok) {
+      const int64_t K2p = round_up((int64_t)g.C * g.Kh, kF16KBlock);
+      const size_t shift_filter_off = (size_t)round_up((int64_t)kStatusBytes + 4 * K2p, 256);
+      const size_t shift_total = (size_t)round_up((int64_t)shift_filter_off + K2p * g.Co * g.Kw * 2, 256);
       const char* force = getenv("IM2WIN_F16_KERNEL");
       const bool use_shift = !(force && strcmp(force, "gather") == 0);
       if (use_shift) {
-        l->f16_shift = true;
-        l->Kp = plan.K2p;
+        l->f16_shift = plan.eligible;
+        l->Kp = K2p;
         l->filter_off = shift_filter_off;
         // the bulk-copy variant shares the filter layout; IM2WIN_F16_KERNEL=shift keeps the gathering one
-        l->f16_raw = plan_f16_raw(g).eligible && !(force && strcmp(force, "shift") == 0);
+        l->f16_raw = plan.eligible && plan_f16_raw(g).eligible && !(force && strcmp(force, "shift") == 0);
+        // layers with one k-block: their own kernel unless another one is forced
+        l->f16_stem = stem_ok && (!force || strcmp(force, "stem") == 0);
       }
       if (shift_total > l->total) l->total = shift_total;
     }
@@ -94,12 +99,14 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
     // with 2-byte gathers) and, in their CTA-pair form, for kernels up to 5 wide with more than 128
     // output channels; IM2WIN_F16_KERNEL=mat forces them wherever they can run (a testing aid)
     const bool want = force ? strcmp(force, "mat") == 0 : (g.s > 1 || (g.Co > 128 && g.Kw <= 5));
+    // (the scratch size covers every layout, whichever kernel is picked or forced)
+    const bool use_mat = want && !l->f16_stem;
     if (mat.eligible) {
-      l->f16_mat = want;
+      l->f16_mat = use_mat;
       const size_t mat_total = (size_t)round_up((int64_t)mat.scratch_bytes, 256);
       if (mat_total > l->total) l->total = mat_total;
     } else if (matc.eligible) {
-      l->f16_matc = want;
+      l->f16_matc = use_mat;
       const size_t matc_total = (size_t)round_up((int64_t)matc.scratch_bytes, 256);
       if (matc_total > l->total) l->total = matc_total;
     }
@@ -131,6 +138,7 @@ static im2win_status conv_common(const void* window, const void* filter, float* 
   cudaError_t e = cudaSuccess;
   if (mode & kDoPack) {
     if (dtype == IM2WIN_F32) e = launch_pack_f32(static_cast<const float*>(filter), scratch, g, l, stream);
+    else if (l.f16_stem) e = launch_pack_f16_shift(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
     else if (l.f16_mat) e = launch_pack_f16_mat(static_cast<const uint16_t*>(filter), scratch, g, stream);
     else if (l.f16_matc) e = launch_pack_f16_matc(static_cast<const uint16_t*>(filter), scratch, g, stream);
     else if (l.f16_raw)
@@ -141,6 +149,7 @@ static im2win_status conv_common(const void* window, const void* filter, float* 
   }
   if (mode & kDoConv) {
     if (dtype == IM2WIN_F32) e = launch_conv_f32(static_cast<const float*>(window), y, scratch, g, l, stream);
+    else if (l.f16_stem) e = launch_conv_f16_stem(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
     else if (l.f16_mat) e = launch_conv_f16_mat(static_cast<const uint16_t*>(window), y, scratch, g, stream);
     else if (l.f16_matc) e = launch_conv_f16_matc(static_cast<const uint16_t*>(window), y, scratch, g, stream);
     else if (l.f16_raw) e = launch_conv_f16_raw(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);

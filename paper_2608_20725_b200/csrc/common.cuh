@@ -38,15 +38,18 @@ struct ScratchLayout {
   bool f16_raw;          // fp16 only: the bulk-copy variant of the shifted-view kernel is used
   bool f16_mat;          // fp16 only: the matrix-transpose variant is used (own scratch layout)
   bool f16_matc;         // fp16 only: its general form (channel classes / batched raw stages) is used
+  bool f16_stem;         // fp16 only: the one-k-block kernel for C*Kh <= 64 is used (filter layout of f16_shift)
 };
 
 // Tile geometry of the fp16 shifted-view kernel for one layer (see conv_f16_shift.cu).
 struct ShiftPlan {
   bool eligible;
-  int32_t Wq;            // virtual positions per strip = Wp / s
+  int32_t Wq;            // virtual positions per strip = ceil(Wp / s)
   int32_t rows;          // rows of one shared-memory sub-tile: 128 + halo, multiple of 8
   int32_t total_rows;    // s * rows
   int32_t items;         // 16-byte chunks each producer thread fills per stage
+  int32_t chunks;        // 16-byte chunks staged per row (8, fewer when one short k-block is all)
+  int32_t nks_last;      // 16-wide MMA steps of the last k-block
   int64_t K2, K2p;       // C*Kh and its round-up to 64
   int64_t VQ;            // N*Ho*Wq virtual positions
 };
@@ -81,6 +84,15 @@ struct MatcPlan {
 };
 MatcPlan plan_f16_matc(const Geometry& g);
 
+// Tile geometry of the one-k-block kernel for layers with C*Kh <= 64 (see conv_f16_stem.cu).
+struct StemPlan {
+  bool eligible;
+  int32_t Wq, ragged, rows, R, nks, chan_region, raw_stage_bytes, a_stage_bytes, b_stage_bytes, bn;
+  int32_t sa, rs, sb, resident, smem_bytes;
+  int64_t VQ;
+};
+StemPlan plan_f16_stem(const Geometry& g);
+
 constexpr int kStatusBytes = 256;
 constexpr int kF32KBlock = 16;     // k-block of the fp32 kernel
 constexpr int kF16KBlock = 64;     // k-block of the fp16 kernel (64 halves = one 128-byte swizzle row)
@@ -110,6 +122,8 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, float* y, void* scratch,
 cudaError_t launch_pack_f16_matc(const uint16_t* filter, void* scratch, const Geometry& g, cudaStream_t stream);
 cudaError_t launch_conv_f16_matc(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                  cudaStream_t stream);
+cudaError_t launch_conv_f16_stem(const uint16_t* window, float* y, void* scratch, const Geometry& g,
+                                 const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_conv_f16_gather(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                    const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratch, const Geometry& g,

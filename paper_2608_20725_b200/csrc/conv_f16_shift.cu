@@ -17,9 +17,11 @@
 // tensor is read from L2/HBM once per output-channel tile and written to shared
 // memory once, instead of Kw times as in an im2col-style expansion.
 //
-// The MMA rows are "virtual positions" q = (n*Ho + ho)*Wq + kq with Wq = Wp/s:
+// The MMA rows are "virtual positions" q = (n*Ho + ho)*Wq + kq with Wq = ceil(Wp/s):
 // q runs over ALL columns of a strip, also the (Wq - Wo) trailing ones that are
-// no output; their accumulator rows are computed and dropped.  Tiles are 128
+// no output; their accumulator rows are computed and dropped.  (When s does not
+// divide Wp the last virtual position of a strip lacks some columns; they are
+// staged as zeros and only dropped rows read them.)  Tiles are 128
 // consecutive q and may span strips and images.  Useful work is Wo/Wq of the
 // MMA work (0.97 for 56-wide rows, 0.78 for 7-wide rows).
 //
@@ -58,7 +60,10 @@ struct ShiftParams {
   uint32_t* status;
   int64_t VQ, img_stride, strip, chan_stride, window_elems;
   int32_t C, N;
-  int32_t Wq, Ho, Wo, HoWo, Co, Kh, Kw, s, num_kb;
+  int32_t Wq, Wp, Ho, Wo, HoWo, Co, Kh, Kw, s, num_kb;
+  int32_t chunks;         // 16-byte chunks of a row that are staged (8, fewer when one short k-block is all)
+  int32_t chunks_last;    // ... of them in the last k-block, = 2 * nks_last
+  int32_t nks_last;       // 16-wide MMA steps of the last k-block
   int32_t halo8;          // halo rows of a sub-tile, rounded up to 8
   int32_t nbig;           // the first nbig tiles are 256 positions tall (two MMA halves), the rest 128
   int32_t a_stage_bytes, sa, sb;
@@ -127,10 +132,14 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
     // image and is masked afterwards) so that the compiler can issue all of a group's
     // loads back to back.
     uint32_t rel[ITEMS], meta[ITEMS];
-    const int n_items = total_rows * 8;
-    const int64_t img_rows = (int64_t)q.Ho * q.Wq;          // virtual positions per image
-    const int64_t n_first = q0 / img_rows;
-    const uint16_t* __restrict__ tile_win = q.win + n_first * q.img_stride;
+    // Rows are numbered in blocks of 8 per sub-tile (row i of sub-tile j <-> strip column i*s + j), so
+    // that the lanes of a warp read 32 neighbouring columns whatever the stride and the eight lanes of
+    // a store phase hit eight different rows of the swizzle pattern.
+    const int n_items = total_rows * q.chunks;
+    const uint32_t img_rows = (uint32_t)(q.Ho * q.Wq);       // virtual positions per image
+    const uint32_t n_first = (uint32_t)q0 / img_rows;
+    const uint16_t* __restrict__ tile_win = q.win + (int64_t)n_first * q.img_stride;
+    const int blk_rows = 8 * q.s;
 #pragma unroll
     for (int it = 0; it < ITEMS; ++it) {
       const int item = threadIdx.x + it * PRODUCER_THREADS;
@@ -139,17 +148,21 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
       if (item < n_items) {
         const int ch = item / total_rows;
         const int ri = item - ch * total_rows;
-        const int sub = ri / rows;
-        const int i = ri - sub * rows;
+        const int blk = ri / blk_rows;
+        const int w = ri - blk * blk_rows;
+        const int sub = w >> 3;
+        const int i = blk * 8 + (w & 7);
         meta[it] = (uint32_t)(sub * sub_bytes + i * 128 + ((ch ^ (i & 7)) << 4)) | (uint32_t)ch;
-        const int64_t vq = q0 + i;
-        if (vq < q.VQ) {
-          const int64_t sg = vq / q.Wq;
-          const int kq = (int)(vq - sg * q.Wq);
-          const int64_t n = sg / q.Ho;
-          const int ho = (int)(sg - n * q.Ho);
-          rel[it] = (uint32_t)((n - n_first) * q.img_stride + ho * q.strip + (int64_t)(kq * q.s + sub) * q.Kh);
-          meta[it] |= 8u;
+        const uint32_t vq = (uint32_t)q0 + (uint32_t)i;
+        if (vq < (uint32_t)q.VQ) {
+          const uint32_t sg = vq / (uint32_t)q.Wq;
+          const int col = (int)(vq - sg * (uint32_t)q.Wq) * q.s + sub;
+          const uint32_t n = sg / (uint32_t)q.Ho;
+          const int ho = (int)(sg - n * (uint32_t)q.Ho);
+          if (col < q.Wp) {                    // the last virtual column of a strip may be cut short
+            rel[it] = (uint32_t)((int64_t)(n - n_first) * q.img_stride + ho * q.strip + (int64_t)col * q.Kh);
+            meta[it] |= 8u;
+          }
         }
       }
     }
@@ -164,7 +177,7 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
     constexpr int G = ITEM_GROUP;
     constexpr int NG = ITEMS / G;
     const uint16_t* __restrict__ zero16 = reinterpret_cast<const uint16_t*>(q.status + 2);
-    auto issue = [&](int kb, int gidx, uint32_t (&h)[G][8]) {
+    auto issue = [&](int kb, int climit, int gidx, uint32_t (&h)[G][8]) {
       const int4* kt = reinterpret_cast<const int4*>(koff_s + kb * KB);   // this k-block's offsets (shared memory)
 #pragma unroll
       for (int gi = 0; gi < G; ++gi) {
@@ -173,16 +186,16 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
         const int4 o0 = kt[ch * 2], o1 = kt[ch * 2 + 1];
         const int32_t off[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
         const uint16_t* src = tile_win + rel[it];
-        const bool row_ok = (meta[it] & 8u) != 0;
+        const bool row_ok = (meta[it] & 8u) != 0 && ch < climit;
 #pragma unroll
         for (int e = 0; e < 8; ++e) h[gi][e] = (uint32_t)__ldg((row_ok && off[e] >= 0) ? src + off[e] : zero16);
       }
     };
-    auto store = [&](uint32_t a_stage, int gidx, const uint32_t (&h)[G][8]) {
+    auto store = [&](uint32_t a_stage, int climit, int gidx, const uint32_t (&h)[G][8]) {
 #pragma unroll
       for (int gi = 0; gi < G; ++gi) {
         const int it = gidx * G + gi;
-        if (meta[it] != 0xffffffffu) {
+        if (meta[it] != 0xffffffffu && (int)(meta[it] & 7u) < climit) {
           const uint32_t w0 = h[gi][0] | (h[gi][1] << 16), w1 = h[gi][2] | (h[gi][3] << 16);
           const uint32_t w2 = h[gi][4] | (h[gi][5] << 16), w3 = h[gi][6] | (h[gi][7] << 16);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_stage + (meta[it] & ~15u)), "r"(w0),
@@ -197,16 +210,17 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
     uint32_t buf[G][8];
     for (int kb = 0; kb < q.num_kb && ok; ++kb) {
       const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
+      const int climit = kb == q.num_kb - 1 ? q.chunks_last : 8;   // the MMAs skip the padded tail of k
 #pragma unroll
       for (int gidx = 0; gidx < NG; ++gidx) {
-        issue(kb, gidx, buf);
+        issue(kb, climit, gidx, buf);
         if (gidx == 0) {
           if (threadIdx.x == 0) TIMER_LAP(2);   // issuing loads
           if (lane == 0) ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
           ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
           if (threadIdx.x == 0) TIMER_LAP(1);   // wait for a free stage
         }
-        if (ok) store(a_stage, gidx, buf);
+        if (ok) store(a_stage, climit, gidx, buf);
       }
       if (!ok) break;
       if (threadIdx.x == 0) TIMER_LAP(3);   // waiting for the loads, pack + store
@@ -229,16 +243,16 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
       const int lq = warp & 3;                 // tensor-memory lane quadrant this warp may read
       const int chalf = warp >> 2;             // which half of the channel tile
       for (int half = 0; half < mt; ++half) {
-        const int64_t vq = q0 + half * TILE_M + lq * 32 + lane;   // accumulator row = virtual position
+        const uint32_t vq = (uint32_t)q0 + (uint32_t)(half * TILE_M + lq * 32 + lane);   // accumulator row = virtual position
         bool valid = false;
         float* yrow = q.y;
-        if (vq < q.VQ) {
-          const int64_t sg = vq / q.Wq;
-          const int kq = (int)(vq - sg * q.Wq);
-          const int64_t n = sg / q.Ho;
-          const int ho = (int)(sg - n * q.Ho);
+        if (vq < (uint32_t)q.VQ) {
+          const uint32_t sg = vq / (uint32_t)q.Wq;
+          const int kq = (int)(vq - sg * (uint32_t)q.Wq);
+          const uint32_t n = sg / (uint32_t)q.Ho;
+          const int ho = (int)(sg - n * (uint32_t)q.Ho);
           valid = kq < q.Wo;                   // trailing columns of a strip are no output
-          yrow += (n * q.Co) * q.HoWo + ho * q.Wo + kq;
+          yrow += ((int64_t)n * q.Co) * q.HoWo + ho * q.Wo + kq;
         }
         const uint32_t lane_base = tmem_acc + ((uint32_t)(lq * 32) << 16) + (uint32_t)(half * BN);
 #pragma unroll 1
@@ -301,6 +315,7 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
       if (!ok) break;
       TIMER_LAP(9);                         // MMA warp: wait for an S stage
       const uint32_t a_lo_stage = a_lo0 + (uint32_t)(sta * (q.a_stage_bytes >> 4));
+      const int nks = kb == q.num_kb - 1 ? q.nks_last : KB / 16;
       uint32_t a_view = 0;                  // offset of kernel column v's view inside the stage
       int sub = 0;
       for (int v = 0; v < q.Kw; ++v) {
@@ -324,7 +339,7 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
           for (int half = 0; half < mt; ++half) {
 #pragma unroll
             for (int j = 0; j < KB / 16; ++j)
-              umma_f16_lohi(acc_col, a_lo + 2 * j, b_lo + 2 * j, idesc, first | (uint32_t)j);
+              if (j < nks) umma_f16_lohi(acc_col, a_lo + 2 * j, b_lo + 2 * j, idesc, first | (uint32_t)j);
             a_lo += (uint32_t)(TILE_M * 128) >> 4;
             acc_col += (uint32_t)BN;
           }
@@ -453,7 +468,7 @@ cudaError_t launch_bn(const CUtensorMap& fmap, const ShiftParams& q0, const Shif
     q.a_stage_bytes = s * (TILE_M + q.halo8) * 128;
   }
   const int rows_all = q.a_stage_bytes / 128;
-  const int items = (rows_all * 8 + PRODUCER_THREADS - 1) / PRODUCER_THREADS;
+  const int items = (rows_all * q.chunks + PRODUCER_THREADS - 1) / PRODUCER_THREADS;
   if (items <= 5) return launch_variant<BN, 5>(fmap, q, plan, co, stream);
   if (items <= 10) return launch_variant<BN, 10>(fmap, q, plan, co, stream);
   if (items <= 15) return launch_variant<BN, 15>(fmap, q, plan, co, stream);
@@ -468,21 +483,23 @@ cudaError_t launch_bn(const CUtensorMap& fmap, const ShiftParams& q0, const Shif
 ShiftPlan plan_f16_shift(const Geometry& g) {
   ShiftPlan p{};
   p.eligible = false;
-  if (g.Wp % g.s != 0) return p;
-  p.Wq = g.Wp / g.s;
+  p.Wq = (g.Wp + g.s - 1) / g.s;
   const int halo = (g.Kw - 1 + g.s - 1) / g.s;
   p.rows = TILE_M + (halo + 7) / 8 * 8;
   p.total_rows = g.s * p.rows;
-  p.items = (p.total_rows * 8 + PRODUCER_THREADS - 1) / PRODUCER_THREADS;
   p.K2 = (int64_t)g.C * g.Kh;
   p.K2p = (p.K2 + KB - 1) / KB * KB;
   p.VQ = (int64_t)g.N * g.Ho * p.Wq;
+  // the MMAs stop at the last 16-wide step that holds real k2; a single short k-block is staged that narrow
+  p.nks_last = (int32_t)((p.K2 - (p.K2p - KB) + 15) / 16);
+  p.chunks = p.K2p == KB ? 2 * p.nks_last : 8;
+  p.items = (p.total_rows * p.chunks + PRODUCER_THREADS - 1) / PRODUCER_THREADS;
   if (p.items > 15) return p;
   if (p.K2p * 4 > 24 * 1024) return p;                    // offset table lives in shared memory
   if (g.img_stride >= ((int64_t)1 << 30)) return p;       // 32-bit offsets relative to the tile's first image
   // two stages of each ring must fit even for the widest channel tile
   if (2 * p.total_rows * 128 + 2 * 256 * KB * 2 + p.K2p * 4 > kSmemBudget - 2048) return p;
-  if ((p.VQ + TILE_M - 1) / TILE_M >= ((int64_t)1 << 31)) return p;
+  if (p.VQ + 2 * TILE_M >= ((int64_t)1 << 31)) return p;   // 32-bit position arithmetic
   p.eligible = true;
   return p;
 }
@@ -514,7 +531,8 @@ cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratc
   q.status = reinterpret_cast<uint32_t*>(base);
   q.VQ = plan.VQ; q.img_stride = g.img_stride; q.strip = g.strip;
   q.chan_stride = g.chan_stride; q.window_elems = g.window_elems; q.C = g.C; q.N = g.N;
-  q.Wq = plan.Wq; q.Ho = g.Ho; q.Wo = g.Wo; q.HoWo = g.Ho * g.Wo; q.Co = g.Co;
+  q.Wq = plan.Wq; q.Wp = g.Wp; q.chunks = plan.chunks; q.nks_last = plan.nks_last;
+  q.chunks_last = 2 * plan.nks_last; q.Ho = g.Ho; q.Wo = g.Wo; q.HoWo = g.Ho * g.Wo; q.Co = g.Co;
   q.Kh = g.Kh; q.Kw = g.Kw; q.s = g.s; q.num_kb = (int32_t)(plan.K2p / KB);
   q.halo8 = plan.rows - TILE_M;
   q.nbig = 0;

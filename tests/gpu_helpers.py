@@ -46,9 +46,9 @@ def gpu_transform(x_cpu: torch.Tensor, dims: dict) -> np.ndarray:
 def gpu_conv(x_cpu: torch.Tensor, f_cpu: torch.Tensor, dims: dict, precision: str):
     """Transform + convolution on the GPU.  precision 'f32', 'f16' (the kernel the library picks),
     'f16-shift' (the gathering shifted-view kernel forced), 'f16-mat' (the matrix-transpose
-    shifted-view kernel forced) or 'f16-gather' (the general fp16 kernel forced); inputs are cast with torch's
+    shifted-view kernel forced), 'f16-stem' (the one-k-block kernel where it can run) or 'f16-gather' (the general fp16 kernel forced); inputs are cast with torch's
     round-to-nearest-even conversion.  Returns (y float32 numpy, x_used, f_used as float32 numpy)."""
-    if precision in ("f16-gather", "f16-shift", "f16-mat"):
+    if precision in ("f16-gather", "f16-shift", "f16-mat", "f16-stem"):
         os.environ["IM2WIN_F16_KERNEL"] = precision.split("-")[1]
         try:
             return gpu_conv(x_cpu, f_cpu, dims, "f16")

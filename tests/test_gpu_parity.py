@@ -51,6 +51,15 @@ SMALL = [
     L("cls2_wide", 3, 10, 9, 10, 260, 3, 3, 1, 1, 35),          # ... with CTA pairs
     L("cls2_deep", 2, 40, 9, 10, 24, 3, 3, 1, 1, 36),           # ... several k-blocks per class (lane tables per class)
     L("cls2_odd", 2, 22, 9, 10, 24, 3, 3, 1, 1, 37),            # ... 11 channels per class: ragged last octet
+    L("rag_s4", 2, 3, 39, 39, 20, 11, 11, 4, 0, 38),            # Wp % s = 3: cut-short last virtual column, one short k-block
+    L("rag_s3", 3, 5, 20, 22, 12, 4, 4, 3, 0, 39),              # Wp % s = 1, K2 = 20: two MMA steps
+    L("rag_s2_deep", 2, 20, 15, 15, 12, 5, 5, 2, 1, 40),        # Wp = 17 with stride 2, two k-blocks (the last one short)
+    L("stem_rag4", 1, 3, 23, 131, 20, 11, 11, 4, 0, 41),        # one-k-block kernel: strip segments, stride 4, tensor ends off a 16-byte boundary
+    L("stem_rag2", 2, 3, 21, 75, 24, 7, 7, 2, 0, 42),           # ... stride 2, odd strips
+    L("stem_rag3", 2, 5, 14, 100, 12, 4, 4, 3, 0, 43),          # ... stride 3, K2 = 20
+    L("stem_c8", 2, 8, 20, 40, 40, 5, 5, 1, 2, 44),             # ... K2 = 40, image segments
+    L("stem_imgs", 6, 3, 8, 8, 16, 3, 3, 1, 1, 45),             # ... a tile that touches three images
+    L("stem_wide", 2, 3, 12, 40, 300, 3, 3, 1, 1, 46),          # ... two channel tiles (filter streamed)
 ]
 
 
@@ -97,7 +106,7 @@ def test_transform_preserves_special_bit_patterns():
 
 
 @pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
-@pytest.mark.parametrize("precision", ["f32", "f16", "f16-shift", "f16-mat", "f16-gather"])
+@pytest.mark.parametrize("precision", ["f32", "f16", "f16-shift", "f16-mat", "f16-stem", "f16-gather"])
 def test_conv_parity_small(layer, precision):
     dims = layer.dims()
     x, f = workloads.make_inputs(layer)
@@ -108,7 +117,7 @@ def test_conv_parity_small(layer, precision):
 
 
 @pytest.mark.parametrize("layer", [SMALL[1], SMALL[2], SMALL[4], SMALL[8], SMALL[10], SMALL[12]], ids=lambda l: l.name)
-@pytest.mark.parametrize("precision", ["f32", "f16", "f16-shift", "f16-mat", "f16-gather"])
+@pytest.mark.parametrize("precision", ["f32", "f16", "f16-shift", "f16-mat", "f16-stem", "f16-gather"])
 def test_conv_exact_on_integer_inputs(layer, precision):
     """x in {-2..2}, filter in {-1,0,1}: every partial sum is a small integer, so any summation
     order gives the oracle's value exactly.  Separates indexing errors from rounding."""
@@ -225,6 +234,38 @@ def test_mat_kernel_with_and_without_cta_pairs(pair, monkeypatch):
         y, _, _ = gpu_conv(x, f, dims, "f16-mat")
         yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
         assert np.array_equal(y.astype(np.float64), yr), layer.name
+
+
+@pytest.mark.parametrize("tall", ["0", "1"])
+def test_shift_kernel_with_and_without_tall_tiles(tall, monkeypatch):
+    """The gathering shifted-view kernel with 128- and 256-position tiles, on layers whose stride
+    divides the strip width and on layers where it does not."""
+    monkeypatch.setenv("IM2WIN_F16_TALL", tall)
+    by_name = {l.name: l for l in SMALL}
+    for name in ("k11", "k5s2", "k147", "rag_s4", "rag_s3", "rag_s2_deep", "wide_row"):
+        layer = by_name[name]
+        dims = layer.dims()
+        x, f = workloads.make_small_integer_inputs(layer)
+        y, _, _ = gpu_conv(x, f, dims, "f16-shift")
+        yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+        assert np.array_equal(y.astype(np.float64), yr), name
+
+
+@pytest.mark.parametrize("generic", ["0", "1"])
+@pytest.mark.parametrize("ctas", ["1", "2"])
+def test_stem_kernel_variants(generic, ctas, monkeypatch):
+    """The one-k-block fp16 kernel with its unrolled (3 channels, Kh in 3/5/7/11) and its table-driven
+    re-layout, one and two CTAs per SM."""
+    monkeypatch.setenv("IM2WIN_F16_STEM_GENERIC", generic)
+    monkeypatch.setenv("IM2WIN_F16_STEM_CTAS", ctas)
+    by_name = {l.name: l for l in SMALL}
+    for name in ("cfg1", "stem_rag4", "stem_rag2", "stem_imgs", "stem_wide", "stem_c8"):
+        layer = by_name[name]
+        dims = layer.dims()
+        x, f = workloads.make_small_integer_inputs(layer)
+        y, _, _ = gpu_conv(x, f, dims, "f16-stem")
+        yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+        assert np.array_equal(y.astype(np.float64), yr), name
 
 
 @pytest.mark.parametrize("name", ["cfg2", "cfg4a", "cfg5k3"])
