@@ -28,8 +28,9 @@
 //
 // Virtual positions q = (n*Ho + ho)*Wq + kq with Wq = ceil(Wp/s); when s does not divide Wp the
 // last virtual column of a strip lacks some columns, which are staged as zeros and only feed
-// accumulator rows that are dropped.  Persistent CTAs, double-buffered accumulator in tensor
-// memory, bounded mbarrier waits.  Warp roles: 0-7 re-layout, 8 filter copies, 9 MMA issue (and
+// accumulator rows that are dropped.  Persistent CTAs; S stage i and accumulator i (two to four of
+// each, in tensor memory) belong together, so that one commit per tile tells the epilogue that the
+// accumulator is complete and the re-layout warps that the S stage is free; bounded mbarrier waits.  Warp roles: 0-7 re-layout, 8 filter copies, 9 MMA issue (and
 // tensor-memory allocation), 10 raw copies, 12-15 epilogue (11 idles).
 #include <cuda.h>
 #include <stdlib.h>
@@ -83,46 +84,37 @@ struct Segment {            // the part of a tile that is one contiguous run per
   int32_t dst;              // byte offset of the run's copy inside a channel region
 };
 
-// Splits the rows of the tile starting at virtual position q0 into contiguous runs.
-__device__ __forceinline__ int split_tile(const StemParams& q, int q0, Segment* segs) {
-  int remaining = q.rows, row0 = 0, g = 0;
-  if (q.ragged) {
-    int sg = q0 / q.Wq, kq = q0 - sg * q.Wq;     // strip (n*Ho + ho) and virtual column inside it
-    const int nstrips = q.N * q.Ho;
-    while (remaining > 0 && sg < nstrips && g < SEG_MAX) {
-      const int cnt = remaining < q.Wq - kq ? remaining : q.Wq - kq;
-      const int n = sg / q.Ho, ho = sg - n * q.Ho;
-      int cend = (kq + cnt) * q.s;
+// Splits the rows of the tile starting at virtual position q0 into contiguous runs: lane g of the
+// calling warp works out run g (no loop: the runs after the first start on strip / image
+// boundaries), writes it to segs[g] and the number of runs is returned to every lane.
+__device__ __forceinline__ int split_tile(const StemParams& q, int q0, Segment* segs, int lane) {
+  const int per = q.ragged ? q.Wq : q.Ho * q.Wq;       // rows of a whole strip / image
+  const int u0 = q0 / per, a0 = q0 - u0 * per;         // first strip / image and the row inside it
+  const int first_cnt = q.rows < per - a0 ? q.rows : per - a0;
+  const int unit = u0 + lane;
+  const int row0 = lane == 0 ? 0 : first_cnt + (lane - 1) * per;
+  const int a = lane == 0 ? a0 : 0;
+  int cnt = q.rows - row0;
+  if (cnt > per - a) cnt = per - a;
+  const bool valid = lane < SEG_MAX && row0 < q.rows && unit < (q.ragged ? q.N * q.Ho : q.N);
+  if (valid) {
+    Segment sg;
+    if (q.ragged) {
+      const int n = unit / q.Ho, ho = unit - n * q.Ho;
+      int cend = (a + cnt) * q.s;
       if (cend > q.Wp) cend = q.Wp;
-      segs[g].e0 = (int64_t)n * q.img_stride + (int64_t)ho * q.strip + (int64_t)kq * q.sKh;
-      segs[g].row0 = row0;
-      segs[g].cnt = cnt;
-      segs[g].elems = cend * q.Kh - kq * q.sKh;
-      segs[g].dst = ((row0 * q.sKh * 2) & ~15) + SEG_GAP * g;
-      row0 += cnt;
-      remaining -= cnt;
-      kq = 0;
-      ++sg;
-      ++g;
+      sg.e0 = (int64_t)n * q.img_stride + (int64_t)ho * q.strip + (int64_t)a * q.sKh;
+      sg.elems = cend * q.Kh - a * q.sKh;
+    } else {
+      sg.e0 = (int64_t)unit * q.img_stride + (int64_t)a * q.sKh;
+      sg.elems = cnt * q.sKh;
     }
-  } else {
-    const int img_rows = q.Ho * q.Wq;
-    int n = q0 / img_rows, a = q0 - n * img_rows;
-    while (remaining > 0 && n < q.N && g < SEG_MAX) {
-      const int cnt = remaining < img_rows - a ? remaining : img_rows - a;
-      segs[g].e0 = (int64_t)n * q.img_stride + (int64_t)a * q.sKh;
-      segs[g].row0 = row0;
-      segs[g].cnt = cnt;
-      segs[g].elems = cnt * q.sKh;
-      segs[g].dst = ((row0 * q.sKh * 2) & ~15) + SEG_GAP * g;
-      row0 += cnt;
-      remaining -= cnt;
-      a = 0;
-      ++n;
-      ++g;
-    }
+    sg.row0 = row0;
+    sg.cnt = cnt;
+    sg.dst = ((row0 * q.sKh * 2) & ~15) + SEG_GAP * lane;
+    segs[lane] = sg;
   }
-  return g;
+  return __popc(__ballot_sync(0xffffffffu, valid));
 }
 
 // One row of S for compile-time (C, Kh): returns the row's K2 halves packed into words.
@@ -150,7 +142,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-  __shared__ __align__(8) uint64_t bars[4 * MAX_STAGES + 2 * MAX_B + 4];
+  __shared__ __align__(8) uint64_t bars[5 * MAX_STAGES + 2 * MAX_B];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile uint32_t abort_flag;
   __shared__ Segment seg_ring[MAX_STAGES][SEG_MAX];      // the segments of the tile in each raw stage (written by the loader)
@@ -165,29 +157,25 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
   const uint32_t a_ring = b_ring + q.sb * q.b_stage_bytes;
   const uint32_t raw_ring = a_ring + q.sa * q.a_stage_bytes;
   const uint32_t a_full0 = smem_u32(&bars[0]);
-  const uint32_t a_empty0 = smem_u32(&bars[MAX_STAGES]);
+  const uint32_t acc_empty0 = smem_u32(&bars[MAX_STAGES]);
   const uint32_t r_full0 = smem_u32(&bars[2 * MAX_STAGES]);
   const uint32_t r_empty0 = smem_u32(&bars[3 * MAX_STAGES]);
   const uint32_t b_full0 = smem_u32(&bars[4 * MAX_STAGES]);
   const uint32_t b_empty0 = smem_u32(&bars[4 * MAX_STAGES + MAX_B]);
-  const uint32_t acc_full0 = smem_u32(&bars[4 * MAX_STAGES + 2 * MAX_B]);
-  const uint32_t acc_empty0 = smem_u32(&bars[4 * MAX_STAGES + 2 * MAX_B + 2]);
+  const uint32_t acc_full0 = smem_u32(&bars[4 * MAX_STAGES + 2 * MAX_B]);   // MAX_STAGES of them
 
   if (threadIdx.x == 0) {
     abort_flag = 0u;
     for (int i = 0; i < MAX_STAGES; ++i) {
       mbar_init(a_full0 + 8 * i, REPACK_WARPS);
-      mbar_init(a_empty0 + 8 * i, 1);
+      mbar_init(acc_empty0 + 8 * i, 4);      // the four epilogue warps
+      mbar_init(acc_full0 + 8 * i, 1);
       mbar_init(r_full0 + 8 * i, 1);
       mbar_init(r_empty0 + 8 * i, REPACK_WARPS);
     }
     for (int i = 0; i < MAX_B; ++i) {
       mbar_init(b_full0 + 8 * i, 1);
       mbar_init(b_empty0 + 8 * i, 1);
-    }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(acc_full0 + 8 * i, 1);
-      mbar_init(acc_empty0 + 8 * i, 4);      // the four epilogue warps
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -221,7 +209,8 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
       if (lane == 0) {
         ok = mbar_wait(r_full0 + 8 * rst, rph, &abort_flag, q.status);
         if (threadIdx.x == 0) TIMER_LAP(1);     // wait for the raw stage
-        if (ok) ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+        // S stage st is free once the MMAs of the tile that used it last are complete
+        if (ok) ok = mbar_wait(acc_full0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
         if (threadIdx.x == 0) TIMER_LAP(2);     // wait for a free S stage
       }
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -329,15 +318,15 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
     bool ok = true;
     int sta = 0, stb = 0;
     uint32_t pha = 0, phb = 0;
-    uint32_t it = 0;                             // work items done by this CTA: accumulator buffer = it & 1
+    uint32_t it = 0;                             // work items done by this CTA
     const uint32_t a_lo0 = smem_desc_lo_noswz(a_ring, (uint32_t)q.R * 16u), b_lo0 = smem_desc_lo(b_ring);
     const uint32_t sub_units = (uint32_t)(q.chunks * q.R);   // 16-byte units per sub-tile
     const uint32_t kstep_units = 2u * (uint32_t)q.R;         // 16-byte units per 16-element k step
     TIMER_DECL;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
-      const uint32_t buf = it & 1u;
+      const uint32_t buf = (uint32_t)sta;       // accumulator i goes with S stage i
       TIMER_LAP(11);
-      ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
+      ok = mbar_wait(acc_empty0 + 8 * buf, pha ^ 1u, &abort_flag, q.status);   // drained by the epilogue
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       TIMER_LAP(9);                              // MMA warp: wait for a free accumulator
@@ -348,34 +337,64 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
       tc_fence_after();
       const uint32_t acc = tmem_acc + buf * (uint32_t)q.bnr;
       const uint32_t a_lo_stage = a_lo0 + (uint32_t)(sta * (q.a_stage_bytes >> 4));
-      uint32_t sub = 0, shift = 0, first = 0;   // kernel column v reads sub-tile v mod s from row v div s on
-      for (int v = 0; v < q.Kw; ++v) {
-        if (!(q.resident && it > 0)) {          // a resident filter is complete after the first work item
-          ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
-          ok = __all_sync(0xffffffffu, ok);
+      // kernel column v reads sub-tile v mod s from row v div s on.  A single thread issuing branchy
+      // code takes hundreds of cycles per kernel column, so the loops below are kept straight-line.
+      if (q.resident) {
+        if (it == 0) {                          // the resident filter is complete after the first wait
+          for (int v = 0; v < q.Kw && ok; ++v) {
+            ok = mbar_wait(b_full0 + 8 * v, 0u, &abort_flag, q.status);
+            ok = __all_sync(0xffffffffu, ok);
+          }
           if (!ok) break;
           tc_fence_after();
         }
         if (leader) {
-          const uint32_t a_lo = a_lo_stage + sub * sub_units + shift;
-          const uint32_t b_lo = b_lo0 + (uint32_t)(stb * (q.b_stage_bytes >> 4));
+          uint32_t a_v = a_lo_stage, b_v = b_lo0, sub = 0, accf = 0;
+          const uint32_t b_step = (uint32_t)(q.b_stage_bytes >> 4);
+          const uint32_t wrap_step = 1u - (uint32_t)(q.s - 1) * sub_units;   // back to sub-tile 0, one row further
+          const uint32_t last_sub = (uint32_t)q.s - 1u;
 #pragma unroll 1
-          for (int j = 0; j < q.nks; ++j)
-            umma_f16_ab(acc, a_lo + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j, kSmemDescHiSw128,
-                        q.idesc, first | (uint32_t)j);
-          first = 1u;
-          if (!q.resident) umma_commit(b_empty0 + 8 * stb);
+          for (int v = 0; v < q.Kw; ++v) {
+#pragma unroll
+            for (int j = 0; j < KB / 16; ++j)
+              if (j < q.nks)
+                umma_f16_ab(acc, a_v + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_v + 2 * j, kSmemDescHiSw128,
+                            q.idesc, accf | (uint32_t)j);
+            accf = 1u;
+            b_v += b_step;
+            const bool wrap = sub == last_sub;
+            a_v += wrap ? wrap_step : sub_units;
+            sub = wrap ? 0u : sub + 1u;
+          }
+          umma_commit(acc_full0 + 8 * buf);     // accumulator complete = S stage free
         }
         __syncwarp();
-        if (++sub == (uint32_t)q.s) { sub = 0; ++shift; }
-        if (++stb == q.sb) { stb = 0; phb ^= 1u; }
+      } else {
+        uint32_t sub = 0, shift = 0, first = 0;
+        for (int v = 0; v < q.Kw; ++v) {
+          ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          if (leader) {
+            const uint32_t a_lo = a_lo_stage + sub * sub_units + shift;
+            const uint32_t b_lo = b_lo0 + (uint32_t)(stb * (q.b_stage_bytes >> 4));
+#pragma unroll
+            for (int j = 0; j < KB / 16; ++j)
+              if (j < q.nks)
+                umma_f16_ab(acc, a_lo + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j, kSmemDescHiSw128,
+                            q.idesc, first | (uint32_t)j);
+            first = 1u;
+            umma_commit(b_empty0 + 8 * stb);
+          }
+          __syncwarp();
+          if (++sub == (uint32_t)q.s) { sub = 0; ++shift; }
+          if (++stb == q.sb) { stb = 0; phb ^= 1u; }
+        }
+        if (!ok) break;
+        if (leader) umma_commit(acc_full0 + 8 * buf);       // accumulator complete = S stage free
+        __syncwarp();
       }
-      if (!ok) break;
-      if (leader) {
-        umma_commit(a_empty0 + 8 * sta);
-        umma_commit(acc_full0 + 8 * buf);
-      }
-      __syncwarp();
       if (++sta == q.sa) { sta = 0; pha ^= 1u; }
     }
     if (leader) { TIMER_LAP(11); TIMER_FLUSH(); }   // MMA warp: filter waits, issue, commits
@@ -395,12 +414,9 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
       if (lane == 0) TIMER_LAP(5);               // raw loader: wait for a free raw stage
       // the tile's segments go with the raw stage: the re-layout warps read them once the stage is full
       Segment* segs = seg_ring[rst];
-      int nseg = 0;
-      if (lane == 0) {
-        nseg = split_tile(q, q0, segs);
-        nseg_ring[rst] = nseg;
-      }
-      nseg = __shfl_sync(0xffffffffu, nseg, 0);
+      const int nseg = split_tile(q, q0, segs, lane);
+      if (lane == 0) nseg_ring[rst] = nseg;
+      __syncwarp();
       const uint32_t bar = r_full0 + 8 * rst;
       const uint32_t stage = raw_ring + rst * q.raw_stage_bytes;
       const int ncopy = nseg * q.C;
@@ -439,8 +455,8 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
     bool ok = true;
     uint32_t it = 0;
     TIMER_DECL;
+    uint32_t buf = 0, eph = 0;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
-      const uint32_t buf = it & 1u;
       const int q0 = (w % q.ntm) * TILE_M;
       const int n0 = (w / q.ntm) * q.bn;
       const int vq = q0 + lq * 32 + lane;        // accumulator row = virtual position
@@ -454,7 +470,7 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
         valid = kq < q.Wo;                       // trailing columns of a strip are no output
         yrow += ((int64_t)n * q.Co + n0) * q.HoWo + ho * q.Wo + kq;
       }
-      if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
+      if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, eph, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
       if (!ok) break;
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(7);   // epilogue: address arithmetic, wait for the accumulator
@@ -475,6 +491,7 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty0 + 8 * buf);
+      if (++buf == (uint32_t)q.sa) { buf = 0; eph ^= 1u; }
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(8);   // epilogue: tensor memory -> global
     }
     if (threadIdx.x == WARP_EPI0 * 32) TIMER_FLUSH();
@@ -540,9 +557,11 @@ StemPlan plan_f16_stem(const Geometry& g) {
   p.b_stage_bytes = p.bn * KB * 2;
   const int nct = (g.Co + p.bn - 1) / p.bn;
   if ((p.VQ + TILE_M - 1) / TILE_M * nct >= ((int64_t)1 << 31)) return p;
-  // rings: S 2, raw 2 (3 if room), filter resident if one channel tile and Kw tiles fit, else 2..4
+  // rings: S stages (= accumulators) 2, raw 2, filter resident if one channel tile and its Kw tiles
+  // fit, else 2..4 stages; then what is left goes to a third raw stage and to more S stages
   const int budget = kSmemMax - 1024 - kStaticSmem;
   const int base = 2 * p.a_stage_bytes + 2 * p.raw_stage_bytes;
+  const int bnr = (p.bn + 31) / 32 * 32;
   p.sa = 2;
   p.rs = 2;
   p.resident = 0;
@@ -554,7 +573,14 @@ StemPlan plan_f16_stem(const Geometry& g) {
     while (p.sb > 2 && base + p.sb * p.b_stage_bytes > budget) --p.sb;
     if (base + p.sb * p.b_stage_bytes > budget) return p;
   }
-  if (base + p.raw_stage_bytes + p.sb * p.b_stage_bytes <= budget) p.rs = 3;
+  int used = base + p.sb * p.b_stage_bytes;
+  if (used + p.raw_stage_bytes <= budget) { p.rs = 3; used += p.raw_stage_bytes; }
+  while (p.sa < MAX_STAGES && (p.sa + 1) * bnr <= 512 && used + p.a_stage_bytes <= budget) {
+    ++p.sa;
+    used += p.a_stage_bytes;
+  }
+  const char* force_sa = getenv("IM2WIN_F16_STEM_STAGES");   // testing aid: S stages / accumulators (2..4)
+  if (force_sa && atoi(force_sa) >= 2 && atoi(force_sa) < p.sa) p.sa = atoi(force_sa);
   p.smem_bytes = p.sa * p.a_stage_bytes + p.rs * p.raw_stage_bytes + p.sb * p.b_stage_bytes + 1024;
   p.eligible = true;
   return p;
@@ -592,7 +618,7 @@ cudaError_t launch_conv_f16_stem(const uint16_t* window, float* y, void* scratch
   q.a_stage_bytes = plan.a_stage_bytes; q.b_stage_bytes = plan.b_stage_bytes;
   q.bn = plan.bn; q.bnr = (plan.bn + 31) / 32 * 32;
   q.tmem_cols = 32;
-  while (q.tmem_cols < 2 * q.bnr) q.tmem_cols *= 2;
+  while (q.tmem_cols < plan.sa * q.bnr) q.tmem_cols *= 2;
   q.idesc = instr_desc_f16(TILE_M, plan.bn);
   q.rs = plan.rs; q.sa = plan.sa; q.sb = plan.sb; q.resident = plan.resident;
   const int64_t ntm = (plan.VQ + TILE_M - 1) / TILE_M;
