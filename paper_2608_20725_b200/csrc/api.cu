@@ -96,9 +96,9 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
     const MatcPlan matc = mat.eligible ? MatcPlan{} : plan_f16_matc(g);
     const char* force = getenv("IM2WIN_F16_KERNEL");
     // measured: the matrix-transpose kernels win for strided layers (the others stage such layers
-    // with 2-byte gathers) and, in their CTA-pair form, for kernels up to 5 wide with more than 128
-    // output channels; IM2WIN_F16_KERNEL=mat forces them wherever they can run (a testing aid)
-    const bool want = force ? strcmp(force, "mat") == 0 : (g.s > 1 || (g.Co > 128 && g.Kw <= 5));
+    // with 2-byte gathers) and for kernels up to 5 wide with 128 output channels or more (CTA pairs
+    // above 128); IM2WIN_F16_KERNEL=mat forces them wherever they can run (a testing aid)
+    const bool want = force ? strcmp(force, "mat") == 0 : (g.s > 1 || (g.Co >= 128 && g.Kw <= 5));
     // (the scratch size covers every layout, whichever kernel is picked or forced)
     const bool use_mat = want && !l->f16_stem;
     if (mat.eligible) {

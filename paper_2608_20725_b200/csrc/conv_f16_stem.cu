@@ -50,7 +50,8 @@ constexpr int REPACK_THREADS = REPACK_WARPS * 32;
 constexpr int WARP_TMA = 8, WARP_MMA = 9, WARP_RAW = 10, WARP_EPI0 = 12;
 constexpr int NUM_WARPS = 16;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
-constexpr int MAX_STAGES = 4;                        // S and raw rings
+constexpr int MAX_STAGES = 4;                        // S stages / accumulators
+constexpr int MAX_RAW = 8;                           // raw stages (small copies are latency bound: many in flight)
 constexpr int MAX_B = 16;                            // filter stages (a resident filter needs Kw of them)
 constexpr int SEG_MAX = 6;                           // strip segments (or images) one tile may touch
 constexpr int SEG_GAP = 48;                          // bytes between the copies of consecutive segments
@@ -142,11 +143,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-  __shared__ __align__(8) uint64_t bars[5 * MAX_STAGES + 2 * MAX_B];
+  __shared__ __align__(8) uint64_t bars[3 * MAX_STAGES + 2 * MAX_RAW + 2 * MAX_B];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile uint32_t abort_flag;
-  __shared__ Segment seg_ring[MAX_STAGES][SEG_MAX];      // the segments of the tile in each raw stage (written by the loader)
-  __shared__ int32_t nseg_ring[MAX_STAGES];
+  __shared__ Segment seg_ring[MAX_RAW][SEG_MAX];      // the segments of the tile in each raw stage (written by the loader)
+  __shared__ int32_t nseg_ring[MAX_RAW];
   __shared__ __align__(16) uint32_t tab_s[KB];           // k2 -> channel region + 2*u | (c*chan_stride mod 8) << 24
   __shared__ __align__(16) uint32_t zero_s[4];           // what padded k2 read
 
@@ -158,11 +159,11 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
   const uint32_t raw_ring = a_ring + q.sa * q.a_stage_bytes;
   const uint32_t a_full0 = smem_u32(&bars[0]);
   const uint32_t acc_empty0 = smem_u32(&bars[MAX_STAGES]);
-  const uint32_t r_full0 = smem_u32(&bars[2 * MAX_STAGES]);
-  const uint32_t r_empty0 = smem_u32(&bars[3 * MAX_STAGES]);
-  const uint32_t b_full0 = smem_u32(&bars[4 * MAX_STAGES]);
-  const uint32_t b_empty0 = smem_u32(&bars[4 * MAX_STAGES + MAX_B]);
-  const uint32_t acc_full0 = smem_u32(&bars[4 * MAX_STAGES + 2 * MAX_B]);   // MAX_STAGES of them
+  const uint32_t acc_full0 = smem_u32(&bars[2 * MAX_STAGES]);
+  const uint32_t r_full0 = smem_u32(&bars[3 * MAX_STAGES]);
+  const uint32_t r_empty0 = smem_u32(&bars[3 * MAX_STAGES + MAX_RAW]);
+  const uint32_t b_full0 = smem_u32(&bars[3 * MAX_STAGES + 2 * MAX_RAW]);
+  const uint32_t b_empty0 = smem_u32(&bars[3 * MAX_STAGES + 2 * MAX_RAW + MAX_B]);
 
   if (threadIdx.x == 0) {
     abort_flag = 0u;
@@ -170,6 +171,8 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
       mbar_init(a_full0 + 8 * i, REPACK_WARPS);
       mbar_init(acc_empty0 + 8 * i, 4);      // the four epilogue warps
       mbar_init(acc_full0 + 8 * i, 1);
+    }
+    for (int i = 0; i < MAX_RAW; ++i) {
       mbar_init(r_full0 + 8 * i, 1);
       mbar_init(r_empty0 + 8 * i, REPACK_WARPS);
     }
@@ -579,6 +582,16 @@ StemPlan plan_f16_stem(const Geometry& g) {
     ++p.sa;
     used += p.a_stage_bytes;
   }
+  // three raw stages by default (measured: eight in flight slow a 3-channel 3x3 layer down from 1.01 ms
+  // to 1.27 ms, as a second CTA per SM does); IM2WIN_F16_STEM_RAW = 2..8 sets another depth (a testing aid)
+  const char* force_rs = getenv("IM2WIN_F16_STEM_RAW");
+  const int rs_max = force_rs && atoi(force_rs) >= 2 && atoi(force_rs) <= MAX_RAW ? atoi(force_rs) : 3;
+  if (rs_max < p.rs) { used -= (p.rs - rs_max) * p.raw_stage_bytes; p.rs = rs_max; }
+  while (p.rs < rs_max && (p.rs + 1) * p.raw_stage_bytes <= 48 * 1024 && used + p.raw_stage_bytes <= budget) {
+    ++p.rs;
+    used += p.raw_stage_bytes;
+  }
+
   const char* force_sa = getenv("IM2WIN_F16_STEM_STAGES");   // testing aid: S stages / accumulators (2..4)
   if (force_sa && atoi(force_sa) >= 2 && atoi(force_sa) < p.sa) p.sa = atoi(force_sa);
   p.smem_bytes = p.sa * p.a_stage_bytes + p.rs * p.raw_stage_bytes + p.sb * p.b_stage_bytes + 1024;
