@@ -306,6 +306,39 @@ def test_full_size_wide_kernels_sampled(name):
         del y
 
 
+# ------------------------------------------------- the paper's Table 1 layers ----
+TABLE1 = [workloads.TABLE1_LAYERS[k].with_batch(n) for k, n in
+          (("cv1", 16), ("cv2", 8), ("cv3", 16), ("cv4", 6), ("cv5", 32), ("cv7", 12), ("cv8", 12), ("cv9", 32),
+           ("cv12", 64))] + [workloads.TABLE1_LAYERS["cv1"], workloads.TABLE1_LAYERS["cv6"]]   # two at the paper's batch of 256
+
+
+@pytest.mark.parametrize("layer", TABLE1, ids=lambda l: f"{l.name}-n{l.N}")
+def test_table1_layers_sampled_outputs(layer):
+    """The paper's benchmark layers (Table 1: no padding, strides 1, 2 and 4, 3 to 512 channels) with
+    their per-image geometry and a batch that still gives several waves of tiles: transform bit for
+    bit on the first and last image, convolution on sampled outputs and on the whole last image."""
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    ho, wo = oracle.out_dims(dims)
+    total = layer.N * layer.Co * ho * wo
+    rng = np.random.default_rng(layer.seed + 3)
+    idx = np.concatenate([rng.integers(0, total, 2048), [0, total - 1, wo - 1, ho * wo - 1, total - ho * wo]])
+    for precision in layer.precisions:
+        tdt = torch.float32 if precision == "f32" else torch.float16
+        raw = x.to(tdt).view(torch.int32 if precision == "f32" else torch.int16)
+        got = gpu_transform(raw, dims)
+        for n in (0, layer.N - 1):
+            want = oracle.transform(raw[n:n + 1].numpy(), dict(dims, N=1))
+            assert np.array_equal(got[n:n + 1], want), (layer.name, precision, n)
+        del got
+        y, _, _ = gpu_conv(x, f, dims, precision)
+        xo, fo = oracle_inputs(x, f, precision)
+        yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
+        check_conv(y.reshape(-1)[idx], yr, ar, precision, layer.name)
+        yi, ai = oracle.conv_im2win(xo[-1:], fo, dict(dims, N=1))
+        check_conv(y[-1:], yi, ai, precision, layer.name + " last image")
+
+
 # ------------------------------------------------------------ full-size layers ----
 FULL = [workloads.LAYERS[k] for k in ("cfg2", "cfg3", "cfg4a", "cfg4b", "cfg4c", "cfg5k1", "cfg5k3", "cfg5k5")]
 
