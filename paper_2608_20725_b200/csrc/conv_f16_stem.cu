@@ -30,8 +30,8 @@
 // last virtual column of a strip lacks some columns, which are staged as zeros and only feed
 // accumulator rows that are dropped.  Persistent CTAs; S stage i and accumulator i (two to four of
 // each, in tensor memory) belong together, so that one commit per tile tells the epilogue that the
-// accumulator is complete and the re-layout warps that the S stage is free; bounded mbarrier waits.  Warp roles: 0-7 re-layout, 8 filter copies, 9 MMA issue (and
-// tensor-memory allocation), 10 raw copies, 12-15 epilogue (11 idles; a second epilogue warp per lane
+// accumulator is complete and the re-layout warps that the S stage is free; bounded mbarrier waits.  Warp roles: 0-7 and 11 re-layout, 8 filter copies, 9 MMA issue (and
+// tensor-memory allocation), 10 raw copies, 12-15 epilogue (a second epilogue warp per lane
 // quadrant was measured: 5 % faster on a 3-channel 3x3 layer, 5-8 % slower on the 7x7 and 11x11 stems).
 #include <cuda.h>
 #include <stdlib.h>
@@ -46,9 +46,9 @@ using namespace ptx;
 
 constexpr int TILE_M = 128;
 constexpr int KB = kF16KBlock;
-constexpr int REPACK_WARPS = 8;
+constexpr int REPACK_WARPS = 9;                      // warps 0-7 and warp 11
 constexpr int REPACK_THREADS = REPACK_WARPS * 32;
-constexpr int WARP_TMA = 8, WARP_MMA = 9, WARP_RAW = 10, WARP_EPI0 = 12;
+constexpr int WARP_TMA = 8, WARP_MMA = 9, WARP_RAW = 10, WARP_REPACK9 = 11, WARP_EPI0 = 12;
 constexpr int NUM_WARPS = 16;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr int MAX_STAGES = 4;                        // S stages / accumulators
@@ -167,8 +167,8 @@ __device__ __forceinline__ void load_row(uint32_t src, uint32_t phase0, uint32_t
   }
 }
 
-// C_ = KH_ = 0: any (C, Kh) with C*Kh <= 64, table-driven re-layout.
-template <int C_, int KH_>
+// C_ = KH_ = KW_ = 0: any (C, Kh, Kw) with C*Kh <= 64: table-driven re-layout, looped MMA issue.
+template <int C_, int KH_, int KW_>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
   extern __shared__ unsigned char smem_dyn[];
@@ -228,7 +228,7 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
   tc_fence_after();
   const uint32_t tmem_acc = tmem_base_slot;
 
-  if (warp < REPACK_WARPS) {
+  if (warp < 8 || warp == WARP_REPACK9) {
     // ---------------- re-layout: raw stage -> S stage ---------------------------
     const uint32_t zero_addr = smem_u32(zero_s);
     const uint32_t r16 = (uint32_t)q.R * 16u;
@@ -237,6 +237,9 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
     int st = 0, rst = 0;
     uint32_t ph = 0, rph = 0;
     const int n_ri = q.s * q.rows;
+    // nine warps: 288 threads take the 262 rows of a 7x7 stride-2 tile in one pass and the 520 rows of
+    // an 11x11 stride-4 tile in two (eight warps need two and three)
+    const int rt = warp < 8 ? (int)threadIdx.x : 256 + lane;
     TIMER_DECL;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
       if (lane == 0) {
@@ -252,7 +255,7 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
       const int nseg = nseg_ring[rst];
       const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
       const uint32_t raw_stage = raw_ring + rst * q.raw_stage_bytes;
-      for (int ri = threadIdx.x; ri < n_ri; ri += REPACK_THREADS) {
+      for (int ri = rt; ri < n_ri; ri += REPACK_THREADS) {
         int sub = 0, i = ri;
         while (i >= q.rows) { i -= q.rows; ++sub; }
         // the segment of row i, the row's record inside the segment's run, the run's phase
@@ -355,6 +358,21 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
     const uint32_t a_lo0 = smem_desc_lo_noswz(a_ring, (uint32_t)q.R * 16u), b_lo0 = smem_desc_lo(b_ring);
     const uint32_t sub_units = (uint32_t)(q.chunks * q.R);   // 16-byte units per sub-tile
     const uint32_t kstep_units = 2u * (uint32_t)q.R;         // 16-byte units per 16-element k step
+    // compile-time kernel width: the issue loops unroll completely and every operand address is a
+    // stage base plus a value worked out here, once (back-to-back MMAs of N = 64 need 48 cycles each,
+    // a looped issue sequence spends twice that per MMA on its own address arithmetic)
+    constexpr int KWU = KW_ > 0 ? KW_ : 1;
+    constexpr int NKS = KW_ > 0 ? (C_ * KH_ + 15) / 16 : 1;
+    uint32_t aoff[KWU];
+    if constexpr (KW_ > 0) {
+      uint32_t sub = 0, shift = 0;
+#pragma unroll
+      for (int v = 0; v < KW_; ++v) {
+        aoff[v] = sub * sub_units + shift;
+        if (++sub == (uint32_t)q.s) { sub = 0; ++shift; }
+      }
+    }
+    const uint32_t b_step = (uint32_t)(q.b_stage_bytes >> 4);
     TIMER_DECL;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
       const uint32_t buf = (uint32_t)sta;       // accumulator i goes with S stage i
@@ -381,9 +399,18 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
           if (!ok) break;
           tc_fence_after();
         }
-        if (leader) {
+        if constexpr (KW_ > 0) {
+          if (leader) {
+#pragma unroll
+            for (int v = 0; v < KW_; ++v)
+#pragma unroll
+              for (int j = 0; j < NKS; ++j)
+                umma_f16_ab(acc, a_lo_stage + aoff[v] + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128,
+                            b_lo0 + (uint32_t)v * b_step + 2 * j, kSmemDescHiSw128, q.idesc, (v | j) ? 1u : 0u);
+            umma_commit(acc_full0 + 8 * buf);   // accumulator complete = S stage free
+          }
+        } else if (leader) {
           uint32_t a_v = a_lo_stage, b_v = b_lo0, sub = 0, accf = 0;
-          const uint32_t b_step = (uint32_t)(q.b_stage_bytes >> 4);
           const uint32_t wrap_step = 1u - (uint32_t)(q.s - 1) * sub_units;   // back to sub-tile 0, one row further
           const uint32_t last_sub = (uint32_t)q.s - 1u;
 #pragma unroll 1
@@ -401,6 +428,27 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
           }
           umma_commit(acc_full0 + 8 * buf);     // accumulator complete = S stage free
         }
+        __syncwarp();
+      } else if constexpr (KW_ > 0) {
+#pragma unroll
+        for (int v = 0; v < KW_; ++v) {
+          ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          if (leader) {
+            const uint32_t b_lo = b_lo0 + (uint32_t)stb * b_step;
+#pragma unroll
+            for (int j = 0; j < NKS; ++j)
+              umma_f16_ab(acc, a_lo_stage + aoff[v] + (uint32_t)j * kstep_units, kSmemDescHiNoSwz128, b_lo + 2 * j,
+                          kSmemDescHiSw128, q.idesc, (v | j) ? 1u : 0u);
+            umma_commit(b_empty0 + 8 * stb);
+          }
+          __syncwarp();
+          if (++stb == q.sb) { stb = 0; phb ^= 1u; }
+        }
+        if (!ok) break;
+        if (leader) umma_commit(acc_full0 + 8 * buf);       // accumulator complete = S stage free
         __syncwarp();
       } else {
         uint32_t sub = 0, shift = 0, first = 0;
@@ -688,13 +736,15 @@ cudaError_t launch_conv_f16_stem(const uint16_t* window, float* y, void* scratch
   q.cbits = 0;
   while ((1 << q.cbits) < g.C) ++q.cbits;
 
-  void (*kernel)(const CUtensorMap, StemParams) = conv_f16_stem_kernel<0, 0>;
-  if (g.C == 3 && g.Kh == 3) kernel = conv_f16_stem_kernel<3, 3>;
-  else if (g.C == 3 && g.Kh == 5) kernel = conv_f16_stem_kernel<3, 5>;
-  else if (g.C == 3 && g.Kh == 7) kernel = conv_f16_stem_kernel<3, 7>;
-  else if (g.C == 3 && g.Kh == 11) kernel = conv_f16_stem_kernel<3, 11>;
+  void (*kernel)(const CUtensorMap, StemParams) = conv_f16_stem_kernel<0, 0, 0>;
+  if (g.C == 3 && g.Kh == g.Kw) {                 // the common stems: square kernels on 3 channels
+    if (g.Kh == 3) kernel = conv_f16_stem_kernel<3, 3, 3>;
+    else if (g.Kh == 5) kernel = conv_f16_stem_kernel<3, 5, 5>;
+    else if (g.Kh == 7) kernel = conv_f16_stem_kernel<3, 7, 7>;
+    else if (g.Kh == 11) kernel = conv_f16_stem_kernel<3, 11, 11>;
+  }
   const char* generic = getenv("IM2WIN_F16_STEM_GENERIC");   // testing aid: the table-driven re-layout everywhere
-  if (generic && atoi(generic)) kernel = conv_f16_stem_kernel<0, 0>;
+  if (generic && atoi(generic)) kernel = conv_f16_stem_kernel<0, 0, 0>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
   if (e != cudaSuccess) return e;
   // persistent CTAs: one per SM (measured: a second CTA per SM, where it fits, only slows the layer
