@@ -88,7 +88,7 @@ MatcPlan plan_f16_matc(const Geometry& g);
 struct StemPlan {
   bool eligible;
   int32_t Wq, ragged, rows, R, nks, chan_region, raw_stage_bytes, a_stage_bytes, b_stage_bytes, bn;
-  int32_t sa, rs, sb, resident, smem_bytes;
+  int32_t sa, rs, sb, resident, smem_bytes, epi_bufs;
   int64_t VQ;
 };
 StemPlan plan_f16_stem(const Geometry& g);

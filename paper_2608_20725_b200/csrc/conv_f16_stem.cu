@@ -56,6 +56,8 @@ constexpr int MAX_RAW = 8;                           // raw stages (small copies
 constexpr int MAX_B = 16;                            // filter stages (a resident filter needs Kw of them)
 constexpr int SEG_MAX = 6;                           // strip segments (or images) one tile may touch
 constexpr int SEG_GAP = 48;                          // bytes between the copies of consecutive segments
+constexpr int EPI_PITCH = 136;                       // floats per output plane in an epilogue staging buffer
+constexpr int EPI_BUF_BYTES = 32 * EPI_PITCH * 4;    // 32 planes x (128 positions + alignment slack)
 
 struct StemParams {
   const uint16_t* __restrict__ win;
@@ -78,6 +80,7 @@ struct StemParams {
   int32_t rs, sa, sb, resident;
   int32_t ntm, nwork;
   int32_t cbits;            // bits of a channel index: ceil(log2 C)
+  int32_t epi_bufs;         // staging buffers of the aligned-store epilogue (0: stores straight from registers)
 };
 
 struct Segment {            // the part of a tile that is one contiguous run per channel
@@ -168,7 +171,8 @@ __device__ __forceinline__ void load_row(uint32_t src, uint32_t phase0, uint32_t
 }
 
 // C_ = KH_ = KW_ = 0: any (C, Kh, Kw) with C*Kh <= 64: table-driven re-layout, looped MMA issue.
-template <int C_, int KH_, int KW_>
+// STAGED: the epilogue that writes aligned runs through a staging buffer (opt-in, see plan_f16_stem).
+template <int C_, int KH_, int KW_, bool STAGED>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
   extern __shared__ unsigned char smem_dyn[];
@@ -187,6 +191,7 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
   const uint32_t b_ring = smem_u32(smem);
   const uint32_t a_ring = b_ring + q.sb * q.b_stage_bytes;
   const uint32_t raw_ring = a_ring + q.sa * q.a_stage_bytes;
+  const uint32_t epi_ring = raw_ring + q.rs * q.raw_stage_bytes;
   const uint32_t a_full0 = smem_u32(&bars[0]);
   const uint32_t acc_empty0 = smem_u32(&bars[MAX_STAGES]);
   const uint32_t acc_full0 = smem_u32(&bars[2 * MAX_STAGES]);
@@ -554,37 +559,150 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
     bool ok = true;
     uint32_t it = 0;
     TIMER_DECL;
-    uint32_t buf = 0, eph = 0;
+    uint32_t buf = 0, eph = 0, chunk_ctr = 0;
+    // Meeting point of the four epilogue warps: hardware barrier 1.  It has no time-out, so the warps
+    // first agree (through the same barrier, which every warp reaches because the wait before it is
+    // bounded) whether all of them got their accumulator; from there on they take the same path.
+    auto epi_sync = [&]() { asm volatile("bar.sync 1, 128;" ::: "memory"); };
+    // ragged run ends: lane -> (plane lane/6, end element lane%6) in two passes of 32
+    const int bi0 = lane / 6, bt0 = lane - 6 * bi0, bi1 = (lane + 32) / 6, bt1 = lane + 32 - 6 * bi1;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x, ++it) {
       const int q0 = (w % q.ntm) * TILE_M;
       const int n0 = (w / q.ntm) * q.bn;
       const int vq = q0 + lq * 32 + lane;        // accumulator row = virtual position
       bool valid = false;
       float* yrow = q.y;
+      int o = 0;                                 // index of the row's output inside its plane
       if (vq < q.VQ) {
         const int sg = vq / q.Wq;
         const int kq = vq - sg * q.Wq;
         const int n = sg / q.Ho;
         const int ho = sg - n * q.Ho;
         valid = kq < q.Wo;                       // trailing columns of a strip are no output
-        yrow += ((int64_t)n * q.Co + n0) * q.HoWo + ho * q.Wo + kq;
+        o = ho * q.Wo + kq;
+        yrow += ((int64_t)n * q.Co + n0) * q.HoWo + o;
+      }
+      // The tile's outputs: first and last valid position (the same for every thread).  When both lie
+      // in one image the outputs are ONE contiguous run of each output plane, [o0, o0 + nv).
+      bool staged = false;
+      int o0 = 0, nv = 0;
+      int64_t plane0 = 0;
+      if constexpr (STAGED) {
+        const int sgF0 = q0 / q.Wq, kqF0 = q0 - sgF0 * q.Wq;
+        const int sgF = kqF0 < q.Wo ? sgF0 : sgF0 + 1;         // a tile that starts on a dropped column
+        const int kqF = kqF0 < q.Wo ? kqF0 : 0;
+        const int nF = sgF / q.Ho, hoF = sgF - nF * q.Ho;
+        const int vqL = q0 + TILE_M - 1 < q.VQ - 1 ? q0 + TILE_M - 1 : q.VQ - 1;
+        const int sgL = vqL / q.Wq, kqL0 = vqL - sgL * q.Wq;
+        const int kqL = kqL0 < q.Wo ? kqL0 : q.Wo - 1;
+        const int nL = sgL / q.Ho, hoL = sgL - nL * q.Ho;
+        o0 = hoF * q.Wo + kqF;
+        nv = hoL * q.Wo + kqL - o0 + 1;
+        staged = nF == nL && nF < q.N && nv > 0;
+        plane0 = ((int64_t)nF * q.Co + n0) * q.HoWo;
       }
       if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, eph, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      if constexpr (STAGED) {
+        uint32_t all_ok;
+        asm volatile(
+            "{\n\t.reg .pred p, pq;\n\t"
+            "setp.ne.b32 pq, %1, 0;\n\t"
+            "bar.red.and.pred p, 1, 128, pq;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(all_ok)
+            : "r"((uint32_t)ok)
+            : "memory");
+        ok = all_ok != 0;
+      }
       if (!ok) break;
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(7);   // epilogue: address arithmetic, wait for the accumulator
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)q.bnr + ((uint32_t)(lq * 32) << 16);
       const int nco = q.Co - n0 < q.bn ? q.Co - n0 : q.bn;   // real channels of this tile
+      if (!STAGED || !staged) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < nco; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(lane_base + (uint32_t)c0, v);
-        if (valid) {
+        for (int c0 = 0; c0 < nco; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(lane_base + (uint32_t)c0, v);
+          if (valid) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c0 + j < nco) yrow[(int64_t)(c0 + j) * q.HoWo] = __uint_as_float(v[j]);
+            for (int j = 0; j < 32; ++j)
+              if (c0 + j < nco) yrow[(int64_t)(c0 + j) * q.HoWo] = __uint_as_float(v[j]);
+          }
         }
+      } else if constexpr (STAGED) {
+        // Through the staging buffer: the rows are compacted (dropped columns leave no gap) and every
+        // plane is shifted by the 16-byte phase of its run, so that the run can be written with aligned
+        // 16-byte stores.  Plane c0 + j starts (g0 + j*hw) mod 4 floats after a 16-byte boundary (c0 is a
+        // multiple of 32); warp lq writes planes lq, lq + 4, ..., which all have the same phase.
+        const uint32_t g0 = (uint32_t)((plane0 + o0) & 3);
+        const uint32_t hw = (uint32_t)q.HoWo & 3u;
+        const int h = (int)((g0 + (uint32_t)lq * hw) & 3u);
+        const int e0 = 4 * lane - h;                         // run element of the lane's first float
+        const bool full = e0 >= 0 && e0 + 3 < nv;
+        const int nhead = h ? 4 - h : 0;                     // floats before the first 16-byte boundary
+        const int tail0 = (h + nv) & ~3, ntail = (h + nv) & 3;   // floats after the last one start at column tail0
+#pragma unroll 1
+        for (int c0 = 0; c0 < nco && ok; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(lane_base + (uint32_t)c0, v);
+          if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(12);   // tmem load
+          const uint32_t stage = epi_ring + (q.epi_bufs == 2 ? (chunk_ctr & 1u) : 0u) * EPI_BUF_BYTES;
+          ++chunk_ctr;
+          if (q.epi_bufs == 1) epi_sync();                    // the readers of the last chunk are done
+          if (valid) {
+            uint32_t colb[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) colb[k] = stage + (uint32_t)((o - o0) + (int)((g0 + (uint32_t)k * hw) & 3u)) * 4u;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c0 + j < nco)
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(colb[j & 3] + (uint32_t)(j * EPI_PITCH * 4)), "r"(v[j])
+                             : "memory");
+          }
+          if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(13);   // staging stores
+          epi_sync();                                        // the chunk is staged
+          if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(14);   // barrier
+          // per lane, the same for every plane: 16-byte store, or which of its four floats exist
+          {
+            const uint32_t src0 = stage + (uint32_t)(lq * EPI_PITCH * 4) + 16u * lane;
+            float* gp0 = q.y + plane0 + (int64_t)(c0 + lq) * q.HoWo + (o0 - h) + 4 * lane;   // 16-byte aligned
+            const int nplanes = (nco - c0 - lq + 3) >> 2 < 8 ? (nco - c0 - lq + 3) >> 2 : 8;   // planes lq, lq+4, .. < nco
+            const int64_t pstep = (int64_t)4 * q.HoWo;
+            uint32_t f[8][4];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              if (i < nplanes)
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(f[i][0]), "=r"(f[i][1]), "=r"(f[i][2]), "=r"(f[i][3])
+                             : "r"(src0 + (uint32_t)(i * 4 * EPI_PITCH * 4)));
+            if (full) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                if (i < nplanes)
+                  *reinterpret_cast<float4*>(gp0 + i * pstep) = make_float4(
+                      __uint_as_float(f[i][0]), __uint_as_float(f[i][1]), __uint_as_float(f[i][2]), __uint_as_float(f[i][3]));
+            }
+            if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(15);   // reads + stores
+            // The ragged ends of the runs (at most three floats before the first and after the last
+            // 16-byte boundary) of all eight planes go out in two store instructions, lane = (plane,
+            // end element): a store instruction costs the warp some 30 cycles however few lanes it
+            // has, so one instruction per element and plane would double the epilogue's time.
+#pragma unroll
+            for (int pass = 0; pass < 2; ++pass) {
+              const int i = pass ? bi1 : bi0, t = pass ? bt1 : bt0;
+              const int col = t < 3 ? h + t : tail0 + t - 3;
+              const bool exists = i < nplanes && (t < 3 ? (t < nhead && col < h + nv) : (t - 3 < ntail && col >= h));
+              if (exists) {
+                uint32_t x;
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(x) : "r"(stage + (uint32_t)(((lq + 4 * i) * EPI_PITCH + col) * 4)));
+                (q.y + plane0 + (int64_t)(c0 + lq + 4 * i) * q.HoWo + (o0 - h))[col] = __uint_as_float(x);
+              }
+            }
+          }
+        }
+        if (!ok) break;
       }
       // the buffer may be overwritten once all four warps have read it
       tc_fence_before();
@@ -690,7 +808,17 @@ StemPlan plan_f16_stem(const Geometry& g) {
 
   const char* force_sa = getenv("IM2WIN_F16_STEM_STAGES");   // testing aid: S stages / accumulators (2..4)
   if (force_sa && atoi(force_sa) >= 2 && atoi(force_sa) < p.sa) p.sa = atoi(force_sa);
-  p.smem_bytes = p.sa * p.a_stage_bytes + p.rs * p.raw_stage_bytes + p.sb * p.b_stage_bytes + 1024;
+  // Staging buffers of the aligned-store epilogue.  Off by default: measured, the staged path is exact
+  // but twice as slow as storing from the registers (cfg3 300 us against 155 us: the two passes through
+  // shared memory and the second tensor-memory round trip cost the epilogue warps more than the aligned
+  // stores save).  IM2WIN_F16_STEM_EPI=1|2 turns it on with one or two buffers where they fit (tests do).
+  p.epi_bufs = 0;
+  const char* want_epi = getenv("IM2WIN_F16_STEM_EPI");
+  const int epi_want = want_epi ? atoi(want_epi) : 0;
+  if (epi_want >= 2 && used + 2 * EPI_BUF_BYTES <= budget) p.epi_bufs = 2;
+  else if (epi_want >= 1 && used + EPI_BUF_BYTES <= budget) p.epi_bufs = 1;
+  p.smem_bytes = p.sa * p.a_stage_bytes + p.rs * p.raw_stage_bytes + p.sb * p.b_stage_bytes +
+                 p.epi_bufs * EPI_BUF_BYTES + 1024;
   p.eligible = true;
   return p;
 }
@@ -733,18 +861,22 @@ cudaError_t launch_conv_f16_stem(const uint16_t* window, float* y, void* scratch
   const int64_t ntm = (plan.VQ + TILE_M - 1) / TILE_M;
   q.ntm = (int32_t)ntm;
   q.nwork = (int32_t)(ntm * ((g.Co + plan.bn - 1) / plan.bn));
+  q.epi_bufs = plan.epi_bufs;
   q.cbits = 0;
   while ((1 << q.cbits) < g.C) ++q.cbits;
 
-  void (*kernel)(const CUtensorMap, StemParams) = conv_f16_stem_kernel<0, 0, 0>;
-  if (g.C == 3 && g.Kh == g.Kw) {                 // the common stems: square kernels on 3 channels
-    if (g.Kh == 3) kernel = conv_f16_stem_kernel<3, 3, 3>;
-    else if (g.Kh == 5) kernel = conv_f16_stem_kernel<3, 5, 5>;
-    else if (g.Kh == 7) kernel = conv_f16_stem_kernel<3, 7, 7>;
-    else if (g.Kh == 11) kernel = conv_f16_stem_kernel<3, 11, 11>;
-  }
   const char* generic = getenv("IM2WIN_F16_STEM_GENERIC");   // testing aid: the table-driven re-layout everywhere
-  if (generic && atoi(generic)) kernel = conv_f16_stem_kernel<0, 0, 0>;
+  int kh = (g.C == 3 && g.Kh == g.Kw && !(generic && atoi(generic))) ? g.Kh : 0;   // the common stems: square kernels on 3 channels
+  if (kh != 3 && kh != 5 && kh != 7 && kh != 11) kh = 0;
+  void (*kernel)(const CUtensorMap, StemParams);
+  if (plan.epi_bufs > 0)
+    kernel = kh == 3 ? conv_f16_stem_kernel<3, 3, 3, true> : kh == 5 ? conv_f16_stem_kernel<3, 5, 5, true>
+           : kh == 7 ? conv_f16_stem_kernel<3, 7, 7, true> : kh == 11 ? conv_f16_stem_kernel<3, 11, 11, true>
+                                                                      : conv_f16_stem_kernel<0, 0, 0, true>;
+  else
+    kernel = kh == 3 ? conv_f16_stem_kernel<3, 3, 3, false> : kh == 5 ? conv_f16_stem_kernel<3, 5, 5, false>
+           : kh == 7 ? conv_f16_stem_kernel<3, 7, 7, false> : kh == 11 ? conv_f16_stem_kernel<3, 11, 11, false>
+                                                                      : conv_f16_stem_kernel<0, 0, 0, false>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
   if (e != cudaSuccess) return e;
   // persistent CTAs: one per SM (measured: a second CTA per SM, where it fits, only slows the layer

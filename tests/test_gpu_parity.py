@@ -268,6 +268,23 @@ def test_stem_kernel_variants(generic, ctas, monkeypatch):
         assert np.array_equal(y.astype(np.float64), yr), name
 
 
+@pytest.mark.parametrize("bufs", ["1", "2"])
+def test_stem_kernel_staged_epilogue(bufs, monkeypatch):
+    """The opt-in epilogue of the one-k-block kernel that writes each output plane's run with aligned
+    16-byte stores through a staging buffer (one or two buffers): runs that start on every 16-byte
+    phase, tiles that straddle images (which store from the registers), several tiles per CTA."""
+    monkeypatch.setenv("IM2WIN_F16_STEM_EPI", bufs)
+    by_name = {l.name: l for l in SMALL}
+    layers = [by_name[n] for n in ("cfg1", "stem_rag4", "stem_rag2", "stem_rag3", "stem_imgs", "stem_wide", "stem_c8")]
+    layers += [workloads.TABLE1_LAYERS["cv3"].with_batch(4), workloads.TABLE1_LAYERS["cv7"].with_batch(3)]
+    for layer in layers:
+        dims = layer.dims()
+        x, f = workloads.make_small_integer_inputs(layer)
+        y, _, _ = gpu_conv(x, f, dims, "f16-stem")
+        yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+        assert np.array_equal(y.astype(np.float64), yr), layer.name
+
+
 @pytest.mark.parametrize("name", ["cfg2", "cfg4a", "cfg5k3"])
 def test_full_size_mat_kernel_sampled(name):
     """The matrix-transpose fp16 kernel forced at benchmark sizes, on sampled outputs."""
