@@ -76,30 +76,39 @@ struct Segment {            // the part of a tile that lies in one image
 };
 
 // Splits the rows of the tile starting at virtual position q0 by image: within an image the
-// columns of one channel are contiguous in the window tensor.
-__device__ __forceinline__ int split_by_image(const RawParams& q, int q0, Segment* segs) {
+// columns of one channel are contiguous in the window tensor.  Lane g of the calling warp works out
+// segment g (the segments after the first start on image boundaries, so there is no loop; a lone
+// lane walking them cost the re-layout warps a quarter of their time on layers with three k-blocks);
+// every lane gets the number of segments.
+__device__ __forceinline__ int split_by_image(const RawParams& q, int q0, Segment* segs, int lane) {
   const int img_rows = q.Ho * q.Wq;               // VQ < 2^31 is a condition of this kernel
-  int n = q0 / img_rows, a = q0 - n * img_rows;
-  int remaining = q.rows, row0 = 0, box0 = 0, g = 0;
-  while (remaining > 0 && n < q.N && g < SEG_MAX) {
-    const int cnt = remaining < img_rows - a ? remaining : img_rows - a;
-    const int f0 = a * q.Kh;                             // element offset inside the channel plane
-    const int span = (f0 & 7) + cnt * q.Kh;
-    segs[g].plane0 = n * q.C;
-    segs[g].x0 = f0 & ~7;
-    segs[g].o0 = f0 & 7;
-    segs[g].row0 = row0;
-    segs[g].cnt = cnt;
-    segs[g].box0 = box0;
-    segs[g].nbox = span <= BOXW ? 1 : (span - (BOXW - BOXSTEP) + BOXSTEP - 1) / BOXSTEP;
-    box0 += segs[g].nbox;
-    row0 += cnt;
-    remaining -= cnt;
-    a = 0;
-    ++n;
-    ++g;
+  const int n0 = q0 / img_rows, a0 = q0 - n0 * img_rows;
+  const int first_cnt = q.rows < img_rows - a0 ? q.rows : img_rows - a0;
+  const int n = n0 + lane;
+  const int a = lane == 0 ? a0 : 0;
+  const int row0 = lane == 0 ? 0 : first_cnt + (lane - 1) * img_rows;
+  int cnt = q.rows - row0;
+  if (cnt > img_rows - a) cnt = img_rows - a;
+  const bool valid = lane < SEG_MAX && row0 < q.rows && n < q.N;
+  const int f0 = a * q.Kh;                               // element offset inside the channel plane
+  const int span = (f0 & 7) + cnt * q.Kh;
+  const int nbox = !valid ? 0 : (span <= BOXW ? 1 : (span - (BOXW - BOXSTEP) + BOXSTEP - 1) / BOXSTEP);
+  int incl = nbox;                                       // inclusive prefix sum over the first SEG_MAX lanes
+  int t = __shfl_up_sync(0xffffffffu, incl, 1);
+  if (lane >= 1) incl += t;
+  t = __shfl_up_sync(0xffffffffu, incl, 2);
+  if (lane >= 2) incl += t;
+  if (valid) {
+    segs[lane].plane0 = n * q.C;
+    segs[lane].x0 = f0 & ~7;
+    segs[lane].o0 = f0 & 7;
+    segs[lane].row0 = row0;
+    segs[lane].cnt = cnt;
+    segs[lane].box0 = incl - nbox;
+    segs[lane].nbox = nbox;
   }
-  return g;
+  __syncwarp();
+  return __popc(__ballot_sync(0xffffffffu, valid));
 }
 
 // Persistent kernel: every CTA walks work items w = blockIdx.x, blockIdx.x + gridDim.x, ...
@@ -191,9 +200,7 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
     TIMER_DECL;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
       const int q0 = (w % q.ntm) * TILE_M;
-      int nseg = 0;
-      if (lane == 0) nseg = split_by_image(q, q0, segs);
-      nseg = __shfl_sync(0xffffffffu, nseg, 0);
+      const int nseg = split_by_image(q, q0, segs, lane);
 #pragma unroll
       for (int it = 0; it < ITEMS; ++it) {
         rbase[it] = 0;
@@ -342,9 +349,13 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
     TIMER_DECL;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
       const int q0 = (w % q.ntm) * TILE_M;
-      int nseg = 0;
-      if (lane == 0) nseg = split_by_image(q, q0, segs);
-      nseg = __shfl_sync(0xffffffffu, nseg, 0);
+      const int nseg = split_by_image(q, q0, segs, lane);
+      int nbox = 0;
+      for (int g = 0; g < nseg; ++g) nbox += segs[g].nbox;
+      // box b of the stage: its segment and its place in it (lane b issues the copy)
+      int bg = 0, bj = lane;
+      while (bg < nseg - 1 && bj >= segs[bg].nbox) { bj -= segs[bg].nbox; ++bg; }
+      const int bx = segs[bg].x0 + bj * BOXSTEP, by = segs[bg].plane0;
       for (int kb = 0; kb < q.num_kb && ok; ++kb) {
         if (leader) TIMER_LAP(6);              // raw loader: issuing copies
         ok = mbar_wait(r_empty0 + 8 * rst, rph ^ 1u, &abort_flag, q.status);
@@ -354,14 +365,18 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
         const uint32_t bar = r_full0 + 8 * rst;
         const int c_lo = (kb * KB) / q.Kh;
         const uint32_t stage = raw_ring + rst * q.raw_stage_bytes;
-        if (leader) {
-          int nbox = 0;
-          for (int g = 0; g < nseg; ++g) nbox += segs[g].nbox;
-          mbar_arrive_expect_tx(bar, (uint32_t)(nbox * q.nslot * 256));
-          for (int g = 0; g < nseg; ++g)
-            for (int j = 0; j < segs[g].nbox; ++j)
-              tma_load_2d(stage + (segs[g].box0 + j) * q.box_bytes, &wmap, segs[g].x0 + j * BOXSTEP,
-                          segs[g].plane0 + c_lo, bar);
+        // one lane announces the bytes, then every lane issues its box (issuing a copy costs a lone
+        // lane several hundred cycles; a stage has up to a dozen)
+        if (leader) mbar_arrive_expect_tx(bar, (uint32_t)(nbox * q.nslot * 256));
+        __syncwarp();
+        for (int b = lane; b < nbox; b += 32) {
+          if (b == lane) {
+            tma_load_2d(stage + b * q.box_bytes, &wmap, bx, by + c_lo, bar);
+          } else {                                 // more than 32 boxes: beyond what the plan allows, kept for safety
+            int g = 0, j = b;
+            while (g < nseg - 1 && j >= segs[g].nbox) { j -= segs[g].nbox; ++g; }
+            tma_load_2d(stage + b * q.box_bytes, &wmap, segs[g].x0 + j * BOXSTEP, segs[g].plane0 + c_lo, bar);
+          }
         }
         __syncwarp();
         if (++rst == q.rs) { rst = 0; rph ^= 1u; }
