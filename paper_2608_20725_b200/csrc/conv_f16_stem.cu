@@ -620,7 +620,7 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)q.bnr + ((uint32_t)(lq * 32) << 16);
       const int nco = q.Co - n0 < q.bn ? q.Co - n0 : q.bn;   // real channels of this tile
-      if (!STAGED || !staged) {
+      if ((!STAGED || !staged) && nco > 64) {
 #pragma unroll 1
         for (int c0 = 0; c0 < nco; c0 += 32) {
           uint32_t v[32];
@@ -629,6 +629,28 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
               if (c0 + j < nco) yrow[(int64_t)(c0 + j) * q.HoWo] = __uint_as_float(v[j]);
+          }
+        }
+      } else if (!STAGED || !staged) {
+        // up to 64 channels: both tensor-memory loads are in flight together (one costs the warp some
+        // 500 cycles when the tensor core is busy with the next tiles); measured 1-3 % on the 64-channel
+        // stems, while wider tiles (96 channels: a dual round and a single one) lost 8 % with it
+#pragma unroll 1
+        for (int c0 = 0; c0 < nco; c0 += 64) {
+          uint32_t v[32], v2[32];
+          tmem_ld32_issue(lane_base + (uint32_t)c0, v);
+          const bool second = c0 + 32 < nco;
+          if (second) tmem_ld32_issue(lane_base + (uint32_t)(c0 + 32), v2);
+          tmem_ld_wait();
+          if (valid) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c0 + j < nco) yrow[(int64_t)(c0 + j) * q.HoWo] = __uint_as_float(v[j]);
+            if (second) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (c0 + 32 + j < nco) yrow[(int64_t)(c0 + 32 + j) * q.HoWo] = __uint_as_float(v2[j]);
+            }
           }
         }
       } else if constexpr (STAGED) {
