@@ -175,7 +175,7 @@ class LayerRunner:
                     events.append((f"{name}_{prec}", e0, e1))
 
     def algorithmic_bytes(self, kernel):
-        """Bytes each kernel must move once (stated per kernel in the design doc)."""
+        """Bytes each kernel must move once: input + window for a transform, window + output (+ filter) for a convolution."""
         l, es = self.layer, (4 if kernel.endswith("f32") else 2)
         x_el = l.N * l.C * l.H * l.W
         win_el = l.N * l.C * self.ho * l.Kh * (l.W + 2 * l.pad)
