@@ -260,13 +260,7 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
           if (n0 + c0 >= q.Co) break;
           uint32_t v[32];
           tmem_ld32(lane_base + (uint32_t)c0, v);
-          if (valid) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int co = n0 + c0 + j;
-              if (co < q.Co) yrow[(int64_t)co * q.HoWo] = __uint_as_float(v[j]);
-            }
-          }
+          if (valid) store_strided32(yrow + (int64_t)(n0 + c0) * q.HoWo, q.HoWo, v, q.Co - n0 - c0);
         }
       }
     }

@@ -625,11 +625,7 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
         for (int c0 = 0; c0 < nco; c0 += 32) {
           uint32_t v[32];
           tmem_ld32(lane_base + (uint32_t)c0, v);
-          if (valid) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c0 + j < nco) yrow[(int64_t)(c0 + j) * q.HoWo] = __uint_as_float(v[j]);
-          }
+          if (valid) store_strided32(yrow + (int64_t)c0 * q.HoWo, q.HoWo, v, nco - c0);
         }
       } else if (!STAGED || !staged) {
         // up to 64 channels: both tensor-memory loads are in flight together (one costs the warp some
@@ -643,14 +639,8 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
           if (second) tmem_ld32_issue(lane_base + (uint32_t)(c0 + 32), v2);
           tmem_ld_wait();
           if (valid) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c0 + j < nco) yrow[(int64_t)(c0 + j) * q.HoWo] = __uint_as_float(v[j]);
-            if (second) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (c0 + 32 + j < nco) yrow[(int64_t)(c0 + 32 + j) * q.HoWo] = __uint_as_float(v2[j]);
-            }
+            store_strided32(yrow + (int64_t)c0 * q.HoWo, q.HoWo, v, nco - c0);
+            if (second) store_strided32(yrow + (int64_t)(c0 + 32) * q.HoWo, q.HoWo, v2, nco - c0 - 32);
           }
         }
       } else if constexpr (STAGED) {
