@@ -811,7 +811,9 @@ StemPlan plan_f16_stem(const Geometry& g) {
   // three raw stages by default (measured: eight in flight slow a 3-channel 3x3 layer down from 1.01 ms
   // to 1.27 ms, as a second CTA per SM does); IM2WIN_F16_STEM_RAW = 2..8 sets another depth (a testing aid)
   const char* force_rs = getenv("IM2WIN_F16_STEM_RAW");
-  const int rs_max = force_rs && atoi(force_rs) >= 2 && atoi(force_rs) <= MAX_RAW ? atoi(force_rs) : 3;
+  // (per-strip runs are many small copies: a fourth stage pays there, 273 -> 250 us on the 7x7 stride-2
+  // layer with 227-wide strips; with per-image runs it changes nothing or costs, see above)
+  const int rs_max = force_rs && atoi(force_rs) >= 2 && atoi(force_rs) <= MAX_RAW ? atoi(force_rs) : (p.ragged ? 4 : 3);
   if (rs_max < p.rs) { used -= (p.rs - rs_max) * p.raw_stage_bytes; p.rs = rs_max; }
   while (p.rs < rs_max && (p.rs + 1) * p.raw_stage_bytes <= 48 * 1024 && used + p.raw_stage_bytes <= budget) {
     ++p.rs;
