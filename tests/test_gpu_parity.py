@@ -326,7 +326,7 @@ def test_full_size_wide_kernels_sampled(name):
 # ------------------------------------------------- the paper's Table 1 layers ----
 TABLE1 = [workloads.TABLE1_LAYERS[k].with_batch(n) for k, n in
           (("cv1", 16), ("cv2", 8), ("cv3", 16), ("cv4", 6), ("cv5", 32), ("cv7", 12), ("cv8", 12), ("cv9", 32),
-           ("cv12", 64))] + [workloads.TABLE1_LAYERS["cv1"], workloads.TABLE1_LAYERS["cv6"]]   # two at the paper's batch of 256
+           ("cv12", 64))] + [workloads.TABLE1_LAYERS[k] for k in ("cv1", "cv3", "cv6", "cv10")]   # four at the paper's batch of 256
 
 
 @pytest.mark.parametrize("layer", TABLE1, ids=lambda l: f"{l.name}-n{l.N}")
