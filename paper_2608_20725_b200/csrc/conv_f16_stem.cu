@@ -256,6 +256,7 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
       }
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
       if (!ok) break;
+      __syncwarp();                             // lane 0 observed the barrier; orders the other lanes' reads after it
       const Segment* segs = seg_ring[rst];      // published by the loader's arrival on the raw stage's barrier
       const int nseg = nseg_ring[rst];
       const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
