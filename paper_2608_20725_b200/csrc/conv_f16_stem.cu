@@ -30,9 +30,10 @@
 // last virtual column of a strip lacks some columns, which are staged as zeros and only feed
 // accumulator rows that are dropped.  Persistent CTAs; S stage i and accumulator i (two to four of
 // each, in tensor memory) belong together, so that one commit per tile tells the epilogue that the
-// accumulator is complete and the re-layout warps that the S stage is free; bounded mbarrier waits.  Warp roles: 0-7 and 11 re-layout, 8 filter copies, 9 MMA issue (and
-// tensor-memory allocation), 10 raw copies, 12-15 epilogue (a second epilogue warp per lane
-// quadrant was measured: 5 % faster on a 3-channel 3x3 layer, 5-8 % slower on the 7x7 and 11x11 stems).
+// accumulator is complete and the re-layout warps that the S stage is free; bounded mbarrier waits.
+// Warp roles: 0-7 and 11 re-layout, 8 filter copies, 9 MMA issue (and tensor-memory allocation),
+// 10 raw copies, 12-15 epilogue (a second epilogue warp per lane quadrant was measured: 5 % faster on
+// a 3-channel 3x3 layer, 5-8 % slower on the 7x7 and 11x11 stems).
 #include <cuda.h>
 #include <stdlib.h>
 
@@ -52,7 +53,7 @@ constexpr int WARP_TMA = 8, WARP_MMA = 9, WARP_RAW = 10, WARP_REPACK9 = 11, WARP
 constexpr int NUM_WARPS = 16;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr int MAX_STAGES = 4;                        // S stages / accumulators
-constexpr int MAX_RAW = 8;                           // raw stages (small copies are latency bound: many in flight)
+constexpr int MAX_RAW = 8;                           // most raw stages a testing switch may ask for (3 or 4 are used)
 constexpr int MAX_B = 16;                            // filter stages (a resident filter needs Kw of them)
 constexpr int SEG_MAX = 6;                           // strip segments (or images) one tile may touch
 constexpr int SEG_GAP = 48;                          // bytes between the copies of consecutive segments
