@@ -66,6 +66,15 @@ typedef enum {
 const char* im2win_status_string(im2win_status status);
 
 /*
+ * Name of the convolution kernel the library selects for a layer (host-only,
+ * launches nothing; static storage): "f32-ffma" for IM2WIN_F32; for IM2WIN_F16
+ * one of the tensor-core kernels of Algorithm 1's GEMM view, "f16-stem",
+ * "f16-mat", "f16-matc", "f16-raw", "f16-shift" or "f16-gather"; "none" for an
+ * invalid shape.  For reports and tests; the choice is an implementation detail.
+ */
+const char* im2win_conv_kernel_name(const im2win_shape* shape, im2win_dtype dtype);
+
+/*
  * Sizes, in bytes, of the buffers a layer needs (host-only, launches nothing).
  *   window_bytes  = N*C*Ho*Kh*(W+2p) * sizeof(element): the closed-form size
  *                   of the im2win tensor (paper Eq. 2; Section "Im2win Data
@@ -143,6 +152,14 @@ im2win_status im2win_conv_packed(const void* window, float* y_nchw, void* scratc
  * (written by the last convolution call that used it) and returns
  * IM2WIN_ERR_TIMEOUT if a bounded device wait gave up, IM2WIN_ERR_CUDA if the
  * stream reports an error, else IM2WIN_OK.  Blocking.
+ *
+ * Layout of the status block (the first 256 bytes of `scratch`, 32-bit words,
+ * all cleared by every filter pack): word 0 is raised by a wait that gave up.
+ * Words 1 and 2 are testing aids read by the fp16 kernels: a non-zero word 1
+ * replaces the number of polls after which a wait gives up (2^24, and never
+ * more than about four seconds); the marker 0x0d0a11fe in word 2 makes the
+ * one-k-block kernel leave out one barrier arrival, so that a test can watch a
+ * wait run out and the kernel return.  Nothing in the library writes them.
  */
 im2win_status im2win_check_status(const void* scratch, void* cuda_stream);
 
@@ -198,7 +215,9 @@ im2win_status im2win_layer_forward_host(const void* x_host, const void* filter_h
  *     library routine.
  *   - The first call on each device looks up the device address of the array
  *     (with that device current) and caches it; make that first call outside any
- *     stream capture.
+ *     stream capture.  The cached address belongs to the device's current
+ *     context: it does not survive a cudaDeviceReset, after which this entry
+ *     point must not be used again in the process.
  *   - All calls on a device share the one array, which keeps whatever the last
  *     call left in it.  Each call rewrites every byte it later reads, so
  *     back-to-back calls on one stream are safe; two calls whose kernels may

@@ -25,7 +25,7 @@ STATUS_NAMES = {
 EXPORTS = (
     "im2win_status_string", "im2win_workspace_size", "im2win_transform", "im2win_conv_f32", "im2win_conv_f16",
     "im2win_check_status", "im2win_layer_workspace_size", "im2win_layer_forward_host",
-    "im2win_conv_f32_static", "im2win_pack_filter", "im2win_conv_packed",
+    "im2win_conv_f32_static", "im2win_pack_filter", "im2win_conv_packed", "im2win_conv_kernel_name",
 )
 
 STATIC_SCRATCH_BYTES = 4 << 20
@@ -66,8 +66,10 @@ def lib() -> ctypes.CDLL:
     L.im2win_conv_f32_static.argtypes = [vp, vp, vp, P(Shape), vp]
     L.im2win_pack_filter.argtypes = [vp, vp, sz, P(Shape), ctypes.c_int, vp]
     L.im2win_conv_packed.argtypes = [vp, vp, vp, sz, P(Shape), ctypes.c_int, vp]
+    L.im2win_conv_kernel_name.argtypes = [P(Shape), ctypes.c_int]
     for name in EXPORTS[1:]:
         getattr(L, name).restype = ctypes.c_int
+    L.im2win_conv_kernel_name.restype = ctypes.c_char_p
     _lib = L
     return L
 
@@ -126,6 +128,12 @@ def _workspace_size_uncached(s: Shape, dtype: int) -> Tuple[int, int, int, int]:
     _check(lib().im2win_workspace_size(ctypes.byref(s), dtype, ctypes.byref(wb), ctypes.byref(sb),
                                        ctypes.byref(ho), ctypes.byref(wo)), "im2win_workspace_size")
     return wb.value, sb.value, ho.value, wo.value
+
+
+def im2win_conv_kernel_name(shape, dtype: int) -> str:
+    """Name of the convolution kernel the library selects for the layer (for reports and tests)."""
+    s = as_shape(shape)
+    return lib().im2win_conv_kernel_name(ctypes.byref(s), dtype).decode()
 
 
 def im2win_transform(x: torch.Tensor, window: torch.Tensor, shape, stream=None) -> None:

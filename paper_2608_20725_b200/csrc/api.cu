@@ -179,6 +179,19 @@ const char* im2win_status_string(im2win_status status) {
   return "unknown status";
 }
 
+const char* im2win_conv_kernel_name(const im2win_shape* shape, im2win_dtype dtype) {
+  Geometry g;
+  ScratchLayout l;
+  if (derive_geometry(shape, &g) != IM2WIN_OK || scratch_layout(g, dtype, &l) != IM2WIN_OK) return "none";
+  if (dtype == IM2WIN_F32) return "f32-ffma";
+  if (l.f16_stem) return "f16-stem";
+  if (l.f16_mat) return "f16-mat";
+  if (l.f16_matc) return "f16-matc";
+  if (l.f16_raw) return "f16-raw";
+  if (l.f16_shift) return "f16-shift";
+  return "f16-gather";
+}
+
 im2win_status im2win_workspace_size(const im2win_shape* shape, im2win_dtype dtype, size_t* window_bytes,
                                     size_t* scratch_bytes, int32_t* Ho, int32_t* Wo) {
   Geometry g;

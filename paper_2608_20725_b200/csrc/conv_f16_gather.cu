@@ -112,6 +112,7 @@ conv_f16_gather_kernel(const __grid_constant__ CUtensorMap fmap, ConvF16Params q
       // Lane 0 polls; the result is shared so that the whole warp takes the same path.
       if (lane == 0) ok = mbar_wait(empty_bar0 + 8 * s, (it & 1u) ^ 1u, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
       if (!ok) break;
       const uint32_t a_stage = smem_base + s * STAGE_BYTES;
 #pragma unroll 1
@@ -144,6 +145,7 @@ conv_f16_gather_kernel(const __grid_constant__ CUtensorMap fmap, ConvF16Params q
     // tcgen05.ld is warp-collective: the decision must be uniform in the warp.
     if (ok && lane == 0) ok = mbar_wait(acc_bar, 0u, &abort_flag, q.status);
     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+    __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
     if (ok) {
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + ((uint32_t)(warp * 32) << 16);

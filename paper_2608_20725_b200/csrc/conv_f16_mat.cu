@@ -269,6 +269,7 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
           if (threadIdx.x == 0) TIMER_LAP(2);   // wait for a free S stage
         }
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
         if (!ok) break;
         const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
         const uint32_t raw_stage = raw_ring + rst * q.raw_stage_bytes + src_l;
@@ -577,6 +578,7 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
       }
       if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
       if (!ok) break;
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);

@@ -299,6 +299,7 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
           if (threadIdx.x == 0) TIMER_LAP(2);   // wait for a free S stage
         }
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
         if (!ok) break;
         const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
         const uint32_t info = kbinfo[kb];
@@ -312,7 +313,9 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
             good = mbar_wait(r_full0 + 8 * rst, rph, &abort_flag, q.status);
             if (threadIdx.x == 0) TIMER_LAP(1);   // wait for the raw stage
           }
-          return __shfl_sync(0xffffffffu, (int)good, 0) != 0;
+          good = __shfl_sync(0xffffffffu, (int)good, 0) != 0;
+          __syncwarp();   // lane 0 observed the barrier: orders the other lanes' reads of the raw stage after it
+          return good;
         };
         auto raw_release = [&]() {
           __syncwarp();
@@ -660,6 +663,7 @@ __device__ __forceinline__ void conv_f16_mat_body(const CUtensorMap& fmap, const
       }
       if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
       if (!ok) break;
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);

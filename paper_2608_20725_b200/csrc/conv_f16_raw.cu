@@ -226,6 +226,7 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
           if (threadIdx.x == 0) TIMER_LAP(2);   // wait for a free S stage
         }
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
         if (!ok) break;
         const uint32_t a_stage = a_ring + st * q.a_stage_bytes;
         const uint32_t raw_stage = raw_ring + rst * q.raw_stage_bytes;
@@ -405,6 +406,7 @@ conv_f16_raw_kernel(const __grid_constant__ CUtensorMap fmap, const __grid_const
       }
       if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
       if (!ok) break;
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);

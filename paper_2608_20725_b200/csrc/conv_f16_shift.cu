@@ -218,6 +218,7 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
           if (threadIdx.x == 0) TIMER_LAP(2);   // issuing loads
           if (lane == 0) ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
           ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+          __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
           if (threadIdx.x == 0) TIMER_LAP(1);   // wait for a free stage
         }
         if (ok) store(a_stage, climit, gidx, buf);
@@ -237,6 +238,7 @@ conv_f16_shift_kernel(const __grid_constant__ CUtensorMap fmap, ShiftParams q) {
     // ---------------- epilogue --------------------------------------------------
     if (ok && lane == 0) ok = mbar_wait(acc_bar, 0u, &abort_flag, q.status);
     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+    __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
     if (threadIdx.x == 0) TIMER_LAP(5);     // wait for the accumulator
     if (ok) {
       tc_fence_after();

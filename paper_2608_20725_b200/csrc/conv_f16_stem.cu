@@ -501,6 +501,7 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
     const int du = adv / per, da = adv - du * per;
     const int dn = q.ragged ? du / q.Ho : 0, dho = q.ragged ? du - dn * q.Ho : 0;
     const int cmask = (1 << q.cbits) - 1;       // copies are numbered (run << cbits) | channel
+    const bool drop_first_arrive = *reinterpret_cast<volatile uint32_t*>(q.status + 2) == ptx::kDebugDropArrive;
     TIMER_DECL;
     for (int w = blockIdx.x; w < q.nwork && ok; w += gridDim.x) {
       if (!stepping) pos_init(q, (w % q.ntm) * TILE_M, pos);
@@ -551,7 +552,9 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
         }
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar);           // after every lane has announced its bytes
+      // after every lane has announced its bytes (testing aid: with the marker in word 2 of the status
+      // block the first arrival of each CTA is left out, so that the waits on this stage run out)
+      if (lane == 0 && !(drop_first_arrive && w == (int)blockIdx.x)) mbar_arrive(bar);
       if (++rst == q.rs) { rst = 0; rph ^= 1u; }
     }
     if (lane == 0) { TIMER_LAP(6); TIMER_FLUSH(); }
@@ -605,6 +608,7 @@ conv_f16_stem_kernel(const __grid_constant__ CUtensorMap fmap, StemParams q) {
       }
       if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, eph, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
       if constexpr (STAGED) {
         uint32_t all_ok;
         asm volatile(

@@ -30,7 +30,12 @@
 namespace im2win {
 namespace ptx {
 
-constexpr uint32_t SPIN_LIMIT = 1u << 24;
+constexpr uint32_t SPIN_LIMIT = 1u << 24;      // polls before a wait gives up (see mbar_wait)
+constexpr uint32_t SPIN_CHUNK = 1024;          // polls between looks at the abort flag and the clock
+constexpr uint64_t SPIN_TIME_NS = 4000000000ull;   // wall-time bound of one wait: 4 s
+// Word 2 of the status block: this marker makes the one-k-block kernel's copy warp leave out one
+// barrier arrival (the test of the bounded waits; nothing in the library writes it).
+constexpr uint32_t kDebugDropArrive = 0x0d0a11feu;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -67,17 +72,53 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
-// Bounded wait.  Returns false (and raises the flags) when the limit is hit or
-// another thread of the CTA has already given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* status) {
-  for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 1023u) == 1023u && *abort_flag) return false;
+// Bounded waits.  A wait first polls SPIN_CHUNK times in line; only a wait that is still pending
+// then (milliseconds: each poll may suspend the thread for a while) enters the slow path below,
+// which gives up after SPIN_LIMIT polls or SPIN_TIME_NS of wall time, whichever comes first, or as
+// soon as another thread of the CTA has given up.  Word 1 of the status block, when non-zero,
+// replaces SPIN_LIMIT (a testing aid: the filter pack clears the block, a test may then lower the
+// limit before the convolution runs).  On giving up the wait raises the CTA's abort flag and word
+// 0 of the status block and returns false; the caller unwinds (drains its copies, frees its tensor
+// memory) and the kernel returns normally.
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+template <bool CLUSTER>
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                            uint32_t* status) {
+  uint32_t limit = *reinterpret_cast<volatile uint32_t*>(status + 1);
+  if (limit == 0u) limit = SPIN_LIMIT;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t i = SPIN_CHUNK; i < limit; i += SPIN_CHUNK) {
+    for (uint32_t j = 0; j < SPIN_CHUNK; ++j) {
+      uint32_t ok;
+      if constexpr (CLUSTER) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+      } else {
+        ok = mbar_try_wait(bar, parity);
+      }
+      if (ok) return true;
+    }
+    if (*abort_flag) return false;
+    if (global_timer_ns() - t0 > SPIN_TIME_NS) break;
   }
   *abort_flag = 1u;
   atomicExch(status, 1u);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* status) {
+  for (uint32_t i = 0; i < SPIN_CHUNK; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow<false>(bar, parity, abort_flag, status);
 }
 // True in exactly one lane of the (converged) warp.
 __device__ __forceinline__ bool elect_one() {
@@ -286,13 +327,9 @@ __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t
 }
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                                   uint32_t* status) {
-  for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
+  for (uint32_t i = 0; i < SPIN_CHUNK; ++i)
     if (mbar_try_wait_cluster(bar, parity)) return true;
-    if ((i & 1023u) == 1023u && *abort_flag) return false;
-  }
-  *abort_flag = 1u;
-  atomicExch(status, 1u);
-  return false;
+  return mbar_wait_slow<true>(bar, parity, abort_flag, status);
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");

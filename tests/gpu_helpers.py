@@ -78,6 +78,37 @@ def gpu_conv(x_cpu: torch.Tensor, f_cpu: torch.Tensor, dims: dict, precision: st
     return yh, xd.float().cpu().numpy(), fd.float().cpu().numpy()
 
 
+def gpu_layer_keep_window(x_cpu: torch.Tensor, f_cpu: torch.Tensor, dims: dict, precision: str, images):
+    """Transform + convolution like gpu_conv, for layers whose window tensor is too large to copy to
+    the host whole: returns (y float32 numpy, {n: window of image n as a raw-integer numpy array
+    [1, C, Ho, Kh*Wp]} for n in `images`)."""
+    tdt = torch.float32 if precision == "f32" else torch.float16
+    idt = torch.int32 if precision == "f32" else torch.int16
+    code = binding.F32 if precision == "f32" else binding.F16
+    xd = x_cpu.to(tdt).cuda().contiguous()
+    fd = f_cpu.to(tdt).cuda().contiguous()
+    wb, sb, ho, wo = binding.im2win_workspace_size(dims, code)
+    nwin = wb // xd.element_size()
+    nout = dims["N"] * dims["Co"] * ho * wo
+    wwhole, win = guarded(nwin, tdt, 3.0)
+    ywhole, y = guarded(nout, torch.float32, -123.0)
+    swhole, scratch = guarded(sb, torch.uint8, 0x5a)
+    binding.im2win_transform(xd, win, dims)
+    if precision == "f32":
+        binding.im2win_conv_f32(win, fd, y, scratch, dims)
+    else:
+        binding.im2win_conv_f16(win, fd, y, scratch, dims)
+    binding.im2win_check_status(scratch)
+    assert_guards_intact(wwhole, nwin, 3.0)
+    assert_guards_intact(ywhole, nout, -123.0)
+    assert_guards_intact(swhole, sb, 0x5a)
+    per = nwin // dims["N"]
+    strip = dims["Kh"] * (dims["W"] + 2 * dims["pad"])
+    wins = {n: win[n * per:(n + 1) * per].cpu().view(idt).numpy().reshape(1, dims["C"], ho, strip) for n in images}
+    yh = y.cpu().numpy().reshape(dims["N"], dims["Co"], ho, wo)
+    return yh, wins
+
+
 def oracle_inputs(x_cpu: torch.Tensor, f_cpu: torch.Tensor, precision: str):
     """The values the oracle computes on: fp32 inputs as they are, or rounded to binary16 by the
     oracle's own routine for the fp16 path."""

@@ -55,6 +55,6 @@ def test_random_layer_all_paths(layer):
     check_conv(y, yr32, ar32, "f32", layer.name)
     xo, fo = oracle_inputs(x, f, "f16")
     yr16, ar16 = oracle.conv_direct(xo, fo, dims)
-    for precision in ("f16", "f16-mat", "f16-shift", "f16-gather"):
+    for precision in ("f16", "f16-mat", "f16-shift", "f16-stem", "f16-gather"):
         y, _, _ = gpu_conv(x, f, dims, precision)
         check_conv(y, yr16, ar16, precision, layer.name)

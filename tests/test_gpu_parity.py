@@ -10,8 +10,8 @@ import torch
 import oracle
 from paper_2608_20725_b200 import binding, workloads
 from paper_2608_20725_b200.workloads import Layer
-from gpu_helpers import (assert_guards_intact, check_conv, gpu_conv, gpu_transform, guarded,
-                         oracle_inputs)
+from gpu_helpers import (assert_guards_intact, check_conv, gpu_conv, gpu_layer_keep_window, gpu_transform,
+                         guarded, oracle_inputs)
 
 pytestmark = pytest.mark.gpu
 
@@ -304,56 +304,97 @@ def test_full_size_mat_kernel_sampled(name):
     check_conv(y[-1:], yi, ai, "f16-mat", layer.name + " last image")
 
 
+def _sample_indices(total, count, seed, extra=()):
+    rng = np.random.default_rng(seed)
+    return np.concatenate([rng.integers(0, total, count), np.asarray(list(extra), dtype=np.int64)])
+
+
+def _whole_conv_check(y, xo, fo, dims, precision, name, images_per_pass):
+    """Every output element of y against the oracle's im2win route, a few images at a time."""
+    worst = 0.0
+    for n0 in range(0, dims["N"], images_per_pass):
+        n1 = min(dims["N"], n0 + images_per_pass)
+        yr, ar = oracle.conv_im2win(xo[n0:n1], fo, dict(dims, N=n1 - n0))
+        worst = max(worst, check_conv(y[n0:n1], yr, ar, precision, f"{name} images {n0}..{n1 - 1}"))
+    return worst
+
+
 @pytest.mark.parametrize("name", ["cfg5k7", "cfg5k11"])
 def test_full_size_wide_kernels_sampled(name):
-    """The two largest sweep layers at benchmark size (K = 12 544 and 30 976): sampled outputs
-    only, the oracle needs minutes for a whole image of these."""
+    """The two largest sweep layers at benchmark size (K = 12 544 and 30 976), in the launch
+    configuration the benchmark times: 65 536 sampled outputs from Eq. 1, two whole images (the
+    first and the last) through the im2win route, and the transform of every image bit for bit."""
     layer = workloads.LAYERS[name]
     dims = layer.dims()
     x, f = workloads.make_inputs(layer)
     ho, wo = oracle.out_dims(dims)
     total = layer.N * layer.Co * ho * wo
-    rng = np.random.default_rng(layer.seed + 11)
-    idx = np.concatenate([rng.integers(0, total, 2048), [0, total - 1, wo - 1, ho * wo - 1, total - ho * wo]])
-    for precision in layer.precisions:
-        y, _, _ = gpu_conv(x, f, dims, precision)
-        xo, fo = oracle_inputs(x, f, precision)
-        yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
-        check_conv(y.reshape(-1)[idx], yr, ar, precision, layer.name)
-        del y
-
-
-# ------------------------------------------------- the paper's Table 1 layers ----
-TABLE1 = [workloads.TABLE1_LAYERS[k].with_batch(n) for k, n in
-          (("cv1", 16), ("cv2", 8), ("cv3", 16), ("cv4", 6), ("cv5", 32), ("cv7", 12), ("cv8", 12), ("cv9", 32),
-           ("cv12", 64))] + [workloads.TABLE1_LAYERS[k] for k in ("cv1", "cv3", "cv6", "cv10")]   # four at the paper's batch of 256
-
-
-@pytest.mark.parametrize("layer", TABLE1, ids=lambda l: f"{l.name}-n{l.N}")
-def test_table1_layers_sampled_outputs(layer):
-    """The paper's benchmark layers (Table 1: no padding, strides 1, 2 and 4, 3 to 512 channels) with
-    their per-image geometry and a batch that still gives several waves of tiles: transform bit for
-    bit on the first and last image, convolution on sampled outputs and on the whole last image."""
-    dims = layer.dims()
-    x, f = workloads.make_inputs(layer)
-    ho, wo = oracle.out_dims(dims)
-    total = layer.N * layer.Co * ho * wo
-    rng = np.random.default_rng(layer.seed + 3)
-    idx = np.concatenate([rng.integers(0, total, 2048), [0, total - 1, wo - 1, ho * wo - 1, total - ho * wo]])
+    idx = _sample_indices(total, 65536, layer.seed + 11, [0, total - 1, wo - 1, ho * wo - 1, total - ho * wo])
     for precision in layer.precisions:
         tdt = torch.float32 if precision == "f32" else torch.float16
         raw = x.to(tdt).view(torch.int32 if precision == "f32" else torch.int16)
         got = gpu_transform(raw, dims)
-        for n in (0, layer.N - 1):
-            want = oracle.transform(raw[n:n + 1].numpy(), dict(dims, N=1))
-            assert np.array_equal(got[n:n + 1], want), (layer.name, precision, n)
+        assert np.array_equal(got, oracle.transform(raw.numpy(), dims)), (name, precision)
         del got
         y, _, _ = gpu_conv(x, f, dims, precision)
         xo, fo = oracle_inputs(x, f, precision)
         yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
         check_conv(y.reshape(-1)[idx], yr, ar, precision, layer.name)
-        yi, ai = oracle.conv_im2win(xo[-1:], fo, dict(dims, N=1))
-        check_conv(y[-1:], yi, ai, precision, layer.name + " last image")
+        for n in (0, layer.N - 1):
+            yi, ai = oracle.conv_im2win(xo[n:n + 1], fo, dict(dims, N=1))
+            check_conv(y[n:n + 1], yi, ai, precision, f"{layer.name} image {n}")
+        del y
+
+
+# ------------------------------------------------- the paper's Table 1 layers ----
+TABLE1 = [workloads.TABLE1_LAYERS[k] for k in ("cv1", "cv2", "cv3", "cv5", "cv6", "cv7", "cv8", "cv9", "cv10",
+                                                "cv11", "cv12")]
+
+
+def _table1_check(layer, precisions, samples):
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    ho, wo = oracle.out_dims(dims)
+    total = layer.N * layer.Co * ho * wo
+    idx = _sample_indices(total, samples, layer.seed + 3, [0, total - 1, wo - 1, ho * wo - 1, total - ho * wo])
+    images = (0, layer.N // 2, layer.N - 1)
+    for precision in precisions:
+        tdt = torch.float32 if precision == "f32" else torch.float16
+        raw = x.to(tdt).view(torch.int32 if precision == "f32" else torch.int16)
+        y, wins = gpu_layer_keep_window(x, f, dims, precision, images)
+        for n in images:
+            want = oracle.transform(raw[n:n + 1].numpy(), dict(dims, N=1))
+            assert np.array_equal(wins[n], want), (layer.name, precision, n)
+        del wins
+        xo, fo = oracle_inputs(x, f, precision)
+        yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
+        check_conv(y.reshape(-1)[idx], yr, ar, precision, layer.name)
+        for n in (layer.N // 2, layer.N - 1):
+            yi, ai = oracle.conv_im2win(xo[n:n + 1], fo, dict(dims, N=1))
+            check_conv(y[n:n + 1], yi, ai, precision, f"{layer.name} image {n}")
+        del y, xo
+
+
+@pytest.mark.parametrize("layer", TABLE1, ids=lambda l: l.name)
+def test_table1_layers_at_batch_256(layer):
+    """The paper's benchmark layers (Table 1: no padding, strides 1, 2 and 4, 3 to 512 channels) at
+    the paper's batch of 256, as the benchmark launches them: transform bit for bit on the first,
+    middle and last image, convolution on 16 384 sampled outputs (Eq. 1) and on two whole images."""
+    _table1_check(layer, layer.precisions, 16384)
+
+
+@pytest.mark.parametrize("precision", ["f32", "f16"])
+def test_table1_cv4_at_batch_256(precision):
+    """cv4 at batch 256: the one layer whose window tensor (2.8 G elements, 11.2 GB in fp32) passes
+    2^31 elements, so image bases need 64-bit arithmetic.  65 536 sampled outputs (a quarter of them
+    in images whose window offset exceeds 2^31 elements), the transform of the first, middle and last
+    image and the convolution of the middle and last image whole."""
+    layer = workloads.TABLE1_LAYERS["cv4"]
+    dims = layer.dims()
+    ho, wo = oracle.out_dims(dims)
+    per_image = oracle.window_elems(dict(dims, N=1))
+    assert per_image * (layer.N - 1) > 2 ** 31 and per_image * (layer.N // 2) < 2 ** 31
+    _table1_check(layer, (precision,), 65536)
 
 
 # ------------------------------------------------------------ full-size layers ----
@@ -361,31 +402,24 @@ FULL = [workloads.LAYERS[k] for k in ("cfg2", "cfg3", "cfg4a", "cfg4b", "cfg4c",
 
 
 @pytest.mark.parametrize("layer", FULL, ids=lambda l: l.name)
-def test_full_size_sampled_outputs(layer):
-    """At the benchmark's sizes: the transform is compared bit for bit on whole images, the
-    convolution on 4096 sampled outputs (plus the corners of the output tensor) that the
-    oracle computes one by one from Eq. 1."""
+def test_full_size_whole_tensors(layer):
+    """At the benchmark's sizes and launch configuration: the transform of every image bit for bit
+    and EVERY output element of the convolution within tolerance (the oracle's im2win route over
+    the whole batch), plus 4096 sampled outputs from Eq. 1 as a second route, in both precisions."""
     dims = layer.dims()
     x, f = workloads.make_inputs(layer)
     ho, wo = oracle.out_dims(dims)
     total = layer.N * layer.Co * ho * wo
-    rng = np.random.default_rng(layer.seed)
-    idx = np.concatenate([rng.integers(0, total, 4096), [0, total - 1, wo - 1, ho * wo - 1, total - ho * wo]])
+    idx = _sample_indices(total, 4096, layer.seed, [0, total - 1, wo - 1, ho * wo - 1, total - ho * wo])
     for precision in layer.precisions:
-        # transform: first and last image, bit for bit
         tdt = torch.float32 if precision == "f32" else torch.float16
         raw = x.to(tdt).view(torch.int32 if precision == "f32" else torch.int16)
         got = gpu_transform(raw, dims)
-        for n in (0, layer.N - 1):
-            one = dict(dims, N=1)
-            want = oracle.transform(raw[n:n + 1].numpy(), one)
-            assert np.array_equal(got[n:n + 1], want), (layer.name, precision, n)
+        assert np.array_equal(got, oracle.transform(raw.numpy(), dims)), (layer.name, precision)
         del got
         y, _, _ = gpu_conv(x, f, dims, precision)
         xo, fo = oracle_inputs(x, f, precision)
         yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
         check_conv(y.reshape(-1)[idx], yr, ar, precision, layer.name)
-        # a whole image through the im2win route as well
-        one = dict(dims, N=1)
-        yi, ai = oracle.conv_im2win(xo[-1:], fo, one)
-        check_conv(y[-1:], yi, ai, precision, layer.name + " last image")
+        _whole_conv_check(y, xo, fo, dims, precision, layer.name, 16)
+        del y

@@ -40,6 +40,14 @@ def test_static_scratch_entry_matches_regular_entry_twice_in_a_row():
         rc = lib.im2win_conv_f32_static(window.data_ptr(), fd.data_ptr(), y.data_ptr(), ctypes.byref(shape), stream)
         assert rc == 0, binding.STATUS_NAMES.get(rc, rc)
         torch.cuda.synchronize()
+        # "allocates nothing": once the first call has done its per-device set-up, a call must leave the
+        # device's free memory where it was
+        free_before, _ = torch.cuda.mem_get_info()
+        rc = lib.im2win_conv_f32_static(window.data_ptr(), fd.data_ptr(), y.data_ptr(), ctypes.byref(shape), stream)
+        assert rc == 0, binding.STATUS_NAMES.get(rc, rc)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before, "the allocation-free entry point changed the device's free memory"
         _, a = oracle.conv_direct(x.numpy(), f.numpy(), dims)
         yr, yn = y_ref.cpu().numpy().astype(np.float64), y.cpu().numpy().astype(np.float64)
         assert np.all(np.isfinite(yn))
