@@ -225,6 +225,7 @@ def kernel_rooflines(runner, avg_ms, peaks, peak_kind):
             else:
                 out[name] = {"bound": "tensor", "achieved": tf, "peak": tensor_peak, "unit": "TFLOP/s",
                              "frac": tf / tensor_peak, "peak_kind": peak_kind, "ms": ms, "tflops": tf}
+            out[name]["frac_of_tensor_peak"] = tf / tensor_peak
     return out
 
 
@@ -375,6 +376,11 @@ def run_gpu_arm(args):
         "clocks": clocks,
     }
     if rank == 0:
+        if world == 1 and not args.no_per_layer:
+            # every BASELINE config, call by call (the metric is "per layer"): 20 launches each
+            del runner, e2e_sets
+            torch.cuda.empty_cache()
+            out["per_layer"] = per_layer_summary(layer_rows(peaks, peak_kind, iters=20, with_packed=False))
         if world == 1 and not args.no_cpu_baseline:
             out["cpu_baseline"] = time_cpu_oracle(layer)
         print(json.dumps(out))
@@ -410,7 +416,9 @@ def time_call(fn, iters, flush):
     return total / iters, best, samples[len(samples) // 2]
 
 
-def write_report(path, peaks, peak_kind, names=None, iters=20):
+def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
+    """Times every call of the named layers (default: all BASELINE configs) one by one: transform and
+    convolution (filter pack included) per precision, L2 flushed before each launch."""
     from paper_2608_20725_b200 import binding
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
     rows = []
@@ -426,25 +434,54 @@ def write_report(path, peaks, peak_kind, names=None, iters=20):
         avg, best, median = {}, {}, {}
         for prec in layer.precisions:
             for kind, fn in (("transform", runner.transform), ("conv", runner.conv)):
-                print(f"[report]   {kind}_{prec}", file=sys.stderr, flush=True)
                 key = f"{kind}_{prec}"
                 avg[key], best[key], median[key] = time_call(lambda: fn(prec), iters, flush)
             binding.im2win_check_status(runner.dev[prec]["scratch"])
-        # the convolution kernel without the filter pack (static weights), for reference
-        packed = {}
-        for prec in layer.precisions:
-            a, b_, m = time_call(lambda: runner.conv_packed(prec), iters, flush)
-            packed[f"conv_{prec}"] = {"avg_ms": a, "best_ms": b_, "median_ms": m}
         row = {"layer": name, "dims": layer.dims(), "gflop": runner.flops / 1e9, "avg_ms": avg, "best_ms": best,
-               "median_ms": median, "conv_without_pack": packed,
-               "kernels": kernel_rooflines(runner, avg, peaks, peak_kind), "memory": runner.memory_report()}
+               "median_ms": median, "kernels": kernel_rooflines(runner, avg, peaks, peak_kind),
+               "conv_kernel": {p: binding.im2win_conv_kernel_name(layer.dims(), binding.F32 if p == "f32" else binding.F16)
+                               for p in layer.precisions},
+               "memory": runner.memory_report()}
+        if with_packed:
+            # the convolution kernel without the filter pack (static weights), for reference
+            packed = {}
+            for prec in layer.precisions:
+                a, b_, m = time_call(lambda: runner.conv_packed(prec), iters, flush)
+                packed[f"conv_{prec}"] = {"avg_ms": a, "best_ms": b_, "median_ms": m}
+            row["conv_without_pack"] = packed
         rows.append(row)
         del runner
         torch.cuda.empty_cache()
+    return rows
+
+
+def write_report(path, peaks, peak_kind, names=None, iters=20):
+    rows = layer_rows(peaks, peak_kind, names, iters)
     os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
     with open(path, "w") as fh:
         for row in rows:
             fh.write(json.dumps(row) + "\n")
+
+
+def per_layer_summary(rows):
+    """The per-layer part of the bench line: for every BASELINE config and each of its calls the
+    device time, the bounding roofline and the fraction reached, plus the memory figures."""
+    out = {}
+    for row in rows:
+        entry = {}
+        for key, k in row["kernels"].items():
+            e = {"ms": round(k["ms"], 5), "bound": k["bound"], "frac": round(k["frac"], 4),
+                 "achieved": round(k["achieved"], 2), "unit": k["unit"]}
+            if key.startswith("conv"):
+                e["tflops"] = round(row["gflop"] / k["ms"], 2)      # GFLOP per ms = TFLOP/s
+                e["kernel"] = row["conv_kernel"][key.split("_")[1]]
+                if key == "conv_f16":
+                    e["frac_of_tensor_peak"] = round(k["frac_of_tensor_peak"], 4)
+            entry[key] = e
+        entry["memory"] = {p: {"window_bytes": m["window_bytes"], "output_bytes": m["output_bytes"],
+                               "im2col_bytes": m["im2col_bytes"]} for p, m in row["memory"].items()}
+        out[row["layer"]] = entry
+    return out
 
 
 def run_kernel_loop(spec, launches=3):
@@ -517,6 +554,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--report", default=None, help="also write a per-layer, per-kernel report (JSON lines)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-layer", action="store_true", help="skip the per-layer timings of the default run")
     ap.add_argument("--kernel-loop", default=None, metavar="LAYER:KERNEL[:BATCH]",
                     help="run a few launches of one kernel (e.g. cfg2:conv_f32) and exit; for profilers")
     ap.add_argument("--report-layers", default=None, help="comma-separated layer names for --report")
