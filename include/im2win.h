@@ -194,6 +194,82 @@ im2win_status im2win_layer_forward_host(const void* x_host, const void* filter_h
                                         const im2win_shape* shape, im2win_dtype dtype,
                                         void* cuda_stream);
 
+/* ------------------------------------------------------------------------
+ * Channel-innermost (NHWC) form of the path, fp16 on tensor cores.
+ *
+ * The paper's tensor-core kernel works on NHWC data (Section "Im2win
+ * Convolution on Tensor Cores"); the index map it prints (Eq. 2) is the NCHW
+ * one.  The reading taken here is Eq. 2 with the channel moved to the fastest
+ * position:
+ *     window[n][ho][k][u][c] = Xpad[n][c][ho*s + u][k],
+ *     k in [0, W+2p), u in [0, Kh), c in [0, Cp),  Cp = C rounded up to 8,
+ * channels C..Cp-1 holding +0.  The Kh x Kw x C window of output (ho, wo) is
+ * then the contiguous run of Kw*Kh*Cp elements that starts (wo*s)*Kh*Cp
+ * elements into strip (n, ho), ordered (v, u, c): height before width as in
+ * Eq. 3, the channel below both.  The tensor has N*Ho*(W+2p)*Kh*Cp elements:
+ * the closed-form im2win size when C is a multiple of 8.
+ */
+typedef enum {
+  IM2WIN_LAYOUT_NCHW = 0,   /* [N][C][H][W] */
+  IM2WIN_LAYOUT_NHWC = 1    /* [N][H][W][C] */
+} im2win_layout;
+
+/*
+ * What a convolution does with its finished fp32 accumulator (the last step
+ * of the paper's Algorithm 1, "write C", whose output type the paper leaves
+ * open): y = acc + bias[co] (if bias is not NULL), then max(y, 0) (if relu),
+ * then the store, as binary32 or rounded once to binary16 (nearest, ties to
+ * even), in NCHW or NHWC order.  A NULL epilogue means no bias, no ReLU,
+ * binary32, NCHW.
+ */
+typedef struct {
+  const float* bias;        /* DEVICE pointer to Co floats, or NULL             */
+  int32_t relu;             /* 0 or 1                                           */
+  int32_t out_dtype;        /* IM2WIN_F32 or IM2WIN_F16: element type of y      */
+  int32_t out_layout;       /* im2win_layout of y                               */
+} im2win_epilogue;
+
+/*
+ * Buffer sizes of the NHWC form (host-only): window_bytes = N*Ho*(W+2p)*Kh*Cp*2,
+ * scratch_bytes for im2win_conv_f16_nhwc (status block + repacked filter), the
+ * output size and the stored channel count Cp.  Any output pointer may be NULL.
+ */
+im2win_status im2win_nhwc_workspace_size(const im2win_shape* shape, size_t* window_bytes, size_t* scratch_bytes,
+                                         int32_t* Ho, int32_t* Wo, int32_t* Cp);
+
+/*
+ * im2win transformation into the NHWC window tensor defined above, from an
+ * input of binary16 bit patterns given as [N][C][H][W] or [N][H][W][C]
+ * (`x_layout`).  Bit patterns are copied verbatim; padding positions and the
+ * channels C..Cp-1 are written as +0.
+ */
+im2win_status im2win_transform_nhwc(const uint16_t* x, im2win_layout x_layout, uint16_t* window,
+                                    const im2win_shape* shape, void* cuda_stream);
+
+/*
+ * Forward convolution over the NHWC window tensor on tensor cores (paper
+ * Algorithm 1 in its GEMM view, M x N x K = positions x Co x Kw*Kh*Cp):
+ *     acc[n][ho][wo][co] = sum_{t < Kw*Kh*Cp} window[n][ho][(wo*s)*Kh*Cp + t] * Fp[co][t],
+ *     Fp[co][(v*Kh + u)*Cp + c] = filter_oihw[co][c][u][v]  (0 for c >= C),
+ * fp16 products, fp32 accumulation, then `epilogue` (may be NULL).  `y` holds
+ * N*Co*Ho*Wo elements of epilogue->out_dtype in epilogue->out_layout.  The
+ * filter is repacked into `scratch` on every call.  Layers with few position
+ * tiles split the reduction over several CTAs, which add their partial sums
+ * into a `y` the call clears first (only without ReLU and with binary32
+ * output; the summation order then varies from run to run).  Waits are
+ * bounded as in im2win_conv_f16 (see im2win_check_status).
+ * im2win_pack_filter_nhwc / im2win_conv_packed_nhwc are the two halves for
+ * static weights.
+ */
+im2win_status im2win_conv_f16_nhwc(const uint16_t* window, const uint16_t* filter_oihw, void* y,
+                                   const im2win_epilogue* epilogue, void* scratch, size_t scratch_bytes,
+                                   const im2win_shape* shape, void* cuda_stream);
+im2win_status im2win_pack_filter_nhwc(const uint16_t* filter_oihw, void* scratch, size_t scratch_bytes,
+                                      const im2win_shape* shape, void* cuda_stream);
+im2win_status im2win_conv_packed_nhwc(const uint16_t* window, void* y, const im2win_epilogue* epilogue,
+                                      void* scratch, size_t scratch_bytes, const im2win_shape* shape,
+                                      void* cuda_stream);
+
 /*
  * fp32 convolution without a scratch argument, for callers that cannot allocate
  * device memory (the paper has no counterpart; this is a convenience of this

@@ -26,6 +26,8 @@ EXPORTS = (
     "im2win_status_string", "im2win_workspace_size", "im2win_transform", "im2win_conv_f32", "im2win_conv_f16",
     "im2win_check_status", "im2win_layer_workspace_size", "im2win_layer_forward_host",
     "im2win_conv_f32_static", "im2win_pack_filter", "im2win_conv_packed", "im2win_conv_kernel_name",
+    "im2win_nhwc_workspace_size", "im2win_transform_nhwc", "im2win_conv_f16_nhwc", "im2win_pack_filter_nhwc",
+    "im2win_conv_packed_nhwc",
 )
 
 STATIC_SCRATCH_BYTES = 4 << 20
@@ -33,6 +35,17 @@ STATIC_SCRATCH_BYTES = 4 << 20
 
 class Shape(ctypes.Structure):
     _fields_ = [(k, ctypes.c_int32) for k in ("N", "C", "H", "W", "Co", "Kh", "Kw", "stride", "pad")]
+
+
+NCHW = 0
+NHWC = 1
+
+
+class Epilogue(ctypes.Structure):
+    """im2win_epilogue: bias (device pointer or NULL), relu, out_dtype (F32/F16), out_layout (NCHW/NHWC)."""
+
+    _fields_ = [("bias", ctypes.c_void_p), ("relu", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
+                ("out_layout", ctypes.c_int32)]
 
 
 class Im2winError(RuntimeError):
@@ -67,6 +80,11 @@ def lib() -> ctypes.CDLL:
     L.im2win_pack_filter.argtypes = [vp, vp, sz, P(Shape), ctypes.c_int, vp]
     L.im2win_conv_packed.argtypes = [vp, vp, vp, sz, P(Shape), ctypes.c_int, vp]
     L.im2win_conv_kernel_name.argtypes = [P(Shape), ctypes.c_int]
+    L.im2win_nhwc_workspace_size.argtypes = [P(Shape), P(sz), P(sz), P(i32), P(i32), P(i32)]
+    L.im2win_transform_nhwc.argtypes = [vp, ctypes.c_int, vp, P(Shape), vp]
+    L.im2win_conv_f16_nhwc.argtypes = [vp, vp, vp, P(Epilogue), vp, sz, P(Shape), vp]
+    L.im2win_pack_filter_nhwc.argtypes = [vp, vp, sz, P(Shape), vp]
+    L.im2win_conv_packed_nhwc.argtypes = [vp, vp, P(Epilogue), vp, sz, P(Shape), vp]
     for name in EXPORTS[1:]:
         getattr(L, name).restype = ctypes.c_int
     L.im2win_conv_kernel_name.restype = ctypes.c_char_p
@@ -224,6 +242,78 @@ def im2win_layer_forward_host(x_host: torch.Tensor, filter_host: torch.Tensor, y
                                            device_workspace.numel() * device_workspace.element_size(),
                                            ctypes.byref(s), code, _stream(stream)),
            "im2win_layer_forward_host")
+
+
+# ------------------------------------------------------- channel-innermost (NHWC) form
+def make_epilogue(bias: Optional[torch.Tensor] = None, relu: bool = False, out_dtype: torch.dtype = torch.float32,
+                  out_layout: int = NCHW) -> Epilogue:
+    if bias is not None:
+        assert bias.is_cuda and bias.dtype == torch.float32 and bias.is_contiguous()
+    return Epilogue(None if bias is None else bias.data_ptr(), int(bool(relu)), _dtype_code(out_dtype), int(out_layout))
+
+
+def im2win_nhwc_workspace_size(shape) -> Tuple[int, int, int, int, int]:
+    """Returns (window_bytes, scratch_bytes, Ho, Wo, Cp) of the NHWC form."""
+    s = as_shape(shape)
+    wb, sb = ctypes.c_size_t(), ctypes.c_size_t()
+    ho, wo, cp = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    _check(lib().im2win_nhwc_workspace_size(ctypes.byref(s), ctypes.byref(wb), ctypes.byref(sb), ctypes.byref(ho),
+                                            ctypes.byref(wo), ctypes.byref(cp)), "im2win_nhwc_workspace_size")
+    return wb.value, sb.value, ho.value, wo.value, cp.value
+
+
+def im2win_transform_nhwc(x: torch.Tensor, x_layout: int, window: torch.Tensor, shape, stream=None) -> None:
+    """x (float16, [N,C,H,W] for NCHW or [N,H,W,C] for NHWC) -> NHWC window tensor (flat float16)."""
+    s = as_shape(shape)
+    assert x.is_cuda and window.is_cuda and x.is_contiguous() and window.is_contiguous()
+    assert x.dtype == torch.float16 and window.dtype == torch.float16
+    wb = im2win_nhwc_workspace_size(s)[0]
+    assert x.numel() == s.N * s.C * s.H * s.W and window.numel() * 2 >= wb
+    _check(lib().im2win_transform_nhwc(x.data_ptr(), int(x_layout), window.data_ptr(), ctypes.byref(s), _stream(stream)),
+           "im2win_transform_nhwc")
+
+
+def _epi_ref(epilogue: Optional[Epilogue]):
+    return None if epilogue is None else ctypes.byref(epilogue)
+
+
+def im2win_conv_f16_nhwc(window, filter_oihw, y, scratch, shape, epilogue: Optional[Epilogue] = None, stream=None) -> None:
+    s = as_shape(shape)
+    for t in (window, filter_oihw, y, scratch):
+        assert t.is_cuda and t.is_contiguous()
+    assert window.dtype == torch.float16 and filter_oihw.dtype == torch.float16
+    want = torch.float32 if epilogue is None or epilogue.out_dtype == F32 else torch.float16
+    assert y.dtype == want
+    _check(lib().im2win_conv_f16_nhwc(window.data_ptr(), filter_oihw.data_ptr(), y.data_ptr(), _epi_ref(epilogue),
+                                      scratch.data_ptr(), scratch.numel() * scratch.element_size(), ctypes.byref(s),
+                                      _stream(stream)), "im2win_conv_f16_nhwc")
+
+
+def im2win_pack_filter_nhwc(filter_oihw, scratch, shape, stream=None) -> None:
+    s = as_shape(shape)
+    assert filter_oihw.is_cuda and filter_oihw.is_contiguous() and filter_oihw.dtype == torch.float16 and scratch.is_cuda
+    _check(lib().im2win_pack_filter_nhwc(filter_oihw.data_ptr(), scratch.data_ptr(),
+                                         scratch.numel() * scratch.element_size(), ctypes.byref(s), _stream(stream)),
+           "im2win_pack_filter_nhwc")
+
+
+def im2win_conv_packed_nhwc(window, y, scratch, shape, epilogue: Optional[Epilogue] = None, stream=None) -> None:
+    s = as_shape(shape)
+    assert window.is_cuda and window.dtype == torch.float16 and y.is_cuda and scratch.is_cuda
+    _check(lib().im2win_conv_packed_nhwc(window.data_ptr(), y.data_ptr(), _epi_ref(epilogue), scratch.data_ptr(),
+                                         scratch.numel() * scratch.element_size(), ctypes.byref(s), _stream(stream)),
+           "im2win_conv_packed_nhwc")
+
+
+def alloc_nhwc_buffers(shape, out_dtype: torch.dtype = torch.float32, out_layout: int = NCHW, device="cuda"):
+    """Allocates (window, scratch, y) for one layer of the NHWC form with torch (device memory only)."""
+    s = as_shape(shape)
+    wb, sb, ho, wo, _ = im2win_nhwc_workspace_size(s)
+    window = torch.empty(wb // 2, dtype=torch.float16, device=device)
+    scratch = torch.empty(sb, dtype=torch.uint8, device=device)
+    yshape = (s.N, s.Co, ho, wo) if out_layout == NCHW else (s.N, ho, wo, s.Co)
+    y = torch.empty(yshape, dtype=out_dtype, device=device)
+    return window, scratch, y
 
 
 # ---------------------------------------------------------------- conveniences

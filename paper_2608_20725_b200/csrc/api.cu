@@ -12,6 +12,11 @@ namespace im2win {
 
 static inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 
+const char* debug_getenv(const char* name) {
+  static const bool enabled = getenv("IM2WIN_DEBUG") != nullptr;   // looked up once per process
+  return enabled ? getenv(name) : nullptr;
+}
+
 im2win_status derive_geometry(const im2win_shape* s, Geometry* g) {
   if (!s) return IM2WIN_ERR_NULL_POINTER;
   if (s->N < 1 || s->C < 1 || s->H < 1 || s->W < 1 || s->Co < 1 || s->Kh < 1 || s->Kw < 1 ||
@@ -79,7 +84,7 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
       const int64_t K2p = round_up((int64_t)g.C * g.Kh, kF16KBlock);
       const size_t shift_filter_off = (size_t)round_up((int64_t)kStatusBytes + 4 * K2p, 256);
       const size_t shift_total = (size_t)round_up((int64_t)shift_filter_off + K2p * g.Co * g.Kw * 2, 256);
-      const char* force = getenv("IM2WIN_F16_KERNEL");
+      const char* force = debug_getenv("IM2WIN_F16_KERNEL");
       const bool use_shift = !(force && strcmp(force, "gather") == 0);
       if (use_shift) {
         l->f16_shift = plan.eligible;
@@ -94,7 +99,7 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
     }
     const MatPlan mat = plan_f16_mat(g);
     const MatcPlan matc = mat.eligible ? MatcPlan{} : plan_f16_matc(g);
-    const char* force = getenv("IM2WIN_F16_KERNEL");
+    const char* force = debug_getenv("IM2WIN_F16_KERNEL");
     // measured: the matrix-transpose kernels win for strided layers (the others stage such layers
     // with 2-byte gathers) and for kernels up to 5 wide with 128 output channels or more (CTA pairs
     // above 128); IM2WIN_F16_KERNEL=mat forces them wherever they can run (a testing aid)
@@ -239,6 +244,89 @@ im2win_status im2win_pack_filter(const void* filter_oihw, void* scratch, size_t 
 im2win_status im2win_conv_packed(const void* window, float* y_nchw, void* scratch, size_t scratch_bytes,
                                  const im2win_shape* shape, im2win_dtype dtype, void* cuda_stream) {
   return conv_common(window, nullptr, y_nchw, scratch, scratch_bytes, shape, dtype, cuda_stream, kDoConv);
+}
+
+// ---- channel-innermost (NHWC) form ------------------------------------------------------------
+static im2win_status epilogue_args(const im2win_epilogue* e, bool nhwc_allowed, EpilogueArgs* out) {
+  out->bias = nullptr; out->relu = 0; out->out16 = 0; out->y_nhwc = 0;
+  if (!e) return IM2WIN_OK;
+  if ((e->relu != 0 && e->relu != 1) || (e->out_dtype != IM2WIN_F32 && e->out_dtype != IM2WIN_F16) ||
+      (e->out_layout != IM2WIN_LAYOUT_NCHW && e->out_layout != IM2WIN_LAYOUT_NHWC))
+    return IM2WIN_ERR_INVALID_ARG;
+  if (e->out_layout == IM2WIN_LAYOUT_NHWC && !nhwc_allowed) return IM2WIN_ERR_UNSUPPORTED;
+  if (e->bias && (reinterpret_cast<uintptr_t>(e->bias) & 3u)) return IM2WIN_ERR_MISALIGNED;
+  out->bias = e->bias; out->relu = e->relu; out->out16 = e->out_dtype == IM2WIN_F16;
+  out->y_nhwc = e->out_layout == IM2WIN_LAYOUT_NHWC;
+  return IM2WIN_OK;
+}
+
+static im2win_status nhwc_common(const uint16_t* window, const uint16_t* filter, void* y, const im2win_epilogue* epilogue,
+                                 void* scratch, size_t scratch_bytes, const im2win_shape* shape, void* cuda_stream,
+                                 int mode) {
+  if (!scratch || !shape) return IM2WIN_ERR_NULL_POINTER;
+  if ((mode & kDoPack) && !filter) return IM2WIN_ERR_NULL_POINTER;
+  if ((mode & kDoConv) && (!window || !y)) return IM2WIN_ERR_NULL_POINTER;
+  Geometry g;
+  im2win_status st = derive_geometry(shape, &g);
+  if (st != IM2WIN_OK) return st;
+  const NhwcPlan plan = plan_nhwc(g);
+  if (!plan.eligible) return IM2WIN_ERR_UNSUPPORTED;
+  EpilogueArgs epi;
+  st = epilogue_args(epilogue, true, &epi);
+  if (st != IM2WIN_OK) return st;
+  if (misaligned(scratch) || ((mode & kDoPack) && misaligned(filter)) ||
+      ((mode & kDoConv) && (misaligned(window) || misaligned(y))))
+    return IM2WIN_ERR_MISALIGNED;
+  if (scratch_bytes < plan.scratch_bytes) return IM2WIN_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if ((mode & kDoPack) && launch_pack_f16_nhwc(filter, scratch, g, stream) != cudaSuccess) return IM2WIN_ERR_CUDA;
+  if ((mode & kDoConv) && launch_conv_f16_nhwc(window, y, scratch, g, epi, stream) != cudaSuccess) return IM2WIN_ERR_CUDA;
+  return IM2WIN_OK;
+}
+
+im2win_status im2win_nhwc_workspace_size(const im2win_shape* shape, size_t* window_bytes, size_t* scratch_bytes,
+                                         int32_t* Ho, int32_t* Wo, int32_t* Cp) {
+  Geometry g;
+  im2win_status st = derive_geometry(shape, &g);
+  if (st != IM2WIN_OK) return st;
+  const NhwcPlan plan = plan_nhwc(g);
+  if (!plan.eligible) return IM2WIN_ERR_UNSUPPORTED;
+  if (window_bytes) *window_bytes = (size_t)plan.window_elems * 2;
+  if (scratch_bytes) *scratch_bytes = plan.scratch_bytes;
+  if (Ho) *Ho = g.Ho;
+  if (Wo) *Wo = g.Wo;
+  if (Cp) *Cp = plan.Cp;
+  return IM2WIN_OK;
+}
+
+im2win_status im2win_transform_nhwc(const uint16_t* x, im2win_layout x_layout, uint16_t* window,
+                                    const im2win_shape* shape, void* cuda_stream) {
+  if (!x || !window || !shape) return IM2WIN_ERR_NULL_POINTER;
+  if (x_layout != IM2WIN_LAYOUT_NCHW && x_layout != IM2WIN_LAYOUT_NHWC) return IM2WIN_ERR_INVALID_ARG;
+  Geometry g;
+  im2win_status st = derive_geometry(shape, &g);
+  if (st != IM2WIN_OK) return st;
+  if (!plan_nhwc(g).eligible) return IM2WIN_ERR_UNSUPPORTED;
+  if (misaligned(x) || misaligned(window)) return IM2WIN_ERR_MISALIGNED;
+  cudaError_t e = launch_transform_nhwc(x, x_layout == IM2WIN_LAYOUT_NHWC, window, g, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? IM2WIN_OK : IM2WIN_ERR_CUDA;
+}
+
+im2win_status im2win_conv_f16_nhwc(const uint16_t* window, const uint16_t* filter_oihw, void* y,
+                                   const im2win_epilogue* epilogue, void* scratch, size_t scratch_bytes,
+                                   const im2win_shape* shape, void* cuda_stream) {
+  return nhwc_common(window, filter_oihw, y, epilogue, scratch, scratch_bytes, shape, cuda_stream, kDoPack | kDoConv);
+}
+
+im2win_status im2win_pack_filter_nhwc(const uint16_t* filter_oihw, void* scratch, size_t scratch_bytes,
+                                      const im2win_shape* shape, void* cuda_stream) {
+  return nhwc_common(nullptr, filter_oihw, nullptr, nullptr, scratch, scratch_bytes, shape, cuda_stream, kDoPack);
+}
+
+im2win_status im2win_conv_packed_nhwc(const uint16_t* window, void* y, const im2win_epilogue* epilogue,
+                                      void* scratch, size_t scratch_bytes, const im2win_shape* shape,
+                                      void* cuda_stream) {
+  return nhwc_common(window, nullptr, y, epilogue, scratch, scratch_bytes, shape, cuda_stream, kDoConv);
 }
 
 im2win_status im2win_check_status(const void* scratch, void* cuda_stream) {

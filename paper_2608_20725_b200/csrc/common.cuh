@@ -93,6 +93,35 @@ struct StemPlan {
 };
 StemPlan plan_f16_stem(const Geometry& g);
 
+// Tile geometry of the channel-innermost (NHWC) path (see nhwc.cu).
+struct NhwcPlan {
+  bool eligible;
+  bool pair;               // CTA pairs (cta_group::2)
+  int32_t Cp;              // stored channels: C rounded up to 8
+  int32_t num_kb;          // 64-wide k-blocks of K
+  int32_t tw, bw, G;       // tw tiles of bw output columns along a strip; G strips per tile
+  int32_t bn, ntn;         // channel tile and their number
+  int32_t ksplit, kb_per_split;
+  int64_t K;               // Kw*Kh*Cp
+  int64_t strip;           // Wp*Kh*Cp halves per (n, ho)
+  int64_t window_elems;    // N*Ho*strip
+  int64_t ntm;             // position tiles
+  size_t scratch_bytes;    // status block + packed filter
+};
+NhwcPlan plan_nhwc(const Geometry& g);
+
+// What the convolution does with a finished accumulator (last step of the paper's Algorithm 1).
+struct EpilogueArgs {
+  const float* bias;       // device, Co floats, or nullptr
+  int32_t relu;            // 1: max(y, 0) after the bias
+  int32_t out16;           // 1: store binary16 (round to nearest even), 0: binary32
+  int32_t y_nhwc;          // 1: y is [N][Ho][Wo][Co], 0: [N][Co][Ho][Wo]
+};
+
+// Environment switches are testing aids: they are looked at only when IM2WIN_DEBUG is set in the
+// environment (checked once per process), so the default call path reads no environment.
+const char* debug_getenv(const char* name);
+
 constexpr int kStatusBytes = 256;
 constexpr int kF32KBlock = 16;     // k-block of the fp32 kernel
 constexpr int kF16KBlock = 64;     // k-block of the fp16 kernel (64 halves = one 128-byte swizzle row)
@@ -128,5 +157,11 @@ cudaError_t launch_conv_f16_gather(const uint16_t* window, float* y, void* scrat
                                    const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                   const ScratchLayout& l, cudaStream_t stream);
+
+cudaError_t launch_transform_nhwc(const uint16_t* x, int x_is_nhwc, uint16_t* window, const Geometry& g,
+                                  cudaStream_t stream);
+cudaError_t launch_pack_f16_nhwc(const uint16_t* filter, void* scratch, const Geometry& g, cudaStream_t stream);
+cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch, const Geometry& g,
+                                 const EpilogueArgs& epi, cudaStream_t stream);
 
 }  // namespace im2win

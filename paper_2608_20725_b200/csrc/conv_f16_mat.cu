@@ -931,7 +931,7 @@ cudaError_t launch_conv_f16_mat(const uint16_t* window, float* y, void* scratch,
   unsigned char* base = static_cast<unsigned char*>(scratch);
   uint16_t* fp = reinterpret_cast<uint16_t*>(base + kStatusBytes);
   const int bn = tile_bn(g);
-  const char* pair_env = getenv("IM2WIN_F16_PAIR");     // testing aid: 0 = never pair CTAs
+  const char* pair_env = debug_getenv("IM2WIN_F16_PAIR");     // testing aid: 0 = never pair CTAs
   // measured: pairing pays for 256-channel tiles (the filter tile halves); narrow tiles gain nothing
   const bool pair = bn == 256 && !(pair_env && pair_env[0] == '0');
   const int ncog = (g.Co + 63) / 64;                    // groups of 64 output channels

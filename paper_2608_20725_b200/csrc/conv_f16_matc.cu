@@ -1035,7 +1035,7 @@ MatcPlan plan_f16_matc(const Geometry& g) {
   if ((p.VQ + TILE_M - 1) / TILE_M * ((g.Co + 63) / 64) >= ((int64_t)1 << 31)) return p;
   p.scratch_bytes = (size_t)kStatusBytes + (size_t)p.K2p * ((g.Co + 63) / 64 * 64) * g.Kw * 2;
   int rs, sa, sb, vg, resident, smem;
-  const char* pair_env = getenv("IM2WIN_F16_PAIR");                  // testing aid: 0 = never pair CTAs
+  const char* pair_env = debug_getenv("IM2WIN_F16_PAIR");                  // testing aid: 0 = never pair CTAs
   const bool pairs = !(pair_env && pair_env[0] == '0');
   const int b_rows = (tile_bn(g) == 256 && pairs) ? 128 : tile_bn(g); // 256-channel tiles run as CTA pairs
   if (!choose_rings(tile_bn(g), b_rows, g.Kw, 2, p, &rs, &sa, &sb, &vg, &resident, &smem)) {
@@ -1082,7 +1082,7 @@ cudaError_t launch_conv_f16_matc(const uint16_t* window, float* y, void* scratch
   unsigned char* base = static_cast<unsigned char*>(scratch);
   uint16_t* fp = reinterpret_cast<uint16_t*>(base + kStatusBytes);
   const int bn = tile_bn(g);
-  const char* pair_env = getenv("IM2WIN_F16_PAIR");     // testing aid: 0 = never pair CTAs
+  const char* pair_env = debug_getenv("IM2WIN_F16_PAIR");     // testing aid: 0 = never pair CTAs
   // measured: pairing pays for 256-channel tiles (the filter tile halves); narrow tiles gain nothing
   const bool pair = bn == 256 && !(pair_env && pair_env[0] == '0');
   const int ncog = (g.Co + 63) / 64;                    // groups of 64 output channels

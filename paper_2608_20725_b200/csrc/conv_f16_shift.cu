@@ -436,7 +436,7 @@ cudaError_t launch_variant(const CUtensorMap& fmap, const ShiftParams& q0, const
 // Number of 256-position tiles: whole waves of tall tiles while two units per slot remain, and
 // in the last round as many tall tiles as it takes for the rest to fit in one wave.
 int choose_nbig(int64_t units, int cotiles, int ctas_per_sm, int kw) {
-  const char* force = getenv("IM2WIN_F16_TALL");     // testing aid: 1 = all tall, 0 = none
+  const char* force = debug_getenv("IM2WIN_F16_TALL");     // testing aid: 1 = all tall, 0 = none
   if (force) return atoi(force) ? (int)(units / 2) : 0;
   // Tall tiles halve the filter traffic per flop, which is what bounds wide kernels (measured:
   // +40 % at 11x11, +25 % at 5x5); with three kernel columns the S producers are the bound and

@@ -816,7 +816,7 @@ StemPlan plan_f16_stem(const Geometry& g) {
   }
   // three raw stages by default (measured: eight in flight slow a 3-channel 3x3 layer down from 1.01 ms
   // to 1.27 ms, as a second CTA per SM does); IM2WIN_F16_STEM_RAW = 2..8 sets another depth (a testing aid)
-  const char* force_rs = getenv("IM2WIN_F16_STEM_RAW");
+  const char* force_rs = debug_getenv("IM2WIN_F16_STEM_RAW");
   // (per-strip runs are many small copies: a fourth stage pays there, 273 -> 250 us on the 7x7 stride-2
   // layer with 227-wide strips; with per-image runs it changes nothing or costs, see above)
   const int rs_max = force_rs && atoi(force_rs) >= 2 && atoi(force_rs) <= MAX_RAW ? atoi(force_rs) : (p.ragged ? 4 : 3);
@@ -826,14 +826,14 @@ StemPlan plan_f16_stem(const Geometry& g) {
     used += p.raw_stage_bytes;
   }
 
-  const char* force_sa = getenv("IM2WIN_F16_STEM_STAGES");   // testing aid: S stages / accumulators (2..4)
+  const char* force_sa = debug_getenv("IM2WIN_F16_STEM_STAGES");   // testing aid: S stages / accumulators (2..4)
   if (force_sa && atoi(force_sa) >= 2 && atoi(force_sa) < p.sa) p.sa = atoi(force_sa);
   // Staging buffers of the aligned-store epilogue.  Off by default: measured, the staged path is exact
   // but twice as slow as storing from the registers (cfg3 300 us against 155 us: the two passes through
   // shared memory and the second tensor-memory round trip cost the epilogue warps more than the aligned
   // stores save).  IM2WIN_F16_STEM_EPI=1|2 turns it on with one or two buffers where they fit (tests do).
   p.epi_bufs = 0;
-  const char* want_epi = getenv("IM2WIN_F16_STEM_EPI");
+  const char* want_epi = debug_getenv("IM2WIN_F16_STEM_EPI");
   const int epi_want = want_epi ? atoi(want_epi) : 0;
   if (epi_want >= 2 && used + 2 * EPI_BUF_BYTES <= budget) p.epi_bufs = 2;
   else if (epi_want >= 1 && used + EPI_BUF_BYTES <= budget) p.epi_bufs = 1;
@@ -885,7 +885,7 @@ cudaError_t launch_conv_f16_stem(const uint16_t* window, float* y, void* scratch
   q.cbits = 0;
   while ((1 << q.cbits) < g.C) ++q.cbits;
 
-  const char* generic = getenv("IM2WIN_F16_STEM_GENERIC");   // testing aid: the table-driven re-layout everywhere
+  const char* generic = debug_getenv("IM2WIN_F16_STEM_GENERIC");   // testing aid: the table-driven re-layout everywhere
   int kh = (g.C == 3 && g.Kh == g.Kw && !(generic && atoi(generic))) ? g.Kh : 0;   // the common stems: square kernels on 3 channels
   if (kh != 3 && kh != 5 && kh != 7 && kh != 11) kh = 0;
   void (*kernel)(const CUtensorMap, StemParams);
@@ -902,7 +902,7 @@ cudaError_t launch_conv_f16_stem(const uint16_t* window, float* y, void* scratch
   // persistent CTAs: one per SM (measured: a second CTA per SM, where it fits, only slows the layer
   // down, 1.30 ms against 1.00 ms on a 3-channel 3x3 layer); IM2WIN_F16_STEM_CTAS=2 asks for two (a testing aid)
   int per_sm = 1;
-  const char* force = getenv("IM2WIN_F16_STEM_CTAS");
+  const char* force = debug_getenv("IM2WIN_F16_STEM_CTAS");
   if (force && atoi(force) == 2) {
     per_sm = (kSmemMax + 1024) / (plan.smem_bytes + kStaticSmem + 1024);
     if (per_sm > 512 / q.tmem_cols) per_sm = 512 / q.tmem_cols;

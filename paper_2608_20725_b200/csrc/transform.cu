@@ -359,7 +359,7 @@ bool plan_strips(const Geometry& g, StripParams* q, size_t* smem_bytes, int* vec
   // vector loads: rows must start 16- (or 8-) byte aligned; IM2WIN_TRANSFORM_SCALAR forces the
   // element-wise form (a testing aid)
   *vec = 0;
-  if (getenv("IM2WIN_TRANSFORM_SCALAR") == nullptr && (ES == 2 || g.Kh <= 3)) {   // fp32, Kh > 3: measured slower
+  if (debug_getenv("IM2WIN_TRANSFORM_SCALAR") == nullptr && (ES == 2 || g.Kh <= 3)) {   // fp32, Kh > 3: measured slower
     if ((g.W * ES) % 16 == 0) *vec = 16;
     else if (ES == 2 && (g.W * ES) % 8 == 0) *vec = 8;      // 8-byte vectors of 4-byte elements measured slower
   }
@@ -451,7 +451,7 @@ cudaError_t launch_transform(const void* x, void* window, const Geometry& g, int
                              cudaStream_t stream) {
   // Strips that fit a staging buffer go to the strip kernel; IM2WIN_TRANSFORM_KERNEL=columns
   // forces the fallback (a testing aid).
-  const char* force = getenv("IM2WIN_TRANSFORM_KERNEL");
+  const char* force = debug_getenv("IM2WIN_TRANSFORM_KERNEL");
   const bool columns = force && strcmp(force, "columns") == 0;
   StripParams q;
   size_t smem = 0;

@@ -3,6 +3,11 @@ import sys
 
 import pytest
 
+# The library's environment switches (testing aids that force a kernel or a tile shape) are read
+# only when IM2WIN_DEBUG is set, and the library looks that up once per process: set it before the
+# first call.
+os.environ.setdefault("IM2WIN_DEBUG", "1")
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)

@@ -134,3 +134,69 @@ def check_conv(y_gpu, y_ref, a_ref, precision, what=""):
     with np.errstate(divide="ignore", invalid="ignore"):
         rel = np.where(a_ref > 0, err / a_ref, 0.0)
     return float(rel.max())
+
+
+# ------------------------------------------------------- channel-innermost (NHWC) form ----
+def gpu_transform_nhwc(x_nchw_bits: torch.Tensor, dims: dict, x_layout: str) -> np.ndarray:
+    """x (int16 CPU tensor [N,C,H,W] of binary16 patterns) -> NHWC window tensor [N,Ho,Wp,Kh,Cp] (int16),
+    feeding the library the input in `x_layout` ("nchw" or "nhwc")."""
+    wb, _, ho, _, cp = binding.im2win_nhwc_workspace_size(dims)
+    n = wb // 2
+    whole, win = guarded(n, torch.float16, 7.0)
+    xin = x_nchw_bits if x_layout == "nchw" else x_nchw_bits.permute(0, 2, 3, 1)
+    xd = xin.contiguous().view(torch.float16).cuda()
+    binding.im2win_transform_nhwc(xd, binding.NCHW if x_layout == "nchw" else binding.NHWC, win, dims)
+    torch.cuda.synchronize()
+    assert_guards_intact(whole, n, 7.0)
+    return win.cpu().view(torch.int16).numpy().reshape(dims["N"], ho, dims["W"] + 2 * dims["pad"], dims["Kh"], cp)
+
+
+def gpu_conv_nhwc(x_cpu: torch.Tensor, f_cpu: torch.Tensor, dims: dict, x_layout="nchw", bias=None, relu=False,
+                  out16=False, y_nhwc=False, packed=False):
+    """NHWC transform + convolution through the C ABI with guard bands.  Returns y as a float64 numpy
+    array in the requested layout ([N,Co,Ho,Wo] or [N,Ho,Wo,Co])."""
+    xh = x_cpu.half()
+    xin = xh if x_layout == "nchw" else xh.permute(0, 2, 3, 1)
+    xd = xin.contiguous().cuda()
+    fd = f_cpu.half().cuda().contiguous()
+    wb, sb, ho, wo, _ = binding.im2win_nhwc_workspace_size(dims)
+    nout = dims["N"] * dims["Co"] * ho * wo
+    odt = torch.float16 if out16 else torch.float32
+    wwhole, win = guarded(wb // 2, torch.float16, 3.0)
+    ywhole, y = guarded(nout, odt, -123.0)
+    swhole, scratch = guarded(sb, torch.uint8, 0x5a)
+    bd = None if bias is None else torch.as_tensor(bias, dtype=torch.float32).cuda().contiguous()
+    epi = binding.make_epilogue(bd, relu, odt, binding.NHWC if y_nhwc else binding.NCHW)
+    binding.im2win_transform_nhwc(xd, binding.NCHW if x_layout == "nchw" else binding.NHWC, win, dims)
+    if packed:
+        binding.im2win_pack_filter_nhwc(fd, scratch, dims)
+        binding.im2win_conv_packed_nhwc(win, y, scratch, dims, epi)
+    else:
+        binding.im2win_conv_f16_nhwc(win, fd, y, scratch, dims, epi)
+    binding.im2win_check_status(scratch)
+    assert_guards_intact(wwhole, wb // 2, 3.0)
+    assert_guards_intact(ywhole, nout, -123.0)
+    assert_guards_intact(swhole, sb, 0x5a)
+    shape = (dims["N"], ho, wo, dims["Co"]) if y_nhwc else (dims["N"], dims["Co"], ho, wo)
+    return y.cpu().double().numpy().reshape(shape)
+
+
+def half_ulp_spacing(v: np.ndarray) -> np.ndarray:
+    """Spacing of binary16 numbers at |v| (2^-24 in the subnormal range)."""
+    with np.errstate(over="ignore"):
+        h = np.minimum(np.abs(v), 65504.0).astype(np.float16)
+    return np.spacing(h).astype(np.float64)
+
+
+def check_fused(y_gpu, y_ref, a_ref, out16, what=""):
+    """|gpu - oracle| <= 2e-3 * (sum|x||w| + |bias|) (+ one binary16 spacing at |y| when the store is
+    binary16), y_ref being the oracle's value BEFORE the store rounding; exact zeros where nothing
+    contributes."""
+    err = np.abs(y_gpu - y_ref)
+    bound = TOL_F16 * a_ref + (half_ulp_spacing(y_ref) if out16 else 0.0)
+    bad = err > bound
+    if bad.any():
+        i = np.unravel_index(np.argmax(err - bound), err.shape)
+        raise AssertionError(f"{what}: {bad.sum()} of {bad.size} outputs out of tolerance; worst at {i}: "
+                             f"gpu={y_gpu[i]!r} oracle={y_ref[i]!r} err={err[i]:.3e} bound={bound[i]:.3e}")
+    assert np.all(y_gpu[a_ref == 0] == 0), f"{what}: outputs with no non-zero term must be exactly 0"

@@ -1,0 +1,177 @@
+"""Parity of the channel-innermost (NHWC) form of the path with the CPU oracle: transform bit for
+bit, convolution (tensor cores, TMA-fed) within the fp16 tolerance, every epilogue option, every
+tile shape the library can be made to take, and the benchmark's deep layers whole."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_20725_b200 import binding, workloads
+from paper_2608_20725_b200.workloads import Layer
+from gpu_helpers import check_conv, check_fused, gpu_conv_nhwc, gpu_transform_nhwc, oracle_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def L(name, N, C, H, W, Co, Kh, Kw, s, p, seed=0, xd="normal01", fd="he_normal"):
+    return Layer(name, N, C, H, W, Co, Kh, Kw, s, p, seed, xd, fd)
+
+
+SMALL = [
+    L("tail_pos", 3, 5, 13, 11, 7, 3, 3, 1, 1, 11),             # C = 5 -> 8 stored channels, ragged tiles
+    L("c8", 2, 8, 12, 12, 72, 3, 3, 1, 1, 13),
+    L("k_tail", 2, 24, 9, 10, 24, 3, 3, 1, 1, 36),              # K = 216: last k-block 24 wide
+    L("co_300", 1, 8, 10, 10, 300, 3, 3, 1, 1, 14),             # Co = 300: two channel tiles, CTA pairs, one ragged
+    L("rect", 2, 4, 9, 14, 10, 2, 5, 1, 2, 15),                 # Kh != Kw
+    L("rect2", 2, 4, 14, 9, 10, 5, 2, 2, 0, 16),
+    L("stride3", 2, 6, 17, 19, 12, 3, 3, 3, 1, 17),
+    L("one_by_one", 3, 40, 7, 7, 33, 1, 1, 1, 0, 18),
+    L("k11", 1, 6, 30, 30, 20, 11, 11, 1, 5, 19),
+    L("k5s2", 2, 10, 21, 21, 24, 5, 5, 2, 2, 20),
+    L("single_out", 1, 3, 3, 3, 2, 3, 3, 1, 0, 21),             # Ho = Wo = 1: 128 strips per tile
+    L("deep", 2, 130, 7, 7, 140, 3, 3, 1, 1, 22),               # K = 1224: 20 k-blocks (K split eligible)
+    L("wide_row", 1, 2, 4, 300, 5, 3, 3, 1, 1, 23),             # one output row longer than a tile: 3 tiles per strip
+    L("uncovered_cols", 1, 3, 10, 12, 4, 3, 4, 3, 0, 24),
+    L("pair_odd", 3, 16, 18, 22, 260, 3, 3, 1, 1, 25),          # odd number of position tiles with CTA pairs
+    L("pair_s2", 2, 24, 16, 14, 200, 3, 3, 2, 1, 26),
+    L("stem7", 2, 3, 37, 37, 64, 7, 7, 2, 3, 12),
+    L("many_kb", 1, 64, 9, 9, 40, 5, 5, 1, 2, 27),              # 25 k-blocks: the stage ring wraps several times
+]
+
+
+@pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
+@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
+def test_transform_nhwc_bit_exact(layer, layout):
+    dims = layer.dims()
+    x, _ = workloads.make_inputs(layer)
+    raw = x.half().view(torch.int16)
+    got = gpu_transform_nhwc(raw, dims, layout)
+    cp = got.shape[-1]
+    want = oracle.transform_nhwc(raw.numpy(), dims, "nchw", cp)
+    assert cp == (layer.C + 7) // 8 * 8 and got.shape == want.shape
+    assert np.array_equal(got, want)
+
+
+def test_transform_nhwc_preserves_special_bit_patterns():
+    layer = L("bits", 2, 11, 9, 10, 1, 3, 3, 2, 2, 30)
+    dims = layer.dims()
+    g = torch.Generator().manual_seed(31)
+    raw = torch.randint(-2 ** 15, 2 ** 15 - 1, (2, 11, 9, 10), generator=g, dtype=torch.int64).to(torch.int16)
+    raw.view(-1)[:3] = torch.tensor([0x7e01, -2 ** 15, -1], dtype=torch.int64).to(torch.int16)
+    for layout in ("nchw", "nhwc"):
+        assert np.array_equal(gpu_transform_nhwc(raw, dims, layout), oracle.transform_nhwc(raw.numpy(), dims, "nchw", 16))
+
+
+def _reference(x, f, dims, bias=None, relu=False, out16=False, y_nhwc=False):
+    xo, fo = oracle_inputs(x, f, "f16")
+    y, a = oracle.conv_direct(xo, fo, dims)
+    # the value before the store rounding, and the rounded one
+    y_pre, a2 = oracle.epilogue(y, a, dims, bias=bias, relu=relu, out16=False, nhwc=y_nhwc)
+    y_post, _ = oracle.epilogue(y, a, dims, bias=bias, relu=relu, out16=out16, nhwc=y_nhwc)
+    return y_pre, y_post, a2
+
+
+@pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
+@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
+def test_conv_nhwc_parity_small(layer, layout):
+    """Plain epilogue (fp32, NCHW out) from either input layout."""
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    y = gpu_conv_nhwc(x, f, dims, x_layout=layout)
+    y_pre, _, a = _reference(x, f, dims)
+    check_conv(y, y_pre, a, "f16", layer.name)
+
+
+@pytest.mark.parametrize("layer", [SMALL[0], SMALL[2], SMALL[3], SMALL[7], SMALL[11], SMALL[14]], ids=lambda l: l.name)
+@pytest.mark.parametrize("bn,pair,ksplit", [("64", "0", "1"), ("128", "0", "1"), ("128", "1", "1"), ("256", "0", "1"),
+                                            ("256", "1", "1"), ("128", "0", "3"), ("256", "1", "2"), ("64", "0", "20")])
+def test_conv_nhwc_exact_on_integer_inputs_every_tile_shape(layer, bn, pair, ksplit, monkeypatch):
+    """Integer-valued inputs (order-independent sums) through every tile width, with and without CTA
+    pairs, with K split over several CTAs (partial sums added with red.global.add.f32)."""
+    monkeypatch.setenv("IM2WIN_NHWC_BN", bn)
+    monkeypatch.setenv("IM2WIN_NHWC_PAIR", pair)
+    monkeypatch.setenv("IM2WIN_NHWC_KSPLIT", ksplit)
+    dims = layer.dims()
+    x, f = workloads.make_small_integer_inputs(layer)
+    yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+    for y_nhwc in (False, True):
+        y = gpu_conv_nhwc(x, f, dims, y_nhwc=y_nhwc)
+        assert np.array_equal(y, yr.transpose(0, 2, 3, 1) if y_nhwc else yr), (layer.name, y_nhwc)
+
+
+@pytest.mark.parametrize("layer", [SMALL[1], SMALL[3], SMALL[6], SMALL[9], SMALL[11]], ids=lambda l: l.name)
+@pytest.mark.parametrize("out16", [False, True])
+@pytest.mark.parametrize("y_nhwc", [False, True])
+@pytest.mark.parametrize("bias,relu", [(False, False), (True, False), (False, True), (True, True)])
+def test_conv_nhwc_epilogue_options(layer, out16, y_nhwc, bias, relu):
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    b = None
+    if bias:
+        b = torch.randn(layer.Co, generator=torch.Generator().manual_seed(layer.seed + 5)).numpy() * 0.5
+    y = gpu_conv_nhwc(x, f, dims, bias=b, relu=relu, out16=out16, y_nhwc=y_nhwc, packed=bias and relu)
+    y_pre, y_post, a = _reference(x, f, dims, b, relu, out16, y_nhwc)
+    check_fused(y, y_pre, a, out16, f"{layer.name} out16={out16} nhwc={y_nhwc} bias={bias} relu={relu}")
+    if relu:
+        assert np.all(y >= 0)
+    if out16:
+        # the stored value is a binary16 number within one spacing of the oracle's own rounding
+        assert np.array_equal(y, y.astype(np.float16).astype(np.float64))
+
+
+def test_conv_nhwc_exact_with_integer_bias_relu_and_half_store():
+    """Small integers all the way: bias, ReLU and the binary16 store must reproduce the oracle exactly."""
+    layer = SMALL[2]
+    dims = layer.dims()
+    x, f = workloads.make_small_integer_inputs(layer)
+    b = np.arange(layer.Co, dtype=np.float32) - 10.0
+    y, a = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+    for y_nhwc in (False, True):
+        want, _ = oracle.epilogue(y, a, dims, bias=b, relu=True, out16=True, nhwc=y_nhwc)
+        got = gpu_conv_nhwc(x, f, dims, bias=b, relu=True, out16=True, y_nhwc=y_nhwc)
+        assert np.abs(want).max() < 2048 and np.array_equal(got, want)
+
+
+def test_nhwc_argument_errors_come_before_any_launch():
+    lib = binding.lib()
+    import ctypes
+    s = binding.as_shape(SMALL[1].dims())
+    e = binding.Epilogue(None, 2, 0, 0)
+    assert lib.im2win_conv_f16_nhwc(ctypes.c_void_p(256), ctypes.c_void_p(512), ctypes.c_void_p(1024), ctypes.byref(e),
+                                    ctypes.c_void_p(2048), 1 << 30, ctypes.byref(s), None) == 1
+    e = binding.Epilogue(None, 0, 5, 0)
+    assert lib.im2win_conv_f16_nhwc(ctypes.c_void_p(256), ctypes.c_void_p(512), ctypes.c_void_p(1024), ctypes.byref(e),
+                                    ctypes.c_void_p(2048), 1 << 30, ctypes.byref(s), None) == 1
+    assert lib.im2win_conv_f16_nhwc(None, ctypes.c_void_p(512), ctypes.c_void_p(1024), None,
+                                    ctypes.c_void_p(2048), 1 << 30, ctypes.byref(s), None) == 2
+    assert lib.im2win_conv_f16_nhwc(ctypes.c_void_p(256), ctypes.c_void_p(512), ctypes.c_void_p(1028), None,
+                                    ctypes.c_void_p(2048), 1 << 30, ctypes.byref(s), None) == 3
+    assert lib.im2win_conv_f16_nhwc(ctypes.c_void_p(256), ctypes.c_void_p(512), ctypes.c_void_p(1024), None,
+                                    ctypes.c_void_p(2048), 16, ctypes.byref(s), None) == 4
+    assert lib.im2win_transform_nhwc(ctypes.c_void_p(256), 7, ctypes.c_void_p(512), ctypes.byref(s), None) == 1
+
+
+FULL = [workloads.LAYERS[k] for k in ("cfg2", "cfg3", "cfg4a", "cfg4b", "cfg4c", "cfg5k1", "cfg5k3", "cfg5k5")]
+
+
+@pytest.mark.parametrize("layer", FULL, ids=lambda l: l.name)
+def test_nhwc_full_size_whole_tensors(layer):
+    """At the benchmark's sizes and launch configuration: the NHWC transform of every image bit for
+    bit and EVERY output element of the convolution within tolerance, plus 4096 outputs from Eq. 1."""
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    ho, wo = oracle.out_dims(dims)
+    raw = x.half().view(torch.int16)
+    got = gpu_transform_nhwc(raw, dims, "nchw")
+    assert np.array_equal(got, oracle.transform_nhwc(raw.numpy(), dims, "nchw", got.shape[-1]))
+    del got
+    y = gpu_conv_nhwc(x, f, dims)
+    xo, fo = oracle_inputs(x, f, "f16")
+    total = layer.N * layer.Co * ho * wo
+    idx = np.concatenate([np.random.default_rng(layer.seed).integers(0, total, 4096), [0, total - 1]])
+    yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
+    check_conv(y.reshape(-1)[idx], yr, ar, "f16", layer.name)
+    for n0 in range(0, layer.N, 16):
+        n1 = min(layer.N, n0 + 16)
+        yi, ai = oracle.conv_im2win(xo[n0:n1], fo, dict(dims, N=n1 - n0))
+        check_conv(y[n0:n1], yi, ai, "f16", f"{layer.name} images {n0}..{n1 - 1}")
