@@ -144,6 +144,28 @@ class LayerRunner:
         _, _, self.ho, self.wo = binding.im2win_workspace_size(self.dims, code)
         self.flops = layer_flops(layer, self.ho, self.wo)
         self.precisions = precisions
+        self.nhwc = None
+
+    def add_nhwc(self):
+        """Buffers of the channel-innermost (NHWC) form of the fp16 path: same NCHW input and OIHW
+        filter, NHWC window tensor, fp32 NCHW output."""
+        b = self.b
+        x, f = workloads.make_inputs(self.layer)
+        window, scratch, y = b.alloc_nhwc_buffers(self.dims)
+        self.nhwc = dict(x=x.half().cuda(), f=f.half().cuda(), window=window, scratch=scratch, y=y,
+                         cp=b.im2win_nhwc_workspace_size(self.dims)[4])
+
+    def transform_nhwc(self, prec=None):
+        d = self.nhwc
+        self.b.im2win_transform_nhwc(d["x"], self.b.NCHW, d["window"], self.dims)
+
+    def conv_nhwc(self, prec=None):
+        d = self.nhwc
+        self.b.im2win_conv_f16_nhwc(d["window"], d["f"], d["y"], d["scratch"], self.dims)
+
+    def conv_nhwc_packed(self, prec=None):
+        d = self.nhwc
+        self.b.im2win_conv_packed_nhwc(d["window"], d["y"], d["scratch"], self.dims)
 
     def transform(self, prec):
         d = self.dev[prec]
@@ -178,7 +200,8 @@ class LayerRunner:
         """Bytes each kernel must move once: input + window for a transform, window + output (+ filter) for a convolution."""
         l, es = self.layer, (4 if kernel.endswith("f32") else 2)
         x_el = l.N * l.C * l.H * l.W
-        win_el = l.N * l.C * self.ho * l.Kh * (l.W + 2 * l.pad)
+        chans = self.nhwc["cp"] if kernel.endswith("nhwc") else l.C        # the NHWC form stores C rounded up to 8
+        win_el = l.N * chans * self.ho * l.Kh * (l.W + 2 * l.pad)
         out_el = l.N * l.Co * self.ho * self.wo
         f_el = l.Co * l.C * l.Kh * l.Kw
         if kernel.startswith("transform"):
@@ -437,6 +460,15 @@ def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
                 key = f"{kind}_{prec}"
                 avg[key], best[key], median[key] = time_call(lambda: fn(prec), iters, flush)
             binding.im2win_check_status(runner.dev[prec]["scratch"])
+        if "f16" in layer.precisions:
+            # the channel-innermost (NHWC) form of the fp16 path on the same layer
+            runner.add_nhwc()
+            for _ in range(3):
+                runner.transform_nhwc()
+                runner.conv_nhwc()
+            for key, fn in (("transform_f16_nhwc", runner.transform_nhwc), ("conv_f16_nhwc", runner.conv_nhwc)):
+                avg[key], best[key], median[key] = time_call(fn, iters, flush)
+            binding.im2win_check_status(runner.nhwc["scratch"])
         row = {"layer": name, "dims": layer.dims(), "gflop": runner.flops / 1e9, "avg_ms": avg, "best_ms": best,
                "median_ms": median, "kernels": kernel_rooflines(runner, avg, peaks, peak_kind),
                "conv_kernel": {p: binding.im2win_conv_kernel_name(layer.dims(), binding.F32 if p == "f32" else binding.F16)
@@ -448,6 +480,9 @@ def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
             for prec in layer.precisions:
                 a, b_, m = time_call(lambda: runner.conv_packed(prec), iters, flush)
                 packed[f"conv_{prec}"] = {"avg_ms": a, "best_ms": b_, "median_ms": m}
+            if runner.nhwc is not None:
+                a, b_, m = time_call(runner.conv_nhwc_packed, iters, flush)
+                packed["conv_f16_nhwc"] = {"avg_ms": a, "best_ms": b_, "median_ms": m}
             row["conv_without_pack"] = packed
         rows.append(row)
         del runner
@@ -474,8 +509,8 @@ def per_layer_summary(rows):
                  "achieved": round(k["achieved"], 2), "unit": k["unit"]}
             if key.startswith("conv"):
                 e["tflops"] = round(row["gflop"] / k["ms"], 2)      # GFLOP per ms = TFLOP/s
-                e["kernel"] = row["conv_kernel"][key.split("_")[1]]
-                if key == "conv_f16":
+                e["kernel"] = "f16-nhwc-tma" if key.endswith("nhwc") else row["conv_kernel"][key.split("_")[1]]
+                if key.startswith("conv_f16"):
                     e["frac_of_tensor_peak"] = round(k["frac_of_tensor_peak"], 4)
             entry[key] = e
         entry["memory"] = {p: {"window_bytes": m["window_bytes"], "output_bytes": m["output_bytes"],
@@ -490,9 +525,20 @@ def run_kernel_loop(spec, launches=3):
     table = dict(workloads.LAYERS)
     table.update(workloads.TABLE1_LAYERS)
     layer = table[parts[0]]
-    kind, prec = parts[1].rsplit("_", 1)
     if len(parts) > 2:
         layer = layer.with_batch(int(parts[2]))
+    if parts[1].endswith("_nhwc"):
+        # the channel-innermost form: transform_f16_nhwc | conv_f16_nhwc
+        runner = LayerRunner(layer, ("f16",))
+        runner.add_nhwc()
+        runner.transform_nhwc()
+        fn = runner.transform_nhwc if parts[1].startswith("transform") else runner.conv_nhwc
+        for _ in range(launches):
+            fn()
+        runner.b.im2win_check_status(runner.nhwc["scratch"])
+        print(f"kernel-loop {spec}: {launches} launches done")
+        return
+    kind, prec = parts[1].rsplit("_", 1)
     runner = LayerRunner(layer, (prec,))
     runner.transform(prec)
     fn = runner.transform if kind == "transform" else runner.conv

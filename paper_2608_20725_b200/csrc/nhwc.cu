@@ -35,7 +35,8 @@ using namespace ptx;
 constexpr int TILE_M = 128;
 constexpr int KB = kF16KBlock;                 // 64 halves = one 128-byte swizzle row
 constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_EPI0 = 2;
-constexpr int NUM_WARPS = 6;
+constexpr int EPI_WARPS = 8;                   // two per tensor-memory lane quadrant: each takes half of the tile's channels
+constexpr int NUM_WARPS = 2 + EPI_WARPS;
 constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr int MAX_STAGES = 8;
 constexpr int A_SLOT_BYTES = TILE_M * KB * 2;  // 16 KB: room for 128 rows even when a tile holds fewer
@@ -49,13 +50,20 @@ struct NhwcParams {
   int32_t Ho, Wo, Co, HoWo;
   int32_t rows_total;        // N*Ho strips
   int32_t bw, G, tw;         // tile = G strips x bw output columns; tw tiles along a strip
-  int32_t num_kb;            // 64-wide k-blocks
-  int32_t nks_last;          // 16-wide MMA steps of the last k-block
-  int32_t ksplit, kb_per_split;
+  int32_t num_kc;            // chunks of KSUB 64-wide k-blocks (one ring stage each)
+  int32_t nks_last;          // 16-wide MMA steps of the last chunk
+  int32_t ksplit, kc_per_split;
   int32_t ntn, nwork;        // channel tiles; work items = position tiles (pairs) x channel tiles x k parts
   int32_t stages;
   uint32_t a_bytes;          // bytes one activation copy brings: G*bw*128
+  int32_t dbg_skip;
 };
+
+// Programmatic dependent launch: the convolution may start while the kernel before it in the stream
+// (the filter pack) is still running, so that its barrier set-up, tensor-memory allocation and
+// descriptor fetches overlap that kernel; every role that touches global memory first waits for the
+// preceding kernel to have completed.
+__device__ __forceinline__ void wait_for_previous_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ void red_add_f32(float* p, float v) {
   asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
@@ -115,11 +123,12 @@ __device__ __forceinline__ void store_chunk(const NhwcParams& q, int64_t base, i
   }
 }
 
-template <int BN, bool PAIR>
+template <int BN, bool PAIR, int KSUB>
 __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CUtensorMap& bmap, const NhwcParams& q) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;              // filter rows (output channels) this CTA stages
   constexpr uint32_t B_BYTES = (uint32_t)B_ROWS * KB * 2;
-  constexpr uint32_t STAGE_BYTES = (uint32_t)A_SLOT_BYTES + B_BYTES;     // a multiple of 1024
+  constexpr uint32_t SUB_BYTES = (uint32_t)A_SLOT_BYTES + B_BYTES;       // one 64-wide k-block of both operands
+  constexpr uint32_t STAGE_BYTES = KSUB * SUB_BYTES;                     // a multiple of 1024
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
   const int w_first = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int w_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
@@ -146,7 +155,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(acc_full0 + 8 * i, 1);
-      mbar_init(acc_empty0 + 8 * i, PAIR ? 8 : 4);        // the four epilogue warps (of each CTA)
+      mbar_init(acc_empty0 + 8 * i, PAIR ? 2 * EPI_WARPS : EPI_WARPS);   // the epilogue warps (of each CTA)
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -163,104 +172,126 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
   const uint32_t acc_empty_dst = PAIR ? mapa_shared(acc_empty0, 0) : acc_empty0;
 
   // work item w -> (position tile (pair) mt, channel tile nt, k part ks), nt and ks fastest so that
-  // the CTAs that share an activation tile run at the same time
+  // the CTAs that share an activation tile run at the same time.  K is walked in chunks of KSUB
+  // 64-wide k-blocks: one ring stage, one pair of barrier operations per chunk.
   const int per_mt = q.ntn * q.ksplit;
 
   if (warp == WARP_TMA) {
     // ---------------- copies of both operands ------------------------------------
-    const bool leader = elect_one();
-    bool ok = true;
-    int st = 0;
-    uint32_t ph = 0;
-    for (int w = w_first; w < q.nwork && ok; w += w_step) {
-      const int mt = w / per_mt, rem = w - mt * per_mt;
-      const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
-      const int mti = PAIR ? 2 * mt + (int)rank : mt;
-      const int rg = mti / q.tw, wt = mti - rg * q.tw;
-      const int z = rg * q.G, yc = wt * q.bw;
-      const int brow = nt * BN + (int)rank * B_ROWS;
-      const int kb0 = ks * q.kb_per_split;
-      const int kb1 = kb0 + q.kb_per_split < q.num_kb ? kb0 + q.kb_per_split : q.num_kb;
-      for (int kb = kb0; kb < kb1; ++kb) {
-        ok = mbar_wait(empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (leader) {
-          const uint32_t a_dst = ring + (uint32_t)st * STAGE_BYTES;
-          const uint32_t b_dst = a_dst + (uint32_t)A_SLOT_BYTES;
-          if (PAIR) {
-            // the leader CTA announces the bytes of both CTAs; every copy reports to its barrier
-            if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, 2u * (q.a_bytes + B_BYTES));
-            tma_load_3d_pair(a_dst, &amap, kb * KB, yc, z, full_dst + 8 * st);
-            tma_load_2d_pair(b_dst, &bmap, kb * KB, brow, full_dst + 8 * st);
-          } else {
-            mbar_arrive_expect_tx(full0 + 8 * st, q.a_bytes + B_BYTES);
-            tma_load_3d(a_dst, &amap, kb * KB, yc, z, full0 + 8 * st);
-            tma_load_2d(b_dst, &bmap, kb * KB, brow, full0 + 8 * st);
+    // Lane 0 polls and issues; the warp meets again after the loop.
+    if (lane == 0) {
+      wait_for_previous_kernel();                // the filter pack (and everything before it) is complete
+      int st = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      TIMER_DECL;
+      for (int w = w_first; w < q.nwork && ok; w += w_step) {
+        const int mt = w / per_mt, rem = w - mt * per_mt;
+        const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
+        const int mti = PAIR ? 2 * mt + (int)rank : mt;
+        const int rg = mti / q.tw, wt = mti - rg * q.tw;
+        const int z = rg * q.G, yc = wt * q.bw;
+        const int brow = nt * BN + (int)rank * B_ROWS;
+        const int kc0 = ks * q.kc_per_split;
+        const int kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
+        for (int kc = kc0; kc < kc1; ++kc) {
+          TIMER_LAP(0);                              // copy thread: issuing
+          ok = mbar_wait(empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+          if (!ok) break;
+          TIMER_LAP(1);                              // copy thread: wait for a free stage
+          const uint32_t dst = ring + (uint32_t)st * STAGE_BYTES;
+          const uint32_t bar = full_dst + 8 * st;
+          // k-blocks beyond K read as zeros (and cost no memory traffic), so every stage brings the
+          // same number of bytes.  In a pair the leader CTA announces the bytes of both CTAs.
+          const uint32_t abytes = (q.dbg_skip & 1) ? 0u : q.a_bytes, bbytes = (q.dbg_skip & 2) ? 0u : B_BYTES;
+          if (!PAIR || rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, (PAIR ? 2u : 1u) * KSUB * (abytes + bbytes));
+#pragma unroll
+          for (int sub = 0; sub < KSUB; ++sub) {
+            const int kx = (kc * KSUB + sub) * KB;
+            if (PAIR) {
+              if (abytes) tma_load_3d_pair(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
+              if (bbytes) tma_load_2d_pair(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
+            } else {
+              if (abytes) tma_load_3d(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
+              if (bbytes) tma_load_2d(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
+            }
           }
+          if (++st == q.stages) { st = 0; ph ^= 1u; }
         }
-        __syncwarp();
-        if (++st == q.stages) { st = 0; ph ^= 1u; }
       }
+      if (blockIdx.x == 0) { TIMER_LAP(0); TIMER_FLUSH(); }
     }
+    __syncwarp();
   } else if (warp == WARP_MMA && rank == 0) {
     // ---------------- MMA issuer (leader CTA of a pair) -----------------------------
+    // One thread runs the whole loop: waits, MMAs and commits are all single-thread operations.
+    // Every byte the MMAs read was written by the copy engine, whose completion the barrier's
+    // transaction count tracks, so CTA-scope waits suffice also for the peer's half.
     constexpr uint32_t idesc = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN);
-    const bool leader = elect_one();
-    bool ok = true;
-    int st = 0;
-    uint32_t ph = 0, it = 0;
-    for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
-      const int rem = w % per_mt;
-      const int ks = rem % q.ksplit;
-      const int kb0 = ks * q.kb_per_split;
-      const int kb1 = kb0 + q.kb_per_split < q.num_kb ? kb0 + q.kb_per_split : q.num_kb;
-      const uint32_t buf = it & 1u;
-      ok = PAIR ? mbar_wait_cluster(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status)
-                : mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t acc = tmem_acc + buf * (uint32_t)BN;
-      uint32_t accumulate = 0;
-      for (int kb = kb0; kb < kb1; ++kb) {
-        ok = PAIR ? mbar_wait_cluster(full0 + 8 * st, ph, &abort_flag, q.status)
-                  : mbar_wait(full0 + 8 * st, ph, &abort_flag, q.status);
-        ok = __all_sync(0xffffffffu, ok);
+    if (lane == 0) {
+      int st = 0;
+      uint32_t ph = 0, it = 0;
+      bool ok = true;
+      const uint32_t a_lo0 = smem_desc_lo(ring), b_lo0 = smem_desc_lo(ring + (uint32_t)A_SLOT_BYTES);
+      TIMER_DECL;
+      for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
+        const int rem = w % per_mt;
+        const int ks = rem % q.ksplit;
+        const int kc0 = ks * q.kc_per_split;
+        const int kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
+        const uint32_t buf = it & 1u;
+        TIMER_LAP(2);                                // MMA thread: issue and bookkeeping
+        ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
         if (!ok) break;
+        TIMER_LAP(3);                                // MMA thread: wait for a free accumulator
         tc_fence_after();
-        if (leader) {
-          const uint32_t a_lo = smem_desc_lo(ring + (uint32_t)st * STAGE_BYTES);
-          const uint32_t b_lo = smem_desc_lo(ring + (uint32_t)st * STAGE_BYTES + (uint32_t)A_SLOT_BYTES);
-          const int nks = kb == q.num_kb - 1 ? q.nks_last : KB / 16;
+        const uint32_t acc = tmem_acc + buf * (uint32_t)BN;
+        uint32_t accumulate = 0;
+        for (int kc = kc0; kc < kc1; ++kc) {
+          TIMER_LAP(2);
+          ok = mbar_wait(full0 + 8 * st, ph, &abort_flag, q.status);
+          if (!ok) break;
+          TIMER_LAP(4);                              // MMA thread: wait for a full stage
+          tc_fence_after();
+          const uint32_t a_lo = a_lo0 + (uint32_t)st * (STAGE_BYTES >> 4);
+          const uint32_t b_lo = b_lo0 + (uint32_t)st * (STAGE_BYTES >> 4);
+          if (kc != q.num_kc - 1) {
 #pragma unroll
-          for (int j = 0; j < KB / 16; ++j) {
-            if (j < nks) {
-              if (PAIR)
-                umma_f16_ab_pair(acc, a_lo + 2 * j, kSmemDescHiSw128, b_lo + 2 * j, kSmemDescHiSw128, idesc, accumulate);
-              else
-                umma_f16_lohi(acc, a_lo + 2 * j, b_lo + 2 * j, idesc, accumulate);
+            for (int j = 0; j < KSUB * (KB / 16); ++j) {
+              const uint32_t off = (uint32_t)(j / 4) * (SUB_BYTES >> 4) + 2u * (uint32_t)(j % 4);
+              if (PAIR) umma_f16_ab_pair(acc, a_lo + off, kSmemDescHiSw128, b_lo + off, kSmemDescHiSw128, idesc, accumulate);
+              else umma_f16_lohi(acc, a_lo + off, b_lo + off, idesc, accumulate);
+              accumulate = 1u;
+            }
+          } else {
+            // the last chunk of K: only the 16-wide steps that hold real k
+            for (int j = 0; j < q.nks_last; ++j) {
+              const uint32_t off = (uint32_t)(j / 4) * (SUB_BYTES >> 4) + 2u * (uint32_t)(j % 4);
+              if (PAIR) umma_f16_ab_pair(acc, a_lo + off, kSmemDescHiSw128, b_lo + off, kSmemDescHiSw128, idesc, accumulate);
+              else umma_f16_lohi(acc, a_lo + off, b_lo + off, idesc, accumulate);
               accumulate = 1u;
             }
           }
           if (PAIR) umma_commit_pair(empty0 + 8 * st);
           else umma_commit(empty0 + 8 * st);
+          if (++st == q.stages) { st = 0; ph ^= 1u; }
         }
-        __syncwarp();
-        if (++st == q.stages) { st = 0; ph ^= 1u; }
+        if (ok) {
+          if (PAIR) umma_commit_pair(acc_full0 + 8 * buf);
+          else umma_commit(acc_full0 + 8 * buf);
+        }
       }
-      if (ok && leader) {
-        if (PAIR) umma_commit_pair(acc_full0 + 8 * buf);
-        else umma_commit(acc_full0 + 8 * buf);
-      }
-      __syncwarp();
+      if (blockIdx.x == 0) { TIMER_LAP(2); TIMER_FLUSH(); }
     }
+    __syncwarp();
   } else if (warp >= WARP_EPI0) {
     // ---------------- epilogue: tensor memory -> output -----------------------------
     const int lq = warp & 3;                     // tensor-memory lane quadrant this warp may read
     const bool vec_ok = q.out16 ? (q.Co % 8 == 0) : (q.Co % 4 == 0);
+    wait_for_previous_kernel();                  // before the first store to y
     bool ok = true;
     uint32_t it = 0;
+    TIMER_DECL;
     for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
       const uint32_t buf = it & 1u;
       const int mt = w / per_mt, rem = w - mt * per_mt;
@@ -283,15 +314,20 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
           base = ((int64_t)n * q.Co + n0) * q.HoWo + ho * q.Wo + wo;
         }
       }
+      if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(5);     // epilogue: draining and storing
       if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
       __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
       if (!ok) break;
+      if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(6);     // epilogue: wait for a finished accumulator
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
       const bool first_part = ks == 0;           // of a split K, only the first part adds the bias
+      // warps 2..5 take the lower half of the tile's channels, warps 6..9 the upper half
+      constexpr int CH = BN / 2;
+      const int cbeg = ((warp - WARP_EPI0) >> 2) * CH;
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int c0 = cbeg; c0 < cbeg + CH; c0 += 32) {
         const int cnt = q.Co - n0 - c0;          // channels left from c0 on
         if (cnt <= 0) break;
         uint32_t v[32];
@@ -315,6 +351,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
         else mbar_arrive(acc_empty0 + 8 * buf);
       }
     }
+    if (threadIdx.x == WARP_EPI0 * 32 && blockIdx.x == 0) { TIMER_LAP(5); TIMER_FLUSH(); }
   }
 
   // ---------------- teardown ---------------------------------------------------
@@ -333,32 +370,67 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
   }
 }
 
-template <int BN>
+template <int BN, int KSUB>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_f16_nhwc_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap, NhwcParams q) {
-  conv_nhwc_body<BN, false>(amap, bmap, q);
+  conv_nhwc_body<BN, false, KSUB>(amap, bmap, q);
 }
 
-template <int BN>
+template <int BN, int KSUB>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 conv_f16_nhwc_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap, NhwcParams q) {
-  conv_nhwc_body<BN, true>(amap, bmap, q);
+  conv_nhwc_body<BN, true, KSUB>(amap, bmap, q);
 }
 
 // Filter pack (paper Section "Im2win Convolution": height before width; here with the channel below
-// both): fp[co][(v*Kh + u)*Cp + c] = f[co][c][u][v], zeros for c >= C.  Thread 0.. of block 0 also
-// clears the status block.
-__global__ void pack_f16_nhwc_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, uint32_t* status,
-                                     int C, int Cp, int Kh, int Kw, int64_t total) {
-  if (blockIdx.x == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
-  const int64_t K = (int64_t)Kw * Kh * Cp;
-  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t co = idx / K;
-    int64_t t = idx - co * K;
-    const int c = (int)(t % Cp);
-    t /= Cp;
-    const int u = (int)(t % Kh), v = (int)(t / Kh);
-    fp[idx] = c < C ? f[((co * C + c) * Kh + u) * Kw + v] : (uint16_t)0;
+// both): fp[co][(v*Kh + u)*Cp + c] = f[co][c][u][v], zeros for c >= C.  One block takes one output
+// channel and a run of `cb` input channels: their cb*Kh*Kw halves are contiguous in the OIHW filter
+// (coalesced reads into shared memory) and leave as Kh*Kw runs of cb channels (coalesced writes).
+// Block (0, 0) also clears the status block.
+__global__ void __launch_bounds__(256)
+pack_f16_nhwc_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, uint32_t* status, int C, int Cp,
+                     int Co, int Kh, int Kw, int cb) {
+  extern __shared__ __align__(16) uint16_t pack_s[];   // [cb][T], after up to 8 halves of phase padding
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
+  const int T = Kh * Kw;
+  const int64_t K = (int64_t)T * Cp;
+  const int c0 = blockIdx.x * cb;
+  const int nc = Cp - c0 < cb ? Cp - c0 : cb;     // stored channels of this block (Cp and cb are multiples of 8)
+  const int nreal = C - c0 < nc ? (C - c0 > 0 ? C - c0 : 0) : nc;
+  const int pairs = nc / 2;
+  for (int co = blockIdx.y; co < Co; co += gridDim.y) {
+    const uint16_t* src = f + ((int64_t)co * C + c0) * T;
+    // the run is read with 16-byte loads from the first 16-byte boundary on (shared-memory copy kept at
+    // the same phase), four loads in flight per thread; the ragged ends element by element
+    const int n = nreal * T;
+    const int head = (int)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(src) & 15u)) & 15u) >> 1);   // halves before the boundary
+    uint16_t* dst = pack_s + 8 - head;              // dst + head is 16-byte aligned (pack_s is)
+    const int nvec = n > head ? (n - head) / 8 : 0;
+    for (int i = threadIdx.x; i < (n < head ? n : head); i += blockDim.x) dst[i] = __ldg(src + i);
+    for (int i = head + nvec * 8 + threadIdx.x; i < n; i += blockDim.x) dst[i] = __ldg(src + i);
+    const uint4* vsrc = reinterpret_cast<const uint4*>(src + head);
+    uint4* vdst = reinterpret_cast<uint4*>(dst + head);
+    for (int i0 = threadIdx.x; i0 < nvec; i0 += 4 * blockDim.x) {
+      uint4 r[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (i0 + j * (int)blockDim.x < nvec) r[j] = __ldg(vsrc + i0 + j * blockDim.x);
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (i0 + j * (int)blockDim.x < nvec) vdst[i0 + j * blockDim.x] = r[j];
+    }
+    const uint16_t* ps = dst;                       // element i of the run is ps[i]
+    __syncthreads();
+    // thread -> (t = v*Kh + u, channel pair): 4-byte stores, consecutive threads along c
+    for (int i = threadIdx.x; i < T * pairs; i += blockDim.x) {
+      const int t = i / pairs, cp2 = i - t * pairs;
+      const int v = t / Kh, u = t - v * Kh;
+      const int c = 2 * cp2;
+      const uint32_t lo = c < nreal ? ps[c * T + u * Kw + v] : 0u;
+      const uint32_t hi = c + 1 < nreal ? ps[(c + 1) * T + u * Kw + v] : 0u;
+      *reinterpret_cast<uint32_t*>(fp + (int64_t)co * K + (int64_t)t * Cp + c0 + c) = lo | (hi << 16);
+    }
+    __syncthreads();
   }
 }
 
@@ -394,40 +466,102 @@ __global__ void transform_nhwc_from_nhwc_kernel(const uint16_t* __restrict__ x, 
   }
 }
 
-// x given NCHW: a transposition.  One block moves the 64 channels x 64 columns of one (n, ho, u):
-// input row h = ho*s + u - p of 64 channels is read along w (coalesced), turned in shared memory and
-// written along c (128 bytes per column k).
-constexpr int TT = 64;
+// x given NCHW: a transposition.  One block builds the part of one strip (n, ho) that covers `kc`
+// columns: phase 1 reads the Kh input rows of every channel along w (coalesced) and stores them in
+// shared memory as [k][u][c] (pitch Cp + 2 halves = an odd number of words); phase 2 walks the
+// strip's 16-byte chunks in output order (c fastest, then u, then k), reads each from shared memory
+// as four words and writes it with one coalesced 16-byte store.  Indices are kept in mixed-radix
+// counters (no division per element); what depends on (u, c) alone is tabulated once per block.
+template <bool VEC2>
 __global__ void __launch_bounds__(256)
 transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ win, int C, int Cp, int H, int W,
-                                int Ho, int Wp, int Kh, int s, int p, int ctiles, int ktiles) {
-  __shared__ uint16_t tile[TT][TT + 2];          // [k][c], 33-word pitch: conflict-free both ways
+                                int Ho, int Wp, int Kh, int s, int p, int kc, int kchunks) {
+  extern __shared__ __align__(16) uint16_t rows_s[];     // [kc][Kh][Cp + 2], then two int tables of Kh*C entries
+  const int PC = Cp + 2;
+  int* rowsrc = reinterpret_cast<int*>(rows_s + (size_t)kc * Kh * PC);   // (c*H + h)*W of row (u, c), -1 outside the image
+  int* rowdst = rowsrc + Kh * C;                                         // u*PC + c
   int64_t b = blockIdx.x;
-  const int kt = (int)(b % ktiles); b /= ktiles;
-  const int ct = (int)(b % ctiles); b /= ctiles;
-  const int u = (int)(b % Kh); b /= Kh;
+  const int kci = (int)(b % kchunks); b /= kchunks;
   const int ho = (int)(b % Ho);
   const int64_t n = b / Ho;
-  const int h = ho * s + u - p;
-  const int k0 = kt * TT, c0 = ct * TT;
-  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;      // 64 x 4
-  const bool row_ok = h >= 0 && h < H;
-  for (int cc = ty; cc < TT; cc += 4) {
-    const int c = c0 + cc, w = k0 + tx - p;
-    uint16_t v = 0;
-    if (row_ok && c < C && w >= 0 && w < W && k0 + tx < Wp) v = __ldg(x + ((n * C + c) * H + h) * (int64_t)W + w);
-    tile[tx][cc] = v;
+  const int k0 = kci * kc;
+  const int nk = Wp - k0 < kc ? Wp - k0 : kc;             // columns of this block
+  // input columns that exist among k0 .. k0 + nk - 1 (k = w + p)
+  const int w_lo = k0 - p > 0 ? k0 - p : 0;
+  const int w_hi = k0 + nk - p < W ? k0 + nk - p : W;     // exclusive
+  const int nw = w_hi > w_lo ? w_hi - w_lo : 0;
+  const int nrows = Kh * C;
+  for (int r = threadIdx.x; r < nrows; r += blockDim.x) {
+    const int u = r / C, c = r - u * C;
+    const int h = ho * s + u - p;
+    rowsrc[r] = (h >= 0 && h < H) ? (c * H + h) * W : -1;
+    rowdst[r] = u * PC + c;
+  }
+  if (Cp > C) {                                           // the zero channels C .. Cp-1
+    const int extra = Cp - C;
+    for (int i = threadIdx.x; i < kc * Kh * extra; i += blockDim.x) {
+      const int r = i / extra, e = i - r * extra;
+      rows_s[r * PC + C + e] = 0;
+    }
   }
   __syncthreads();
-  // write: thread -> (column k, channel pair): 32 lanes write 128 contiguous bytes of one column
-  const int cw = (Cp - c0 < TT ? Cp - c0 : TT) / 2;            // channel pairs of this tile (Cp is even)
-  const int lane2 = threadIdx.x & 31, kq = threadIdx.x >> 5;   // 32 x 8
-  for (int kk = kq; kk < TT; kk += 8) {
-    const int k = k0 + kk;
-    if (k >= Wp || lane2 >= cw) continue;
-    const uint32_t v = *reinterpret_cast<const uint32_t*>(&tile[kk][2 * lane2]);    // rows are 132 bytes: 4-byte aligned
-    uint16_t* dst = win + ((((n * Ho + ho) * Wp + k) * Kh + u) * (int64_t)Cp) + c0 + 2 * lane2;
-    *reinterpret_cast<uint32_t*>(dst) = v;
+  const uint16_t* ximg = x + n * ((int64_t)C * H * W);
+  // phase 1: item -> (row = (u, c), column (pair)), columns fastest; 8 loads in flight per thread
+  {
+    constexpr int E = VEC2 ? 2 : 1;                       // columns per item (VEC2: W, w_lo and nw are even)
+    const int nwi = nw / E;
+    const int items = nrows * nwi;
+    const int step = (int)blockDim.x;
+    const int d_row = nwi > 0 ? step / nwi : 0, d_col = nwi > 0 ? step - d_row * nwi : 0;
+    int row = nwi > 0 ? (int)threadIdx.x / nwi : 0, col = nwi > 0 ? (int)threadIdx.x - row * nwi : 0;
+    for (int i0 = threadIdx.x; i0 < items; i0 += 8 * step) {
+      uint32_t r[8];
+      int dsts[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        r[j] = 0u;
+        dsts[j] = -1;
+        if (i0 + j * step < items) {
+          const int src = rowsrc[row];
+          const int wcol = w_lo + E * col;
+          dsts[j] = ((wcol + p - k0) * Kh) * PC + rowdst[row];
+          if (src >= 0) {
+            if (VEC2) r[j] = __ldg(reinterpret_cast<const uint32_t*>(ximg + src + wcol));
+            else r[j] = __ldg(ximg + src + wcol);
+          }
+        }
+        col += d_col; row += d_row;
+        if (col >= nwi) { col -= nwi; ++row; }
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (dsts[j] >= 0) {
+          rows_s[dsts[j]] = (uint16_t)(r[j] & 0xffffu);
+          if (VEC2) rows_s[dsts[j] + Kh * PC] = (uint16_t)(r[j] >> 16);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  // phase 2: chunk j = t*octs + oct with t = kk*Kh + u: consecutive threads write consecutive 16 bytes
+  const int octs = Cp / 8;
+  const int chunks = nk * Kh * octs;
+  const int t_lo = (p - k0 > 0 ? p - k0 : 0) * Kh, t_hi = (W + p - k0) * Kh;   // columns inside the image
+  uint4* out = reinterpret_cast<uint4*>(win + (((n * Ho + ho) * (int64_t)Wp + k0) * Kh) * Cp);
+  {
+    const int step = (int)blockDim.x;
+    const int d_t = step / octs, d_o = step - d_t * octs;
+    int t = (int)threadIdx.x / octs, oct = (int)threadIdx.x - t * octs;
+    for (int j = threadIdx.x; j < chunks; j += step) {
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (t >= t_lo && t < t_hi) {                        // rows outside the image were stored as zeros in phase 1
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(rows_s + t * PC + 8 * oct);
+        v = make_uint4(src[0], src[1], src[2], src[3]);
+      }
+      out[j] = v;
+      oct += d_o; t += d_t;
+      if (oct >= octs) { oct -= octs; ++t; }
+    }
   }
 }
 
@@ -449,41 +583,89 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-template <int BN, bool PAIR>
-cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, NhwcParams q, int slots, cudaStream_t stream) {
+template <int BN, bool PAIR, int KSUB>
+cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, NhwcParams q, const NhwcPlan& plan,
+                           cudaStream_t stream) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;
-  constexpr int STAGE = A_SLOT_BYTES + B_ROWS * KB * 2;
+  constexpr int STAGE = KSUB * (A_SLOT_BYTES + B_ROWS * KB * 2);
   int stages = (kSmemMax - 2048) / STAGE;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) return cudaErrorInvalidValue;
   q.stages = stages;
+  // K in chunks of KSUB k-blocks; a K split hands out whole chunks
+  q.num_kc = (plan.num_kb + KSUB - 1) / KSUB;
+  q.nks_last = (int32_t)((plan.K - (int64_t)(q.num_kc - 1) * KSUB * KB + 15) / 16);
+  q.kc_per_split = (q.num_kc + q.ksplit - 1) / q.ksplit;
+  q.ksplit = (q.num_kc + q.kc_per_split - 1) / q.kc_per_split;
+  const int64_t ntm_eff = PAIR ? (plan.ntm + 1) / 2 : plan.ntm;
+  const int64_t nwork = ntm_eff * q.ntn * q.ksplit;
+  if (nwork >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
+  q.nwork = (int32_t)nwork;
+  const int slots = PAIR ? 74 : 148;
   const int smem_bytes = stages * STAGE + 1024;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(NUM_THREADS, 1, 1);
   cfg.dynamicSmemBytes = (size_t)smem_bytes;
   cfg.stream = stream;
+  // per device and kernel variant, done once: the shared-memory opt-in and the number of CTA pairs
+  // that can be resident together (both are host-side queries that would otherwise sit between the
+  // filter pack and this launch on every call)
+  static int cached_clusters[64] = {};           // 0 = not yet asked
+  static bool attr_done[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   if (PAIR) {
-    cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-    if (e != cudaSuccess) return e;
-    cudaLaunchAttribute attr[1];
+    cudaError_t e = cudaSuccess;
+    if (!attr_done[dev]) {
+      e = cudaFuncSetAttribute(conv_f16_nhwc_pair_kernel<BN, KSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+      if (e != cudaSuccess) return e;
+      attr_done[dev] = true;
+    }
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.gridDim = dim3(148, 1, 1);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    int clusters = 0;                           // as many pairs as can be resident at once
-    e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_nhwc_pair_kernel<BN>, &cfg);
-    if (e != cudaSuccess) return e;
-    if (clusters < 1) return cudaErrorInvalidValue;
+    int clusters = cached_clusters[dev];        // as many pairs as can be resident at once
+    if (clusters == 0) {
+      e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_nhwc_pair_kernel<BN, KSUB>, &cfg);
+      if (e != cudaSuccess) return e;
+      if (clusters < 1) return cudaErrorInvalidValue;
+      cached_clusters[dev] = clusters;
+    }
     if (clusters > slots) clusters = slots;
     if (clusters > q.nwork) clusters = q.nwork;
     cfg.gridDim = dim3(2 * clusters, 1, 1);
-    return cudaLaunchKernelEx(&cfg, conv_f16_nhwc_pair_kernel<BN>, amap, bmap, q);
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, conv_f16_nhwc_pair_kernel<BN, KSUB>, amap, bmap, q);
   }
-  cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-  if (e != cudaSuccess) return e;
+  if (!attr_done[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_kernel<BN, KSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (e != cudaSuccess) return e;
+    attr_done[dev] = true;
+  }
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   cfg.gridDim = dim3((unsigned)(slots < q.nwork ? slots : q.nwork), 1, 1);
-  return cudaLaunchKernelEx(&cfg, conv_f16_nhwc_kernel<BN>, amap, bmap, q);
+  return cudaLaunchKernelEx(&cfg, conv_f16_nhwc_kernel<BN, KSUB>, amap, bmap, q);
+}
+
+template <int KSUB>
+cudaError_t launch_ksub(const CUtensorMap& amap, const CUtensorMap& bmap, const NhwcParams& q, const NhwcPlan& plan,
+                        cudaStream_t stream) {
+  if (plan.pair) {
+    if (plan.bn == 256) return launch_variant<256, true, KSUB>(amap, bmap, q, plan, stream);
+    return launch_variant<128, true, KSUB>(amap, bmap, q, plan, stream);
+  }
+  if (plan.bn == 64) return launch_variant<64, false, KSUB>(amap, bmap, q, plan, stream);
+  if (plan.bn == 128) return launch_variant<128, false, KSUB>(amap, bmap, q, plan, stream);
+  return launch_variant<256, false, KSUB>(amap, bmap, q, plan, stream);
 }
 
 }  // namespace
@@ -500,6 +682,9 @@ NhwcPlan plan_nhwc(const Geometry& g) {
   p.window_elems = (int64_t)g.N * g.Ho * p.strip;
   if ((int64_t)g.N * g.Ho >= lim || p.strip >= lim) return p;
   if ((int64_t)g.s * g.Kh * p.Cp * 2 >= ((int64_t)1 << 40) || p.strip * 2 >= ((int64_t)1 << 40)) return p;
+  // the transform from NCHW tabulates one entry per (u, c) in shared memory and indexes an image with 32 bits
+  if ((int64_t)g.Kh * g.C * 8 > 48 * 1024 || (int64_t)g.C * g.H * g.W >= lim) return p;
+  if ((int64_t)g.Kh * (p.Cp + 2) * 2 > 56 * 1024) return p;
   // position tiles: tw tiles along a strip of bw columns each (one when the strip fits 128 rows),
   // G whole strips per tile when a strip is short
   p.tw = (g.Wo + TILE_M - 1) / TILE_M;
@@ -517,24 +702,24 @@ NhwcPlan plan_nhwc(const Geometry& g) {
   const int64_t ntm_eff = p.pair ? (p.ntm + 1) / 2 : p.ntm;
   const int slots = p.pair ? 74 : 148;
   const int64_t tiles = ntm_eff * p.ntn;
-  // K is split when the tiles alone leave most of a wave empty or the last wave nearly so: parts of
-  // at least 8 k-blocks, as many as bring the number of work items to a whole number of waves
-  if (tiles < 2 * slots && p.num_kb >= 16) {
+  // K is split over several CTAs only where the parts stay long (48 k-blocks or more): the partial
+  // sums are added with atomics, which was measured to cost more than the fuller waves gain unless
+  // a long main loop of other items hides it.  Among the admissible splits the one with the best
+  // wave efficiency wins.
+  if (tiles < 4 * slots) {
     double best = 0.0;
     for (int ks = 1; ks <= 8; ++ks) {
       const int per = (p.num_kb + ks - 1) / ks;
-      if (per < 8 && ks > 1) break;
+      if (ks > 1 && per < 48) break;
       const int parts = (p.num_kb + per - 1) / per;
       const int64_t items = tiles * parts;
       const int64_t waves = (items + slots - 1) / slots;
-      // time ~ waves * (k-blocks per part + fixed cost of an item in k-block units)
-      const double t = (double)waves * (per + 3.0 + (parts > 1 ? 1.5 : 0.0));
+      const double t = (double)waves * (per + 4.0 + (parts > 1 ? 2.0 : 0.0));     // in k-blocks
       const double eff = (double)tiles * p.num_kb / slots / t;
-      if (eff > best + 1e-9) { best = eff; p.ksplit = parts; }
+      if (eff > best + 0.02) { best = eff; p.ksplit = parts; }
     }
   }
   p.kb_per_split = (p.num_kb + p.ksplit - 1) / p.ksplit;
-  p.ksplit = (p.num_kb + p.kb_per_split - 1) / p.kb_per_split;
   if (tiles * p.ksplit >= lim) return p;
   p.scratch_bytes = (size_t)kStatusBytes + (size_t)g.Co * p.K * 2;
   p.scratch_bytes = (p.scratch_bytes + 255) / 256 * 256;
@@ -554,11 +739,34 @@ cudaError_t launch_transform_nhwc(const uint16_t* x, int x_is_nhwc, uint16_t* wi
                                                                           g.Kh, g.s, g.p, chunks);
     return cudaGetLastError();
   }
-  const int ctiles = (plan.Cp + TT - 1) / TT, ktiles = (g.Wp + TT - 1) / TT;
-  const int64_t blocks = (int64_t)g.N * g.Ho * g.Kh * ctiles * ktiles;
+  // columns per block: the whole strip when its Kh rows of Cp + 2 halves fit 64 KB of shared memory
+  const int64_t per_col = (int64_t)g.Kh * (plan.Cp + 2) * 2;
+  const int64_t tables = (int64_t)g.Kh * g.C * 8;
+  if ((int64_t)g.C * g.H * g.W >= ((int64_t)1 << 31) || tables > 48 * 1024) return cudaErrorInvalidValue;
+  int kc = (int)((112 * 1024 - tables) / per_col);
+  if (kc < 1) return cudaErrorInvalidValue;
+  if (kc > g.Wp) kc = g.Wp;
+  // with two columns per load the chunk boundaries must stay even
+  const bool vec2 = (g.W % 2 == 0) && (g.p % 2 == 0) && (kc % 2 == 0 || kc == g.Wp);
+  const int kchunks = (g.Wp + kc - 1) / kc;
+  const int64_t blocks = (int64_t)g.N * g.Ho * kchunks;
   if (blocks >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
-  transform_nhwc_from_nchw_kernel<<<(unsigned)blocks, 256, 0, stream>>>(x, window, g.C, plan.Cp, g.H, g.W, g.Ho, g.Wp,
-                                                                        g.Kh, g.s, g.p, ctiles, ktiles);
+  const size_t smem = (size_t)(per_col * kc + tables);
+  static bool attr_done[64][2] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!attr_done[dev][vec2]) {
+    cudaError_t e = vec2 ? cudaFuncSetAttribute(transform_nhwc_from_nchw_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024)
+                         : cudaFuncSetAttribute(transform_nhwc_from_nchw_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_done[dev][vec2] = true;
+  }
+  if (vec2)
+    transform_nhwc_from_nchw_kernel<true><<<(unsigned)blocks, 256, smem, stream>>>(x, window, g.C, plan.Cp, g.H, g.W, g.Ho, g.Wp,
+                                                                                   g.Kh, g.s, g.p, kc, kchunks);
+  else
+    transform_nhwc_from_nchw_kernel<false><<<(unsigned)blocks, 256, smem, stream>>>(x, window, g.C, plan.Cp, g.H, g.W, g.Ho, g.Wp,
+                                                                                    g.Kh, g.s, g.p, kc, kchunks);
   return cudaGetLastError();
 }
 
@@ -566,11 +774,19 @@ cudaError_t launch_pack_f16_nhwc(const uint16_t* filter, void* scratch, const Ge
   const NhwcPlan plan = plan_nhwc(g);
   if (!plan.eligible) return cudaErrorInvalidValue;
   unsigned char* base = static_cast<unsigned char*>(scratch);
-  const int64_t total = (int64_t)g.Co * plan.K;
-  int64_t blocks = (total + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
-  pack_f16_nhwc_kernel<<<(unsigned)blocks, 256, 0, stream>>>(filter, reinterpret_cast<uint16_t*>(base + kStatusBytes),
-                                                             reinterpret_cast<uint32_t*>(base), g.C, plan.Cp, g.Kh, g.Kw, total);
+  // channels per block: as many as fit 32 KB of staging, a multiple of 8, at least 8
+  int cb = (32 * 1024 / 2 / g.T) / 8 * 8;
+  if (cb < 8) cb = 8;
+  if (cb > plan.Cp) cb = plan.Cp;
+  const size_t smem = (size_t)cb * g.T * 2 + 32;
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(pack_f16_nhwc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid((unsigned)((plan.Cp + cb - 1) / cb), (unsigned)(g.Co < 32768 ? g.Co : 32768));
+  pack_f16_nhwc_kernel<<<grid, 256, smem, stream>>>(filter, reinterpret_cast<uint16_t*>(base + kStatusBytes),
+                                                     reinterpret_cast<uint32_t*>(base), g.C, plan.Cp, g.Co, g.Kh, g.Kw, cb);
   return cudaGetLastError();
 }
 
@@ -589,14 +805,11 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   }
   if (const char* v = debug_getenv("IM2WIN_NHWC_PAIR")) plan.pair = v[0] == '1' && plan.bn >= 128;
   if (const char* v = debug_getenv("IM2WIN_NHWC_KSPLIT")) {
-    int ks = atoi(v);
-    if (ks >= 1 && ks <= plan.num_kb) {
-      plan.kb_per_split = (plan.num_kb + ks - 1) / ks;
-      plan.ksplit = (plan.num_kb + plan.kb_per_split - 1) / plan.kb_per_split;
-    }
+    const int ks = atoi(v);
+    if (ks >= 1 && ks <= plan.num_kb) plan.ksplit = ks;
   }
   const bool split = plan.ksplit > 1 && !epi.relu && !epi.out16;   // partial sums cannot pass a ReLU or a rounding
-  if (!split) { plan.ksplit = 1; plan.kb_per_split = plan.num_kb; }
+  if (!split) plan.ksplit = 1;
 
   // Activation operand: (k, wo, strip) with OVERLAPPING rows: the row of output column wo starts
   // s*Kh*Cp halves after that of wo-1.  k beyond K, columns beyond Wo and strips beyond N*Ho read
@@ -632,26 +845,18 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   q.Ho = g.Ho; q.Wo = g.Wo; q.Co = g.Co; q.HoWo = g.Ho * g.Wo;
   q.rows_total = g.N * g.Ho;
   q.bw = plan.bw; q.G = plan.G; q.tw = plan.tw;
-  q.num_kb = plan.num_kb;
-  q.nks_last = (int32_t)((plan.K - (int64_t)(plan.num_kb - 1) * KB + 15) / 16);
-  q.ksplit = plan.ksplit; q.kb_per_split = plan.kb_per_split;
+  q.ksplit = plan.ksplit;
   q.ntn = plan.ntn;
-  const int64_t ntm_eff = plan.pair ? (plan.ntm + 1) / 2 : plan.ntm;
-  const int64_t nwork = ntm_eff * plan.ntn * plan.ksplit;
-  if (nwork >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
-  q.nwork = (int32_t)nwork;
   q.a_bytes = (uint32_t)(plan.G * plan.bw * KB * 2);
   if (split) {
     cudaError_t e = cudaMemsetAsync(y, 0, (size_t)g.out_elems * 4, stream);
     if (e != cudaSuccess) return e;
   }
-  if (plan.pair) {
-    if (plan.bn == 256) return launch_variant<256, true>(amap, bmap, q, 74, stream);
-    return launch_variant<128, true>(amap, bmap, q, 74, stream);
-  }
-  if (plan.bn == 64) return launch_variant<64, false>(amap, bmap, q, 148, stream);
-  if (plan.bn == 128) return launch_variant<128, false>(amap, bmap, q, 148, stream);
-  return launch_variant<256, false>(amap, bmap, q, 148, stream);
+  if (const char* v = debug_getenv("IM2WIN_NHWC_SKIP")) q.dbg_skip = atoi(v);
+  int ksub = 2;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_KSUB")) ksub = atoi(v) == 1 ? 1 : 2;
+  if (ksub == 1) return launch_ksub<1>(amap, bmap, q, plan, stream);
+  return launch_ksub<2>(amap, bmap, q, plan, stream);
 }
 
 }  // namespace im2win
