@@ -22,7 +22,9 @@
 // into an output that was cleared first.  Every mbarrier wait is bounded.
 #include <cuda.h>
 #include <cuda_fp16.h>
+#include <stdio.h>
 #include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
@@ -42,13 +44,18 @@ constexpr int MAX_STAGES = 8;
 constexpr int A_SLOT_BYTES = TILE_M * KB * 2;  // 16 KB: room for 128 rows even when a tile holds fewer
 constexpr int kSmemMax = 227 * 1024;
 
-struct NhwcParams {
+// What the epilogue needs to know about the output (shared by both kernels of this file).
+struct EpiParams {
   void* y;
   const float* bias;
-  uint32_t* status;
   int32_t relu, out16, y_nhwc, atomic;
   int32_t Ho, Wo, Co, HoWo;
   int32_t rows_total;        // N*Ho strips
+};
+
+struct NhwcParams {
+  EpiParams e;
+  uint32_t* status;
   int32_t bw, G, tw;         // tile = G strips x bw output columns; tw tiles along a strip
   int32_t num_kc;            // chunks of KSUB 64-wide k-blocks (one ring stage each)
   int32_t nks_last;          // 16-wide MMA steps of the last chunk
@@ -56,7 +63,7 @@ struct NhwcParams {
   int32_t ntn, nwork;        // channel tiles; work items = position tiles (pairs) x channel tiles x k parts
   int32_t stages;
   uint32_t a_bytes;          // bytes one activation copy brings: G*bw*128
-  int32_t dbg_skip;
+  int32_t ww;
 };
 
 // Programmatic dependent launch: the convolution may start while the kernel before it in the stream
@@ -72,7 +79,7 @@ __device__ __forceinline__ void red_add_f32(float* p, float v) {
 // Epilogue of one accumulator row chunk: v[j] belongs to output channel c0 + j (j < cnt) of the
 // row's position; `base` is the element index of channel c0 at that position and `cs` the element
 // distance between channels (Ho*Wo for NCHW, 1 for NHWC).
-__device__ __forceinline__ void store_chunk(const NhwcParams& q, int64_t base, int64_t cs, const uint32_t (&v)[32],
+__device__ __forceinline__ void store_chunk(const EpiParams& q, int64_t base, int64_t cs, const uint32_t (&v)[32],
                                             int cnt, bool vec_ok) {
   if (q.atomic) {
     float* p = reinterpret_cast<float*>(q.y) + base;
@@ -120,6 +127,34 @@ __device__ __forceinline__ void store_chunk(const NhwcParams& q, int64_t base, i
       for (int j = 0; j < 32; ++j)
         if (j < cnt) p[j] = __float2half_rn(__uint_as_float(v[j]));
     }
+  }
+}
+
+// One epilogue warp's share of a finished accumulator: tensor-memory lane quadrant warp % 4, the
+// lower (warps 2..5) or upper (warps 6..9) half of the tile's BN channels, 32 channels at a time:
+// bias (first K part only), ReLU, store.  `base` is the element index of the tile's first channel
+// at this lane's position, `cs` the element distance between channels.
+template <int BN>
+__device__ __forceinline__ void drain_accumulator(const EpiParams& e, int warp, int lane, uint32_t lane_base, bool valid,
+                                                  int64_t base, int64_t cs, int n0, bool first_part, bool vec_ok) {
+  constexpr int CH = BN / 2;
+  const int cbeg = ((warp - WARP_EPI0) >> 2) * CH;
+#pragma unroll 1
+  for (int c0 = cbeg; c0 < cbeg + CH; c0 += 32) {
+    const int cnt = e.Co - n0 - c0;              // channels left from c0 on
+    if (cnt <= 0) break;
+    uint32_t v[32];
+    tmem_ld32(lane_base + (uint32_t)c0, v);
+    if (e.bias != nullptr && first_part) {
+      const float b = lane < cnt ? __ldg(e.bias + n0 + c0 + lane) : 0.0f;
+#pragma unroll
+      for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(__uint_as_float(v[t]) + __shfl_sync(0xffffffffu, b, t));
+    }
+    if (e.relu) {
+#pragma unroll
+      for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(fmaxf(__uint_as_float(v[t]), 0.0f));
+    }
+    if (valid) store_chunk(e, base + (int64_t)c0 * cs, cs, v, cnt < 32 ? cnt : 32, vec_ok);
   }
 }
 
@@ -203,17 +238,16 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
           const uint32_t bar = full_dst + 8 * st;
           // k-blocks beyond K read as zeros (and cost no memory traffic), so every stage brings the
           // same number of bytes.  In a pair the leader CTA announces the bytes of both CTAs.
-          const uint32_t abytes = (q.dbg_skip & 1) ? 0u : q.a_bytes, bbytes = (q.dbg_skip & 2) ? 0u : B_BYTES;
-          if (!PAIR || rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, (PAIR ? 2u : 1u) * KSUB * (abytes + bbytes));
+          if (!PAIR || rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, (PAIR ? 2u : 1u) * KSUB * (q.a_bytes + B_BYTES));
 #pragma unroll
           for (int sub = 0; sub < KSUB; ++sub) {
             const int kx = (kc * KSUB + sub) * KB;
             if (PAIR) {
-              if (abytes) tma_load_3d_pair(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
-              if (bbytes) tma_load_2d_pair(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
+              tma_load_3d_pair(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
+              tma_load_2d_pair(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
             } else {
-              if (abytes) tma_load_3d(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
-              if (bbytes) tma_load_2d(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
+              tma_load_3d(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
+              tma_load_2d(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
             }
           }
           if (++st == q.stages) { st = 0; ph ^= 1u; }
@@ -228,7 +262,55 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
     // Every byte the MMAs read was written by the copy engine, whose completion the barrier's
     // transaction count tracks, so CTA-scope waits suffice also for the peer's half.
     constexpr uint32_t idesc = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN);
-    if (lane == 0) {
+    if (q.ww) {
+      // experiment: the whole warp walks the loop, one elected lane issues
+      const bool leader = elect_one();
+      int st = 0;
+      uint32_t ph = 0, it = 0;
+      bool ok = true;
+      const uint32_t a_lo0 = smem_desc_lo(ring), b_lo0 = smem_desc_lo(ring + (uint32_t)A_SLOT_BYTES);
+      for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
+        const int rem = w % per_mt;
+        const int ks = rem % q.ksplit;
+        const int kc0 = ks * q.kc_per_split;
+        const int kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
+        const uint32_t buf = it & 1u;
+        ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t acc = tmem_acc + buf * (uint32_t)BN;
+        uint32_t accumulate = 0;
+        for (int kc = kc0; kc < kc1; ++kc) {
+          ok = mbar_wait(full0 + 8 * st, ph, &abort_flag, q.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          const uint32_t a_lo = a_lo0 + (uint32_t)st * (STAGE_BYTES >> 4);
+          const uint32_t b_lo = b_lo0 + (uint32_t)st * (STAGE_BYTES >> 4);
+          if (leader) {
+            const int nks = kc != q.num_kc - 1 ? KSUB * (KB / 16) : q.nks_last;
+#pragma unroll
+            for (int j = 0; j < KSUB * (KB / 16); ++j) {
+              if (j < nks) {
+                const uint32_t off = (uint32_t)(j / 4) * (SUB_BYTES >> 4) + 2u * (uint32_t)(j % 4);
+                if (PAIR) umma_f16_ab_pair(acc, a_lo + off, kSmemDescHiSw128, b_lo + off, kSmemDescHiSw128, idesc, accumulate);
+                else umma_f16_lohi(acc, a_lo + off, b_lo + off, idesc, accumulate);
+                accumulate = 1u;
+              }
+            }
+            if (PAIR) umma_commit_pair(empty0 + 8 * st);
+            else umma_commit(empty0 + 8 * st);
+          }
+          __syncwarp();
+          if (++st == q.stages) { st = 0; ph ^= 1u; }
+        }
+        if (ok && leader) {
+          if (PAIR) umma_commit_pair(acc_full0 + 8 * buf);
+          else umma_commit(acc_full0 + 8 * buf);
+        }
+        __syncwarp();
+      }
+    } else if (lane == 0) {
       int st = 0;
       uint32_t ph = 0, it = 0;
       bool ok = true;
@@ -252,7 +334,6 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
           ok = mbar_wait(full0 + 8 * st, ph, &abort_flag, q.status);
           if (!ok) break;
           TIMER_LAP(4);                              // MMA thread: wait for a full stage
-          tc_fence_after();
           const uint32_t a_lo = a_lo0 + (uint32_t)st * (STAGE_BYTES >> 4);
           const uint32_t b_lo = b_lo0 + (uint32_t)st * (STAGE_BYTES >> 4);
           if (kc != q.num_kc - 1) {
@@ -287,7 +368,8 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
   } else if (warp >= WARP_EPI0) {
     // ---------------- epilogue: tensor memory -> output -----------------------------
     const int lq = warp & 3;                     // tensor-memory lane quadrant this warp may read
-    const bool vec_ok = q.out16 ? (q.Co % 8 == 0) : (q.Co % 4 == 0);
+    const EpiParams& e = q.e;
+    const bool vec_ok = e.out16 ? (e.Co % 8 == 0) : (e.Co % 4 == 0);
     wait_for_previous_kernel();                  // before the first store to y
     bool ok = true;
     uint32_t it = 0;
@@ -303,15 +385,15 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       const int r = lq * 32 + lane;
       const int j = r / q.bw, i = r - j * q.bw;
       const int strip = rg * q.G + j, wo = wt * q.bw + i;
-      const bool valid = j < q.G && strip < q.rows_total && wo < q.Wo;
+      const bool valid = j < q.G && strip < e.rows_total && wo < e.Wo;
       int64_t base = 0, cs = 1;
       if (valid) {
-        if (q.y_nhwc) {
-          base = ((int64_t)strip * q.Wo + wo) * q.Co + n0;
+        if (e.y_nhwc) {
+          base = ((int64_t)strip * e.Wo + wo) * e.Co + n0;
         } else {
-          const int n = strip / q.Ho, ho = strip - n * q.Ho;
-          cs = q.HoWo;
-          base = ((int64_t)n * q.Co + n0) * q.HoWo + ho * q.Wo + wo;
+          const int n = strip / e.Ho, ho = strip - n * e.Ho;
+          cs = e.HoWo;
+          base = ((int64_t)n * e.Co + n0) * e.HoWo + ho * e.Wo + wo;
         }
       }
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(5);     // epilogue: draining and storing
@@ -322,27 +404,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(6);     // epilogue: wait for a finished accumulator
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
-      const bool first_part = ks == 0;           // of a split K, only the first part adds the bias
-      // warps 2..5 take the lower half of the tile's channels, warps 6..9 the upper half
-      constexpr int CH = BN / 2;
-      const int cbeg = ((warp - WARP_EPI0) >> 2) * CH;
-#pragma unroll 1
-      for (int c0 = cbeg; c0 < cbeg + CH; c0 += 32) {
-        const int cnt = q.Co - n0 - c0;          // channels left from c0 on
-        if (cnt <= 0) break;
-        uint32_t v[32];
-        tmem_ld32(lane_base + (uint32_t)c0, v);
-        if (q.bias != nullptr && first_part) {
-          const float b = lane < cnt ? __ldg(q.bias + n0 + c0 + lane) : 0.0f;
-#pragma unroll
-          for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(__uint_as_float(v[t]) + __shfl_sync(0xffffffffu, b, t));
-        }
-        if (q.relu) {
-#pragma unroll
-          for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(fmaxf(__uint_as_float(v[t]), 0.0f));
-        }
-        if (valid) store_chunk(q, base + (int64_t)c0 * cs, cs, v, cnt < 32 ? cnt : 32, vec_ok);
-      }
+      drain_accumulator<BN>(e, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
       // the buffer may be overwritten once all four warps (of both CTAs) have read it
       tc_fence_before();
       __syncwarp();
@@ -380,6 +442,319 @@ template <int BN, int KSUB>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 conv_f16_nhwc_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap, NhwcParams q) {
   conv_nhwc_body<BN, true, KSUB>(amap, bmap, q);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Second kernel: shifted views.  The copies above bring every element of a strip into shared
+// memory Kw/s times (the rows of the activation operand overlap).  The im2win layout lets the MMA
+// use that overlap instead: stage every COLUMN of the strips once,
+//     S[sub-tile t][row = virtual position q][64 halves of k2 = (u, c)],   column k = q*s + t,
+// and multiply kernel column v against the view of sub-tile v mod s that starts v div s rows
+// further down (the 128-byte swizzle is a function of the shared-memory address, so a view may start
+// at any row).  One MMA row is one virtual position q = strip*Wq + i, Wq = Wp/s; positions with
+// i >= Wo are computed and dropped (useful fraction Wo/Wq).  Per k2-block the activation bytes that
+// cross from L2 to the SM shrink from Kw*16 KB to 16 KB + halo; the filter tiles (one per (k2-block,
+// kernel column), streamed through their own ring, or resident when the layer's whole filter
+// fits) stay as they were.  Needs s | Wp and Kw >= 2.
+constexpr int MAX_SA = 6, MAX_SB = 12;
+constexpr int WARP_BLOAD = 2 + EPI_WARPS;      // the filter-copy warp of this kernel
+constexpr int SHIFT_THREADS = (NUM_WARPS + 1) * 32;
+
+struct ShiftViewParams {
+  EpiParams e;
+  uint32_t* status;
+  int64_t VQ;                // N*Ho*Wq virtual positions
+  int32_t Wq;                // virtual positions per strip
+  int32_t s, Kw;
+  int32_t rows;              // rows of a sub-tile: 128 + (Kw-1)/s
+  uint32_t subt_bytes;       // rows*128 rounded up to 1024
+  uint32_t a_stage_bytes;    // s*subt_bytes
+  int32_t nkb2;              // 64-wide blocks of k2 = Kh*Cp
+  int32_t nks_last;          // 16-wide MMA steps of the last block
+  int32_t bu;                // (k2-block, kernel column) units per filter stage
+  int32_t sa, sb;            // ring depths
+  int32_t resident;          // 1: the filter ring holds the layer's whole filter, loaded once per CTA
+  int32_t ksplit, kb_per_split;
+  int32_t ntn, nwork;
+};
+
+template <int BN, bool PAIR>
+__device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const CUtensorMap& bmap, const ShiftViewParams& q) {
+  constexpr int B_ROWS = PAIR ? BN / 2 : BN;
+  constexpr uint32_t B_BYTES = (uint32_t)B_ROWS * KB * 2;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const int w_first = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int w_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+  __shared__ __align__(8) uint64_t bars[2 * MAX_SA + 2 * MAX_SB + 4];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ volatile uint32_t abort_flag;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t a_ring = smem_u32(smem);
+  const uint32_t b_ring = a_ring + (uint32_t)q.sa * q.a_stage_bytes;
+  const uint32_t b_stage_bytes = (uint32_t)q.bu * B_BYTES;
+  const uint32_t a_full0 = smem_u32(&bars[0]);
+  const uint32_t a_empty0 = smem_u32(&bars[MAX_SA]);
+  const uint32_t b_full0 = smem_u32(&bars[2 * MAX_SA]);
+  const uint32_t b_empty0 = smem_u32(&bars[2 * MAX_SA + MAX_SB]);
+  const uint32_t acc_full0 = smem_u32(&bars[2 * MAX_SA + 2 * MAX_SB]);
+  const uint32_t acc_empty0 = smem_u32(&bars[2 * MAX_SA + 2 * MAX_SB + 2]);
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0u;
+    for (int i = 0; i < MAX_SA; ++i) { mbar_init(a_full0 + 8 * i, 1); mbar_init(a_empty0 + 8 * i, 1); }
+    for (int i = 0; i < MAX_SB; ++i) { mbar_init(b_full0 + 8 * i, 1); mbar_init(b_empty0 + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(acc_full0 + 8 * i, 1);
+      mbar_init(acc_empty0 + 8 * i, PAIR ? 2 * EPI_WARPS : EPI_WARPS);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == WARP_MMA) {
+    if (PAIR) tmem_alloc_pair(smem_u32(&tmem_base_slot), 2 * BN);
+    else tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (PAIR) cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_acc = tmem_base_slot;
+  const uint32_t a_full_dst = PAIR ? mapa_shared(a_full0, 0) : a_full0;     // the leader's barriers
+  const uint32_t b_full_dst = PAIR ? mapa_shared(b_full0, 0) : b_full0;
+  const uint32_t acc_empty_dst = PAIR ? mapa_shared(acc_empty0, 0) : acc_empty0;
+  const int per_mt = q.ntn * q.ksplit;
+
+  if (warp == WARP_TMA) {
+    // ---------------- activation copies: s sub-tiles per k2-block -------------------
+    // (the whole warp walks the loops and takes the waits, one elected lane issues)
+    {
+      const bool leader = elect_one();
+      wait_for_previous_kernel();
+      int st = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int w = w_first; w < q.nwork && ok; w += w_step) {
+        const int mt = w / per_mt, rem = w - mt * per_mt;
+        const int ks = rem % q.ksplit;
+        const int q0 = (PAIR ? 2 * mt + (int)rank : mt) * TILE_M;
+        const int kb0 = ks * q.kb_per_split;
+        const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          if (leader) {
+            const uint32_t dst = a_ring + (uint32_t)st * q.a_stage_bytes;
+            const uint32_t bar = a_full_dst + 8 * st;
+            if (!PAIR || rank == 0)
+              mbar_arrive_expect_tx(a_full0 + 8 * st, (PAIR ? 2u : 1u) * (uint32_t)(q.s * q.rows * KB * 2));
+            for (int t = 0; t < q.s; ++t) {
+              if (PAIR) tma_load_3d_pair(dst + (uint32_t)t * q.subt_bytes, &amap, kb * KB, t, q0, bar);
+              else tma_load_3d(dst + (uint32_t)t * q.subt_bytes, &amap, kb * KB, t, q0, bar);
+            }
+          }
+          __syncwarp();
+          if (++st == q.sa) { st = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == WARP_BLOAD) {
+    // ---------------- filter copies: bu (k2-block, kernel column) units per stage ----
+    {
+      const bool leader = elect_one();
+      wait_for_previous_kernel();
+      int st = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int w = w_first; w < q.nwork && ok; w += w_step) {
+        const int rem = w % per_mt;
+        const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
+        const int brow = nt * BN + (int)rank * B_ROWS;
+        const int kb0 = ks * q.kb_per_split;
+        const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
+        int kb = kb0, v = 0;
+        for (int left = (kb1 - kb0) * q.Kw; left > 0 && ok; left -= q.bu) {
+          const int nu = left < q.bu ? left : q.bu;             // units of this stage
+          ok = mbar_wait(b_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          const uint32_t dst = b_ring + (uint32_t)st * b_stage_bytes;
+          const uint32_t bar = b_full_dst + 8 * st;
+          if (leader && (!PAIR || rank == 0))
+            mbar_arrive_expect_tx(b_full0 + 8 * st, (PAIR ? 2u : 1u) * (uint32_t)nu * B_BYTES);
+          for (int j = 0; j < nu; ++j) {
+            if (leader) {
+              if (PAIR) tma_load_3d_pair(dst + (uint32_t)j * B_BYTES, &bmap, kb * KB, v, brow, bar);
+              else tma_load_3d(dst + (uint32_t)j * B_BYTES, &bmap, kb * KB, v, brow, bar);
+            }
+            if (++v == q.Kw) { v = 0; ++kb; }
+          }
+          __syncwarp();
+          if (++st == q.sb) { st = 0; ph ^= 1u; }
+        }
+        if (q.resident) break;                   // every stage now holds its units for good
+      }
+    }
+  } else if (warp == WARP_MMA && rank == 0) {
+    // ---------------- MMA issuer ------------------------------------------------------
+    // The whole warp walks the loop (waits are taken by every lane), one elected lane issues the
+    // MMAs and commits: measured faster than a lone lane, whose satisfied waits cost more.
+    constexpr uint32_t idesc = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN);
+    {
+      const bool leader = elect_one();
+      int sta = 0, stb = 0;
+      uint32_t pha = 0, phb = 0, it = 0;
+      bool ok = true;
+      const uint32_t a_lo0 = smem_desc_lo(a_ring), b_lo0 = smem_desc_lo(b_ring);
+      const uint32_t subt16 = q.subt_bytes >> 4, astage16 = q.a_stage_bytes >> 4, bstage16 = b_stage_bytes >> 4;
+      for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
+        const int rem = w % per_mt;
+        const int ks = rem % q.ksplit;
+        const int kb0 = ks * q.kb_per_split;
+        const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
+        const uint32_t buf = it & 1u;
+        ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t acc = tmem_acc + buf * (uint32_t)BN;
+        uint32_t accumulate = 0;
+        if (q.resident) stb = 0;
+        // the item's units (k2-block, kernel column) in order, bu per filter stage
+        int kb = kb0, v = 0, sub = 0;
+        uint32_t a_tap = 0, a_stage = 0;         // view of the current kernel column inside the activation stage
+        int nks = KB / 16;
+        for (int left = (kb1 - kb0) * q.Kw; left > 0 && ok; left -= q.bu) {
+          const int nu = left < q.bu ? left : q.bu;
+          if (!(q.resident && it > 0)) {         // a resident filter is complete after the first item
+            ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          uint32_t b_lo = b_lo0 + (uint32_t)stb * bstage16;
+          for (int j = 0; j < nu; ++j) {
+            if (v == 0) {
+              ok = mbar_wait(a_full0 + 8 * sta, pha, &abort_flag, q.status);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              a_stage = a_lo0 + (uint32_t)sta * astage16;
+              nks = kb == q.nkb2 - 1 ? q.nks_last : KB / 16;
+            }
+            if (leader) {
+              const uint32_t a_lo = a_stage + a_tap;
+#pragma unroll
+              for (int t = 0; t < KB / 16; ++t) {
+                if (t < nks) {
+                  if (PAIR) umma_f16_ab_pair(acc, a_lo + 2 * t, kSmemDescHiSw128, b_lo + 2 * t, kSmemDescHiSw128, idesc, accumulate);
+                  else umma_f16_lohi(acc, a_lo + 2 * t, b_lo + 2 * t, idesc, accumulate);
+                  accumulate = 1u;
+                }
+              }
+            }
+            b_lo += B_BYTES >> 4;
+            // next kernel column: sub-tile v mod s, view starting v div s rows further down
+            ++v;
+            if (++sub == q.s) { sub = 0; a_tap += (KB * 2 >> 4) - (uint32_t)(q.s - 1) * subt16; }
+            else a_tap += subt16;
+            if (v == q.Kw) {
+              v = 0; sub = 0; a_tap = 0; ++kb;
+              if (leader) {
+                if (PAIR) umma_commit_pair(a_empty0 + 8 * sta);
+                else umma_commit(a_empty0 + 8 * sta);
+              }
+              if (++sta == q.sa) { sta = 0; pha ^= 1u; }
+            }
+          }
+          if (!ok) break;
+          if (leader && !q.resident) {
+            if (PAIR) umma_commit_pair(b_empty0 + 8 * stb);
+            else umma_commit(b_empty0 + 8 * stb);
+          }
+          __syncwarp();
+          if (++stb == q.sb) { stb = 0; phb ^= 1u; }
+        }
+        if (ok && leader) {
+          if (PAIR) umma_commit_pair(acc_full0 + 8 * buf);
+          else umma_commit(acc_full0 + 8 * buf);
+        }
+        __syncwarp();
+      }
+    }
+  } else if (warp >= WARP_EPI0 && warp < WARP_EPI0 + EPI_WARPS) {
+    // ---------------- epilogue ----------------------------------------------------------
+    const int lq = warp & 3;
+    const EpiParams& e = q.e;
+    const bool vec_ok = e.out16 ? (e.Co % 8 == 0) : (e.Co % 4 == 0);
+    wait_for_previous_kernel();
+    bool ok = true;
+    uint32_t it = 0;
+    for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
+      const uint32_t buf = it & 1u;
+      const int mt = w / per_mt, rem = w - mt * per_mt;
+      const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
+      const int n0 = nt * BN;
+      // accumulator row = virtual position vq = strip*Wq + i; columns i >= Wo of a strip are no output
+      const int64_t vq = (int64_t)(PAIR ? 2 * mt + (int)rank : mt) * TILE_M + lq * 32 + lane;
+      bool valid = false;
+      int64_t base = 0, cs = 1;
+      if (vq < q.VQ) {
+        const int strip = (int)(vq / q.Wq), i = (int)(vq - (int64_t)strip * q.Wq);
+        valid = i < e.Wo;
+        if (e.y_nhwc) {
+          base = ((int64_t)strip * e.Wo + i) * e.Co + n0;
+        } else {
+          const int n = strip / e.Ho, ho = strip - n * e.Ho;
+          cs = e.HoWo;
+          base = ((int64_t)n * e.Co + n0) * e.HoWo + ho * e.Wo + i;
+        }
+      }
+      if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
+      ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+      __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
+      drain_accumulator<BN>(e, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_cluster(acc_empty_dst + 8 * buf);
+        else mbar_arrive(acc_empty0 + 8 * buf);
+      }
+    }
+  }
+
+  // ---------------- teardown ---------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);     // copies in flight land before the CTA leaves
+    __syncthreads();
+  }
+  if (PAIR) cluster_sync_all();
+  if (warp == WARP_MMA) {
+    __syncwarp();
+    tc_fence_after();
+    if (PAIR) tmem_dealloc_pair(tmem_acc, 2 * BN);
+    else tmem_dealloc(tmem_acc, 2 * BN);
+  }
+}
+
+template <int BN>
+__global__ void __launch_bounds__(SHIFT_THREADS, 1)
+conv_f16_nhwc_shift_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap, ShiftViewParams q) {
+  conv_shift_body<BN, false>(amap, bmap, q);
+}
+
+template <int BN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(SHIFT_THREADS, 1)
+conv_f16_nhwc_shift_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
+                                ShiftViewParams q) {
+  conv_shift_body<BN, true>(amap, bmap, q);
 }
 
 // Filter pack (paper Section "Im2win Convolution": height before width; here with the channel below
@@ -566,6 +941,12 @@ transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __rest
 }
 
 // ------------------------------------------------------------------- host side
+// Testing aid: with IM2WIN_DEBUG and IM2WIN_VERBOSE set, a failed host-side step says what failed.
+cudaError_t report(cudaError_t e, const char* what) {
+  if (e != cudaSuccess && debug_getenv("IM2WIN_VERBOSE")) fprintf(stderr, "im2win nhwc: %s: %s\n", what, cudaGetErrorString(e));
+  return e;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -666,6 +1047,172 @@ cudaError_t launch_ksub(const CUtensorMap& amap, const CUtensorMap& bmap, const 
   if (plan.bn == 64) return launch_variant<64, false, KSUB>(amap, bmap, q, plan, stream);
   if (plan.bn == 128) return launch_variant<128, false, KSUB>(amap, bmap, q, plan, stream);
   return launch_variant<256, false, KSUB>(amap, bmap, q, plan, stream);
+}
+
+// Geometry of the shifted-view kernel for a layer (host side).
+struct ShiftViewPlan {
+  bool eligible;
+  int32_t Wq, rows, nkb2, nks_last, bu;
+  uint32_t subt_bytes, a_stage_bytes;
+  int64_t VQ, K2;
+  double m_eff;              // useful fraction of the MMA rows
+};
+
+ShiftViewPlan plan_shift_view(const Geometry& g, const NhwcPlan& plan) {
+  ShiftViewPlan p{};
+  p.eligible = false;
+  if (g.Kw < 2 || g.Wp % g.s != 0 || g.s > 16) return p;
+  p.Wq = g.Wp / g.s;
+  p.VQ = (int64_t)g.N * g.Ho * p.Wq;
+  if (p.VQ >= ((int64_t)1 << 31) - 4 * TILE_M) return p;
+  p.rows = TILE_M + (g.Kw - 1) / g.s;
+  if (p.rows > 256) return p;
+  p.subt_bytes = (uint32_t)((p.rows * KB * 2 + 1023) / 1024 * 1024);
+  p.a_stage_bytes = (uint32_t)g.s * p.subt_bytes;
+  p.K2 = (int64_t)g.Kh * plan.Cp;
+  p.nkb2 = (int32_t)((p.K2 + KB - 1) / KB);
+  p.nks_last = (int32_t)((p.K2 - (int64_t)(p.nkb2 - 1) * KB + 15) / 16);
+  p.bu = g.Kw % 3 == 0 ? 3 : 2;
+  if (2 * (int64_t)p.a_stage_bytes + 2 * (int64_t)p.bu * 256 * KB * 2 / 2 > kSmemMax - 2048) return p;
+  p.m_eff = (double)g.Wo / p.Wq;
+  p.eligible = true;
+  return p;
+}
+
+template <int BN, bool PAIR>
+cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bmap, ShiftViewParams q, const NhwcPlan& plan,
+                                 const ShiftViewPlan& sp, cudaStream_t stream) {
+  constexpr int B_ROWS = PAIR ? BN / 2 : BN;
+  constexpr int B_BYTES = B_ROWS * KB * 2;
+  const int budget = kSmemMax - 2048;
+  // units per filter stage: as planned, fewer when two activation stages and three filter stages
+  // of that size do not fit (wide tiles without pairing)
+  while (q.bu > 1 && 2 * (int64_t)sp.a_stage_bytes + 3 * (int64_t)q.bu * B_BYTES > budget) --q.bu;
+  const int b_stage = q.bu * B_BYTES;
+  // K split: whole k2-blocks
+  q.kb_per_split = (sp.nkb2 + q.ksplit - 1) / q.ksplit;
+  q.ksplit = (sp.nkb2 + q.kb_per_split - 1) / q.kb_per_split;
+  const int64_t ntm = (sp.VQ + TILE_M - 1) / TILE_M;
+  const int64_t ntm_eff = PAIR ? (ntm + 1) / 2 : ntm;
+  const int64_t nwork = ntm_eff * q.ntn * q.ksplit;
+  if (nwork >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
+  q.nwork = (int32_t)nwork;
+  // rings: the whole filter resident when the layer has one channel tile and it fits beside two
+  // activation stages; otherwise two or three activation stages and the rest for filter stages
+  const int groups = (sp.nkb2 * q.Kw + q.bu - 1) / q.bu;
+  q.resident = 0;
+  if (q.ntn == 1 && q.ksplit == 1 && groups <= MAX_SB &&
+      (int64_t)groups * b_stage + 2 * (int64_t)sp.a_stage_bytes <= budget) {
+    q.resident = 1;
+    q.sb = groups;
+    q.sa = (int)((budget - (int64_t)groups * b_stage) / sp.a_stage_bytes);
+    if (q.sa > MAX_SA) q.sa = MAX_SA;
+  } else {
+    q.sa = sp.a_stage_bytes <= 20 * 1024 ? 3 : 2;
+    q.sb = (int)((budget - (int64_t)q.sa * sp.a_stage_bytes) / b_stage);
+    if (q.sb > MAX_SB) q.sb = MAX_SB;
+    if (q.sb < 2) { q.sa = 2; q.sb = (int)((budget - 2 * (int64_t)sp.a_stage_bytes) / b_stage); }
+    if (q.sb < 2) return report(cudaErrorInvalidValue, "rings do not fit (shifted view)");
+  }
+  const int smem_bytes = q.sa * (int)sp.a_stage_bytes + q.sb * b_stage + 1024;
+  const int slots = PAIR ? 74 : 148;
+  static int cached_clusters[64] = {};
+  static int attr_bytes[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(SHIFT_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  if (PAIR) {
+    if (attr_bytes[dev] < smem_bytes) {
+      cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
+      if (e != cudaSuccess) return report(e, "shared-memory opt-in (shifted view, pairs)");
+      attr_bytes[dev] = kSmemMax - 1024;
+    }
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    int clusters = cached_clusters[dev];
+    if (clusters == 0) {
+      cudaLaunchConfig_t probe = cfg;
+      probe.gridDim = dim3(148, 1, 1);
+      probe.dynamicSmemBytes = (size_t)(kSmemMax - 1024);   // the worst case: one CTA per SM either way
+      probe.numAttrs = 1;
+      cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_nhwc_shift_pair_kernel<BN>, &probe);
+      if (e != cudaSuccess) return e;
+      if (clusters < 1) return cudaErrorInvalidValue;
+      cached_clusters[dev] = clusters;
+    }
+    if (clusters > slots) clusters = slots;
+    if (clusters > q.nwork) clusters = q.nwork;
+    cfg.gridDim = dim3(2 * clusters, 1, 1);
+    cfg.numAttrs = 2;
+    return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_pair_kernel<BN>, amap, bmap, q), "pair launch (shifted view)");
+  }
+  if (attr_bytes[dev] < smem_bytes) {
+    cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
+    if (e != cudaSuccess) return report(e, "shared-memory opt-in (shifted view)");
+    attr_bytes[dev] = kSmemMax - 1024;
+  }
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)(slots < q.nwork ? slots : q.nwork), 1, 1);
+  return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_kernel<BN>, amap, bmap, q), "launch (shifted view)");
+}
+
+cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* y, uint32_t* status, const Geometry& g,
+                              const NhwcPlan& plan, const ShiftViewPlan& sp, const EpilogueArgs& epi, bool split,
+                              EncodeTiledFn encode, cudaStream_t stream) {
+  // Activation operand: (k2, column class t, virtual position q): column k = q*s + t of the flat
+  // sequence of all strips' columns; filter: (k2, kernel column v, output channel).  Out-of-range
+  // coordinates read as zeros.
+  CUtensorMap amap, bmap;
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)sp.K2, (cuuint64_t)g.s, (cuuint64_t)sp.VQ};
+    const cuuint64_t strides[2] = {(cuuint64_t)sp.K2 * 2, (cuuint64_t)g.s * sp.K2 * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)KB, 1, (cuuint32_t)sp.rows};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult cr = encode(&amap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<uint16_t*>(window), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return report(cudaErrorInvalidValue, "activation tensor map (shifted view)");
+  }
+  const int b_rows = plan.pair ? plan.bn / 2 : plan.bn;
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)sp.K2, (cuuint64_t)g.Kw, (cuuint64_t)g.Co};
+    const cuuint64_t strides[2] = {(cuuint64_t)sp.K2 * 2, (cuuint64_t)g.Kw * sp.K2 * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)KB, 1, (cuuint32_t)b_rows};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult cr = encode(&bmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<uint16_t*>(fp), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return report(cudaErrorInvalidValue, "filter tensor map (shifted view)");
+  }
+  ShiftViewParams q{};
+  q.e.y = y; q.e.bias = epi.bias;
+  q.e.relu = epi.relu; q.e.out16 = epi.out16; q.e.y_nhwc = epi.y_nhwc; q.e.atomic = split ? 1 : 0;
+  q.e.Ho = g.Ho; q.e.Wo = g.Wo; q.e.Co = g.Co; q.e.HoWo = g.Ho * g.Wo;
+  q.e.rows_total = g.N * g.Ho;
+  q.status = status;
+  q.VQ = sp.VQ; q.Wq = sp.Wq; q.s = g.s; q.Kw = g.Kw;
+  q.rows = sp.rows; q.subt_bytes = sp.subt_bytes; q.a_stage_bytes = sp.a_stage_bytes;
+  q.nkb2 = sp.nkb2; q.nks_last = sp.nks_last; q.bu = sp.bu;
+  q.ksplit = split ? plan.ksplit : 1;
+  q.ntn = plan.ntn;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_BU")) { const int bu = atoi(v); if (bu >= 1 && bu <= 8) q.bu = bu; }
+  if (plan.pair) {
+    if (plan.bn == 256) return launch_shift_variant<256, true>(amap, bmap, q, plan, sp, stream);
+    return launch_shift_variant<128, true>(amap, bmap, q, plan, sp, stream);
+  }
+  if (plan.bn == 64) return launch_shift_variant<64, false>(amap, bmap, q, plan, sp, stream);
+  if (plan.bn == 128) return launch_shift_variant<128, false>(amap, bmap, q, plan, sp, stream);
+  return launch_shift_variant<256, false>(amap, bmap, q, plan, sp, stream);
 }
 
 }  // namespace
@@ -810,6 +1357,22 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   }
   const bool split = plan.ksplit > 1 && !epi.relu && !epi.out16;   // partial sums cannot pass a ReLU or a rounding
   if (!split) plan.ksplit = 1;
+  if (split) {
+    cudaError_t e = cudaMemsetAsync(y, 0, (size_t)g.out_elems * 4, stream);
+    if (e != cudaSuccess) return e;
+  }
+  // Which kernel: the shifted-view kernel moves 1/Kw..s/Kw of the activation bytes into the SM but
+  // computes Wq rows per strip for Wo outputs; the overlapping-row kernel computes whole strips
+  // (G*bw of 128 rows).  The shifted view is taken unless it wastes clearly more rows.
+  const ShiftViewPlan sp = plan_shift_view(g, plan);
+  const double m_eff_overlap = (double)plan.G * plan.bw / TILE_M;
+  bool use_shift = sp.eligible && sp.m_eff >= m_eff_overlap - 0.06;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_KERNEL")) {
+    if (strcmp(v, "shift") == 0) use_shift = sp.eligible;
+    else if (strcmp(v, "overlap") == 0) use_shift = false;
+  }
+  if (use_shift)
+    return launch_shift_view(window, fp, y, reinterpret_cast<uint32_t*>(base), g, plan, sp, epi, split, encode, stream);
 
   // Activation operand: (k, wo, strip) with OVERLAPPING rows: the row of output column wo starts
   // s*Kh*Cp halves after that of wo-1.  k beyond K, columns beyond Wo and strips beyond N*Ho read
@@ -838,21 +1401,17 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   }
 
   NhwcParams q{};
-  q.y = y;
-  q.bias = epi.bias;
+  q.e.y = y;
+  q.e.bias = epi.bias;
   q.status = reinterpret_cast<uint32_t*>(base);
-  q.relu = epi.relu; q.out16 = epi.out16; q.y_nhwc = epi.y_nhwc; q.atomic = split ? 1 : 0;
-  q.Ho = g.Ho; q.Wo = g.Wo; q.Co = g.Co; q.HoWo = g.Ho * g.Wo;
-  q.rows_total = g.N * g.Ho;
+  q.e.relu = epi.relu; q.e.out16 = epi.out16; q.e.y_nhwc = epi.y_nhwc; q.e.atomic = split ? 1 : 0;
+  q.e.Ho = g.Ho; q.e.Wo = g.Wo; q.e.Co = g.Co; q.e.HoWo = g.Ho * g.Wo;
+  q.e.rows_total = g.N * g.Ho;
   q.bw = plan.bw; q.G = plan.G; q.tw = plan.tw;
   q.ksplit = plan.ksplit;
   q.ntn = plan.ntn;
   q.a_bytes = (uint32_t)(plan.G * plan.bw * KB * 2);
-  if (split) {
-    cudaError_t e = cudaMemsetAsync(y, 0, (size_t)g.out_elems * 4, stream);
-    if (e != cudaSuccess) return e;
-  }
-  if (const char* v = debug_getenv("IM2WIN_NHWC_SKIP")) q.dbg_skip = atoi(v);
+  if (const char* v = debug_getenv("IM2WIN_NHWC_WW")) q.ww = atoi(v);
   int ksub = 2;
   if (const char* v = debug_getenv("IM2WIN_NHWC_KSUB")) ksub = atoi(v) == 1 ? 1 : 2;
   if (ksub == 1) return launch_ksub<1>(amap, bmap, q, plan, stream);

@@ -72,9 +72,12 @@ def _reference(x, f, dims, bias=None, relu=False, out16=False, y_nhwc=False):
 
 
 @pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
-@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
-def test_conv_nhwc_parity_small(layer, layout):
-    """Plain epilogue (fp32, NCHW out) from either input layout."""
+@pytest.mark.parametrize("layout,kernel", [("nchw", "overlap"), ("nhwc", "shift"), ("nchw", "default")])
+def test_conv_nhwc_parity_small(layer, layout, kernel, monkeypatch):
+    """Plain epilogue (fp32, NCHW out) from either input layout, through either kernel and the one
+    the library picks."""
+    if kernel != "default":
+        monkeypatch.setenv("IM2WIN_NHWC_KERNEL", kernel)
     dims = layer.dims()
     x, f = workloads.make_inputs(layer)
     y = gpu_conv_nhwc(x, f, dims, x_layout=layout)
@@ -82,12 +85,17 @@ def test_conv_nhwc_parity_small(layer, layout):
     check_conv(y, y_pre, a, "f16", layer.name)
 
 
-@pytest.mark.parametrize("layer", [SMALL[0], SMALL[2], SMALL[3], SMALL[7], SMALL[11], SMALL[14]], ids=lambda l: l.name)
+@pytest.mark.parametrize("layer", [SMALL[0], SMALL[2], SMALL[3], SMALL[4], SMALL[6], SMALL[7], SMALL[9], SMALL[11],
+                                   SMALL[12], SMALL[14], SMALL[15]], ids=lambda l: l.name)
+@pytest.mark.parametrize("kernel", ["overlap", "shift"])
 @pytest.mark.parametrize("bn,pair,ksplit", [("64", "0", "1"), ("128", "0", "1"), ("128", "1", "1"), ("256", "0", "1"),
                                             ("256", "1", "1"), ("128", "0", "3"), ("256", "1", "2"), ("64", "0", "20")])
-def test_conv_nhwc_exact_on_integer_inputs_every_tile_shape(layer, bn, pair, ksplit, monkeypatch):
-    """Integer-valued inputs (order-independent sums) through every tile width, with and without CTA
-    pairs, with K split over several CTAs (partial sums added with red.global.add.f32)."""
+def test_conv_nhwc_exact_on_integer_inputs_every_tile_shape(layer, kernel, bn, pair, ksplit, monkeypatch):
+    """Integer-valued inputs (order-independent sums) through both kernels (overlapping-row copies
+    and shifted views; a layer the shifted-view kernel cannot take runs the other one), every tile
+    width, with and without CTA pairs, with K split over several CTAs (partial sums added with
+    red.global.add.f32)."""
+    monkeypatch.setenv("IM2WIN_NHWC_KERNEL", kernel)
     monkeypatch.setenv("IM2WIN_NHWC_BN", bn)
     monkeypatch.setenv("IM2WIN_NHWC_PAIR", pair)
     monkeypatch.setenv("IM2WIN_NHWC_KSPLIT", ksplit)
@@ -103,7 +111,8 @@ def test_conv_nhwc_exact_on_integer_inputs_every_tile_shape(layer, bn, pair, ksp
 @pytest.mark.parametrize("out16", [False, True])
 @pytest.mark.parametrize("y_nhwc", [False, True])
 @pytest.mark.parametrize("bias,relu", [(False, False), (True, False), (False, True), (True, True)])
-def test_conv_nhwc_epilogue_options(layer, out16, y_nhwc, bias, relu):
+def test_conv_nhwc_epilogue_options(layer, out16, y_nhwc, bias, relu, monkeypatch):
+    monkeypatch.setenv("IM2WIN_NHWC_KERNEL", "shift" if (bias != relu) else "overlap")
     dims = layer.dims()
     x, f = workloads.make_inputs(layer)
     b = None
@@ -175,3 +184,24 @@ def test_nhwc_full_size_whole_tensors(layer):
         n1 = min(layer.N, n0 + 16)
         yi, ai = oracle.conv_im2win(xo[n0:n1], fo, dict(dims, N=n1 - n0))
         check_conv(y[n0:n1], yi, ai, "f16", f"{layer.name} images {n0}..{n1 - 1}")
+
+
+@pytest.mark.parametrize("name,kernel", [("cfg2", "overlap"), ("cfg4a", "shift"), ("cfg4b", "shift"), ("cfg4c", "shift"),
+                                         ("cfg4c", "overlap"), ("cfg5k3", "overlap"), ("cfg5k3", "shift"), ("cfg5k5", "shift")])
+def test_nhwc_full_size_forced_kernel_sampled(name, kernel, monkeypatch):
+    """Both kernels at benchmark size wherever the library would pick the other one: 16 384 sampled
+    outputs from Eq. 1 and two whole images."""
+    monkeypatch.setenv("IM2WIN_NHWC_KERNEL", kernel)
+    layer = workloads.LAYERS[name]
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    ho, wo = oracle.out_dims(dims)
+    y = gpu_conv_nhwc(x, f, dims)
+    xo, fo = oracle_inputs(x, f, "f16")
+    total = layer.N * layer.Co * ho * wo
+    idx = np.concatenate([np.random.default_rng(layer.seed + 1).integers(0, total, 16384), [0, total - 1]])
+    yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
+    check_conv(y.reshape(-1)[idx], yr, ar, "f16", f"{name} {kernel}")
+    for n in (0, layer.N - 1):
+        yi, ai = oracle.conv_im2win(xo[n:n + 1], fo, dict(dims, N=1))
+        check_conv(y[n:n + 1], yi, ai, "f16", f"{name} {kernel} image {n}")
