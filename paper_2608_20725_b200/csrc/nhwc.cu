@@ -63,7 +63,6 @@ struct NhwcParams {
   int32_t ntn, nwork;        // channel tiles; work items = position tiles (pairs) x channel tiles x k parts
   int32_t stages;
   uint32_t a_bytes;          // bytes one activation copy brings: G*bw*128
-  int32_t ww;
 };
 
 // Programmatic dependent launch: the convolution may start while the kernel before it in the stream
@@ -213,13 +212,12 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
 
   if (warp == WARP_TMA) {
     // ---------------- copies of both operands ------------------------------------
-    // Lane 0 polls and issues; the warp meets again after the loop.
-    if (lane == 0) {
+    {
+      const bool leader = elect_one();
       wait_for_previous_kernel();                // the filter pack (and everything before it) is complete
       int st = 0;
       uint32_t ph = 0;
       bool ok = true;
-      TIMER_DECL;
       for (int w = w_first; w < q.nwork && ok; w += w_step) {
         const int mt = w / per_mt, rem = w - mt * per_mt;
         const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
@@ -230,40 +228,40 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
         const int kc0 = ks * q.kc_per_split;
         const int kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
         for (int kc = kc0; kc < kc1; ++kc) {
-          TIMER_LAP(0);                              // copy thread: issuing
           ok = mbar_wait(empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          TIMER_LAP(1);                              // copy thread: wait for a free stage
-          const uint32_t dst = ring + (uint32_t)st * STAGE_BYTES;
-          const uint32_t bar = full_dst + 8 * st;
-          // k-blocks beyond K read as zeros (and cost no memory traffic), so every stage brings the
-          // same number of bytes.  In a pair the leader CTA announces the bytes of both CTAs.
-          if (!PAIR || rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, (PAIR ? 2u : 1u) * KSUB * (q.a_bytes + B_BYTES));
+          if (leader) {
+            const uint32_t dst = ring + (uint32_t)st * STAGE_BYTES;
+            const uint32_t bar = full_dst + 8 * st;
+            // k-blocks beyond K read as zeros (and cost no memory traffic), so every stage brings the
+            // same number of bytes.  In a pair the leader CTA announces the bytes of both CTAs.
+            if (!PAIR || rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, (PAIR ? 2u : 1u) * KSUB * (q.a_bytes + B_BYTES));
 #pragma unroll
-          for (int sub = 0; sub < KSUB; ++sub) {
-            const int kx = (kc * KSUB + sub) * KB;
-            if (PAIR) {
-              tma_load_3d_pair(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
-              tma_load_2d_pair(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
-            } else {
-              tma_load_3d(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
-              tma_load_2d(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
+            for (int sub = 0; sub < KSUB; ++sub) {
+              const int kx = (kc * KSUB + sub) * KB;
+              if (PAIR) {
+                tma_load_3d_pair(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
+                tma_load_2d_pair(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
+              } else {
+                tma_load_3d(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
+                tma_load_2d(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
+              }
             }
           }
+          __syncwarp();
           if (++st == q.stages) { st = 0; ph ^= 1u; }
         }
       }
-      if (blockIdx.x == 0) { TIMER_LAP(0); TIMER_FLUSH(); }
     }
-    __syncwarp();
   } else if (warp == WARP_MMA && rank == 0) {
     // ---------------- MMA issuer (leader CTA of a pair) -----------------------------
-    // One thread runs the whole loop: waits, MMAs and commits are all single-thread operations.
     // Every byte the MMAs read was written by the copy engine, whose completion the barrier's
     // transaction count tracks, so CTA-scope waits suffice also for the peer's half.
     constexpr uint32_t idesc = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN);
-    if (q.ww) {
-      // experiment: the whole warp walks the loop, one elected lane issues
+    {
+      // the whole warp walks the loop and takes the waits, one elected lane issues (measured faster
+      // than a lone lane, whose satisfied waits cost more)
       const bool leader = elect_one();
       int st = 0;
       uint32_t ph = 0, it = 0;
@@ -310,61 +308,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
         }
         __syncwarp();
       }
-    } else if (lane == 0) {
-      int st = 0;
-      uint32_t ph = 0, it = 0;
-      bool ok = true;
-      const uint32_t a_lo0 = smem_desc_lo(ring), b_lo0 = smem_desc_lo(ring + (uint32_t)A_SLOT_BYTES);
-      TIMER_DECL;
-      for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
-        const int rem = w % per_mt;
-        const int ks = rem % q.ksplit;
-        const int kc0 = ks * q.kc_per_split;
-        const int kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
-        const uint32_t buf = it & 1u;
-        TIMER_LAP(2);                                // MMA thread: issue and bookkeeping
-        ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
-        if (!ok) break;
-        TIMER_LAP(3);                                // MMA thread: wait for a free accumulator
-        tc_fence_after();
-        const uint32_t acc = tmem_acc + buf * (uint32_t)BN;
-        uint32_t accumulate = 0;
-        for (int kc = kc0; kc < kc1; ++kc) {
-          TIMER_LAP(2);
-          ok = mbar_wait(full0 + 8 * st, ph, &abort_flag, q.status);
-          if (!ok) break;
-          TIMER_LAP(4);                              // MMA thread: wait for a full stage
-          const uint32_t a_lo = a_lo0 + (uint32_t)st * (STAGE_BYTES >> 4);
-          const uint32_t b_lo = b_lo0 + (uint32_t)st * (STAGE_BYTES >> 4);
-          if (kc != q.num_kc - 1) {
-#pragma unroll
-            for (int j = 0; j < KSUB * (KB / 16); ++j) {
-              const uint32_t off = (uint32_t)(j / 4) * (SUB_BYTES >> 4) + 2u * (uint32_t)(j % 4);
-              if (PAIR) umma_f16_ab_pair(acc, a_lo + off, kSmemDescHiSw128, b_lo + off, kSmemDescHiSw128, idesc, accumulate);
-              else umma_f16_lohi(acc, a_lo + off, b_lo + off, idesc, accumulate);
-              accumulate = 1u;
-            }
-          } else {
-            // the last chunk of K: only the 16-wide steps that hold real k
-            for (int j = 0; j < q.nks_last; ++j) {
-              const uint32_t off = (uint32_t)(j / 4) * (SUB_BYTES >> 4) + 2u * (uint32_t)(j % 4);
-              if (PAIR) umma_f16_ab_pair(acc, a_lo + off, kSmemDescHiSw128, b_lo + off, kSmemDescHiSw128, idesc, accumulate);
-              else umma_f16_lohi(acc, a_lo + off, b_lo + off, idesc, accumulate);
-              accumulate = 1u;
-            }
-          }
-          if (PAIR) umma_commit_pair(empty0 + 8 * st);
-          else umma_commit(empty0 + 8 * st);
-          if (++st == q.stages) { st = 0; ph ^= 1u; }
-        }
-        if (ok) {
-          if (PAIR) umma_commit_pair(acc_full0 + 8 * buf);
-          else umma_commit(acc_full0 + 8 * buf);
-        }
-      }
-      if (blockIdx.x == 0) { TIMER_LAP(2); TIMER_FLUSH(); }
     }
-    __syncwarp();
   } else if (warp >= WARP_EPI0) {
     // ---------------- epilogue: tensor memory -> output -----------------------------
     const int lq = warp & 3;                     // tensor-memory lane quadrant this warp may read
@@ -457,6 +401,7 @@ conv_f16_nhwc_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid
 // kernel column), streamed through their own ring, or resident when the layer's whole filter
 // fits) stay as they were.  Needs s | Wp and Kw >= 2.
 constexpr int MAX_SA = 6, MAX_SB = 12;
+constexpr int MAX_KW = 64;                     // kernel widths the shifted-view kernel takes
 constexpr int WARP_BLOAD = 2 + EPI_WARPS;      // the filter-copy warp of this kernel
 constexpr int SHIFT_THREADS = (NUM_WARPS + 1) * 32;
 
@@ -476,6 +421,7 @@ struct ShiftViewParams {
   int32_t resident;          // 1: the filter ring holds the layer's whole filter, loaded once per CTA
   int32_t ksplit, kb_per_split;
   int32_t ntn, nwork;
+  int32_t bu_forced;         // testing aid: bu was given, do not choose it
 };
 
 template <int BN, bool PAIR>
@@ -491,6 +437,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
   __shared__ __align__(8) uint64_t bars[2 * MAX_SA + 2 * MAX_SB + 4];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile uint32_t abort_flag;
+  __shared__ uint32_t tap16[MAX_KW];           // view of kernel column v inside an activation stage, in 16-byte units
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -506,6 +453,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
 
   if (threadIdx.x == 0) {
     abort_flag = 0u;
+    // kernel column v reads sub-tile v mod s from row v div s on
+    for (int v = 0; v < q.Kw; ++v) tap16[v] = (uint32_t)(v % q.s) * (q.subt_bytes >> 4) + (uint32_t)(v / q.s) * (KB * 2 >> 4);
     for (int i = 0; i < MAX_SA; ++i) { mbar_init(a_full0 + 8 * i, 1); mbar_init(a_empty0 + 8 * i, 1); }
     for (int i = 0; i < MAX_SB; ++i) { mbar_init(b_full0 + 8 * i, 1); mbar_init(b_empty0 + 8 * i, 1); }
     for (int i = 0; i < 2; ++i) {
@@ -537,6 +486,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       int st = 0;
       uint32_t ph = 0;
       bool ok = true;
+      TIMER_DECL;
       for (int w = w_first; w < q.nwork && ok; w += w_step) {
         const int mt = w / per_mt, rem = w - mt * per_mt;
         const int ks = rem % q.ksplit;
@@ -544,9 +494,11 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
         const int kb0 = ks * q.kb_per_split;
         const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
         for (int kb = kb0; kb < kb1; ++kb) {
+          if (lane == 0) TIMER_LAP(0);                   // activation copies: issuing
           ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
+          if (lane == 0) TIMER_LAP(1);                   // activation copies: wait for a free stage
           if (leader) {
             const uint32_t dst = a_ring + (uint32_t)st * q.a_stage_bytes;
             const uint32_t bar = a_full_dst + 8 * st;
@@ -561,6 +513,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
           if (++st == q.sa) { st = 0; ph ^= 1u; }
         }
       }
+      if (lane == 0 && blockIdx.x == 0) { TIMER_LAP(0); TIMER_FLUSH(); }
     }
   } else if (warp == WARP_BLOAD) {
     // ---------------- filter copies: bu (k2-block, kernel column) units per stage ----
@@ -611,41 +564,94 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       bool ok = true;
       const uint32_t a_lo0 = smem_desc_lo(a_ring), b_lo0 = smem_desc_lo(b_ring);
       const uint32_t subt16 = q.subt_bytes >> 4, astage16 = q.a_stage_bytes >> 4, bstage16 = b_stage_bytes >> 4;
+      TIMER_DECL;
       for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
         const int rem = w % per_mt;
         const int ks = rem % q.ksplit;
         const int kb0 = ks * q.kb_per_split;
         const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
         const uint32_t buf = it & 1u;
+        if (lane == 0) TIMER_LAP(2);                     // MMA warp: issue and bookkeeping
         ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
+        if (lane == 0) TIMER_LAP(3);                     // MMA warp: wait for a free accumulator
         tc_fence_after();
         const uint32_t acc = tmem_acc + buf * (uint32_t)BN;
         uint32_t accumulate = 0;
         if (q.resident) stb = 0;
+        if (q.bu == q.Kw) {
+          // one filter stage per k2-block (all its kernel columns): two waits and two commits per block
+          for (int kb = kb0; kb < kb1; ++kb) {
+            if (lane == 0) TIMER_LAP(2);
+            ok = mbar_wait(a_full0 + 8 * sta, pha, &abort_flag, q.status);
+            if (ok && !(q.resident && it > 0)) ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (lane == 0) TIMER_LAP(4);               // MMA warp: wait for the stages
+            if (leader) {
+              const uint32_t a_stage = a_lo0 + (uint32_t)sta * astage16;
+              uint32_t b_lo = b_lo0 + (uint32_t)stb * bstage16;
+              if (kb != q.nkb2 - 1 || q.nks_last == KB / 16) {
+                for (int v = 0; v < q.Kw; ++v) {
+                  const uint32_t a_lo = a_stage + tap16[v];
+#pragma unroll
+                  for (int t = 0; t < KB / 16; ++t) {
+                    if (PAIR) umma_f16_ab_pair(acc, a_lo + 2 * t, kSmemDescHiSw128, b_lo + 2 * t, kSmemDescHiSw128, idesc, accumulate);
+                    else umma_f16_lohi(acc, a_lo + 2 * t, b_lo + 2 * t, idesc, accumulate);
+                    accumulate = 1u;
+                  }
+                  b_lo += B_BYTES >> 4;
+                }
+              } else {
+                for (int v = 0; v < q.Kw; ++v) {
+                  const uint32_t a_lo = a_stage + tap16[v];
+                  for (int t = 0; t < q.nks_last; ++t) {
+                    if (PAIR) umma_f16_ab_pair(acc, a_lo + 2 * t, kSmemDescHiSw128, b_lo + 2 * t, kSmemDescHiSw128, idesc, accumulate);
+                    else umma_f16_lohi(acc, a_lo + 2 * t, b_lo + 2 * t, idesc, accumulate);
+                    accumulate = 1u;
+                  }
+                  b_lo += B_BYTES >> 4;
+                }
+              }
+              if (PAIR) umma_commit_pair(a_empty0 + 8 * sta);
+              else umma_commit(a_empty0 + 8 * sta);
+              if (!q.resident) {
+                if (PAIR) umma_commit_pair(b_empty0 + 8 * stb);
+                else umma_commit(b_empty0 + 8 * stb);
+              }
+            }
+            __syncwarp();
+            if (++sta == q.sa) { sta = 0; pha ^= 1u; }
+            if (++stb == q.sb) { stb = 0; phb ^= 1u; }
+          }
+        } else {
         // the item's units (k2-block, kernel column) in order, bu per filter stage
-        int kb = kb0, v = 0, sub = 0;
-        uint32_t a_tap = 0, a_stage = 0;         // view of the current kernel column inside the activation stage
+        int kb = kb0, v = 0;
+        uint32_t a_stage = 0;
         int nks = KB / 16;
         for (int left = (kb1 - kb0) * q.Kw; left > 0 && ok; left -= q.bu) {
           const int nu = left < q.bu ? left : q.bu;
           if (!(q.resident && it > 0)) {         // a resident filter is complete after the first item
+            if (lane == 0) TIMER_LAP(2);
             ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
+            if (lane == 0) TIMER_LAP(7);                 // MMA warp: wait for a filter stage
           }
           uint32_t b_lo = b_lo0 + (uint32_t)stb * bstage16;
           for (int j = 0; j < nu; ++j) {
             if (v == 0) {
+              if (lane == 0) TIMER_LAP(2);
               ok = mbar_wait(a_full0 + 8 * sta, pha, &abort_flag, q.status);
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) break;
+              if (lane == 0) TIMER_LAP(4);               // MMA warp: wait for an activation stage
               a_stage = a_lo0 + (uint32_t)sta * astage16;
               nks = kb == q.nkb2 - 1 ? q.nks_last : KB / 16;
             }
             if (leader) {
-              const uint32_t a_lo = a_stage + a_tap;
+              const uint32_t a_lo = a_stage + tap16[v];
 #pragma unroll
               for (int t = 0; t < KB / 16; ++t) {
                 if (t < nks) {
@@ -656,12 +662,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
               }
             }
             b_lo += B_BYTES >> 4;
-            // next kernel column: sub-tile v mod s, view starting v div s rows further down
-            ++v;
-            if (++sub == q.s) { sub = 0; a_tap += (KB * 2 >> 4) - (uint32_t)(q.s - 1) * subt16; }
-            else a_tap += subt16;
-            if (v == q.Kw) {
-              v = 0; sub = 0; a_tap = 0; ++kb;
+            if (++v == q.Kw) {
+              v = 0; ++kb;
               if (leader) {
                 if (PAIR) umma_commit_pair(a_empty0 + 8 * sta);
                 else umma_commit(a_empty0 + 8 * sta);
@@ -677,12 +679,14 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
           __syncwarp();
           if (++stb == q.sb) { stb = 0; phb ^= 1u; }
         }
+        }
         if (ok && leader) {
           if (PAIR) umma_commit_pair(acc_full0 + 8 * buf);
           else umma_commit(acc_full0 + 8 * buf);
         }
         __syncwarp();
       }
+      if (lane == 0 && blockIdx.x == 0) { TIMER_LAP(2); TIMER_FLUSH(); }
     }
   } else if (warp >= WARP_EPI0 && warp < WARP_EPI0 + EPI_WARPS) {
     // ---------------- epilogue ----------------------------------------------------------
@@ -692,6 +696,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
     wait_for_previous_kernel();
     bool ok = true;
     uint32_t it = 0;
+    TIMER_DECL;
     for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
       const uint32_t buf = it & 1u;
       const int mt = w / per_mt, rem = w - mt * per_mt;
@@ -712,10 +717,12 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
           base = ((int64_t)n * e.Co + n0) * e.HoWo + ho * e.Wo + i;
         }
       }
+      if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(5);     // epilogue: draining and storing
       if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
       __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
       if (!ok) break;
+      if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(6);     // epilogue: wait for a finished accumulator
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
       drain_accumulator<BN>(e, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
@@ -726,6 +733,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
         else mbar_arrive(acc_empty0 + 8 * buf);
       }
     }
+    if (threadIdx.x == WARP_EPI0 * 32 && blockIdx.x == 0) { TIMER_LAP(5); TIMER_FLUSH(); }
   }
 
   // ---------------- teardown ---------------------------------------------------
@@ -1042,7 +1050,8 @@ cudaError_t launch_ksub(const CUtensorMap& amap, const CUtensorMap& bmap, const 
                         cudaStream_t stream) {
   if (plan.pair) {
     if (plan.bn == 256) return launch_variant<256, true, KSUB>(amap, bmap, q, plan, stream);
-    return launch_variant<128, true, KSUB>(amap, bmap, q, plan, stream);
+    if (plan.bn == 128) return launch_variant<128, true, KSUB>(amap, bmap, q, plan, stream);
+    return launch_variant<64, true, KSUB>(amap, bmap, q, plan, stream);
   }
   if (plan.bn == 64) return launch_variant<64, false, KSUB>(amap, bmap, q, plan, stream);
   if (plan.bn == 128) return launch_variant<128, false, KSUB>(amap, bmap, q, plan, stream);
@@ -1061,7 +1070,7 @@ struct ShiftViewPlan {
 ShiftViewPlan plan_shift_view(const Geometry& g, const NhwcPlan& plan) {
   ShiftViewPlan p{};
   p.eligible = false;
-  if (g.Kw < 2 || g.Wp % g.s != 0 || g.s > 16) return p;
+  if (g.Kw < 2 || g.Kw > MAX_KW || g.Wp % g.s != 0 || g.s > 16) return p;
   p.Wq = g.Wp / g.s;
   p.VQ = (int64_t)g.N * g.Ho * p.Wq;
   if (p.VQ >= ((int64_t)1 << 31) - 4 * TILE_M) return p;
@@ -1085,9 +1094,13 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;
   constexpr int B_BYTES = B_ROWS * KB * 2;
   const int budget = kSmemMax - 2048;
-  // units per filter stage: as planned, fewer when two activation stages and three filter stages
-  // of that size do not fit (wide tiles without pairing)
-  while (q.bu > 1 && 2 * (int64_t)sp.a_stage_bytes + 3 * (int64_t)q.bu * B_BYTES > budget) --q.bu;
+  // units per filter stage: all kernel columns of a k2-block when two such stages fit beside two
+  // activation stages (the MMA warp then pays two waits and two commits per block); otherwise three,
+  // or fewer when three stages of that size do not fit (wide tiles without pairing)
+  const bool whole_blocks = 2 * (int64_t)sp.a_stage_bytes + 2 * (int64_t)q.Kw * B_BYTES <= budget;
+  if (!q.bu_forced) q.bu = whole_blocks ? q.Kw : 3;
+  if (!(whole_blocks && q.bu == q.Kw))
+    while (q.bu > 1 && 2 * (int64_t)sp.a_stage_bytes + 3 * (int64_t)q.bu * B_BYTES > budget) --q.bu;
   const int b_stage = q.bu * B_BYTES;
   // K split: whole k2-blocks
   q.kb_per_split = (sp.nkb2 + q.ksplit - 1) / q.ksplit;
@@ -1205,10 +1218,11 @@ cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* 
   q.nkb2 = sp.nkb2; q.nks_last = sp.nks_last; q.bu = sp.bu;
   q.ksplit = split ? plan.ksplit : 1;
   q.ntn = plan.ntn;
-  if (const char* v = debug_getenv("IM2WIN_NHWC_BU")) { const int bu = atoi(v); if (bu >= 1 && bu <= 8) q.bu = bu; }
+  if (const char* v = debug_getenv("IM2WIN_NHWC_BU")) { const int bu = atoi(v); if (bu >= 1 && bu <= 8) { q.bu = bu; q.bu_forced = 1; } }
   if (plan.pair) {
     if (plan.bn == 256) return launch_shift_variant<256, true>(amap, bmap, q, plan, sp, stream);
-    return launch_shift_variant<128, true>(amap, bmap, q, plan, sp, stream);
+    if (plan.bn == 128) return launch_shift_variant<128, true>(amap, bmap, q, plan, sp, stream);
+    return launch_shift_variant<64, true>(amap, bmap, q, plan, sp, stream);
   }
   if (plan.bn == 64) return launch_shift_variant<64, false>(amap, bmap, q, plan, sp, stream);
   if (plan.bn == 128) return launch_shift_variant<128, false>(amap, bmap, q, plan, sp, stream);
@@ -1240,10 +1254,9 @@ NhwcPlan plan_nhwc(const Geometry& g) {
   if (p.G > 256) p.G = 256;
   const int64_t groups = ((int64_t)g.N * g.Ho + p.G - 1) / p.G;
   p.ntm = groups * p.tw;
-  // channel tile: the narrowest MMA N that covers Co, at most 256; tiles of 256 run as CTA pairs
-  // (each CTA stages half of the filter tile)
+  // channel tile: the narrowest MMA N that covers Co, at most 256; CTA pairs (cta_group::2, M = 256)
   p.bn = g.Co <= 64 ? 64 : (g.Co <= 128 ? 128 : 256);
-  p.pair = p.bn == 256;
+  p.pair = p.ntm >= 2;       // pairs at every width: half the filter bytes per CTA and half the MMA instructions per flop
   p.ntn = (g.Co + p.bn - 1) / p.bn;
   p.ksplit = 1;
   const int64_t ntm_eff = p.pair ? (p.ntm + 1) / 2 : p.ntm;
@@ -1348,9 +1361,9 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   // testing aids (read only when IM2WIN_DEBUG is set): tile width, pairing and K split
   if (const char* v = debug_getenv("IM2WIN_NHWC_BN")) {
     const int bn = atoi(v);
-    if (bn == 64 || bn == 128 || bn == 256) { plan.bn = bn; plan.ntn = (g.Co + bn - 1) / bn; plan.pair = bn == 256; }
+    if (bn == 64 || bn == 128 || bn == 256) { plan.bn = bn; plan.ntn = (g.Co + bn - 1) / bn; }
   }
-  if (const char* v = debug_getenv("IM2WIN_NHWC_PAIR")) plan.pair = v[0] == '1' && plan.bn >= 128;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_PAIR")) plan.pair = v[0] == '1';
   if (const char* v = debug_getenv("IM2WIN_NHWC_KSPLIT")) {
     const int ks = atoi(v);
     if (ks >= 1 && ks <= plan.num_kb) plan.ksplit = ks;
@@ -1361,12 +1374,15 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
     cudaError_t e = cudaMemsetAsync(y, 0, (size_t)g.out_elems * 4, stream);
     if (e != cudaSuccess) return e;
   }
-  // Which kernel: the shifted-view kernel moves 1/Kw..s/Kw of the activation bytes into the SM but
-  // computes Wq rows per strip for Wo outputs; the overlapping-row kernel computes whole strips
-  // (G*bw of 128 rows).  The shifted view is taken unless it wastes clearly more rows.
+  // Which kernel.  The shifted-view kernel brings s/Kw of the activation bytes into the SM but computes
+  // Wq rows per strip for Wo outputs, and it needs one filter stage per k2-block (all kernel columns)
+  // to keep its MMA warp's barrier traffic low.  Measured: it wins where every column is reused by
+  // three kernel columns or more (Kw >= 3s) and two such filter stages fit beside two activation
+  // stages; elsewhere the overlapping-row kernel is as fast or faster.
   const ShiftViewPlan sp = plan_shift_view(g, plan);
-  const double m_eff_overlap = (double)plan.G * plan.bw / TILE_M;
-  bool use_shift = sp.eligible && sp.m_eff >= m_eff_overlap - 0.06;
+  const int64_t b_bytes = (int64_t)(plan.pair ? plan.bn / 2 : plan.bn) * KB * 2;
+  bool use_shift = sp.eligible && g.Kw >= 3 * g.s &&
+                   2 * (int64_t)sp.a_stage_bytes + 2 * (int64_t)g.Kw * b_bytes <= kSmemMax - 2048;
   if (const char* v = debug_getenv("IM2WIN_NHWC_KERNEL")) {
     if (strcmp(v, "shift") == 0) use_shift = sp.eligible;
     else if (strcmp(v, "overlap") == 0) use_shift = false;
@@ -1411,8 +1427,7 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   q.ksplit = plan.ksplit;
   q.ntn = plan.ntn;
   q.a_bytes = (uint32_t)(plan.G * plan.bw * KB * 2);
-  if (const char* v = debug_getenv("IM2WIN_NHWC_WW")) q.ww = atoi(v);
-  int ksub = 2;
+  int ksub = 1;
   if (const char* v = debug_getenv("IM2WIN_NHWC_KSUB")) ksub = atoi(v) == 1 ? 1 : 2;
   if (ksub == 1) return launch_ksub<1>(amap, bmap, q, plan, stream);
   return launch_ksub<2>(amap, bmap, q, plan, stream);
