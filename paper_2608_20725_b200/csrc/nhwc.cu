@@ -818,6 +818,12 @@ pack_f16_nhwc_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, 
 }
 
 // ---------------------------------------------------------------- transform ----
+template <int VEC> struct VecType;
+template <> struct VecType<8> { typedef uint4 type; };
+template <> struct VecType<4> { typedef uint2 type; };
+template <> struct VecType<2> { typedef uint32_t type; };
+template <> struct VecType<1> { typedef uint16_t type; };
+
 // x given NHWC: every (n, ho, k, u) of the window tensor is the channel vector of one input pixel
 // (or zeros in the padding): 16-byte chunks, one per thread, consecutive threads along (k, u, c).
 __global__ void transform_nhwc_from_nhwc_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ win, int C, int Cp,
@@ -849,101 +855,97 @@ __global__ void transform_nhwc_from_nhwc_kernel(const uint16_t* __restrict__ x, 
   }
 }
 
-// x given NCHW: a transposition.  One block builds the part of one strip (n, ho) that covers `kc`
-// columns: phase 1 reads the Kh input rows of every channel along w (coalesced) and stores them in
-// shared memory as [k][u][c] (pitch Cp + 2 halves = an odd number of words); phase 2 walks the
-// strip's 16-byte chunks in output order (c fastest, then u, then k), reads each from shared memory
-// as four words and writes it with one coalesced 16-byte store.  Indices are kept in mixed-radix
-// counters (no division per element); what depends on (u, c) alone is tabulated once per block.
+// x given NCHW: a transposition.  One block takes one row h of the padded input of one image (all
+// channels, a chunk of columns when the row is long): phase 1 reads it along w (coalesced) and
+// stores it in shared memory as T[w][c] (pitch Cp + 2 halves = an odd number of words:
+// conflict-free); phase 2 writes T to every place of the window tensor that holds this input row,
+// i.e. once per (ho, u) with ho*s + u = h + p (Kh/s places): 16-byte chunks in output order (c
+// fastest), so consecutive threads write consecutive bytes of a column.  Every input element is
+// read once and transposed once; blocks of rows outside the image only write zeros.  Indices are
+// kept in mixed-radix counters (no division per element).
 template <bool VEC2>
 __global__ void __launch_bounds__(256)
 transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ win, int C, int Cp, int H, int W,
                                 int Ho, int Wp, int Kh, int s, int p, int kc, int kchunks) {
-  extern __shared__ __align__(16) uint16_t rows_s[];     // [kc][Kh][Cp + 2], then two int tables of Kh*C entries
+  extern __shared__ __align__(16) uint16_t rows_s[];     // T[kc][Cp + 2]
   const int PC = Cp + 2;
-  int* rowsrc = reinterpret_cast<int*>(rows_s + (size_t)kc * Kh * PC);   // (c*H + h)*W of row (u, c), -1 outside the image
-  int* rowdst = rowsrc + Kh * C;                                         // u*PC + c
   int64_t b = blockIdx.x;
   const int kci = (int)(b % kchunks); b /= kchunks;
-  const int ho = (int)(b % Ho);
-  const int64_t n = b / Ho;
-  const int k0 = kci * kc;
-  const int nk = Wp - k0 < kc ? Wp - k0 : kc;             // columns of this block
-  // input columns that exist among k0 .. k0 + nk - 1 (k = w + p)
-  const int w_lo = k0 - p > 0 ? k0 - p : 0;
-  const int w_hi = k0 + nk - p < W ? k0 + nk - p : W;     // exclusive
-  const int nw = w_hi > w_lo ? w_hi - w_lo : 0;
-  const int nrows = Kh * C;
-  for (int r = threadIdx.x; r < nrows; r += blockDim.x) {
-    const int u = r / C, c = r - u * C;
-    const int h = ho * s + u - p;
-    rowsrc[r] = (h >= 0 && h < H) ? (c * H + h) * W : -1;
-    rowdst[r] = u * PC + c;
-  }
-  if (Cp > C) {                                           // the zero channels C .. Cp-1
-    const int extra = Cp - C;
-    for (int i = threadIdx.x; i < kc * Kh * extra; i += blockDim.x) {
-      const int r = i / extra, e = i - r * extra;
-      rows_s[r * PC + C + e] = 0;
+  const int hp = (int)(b % (H + 2 * p));                  // row of the padded input
+  const int64_t n = b / (H + 2 * p);
+  const int h = hp - p;
+  const bool row_ok = h >= 0 && h < H;
+  // the strips that hold this row: ho*s + u = hp with 0 <= u < Kh
+  const int ho_hi = hp / s < Ho - 1 ? hp / s : Ho - 1;
+  int ho_lo = hp - Kh + 1 > 0 ? (hp - Kh + 1 + s - 1) / s : 0;
+  if (ho_lo > ho_hi) return;                              // a row no window reaches
+  const int w0 = kci * kc;
+  const int nw = W - w0 < kc ? W - w0 : kc;               // input columns of this block
+  // its columns of the window tensor: k = w + p, plus the left padding for the first chunk and the
+  // right padding for the last
+  const int k_lo = kci == 0 ? 0 : w0 + p;
+  const int k_hi = kci == kchunks - 1 ? Wp : w0 + nw + p; // exclusive
+  if (row_ok) {
+    if (Cp > C) {                                         // the zero channels C .. Cp-1
+      const int extra = Cp - C;
+      for (int i = threadIdx.x; i < nw * extra; i += blockDim.x) {
+        const int r = i / extra, e = i - r * extra;
+        rows_s[r * PC + C + e] = 0;
+      }
     }
-  }
-  __syncthreads();
-  const uint16_t* ximg = x + n * ((int64_t)C * H * W);
-  // phase 1: item -> (row = (u, c), column (pair)), columns fastest; 8 loads in flight per thread
-  {
-    constexpr int E = VEC2 ? 2 : 1;                       // columns per item (VEC2: W, w_lo and nw are even)
+    // phase 1: item -> (c, column (pair)), columns fastest; 8 loads in flight per thread
+    constexpr int E = VEC2 ? 2 : 1;                       // columns per item (VEC2: W, w0 and nw are even)
     const int nwi = nw / E;
-    const int items = nrows * nwi;
+    const int items = C * nwi;
     const int step = (int)blockDim.x;
-    const int d_row = nwi > 0 ? step / nwi : 0, d_col = nwi > 0 ? step - d_row * nwi : 0;
-    int row = nwi > 0 ? (int)threadIdx.x / nwi : 0, col = nwi > 0 ? (int)threadIdx.x - row * nwi : 0;
+    const int d_c = step / nwi, d_col = step - d_c * nwi;
+    int c = (int)threadIdx.x / nwi, col = (int)threadIdx.x - c * nwi;
+    const uint16_t* xrow = x + ((n * C) * H + h) * (int64_t)W + w0;      // channel c: + c*H*W
+    const int64_t cstride = (int64_t)H * W;
     for (int i0 = threadIdx.x; i0 < items; i0 += 8 * step) {
       uint32_t r[8];
       int dsts[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        r[j] = 0u;
         dsts[j] = -1;
         if (i0 + j * step < items) {
-          const int src = rowsrc[row];
-          const int wcol = w_lo + E * col;
-          dsts[j] = ((wcol + p - k0) * Kh) * PC + rowdst[row];
-          if (src >= 0) {
-            if (VEC2) r[j] = __ldg(reinterpret_cast<const uint32_t*>(ximg + src + wcol));
-            else r[j] = __ldg(ximg + src + wcol);
-          }
+          dsts[j] = (E * col) * PC + c;
+          if (VEC2) r[j] = __ldg(reinterpret_cast<const uint32_t*>(xrow + c * cstride + E * col));
+          else r[j] = __ldg(xrow + c * cstride + col);
         }
-        col += d_col; row += d_row;
-        if (col >= nwi) { col -= nwi; ++row; }
+        col += d_col; c += d_c;
+        if (col >= nwi) { col -= nwi; ++c; }
       }
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         if (dsts[j] >= 0) {
           rows_s[dsts[j]] = (uint16_t)(r[j] & 0xffffu);
-          if (VEC2) rows_s[dsts[j] + Kh * PC] = (uint16_t)(r[j] >> 16);
+          if (VEC2) rows_s[dsts[j] + PC] = (uint16_t)(r[j] >> 16);
         }
       }
     }
   }
   __syncthreads();
-  // phase 2: chunk j = t*octs + oct with t = kk*Kh + u: consecutive threads write consecutive 16 bytes
+  // phase 2: for every (ho, u) that holds the row, chunk j = (k - k_lo)*octs + oct
   const int octs = Cp / 8;
-  const int chunks = nk * Kh * octs;
-  const int t_lo = (p - k0 > 0 ? p - k0 : 0) * Kh, t_hi = (W + p - k0) * Kh;   // columns inside the image
-  uint4* out = reinterpret_cast<uint4*>(win + (((n * Ho + ho) * (int64_t)Wp + k0) * Kh) * Cp);
-  {
-    const int step = (int)blockDim.x;
-    const int d_t = step / octs, d_o = step - d_t * octs;
-    int t = (int)threadIdx.x / octs, oct = (int)threadIdx.x - t * octs;
+  const int chunks = (k_hi - k_lo) * octs;
+  const int step = (int)blockDim.x;
+  const int d_k = step / octs, d_o = step - d_k * octs;
+  for (int ho = ho_lo; ho <= ho_hi; ++ho) {
+    const int u = hp - ho * s;
+    // chunk (k, oct) of strip (n, ho): ((k*Kh + u)*Cp + 8*oct) halves into the strip
+    uint16_t* strip = win + ((n * Ho + ho) * (int64_t)Wp) * Kh * Cp + (int64_t)u * Cp;
+    int k = k_lo + (int)threadIdx.x / octs, oct = (int)threadIdx.x % octs;
     for (int j = threadIdx.x; j < chunks; j += step) {
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (t >= t_lo && t < t_hi) {                        // rows outside the image were stored as zeros in phase 1
-        const uint32_t* src = reinterpret_cast<const uint32_t*>(rows_s + t * PC + 8 * oct);
+      const int w = k - p;
+      if (row_ok && w >= w0 && w < w0 + nw) {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(rows_s + (w - w0) * PC + 8 * oct);
         v = make_uint4(src[0], src[1], src[2], src[3]);
       }
-      out[j] = v;
-      oct += d_o; t += d_t;
-      if (oct >= octs) { oct -= octs; ++t; }
+      *reinterpret_cast<uint4*>(strip + (int64_t)k * Kh * Cp + 8 * oct) = v;
+      oct += d_o; k += d_k;
+      if (oct >= octs) { oct -= octs; ++k; }
     }
   }
 }
@@ -1243,9 +1245,8 @@ NhwcPlan plan_nhwc(const Geometry& g) {
   p.window_elems = (int64_t)g.N * g.Ho * p.strip;
   if ((int64_t)g.N * g.Ho >= lim || p.strip >= lim) return p;
   if ((int64_t)g.s * g.Kh * p.Cp * 2 >= ((int64_t)1 << 40) || p.strip * 2 >= ((int64_t)1 << 40)) return p;
-  // the transform from NCHW tabulates one entry per (u, c) in shared memory and indexes an image with 32 bits
-  if ((int64_t)g.Kh * g.C * 8 > 48 * 1024 || (int64_t)g.C * g.H * g.W >= lim) return p;
-  if ((int64_t)g.Kh * (p.Cp + 2) * 2 > 56 * 1024) return p;
+  // the transform from NCHW stages at least two columns of Cp + 2 channels in 48 KB of shared memory
+  if ((int64_t)(p.Cp + 2) * 2 * 2 > 48 * 1024) return p;
   // position tiles: tw tiles along a strip of bw columns each (one when the strip fits 128 rows),
   // G whole strips per tile when a strip is short
   p.tw = (g.Wo + TILE_M - 1) / TILE_M;
@@ -1299,28 +1300,17 @@ cudaError_t launch_transform_nhwc(const uint16_t* x, int x_is_nhwc, uint16_t* wi
                                                                           g.Kh, g.s, g.p, chunks);
     return cudaGetLastError();
   }
-  // columns per block: the whole strip when its Kh rows of Cp + 2 halves fit 64 KB of shared memory
-  const int64_t per_col = (int64_t)g.Kh * (plan.Cp + 2) * 2;
-  const int64_t tables = (int64_t)g.Kh * g.C * 8;
-  if ((int64_t)g.C * g.H * g.W >= ((int64_t)1 << 31) || tables > 48 * 1024) return cudaErrorInvalidValue;
-  int kc = (int)((112 * 1024 - tables) / per_col);
-  if (kc < 1) return cudaErrorInvalidValue;
-  if (kc > g.Wp) kc = g.Wp;
-  // with two columns per load the chunk boundaries must stay even
-  const bool vec2 = (g.W % 2 == 0) && (g.p % 2 == 0) && (kc % 2 == 0 || kc == g.Wp);
-  const int kchunks = (g.Wp + kc - 1) / kc;
-  const int64_t blocks = (int64_t)g.N * g.Ho * kchunks;
+  // columns per block: the whole row when it fits 48 KB of shared memory as T[w][Cp + 2]
+  const int64_t per_col = (int64_t)(plan.Cp + 2) * 2;
+  int kc = (int)((48 * 1024) / per_col);
+  if (kc < 2) return cudaErrorInvalidValue;
+  if (kc > g.W) kc = g.W;
+  else kc &= ~1;                                           // chunk boundaries stay even for the two-column loads
+  const bool vec2 = g.W % 2 == 0;
+  const int kchunks = (g.W + kc - 1) / kc;
+  const int64_t blocks = (int64_t)g.N * (g.H + 2 * g.p) * kchunks;
   if (blocks >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
-  const size_t smem = (size_t)(per_col * kc + tables);
-  static bool attr_done[64][2] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!attr_done[dev][vec2]) {
-    cudaError_t e = vec2 ? cudaFuncSetAttribute(transform_nhwc_from_nchw_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024)
-                         : cudaFuncSetAttribute(transform_nhwc_from_nchw_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_done[dev][vec2] = true;
-  }
+  const size_t smem = (size_t)(per_col * kc);
   if (vec2)
     transform_nhwc_from_nchw_kernel<true><<<(unsigned)blocks, 256, smem, stream>>>(x, window, g.C, plan.Cp, g.H, g.W, g.Ho, g.Wp,
                                                                                    g.Kh, g.s, g.p, kc, kchunks);
