@@ -153,7 +153,10 @@ class LayerRunner:
         x, f = workloads.make_inputs(self.layer)
         window, scratch, y = b.alloc_nhwc_buffers(self.dims)
         self.nhwc = dict(x=x.half().cuda(), f=f.half().cuda(), window=window, scratch=scratch, y=y,
-                         cp=b.im2win_nhwc_workspace_size(self.dims)[4])
+                         cp=b.im2win_nhwc_workspace_size(self.dims)[4],
+                         y16=torch.empty(y.shape, dtype=torch.float16, device="cuda"),
+                         bias=torch.zeros(self.layer.Co, dtype=torch.float32, device="cuda"))
+        self.nhwc["epi16"] = b.make_epilogue(self.nhwc["bias"], True, torch.float16, b.NCHW)
 
     def transform_nhwc(self, prec=None):
         d = self.nhwc
@@ -162,6 +165,11 @@ class LayerRunner:
     def conv_nhwc(self, prec=None):
         d = self.nhwc
         self.b.im2win_conv_f16_nhwc(d["window"], d["f"], d["y"], d["scratch"], self.dims)
+
+    def conv_nhwc_out16(self, prec=None):
+        """The same convolution with the fused epilogue: bias, ReLU, binary16 NCHW output."""
+        d = self.nhwc
+        self.b.im2win_conv_f16_nhwc(d["window"], d["f"], d["y16"], d["scratch"], self.dims, d["epi16"])
 
     def conv_nhwc_packed(self, prec=None):
         d = self.nhwc
@@ -206,6 +214,8 @@ class LayerRunner:
         f_el = l.Co * l.C * l.Kh * l.Kw
         if kernel.startswith("transform"):
             return (x_el + win_el) * es
+        if kernel.endswith("out16_nhwc"):
+            return win_el * es + f_el * es + out_el * 2 + l.Co * 4
         return win_el * es + f_el * es + out_el * 4
 
     def memory_report(self):
@@ -218,6 +228,12 @@ class LayerRunner:
             rep[prec] = {"window_bytes": win, "output_bytes": out, "window_plus_output_bytes": win + out,
                          "scratch_bytes": self.dev[prec]["scratch"].numel(),
                          "im2col_bytes": l.N * l.C * l.Kh * l.Kw * self.ho * self.wo * es}
+        if self.nhwc is not None:
+            win = l.N * self.nhwc["cp"] * self.ho * l.Kh * (l.W + 2 * l.pad) * 2
+            out = l.N * l.Co * self.ho * self.wo * 4
+            rep["f16_nhwc"] = {"window_bytes": win, "output_bytes": out, "window_plus_output_bytes": win + out,
+                               "scratch_bytes": self.nhwc["scratch"].numel(),
+                               "im2col_bytes": l.N * l.C * l.Kh * l.Kw * self.ho * self.wo * 2}
         return rep
 
 
@@ -466,7 +482,8 @@ def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
             for _ in range(3):
                 runner.transform_nhwc()
                 runner.conv_nhwc()
-            for key, fn in (("transform_f16_nhwc", runner.transform_nhwc), ("conv_f16_nhwc", runner.conv_nhwc)):
+            for key, fn in (("transform_f16_nhwc", runner.transform_nhwc), ("conv_f16_nhwc", runner.conv_nhwc),
+                            ("conv_f16_out16_nhwc", runner.conv_nhwc_out16)):
                 avg[key], best[key], median[key] = time_call(fn, iters, flush)
             binding.im2win_check_status(runner.nhwc["scratch"])
         row = {"layer": name, "dims": layer.dims(), "gflop": runner.flops / 1e9, "avg_ms": avg, "best_ms": best,

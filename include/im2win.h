@@ -69,7 +69,7 @@ const char* im2win_status_string(im2win_status status);
  * Name of the convolution kernel the library selects for a layer (host-only,
  * launches nothing; static storage): "f32-ffma" for IM2WIN_F32; for IM2WIN_F16
  * one of the tensor-core kernels of Algorithm 1's GEMM view, "f16-stem",
- * "f16-mat", "f16-matc", "f16-raw", "f16-shift" or "f16-gather"; "none" for an
+ * "f16-mat", "f16-raw", "f16-shift" or "f16-gather"; "none" for an
  * invalid shape.  For reports and tests; the choice is an implementation detail.
  */
 const char* im2win_conv_kernel_name(const im2win_shape* shape, im2win_dtype dtype);

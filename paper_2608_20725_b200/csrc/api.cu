@@ -69,7 +69,6 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
   l->f16_shift = false;
   l->f16_raw = false;
   l->f16_mat = false;
-  l->f16_matc = false;
   l->f16_stem = false;
   l->koff_off = kStatusBytes;
   l->filter_off = (size_t)round_up((int64_t)l->koff_off + 4 * l->Kp, 256);
@@ -98,22 +97,16 @@ im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayou
       if (shift_total > l->total) l->total = shift_total;
     }
     const MatPlan mat = plan_f16_mat(g);
-    const MatcPlan matc = mat.eligible ? MatcPlan{} : plan_f16_matc(g);
     const char* force = debug_getenv("IM2WIN_F16_KERNEL");
-    // measured: the matrix-transpose kernels win for strided layers (the others stage such layers
+    // measured: the matrix-transpose kernel wins for strided layers (the others stage such layers
     // with 2-byte gathers) and for kernels up to 5 wide with 128 output channels or more (CTA pairs
-    // above 128); IM2WIN_F16_KERNEL=mat forces them wherever they can run (a testing aid)
+    // above 128); IM2WIN_F16_KERNEL=mat forces it wherever it can run (a testing aid)
     const bool want = force ? strcmp(force, "mat") == 0 : (g.s > 1 || (g.Co >= 128 && g.Kw <= 5));
     // (the scratch size covers every layout, whichever kernel is picked or forced)
-    const bool use_mat = want && !l->f16_stem;
     if (mat.eligible) {
-      l->f16_mat = use_mat;
+      l->f16_mat = want && !l->f16_stem;
       const size_t mat_total = (size_t)round_up((int64_t)mat.scratch_bytes, 256);
       if (mat_total > l->total) l->total = mat_total;
-    } else if (matc.eligible) {
-      l->f16_matc = use_mat;
-      const size_t matc_total = (size_t)round_up((int64_t)matc.scratch_bytes, 256);
-      if (matc_total > l->total) l->total = matc_total;
     }
   }
   return IM2WIN_OK;
@@ -145,7 +138,6 @@ static im2win_status conv_common(const void* window, const void* filter, float* 
     if (dtype == IM2WIN_F32) e = launch_pack_f32(static_cast<const float*>(filter), scratch, g, l, stream);
     else if (l.f16_stem) e = launch_pack_f16_shift(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
     else if (l.f16_mat) e = launch_pack_f16_mat(static_cast<const uint16_t*>(filter), scratch, g, stream);
-    else if (l.f16_matc) e = launch_pack_f16_matc(static_cast<const uint16_t*>(filter), scratch, g, stream);
     else if (l.f16_raw)
       e = launch_pack_f16_raw(static_cast<const uint16_t*>(filter), scratch, g, l, plan_f16_raw(g), stream);
     else if (l.f16_shift) e = launch_pack_f16_shift(static_cast<const uint16_t*>(filter), scratch, g, l, stream);
@@ -156,7 +148,6 @@ static im2win_status conv_common(const void* window, const void* filter, float* 
     if (dtype == IM2WIN_F32) e = launch_conv_f32(static_cast<const float*>(window), y, scratch, g, l, stream);
     else if (l.f16_stem) e = launch_conv_f16_stem(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
     else if (l.f16_mat) e = launch_conv_f16_mat(static_cast<const uint16_t*>(window), y, scratch, g, stream);
-    else if (l.f16_matc) e = launch_conv_f16_matc(static_cast<const uint16_t*>(window), y, scratch, g, stream);
     else if (l.f16_raw) e = launch_conv_f16_raw(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
     else if (l.f16_shift) e = launch_conv_f16_shift(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
     else e = launch_conv_f16_gather(static_cast<const uint16_t*>(window), y, scratch, g, l, stream);
@@ -191,7 +182,6 @@ const char* im2win_conv_kernel_name(const im2win_shape* shape, im2win_dtype dtyp
   if (dtype == IM2WIN_F32) return "f32-ffma";
   if (l.f16_stem) return "f16-stem";
   if (l.f16_mat) return "f16-mat";
-  if (l.f16_matc) return "f16-matc";
   if (l.f16_raw) return "f16-raw";
   if (l.f16_shift) return "f16-shift";
   return "f16-gather";

@@ -37,7 +37,6 @@ struct ScratchLayout {
   bool f16_shift;        // fp16 only: a shifted-view kernel (and its filter layout) is used
   bool f16_raw;          // fp16 only: the bulk-copy variant of the shifted-view kernel is used
   bool f16_mat;          // fp16 only: the matrix-transpose variant is used (own scratch layout)
-  bool f16_matc;         // fp16 only: its general form (channel classes / batched raw stages) is used
   bool f16_stem;         // fp16 only: the one-k-block kernel for C*Kh <= 64 is used (filter layout of f16_shift)
 };
 
@@ -72,17 +71,6 @@ struct MatPlan {
   size_t scratch_bytes;  // status block + packed filter
 };
 MatPlan plan_f16_mat(const Geometry& g);
-
-// Tile geometry of the general matrix-transpose kernel (channel classes, batched raw stages; see
-// conv_f16_matc.cu).
-struct MatcPlan {
-  bool eligible;
-  int32_t Wq, rows, R, nplanes, rawbox, box_bytes, raw_stage_bytes, a_stage_bytes, num_kb;
-  int32_t P, shift1, kbpc, units0, units1;   // channel classes (conv_f16_matc.cu, WinMaps)
-  int64_t K2p, VQ;
-  size_t scratch_bytes;  // status block + packed filter
-};
-MatcPlan plan_f16_matc(const Geometry& g);
 
 // Tile geometry of the one-k-block kernel for layers with C*Kh <= 64 (see conv_f16_stem.cu).
 struct StemPlan {
@@ -148,9 +136,6 @@ cudaError_t launch_conv_f16_raw(const uint16_t* window, float* y, void* scratch,
 cudaError_t launch_pack_f16_mat(const uint16_t* filter, void* scratch, const Geometry& g, cudaStream_t stream);
 cudaError_t launch_conv_f16_mat(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                 cudaStream_t stream);
-cudaError_t launch_pack_f16_matc(const uint16_t* filter, void* scratch, const Geometry& g, cudaStream_t stream);
-cudaError_t launch_conv_f16_matc(const uint16_t* window, float* y, void* scratch, const Geometry& g,
-                                 cudaStream_t stream);
 cudaError_t launch_conv_f16_stem(const uint16_t* window, float* y, void* scratch, const Geometry& g,
                                  const ScratchLayout& l, cudaStream_t stream);
 cudaError_t launch_conv_f16_gather(const uint16_t* window, float* y, void* scratch, const Geometry& g,

@@ -774,6 +774,9 @@ __global__ void __launch_bounds__(256)
 pack_f16_nhwc_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, uint32_t* status, int C, int Cp,
                      int Co, int Kh, int Kw, int cb) {
   extern __shared__ __align__(16) uint16_t pack_s[];   // [cb][T], after up to 8 halves of phase padding
+  // the convolution that follows in the stream may be launched now: its set-up overlaps this kernel,
+  // and every role of it that touches memory first waits for this grid to have completed
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
   const int T = Kh * Kw;
   const int64_t K = (int64_t)T * Cp;
