@@ -578,7 +578,7 @@ def run_reference_arm(args):
     sets = {"f32": (x.numpy(), f.numpy()), "f16": (x16, f16)}
     dims = layer.dims()
     ho, wo = oracle.out_dims(dims)
-    n_img = 2                                   # images per precision per step: a bounded sample of the batch
+    n_img = 16                                  # images per precision per step: a bounded sample of the batch
     flops_step = 2 * n_img * layer_flops(layer, ho, wo) / layer.N
 
     def step(i):
