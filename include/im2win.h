@@ -187,7 +187,10 @@ im2win_status im2win_layer_workspace_size(const im2win_shape* shape, im2win_dtyp
  * that the library creates once per device and keeps; they are ordered after
  * everything queued on `cuda_stream` before the call, and `cuda_stream` waits
  * for the last of them, so synchronising `cuda_stream` still completes the
- * call.  The result does not depend on the chunking.
+ * call.  The result does not depend on the chunking.  Arguments and every
+ * chunk's geometry are validated before anything is queued; should a CUDA call
+ * fail after the first chunk was queued, the call still makes `cuda_stream`
+ * wait for the auxiliary streams before it returns the error.
  */
 im2win_status im2win_layer_forward_host(const void* x_host, const void* filter_host, float* y_host,
                                         void* device_workspace, size_t device_workspace_bytes,

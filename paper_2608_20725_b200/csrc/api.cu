@@ -440,11 +440,27 @@ im2win_status im2win_layer_forward_host(const void* x_host, const void* filter_h
     cudaEventDestroy(ev);                                              // released once it has completed
     return ok;
   };
-  if (!fence(stream, aux.in) || !fence(stream, aux.out)) return IM2WIN_ERR_CUDA;
-  if (cudaMemcpyAsync(ws + L.f_off, filter_host, L.f_bytes, cudaMemcpyHostToDevice, aux.in) != cudaSuccess)
-    return IM2WIN_ERR_CUDA;
   const int per = ((g.N + nchunk - 1) / nchunk + unit - 1) / unit * unit;
+  // Every distinct chunk size is validated before anything is queued: its geometry must derive and
+  // the scratch its kernels want (the kernel choice can depend on N) must fit the scratch that was
+  // sized for the whole batch.
   for (int n0 = 0; n0 < g.N; n0 += per) {
+    im2win_shape part = *shape;
+    part.N = n0 + per < g.N ? per : g.N - n0;
+    Geometry gp;
+    ScratchLayout lp;
+    st = derive_geometry(&part, &gp);
+    if (st == IM2WIN_OK) st = scratch_layout(gp, dtype, &lp);
+    if (st != IM2WIN_OK) return st;
+    if (lp.total > L.scratch_bytes) return IM2WIN_ERR_WORKSPACE_TOO_SMALL;
+  }
+  if (!fence(stream, aux.in) || !fence(stream, aux.out)) return IM2WIN_ERR_CUDA;
+  // From here on work is queued on the auxiliary streams: on any failure `stream` is still made to
+  // wait for both of them, so that synchronising `stream` completes whatever was queued.
+  im2win_status result = IM2WIN_OK;
+  if (cudaMemcpyAsync(ws + L.f_off, filter_host, L.f_bytes, cudaMemcpyHostToDevice, aux.in) != cudaSuccess)
+    result = IM2WIN_ERR_CUDA;
+  for (int n0 = 0; n0 < g.N && result == IM2WIN_OK; n0 += per) {
     const int n1 = n0 + per < g.N ? n0 + per : g.N;
     im2win_shape part = *shape;
     part.N = n1 - n0;
@@ -452,21 +468,23 @@ im2win_status im2win_layer_forward_host(const void* x_host, const void* filter_h
     unsigned char* wd = ws + L.win_off + (size_t)n0 * w_img;
     unsigned char* yd = ws + L.y_off + (size_t)n0 * y_img;
     if (cudaMemcpyAsync(xd, static_cast<const unsigned char*>(x_host) + (size_t)n0 * x_img, (size_t)part.N * x_img,
-                        cudaMemcpyHostToDevice, aux.in) != cudaSuccess)
-      return IM2WIN_ERR_CUDA;
-    if (!fence(aux.in, stream)) return IM2WIN_ERR_CUDA;
-    st = im2win_transform(xd, wd, &part, dtype, cuda_stream);
-    if (st != IM2WIN_OK) return st;
-    st = conv_common(wd, ws + L.f_off, reinterpret_cast<float*>(yd), ws + L.scratch_off, L.scratch_bytes, &part, dtype,
-                     cuda_stream);
-    if (st != IM2WIN_OK) return st;
-    if (!fence(stream, aux.out)) return IM2WIN_ERR_CUDA;
-    if (cudaMemcpyAsync(reinterpret_cast<unsigned char*>(y_host) + (size_t)n0 * y_img, yd, (size_t)part.N * y_img,
+                        cudaMemcpyHostToDevice, aux.in) != cudaSuccess || !fence(aux.in, stream)) {
+      result = IM2WIN_ERR_CUDA;
+      break;
+    }
+    result = im2win_transform(xd, wd, &part, dtype, cuda_stream);
+    if (result != IM2WIN_OK) break;
+    result = conv_common(wd, ws + L.f_off, reinterpret_cast<float*>(yd), ws + L.scratch_off, L.scratch_bytes, &part,
+                         dtype, cuda_stream);
+    if (result != IM2WIN_OK) break;
+    if (!fence(stream, aux.out) ||
+        cudaMemcpyAsync(reinterpret_cast<unsigned char*>(y_host) + (size_t)n0 * y_img, yd, (size_t)part.N * y_img,
                         cudaMemcpyDeviceToHost, aux.out) != cudaSuccess)
-      return IM2WIN_ERR_CUDA;
+      result = IM2WIN_ERR_CUDA;
   }
-  if (!fence(aux.out, stream) || !fence(aux.in, stream)) return IM2WIN_ERR_CUDA;
-  return IM2WIN_OK;
+  const bool joined = fence(aux.out, stream) & fence(aux.in, stream);
+  if (result == IM2WIN_OK && !joined) result = IM2WIN_ERR_CUDA;
+  return result;
 }
 
 }  // extern "C"
