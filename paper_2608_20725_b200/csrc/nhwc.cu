@@ -63,6 +63,9 @@ struct NhwcParams {
   int32_t ntn, nwork;        // channel tiles; work items = position tiles (pairs) x channel tiles x k parts
   int32_t stages;
   uint32_t a_bytes;          // bytes one activation copy brings: G*bw*128
+  int32_t tail_halves;       // host only: the last round's tiles may be handed out as halves
+  int32_t n_main;            // work items below this index are whole tiles; each whole tile above it is two
+                             // items, one per half of its channels (fills the last, short round of tiles)
 };
 
 // Programmatic dependent launch: the convolution may start while the kernel before it in the stream
@@ -130,13 +133,12 @@ __device__ __forceinline__ void store_chunk(const EpiParams& q, int64_t base, in
 }
 
 // One epilogue warp's share of a finished accumulator: tensor-memory lane quadrant warp % 4, the
-// lower (warps 2..5) or upper (warps 6..9) half of the tile's BN channels, 32 channels at a time:
+// lower (warps 2..5) or upper (warps 6..9) half of the tile's `cols` channels, 32 channels at a time:
 // bias (first K part only), ReLU, store.  `base` is the element index of the tile's first channel
 // at this lane's position, `cs` the element distance between channels.
-template <int BN>
-__device__ __forceinline__ void drain_accumulator(const EpiParams& e, int warp, int lane, uint32_t lane_base, bool valid,
-                                                  int64_t base, int64_t cs, int n0, bool first_part, bool vec_ok) {
-  constexpr int CH = BN / 2;
+__device__ __forceinline__ void drain_accumulator(const EpiParams& e, int cols, int warp, int lane, uint32_t lane_base,
+                                                  bool valid, int64_t base, int64_t cs, int n0, bool first_part, bool vec_ok) {
+  const int CH = cols / 2;                       // cols is a multiple of 64
   const int cbeg = ((warp - WARP_EPI0) >> 2) * CH;
 #pragma unroll 1
   for (int c0 = cbeg; c0 < cbeg + CH; c0 += 32) {
@@ -157,8 +159,16 @@ __device__ __forceinline__ void drain_accumulator(const EpiParams& e, int warp, 
   }
 }
 
+// Work item w of the overlapping-row kernel -> whole tile index and which part of its channels:
+// half = -1 the whole tile, 0 / 1 its lower / upper half.
+__device__ __forceinline__ void decode_item(const NhwcParams& q, int w, int* whole, int* half) {
+  if (w < q.n_main) { *whole = w; *half = -1; }
+  else { const int t = w - q.n_main; *whole = q.n_main + (t >> 1); *half = t & 1; }
+}
+
 template <int BN, bool PAIR, int KSUB>
-__device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CUtensorMap& bmap, const NhwcParams& q) {
+__device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CUtensorMap& bmap, const CUtensorMap& bmap_h,
+                                               const NhwcParams& q) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;              // filter rows (output channels) this CTA stages
   constexpr uint32_t B_BYTES = (uint32_t)B_ROWS * KB * 2;
   constexpr uint32_t SUB_BYTES = (uint32_t)A_SLOT_BYTES + B_BYTES;       // one 64-wide k-block of both operands
@@ -219,12 +229,17 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       uint32_t ph = 0;
       bool ok = true;
       for (int w = w_first; w < q.nwork && ok; w += w_step) {
-        const int mt = w / per_mt, rem = w - mt * per_mt;
+        int whole, half;
+        decode_item(q, w, &whole, &half);
+        const int mt = whole / per_mt, rem = whole - mt * per_mt;
         const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
         const int mti = PAIR ? 2 * mt + (int)rank : mt;
         const int rg = mti / q.tw, wt = mti - rg * q.tw;
         const int z = rg * q.G, yc = wt * q.bw;
-        const int brow = nt * BN + (int)rank * B_ROWS;
+        // filter rows of this CTA: its share of the tile's channels, or of one half of them
+        const int brow = half < 0 ? nt * BN + (int)rank * B_ROWS : nt * BN + half * (BN / 2) + (int)rank * (B_ROWS / 2);
+        const uint32_t b_bytes = half < 0 ? B_BYTES : B_BYTES / 2;
+        const CUtensorMap* bm = half < 0 ? &bmap : &bmap_h;
         const int kc0 = ks * q.kc_per_split;
         const int kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
         for (int kc = kc0; kc < kc1; ++kc) {
@@ -236,16 +251,16 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
             const uint32_t bar = full_dst + 8 * st;
             // k-blocks beyond K read as zeros (and cost no memory traffic), so every stage brings the
             // same number of bytes.  In a pair the leader CTA announces the bytes of both CTAs.
-            if (!PAIR || rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, (PAIR ? 2u : 1u) * KSUB * (q.a_bytes + B_BYTES));
+            if (!PAIR || rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, (PAIR ? 2u : 1u) * KSUB * (q.a_bytes + b_bytes));
 #pragma unroll
             for (int sub = 0; sub < KSUB; ++sub) {
               const int kx = (kc * KSUB + sub) * KB;
               if (PAIR) {
                 tma_load_3d_pair(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
-                tma_load_2d_pair(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
+                tma_load_2d_pair(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, bm, kx, brow, bar);
               } else {
                 tma_load_3d(dst + sub * SUB_BYTES, &amap, kx, yc, z, bar);
-                tma_load_2d(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, &bmap, kx, brow, bar);
+                tma_load_2d(dst + sub * SUB_BYTES + (uint32_t)A_SLOT_BYTES, bm, kx, brow, bar);
               }
             }
           }
@@ -258,7 +273,8 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
     // ---------------- MMA issuer (leader CTA of a pair) -----------------------------
     // Every byte the MMAs read was written by the copy engine, whose completion the barrier's
     // transaction count tracks, so CTA-scope waits suffice also for the peer's half.
-    constexpr uint32_t idesc = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN);
+    constexpr uint32_t idesc_whole = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN);
+    constexpr uint32_t idesc_half = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN / 2);
     {
       // the whole warp walks the loop and takes the waits, one elected lane issues (measured faster
       // than a lone lane, whose satisfied waits cost more)
@@ -268,7 +284,10 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       bool ok = true;
       const uint32_t a_lo0 = smem_desc_lo(ring), b_lo0 = smem_desc_lo(ring + (uint32_t)A_SLOT_BYTES);
       for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
-        const int rem = w % per_mt;
+        int whole, half;
+        decode_item(q, w, &whole, &half);
+        const uint32_t idesc = half < 0 ? idesc_whole : idesc_half;
+        const int rem = whole % per_mt;
         const int ks = rem % q.ksplit;
         const int kc0 = ks * q.kc_per_split;
         const int kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
@@ -320,11 +339,14 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
     TIMER_DECL;
     for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
       const uint32_t buf = it & 1u;
-      const int mt = w / per_mt, rem = w - mt * per_mt;
+      int whole, half;
+      decode_item(q, w, &whole, &half);
+      const int mt = whole / per_mt, rem = whole - mt * per_mt;
       const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
       const int mti = PAIR ? 2 * mt + (int)rank : mt;
       const int rg = mti / q.tw, wt = mti - rg * q.tw;
-      const int n0 = nt * BN;
+      const int n0 = nt * BN + (half > 0 ? BN / 2 : 0);
+      const int cols = half < 0 ? BN : BN / 2;
       // accumulator row r = lane of tensor memory = (strip j of the tile, column i of the tile)
       const int r = lq * 32 + lane;
       const int j = r / q.bw, i = r - j * q.bw;
@@ -348,7 +370,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(6);     // epilogue: wait for a finished accumulator
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
-      drain_accumulator<BN>(e, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
+      drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
       // the buffer may be overwritten once all four warps (of both CTAs) have read it
       tc_fence_before();
       __syncwarp();
@@ -378,14 +400,16 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
 
 template <int BN, int KSUB>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-conv_f16_nhwc_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap, NhwcParams q) {
-  conv_nhwc_body<BN, false, KSUB>(amap, bmap, q);
+conv_f16_nhwc_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
+                     const __grid_constant__ CUtensorMap bmap_h, NhwcParams q) {
+  conv_nhwc_body<BN, false, KSUB>(amap, bmap, bmap_h, q);
 }
 
 template <int BN, int KSUB>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
-conv_f16_nhwc_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap, NhwcParams q) {
-  conv_nhwc_body<BN, true, KSUB>(amap, bmap, q);
+conv_f16_nhwc_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
+                          const __grid_constant__ CUtensorMap bmap_h, NhwcParams q) {
+  conv_nhwc_body<BN, true, KSUB>(amap, bmap, bmap_h, q);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -725,7 +749,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(6);     // epilogue: wait for a finished accumulator
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
-      drain_accumulator<BN>(e, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
+      drain_accumulator(e, BN, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
@@ -978,8 +1002,8 @@ EncodeTiledFn get_encode_fn() {
 }
 
 template <int BN, bool PAIR, int KSUB>
-cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, NhwcParams q, const NhwcPlan& plan,
-                           cudaStream_t stream) {
+cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, const CUtensorMap& bmap_h, NhwcParams q,
+                           const NhwcPlan& plan, cudaStream_t stream) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;
   constexpr int STAGE = KSUB * (A_SLOT_BYTES + B_ROWS * KB * 2);
   int stages = (kSmemMax - 2048) / STAGE;
@@ -993,14 +1017,11 @@ cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, Nhw
   q.ksplit = (q.num_kc + q.kc_per_split - 1) / q.kc_per_split;
   const int64_t ntm_eff = PAIR ? (plan.ntm + 1) / 2 : plan.ntm;
   const int64_t nwork = ntm_eff * q.ntn * q.ksplit;
-  if (nwork >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
+  if (nwork >= ((int64_t)1 << 30)) return cudaErrorInvalidValue;
   q.nwork = (int32_t)nwork;
-  const int slots = PAIR ? 74 : 148;
+  q.n_main = q.nwork;
+  int slots = PAIR ? 74 : 148;
   const int smem_bytes = stages * STAGE + 1024;
-  cudaLaunchConfig_t cfg = {};
-  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = (size_t)smem_bytes;
-  cfg.stream = stream;
   // per device and kernel variant, done once: the shared-memory opt-in and the number of CTA pairs
   // that can be resident together (both are host-side queries that would otherwise sit between the
   // filter pack and this launch on every call)
@@ -1008,6 +1029,11 @@ cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, Nhw
   static bool attr_done[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
   if (PAIR) {
     cudaError_t e = cudaSuccess;
     if (!attr_done[dev]) {
@@ -1015,7 +1041,6 @@ cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, Nhw
       if (e != cudaSuccess) return e;
       attr_done[dev] = true;
     }
-    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -1030,37 +1055,47 @@ cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, Nhw
       if (clusters < 1) return cudaErrorInvalidValue;
       cached_clusters[dev] = clusters;
     }
-    if (clusters > slots) clusters = slots;
-    if (clusters > q.nwork) clusters = q.nwork;
-    cfg.gridDim = dim3(2 * clusters, 1, 1);
-    cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, conv_f16_nhwc_pair_kernel<BN, KSUB>, amap, bmap, q);
-  }
-  if (!attr_done[dev]) {
+    if (clusters < slots) slots = clusters;
+  } else if (!attr_done[dev]) {
     cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_kernel<BN, KSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
     attr_done[dev] = true;
   }
-  cudaLaunchAttribute attr[1];
+  // The last round of tiles: when it would fill at most half of the CTAs (or pairs), each of its tiles
+  // is handed out as two items of half the channels, so the round takes half as long.  (Not with a K
+  // split, whose parts already are the finer grain.)
+  if (BN >= 128 && q.ksplit == 1 && q.tail_halves) {
+    const int tail = q.nwork % slots;
+    if (tail > 0 && 2 * tail <= slots) {
+      q.n_main = q.nwork - tail;
+      q.nwork += tail;
+    }
+  }
+  const int ctas = slots < q.nwork ? slots : q.nwork;
+  if (PAIR) {
+    cfg.gridDim = dim3(2 * ctas, 1, 1);
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, conv_f16_nhwc_pair_kernel<BN, KSUB>, amap, bmap, bmap_h, q);
+  }
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cfg.gridDim = dim3((unsigned)(slots < q.nwork ? slots : q.nwork), 1, 1);
-  return cudaLaunchKernelEx(&cfg, conv_f16_nhwc_kernel<BN, KSUB>, amap, bmap, q);
+  cfg.gridDim = dim3((unsigned)ctas, 1, 1);
+  return cudaLaunchKernelEx(&cfg, conv_f16_nhwc_kernel<BN, KSUB>, amap, bmap, bmap_h, q);
 }
 
 template <int KSUB>
-cudaError_t launch_ksub(const CUtensorMap& amap, const CUtensorMap& bmap, const NhwcParams& q, const NhwcPlan& plan,
-                        cudaStream_t stream) {
+cudaError_t launch_ksub(const CUtensorMap& amap, const CUtensorMap& bmap, const CUtensorMap& bmap_h, const NhwcParams& q,
+                        const NhwcPlan& plan, cudaStream_t stream) {
   if (plan.pair) {
-    if (plan.bn == 256) return launch_variant<256, true, KSUB>(amap, bmap, q, plan, stream);
-    if (plan.bn == 128) return launch_variant<128, true, KSUB>(amap, bmap, q, plan, stream);
-    return launch_variant<64, true, KSUB>(amap, bmap, q, plan, stream);
+    if (plan.bn == 256) return launch_variant<256, true, KSUB>(amap, bmap, bmap_h, q, plan, stream);
+    if (plan.bn == 128) return launch_variant<128, true, KSUB>(amap, bmap, bmap_h, q, plan, stream);
+    return launch_variant<64, true, KSUB>(amap, bmap, bmap_h, q, plan, stream);
   }
-  if (plan.bn == 64) return launch_variant<64, false, KSUB>(amap, bmap, q, plan, stream);
-  if (plan.bn == 128) return launch_variant<128, false, KSUB>(amap, bmap, q, plan, stream);
-  return launch_variant<256, false, KSUB>(amap, bmap, q, plan, stream);
+  if (plan.bn == 64) return launch_variant<64, false, KSUB>(amap, bmap, bmap_h, q, plan, stream);
+  if (plan.bn == 128) return launch_variant<128, false, KSUB>(amap, bmap, bmap_h, q, plan, stream);
+  return launch_variant<256, false, KSUB>(amap, bmap, bmap_h, q, plan, stream);
 }
 
 // Geometry of the shifted-view kernel for a layer (host side).
@@ -1376,6 +1411,19 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   const int64_t b_bytes = (int64_t)(plan.pair ? plan.bn / 2 : plan.bn) * KB * 2;
   bool use_shift = sp.eligible && g.Kw >= 3 * g.s &&
                    2 * (int64_t)sp.a_stage_bytes + 2 * (int64_t)g.Kw * b_bytes <= kSmemMax - 2048;
+  if (use_shift && plan.ksplit == 1) {
+    // Rounds of tiles on the CTAs (pairs): the overlapping-row kernel can hand the tiles of a last round
+    // that is at most half full out as half tiles, the shifted-view kernel cannot; where that saves
+    // more than the shifted view's lower traffic is worth (measured: about 15 % per round), take it.
+    const int slots = plan.pair ? 74 : 148;
+    const int64_t it_o = (plan.pair ? (plan.ntm + 1) / 2 : plan.ntm) * plan.ntn;
+    const int64_t tiles_s = (sp.VQ + TILE_M - 1) / TILE_M;
+    const int64_t it_s = (plan.pair ? (tiles_s + 1) / 2 : tiles_s) * plan.ntn;
+    const int64_t tail = it_o % slots;
+    const double r_o = (double)(it_o / slots) + (tail == 0 ? 0.0 : (plan.bn >= 128 && 2 * tail <= slots ? 0.55 : 1.0));
+    const double r_s = (double)((it_s + slots - 1) / slots);
+    if (r_o < 0.85 * r_s) use_shift = false;
+  }
   if (const char* v = debug_getenv("IM2WIN_NHWC_KERNEL")) {
     if (strcmp(v, "shift") == 0) use_shift = sp.eligible;
     else if (strcmp(v, "overlap") == 0) use_shift = false;
@@ -1398,12 +1446,13 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
     if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
   const int b_rows = plan.pair ? plan.bn / 2 : plan.bn;
-  {
+  CUtensorMap bmap_h;                            // the same filter with boxes of half as many channels
+  for (int half = 0; half < 2; ++half) {
     const cuuint64_t dims[2] = {(cuuint64_t)plan.K, (cuuint64_t)g.Co};
     const cuuint64_t strides[1] = {(cuuint64_t)plan.K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)KB, (cuuint32_t)b_rows};
+    const cuuint32_t box[2] = {(cuuint32_t)KB, (cuuint32_t)(half ? b_rows / 2 : b_rows)};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult cr = encode(&bmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, fp, dims, strides, box, estr,
+    CUresult cr = encode(half ? &bmap_h : &bmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, fp, dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
@@ -1422,8 +1471,10 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   q.a_bytes = (uint32_t)(plan.G * plan.bw * KB * 2);
   int ksub = 1;
   if (const char* v = debug_getenv("IM2WIN_NHWC_KSUB")) ksub = atoi(v) == 1 ? 1 : 2;
-  if (ksub == 1) return launch_ksub<1>(amap, bmap, q, plan, stream);
-  return launch_ksub<2>(amap, bmap, q, plan, stream);
+  q.tail_halves = 1;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_TAIL")) q.tail_halves = v[0] != '0';
+  if (ksub == 1) return launch_ksub<1>(amap, bmap, bmap_h, q, plan, stream);
+  return launch_ksub<2>(amap, bmap, bmap_h, q, plan, stream);
 }
 
 }  // namespace im2win
