@@ -226,7 +226,7 @@ typedef enum {
  * binary32, NCHW.
  */
 typedef struct {
-  const float* bias;        /* DEVICE pointer to Co floats, or NULL             */
+  const float* bias;        /* DEVICE pointer to Co floats (16-byte aligned), or NULL */
   int32_t relu;             /* 0 or 1                                           */
   int32_t out_dtype;        /* IM2WIN_F32 or IM2WIN_F16: element type of y      */
   int32_t out_layout;       /* im2win_layout of y                               */

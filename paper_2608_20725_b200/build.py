@@ -55,15 +55,17 @@ def is_stale() -> bool:
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
     """Compile every .cu under csrc/ and link them into one shared library; returns its path."""
-    if not force and not is_stale():
-        return LIB_PATH
     nvcc = os.environ.get("NVCC", "nvcc")
-    extra = os.environ.get("IM2WIN_EXTRA_NVCC_FLAGS", "").split()     # e.g. -DIM2WIN_BOUNDS_DEBUG
-    os.makedirs(OBJ_DIR, exist_ok=True)
-    # objects built with other flags must not be reused
+    extra = os.environ.get("IM2WIN_EXTRA_NVCC_FLAGS", "").split()     # e.g. -DIM2WIN_F16_TIMERS
+    # objects built with other flags must not be reused; extra flags always mean a rebuild, and so does
+    # a library that was last built with extra flags
     stamp = os.path.join(OBJ_DIR, "flags.txt")
     flags_now = " ".join(NVCC_COMPILE_FLAGS + extra)
     flags_old = open(stamp).read() if os.path.exists(stamp) else None
+    flags_changed = flags_old is not None and flags_old != flags_now
+    if not force and not flags_changed and not extra and not is_stale():
+        return LIB_PATH
+    os.makedirs(OBJ_DIR, exist_ok=True)
     rebuild_all = force or flags_old != flags_now
 
     def compile_one(src: str):

@@ -244,7 +244,7 @@ static im2win_status epilogue_args(const im2win_epilogue* e, bool nhwc_allowed, 
       (e->out_layout != IM2WIN_LAYOUT_NCHW && e->out_layout != IM2WIN_LAYOUT_NHWC))
     return IM2WIN_ERR_INVALID_ARG;
   if (e->out_layout == IM2WIN_LAYOUT_NHWC && !nhwc_allowed) return IM2WIN_ERR_UNSUPPORTED;
-  if (e->bias && (reinterpret_cast<uintptr_t>(e->bias) & 3u)) return IM2WIN_ERR_MISALIGNED;
+  if (e->bias && (reinterpret_cast<uintptr_t>(e->bias) & 15u)) return IM2WIN_ERR_MISALIGNED;
   out->bias = e->bias; out->relu = e->relu; out->out16 = e->out_dtype == IM2WIN_F16;
   out->y_nhwc = e->out_layout == IM2WIN_LAYOUT_NHWC;
   return IM2WIN_OK;

@@ -43,6 +43,8 @@ constexpr int NUM_THREADS = NUM_WARPS * 32;
 constexpr int MAX_STAGES = 8;
 constexpr int A_SLOT_BYTES = TILE_M * KB * 2;  // 16 KB: room for 128 rows even when a tile holds fewer
 constexpr int kSmemMax = 227 * 1024;
+constexpr int MAX_ACC = 8;                     // accumulator buffers in tensor memory: 512 columns / BN, at most 8
+__host__ __device__ constexpr int acc_buffers(int bn) { return 512 / bn < MAX_ACC ? 512 / bn : MAX_ACC; }
 
 // What the epilogue needs to know about the output (shared by both kernels of this file).
 struct EpiParams {
@@ -147,9 +149,23 @@ __device__ __forceinline__ void drain_accumulator(const EpiParams& e, int cols, 
     uint32_t v[32];
     tmem_ld32(lane_base + (uint32_t)c0, v);
     if (e.bias != nullptr && first_part) {
-      const float b = lane < cnt ? __ldg(e.bias + n0 + c0 + lane) : 0.0f;
+      // every lane adds the same 32 channel values: uniform 16-byte loads (the bias is 16-byte aligned
+      // and n0 + c0 a multiple of 32), element by element at the ragged end
+      if (cnt >= 32) {
+        const float4* b4 = reinterpret_cast<const float4*>(e.bias + n0 + c0);
 #pragma unroll
-      for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(__uint_as_float(v[t]) + __shfl_sync(0xffffffffu, b, t));
+        for (int t = 0; t < 32; t += 4) {
+          const float4 b = __ldg(b4 + t / 4);
+          v[t] = __float_as_uint(__uint_as_float(v[t]) + b.x);
+          v[t + 1] = __float_as_uint(__uint_as_float(v[t + 1]) + b.y);
+          v[t + 2] = __float_as_uint(__uint_as_float(v[t + 2]) + b.z);
+          v[t + 3] = __float_as_uint(__uint_as_float(v[t + 3]) + b.w);
+        }
+      } else {
+#pragma unroll
+        for (int t = 0; t < 32; ++t)
+          if (t < cnt) v[t] = __float_as_uint(__uint_as_float(v[t]) + __ldg(e.bias + n0 + c0 + t));
+      }
     }
     if (e.relu) {
 #pragma unroll
@@ -170,6 +186,7 @@ template <int BN, bool PAIR, int KSUB>
 __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CUtensorMap& bmap, const CUtensorMap& bmap_h,
                                                const NhwcParams& q) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;              // filter rows (output channels) this CTA stages
+  constexpr int NACC = acc_buffers(BN);                   // accumulator ring: the epilogue's latency is hidden behind NACC - 1 tiles
   constexpr uint32_t B_BYTES = (uint32_t)B_ROWS * KB * 2;
   constexpr uint32_t SUB_BYTES = (uint32_t)A_SLOT_BYTES + B_BYTES;       // one 64-wide k-block of both operands
   constexpr uint32_t STAGE_BYTES = KSUB * SUB_BYTES;                     // a multiple of 1024
@@ -179,7 +196,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
+  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 2 * MAX_ACC];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile uint32_t abort_flag;
 
@@ -189,7 +206,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
   const uint32_t full0 = smem_u32(&bars[0]);
   const uint32_t empty0 = smem_u32(&bars[MAX_STAGES]);
   const uint32_t acc_full0 = smem_u32(&bars[2 * MAX_STAGES]);
-  const uint32_t acc_empty0 = smem_u32(&bars[2 * MAX_STAGES + 2]);
+  const uint32_t acc_empty0 = smem_u32(&bars[2 * MAX_STAGES + MAX_ACC]);
 
   if (threadIdx.x == 0) {
     abort_flag = 0u;
@@ -197,15 +214,15 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       mbar_init(full0 + 8 * i, 1);
       mbar_init(empty0 + 8 * i, 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < MAX_ACC; ++i) {
       mbar_init(acc_full0 + 8 * i, 1);
       mbar_init(acc_empty0 + 8 * i, PAIR ? 2 * EPI_WARPS : EPI_WARPS);   // the epilogue warps (of each CTA)
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == WARP_MMA) {
-    if (PAIR) tmem_alloc_pair(smem_u32(&tmem_base_slot), 2 * BN);
-    else tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
+    if (PAIR) tmem_alloc_pair(smem_u32(&tmem_base_slot), NACC * BN);
+    else tmem_alloc(smem_u32(&tmem_base_slot), NACC * BN);
   }
   tc_fence_before();
   __syncthreads();
@@ -291,8 +308,8 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
         const int ks = rem % q.ksplit;
         const int kc0 = ks * q.kc_per_split;
         const int kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
-        const uint32_t buf = it & 1u;
-        ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);
+        const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
+        ok = mbar_wait(acc_empty0 + 8 * buf, aph ^ 1u, &abort_flag, q.status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
@@ -338,7 +355,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
     uint32_t it = 0;
     TIMER_DECL;
     for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
-      const uint32_t buf = it & 1u;
+      const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
       int whole, half;
       decode_item(q, w, &whole, &half);
       const int mt = whole / per_mt, rem = whole - mt * per_mt;
@@ -363,7 +380,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
         }
       }
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(5);     // epilogue: draining and storing
-      if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
+      if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, aph, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
       __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
       if (!ok) break;
@@ -393,8 +410,8 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
   if (warp == WARP_MMA) {
     __syncwarp();
     tc_fence_after();
-    if (PAIR) tmem_dealloc_pair(tmem_acc, 2 * BN);
-    else tmem_dealloc(tmem_acc, 2 * BN);
+    if (PAIR) tmem_dealloc_pair(tmem_acc, NACC * BN);
+    else tmem_dealloc(tmem_acc, NACC * BN);
   }
 }
 
@@ -448,9 +465,28 @@ struct ShiftViewParams {
   int32_t bu_forced;         // testing aid: bu was given, do not choose it
 };
 
+// All MMAs of one full k2-block whose KW kernel columns sit in one filter stage, unrolled for a
+// compile-time kernel width (view offsets from registers, filter tiles B16 sixteen-byte units apart):
+// the issuing lane then spends a handful of instructions per MMA, which is what narrow tiles need
+// (an N = 64 MMA occupies the tensor pipe for 48 cycles only).
+template <int KW, bool PAIR>
+__device__ __forceinline__ void issue_k2_block(uint32_t acc, uint32_t a_stage, uint32_t b_lo, const uint32_t (&tap)[7],
+                                               uint32_t b16, uint32_t idesc, uint32_t& accumulate) {
+#pragma unroll
+  for (int v = 0; v < KW; ++v) {
+#pragma unroll
+    for (int t = 0; t < KB / 16; ++t) {
+      if (PAIR) umma_f16_ab_pair(acc, a_stage + tap[v] + 2 * t, kSmemDescHiSw128, b_lo + v * b16 + 2 * t, kSmemDescHiSw128, idesc, accumulate);
+      else umma_f16_lohi(acc, a_stage + tap[v] + 2 * t, b_lo + v * b16 + 2 * t, idesc, accumulate);
+      accumulate = 1u;
+    }
+  }
+}
+
 template <int BN, bool PAIR>
 __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const CUtensorMap& bmap, const ShiftViewParams& q) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;
+  constexpr int NACC = acc_buffers(BN);
   constexpr uint32_t B_BYTES = (uint32_t)B_ROWS * KB * 2;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
   const int w_first = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
@@ -458,7 +494,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-  __shared__ __align__(8) uint64_t bars[2 * MAX_SA + 2 * MAX_SB + 4];
+  __shared__ __align__(8) uint64_t bars[2 * MAX_SA + 2 * MAX_SB + 2 * MAX_ACC];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile uint32_t abort_flag;
   __shared__ uint32_t tap16[MAX_KW];           // view of kernel column v inside an activation stage, in 16-byte units
@@ -473,7 +509,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
   const uint32_t b_full0 = smem_u32(&bars[2 * MAX_SA]);
   const uint32_t b_empty0 = smem_u32(&bars[2 * MAX_SA + MAX_SB]);
   const uint32_t acc_full0 = smem_u32(&bars[2 * MAX_SA + 2 * MAX_SB]);
-  const uint32_t acc_empty0 = smem_u32(&bars[2 * MAX_SA + 2 * MAX_SB + 2]);
+  const uint32_t acc_empty0 = smem_u32(&bars[2 * MAX_SA + 2 * MAX_SB + MAX_ACC]);
 
   if (threadIdx.x == 0) {
     abort_flag = 0u;
@@ -481,15 +517,15 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
     for (int v = 0; v < q.Kw; ++v) tap16[v] = (uint32_t)(v % q.s) * (q.subt_bytes >> 4) + (uint32_t)(v / q.s) * (KB * 2 >> 4);
     for (int i = 0; i < MAX_SA; ++i) { mbar_init(a_full0 + 8 * i, 1); mbar_init(a_empty0 + 8 * i, 1); }
     for (int i = 0; i < MAX_SB; ++i) { mbar_init(b_full0 + 8 * i, 1); mbar_init(b_empty0 + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < MAX_ACC; ++i) {
       mbar_init(acc_full0 + 8 * i, 1);
       mbar_init(acc_empty0 + 8 * i, PAIR ? 2 * EPI_WARPS : EPI_WARPS);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == WARP_MMA) {
-    if (PAIR) tmem_alloc_pair(smem_u32(&tmem_base_slot), 2 * BN);
-    else tmem_alloc(smem_u32(&tmem_base_slot), 2 * BN);
+    if (PAIR) tmem_alloc_pair(smem_u32(&tmem_base_slot), NACC * BN);
+    else tmem_alloc(smem_u32(&tmem_base_slot), NACC * BN);
   }
   tc_fence_before();
   __syncthreads();
@@ -588,15 +624,18 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       bool ok = true;
       const uint32_t a_lo0 = smem_desc_lo(a_ring), b_lo0 = smem_desc_lo(b_ring);
       const uint32_t subt16 = q.subt_bytes >> 4, astage16 = q.a_stage_bytes >> 4, bstage16 = b_stage_bytes >> 4;
+      uint32_t tapr[7];                          // the first seven view offsets in registers (unrolled issue paths)
+#pragma unroll
+      for (int v = 0; v < 7; ++v) tapr[v] = v < q.Kw ? tap16[v] : 0u;
       TIMER_DECL;
       for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
         const int rem = w % per_mt;
         const int ks = rem % q.ksplit;
         const int kb0 = ks * q.kb_per_split;
         const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
-        const uint32_t buf = it & 1u;
+        const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
         if (lane == 0) TIMER_LAP(2);                     // MMA warp: issue and bookkeeping
-        ok = mbar_wait(acc_empty0 + 8 * buf, ((it >> 1) & 1u) ^ 1u, &abort_flag, q.status);   // drained by the epilogue
+        ok = mbar_wait(acc_empty0 + 8 * buf, aph ^ 1u, &abort_flag, q.status);   // drained by the epilogue
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         if (lane == 0) TIMER_LAP(3);                     // MMA warp: wait for a free accumulator
@@ -617,15 +656,20 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
               const uint32_t a_stage = a_lo0 + (uint32_t)sta * astage16;
               uint32_t b_lo = b_lo0 + (uint32_t)stb * bstage16;
               if (kb != q.nkb2 - 1 || q.nks_last == KB / 16) {
-                for (int v = 0; v < q.Kw; ++v) {
-                  const uint32_t a_lo = a_stage + tap16[v];
+                if (q.Kw == 3) issue_k2_block<3, PAIR>(acc, a_stage, b_lo, tapr, B_BYTES >> 4, idesc, accumulate);
+                else if (q.Kw == 5) issue_k2_block<5, PAIR>(acc, a_stage, b_lo, tapr, B_BYTES >> 4, idesc, accumulate);
+                else if (q.Kw == 7) issue_k2_block<7, PAIR>(acc, a_stage, b_lo, tapr, B_BYTES >> 4, idesc, accumulate);
+                else {
+                  for (int v = 0; v < q.Kw; ++v) {
+                    const uint32_t a_lo = a_stage + tap16[v];
 #pragma unroll
-                  for (int t = 0; t < KB / 16; ++t) {
-                    if (PAIR) umma_f16_ab_pair(acc, a_lo + 2 * t, kSmemDescHiSw128, b_lo + 2 * t, kSmemDescHiSw128, idesc, accumulate);
-                    else umma_f16_lohi(acc, a_lo + 2 * t, b_lo + 2 * t, idesc, accumulate);
-                    accumulate = 1u;
+                    for (int t = 0; t < KB / 16; ++t) {
+                      if (PAIR) umma_f16_ab_pair(acc, a_lo + 2 * t, kSmemDescHiSw128, b_lo + 2 * t, kSmemDescHiSw128, idesc, accumulate);
+                      else umma_f16_lohi(acc, a_lo + 2 * t, b_lo + 2 * t, idesc, accumulate);
+                      accumulate = 1u;
+                    }
+                    b_lo += B_BYTES >> 4;
                   }
-                  b_lo += B_BYTES >> 4;
                 }
               } else {
                 for (int v = 0; v < q.Kw; ++v) {
@@ -722,7 +766,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
     uint32_t it = 0;
     TIMER_DECL;
     for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
-      const uint32_t buf = it & 1u;
+      const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
       const int mt = w / per_mt, rem = w - mt * per_mt;
       const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
       const int n0 = nt * BN;
@@ -742,7 +786,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
         }
       }
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(5);     // epilogue: draining and storing
-      if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, (it >> 1) & 1u, &abort_flag, q.status);
+      if (lane == 0) ok = mbar_wait(acc_full0 + 8 * buf, aph, &abort_flag, q.status);
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
       __syncwarp();   // lane 0 observed the barrier: orders the other lanes' accesses after it
       if (!ok) break;
@@ -771,8 +815,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
   if (warp == WARP_MMA) {
     __syncwarp();
     tc_fence_after();
-    if (PAIR) tmem_dealloc_pair(tmem_acc, 2 * BN);
-    else tmem_dealloc(tmem_acc, 2 * BN);
+    if (PAIR) tmem_dealloc_pair(tmem_acc, NACC * BN);
+    else tmem_dealloc(tmem_acc, NACC * BN);
   }
 }
 
