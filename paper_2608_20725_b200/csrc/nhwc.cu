@@ -934,7 +934,7 @@ __global__ void transform_nhwc_from_nhwc_kernel(const uint16_t* __restrict__ x, 
 // fastest), so consecutive threads write consecutive bytes of a column.  Every input element is
 // read once and transposed once; blocks of rows outside the image only write zeros.  Indices are
 // kept in mixed-radix counters (no division per element).
-template <bool VEC2>
+template <int VEC>
 __global__ void __launch_bounds__(256)
 transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ win, int C, int Cp, int H, int W,
                                 int Ho, int Wp, int Kh, int s, int p, int kc, int kchunks) {
@@ -964,34 +964,35 @@ transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __rest
         rows_s[r * PC + C + e] = 0;
       }
     }
-    // phase 1: item -> (c, column (pair)), columns fastest; 8 loads in flight per thread
-    constexpr int E = VEC2 ? 2 : 1;                       // columns per item (VEC2: W, w0 and nw are even)
-    const int nwi = nw / E;
+    // phase 1: item -> (c, group of VEC columns), columns fastest (W, w0 and nw are multiples of
+    // VEC): one VEC*2-byte load, VEC transposing 2-byte stores; four loads in flight per thread
+    typedef typename VecType<VEC>::type V;
+    const int nwi = nw / VEC;
     const int items = C * nwi;
     const int step = (int)blockDim.x;
     const int d_c = step / nwi, d_col = step - d_c * nwi;
     int c = (int)threadIdx.x / nwi, col = (int)threadIdx.x - c * nwi;
     const uint16_t* xrow = x + ((n * C) * H + h) * (int64_t)W + w0;      // channel c: + c*H*W
     const int64_t cstride = (int64_t)H * W;
-    for (int i0 = threadIdx.x; i0 < items; i0 += 8 * step) {
-      uint32_t r[8];
-      int dsts[8];
+    for (int i0 = threadIdx.x; i0 < items; i0 += 4 * step) {
+      V r[4];
+      int dsts[4];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < 4; ++j) {
         dsts[j] = -1;
         if (i0 + j * step < items) {
-          dsts[j] = (E * col) * PC + c;
-          if (VEC2) r[j] = __ldg(reinterpret_cast<const uint32_t*>(xrow + c * cstride + E * col));
-          else r[j] = __ldg(xrow + c * cstride + col);
+          dsts[j] = (VEC * col) * PC + c;
+          r[j] = __ldg(reinterpret_cast<const V*>(xrow + c * cstride + VEC * col));
         }
         col += d_col; c += d_c;
         if (col >= nwi) { col -= nwi; ++c; }
       }
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < 4; ++j) {
         if (dsts[j] >= 0) {
-          rows_s[dsts[j]] = (uint16_t)(r[j] & 0xffffu);
-          if (VEC2) rows_s[dsts[j] + PC] = (uint16_t)(r[j] >> 16);
+          const uint16_t* e = reinterpret_cast<const uint16_t*>(&r[j]);
+#pragma unroll
+          for (int t = 0; t < VEC; ++t) rows_s[dsts[j] + t * PC] = e[t];
         }
       }
     }
@@ -1327,8 +1328,8 @@ NhwcPlan plan_nhwc(const Geometry& g) {
   p.window_elems = (int64_t)g.N * g.Ho * p.strip;
   if ((int64_t)g.N * g.Ho >= lim || p.strip >= lim) return p;
   if ((int64_t)g.s * g.Kh * p.Cp * 2 >= ((int64_t)1 << 40) || p.strip * 2 >= ((int64_t)1 << 40)) return p;
-  // the transform from NCHW stages at least two columns of Cp + 2 channels in 48 KB of shared memory
-  if ((int64_t)(p.Cp + 2) * 2 * 2 > 48 * 1024) return p;
+  // the transform from NCHW stages at least eight columns of Cp + 2 channels in 48 KB of shared memory
+  if ((int64_t)(p.Cp + 2) * 2 * 8 > 48 * 1024) return p;
   // position tiles: tw tiles along a strip of bw columns each (one when the strip fits 128 rows),
   // G whole strips per tile when a strip is short
   p.tw = (g.Wo + TILE_M - 1) / TILE_M;
@@ -1385,20 +1386,24 @@ cudaError_t launch_transform_nhwc(const uint16_t* x, int x_is_nhwc, uint16_t* wi
   // columns per block: the whole row when it fits 48 KB of shared memory as T[w][Cp + 2]
   const int64_t per_col = (int64_t)(plan.Cp + 2) * 2;
   int kc = (int)((48 * 1024) / per_col);
-  if (kc < 2) return cudaErrorInvalidValue;
+  if (kc < 8) return cudaErrorInvalidValue;
   if (kc > g.W) kc = g.W;
-  else kc &= ~1;                                           // chunk boundaries stay even for the two-column loads
-  const bool vec2 = g.W % 2 == 0;
+  else kc &= ~7;                                           // chunk boundaries stay multiples of 8 for the vector loads
+  if (kc < 1) return cudaErrorInvalidValue;
+  // columns per load: rows must start on a multiple of it (W a multiple) and so must the chunks
+  const int vec = g.W % 8 == 0 ? 8 : (g.W % 4 == 0 ? 4 : (g.W % 2 == 0 ? 2 : 1));
   const int kchunks = (g.W + kc - 1) / kc;
   const int64_t blocks = (int64_t)g.N * (g.H + 2 * g.p) * kchunks;
   if (blocks >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
   const size_t smem = (size_t)(per_col * kc);
-  if (vec2)
-    transform_nhwc_from_nchw_kernel<true><<<(unsigned)blocks, 256, smem, stream>>>(x, window, g.C, plan.Cp, g.H, g.W, g.Ho, g.Wp,
-                                                                                   g.Kh, g.s, g.p, kc, kchunks);
-  else
-    transform_nhwc_from_nchw_kernel<false><<<(unsigned)blocks, 256, smem, stream>>>(x, window, g.C, plan.Cp, g.H, g.W, g.Ho, g.Wp,
-                                                                                    g.Kh, g.s, g.p, kc, kchunks);
+#define IM2WIN_LAUNCH_T(V)                                                                                          \
+  transform_nhwc_from_nchw_kernel<V><<<(unsigned)blocks, 256, smem, stream>>>(x, window, g.C, plan.Cp, g.H, g.W, g.Ho, \
+                                                                            g.Wp, g.Kh, g.s, g.p, kc, kchunks)
+  if (vec == 8) IM2WIN_LAUNCH_T(8);
+  else if (vec == 4) IM2WIN_LAUNCH_T(4);
+  else if (vec == 2) IM2WIN_LAUNCH_T(2);
+  else IM2WIN_LAUNCH_T(1);
+#undef IM2WIN_LAUNCH_T
   return cudaGetLastError();
 }
 
