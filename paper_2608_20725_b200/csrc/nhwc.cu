@@ -134,44 +134,58 @@ __device__ __forceinline__ void store_chunk(const EpiParams& q, int64_t base, in
   }
 }
 
+// Bias (first K part only), ReLU and store of 32 channels from c0 on of one accumulator row.
+__device__ __forceinline__ void finish_chunk(const EpiParams& e, uint32_t (&v)[32], int c0, int n0, bool first_part,
+                                             bool valid, int64_t base, int64_t cs, bool vec_ok) {
+  const int cnt = e.Co - n0 - c0;                // channels left from c0 on
+  if (cnt <= 0) return;
+  if (e.bias != nullptr && first_part) {
+    // every lane adds the same 32 channel values: uniform 16-byte loads (the bias is 16-byte aligned
+    // and n0 + c0 a multiple of 32), element by element at the ragged end
+    if (cnt >= 32) {
+      const float4* b4 = reinterpret_cast<const float4*>(e.bias + n0 + c0);
+#pragma unroll
+      for (int t = 0; t < 32; t += 4) {
+        const float4 b = __ldg(b4 + t / 4);
+        v[t] = __float_as_uint(__uint_as_float(v[t]) + b.x);
+        v[t + 1] = __float_as_uint(__uint_as_float(v[t + 1]) + b.y);
+        v[t + 2] = __float_as_uint(__uint_as_float(v[t + 2]) + b.z);
+        v[t + 3] = __float_as_uint(__uint_as_float(v[t + 3]) + b.w);
+      }
+    } else {
+#pragma unroll
+      for (int t = 0; t < 32; ++t)
+        if (t < cnt) v[t] = __float_as_uint(__uint_as_float(v[t]) + __ldg(e.bias + n0 + c0 + t));
+    }
+  }
+  if (e.relu) {
+#pragma unroll
+    for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(fmaxf(__uint_as_float(v[t]), 0.0f));
+  }
+  if (valid) store_chunk(e, base + (int64_t)c0 * cs, cs, v, cnt < 32 ? cnt : 32, vec_ok);
+}
+
 // One epilogue warp's share of a finished accumulator: tensor-memory lane quadrant warp % 4, the
 // lower (warps 2..5) or upper (warps 6..9) half of the tile's `cols` channels, 32 channels at a time:
-// bias (first K part only), ReLU, store.  `base` is the element index of the tile's first channel
-// at this lane's position, `cs` the element distance between channels.
+// bias, ReLU, store.  The tensor-memory load of the next 32 channels is in flight while the current
+// ones are stored (two register sets, taken in turn).  `base` is the element index of the tile's first
+// channel at this lane's position, `cs` the element distance between channels.
 __device__ __forceinline__ void drain_accumulator(const EpiParams& e, int cols, int warp, int lane, uint32_t lane_base,
                                                   bool valid, int64_t base, int64_t cs, int n0, bool first_part, bool vec_ok) {
-  const int CH = cols / 2;                       // cols is a multiple of 64
+  const int CH = cols / 2;                       // a multiple of 32
   const int cbeg = ((warp - WARP_EPI0) >> 2) * CH;
+  const int cend = cbeg + CH;
+  uint32_t va[32], vb[32];
+  tmem_ld32_issue(lane_base + (uint32_t)cbeg, va);
 #pragma unroll 1
-  for (int c0 = cbeg; c0 < cbeg + CH; c0 += 32) {
-    const int cnt = e.Co - n0 - c0;              // channels left from c0 on
-    if (cnt <= 0) break;
-    uint32_t v[32];
-    tmem_ld32(lane_base + (uint32_t)c0, v);
-    if (e.bias != nullptr && first_part) {
-      // every lane adds the same 32 channel values: uniform 16-byte loads (the bias is 16-byte aligned
-      // and n0 + c0 a multiple of 32), element by element at the ragged end
-      if (cnt >= 32) {
-        const float4* b4 = reinterpret_cast<const float4*>(e.bias + n0 + c0);
-#pragma unroll
-        for (int t = 0; t < 32; t += 4) {
-          const float4 b = __ldg(b4 + t / 4);
-          v[t] = __float_as_uint(__uint_as_float(v[t]) + b.x);
-          v[t + 1] = __float_as_uint(__uint_as_float(v[t + 1]) + b.y);
-          v[t + 2] = __float_as_uint(__uint_as_float(v[t + 2]) + b.z);
-          v[t + 3] = __float_as_uint(__uint_as_float(v[t + 3]) + b.w);
-        }
-      } else {
-#pragma unroll
-        for (int t = 0; t < 32; ++t)
-          if (t < cnt) v[t] = __float_as_uint(__uint_as_float(v[t]) + __ldg(e.bias + n0 + c0 + t));
-      }
-    }
-    if (e.relu) {
-#pragma unroll
-      for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(fmaxf(__uint_as_float(v[t]), 0.0f));
-    }
-    if (valid) store_chunk(e, base + (int64_t)c0 * cs, cs, v, cnt < 32 ? cnt : 32, vec_ok);
+  for (int c0 = cbeg; c0 < cend; c0 += 64) {
+    tmem_ld_wait_for(va);
+    if (c0 + 32 < cend) tmem_ld32_issue(lane_base + (uint32_t)(c0 + 32), vb);
+    finish_chunk(e, va, c0, n0, first_part, valid, base, cs, vec_ok);
+    if (c0 + 32 >= cend) break;
+    tmem_ld_wait_for(vb);
+    if (c0 + 64 < cend) tmem_ld32_issue(lane_base + (uint32_t)(c0 + 64), va);
+    finish_chunk(e, vb, c0 + 32, n0, first_part, valid, base, cs, vec_ok);
   }
 }
 
