@@ -126,19 +126,27 @@ class ClockSampler:
 class LayerRunner:
     """Device-resident buffers of one layer and the four calls of a step."""
 
-    def __init__(self, layer, precisions=("f32", "f16")):
+    def __init__(self, layer, precisions=("f32", "f16"), sets=1):
+        """`sets` > 1 keeps that many copies of every device buffer (inputs included), so that
+        launches queued back to back can each work on memory the one before did not touch."""
         from paper_2608_20725_b200 import binding
         self.b = binding
         self.layer = layer
         self.dims = layer.dims()
+        self.sets = sets
         x, f = workloads.make_inputs(layer)
         self.host = {}
         self.dev = {}
+        self.dev_sets = {}
         for prec in precisions:
             tdt = torch.float32 if prec == "f32" else torch.float16
             xh, fh = x.to(tdt).contiguous(), f.to(tdt).contiguous()
-            window, scratch, y = binding.alloc_layer_buffers(self.dims, tdt)
-            self.dev[prec] = dict(x=xh.cuda(), f=fh.cuda(), window=window, scratch=scratch, y=y)
+            self.dev_sets[prec] = []
+            for i in range(sets):
+                window, scratch, y = binding.alloc_layer_buffers(self.dims, tdt)
+                xd = xh.cuda() if i == 0 else self.dev_sets[prec][0]["x"].clone()
+                self.dev_sets[prec].append(dict(x=xd, f=fh.cuda(), window=window, scratch=scratch, y=y))
+            self.dev[prec] = self.dev_sets[prec][0]
             self.host[prec] = (xh, fh)
         code = binding.F32 if "f32" in precisions else binding.F16
         _, _, self.ho, self.wo = binding.im2win_workspace_size(self.dims, code)
@@ -151,44 +159,49 @@ class LayerRunner:
         filter, NHWC window tensor, fp32 NCHW output."""
         b = self.b
         x, f = workloads.make_inputs(self.layer)
-        window, scratch, y = b.alloc_nhwc_buffers(self.dims)
-        self.nhwc = dict(x=x.half().cuda(), f=f.half().cuda(), window=window, scratch=scratch, y=y,
-                         cp=b.im2win_nhwc_workspace_size(self.dims)[4],
-                         y16=torch.empty(y.shape, dtype=torch.float16, device="cuda"),
-                         bias=torch.zeros(self.layer.Co, dtype=torch.float32, device="cuda"))
-        self.nhwc["epi16"] = b.make_epilogue(self.nhwc["bias"], True, torch.float16, b.NCHW)
+        x16, f16 = x.half().cuda(), f.half().cuda()
+        cp = b.im2win_nhwc_workspace_size(self.dims)[4]
+        self.nhwc_sets = []
+        for i in range(self.sets):
+            window, scratch, y = b.alloc_nhwc_buffers(self.dims)
+            d = dict(x=x16 if i == 0 else x16.clone(), f=f16 if i == 0 else f16.clone(), window=window,
+                     scratch=scratch, y=y, cp=cp, y16=torch.empty(y.shape, dtype=torch.float16, device="cuda"),
+                     bias=torch.zeros(self.layer.Co, dtype=torch.float32, device="cuda"))
+            d["epi16"] = b.make_epilogue(d["bias"], True, torch.float16, b.NCHW)
+            self.nhwc_sets.append(d)
+        self.nhwc = self.nhwc_sets[0]
 
-    def transform_nhwc(self, prec=None):
-        d = self.nhwc
+    def transform_nhwc(self, prec=None, i=0):
+        d = self.nhwc_sets[i]
         self.b.im2win_transform_nhwc(d["x"], self.b.NCHW, d["window"], self.dims)
 
-    def conv_nhwc(self, prec=None):
-        d = self.nhwc
+    def conv_nhwc(self, prec=None, i=0):
+        d = self.nhwc_sets[i]
         self.b.im2win_conv_f16_nhwc(d["window"], d["f"], d["y"], d["scratch"], self.dims)
 
-    def conv_nhwc_out16(self, prec=None):
+    def conv_nhwc_out16(self, prec=None, i=0):
         """The same convolution with the fused epilogue: bias, ReLU, binary16 NCHW output."""
-        d = self.nhwc
+        d = self.nhwc_sets[i]
         self.b.im2win_conv_f16_nhwc(d["window"], d["f"], d["y16"], d["scratch"], self.dims, d["epi16"])
 
-    def conv_nhwc_packed(self, prec=None):
-        d = self.nhwc
+    def conv_nhwc_packed(self, prec=None, i=0):
+        d = self.nhwc_sets[i]
         self.b.im2win_conv_packed_nhwc(d["window"], d["y"], d["scratch"], self.dims)
 
-    def transform(self, prec):
-        d = self.dev[prec]
+    def transform(self, prec, i=0):
+        d = self.dev_sets[prec][i]
         self.b.im2win_transform(d["x"], d["window"], self.dims)
 
-    def conv(self, prec):
-        d = self.dev[prec]
+    def conv(self, prec, i=0):
+        d = self.dev_sets[prec][i]
         if prec == "f32":
             self.b.im2win_conv_f32(d["window"], d["f"], d["y"], d["scratch"], self.dims)
         else:
             self.b.im2win_conv_f16(d["window"], d["f"], d["y"], d["scratch"], self.dims)
 
-    def conv_packed(self, prec):
+    def conv_packed(self, prec, i=0):
         """The convolution alone, on the filter the last conv() call left packed in scratch."""
-        d = self.dev[prec]
+        d = self.dev_sets[prec][i]
         self.b.im2win_conv_packed(d["window"], d["y"], d["scratch"], self.dims)
 
     def step(self, events=None):
@@ -455,9 +468,45 @@ def time_call(fn, iters, flush):
     return total / iters, best, samples[len(samples) // 2]
 
 
+def time_back_to_back(fn, sets, launches):
+    """Device time per launch (ms) of `launches` calls fn(i) queued back to back between one pair of
+    events, call j on buffer set j % sets.  The sets together exceed the L2 several times (or one
+    call's own buffers do), so no call finds its inputs cached; unlike time_call the figure leaves out
+    the fixed cost of an isolated launch (event bracket, idle-GPU start, nothing queued behind it)."""
+    for i in range(sets):
+        fn(i)
+    torch.cuda.synchronize()
+    torch.cuda._sleep(600_000)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for j in range(launches):
+        fn(j % sets)
+    e1.record()
+    e1.synchronize()
+    return e0.elapsed_time(e1) / launches
+
+
+L2_BYTES = 126 << 20
+
+
+def buffer_sets_for(layer):
+    """Buffer sets for back-to-back timing: one when a single call already moves two L2 sizes, else
+    enough (at most 12) that the sets a call does not touch hold three L2 sizes."""
+    from paper_2608_20725_b200 import binding
+    _, _, ho, wo = binding.im2win_workspace_size(layer.dims(), binding.F32 if "f32" in layer.precisions else binding.F16)
+    x_el = layer.N * layer.C * layer.H * layer.W
+    win_el = layer.N * layer.C * ho * layer.Kh * (layer.W + 2 * layer.pad)
+    out_el = layer.N * layer.Co * ho * wo
+    smallest = min((x_el + win_el) * 2, win_el * 2 + out_el * 2)     # fewest bytes a timed call touches (fp16 sizes)
+    if smallest >= 2 * L2_BYTES:
+        return 1
+    return max(2, min(12, 1 + -(-3 * L2_BYTES // smallest)))
+
+
 def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
     """Times every call of the named layers (default: all BASELINE configs) one by one: transform and
-    convolution (filter pack included) per precision, L2 flushed before each launch."""
+    convolution (filter pack included) per precision, L2 flushed before each launch; then the same
+    calls queued back to back over rotating buffer sets."""
     from paper_2608_20725_b200 import binding
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
     rows = []
@@ -466,16 +515,19 @@ def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
     for name in (names or list(workloads.LAYERS)):
         layer = table[name]
         print(f"[report] {name}", file=sys.stderr, flush=True)
-        runner = LayerRunner(layer, layer.precisions)
+        sets = buffer_sets_for(layer)
+        runner = LayerRunner(layer, layer.precisions, sets=sets)
         for _ in range(3):
             runner.step()
         torch.cuda.synchronize()
-        avg, best, median = {}, {}, {}
+        avg, best, median, b2b = {}, {}, {}, {}
         for prec in layer.precisions:
             for kind, fn in (("transform", runner.transform), ("conv", runner.conv)):
                 key = f"{kind}_{prec}"
                 avg[key], best[key], median[key] = time_call(lambda: fn(prec), iters, flush)
-            binding.im2win_check_status(runner.dev[prec]["scratch"])
+                b2b[key] = time_back_to_back(lambda i: fn(prec, i), sets, iters)
+            for d in runner.dev_sets[prec]:
+                binding.im2win_check_status(d["scratch"])
         if "f16" in layer.precisions:
             # the channel-innermost (NHWC) form of the fp16 path on the same layer
             runner.add_nhwc()
@@ -485,9 +537,13 @@ def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
             for key, fn in (("transform_f16_nhwc", runner.transform_nhwc), ("conv_f16_nhwc", runner.conv_nhwc),
                             ("conv_f16_out16_nhwc", runner.conv_nhwc_out16)):
                 avg[key], best[key], median[key] = time_call(fn, iters, flush)
-            binding.im2win_check_status(runner.nhwc["scratch"])
+                b2b[key] = time_back_to_back(lambda i: fn(None, i), sets, iters)
+            for d in runner.nhwc_sets:
+                binding.im2win_check_status(d["scratch"])
         row = {"layer": name, "dims": layer.dims(), "gflop": runner.flops / 1e9, "avg_ms": avg, "best_ms": best,
-               "median_ms": median, "kernels": kernel_rooflines(runner, avg, peaks, peak_kind),
+               "median_ms": median, "back_to_back_ms": b2b, "buffer_sets": sets,
+               "kernels": kernel_rooflines(runner, avg, peaks, peak_kind),
+               "kernels_back_to_back": kernel_rooflines(runner, b2b, peaks, peak_kind),
                "conv_kernel": {p: binding.im2win_conv_kernel_name(layer.dims(), binding.F32 if p == "f32" else binding.F16)
                                for p in layer.precisions},
                "memory": runner.memory_report()}
@@ -499,7 +555,8 @@ def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
                 packed[f"conv_{prec}"] = {"avg_ms": a, "best_ms": b_, "median_ms": m}
             if runner.nhwc is not None:
                 a, b_, m = time_call(runner.conv_nhwc_packed, iters, flush)
-                packed["conv_f16_nhwc"] = {"avg_ms": a, "best_ms": b_, "median_ms": m}
+                packed["conv_f16_nhwc"] = {"avg_ms": a, "best_ms": b_, "median_ms": m,
+                                           "back_to_back_ms": time_back_to_back(lambda i: runner.conv_nhwc_packed(None, i), sets, iters)}
             row["conv_without_pack"] = packed
         rows.append(row)
         del runner
@@ -524,12 +581,16 @@ def per_layer_summary(rows):
         for key, k in row["kernels"].items():
             e = {"ms": round(k["ms"], 5), "bound": k["bound"], "frac": round(k["frac"], 4),
                  "achieved": round(k["achieved"], 2), "unit": k["unit"]}
+            kb = row["kernels_back_to_back"][key]
+            # the same call queued back to back over `buffer_sets` rotating buffer sets (no isolated-launch cost)
+            e["back_to_back"] = {"ms": round(kb["ms"], 5), "bound": kb["bound"], "frac": round(kb["frac"], 4)}
             if key.startswith("conv"):
                 e["tflops"] = round(row["gflop"] / k["ms"], 2)      # GFLOP per ms = TFLOP/s
                 e["kernel"] = "f16-nhwc-tma" if key.endswith("nhwc") else row["conv_kernel"][key.split("_")[1]]
                 if key.startswith("conv_f16"):
                     e["frac_of_tensor_peak"] = round(k["frac_of_tensor_peak"], 4)
             entry[key] = e
+        entry["buffer_sets"] = row["buffer_sets"]
         entry["memory"] = {p: {"window_bytes": m["window_bytes"], "output_bytes": m["output_bytes"],
                                "im2col_bytes": m["im2col_bytes"]} for p, m in row["memory"].items()}
         out[row["layer"]] = entry

@@ -866,6 +866,9 @@ pack_f16_nhwc_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, 
   const int nc = Cp - c0 < cb ? Cp - c0 : cb;     // stored channels of this block (Cp and cb are multiples of 8)
   const int nreal = C - c0 < nc ? (C - c0 > 0 ? C - c0 : 0) : nc;
   const int pairs = nc / 2;
+  int ncc_log2 = 0;
+  while ((1 << ncc_log2) < pairs && (1 << ncc_log2) < (int)blockDim.x) ++ncc_log2;
+  const int ncc = 1 << ncc_log2, ntt = (int)blockDim.x >> ncc_log2;   // blockDim.x is a power of two
   for (int co = blockIdx.y; co < Co; co += gridDim.y) {
     const uint16_t* src = f + ((int64_t)co * C + c0) * T;
     // the run is read with 16-byte loads from the first 16-byte boundary on (shared-memory copy kept at
@@ -889,14 +892,26 @@ pack_f16_nhwc_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, 
     }
     const uint16_t* ps = dst;                       // element i of the run is ps[i]
     __syncthreads();
-    // thread -> (t = v*Kh + u, channel pair): 4-byte stores, consecutive threads along c
-    for (int i = threadIdx.x; i < T * pairs; i += blockDim.x) {
-      const int t = i / pairs, cp2 = i - t * pairs;
-      const int v = t / Kh, u = t - v * Kh;
-      const int c = 2 * cp2;
-      const uint32_t lo = c < nreal ? ps[c * T + u * Kw + v] : 0u;
-      const uint32_t hi = c + 1 < nreal ? ps[(c + 1) * T + u * Kw + v] : 0u;
-      *reinterpret_cast<uint32_t*>(fp + (int64_t)co * K + (int64_t)t * Cp + c0 + c) = lo | (hi << 16);
+    // 4-byte stores (a channel pair each), consecutive threads along c.  The threads form ntt rows of
+    // ncc (a power of two): a row walks t = v*Kh + u in steps of ntt, its threads the channel pairs;
+    // (v, u) advance by additions, so that the loop holds no division.
+    {
+      uint32_t* out_co = reinterpret_cast<uint32_t*>(fp + (int64_t)co * K + c0);
+      const int tx = (int)threadIdx.x & (ncc - 1), ty = (int)threadIdx.x >> ncc_log2;
+      const int dv = ntt / Kh, du = ntt - dv * Kh;
+      int v = ty / Kh, u = ty - v * Kh;
+      for (int t = ty; t < T; t += ntt) {
+        const uint16_t* pt = ps + u * Kw + v;
+        uint32_t* orow = out_co + ((t * Cp) >> 1);
+        for (int cp2 = tx; cp2 < pairs; cp2 += ncc) {
+          const int c = 2 * cp2;
+          const uint32_t lo = c < nreal ? pt[c * T] : 0u;
+          const uint32_t hi = c + 1 < nreal ? pt[(c + 1) * T] : 0u;
+          orow[cp2] = lo | (hi << 16);
+        }
+        u += du; v += dv;
+        if (u >= Kh) { u -= Kh; ++v; }
+      }
     }
     __syncthreads();
   }
