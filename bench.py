@@ -534,8 +534,11 @@ def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
             for _ in range(3):
                 runner.transform_nhwc()
                 runner.conv_nhwc()
+            # conv_packed_*: the convolution on a filter packed beforehand (static weights), i.e. without
+            # the pack kernel that conv_f16_nhwc runs on every call
             for key, fn in (("transform_f16_nhwc", runner.transform_nhwc), ("conv_f16_nhwc", runner.conv_nhwc),
-                            ("conv_f16_out16_nhwc", runner.conv_nhwc_out16)):
+                            ("conv_f16_out16_nhwc", runner.conv_nhwc_out16),
+                            ("conv_packed_f16_nhwc", runner.conv_nhwc_packed)):
                 avg[key], best[key], median[key] = time_call(fn, iters, flush)
                 b2b[key] = time_back_to_back(lambda i: fn(None, i), sets, iters)
             for d in runner.nhwc_sets:
@@ -587,7 +590,7 @@ def per_layer_summary(rows):
             if key.startswith("conv"):
                 e["tflops"] = round(row["gflop"] / k["ms"], 2)      # GFLOP per ms = TFLOP/s
                 e["kernel"] = "f16-nhwc-tma" if key.endswith("nhwc") else row["conv_kernel"][key.split("_")[1]]
-                if key.startswith("conv_f16"):
+                if "f16" in key:
                     e["frac_of_tensor_peak"] = round(k["frac_of_tensor_peak"], 4)
             entry[key] = e
         entry["buffer_sets"] = row["buffer_sets"]

@@ -454,7 +454,8 @@ conv_f16_nhwc_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid
 // i >= Wo are computed and dropped (useful fraction Wo/Wq).  Per k2-block the activation bytes that
 // cross from L2 to the SM shrink from Kw*16 KB to 16 KB + halo; the filter tiles (one per (k2-block,
 // kernel column), streamed through their own ring, or resident when the layer's whole filter
-// fits) stay as they were.  Needs s | Wp and Kw >= 2.
+// fits) stay as they were.  Needs s | Wp.  Of the s column classes only those some kernel column reads
+// (min(s, Kw)) are copied; a 1x1 layer is then a plain product over full 128-position tiles.
 constexpr int MAX_SA = 6, MAX_SB = 12;
 constexpr int MAX_KW = 64;                     // kernel widths the shifted-view kernel takes
 constexpr int WARP_BLOAD = 2 + EPI_WARPS;      // the filter-copy warp of this kernel
@@ -556,6 +557,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
     // (the whole warp walks the loops and takes the waits, one elected lane issues)
     {
       const bool leader = elect_one();
+      const int ncls = q.s < q.Kw ? q.s : q.Kw;   // column classes some kernel column reads
       wait_for_previous_kernel();
       int st = 0;
       uint32_t ph = 0;
@@ -577,8 +579,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
             const uint32_t dst = a_ring + (uint32_t)st * q.a_stage_bytes;
             const uint32_t bar = a_full_dst + 8 * st;
             if (!PAIR || rank == 0)
-              mbar_arrive_expect_tx(a_full0 + 8 * st, (PAIR ? 2u : 1u) * (uint32_t)(q.s * q.rows * KB * 2));
-            for (int t = 0; t < q.s; ++t) {
+              mbar_arrive_expect_tx(a_full0 + 8 * st, (PAIR ? 2u : 1u) * (uint32_t)(ncls * q.rows * KB * 2));
+            for (int t = 0; t < ncls; ++t) {
               if (PAIR) tma_load_3d_pair(dst + (uint32_t)t * q.subt_bytes, &amap, kb * KB, t, q0, bar);
               else tma_load_3d(dst + (uint32_t)t * q.subt_bytes, &amap, kb * KB, t, q0, bar);
             }
@@ -1051,6 +1053,108 @@ transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __rest
   }
 }
 
+// x given NCHW with at most 8 channels (Cp = 8, the 3-channel stems): a column of the window tensor is
+// one 16-byte chunk per (k, u), and the per-row kernel above would scatter such chunks Kh*16 bytes
+// apart.  Here one block builds one whole strip (n, ho) in shared memory in output order and writes
+// it out as one contiguous run.  The input rows a strip needs are, per channel, one contiguous run
+// of the input (rows ho*s - p .. + Kh - 1, clipped to the image): the C runs are brought into a
+// staging area with 16-byte loads from their first 16-byte boundary on (all in flight together; a
+// run is read by the Kh/s strips that hold its rows, from L2 after the first), then scattered inside
+// shared memory to S[k][u][c]; everything else (padding, channels C..7) stays zero.  A column of S is
+// PW = 4*Kh + 1 words apart, an odd number, so that the scatter and the read-out spread over the
+// banks.
+__global__ void __launch_bounds__(256)
+transform_nhwc_strip_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ win, int C, int H, int W, int Ho,
+                            int Wp, int Kh, int s, int p, int SP) {
+  extern __shared__ __align__(16) uint32_t strip_s[];     // [Wp][PW] words, then the staging area [C][SP] halves
+  const int PW = 4 * Kh + 1;
+  const int strip_words = (Wp * PW + 3) & ~3;
+  uint16_t* stage = reinterpret_cast<uint16_t*>(strip_s + strip_words);
+  const int64_t n = blockIdx.x / Ho;
+  const int ho = (int)(blockIdx.x - n * Ho);
+  // rows of the image this strip holds: u_lo .. u_hi of its Kh rows
+  const int h0 = ho * s - p;
+  const int u_lo = h0 < 0 ? -h0 : 0;
+  const int u_hi = h0 + Kh - 1 < H ? Kh - 1 : H - 1 - h0;
+  const int L = (u_hi - u_lo + 1) * W;                    // halves per channel run (<= 0: none)
+  const int NV = L > 0 ? L / 8 + 1 : 0;                   // 16-byte pieces a run may span after its head
+  const int step = (int)blockDim.x;
+  const uint16_t* run0 = x + ((n * C) * H + (h0 + u_lo)) * (int64_t)W;         // channel c: + c*H*W
+  const int64_t cstride = (int64_t)H * W;
+  // halves before the first 16-byte boundary of channel c's run
+  const int ph0 = (int)((reinterpret_cast<uintptr_t>(run0) >> 1) & 7u), cs7 = (int)(cstride & 7);
+  auto head_of = [&](int c) { return (8 - ((ph0 + c * cs7) & 7)) & 7; };
+  if (L > 0) {
+    // 16-byte pieces, four in flight per thread: item -> (c, piece)
+    for (int i0 = threadIdx.x; i0 < C * NV; i0 += 4 * step) {
+      uint4 r[4];
+      int dsts[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        dsts[j] = -1;
+        const int i = i0 + j * step;
+        if (i < C * NV) {
+          const int c = i / NV, v = i - c * NV;
+          const uint16_t* src = run0 + c * cstride;
+          const int head = head_of(c);
+          if (head + 8 * v + 8 <= L) {
+            dsts[j] = c * SP + 8 + 8 * v;                 // the staged run keeps the phase: element e at c*SP + 8 - head + e
+            r[j] = __ldg(reinterpret_cast<const uint4*>(src + head + 8 * v));
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (dsts[j] >= 0) *reinterpret_cast<uint4*>(stage + dsts[j]) = r[j];
+    }
+    // the ragged ends of every run, element by element: at most 7 + 7 halves per channel
+    for (int i = threadIdx.x; i < C * 16; i += step) {
+      const int c = i >> 4, e = i & 15;
+      const uint16_t* src = run0 + c * cstride;
+      const int head = head_of(c);
+      const int nvec = L > head ? (L - head) / 8 : 0;
+      int idx = -1;
+      if (e < 8) { if (e < head && e < L) idx = e; }                        // before the boundary
+      else { const int t = head + 8 * nvec + (e - 8); if (t < L && t >= head) idx = t; }   // after the last whole piece
+      if (idx >= 0) stage[c * SP + 8 - head + idx] = __ldg(src + idx);
+    }
+  }
+  {
+    const int total = Wp * PW, quads = total / 4;
+    for (int i = threadIdx.x; i < quads; i += step) reinterpret_cast<uint4*>(strip_s)[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = 4 * quads + threadIdx.x; i < total; i += step) strip_s[i] = 0u;
+  }
+  __syncthreads();
+  // scatter inside shared memory: a warp takes the rows (c, u) in turn, its lanes walk the columns
+  if (L > 0) {
+    uint16_t* sh = reinterpret_cast<uint16_t*>(strip_s);
+    const int rows = u_hi - u_lo + 1;
+    const int warp = (int)threadIdx.x >> 5, lane = (int)threadIdx.x & 31, nwarps = step >> 5;
+    for (int c = 0; c < C; ++c) {
+      const uint16_t* src_c = stage + c * SP + 8 - head_of(c);       // element 0 of channel c's run
+      for (int r = warp; r < rows; r += nwarps) {
+        const uint16_t* src = src_c + r * W;
+        uint16_t* dst = sh + (p * PW + 4 * (r + u_lo)) * 2 + c;
+        for (int w = lane; w < W; w += 32) dst[w * PW * 2] = src[w];
+      }
+    }
+  }
+  __syncthreads();
+  // read-out: chunk j = k*Kh + u of the strip, consecutive threads consecutive chunks
+  {
+    uint4* dst = reinterpret_cast<uint4*>(win + (n * Ho + ho) * (int64_t)Wp * Kh * 8);
+    const int chunks = Wp * Kh;
+    const int d_k = step / Kh, d_u = step - d_k * Kh;
+    int k = (int)threadIdx.x / Kh, u = (int)threadIdx.x - k * Kh;
+    for (int j = threadIdx.x; j < chunks; j += step) {
+      const uint32_t* src = strip_s + k * PW + 4 * u;
+      dst[j] = make_uint4(src[0], src[1], src[2], src[3]);
+      u += d_u; k += d_k;
+      if (u >= Kh) { u -= Kh; ++k; }
+    }
+  }
+}
+
 // ------------------------------------------------------------------- host side
 // Testing aid: with IM2WIN_DEBUG and IM2WIN_VERBOSE set, a failed host-side step says what failed.
 cudaError_t report(cudaError_t e, const char* what) {
@@ -1184,14 +1288,14 @@ struct ShiftViewPlan {
 ShiftViewPlan plan_shift_view(const Geometry& g, const NhwcPlan& plan) {
   ShiftViewPlan p{};
   p.eligible = false;
-  if (g.Kw < 2 || g.Kw > MAX_KW || g.Wp % g.s != 0 || g.s > 16) return p;
+  if (g.Kw > MAX_KW || g.Wp % g.s != 0 || g.s > 16) return p;
   p.Wq = g.Wp / g.s;
   p.VQ = (int64_t)g.N * g.Ho * p.Wq;
   if (p.VQ >= ((int64_t)1 << 31) - 4 * TILE_M) return p;
   p.rows = TILE_M + (g.Kw - 1) / g.s;
   if (p.rows > 256) return p;
   p.subt_bytes = (uint32_t)((p.rows * KB * 2 + 1023) / 1024 * 1024);
-  p.a_stage_bytes = (uint32_t)g.s * p.subt_bytes;
+  p.a_stage_bytes = (uint32_t)(g.s < g.Kw ? g.s : g.Kw) * p.subt_bytes;
   p.K2 = (int64_t)g.Kh * plan.Cp;
   p.nkb2 = (int32_t)((p.K2 + KB - 1) / KB);
   p.nks_last = (int32_t)((p.K2 - (int64_t)(p.nkb2 - 1) * KB + 15) / 16);
@@ -1412,6 +1516,24 @@ cudaError_t launch_transform_nhwc(const uint16_t* x, int x_is_nhwc, uint16_t* wi
                                                                           g.Kh, g.s, g.p, chunks);
     return cudaGetLastError();
   }
+  // at most 8 channels: one block per strip, built in shared memory and written as one run
+  const int SP = (g.Kh * g.W + 16 + 7) & ~7;              // staged halves per channel: a run plus the phase padding
+  const int64_t strip_smem = (((int64_t)g.Wp * (4 * g.Kh + 1) + 3) & ~(int64_t)3) * 4 + (int64_t)g.C * SP * 2;
+  bool by_strip = plan.Cp == 8 && strip_smem <= 100 * 1024 && (int64_t)g.N * g.Ho < ((int64_t)1 << 31);
+  if (const char* v = debug_getenv("IM2WIN_NHWC_TRANSFORM")) by_strip = by_strip && strcmp(v, "rows") != 0;
+  if (by_strip) {
+    static bool attr_done[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (strip_smem > 48 * 1024 && !attr_done[dev]) {
+      cudaError_t e = cudaFuncSetAttribute(transform_nhwc_strip_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+      if (e != cudaSuccess) return e;
+      attr_done[dev] = true;
+    }
+    transform_nhwc_strip_kernel<<<(unsigned)((int64_t)g.N * g.Ho), 256, (size_t)strip_smem, stream>>>(
+        x, window, g.C, g.H, g.W, g.Ho, g.Wp, g.Kh, g.s, g.p, SP);
+    return cudaGetLastError();
+  }
   // columns per block: the whole row when it fits 48 KB of shared memory as T[w][Cp + 2]
   const int64_t per_col = (int64_t)(plan.Cp + 2) * 2;
   int kc = (int)((48 * 1024) / per_col);
@@ -1487,7 +1609,11 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   // stages; elsewhere the overlapping-row kernel is as fast or faster.
   const ShiftViewPlan sp = plan_shift_view(g, plan);
   const int64_t b_bytes = (int64_t)(plan.pair ? plan.bn / 2 : plan.bn) * KB * 2;
-  bool use_shift = sp.eligible && g.Kw >= 3 * g.s &&
+  // Kernels no wider than the stride read every column once in either kernel; there the shifted view
+  // is taken when its full 128-position tiles need fewer rounds than the overlapping-row kernel's
+  // tiles of whole strips.
+  const bool reuse = g.Kw >= 3 * g.s, once = g.Kw <= g.s;
+  bool use_shift = sp.eligible && (reuse || (once && plan.ksplit == 1)) &&
                    2 * (int64_t)sp.a_stage_bytes + 2 * (int64_t)g.Kw * b_bytes <= kSmemMax - 2048;
   if (use_shift && plan.ksplit == 1) {
     // Rounds of tiles on the CTAs (pairs): the overlapping-row kernel can hand the tiles of a last round
@@ -1500,7 +1626,7 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
     const int64_t tail = it_o % slots;
     const double r_o = (double)(it_o / slots) + (tail == 0 ? 0.0 : (plan.bn >= 128 && 2 * tail <= slots ? 0.55 : 1.0));
     const double r_s = (double)((it_s + slots - 1) / slots);
-    if (r_o < 0.85 * r_s) use_shift = false;
+    if (reuse ? r_o < 0.85 * r_s : r_o <= r_s) use_shift = false;
   }
   if (const char* v = debug_getenv("IM2WIN_NHWC_KERNEL")) {
     if (strcmp(v, "shift") == 0) use_shift = sp.eligible;

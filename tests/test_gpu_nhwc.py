@@ -36,12 +36,18 @@ SMALL = [
     L("pair_s2", 2, 24, 16, 14, 200, 3, 3, 2, 1, 26),
     L("stem7", 2, 3, 37, 37, 64, 7, 7, 2, 3, 12),
     L("many_kb", 1, 64, 9, 9, 40, 5, 5, 1, 2, 27),              # 25 k-blocks: the stage ring wraps several times
+    L("one_by_one_s2", 2, 24, 14, 14, 40, 1, 1, 2, 0, 28),      # kernel narrower than the stride: one column class of two is read
+    L("one_by_one_big", 5, 72, 13, 13, 136, 1, 1, 1, 0, 29),    # 1x1 over several full position tiles
 ]
 
 
 @pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
-@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
-def test_transform_nhwc_bit_exact(layer, layout):
+@pytest.mark.parametrize("layout,variant", [("nchw", "default"), ("nchw", "rows"), ("nhwc", "default")])
+def test_transform_nhwc_bit_exact(layer, layout, variant, monkeypatch):
+    """From either input layout; from NCHW through the kernel the library picks (one block per strip
+    for up to 8 channels, else one block per input row) and through the per-row kernel forced."""
+    if variant != "default":
+        monkeypatch.setenv("IM2WIN_NHWC_TRANSFORM", variant)
     dims = layer.dims()
     x, _ = workloads.make_inputs(layer)
     raw = x.half().view(torch.int16)
@@ -86,7 +92,7 @@ def test_conv_nhwc_parity_small(layer, layout, kernel, monkeypatch):
 
 
 @pytest.mark.parametrize("layer", [SMALL[0], SMALL[2], SMALL[3], SMALL[4], SMALL[6], SMALL[7], SMALL[9], SMALL[11],
-                                   SMALL[12], SMALL[14], SMALL[15]], ids=lambda l: l.name)
+                                   SMALL[12], SMALL[14], SMALL[15], SMALL[18], SMALL[19]], ids=lambda l: l.name)
 @pytest.mark.parametrize("kernel", ["overlap", "shift"])
 @pytest.mark.parametrize("bn,pair,ksplit", [("64", "0", "1"), ("128", "0", "1"), ("128", "1", "1"), ("256", "0", "1"),
                                             ("256", "1", "1"), ("128", "0", "3"), ("256", "1", "2"), ("64", "0", "20")])
