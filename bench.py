@@ -334,8 +334,8 @@ def run_gpu_arm(args):
         torch.cuda.synchronize()
 
     layer = workloads.LAYERS[workloads.BENCH_LAYER]
-    runner = LayerRunner(layer)
     peaks, peak_kind = load_peaks()
+    runner = LayerRunner(layer)
     torch.cuda.reset_peak_memory_stats()
 
     for _ in range(args.warmup):
