@@ -38,6 +38,7 @@
 #include <stdlib.h>
 
 #include "common.cuh"
+#define IM2WIN_INLINE_SLOW_WAIT   // the slow path of the bounded waits expanded in place: faster in this kernel
 #include "ptx_sm100.cuh"
 
 namespace im2win {
