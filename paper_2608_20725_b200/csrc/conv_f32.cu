@@ -46,7 +46,7 @@ __device__ __forceinline__ float2 unpack2(unsigned long long v) {
 }
 
 template <int BM, int BN>
-__global__ void __launch_bounds__((BM / 8) * (BN / 8), ((BM / 8) * (BN / 8) == 256 ? 2 : 1))
+__global__ void __launch_bounds__((BM / 8) * (BN / 8), ((BM / 8) * (BN / 8) == 256 ? 2 : 3))
 conv_f32_kernel(ConvF32Params q) {
   constexpr int THREADS = (BM / 8) * (BN / 8);
   constexpr int A_PER_THREAD = BK * BM / THREADS;         // scalar gathers per k-block
@@ -216,7 +216,13 @@ cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, 
     const int64_t tiles = (g.P + bm - 1) / bm * cot;
     return (double)((tiles + 147) / 148) * bm;
   };
-  const bool small_m = waves_cost(64) < 0.9 * waves_cost(128);
+  bool small_m = waves_cost(64) < 0.9 * waves_cost(128);
+  // 128-channel tiles: with four to eight 128-position tiles per SM the partly filled last round of
+  // 256-thread CTAs costs more than the 64-position tile's extra filter traffic (measured on 3x3 to
+  // 7x7 layers at 28x28 and 10x10: 3-5 % faster; larger grids are 3-4 % faster with 128 positions)
+  const int64_t tiles128 = (g.P + 127) / 128 * cot;
+  if (wide && tiles128 >= 4 * 148 && tiles128 < 8 * 148) small_m = true;
+  if (const char* v = debug_getenv("IM2WIN_F32_BM")) small_m = atoi(v) == 64;   // testing aid
   const int bm = small_m ? 64 : 128;
   dim3 grid((unsigned)((g.P + bm - 1) / bm), (unsigned)cot);
   const int threads = (bm / 8) * (bn / 8);

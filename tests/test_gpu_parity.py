@@ -128,6 +128,23 @@ def test_conv_exact_on_integer_inputs(layer, precision):
     assert np.array_equal(y.astype(np.float64), yr)
 
 
+@pytest.mark.parametrize("layer", [SMALL[1], SMALL[2], L("wide_co", 3, 20, 11, 13, 150, 3, 3, 1, 1, 47)], ids=lambda l: l.name)
+@pytest.mark.parametrize("bm", ["64", "128"])
+def test_conv_f32_both_tile_heights(layer, bm, monkeypatch):
+    """The fp32 kernel's 64- and 128-position tiles (the library picks by grid size), on 64- and
+    128-channel tiles: exact on integer-valued inputs, within tolerance on the seeded ones."""
+    monkeypatch.setenv("IM2WIN_F32_BM", bm)
+    dims = layer.dims()
+    x, f = workloads.make_small_integer_inputs(layer)
+    y, _, _ = gpu_conv(x, f, dims, "f32")
+    yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+    assert np.array_equal(y.astype(np.float64), yr)
+    x, f = workloads.make_inputs(layer)
+    y, _, _ = gpu_conv(x, f, dims, "f32")
+    yr, ar = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+    check_conv(y, yr, ar, "f32", layer.name)
+
+
 def test_f16_inputs_are_the_oracles_rounding():
     """The cast that feeds the fp16 path (torch .half()) and the oracle's rounding agree bit for bit."""
     layer = workloads.LAYERS["cfg5k11"].with_batch(1)
