@@ -968,87 +968,106 @@ __global__ void transform_nhwc_from_nhwc_kernel(const uint16_t* __restrict__ x, 
 template <int VEC>
 __global__ void __launch_bounds__(256)
 transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ win, int C, int Cp, int H, int W,
-                                int Ho, int Wp, int Kh, int s, int p, int kc, int kchunks) {
+                                int Ho, int Wp, int Kh, int s, int p, int kc, int kchunks, int R, int rgroups) {
   extern __shared__ __align__(16) uint16_t rows_s[];     // T[kc][Cp + 2]
   const int PC = Cp + 2;
-  int64_t b = blockIdx.x;
-  const int kci = (int)(b % kchunks); b /= kchunks;
-  const int hp = (int)(b % (H + 2 * p));                  // row of the padded input
-  const int64_t n = b / (H + 2 * p);
-  const int h = hp - p;
-  const bool row_ok = h >= 0 && h < H;
-  // the strips that hold this row: ho*s + u = hp with 0 <= u < Kh
-  const int ho_hi = hp / s < Ho - 1 ? hp / s : Ho - 1;
-  int ho_lo = hp - Kh + 1 > 0 ? (hp - Kh + 1 + s - 1) / s : 0;
-  if (ho_lo > ho_hi) return;                              // a row no window reaches
+  // block -> (image n, group of R consecutive rows of the padded input, column chunk); 32-bit
+  // arithmetic (the host keeps the block count below 2^31): the set-up is paid by every thread of
+  // every block, and a block's own work is only a few instructions per thread and row
+  uint32_t b = blockIdx.x;
+  const int kci = (int)(b % (uint32_t)kchunks); b /= (uint32_t)kchunks;
+  const int rg = (int)(b % (uint32_t)rgroups);
+  const int64_t n = b / (uint32_t)rgroups;
   const int w0 = kci * kc;
   const int nw = W - w0 < kc ? W - w0 : kc;               // input columns of this block
   // its columns of the window tensor: k = w + p, plus the left padding for the first chunk and the
   // right padding for the last
   const int k_lo = kci == 0 ? 0 : w0 + p;
   const int k_hi = kci == kchunks - 1 ? Wp : w0 + nw + p; // exclusive
-  if (row_ok) {
-    if (Cp > C) {                                         // the zero channels C .. Cp-1
-      const int extra = Cp - C;
-      for (int i = threadIdx.x; i < nw * extra; i += blockDim.x) {
-        const int r = i / extra, e = i - r * extra;
-        rows_s[r * PC + C + e] = 0;
-      }
-    }
-    // phase 1: item -> (c, group of VEC columns), columns fastest (W, w0 and nw are multiples of
-    // VEC): one VEC*2-byte load, VEC transposing 2-byte stores; four loads in flight per thread
-    typedef typename VecType<VEC>::type V;
-    const int nwi = nw / VEC;
-    const int items = C * nwi;
-    const int step = (int)blockDim.x;
-    const int d_c = step / nwi, d_col = step - d_c * nwi;
-    int c = (int)threadIdx.x / nwi, col = (int)threadIdx.x - c * nwi;
-    const uint16_t* xrow = x + ((n * C) * H + h) * (int64_t)W + w0;      // channel c: + c*H*W
-    const int64_t cstride = (int64_t)H * W;
-    for (int i0 = threadIdx.x; i0 < items; i0 += 4 * step) {
-      V r[4];
-      int dsts[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        dsts[j] = -1;
-        if (i0 + j * step < items) {
-          dsts[j] = (VEC * col) * PC + c;
-          r[j] = __ldg(reinterpret_cast<const V*>(xrow + c * cstride + VEC * col));
-        }
-        col += d_col; c += d_c;
-        if (col >= nwi) { col -= nwi; ++c; }
-      }
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        if (dsts[j] >= 0) {
-          const uint16_t* e = reinterpret_cast<const uint16_t*>(&r[j]);
-#pragma unroll
-          for (int t = 0; t < VEC; ++t) rows_s[dsts[j] + t * PC] = e[t];
-        }
-      }
-    }
-  }
-  __syncthreads();
-  // phase 2: for every (ho, u) that holds the row, chunk j = (k - k_lo)*octs + oct
+  const int step = (int)blockDim.x;
+  // phase 1 counters: item -> (channel pair, group of VEC columns), columns fastest
+  typedef typename VecType<VEC>::type V;
+  const int nwi = nw / VEC;
+  const int cpairs = (C + 1) / 2;
+  const int items = cpairs * nwi;
+  const int d_c = step / nwi, d_col = step - d_c * nwi;
+  const int cp_first = (int)threadIdx.x / nwi, col_first = (int)threadIdx.x - cp_first * nwi;
+  const int64_t cstride = (int64_t)H * W;
+  // phase 2 counters: chunk j = (k - k_lo)*octs + oct
   const int octs = Cp / 8;
   const int chunks = (k_hi - k_lo) * octs;
-  const int step = (int)blockDim.x;
   const int d_k = step / octs, d_o = step - d_k * octs;
-  for (int ho = ho_lo; ho <= ho_hi; ++ho) {
-    const int u = hp - ho * s;
-    // chunk (k, oct) of strip (n, ho): ((k*Kh + u)*Cp + 8*oct) halves into the strip
-    uint16_t* strip = win + ((n * Ho + ho) * (int64_t)Wp) * Kh * Cp + (int64_t)u * Cp;
-    int k = k_lo + (int)threadIdx.x / octs, oct = (int)threadIdx.x % octs;
-    for (int j = threadIdx.x; j < chunks; j += step) {
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      const int w = k - p;
-      if (row_ok && w >= w0 && w < w0 + nw) {
-        const uint32_t* src = reinterpret_cast<const uint32_t*>(rows_s + (w - w0) * PC + 8 * oct);
-        v = make_uint4(src[0], src[1], src[2], src[3]);
+  const int k_first = k_lo + (int)threadIdx.x / octs, oct_first = (int)threadIdx.x % octs;
+
+  const int hp_end = (rg + 1) * R < H + 2 * p ? (rg + 1) * R : H + 2 * p;
+  for (int hp = rg * R; hp < hp_end; ++hp) {              // row of the padded input
+    const int h = hp - p;
+    const bool row_ok = h >= 0 && h < H;
+    // the strips that hold this row: ho*s + u = hp with 0 <= u < Kh
+    const int ho_hi = hp / s < Ho - 1 ? hp / s : Ho - 1;
+    const int ho_lo = hp - Kh + 1 > 0 ? (hp - Kh + 1 + s - 1) / s : 0;
+    if (ho_lo > ho_hi) continue;                          // a row no window reaches (the same for every thread)
+    __syncthreads();                                      // the row before has been written out
+    if (row_ok) {
+      if (Cp > C) {                                       // the zero channels C .. Cp-1 (an odd C's last pair store
+                                                          // writes a zero to channel C as well: same value)
+        const int extra = Cp - C;
+        for (int i = threadIdx.x; i < nw * extra; i += step) {
+          const int r = i / extra, e = i - r * extra;
+          rows_s[r * PC + C + e] = 0;
+        }
       }
-      *reinterpret_cast<uint4*>(strip + (int64_t)k * Kh * Cp + 8 * oct) = v;
-      oct += d_o; k += d_k;
-      if (oct >= octs) { oct -= octs; ++k; }
+      // phase 1 (W, w0 and nw are multiples of VEC): two VEC*2-byte loads (the second channel's only
+      // when it exists), VEC transposing 4-byte stores of a channel pair each; two items in flight
+      int cp = cp_first, col = col_first;
+      const uint16_t* xrow = x + ((n * C) * H + h) * (int64_t)W + w0;    // channel c: + c*H*W
+      for (int i0 = threadIdx.x; i0 < items; i0 += 2 * step) {
+        V r0[2], r1[2];
+        int dsts[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          dsts[j] = -1;
+          if (i0 + j * step < items) {
+            const int c = 2 * cp;
+            dsts[j] = (VEC * col) * PC + c;
+            const uint16_t* src = xrow + c * cstride + VEC * col;
+            r0[j] = __ldg(reinterpret_cast<const V*>(src));
+            if (c + 1 < C) r1[j] = __ldg(reinterpret_cast<const V*>(src + cstride));
+            else memset(&r1[j], 0, sizeof(V));
+          }
+          col += d_col; cp += d_c;
+          if (col >= nwi) { col -= nwi; ++cp; }
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          if (dsts[j] >= 0) {
+            const uint16_t* e0 = reinterpret_cast<const uint16_t*>(&r0[j]);
+            const uint16_t* e1 = reinterpret_cast<const uint16_t*>(&r1[j]);
+#pragma unroll
+            for (int t = 0; t < VEC; ++t)
+              *reinterpret_cast<uint32_t*>(rows_s + dsts[j] + t * PC) = (uint32_t)e0[t] | ((uint32_t)e1[t] << 16);
+          }
+        }
+      }
+    }
+    __syncthreads();
+    // phase 2: for every (ho, u) that holds the row
+    for (int ho = ho_lo; ho <= ho_hi; ++ho) {
+      const int u = hp - ho * s;
+      // chunk (k, oct) of strip (n, ho): ((k*Kh + u)*Cp + 8*oct) halves into the strip
+      uint16_t* strip = win + ((n * Ho + ho) * (int64_t)Wp) * Kh * Cp + (int64_t)u * Cp;
+      int k = k_first, oct = oct_first;
+      for (int j = threadIdx.x; j < chunks; j += step) {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        const int w = k - p;
+        if (row_ok && w >= w0 && w < w0 + nw) {
+          const uint32_t* src = reinterpret_cast<const uint32_t*>(rows_s + (w - w0) * PC + 8 * oct);
+          v = make_uint4(src[0], src[1], src[2], src[3]);
+        }
+        *reinterpret_cast<uint4*>(strip + (int64_t)k * Kh * Cp + 8 * oct) = v;
+        oct += d_o; k += d_k;
+        if (oct >= octs) { oct -= octs; ++k; }
+      }
     }
   }
 }
@@ -1544,12 +1563,19 @@ cudaError_t launch_transform_nhwc(const uint16_t* x, int x_is_nhwc, uint16_t* wi
   // columns per load: rows must start on a multiple of it (W a multiple) and so must the chunks
   const int vec = g.W % 8 == 0 ? 8 : (g.W % 4 == 0 ? 4 : (g.W % 2 == 0 ? 2 : 1));
   const int kchunks = (g.W + kc - 1) / kc;
-  const int64_t blocks = (int64_t)g.N * (g.H + 2 * g.p) * kchunks;
+  // rows per block: two (a block's set-up then serves both) when there are many more row blocks than
+  // the GPU holds at once and a row is written to few places; measured 4-10 % faster on 3x3 and 5x5
+  // layers with 56x56 and 24x24 images, slower from three rows on and for tall kernels
+  const int rows_total = g.H + 2 * g.p;
+  int R = ((int64_t)g.N * rows_total * kchunks >= 148 * 16 && g.Kh <= 5) ? 2 : 1;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_TRANSFORM_ROWS")) { const int r = atoi(v); if (r >= 1 && r <= 64) R = r; }   // testing aid
+  const int rgroups = (rows_total + R - 1) / R;
+  const int64_t blocks = (int64_t)g.N * rgroups * kchunks;
   if (blocks >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
   const size_t smem = (size_t)(per_col * kc);
 #define IM2WIN_LAUNCH_T(V)                                                                                          \
   transform_nhwc_from_nchw_kernel<V><<<(unsigned)blocks, 256, smem, stream>>>(x, window, g.C, plan.Cp, g.H, g.W, g.Ho, \
-                                                                            g.Wp, g.Kh, g.s, g.p, kc, kchunks)
+                                                                            g.Wp, g.Kh, g.s, g.p, kc, kchunks, R, rgroups)
   if (vec == 8) IM2WIN_LAUNCH_T(8);
   else if (vec == 4) IM2WIN_LAUNCH_T(4);
   else if (vec == 2) IM2WIN_LAUNCH_T(2);

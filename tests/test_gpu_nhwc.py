@@ -42,12 +42,15 @@ SMALL = [
 
 
 @pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
-@pytest.mark.parametrize("layout,variant", [("nchw", "default"), ("nchw", "rows"), ("nhwc", "default")])
+@pytest.mark.parametrize("layout,variant", [("nchw", "default"), ("nchw", "rows"), ("nchw", "rows3"), ("nhwc", "default")])
 def test_transform_nhwc_bit_exact(layer, layout, variant, monkeypatch):
     """From either input layout; from NCHW through the kernel the library picks (one block per strip
-    for up to 8 channels, else one block per input row) and through the per-row kernel forced."""
+    for up to 8 channels, else blocks of input rows) and through the per-row kernel forced, with
+    one and with three rows per block."""
     if variant != "default":
-        monkeypatch.setenv("IM2WIN_NHWC_TRANSFORM", variant)
+        monkeypatch.setenv("IM2WIN_NHWC_TRANSFORM", "rows")
+    if variant == "rows3":
+        monkeypatch.setenv("IM2WIN_NHWC_TRANSFORM_ROWS", "3")
     dims = layer.dims()
     x, _ = workloads.make_inputs(layer)
     raw = x.half().view(torch.int16)
