@@ -45,6 +45,19 @@ __device__ __forceinline__ float2 unpack2(unsigned long long v) {
   return r;
 }
 
+// Position p -> (image n, offset r inside the image's Ho*Wo outputs).  A 64-bit division costs about a
+// hundred instructions; with fewer than 2^31 positions (every layer but the very largest) a 32-bit one does.
+__device__ __forceinline__ void split_position(int64_t p, const ConvF32Params& q, int64_t& n, int& r) {
+  if (q.P < ((int64_t)1 << 31)) {
+    const uint32_t nq = (uint32_t)p / (uint32_t)q.HoWo;
+    n = nq;
+    r = (int)((uint32_t)p - nq * (uint32_t)q.HoWo);
+  } else {
+    n = p / q.HoWo;
+    r = (int)(p - n * q.HoWo);
+  }
+}
+
 template <int BM, int BN>
 __global__ void __launch_bounds__((BM / 8) * (BN / 8), ((BM / 8) * (BN / 8) == 256 ? 2 : 3))
 conv_f32_kernel(ConvF32Params q) {
@@ -71,8 +84,9 @@ conv_f32_kernel(ConvF32Params q) {
   const bool lvalid = lp < q.P;
   const float* abase = q.win;
   if (lvalid) {
-    const int64_t n = lp / q.HoWo;
-    const int r = (int)(lp - n * q.HoWo);
+    int64_t n;
+    int r;
+    split_position(lp, q, n, r);
     const int ho = r / q.Wo;
     const int wo = r - ho * q.Wo;
     abase += n * q.img_stride + ho * q.strip + (int64_t)wo * q.sKh;
@@ -172,8 +186,17 @@ conv_f32_kernel(ConvF32Params q) {
   for (int hm = 0; hm < 2; ++hm) {
     const int64_t p = m0 + hm * (BM / 2) + tm * 4;
     if (p >= q.P) continue;
-    const int64_t n = p / q.HoWo;
-    const int r = (int)(p - n * q.HoWo);
+    int64_t n;
+    int r;
+    split_position(p, q, n, r);
+    // (image, offset) of the four positions: the offset advances by one and wraps into the next image
+    int64_t nn[4];
+    int rr[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      nn[i] = n; rr[i] = r + i;
+      while (rr[i] >= q.HoWo) { rr[i] -= q.HoWo; ++nn[i]; }
+    }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int co = n0 + (j / 4) * (BN / 2) + tn * 4 + (j % 4);
@@ -184,11 +207,8 @@ conv_f32_kernel(ConvF32Params q) {
       } else {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int64_t pi = p + i;
-          if (pi >= q.P) break;
-          const int64_t ni = pi / q.HoWo;
-          const int ri = (int)(pi - ni * q.HoWo);
-          q.y[(ni * q.Co + co) * q.HoWo + ri] = acc[hm * 4 + i][j];
+          if (p + i >= q.P) break;
+          q.y[(nn[i] * q.Co + co) * q.HoWo + rr[i]] = acc[hm * 4 + i][j];
         }
       }
     }
