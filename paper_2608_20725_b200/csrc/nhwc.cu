@@ -478,6 +478,7 @@ struct ShiftViewParams {
   int32_t ksplit, kb_per_split;
   int32_t ntn, nwork;
   int32_t bu_forced;         // testing aid: bu was given, do not choose it
+  int32_t dual;              // 1: two MMA-issuing warps, each with half of the activation ring (resident filter only)
 };
 
 // All MMAs of one full k2-block whose KW kernel columns sit in one filter stage, unrolled for a
@@ -559,19 +560,24 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       const bool leader = elect_one();
       const int ncls = q.s < q.Kw ? q.s : q.Kw;   // column classes some kernel column reads
       wait_for_previous_kernel();
-      int st = 0;
-      uint32_t ph = 0;
+      // with two issuing warps the ring is two rings of half the stages: even items fill one, odd items the other
+      const int nst = q.dual ? q.sa / 2 : q.sa;
+      int st2[2] = {0, 0};
+      uint32_t ph2[2] = {0u, 0u};
+      uint32_t it = 0;
       bool ok = true;
       TIMER_DECL;
-      for (int w = w_first; w < q.nwork && ok; w += w_step) {
+      for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
         const int mt = w / per_mt, rem = w - mt * per_mt;
         const int ks = rem % q.ksplit;
         const int q0 = (PAIR ? 2 * mt + (int)rank : mt) * TILE_M;
         const int kb0 = ks * q.kb_per_split;
         const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
+        const int r = q.dual ? (int)(it & 1u) : 0;
         for (int kb = kb0; kb < kb1; ++kb) {
+          const int st = r * nst + st2[r];
           if (lane == 0) TIMER_LAP(0);                   // activation copies: issuing
-          ok = mbar_wait(a_empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
+          ok = mbar_wait(a_empty0 + 8 * st, ph2[r] ^ 1u, &abort_flag, q.status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           if (lane == 0) TIMER_LAP(1);                   // activation copies: wait for a free stage
@@ -586,7 +592,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
             }
           }
           __syncwarp();
-          if (++st == q.sa) { st = 0; ph ^= 1u; }
+          if (++st2[r] == nst) { st2[r] = 0; ph2[r] ^= 1u; }
         }
       }
       if (lane == 0 && blockIdx.x == 0) { TIMER_LAP(0); TIMER_FLUSH(); }
@@ -628,15 +634,25 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
         if (q.resident) break;                   // every stage now holds its units for good
       }
     }
-  } else if (warp == WARP_MMA && rank == 0) {
+  }
+  if ((warp == WARP_MMA || (warp == WARP_BLOAD && q.dual)) && rank == 0) {
     // ---------------- MMA issuer ------------------------------------------------------
     // The whole warp walks the loop (waits are taken by every lane), one elected lane issues the
     // MMAs and commits: measured faster than a lone lane, whose satisfied waits cost more.
+    // With a resident filter the filter-copy warp is idle after the first item and becomes a second
+    // issuer (q.dual): issuer 0 takes the even items, issuer 1 the odd ones, each with its own half of
+    // the activation ring and its own accumulators (the accumulator ring has an even length), so the
+    // two instruction streams are independent: while one issuer waits for its stages or an accumulator
+    // the other keeps the tensor pipe fed (short items of 64-channel layers).
     constexpr uint32_t idesc = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN);
     {
       const bool leader = elect_one();
+      const int mid = warp == WARP_MMA ? 0 : 1;
+      const int nroles = q.dual ? 2 : 1;
+      const int nst = q.dual ? q.sa / 2 : q.sa;      // activation stages of this issuer
+      const int abase = mid * nst;
       int sta = 0, stb = 0;
-      uint32_t pha = 0, phb = 0, it = 0;
+      uint32_t pha = 0, phb = 0, it = (uint32_t)mid;
       bool ok = true;
       const uint32_t a_lo0 = smem_desc_lo(a_ring), b_lo0 = smem_desc_lo(b_ring);
       const uint32_t subt16 = q.subt_bytes >> 4, astage16 = q.a_stage_bytes >> 4, bstage16 = b_stage_bytes >> 4;
@@ -644,12 +660,13 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
 #pragma unroll
       for (int v = 0; v < 7; ++v) tapr[v] = v < q.Kw ? tap16[v] : 0u;
       TIMER_DECL;
-      for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
+      for (int w = w_first + mid * w_step; w < q.nwork && ok; w += nroles * w_step, it += (uint32_t)nroles) {
         const int rem = w % per_mt;
         const int ks = rem % q.ksplit;
         const int kb0 = ks * q.kb_per_split;
         const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
         const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
+        const bool first_item = it < (uint32_t)nroles;   // this issuer's first item: a resident filter is still arriving
         if (lane == 0) TIMER_LAP(2);                     // MMA warp: issue and bookkeeping
         ok = mbar_wait(acc_empty0 + 8 * buf, aph ^ 1u, &abort_flag, q.status);   // drained by the epilogue
         ok = __all_sync(0xffffffffu, ok);
@@ -663,13 +680,13 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
           // one filter stage per k2-block (all its kernel columns): two waits and two commits per block
           for (int kb = kb0; kb < kb1; ++kb) {
             if (lane == 0) TIMER_LAP(2);
-            ok = mbar_wait(a_full0 + 8 * sta, pha, &abort_flag, q.status);
-            if (ok && !(q.resident && it > 0)) ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
+            ok = mbar_wait(a_full0 + 8 * (abase + sta), pha, &abort_flag, q.status);
+            if (ok && !(q.resident && !first_item)) ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             if (lane == 0) TIMER_LAP(4);               // MMA warp: wait for the stages
             if (leader) {
-              const uint32_t a_stage = a_lo0 + (uint32_t)sta * astage16;
+              const uint32_t a_stage = a_lo0 + (uint32_t)(abase + sta) * astage16;
               uint32_t b_lo = b_lo0 + (uint32_t)stb * bstage16;
               if (kb != q.nkb2 - 1 || q.nks_last == KB / 16) {
                 if (q.Kw == 3) issue_k2_block<3, PAIR>(acc, a_stage, b_lo, tapr, B_BYTES >> 4, idesc, accumulate);
@@ -698,15 +715,15 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
                   b_lo += B_BYTES >> 4;
                 }
               }
-              if (PAIR) umma_commit_pair(a_empty0 + 8 * sta);
-              else umma_commit(a_empty0 + 8 * sta);
+              if (PAIR) umma_commit_pair(a_empty0 + 8 * (abase + sta));
+              else umma_commit(a_empty0 + 8 * (abase + sta));
               if (!q.resident) {
                 if (PAIR) umma_commit_pair(b_empty0 + 8 * stb);
                 else umma_commit(b_empty0 + 8 * stb);
               }
             }
             __syncwarp();
-            if (++sta == q.sa) { sta = 0; pha ^= 1u; }
+            if (++sta == nst) { sta = 0; pha ^= 1u; }
             if (++stb == q.sb) { stb = 0; phb ^= 1u; }
           }
         } else {
@@ -716,7 +733,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
         int nks = KB / 16;
         for (int left = (kb1 - kb0) * q.Kw; left > 0 && ok; left -= q.bu) {
           const int nu = left < q.bu ? left : q.bu;
-          if (!(q.resident && it > 0)) {         // a resident filter is complete after the first item
+          if (!(q.resident && !first_item)) {    // a resident filter is complete after the first item
             if (lane == 0) TIMER_LAP(2);
             ok = mbar_wait(b_full0 + 8 * stb, phb, &abort_flag, q.status);
             ok = __all_sync(0xffffffffu, ok);
@@ -770,9 +787,10 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
         }
         __syncwarp();
       }
-      if (lane == 0 && blockIdx.x == 0) { TIMER_LAP(2); TIMER_FLUSH(); }
+      if (lane == 0 && blockIdx.x == 0 && mid == 0) { TIMER_LAP(2); TIMER_FLUSH(); }
     }
-  } else if (warp >= WARP_EPI0 && warp < WARP_EPI0 + EPI_WARPS) {
+  }
+  if (warp >= WARP_EPI0 && warp < WARP_EPI0 + EPI_WARPS) {
     // ---------------- epilogue ----------------------------------------------------------
     const int lq = warp & 3;
     const EpiParams& e = q.e;
@@ -1364,6 +1382,11 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
     if (q.sb < 2) { q.sa = 2; q.sb = (int)((budget - 2 * (int64_t)sp.a_stage_bytes) / b_stage); }
     if (q.sb < 2) return report(cudaErrorInvalidValue, "rings do not fit (shifted view)");
   }
+  // two MMA issuers (see the kernel): a resident filter held as whole k2-blocks, and for each issuer
+  // activation stages for a whole item (measured: 2-5 % faster then, cfg3 148 -> 142 us, a 3x3 layer
+  // with 56x56 images and 64 channels 90 -> 86; with half-item rings a 128-channel layer lost 27 %)
+  q.dual = (q.resident && q.bu == q.Kw && q.sa / 2 >= sp.nkb2 && q.nwork >= 2) ? 1 : 0;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_DUAL")) q.dual = (q.dual && v[0] != '0') ? 1 : 0;
   const int smem_bytes = q.sa * (int)sp.a_stage_bytes + q.sb * b_stage + 1024;
   const int slots = PAIR ? 74 : 148;
   static int cached_clusters[64] = {};

@@ -137,6 +137,24 @@ def test_conv_nhwc_epilogue_options(layer, out16, y_nhwc, bias, relu, monkeypatc
         assert np.array_equal(y, y.astype(np.float16).astype(np.float64))
 
 
+@pytest.mark.parametrize("layer", [L("many_items", 16, 16, 40, 40, 48, 3, 3, 1, 1, 60),
+                                   L("many_items_s2", 12, 8, 61, 62, 20, 5, 5, 2, 2, 61)], ids=lambda l: l.name)
+@pytest.mark.parametrize("dual", ["0", "1"])
+def test_conv_nhwc_two_mma_issuers(layer, dual, monkeypatch):
+    """More tile pairs than CTA pairs with a resident filter: every CTA works through several items,
+    with one MMA-issuing warp and with two (even and odd items on halves of the activation ring).
+    Exact on integer-valued inputs, within tolerance on the seeded ones."""
+    monkeypatch.setenv("IM2WIN_NHWC_KERNEL", "shift")
+    monkeypatch.setenv("IM2WIN_NHWC_DUAL", dual)
+    dims = layer.dims()
+    x, f = workloads.make_small_integer_inputs(layer)
+    yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+    assert np.array_equal(gpu_conv_nhwc(x, f, dims), yr)
+    x, f = workloads.make_inputs(layer)
+    y_pre, _, a = _reference(x, f, dims)
+    check_conv(gpu_conv_nhwc(x, f, dims), y_pre, a, "f16", layer.name)
+
+
 def test_conv_nhwc_exact_with_integer_bias_relu_and_half_store():
     """Small integers all the way: bias, ReLU and the binary16 store must reproduce the oracle exactly."""
     layer = SMALL[2]
