@@ -479,7 +479,16 @@ struct ShiftViewParams {
   int32_t ntn, nwork;
   int32_t bu_forced;         // testing aid: bu was given, do not choose it
   int32_t dual;              // 1: two MMA-issuing warps, each with half of the activation ring (resident filter only)
+  int32_t n_main;            // work items below this index are whole tiles; each whole tile above it is handed out as
+  int32_t tail_log2;         // 2^tail_log2 items of BN >> tail_log2 channels (fills the last, short round of tiles)
 };
+
+// Work item w of the shifted-view kernel -> whole item index and which part of its channels
+// (-1: all of them).
+__device__ __forceinline__ void decode_shift_item(const ShiftViewParams& q, int w, int* whole, int* part) {
+  if (w < q.n_main) { *whole = w; *part = -1; }
+  else { const int t = w - q.n_main; *whole = q.n_main + (t >> q.tail_log2); *part = t & ((1 << q.tail_log2) - 1); }
+}
 
 // All MMAs of one full k2-block whose KW kernel columns sit in one filter stage, unrolled for a
 // compile-time kernel width (view offsets from registers, filter tiles B16 sixteen-byte units apart):
@@ -500,7 +509,8 @@ __device__ __forceinline__ void issue_k2_block(uint32_t acc, uint32_t a_stage, u
 }
 
 template <int BN, bool PAIR>
-__device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const CUtensorMap& bmap, const ShiftViewParams& q) {
+__device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const CUtensorMap& bmap, const CUtensorMap& bmap_h,
+                                                const CUtensorMap& bmap_q, const ShiftViewParams& q) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;
   constexpr int NACC = acc_buffers(BN);
   constexpr uint32_t B_BYTES = (uint32_t)B_ROWS * KB * 2;
@@ -568,7 +578,9 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       bool ok = true;
       TIMER_DECL;
       for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
-        const int mt = w / per_mt, rem = w - mt * per_mt;
+        int whole, part;
+        decode_shift_item(q, w, &whole, &part);
+        const int mt = whole / per_mt, rem = whole - mt * per_mt;
         const int ks = rem % q.ksplit;
         const int q0 = (PAIR ? 2 * mt + (int)rank : mt) * TILE_M;
         const int kb0 = ks * q.kb_per_split;
@@ -606,9 +618,15 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       uint32_t ph = 0;
       bool ok = true;
       for (int w = w_first; w < q.nwork && ok; w += w_step) {
-        const int rem = w % per_mt;
+        int whole, part;
+        decode_shift_item(q, w, &whole, &part);
+        const int rem = whole % per_mt;
         const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
-        const int brow = nt * BN + (int)rank * B_ROWS;
+        // filter rows of this CTA: its share of the tile's channels, or of one part of them
+        const int brow = part < 0 ? nt * BN + (int)rank * B_ROWS
+                                  : nt * BN + part * (BN >> q.tail_log2) + (int)rank * (B_ROWS >> q.tail_log2);
+        const uint32_t unit_bytes = part < 0 ? B_BYTES : B_BYTES >> q.tail_log2;
+        const CUtensorMap* bm = part < 0 ? &bmap : (q.tail_log2 == 1 ? &bmap_h : &bmap_q);
         const int kb0 = ks * q.kb_per_split;
         const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
         int kb = kb0, v = 0;
@@ -620,11 +638,11 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
           const uint32_t dst = b_ring + (uint32_t)st * b_stage_bytes;
           const uint32_t bar = b_full_dst + 8 * st;
           if (leader && (!PAIR || rank == 0))
-            mbar_arrive_expect_tx(b_full0 + 8 * st, (PAIR ? 2u : 1u) * (uint32_t)nu * B_BYTES);
+            mbar_arrive_expect_tx(b_full0 + 8 * st, (PAIR ? 2u : 1u) * (uint32_t)nu * unit_bytes);
           for (int j = 0; j < nu; ++j) {
             if (leader) {
-              if (PAIR) tma_load_3d_pair(dst + (uint32_t)j * B_BYTES, &bmap, kb * KB, v, brow, bar);
-              else tma_load_3d(dst + (uint32_t)j * B_BYTES, &bmap, kb * KB, v, brow, bar);
+              if (PAIR) tma_load_3d_pair(dst + (uint32_t)j * B_BYTES, bm, kb * KB, v, brow, bar);
+              else tma_load_3d(dst + (uint32_t)j * B_BYTES, bm, kb * KB, v, brow, bar);
             }
             if (++v == q.Kw) { v = 0; ++kb; }
           }
@@ -644,7 +662,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
     // the activation ring and its own accumulators (the accumulator ring has an even length), so the
     // two instruction streams are independent: while one issuer waits for its stages or an accumulator
     // the other keeps the tensor pipe fed (short items of 64-channel layers).
-    constexpr uint32_t idesc = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN);
+    constexpr uint32_t idesc_whole = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, BN);
+    const uint32_t idesc_part = instr_desc_f16(PAIR ? 2 * TILE_M : TILE_M, 0) | ((uint32_t)((BN >> q.tail_log2) >> 3) << 17);
     {
       const bool leader = elect_one();
       const int mid = warp == WARP_MMA ? 0 : 1;
@@ -661,7 +680,10 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       for (int v = 0; v < 7; ++v) tapr[v] = v < q.Kw ? tap16[v] : 0u;
       TIMER_DECL;
       for (int w = w_first + mid * w_step; w < q.nwork && ok; w += nroles * w_step, it += (uint32_t)nroles) {
-        const int rem = w % per_mt;
+        int whole, part;
+        decode_shift_item(q, w, &whole, &part);
+        const uint32_t idesc = part < 0 ? idesc_whole : idesc_part;
+        const int rem = whole % per_mt;
         const int ks = rem % q.ksplit;
         const int kb0 = ks * q.kb_per_split;
         const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
@@ -801,9 +823,12 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
     TIMER_DECL;
     for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
       const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
-      const int mt = w / per_mt, rem = w - mt * per_mt;
+      int whole, part;
+      decode_shift_item(q, w, &whole, &part);
+      const int mt = whole / per_mt, rem = whole - mt * per_mt;
       const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
-      const int n0 = nt * BN;
+      const int n0 = nt * BN + (part > 0 ? part * (BN >> q.tail_log2) : 0);
+      const int cols = part < 0 ? BN : BN >> q.tail_log2;
       // accumulator row = virtual position vq = strip*Wq + i; columns i >= Wo of a strip are no output
       const int64_t vq = (int64_t)(PAIR ? 2 * mt + (int)rank : mt) * TILE_M + lq * 32 + lane;
       bool valid = false;
@@ -827,7 +852,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(6);     // epilogue: wait for a finished accumulator
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
-      drain_accumulator(e, BN, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
+      drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
@@ -856,15 +881,18 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
 
 template <int BN>
 __global__ void __launch_bounds__(SHIFT_THREADS, 1)
-conv_f16_nhwc_shift_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap, ShiftViewParams q) {
-  conv_shift_body<BN, false>(amap, bmap, q);
+conv_f16_nhwc_shift_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
+                           const __grid_constant__ CUtensorMap bmap_h, const __grid_constant__ CUtensorMap bmap_q,
+                           ShiftViewParams q) {
+  conv_shift_body<BN, false>(amap, bmap, bmap_h, bmap_q, q);
 }
 
 template <int BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(SHIFT_THREADS, 1)
 conv_f16_nhwc_shift_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
+                                const __grid_constant__ CUtensorMap bmap_h, const __grid_constant__ CUtensorMap bmap_q,
                                 ShiftViewParams q) {
-  conv_shift_body<BN, true>(amap, bmap, q);
+  conv_shift_body<BN, true>(amap, bmap, bmap_h, bmap_q, q);
 }
 
 // Filter pack (paper Section "Im2win Convolution": height before width; here with the channel below
@@ -1344,7 +1372,8 @@ ShiftViewPlan plan_shift_view(const Geometry& g, const NhwcPlan& plan) {
 }
 
 template <int BN, bool PAIR>
-cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bmap, ShiftViewParams q, const NhwcPlan& plan,
+cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bmap, const CUtensorMap& bmap_h,
+                                 const CUtensorMap& bmap_q, ShiftViewParams q, const NhwcPlan& plan,
                                  const ShiftViewPlan& sp, cudaStream_t stream) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;
   constexpr int B_BYTES = B_ROWS * KB * 2;
@@ -1389,6 +1418,24 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
   if (const char* v = debug_getenv("IM2WIN_NHWC_DUAL")) q.dual = (q.dual && v[0] != '0') ? 1 : 0;
   const int smem_bytes = q.sa * (int)sp.a_stage_bytes + q.sb * b_stage + 1024;
   const int slots = PAIR ? 74 : 148;
+  // The last round of tiles: when it is short, each of its tiles is handed out as two or four items
+  // of half or a quarter of the channels (at least 64), so that the round takes a fraction of a
+  // tile's time.  Streamed filters only (a resident one is laid out for whole tiles), no K split.
+  q.n_main = q.nwork;
+  q.tail_log2 = 0;
+  bool tail_parts = true;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_TAIL")) tail_parts = v[0] != '0';
+  if (tail_parts && !q.resident && q.ksplit == 1 && BN >= 128) {
+    const int tail = q.nwork % slots;
+    int lg = 0;
+    if (tail > 0 && BN >= 256 && 4 * tail <= slots) lg = 2;
+    else if (tail > 0 && 2 * tail <= slots) lg = 1;
+    if (lg > 0) {
+      q.n_main = q.nwork - tail;
+      q.nwork += tail * ((1 << lg) - 1);
+      q.tail_log2 = lg;
+    }
+  }
   static int cached_clusters[64] = {};
   static int attr_bytes[64] = {};
   int dev = 0;
@@ -1424,7 +1471,7 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
     if (clusters > q.nwork) clusters = q.nwork;
     cfg.gridDim = dim3(2 * clusters, 1, 1);
     cfg.numAttrs = 2;
-    return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_pair_kernel<BN>, amap, bmap, q), "pair launch (shifted view)");
+    return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_pair_kernel<BN>, amap, bmap, bmap_h, bmap_q, q), "pair launch (shifted view)");
   }
   if (attr_bytes[dev] < smem_bytes) {
     cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
@@ -1436,7 +1483,7 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cfg.gridDim = dim3((unsigned)(slots < q.nwork ? slots : q.nwork), 1, 1);
-  return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_kernel<BN>, amap, bmap, q), "launch (shifted view)");
+  return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_kernel<BN>, amap, bmap, bmap_h, bmap_q, q), "launch (shifted view)");
 }
 
 cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* y, uint32_t* status, const Geometry& g,
@@ -1445,7 +1492,7 @@ cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* 
   // Activation operand: (k2, column class t, virtual position q): column k = q*s + t of the flat
   // sequence of all strips' columns; filter: (k2, kernel column v, output channel).  Out-of-range
   // coordinates read as zeros.
-  CUtensorMap amap, bmap;
+  CUtensorMap amap, bmap, bmap_h, bmap_q;
   {
     const cuuint64_t dims[3] = {(cuuint64_t)sp.K2, (cuuint64_t)g.s, (cuuint64_t)sp.VQ};
     const cuuint64_t strides[2] = {(cuuint64_t)sp.K2 * 2, (cuuint64_t)g.s * sp.K2 * 2};
@@ -1457,14 +1504,16 @@ cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* 
     if (cr != CUDA_SUCCESS) return report(cudaErrorInvalidValue, "activation tensor map (shifted view)");
   }
   const int b_rows = plan.pair ? plan.bn / 2 : plan.bn;
-  {
+  // the filter with boxes of a CTA's whole share of a tile's channels, of half and of a quarter of it
+  // (the last two for the items of a short last round)
+  for (int lg = 0; lg < 3; ++lg) {
     const cuuint64_t dims[3] = {(cuuint64_t)sp.K2, (cuuint64_t)g.Kw, (cuuint64_t)g.Co};
     const cuuint64_t strides[2] = {(cuuint64_t)sp.K2 * 2, (cuuint64_t)g.Kw * sp.K2 * 2};
-    const cuuint32_t box[3] = {(cuuint32_t)KB, 1, (cuuint32_t)b_rows};
+    const cuuint32_t box[3] = {(cuuint32_t)KB, 1, (cuuint32_t)(b_rows >> lg)};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult cr = encode(&bmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<uint16_t*>(fp), dims, strides, box, estr,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult cr = encode(lg == 0 ? &bmap : (lg == 1 ? &bmap_h : &bmap_q), CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
+                         const_cast<uint16_t*>(fp), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) return report(cudaErrorInvalidValue, "filter tensor map (shifted view)");
   }
   ShiftViewParams q{};
@@ -1480,13 +1529,13 @@ cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* 
   q.ntn = plan.ntn;
   if (const char* v = debug_getenv("IM2WIN_NHWC_BU")) { const int bu = atoi(v); if (bu >= 1 && bu <= 8) { q.bu = bu; q.bu_forced = 1; } }
   if (plan.pair) {
-    if (plan.bn == 256) return launch_shift_variant<256, true>(amap, bmap, q, plan, sp, stream);
-    if (plan.bn == 128) return launch_shift_variant<128, true>(amap, bmap, q, plan, sp, stream);
-    return launch_shift_variant<64, true>(amap, bmap, q, plan, sp, stream);
+    if (plan.bn == 256) return launch_shift_variant<256, true>(amap, bmap, bmap_h, bmap_q, q, plan, sp, stream);
+    if (plan.bn == 128) return launch_shift_variant<128, true>(amap, bmap, bmap_h, bmap_q, q, plan, sp, stream);
+    return launch_shift_variant<64, true>(amap, bmap, bmap_h, bmap_q, q, plan, sp, stream);
   }
-  if (plan.bn == 64) return launch_shift_variant<64, false>(amap, bmap, q, plan, sp, stream);
-  if (plan.bn == 128) return launch_shift_variant<128, false>(amap, bmap, q, plan, sp, stream);
-  return launch_shift_variant<256, false>(amap, bmap, q, plan, sp, stream);
+  if (plan.bn == 64) return launch_shift_variant<64, false>(amap, bmap, bmap_h, bmap_q, q, plan, sp, stream);
+  if (plan.bn == 128) return launch_shift_variant<128, false>(amap, bmap, bmap_h, bmap_q, q, plan, sp, stream);
+  return launch_shift_variant<256, false>(amap, bmap, bmap_h, bmap_q, q, plan, sp, stream);
 }
 
 }  // namespace
@@ -1674,7 +1723,9 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
     const int64_t it_s = (plan.pair ? (tiles_s + 1) / 2 : tiles_s) * plan.ntn;
     const int64_t tail = it_o % slots;
     const double r_o = (double)(it_o / slots) + (tail == 0 ? 0.0 : (plan.bn >= 128 && 2 * tail <= slots ? 0.55 : 1.0));
-    const double r_s = (double)((it_s + slots - 1) / slots);
+    // (the shifted-view kernel hands a short last round out as quarter or half tiles when its filter is streamed)
+    const int64_t tail_s = it_s % slots;
+    const double r_s = (double)(it_s / slots) + (tail_s == 0 ? 0.0 : (plan.bn >= 256 && 4 * tail_s <= slots ? 0.4 : (plan.bn >= 128 && 2 * tail_s <= slots ? 0.55 : 1.0)));
     if (reuse ? r_o < 0.85 * r_s : r_o <= r_s) use_shift = false;
   }
   if (const char* v = debug_getenv("IM2WIN_NHWC_KERNEL")) {
