@@ -94,7 +94,8 @@ struct NhwcPlan {
   int64_t strip;           // Wp*Kh*Cp halves per (n, ho)
   int64_t window_elems;    // N*Ho*strip
   int64_t ntm;             // position tiles
-  size_t scratch_bytes;    // status block + packed filter
+  size_t flags_off;        // byte offset of the tail-tile flag words inside the scratch
+  size_t scratch_bytes;    // status block + packed filter + flag words
 };
 NhwcPlan plan_nhwc(const Geometry& g);
 

@@ -26,6 +26,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 
@@ -84,8 +86,8 @@ __device__ __forceinline__ void red_add_f32(float* p, float v) {
 // row's position; `base` is the element index of channel c0 at that position and `cs` the element
 // distance between channels (Ho*Wo for NCHW, 1 for NHWC).
 __device__ __forceinline__ void store_chunk(const EpiParams& q, int64_t base, int64_t cs, const uint32_t (&v)[32],
-                                            int cnt, bool vec_ok) {
-  if (q.atomic) {
+                                            int cnt, bool vec_ok, bool add = false) {
+  if (q.atomic || add) {
     float* p = reinterpret_cast<float*>(q.y) + base;
 #pragma unroll
     for (int j = 0; j < 32; ++j)
@@ -136,7 +138,7 @@ __device__ __forceinline__ void store_chunk(const EpiParams& q, int64_t base, in
 
 // Bias (first K part only), ReLU and store of 32 channels from c0 on of one accumulator row.
 __device__ __forceinline__ void finish_chunk(const EpiParams& e, uint32_t (&v)[32], int c0, int n0, bool first_part,
-                                             bool valid, int64_t base, int64_t cs, bool vec_ok) {
+                                             bool valid, int64_t base, int64_t cs, bool vec_ok, bool add = false) {
   const int cnt = e.Co - n0 - c0;                // channels left from c0 on
   if (cnt <= 0) return;
   if (e.bias != nullptr && first_part) {
@@ -162,7 +164,7 @@ __device__ __forceinline__ void finish_chunk(const EpiParams& e, uint32_t (&v)[3
 #pragma unroll
     for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(fmaxf(__uint_as_float(v[t]), 0.0f));
   }
-  if (valid) store_chunk(e, base + (int64_t)c0 * cs, cs, v, cnt < 32 ? cnt : 32, vec_ok);
+  if (valid) store_chunk(e, base + (int64_t)c0 * cs, cs, v, cnt < 32 ? cnt : 32, vec_ok, add);
 }
 
 // One epilogue warp's share of a finished accumulator: tensor-memory lane quadrant warp % 4, the
@@ -171,7 +173,8 @@ __device__ __forceinline__ void finish_chunk(const EpiParams& e, uint32_t (&v)[3
 // ones are stored (two register sets, taken in turn).  `base` is the element index of the tile's first
 // channel at this lane's position, `cs` the element distance between channels.
 __device__ __forceinline__ void drain_accumulator(const EpiParams& e, int cols, int warp, int lane, uint32_t lane_base,
-                                                  bool valid, int64_t base, int64_t cs, int n0, bool first_part, bool vec_ok) {
+                                                  bool valid, int64_t base, int64_t cs, int n0, bool first_part, bool vec_ok,
+                                                  bool add = false) {
   const int CH = cols / 2;                       // a multiple of 32
   const int cbeg = ((warp - WARP_EPI0) >> 2) * CH;
   const int cend = cbeg + CH;
@@ -181,11 +184,11 @@ __device__ __forceinline__ void drain_accumulator(const EpiParams& e, int cols, 
   for (int c0 = cbeg; c0 < cend; c0 += 64) {
     tmem_ld_wait_for(va);
     if (c0 + 32 < cend) tmem_ld32_issue(lane_base + (uint32_t)(c0 + 32), vb);
-    finish_chunk(e, va, c0, n0, first_part, valid, base, cs, vec_ok);
+    finish_chunk(e, va, c0, n0, first_part, valid, base, cs, vec_ok, add);
     if (c0 + 32 >= cend) break;
     tmem_ld_wait_for(vb);
     if (c0 + 64 < cend) tmem_ld32_issue(lane_base + (uint32_t)(c0 + 64), va);
-    finish_chunk(e, vb, c0 + 32, n0, first_part, valid, base, cs, vec_ok);
+    finish_chunk(e, vb, c0 + 32, n0, first_part, valid, base, cs, vec_ok, add);
   }
 }
 
@@ -457,6 +460,7 @@ conv_f16_nhwc_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid
 // fits) stay as they were.  Needs s | Wp.  Of the s column classes only those some kernel column reads
 // (min(s, Kw)) are copied; a 1x1 layer is then a plain product over full 128-position tiles.
 constexpr int MAX_SA = 6, MAX_SB = 12;
+constexpr int kTailFlagBytes = 1024;           // 256 flag words: two per tile of a short last round (at most 37 of them)
 constexpr int MAX_KW = 64;                     // kernel widths the shifted-view kernel takes
 constexpr int WARP_BLOAD = 2 + EPI_WARPS;      // the filter-copy warp of this kernel
 constexpr int SHIFT_THREADS = (NUM_WARPS + 1) * 32;
@@ -481,7 +485,44 @@ struct ShiftViewParams {
   int32_t dual;              // 1: two MMA-issuing warps, each with half of the activation ring (resident filter only)
   int32_t n_main;            // work items below this index are whole tiles; each whole tile above it is handed out as
   int32_t tail_log2;         // 2^tail_log2 items of BN >> tail_log2 channels (fills the last, short round of tiles)
+  int32_t tail_k;            // 1: the tail items split the reduction instead (tail_kb k2-blocks each, all channels):
+  int32_t tail_kb;           //    part 0 stores, raises the tile's flag; the others wait for it and add atomically
+  uint32_t* flags;           // two words per tail tile (one per CTA of a pair), compared with `epoch`
+  uint32_t epoch;            // distinct per launch, so that flags need no clearing between launches
 };
+
+// k2-blocks [kb0, kb1) of an item: its K part (ks of q.ksplit), or for a tail part that splits the
+// reduction its tail_kb blocks.
+__device__ __forceinline__ void item_blocks(const ShiftViewParams& q, int ks, int part, int* kb0, int* kb1) {
+  const int per = (q.tail_k && part >= 0) ? q.tail_kb : q.kb_per_split;
+  const int first = ((q.tail_k && part >= 0) ? part : ks) * per;
+  *kb0 = first;
+  *kb1 = first + per < q.nkb2 ? first + per : q.nkb2;
+}
+
+// Bounded wait for a flag word to hold `value` (written with release semantics by another CTA).
+__device__ __noinline__ bool wait_flag(const uint32_t* flag, uint32_t value, volatile uint32_t* abort_flag, uint32_t* status) {
+  uint32_t limit = *reinterpret_cast<volatile uint32_t*>(status + 1);
+  if (limit == 0u) limit = SPIN_LIMIT;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t i = 0; i < limit; ++i) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v == value) return true;
+    if ((i & 255u) == 255u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > SPIN_TIME_NS) break;
+    }
+    __nanosleep(64);
+  }
+  *abort_flag = 1u;
+  atomicExch(status, 1u);
+  return false;
+}
+
+__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 
 // Work item w of the shifted-view kernel -> whole item index and which part of its channels
 // (-1: all of them).
@@ -583,8 +624,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
         const int mt = whole / per_mt, rem = whole - mt * per_mt;
         const int ks = rem % q.ksplit;
         const int q0 = (PAIR ? 2 * mt + (int)rank : mt) * TILE_M;
-        const int kb0 = ks * q.kb_per_split;
-        const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
+        int kb0, kb1;
+        item_blocks(q, ks, part, &kb0, &kb1);
         const int r = q.dual ? (int)(it & 1u) : 0;
         for (int kb = kb0; kb < kb1; ++kb) {
           const int st = r * nst + st2[r];
@@ -623,12 +664,13 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
         const int rem = whole % per_mt;
         const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
         // filter rows of this CTA: its share of the tile's channels, or of one part of them
-        const int brow = part < 0 ? nt * BN + (int)rank * B_ROWS
-                                  : nt * BN + part * (BN >> q.tail_log2) + (int)rank * (B_ROWS >> q.tail_log2);
-        const uint32_t unit_bytes = part < 0 ? B_BYTES : B_BYTES >> q.tail_log2;
-        const CUtensorMap* bm = part < 0 ? &bmap : (q.tail_log2 == 1 ? &bmap_h : &bmap_q);
-        const int kb0 = ks * q.kb_per_split;
-        const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
+        const bool npart = part >= 0 && !q.tail_k;       // a part of the channels (a K part keeps them all)
+        const int brow = !npart ? nt * BN + (int)rank * B_ROWS
+                                : nt * BN + part * (BN >> q.tail_log2) + (int)rank * (B_ROWS >> q.tail_log2);
+        const uint32_t unit_bytes = !npart ? B_BYTES : B_BYTES >> q.tail_log2;
+        const CUtensorMap* bm = !npart ? &bmap : (q.tail_log2 == 1 ? &bmap_h : &bmap_q);
+        int kb0, kb1;
+        item_blocks(q, ks, part, &kb0, &kb1);
         int kb = kb0, v = 0;
         for (int left = (kb1 - kb0) * q.Kw; left > 0 && ok; left -= q.bu) {
           const int nu = left < q.bu ? left : q.bu;             // units of this stage
@@ -682,11 +724,11 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       for (int w = w_first + mid * w_step; w < q.nwork && ok; w += nroles * w_step, it += (uint32_t)nroles) {
         int whole, part;
         decode_shift_item(q, w, &whole, &part);
-        const uint32_t idesc = part < 0 ? idesc_whole : idesc_part;
+        const uint32_t idesc = (part < 0 || q.tail_k) ? idesc_whole : idesc_part;
         const int rem = whole % per_mt;
         const int ks = rem % q.ksplit;
-        const int kb0 = ks * q.kb_per_split;
-        const int kb1 = kb0 + q.kb_per_split < q.nkb2 ? kb0 + q.kb_per_split : q.nkb2;
+        int kb0, kb1;
+        item_blocks(q, ks, part, &kb0, &kb1);
         const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
         const bool first_item = it < (uint32_t)nroles;   // this issuer's first item: a resident filter is still arriving
         if (lane == 0) TIMER_LAP(2);                     // MMA warp: issue and bookkeeping
@@ -827,8 +869,9 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       decode_shift_item(q, w, &whole, &part);
       const int mt = whole / per_mt, rem = whole - mt * per_mt;
       const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
-      const int n0 = nt * BN + (part > 0 ? part * (BN >> q.tail_log2) : 0);
-      const int cols = part < 0 ? BN : BN >> q.tail_log2;
+      const bool kpart = q.tail_k && part >= 0;        // a tail item that holds one K part of all channels
+      const int n0 = nt * BN + ((part > 0 && !kpart) ? part * (BN >> q.tail_log2) : 0);
+      const int cols = (part < 0 || kpart) ? BN : BN >> q.tail_log2;
       // accumulator row = virtual position vq = strip*Wq + i; columns i >= Wo of a strip are no output
       const int64_t vq = (int64_t)(PAIR ? 2 * mt + (int)rank : mt) * TILE_M + lq * 32 + lane;
       bool valid = false;
@@ -852,7 +895,21 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(6);     // epilogue: wait for a finished accumulator
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
-      drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
+      // K parts of a tail tile: part 0 stores (with the bias) and then raises this CTA's flag of the
+      // tile; the other parts wait for that flag and add their sums with red.global.add.f32
+      uint32_t* flag = q.flags + 2 * (whole - q.n_main) + (PAIR ? (int)rank : 0);
+      const bool adds = kpart && part > 0;
+      if (adds) {
+        if (lane == 0) ok = wait_flag(flag, q.epoch, &abort_flag, q.status);
+        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        __syncwarp();
+      }
+      if (ok) drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, kpart ? part == 0 : ks == 0, vec_ok, adds);
+      if (kpart && part == 0) {
+        __threadfence();
+        named_barrier_sync(1, EPI_WARPS * 32);          // all eight epilogue warps have stored
+        if (threadIdx.x == WARP_EPI0 * 32) asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(q.epoch) : "memory");
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
@@ -901,13 +958,16 @@ conv_f16_nhwc_shift_pair_kernel(const __grid_constant__ CUtensorMap amap, const 
 // (coalesced reads into shared memory) and leave as Kh*Kw runs of cb channels (coalesced writes).
 // Block (0, 0) also clears the status block.
 __global__ void __launch_bounds__(256)
-pack_f16_nhwc_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, uint32_t* status, int C, int Cp,
-                     int Co, int Kh, int Kw, int cb) {
+pack_f16_nhwc_kernel(const uint16_t* __restrict__ f, uint16_t* __restrict__ fp, uint32_t* status, uint32_t* flags,
+                     int C, int Cp, int Co, int Kh, int Kw, int cb) {
   extern __shared__ __align__(16) uint16_t pack_s[];   // [cb][T], after up to 8 halves of phase padding
   // the convolution that follows in the stream may be launched now: its set-up overlaps this kernel,
   // and every role of it that touches memory first waits for this grid to have completed
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
+  if (blockIdx.x == 0 && blockIdx.y == 0) {
+    if (threadIdx.x < kStatusBytes / 4) status[threadIdx.x] = 0u;
+    for (int i = threadIdx.x; i < kTailFlagBytes / 4; i += blockDim.x) flags[i] = 0u;
+  }
   const int T = Kh * Kw;
   const int64_t K = (int64_t)T * Cp;
   const int c0 = blockIdx.x * cb;
@@ -1417,7 +1477,37 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
   q.dual = (q.resident && q.bu == q.Kw && q.sa / 2 >= sp.nkb2 && q.nwork >= 2) ? 1 : 0;
   if (const char* v = debug_getenv("IM2WIN_NHWC_DUAL")) q.dual = (q.dual && v[0] != '0') ? 1 : 0;
   const int smem_bytes = q.sa * (int)sp.a_stage_bytes + q.sb * b_stage + 1024;
-  const int slots = PAIR ? 74 : 148;
+  static int cached_clusters[64] = {};
+  static int attr_bytes[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  // CTAs (pairs) that are resident together: the grid, and what "a round of tiles" means below.  The
+  // items of a split last round wait for one another, so every one of them must have a CTA of its own.
+  int slots = PAIR ? 74 : 148;
+  if (PAIR) {
+    if (attr_bytes[dev] < smem_bytes) {
+      cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
+      if (e != cudaSuccess) return report(e, "shared-memory opt-in (shifted view, pairs)");
+      attr_bytes[dev] = kSmemMax - 1024;
+    }
+    int clusters = cached_clusters[dev];
+    if (clusters == 0) {
+      cudaLaunchConfig_t probe = {};
+      cudaLaunchAttribute pattr[1];
+      pattr[0].id = cudaLaunchAttributeClusterDimension;
+      pattr[0].val.clusterDim.x = 2; pattr[0].val.clusterDim.y = 1; pattr[0].val.clusterDim.z = 1;
+      probe.blockDim = dim3(SHIFT_THREADS, 1, 1);
+      probe.gridDim = dim3(148, 1, 1);
+      probe.dynamicSmemBytes = (size_t)(kSmemMax - 1024);   // the worst case: one CTA per SM either way
+      probe.attrs = pattr;
+      probe.numAttrs = 1;
+      cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_nhwc_shift_pair_kernel<BN>, &probe);
+      if (e != cudaSuccess) return e;
+      if (clusters < 1) return cudaErrorInvalidValue;
+      cached_clusters[dev] = clusters;
+    }
+    if (clusters < slots) slots = clusters;
+  }
   // The last round of tiles: when it is short, each of its tiles is handed out as two or four items
   // of half or a quarter of the channels (at least 64), so that the round takes a fraction of a
   // tile's time.  Streamed filters only (a resident one is laid out for whole tiles), no K split.
@@ -1425,50 +1515,52 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
   q.tail_log2 = 0;
   bool tail_parts = true;
   if (const char* v = debug_getenv("IM2WIN_NHWC_TAIL")) tail_parts = v[0] != '0';
-  if (tail_parts && !q.resident && q.ksplit == 1 && BN >= 128) {
+  q.tail_k = 0;
+  q.tail_kb = 0;
+  if (tail_parts && !q.resident && q.ksplit == 1) {
     const int tail = q.nwork % slots;
+    // Preferred: parts of the reduction (every MMA stays as wide as the tile; the parts meet through
+    // the tile's flag and red.global.add.f32), up to eight per tile, each at least two k2-blocks long.
+    // Not under a ReLU or a rounding store (partial sums cannot pass them): then, or when K is short,
+    // parts of the channels.
+    // (and only for long items, 96 (k2-block, kernel column) units or more: measured, the wait for part 0
+    // and the atomics cost short items more than the narrower MMAs of channel parts do:
+    // 5x5 on 96 channels 121 against 115 us, 3x3 on 256 channels 71 against 61; 7x7 on 256: 265 against 300)
+    bool k_parts = !q.e.relu && !q.e.out16 && q.flags != nullptr && 2 * tail * (int)sizeof(uint32_t) <= kTailFlagBytes &&
+                   sp.nkb2 * q.Kw >= 96;
+    if (const char* v = debug_getenv("IM2WIN_NHWC_TAIL_K")) k_parts = k_parts && v[0] != '0';
     int lg = 0;
-    if (tail > 0 && BN >= 256 && 4 * tail <= slots) lg = 2;
-    else if (tail > 0 && 2 * tail <= slots) lg = 1;
+    if (tail > 0 && k_parts) {
+      for (int c = 3; c >= 1; --c)
+        if ((tail << c) <= slots && sp.nkb2 >= 2 * (1 << c)) { lg = c; break; }
+      if (lg > 0) {
+        q.tail_k = 1;
+        q.tail_kb = (sp.nkb2 + (1 << lg) - 1) >> lg;
+        if (((1 << lg) - 1) * q.tail_kb >= sp.nkb2) { q.tail_k = 0; lg = 0; }      // a part would be empty
+      }
+    }
+    if (lg == 0 && tail > 0 && BN >= 128) {
+      if (BN >= 256 && 4 * tail <= slots) lg = 2;
+      else if (2 * tail <= slots) lg = 1;
+    }
     if (lg > 0) {
       q.n_main = q.nwork - tail;
       q.nwork += tail * ((1 << lg) - 1);
       q.tail_log2 = lg;
     }
   }
-  static int cached_clusters[64] = {};
-  static int attr_bytes[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(SHIFT_THREADS, 1, 1);
   cfg.dynamicSmemBytes = (size_t)smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   if (PAIR) {
-    if (attr_bytes[dev] < smem_bytes) {
-      cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
-      if (e != cudaSuccess) return report(e, "shared-memory opt-in (shifted view, pairs)");
-      attr_bytes[dev] = kSmemMax - 1024;
-    }
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    int clusters = cached_clusters[dev];
-    if (clusters == 0) {
-      cudaLaunchConfig_t probe = cfg;
-      probe.gridDim = dim3(148, 1, 1);
-      probe.dynamicSmemBytes = (size_t)(kSmemMax - 1024);   // the worst case: one CTA per SM either way
-      probe.numAttrs = 1;
-      cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_nhwc_shift_pair_kernel<BN>, &probe);
-      if (e != cudaSuccess) return e;
-      if (clusters < 1) return cudaErrorInvalidValue;
-      cached_clusters[dev] = clusters;
-    }
-    if (clusters > slots) clusters = slots;
-    if (clusters > q.nwork) clusters = q.nwork;
+    const int clusters = slots < q.nwork ? slots : q.nwork;
     cfg.gridDim = dim3(2 * clusters, 1, 1);
     cfg.numAttrs = 2;
     return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_pair_kernel<BN>, amap, bmap, bmap_h, bmap_q, q), "pair launch (shifted view)");
@@ -1486,9 +1578,9 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
   return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_kernel<BN>, amap, bmap, bmap_h, bmap_q, q), "launch (shifted view)");
 }
 
-cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* y, uint32_t* status, const Geometry& g,
-                              const NhwcPlan& plan, const ShiftViewPlan& sp, const EpilogueArgs& epi, bool split,
-                              EncodeTiledFn encode, cudaStream_t stream) {
+cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* y, uint32_t* status, uint32_t* flags,
+                              const Geometry& g, const NhwcPlan& plan, const ShiftViewPlan& sp, const EpilogueArgs& epi,
+                              bool split, EncodeTiledFn encode, cudaStream_t stream) {
   // Activation operand: (k2, column class t, virtual position q): column k = q*s + t of the flat
   // sequence of all strips' columns; filter: (k2, kernel column v, output channel).  Out-of-range
   // coordinates read as zeros.
@@ -1527,6 +1619,13 @@ cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* 
   q.nkb2 = sp.nkb2; q.nks_last = sp.nks_last; q.bu = sp.bu;
   q.ksplit = split ? plan.ksplit : 1;
   q.ntn = plan.ntn;
+  {
+    static std::atomic<uint32_t> launches{0};
+    uint32_t e = ++launches;
+    if (e == 0) e = ++launches;                 // 0 is what cleared flags hold
+    q.epoch = e;
+    q.flags = flags;
+  }
   if (const char* v = debug_getenv("IM2WIN_NHWC_BU")) { const int bu = atoi(v); if (bu >= 1 && bu <= 8) { q.bu = bu; q.bu_forced = 1; } }
   if (plan.pair) {
     if (plan.bn == 256) return launch_shift_variant<256, true>(amap, bmap, bmap_h, bmap_q, q, plan, sp, stream);
@@ -1589,8 +1688,10 @@ NhwcPlan plan_nhwc(const Geometry& g) {
   }
   p.kb_per_split = (p.num_kb + p.ksplit - 1) / p.ksplit;
   if (tiles * p.ksplit >= lim) return p;
-  p.scratch_bytes = (size_t)kStatusBytes + (size_t)g.Co * p.K * 2;
-  p.scratch_bytes = (p.scratch_bytes + 255) / 256 * 256;
+  // status block, packed filter, then kTailFlagBytes of flag words (hand-off between the CTAs that share
+  // a tile of a short last round; cleared by the filter pack)
+  p.flags_off = ((size_t)kStatusBytes + (size_t)g.Co * p.K * 2 + 255) / 256 * 256;
+  p.scratch_bytes = p.flags_off + kTailFlagBytes;
   p.eligible = true;
   return p;
 }
@@ -1672,7 +1773,9 @@ cudaError_t launch_pack_f16_nhwc(const uint16_t* filter, void* scratch, const Ge
   }
   dim3 grid((unsigned)((plan.Cp + cb - 1) / cb), (unsigned)(g.Co < 32768 ? g.Co : 32768));
   pack_f16_nhwc_kernel<<<grid, 256, smem, stream>>>(filter, reinterpret_cast<uint16_t*>(base + kStatusBytes),
-                                                     reinterpret_cast<uint32_t*>(base), g.C, plan.Cp, g.Co, g.Kh, g.Kw, cb);
+                                                     reinterpret_cast<uint32_t*>(base),
+                                                     reinterpret_cast<uint32_t*>(base + plan.flags_off), g.C, plan.Cp, g.Co,
+                                                     g.Kh, g.Kw, cb);
   return cudaGetLastError();
 }
 
@@ -1694,12 +1797,8 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
     const int ks = atoi(v);
     if (ks >= 1 && ks <= plan.num_kb) plan.ksplit = ks;
   }
-  const bool split = plan.ksplit > 1 && !epi.relu && !epi.out16;   // partial sums cannot pass a ReLU or a rounding
+  bool split = plan.ksplit > 1 && !epi.relu && !epi.out16;   // partial sums cannot pass a ReLU or a rounding
   if (!split) plan.ksplit = 1;
-  if (split) {
-    cudaError_t e = cudaMemsetAsync(y, 0, (size_t)g.out_elems * 4, stream);
-    if (e != cudaSuccess) return e;
-  }
   // Which kernel.  The shifted-view kernel brings s/Kw of the activation bytes into the SM but computes
   // Wq rows per strip for Wo outputs, and it needs one filter stage per k2-block (all kernel columns)
   // to keep its MMA warp's barrier traffic low.  Measured: it wins where every column is reused by
@@ -1732,8 +1831,29 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
     if (strcmp(v, "shift") == 0) use_shift = sp.eligible;
     else if (strcmp(v, "overlap") == 0) use_shift = false;
   }
+  if (use_shift && split) {
+    // The shifted-view kernel can also split K for the tiles of a short last round only (parts meet
+    // through a flag, no cleared output, atomics on those tiles only).  Rounds, in tile times: whole
+    // rounds plus 1/P + 0.1 for a last round handed out as P parts, against the parts of a split of
+    // every tile plus 0.1 for clearing the output and the atomics.  (Measured: cfg5k5 135 against 148 us.)
+    const int slots = plan.pair ? 74 : 148;
+    const int64_t tiles_s = (sp.VQ + TILE_M - 1) / TILE_M;
+    const int64_t it_s = (plan.pair ? (tiles_s + 1) / 2 : tiles_s) * plan.ntn;
+    const int64_t tail_s = it_s % slots;
+    double frac = tail_s == 0 ? 0.0 : 1.0;
+    for (int c = 3; c >= 1 && tail_s > 0 && sp.nkb2 * g.Kw >= 96; --c)
+      if ((tail_s << c) <= slots && sp.nkb2 >= 2 * (1 << c)) { frac = 1.0 / (1 << c) + 0.1; break; }
+    const double r_tail = (double)(it_s / slots) + frac;
+    const double r_split = (double)((it_s * plan.ksplit + slots - 1) / slots) / plan.ksplit + 0.1;
+    if (r_tail <= r_split) { split = false; plan.ksplit = 1; }
+  }
+  if (split) {
+    cudaError_t e = cudaMemsetAsync(y, 0, (size_t)g.out_elems * 4, stream);
+    if (e != cudaSuccess) return e;
+  }
   if (use_shift)
-    return launch_shift_view(window, fp, y, reinterpret_cast<uint32_t*>(base), g, plan, sp, epi, split, encode, stream);
+    return launch_shift_view(window, fp, y, reinterpret_cast<uint32_t*>(base), reinterpret_cast<uint32_t*>(base + plan.flags_off),
+                             g, plan, sp, epi, split, encode, stream);
 
   // Activation operand: (k, wo, strip) with OVERLAPPING rows: the row of output column wo starts
   // s*Kh*Cp halves after that of wo-1.  k beyond K, columns beyond Wo and strips beyond N*Ho read

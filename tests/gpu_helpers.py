@@ -152,7 +152,7 @@ def gpu_transform_nhwc(x_nchw_bits: torch.Tensor, dims: dict, x_layout: str) -> 
 
 
 def gpu_conv_nhwc(x_cpu: torch.Tensor, f_cpu: torch.Tensor, dims: dict, x_layout="nchw", bias=None, relu=False,
-                  out16=False, y_nhwc=False, packed=False):
+                  out16=False, y_nhwc=False, packed=False, repeat=1):
     """NHWC transform + convolution through the C ABI with guard bands.  Returns y as a float64 numpy
     array in the requested layout ([N,Co,Ho,Wo] or [N,Ho,Wo,Co])."""
     xh = x_cpu.half()
@@ -170,7 +170,8 @@ def gpu_conv_nhwc(x_cpu: torch.Tensor, f_cpu: torch.Tensor, dims: dict, x_layout
     binding.im2win_transform_nhwc(xd, binding.NCHW if x_layout == "nchw" else binding.NHWC, win, dims)
     if packed:
         binding.im2win_pack_filter_nhwc(fd, scratch, dims)
-        binding.im2win_conv_packed_nhwc(win, y, scratch, dims, epi)
+        for _ in range(repeat):                      # the same packed filter and scratch, call after call
+            binding.im2win_conv_packed_nhwc(win, y, scratch, dims, epi)
     else:
         binding.im2win_conv_f16_nhwc(win, fd, y, scratch, dims, epi)
     binding.im2win_check_status(scratch)

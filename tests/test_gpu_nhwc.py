@@ -155,6 +155,42 @@ def test_conv_nhwc_two_mma_issuers(layer, dual, monkeypatch):
     check_conv(gpu_conv_nhwc(x, f, dims), y_pre, a, "f16", layer.name)
 
 
+_SHORT_LAST_ROUND = L("short_last_round", 13, 128, 24, 26, 300, 7, 7, 1, 3, 62)    # 14 k2-blocks x 7 kernel columns per item
+_short_last_round_refs = {}
+
+
+def _short_last_round_reference():
+    """The oracle's results for the layer above, computed once for all variants of the test."""
+    if not _short_last_round_refs:
+        dims = _SHORT_LAST_ROUND.dims()
+        xi, fi = workloads.make_small_integer_inputs(_SHORT_LAST_ROUND)
+        yi, _ = oracle.conv_direct(xi.numpy(), fi.numpy(), dims)
+        x, f = workloads.make_inputs(_SHORT_LAST_ROUND)
+        y_pre, _, a = _reference(x, f, dims)
+        _short_last_round_refs.update(xi=xi, fi=fi, yi=yi, x=x, f=f, y_pre=y_pre, a=a)
+    return _short_last_round_refs
+
+
+@pytest.mark.parametrize("tail", ["k", "n", "off"])
+def test_conv_nhwc_short_last_round(tail, monkeypatch):
+    """78 tile items on 74 CTA pairs with a streamed filter: the four tiles of the last round are handed
+    out as K parts (part 0 stores and raises the tile's flag, the others wait for it and add with
+    red.global.add.f32), as channel parts, or whole.  Exact on integer-valued inputs (three calls on
+    the same scratch: the flags carry a per-launch value), within tolerance on the seeded ones; with a
+    ReLU the K parts must not be taken (the result stays exact)."""
+    monkeypatch.setenv("IM2WIN_NHWC_KERNEL", "shift")
+    if tail == "off":
+        monkeypatch.setenv("IM2WIN_NHWC_TAIL", "0")
+    if tail == "n":
+        monkeypatch.setenv("IM2WIN_NHWC_TAIL_K", "0")
+    dims = _SHORT_LAST_ROUND.dims()
+    r = _short_last_round_reference()
+    assert np.array_equal(gpu_conv_nhwc(r["xi"], r["fi"], dims), r["yi"])
+    assert np.array_equal(gpu_conv_nhwc(r["xi"], r["fi"], dims, packed=True, repeat=3), r["yi"])
+    assert np.array_equal(gpu_conv_nhwc(r["xi"], r["fi"], dims, relu=True), np.maximum(r["yi"], 0))
+    check_conv(gpu_conv_nhwc(r["x"], r["f"], dims), r["y_pre"], r["a"], "f16", _SHORT_LAST_ROUND.name)
+
+
 def test_conv_nhwc_exact_with_integer_bias_relu_and_half_store():
     """Small integers all the way: bias, ReLU and the binary16 store must reproduce the oracle exactly."""
     layer = SMALL[2]
