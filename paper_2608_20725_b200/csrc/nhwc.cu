@@ -494,8 +494,8 @@ struct ShiftViewParams {
 // k2-blocks [kb0, kb1) of an item: its K part (ks of q.ksplit), or for a tail part that splits the
 // reduction its tail_kb blocks.
 __device__ __forceinline__ void item_blocks(const ShiftViewParams& q, int ks, int part, int* kb0, int* kb1) {
-  const int per = (q.tail_k && part >= 0) ? q.tail_kb : q.kb_per_split;
-  const int first = ((q.tail_k && part >= 0) ? part : ks) * per;
+  const int per = (part >= 0 && q.tail_k) ? q.tail_kb : q.kb_per_split;     // (part is the constant -1 in kernels without tail items)
+  const int first = ((part >= 0 && q.tail_k) ? part : ks) * per;
   *kb0 = first;
   *kb1 = first + per < q.nkb2 ? first + per : q.nkb2;
 }
@@ -549,7 +549,10 @@ __device__ __forceinline__ void issue_k2_block(uint32_t acc, uint32_t a_stage, u
   }
 }
 
-template <int BN, bool PAIR>
+// TAIL: the launch has items that are parts of a tile (a short last round, see decode_shift_item); without
+// them every item is a whole tile and the part handling drops out of the code (layers with very short
+// items, a 3x3 stem has six MMAs per item, pay for every instruction in the per-item paths).
+template <int BN, bool PAIR, bool TAIL>
 __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const CUtensorMap& bmap, const CUtensorMap& bmap_h,
                                                 const CUtensorMap& bmap_q, const ShiftViewParams& q) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;
@@ -613,24 +616,26 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       wait_for_previous_kernel();
       // with two issuing warps the ring is two rings of half the stages: even items fill one, odd items the other
       const int nst = q.dual ? q.sa / 2 : q.sa;
-      int st2[2] = {0, 0};
-      uint32_t ph2[2] = {0u, 0u};
+      int st_even = 0, st_odd = 0;             // (scalars, not an array indexed by the ring: that would live in local memory)
+      uint32_t ph_even = 0u, ph_odd = 0u;
       uint32_t it = 0;
       bool ok = true;
       TIMER_DECL;
       for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
-        int whole, part;
-        decode_shift_item(q, w, &whole, &part);
+        int whole = w, part = -1;
+        if (TAIL) decode_shift_item(q, w, &whole, &part);
         const int mt = whole / per_mt, rem = whole - mt * per_mt;
         const int ks = rem % q.ksplit;
         const int q0 = (PAIR ? 2 * mt + (int)rank : mt) * TILE_M;
         int kb0, kb1;
         item_blocks(q, ks, part, &kb0, &kb1);
-        const int r = q.dual ? (int)(it & 1u) : 0;
+        const bool odd = q.dual && (it & 1u);
+        int stl = odd ? st_odd : st_even;
+        uint32_t phl = odd ? ph_odd : ph_even;
         for (int kb = kb0; kb < kb1; ++kb) {
-          const int st = r * nst + st2[r];
+          const int st = (odd ? nst : 0) + stl;
           if (lane == 0) TIMER_LAP(0);                   // activation copies: issuing
-          ok = mbar_wait(a_empty0 + 8 * st, ph2[r] ^ 1u, &abort_flag, q.status);
+          ok = mbar_wait(a_empty0 + 8 * st, phl ^ 1u, &abort_flag, q.status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           if (lane == 0) TIMER_LAP(1);                   // activation copies: wait for a free stage
@@ -645,8 +650,9 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
             }
           }
           __syncwarp();
-          if (++st2[r] == nst) { st2[r] = 0; ph2[r] ^= 1u; }
+          if (++stl == nst) { stl = 0; phl ^= 1u; }
         }
+        if (odd) { st_odd = stl; ph_odd = phl; } else { st_even = stl; ph_even = phl; }
       }
       if (lane == 0 && blockIdx.x == 0) { TIMER_LAP(0); TIMER_FLUSH(); }
     }
@@ -659,8 +665,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       uint32_t ph = 0;
       bool ok = true;
       for (int w = w_first; w < q.nwork && ok; w += w_step) {
-        int whole, part;
-        decode_shift_item(q, w, &whole, &part);
+        int whole = w, part = -1;
+        if (TAIL) decode_shift_item(q, w, &whole, &part);
         const int rem = whole % per_mt;
         const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
         // filter rows of this CTA: its share of the tile's channels, or of one part of them
@@ -722,8 +728,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       for (int v = 0; v < 7; ++v) tapr[v] = v < q.Kw ? tap16[v] : 0u;
       TIMER_DECL;
       for (int w = w_first + mid * w_step; w < q.nwork && ok; w += nroles * w_step, it += (uint32_t)nroles) {
-        int whole, part;
-        decode_shift_item(q, w, &whole, &part);
+        int whole = w, part = -1;
+        if (TAIL) decode_shift_item(q, w, &whole, &part);
         const uint32_t idesc = (part < 0 || q.tail_k) ? idesc_whole : idesc_part;
         const int rem = whole % per_mt;
         const int ks = rem % q.ksplit;
@@ -865,11 +871,11 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
     TIMER_DECL;
     for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
       const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
-      int whole, part;
-      decode_shift_item(q, w, &whole, &part);
+      int whole = w, part = -1;
+      if (TAIL) decode_shift_item(q, w, &whole, &part);
       const int mt = whole / per_mt, rem = whole - mt * per_mt;
       const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
-      const bool kpart = q.tail_k && part >= 0;        // a tail item that holds one K part of all channels
+      const bool kpart = TAIL && q.tail_k && part >= 0;        // a tail item that holds one K part of all channels
       const int n0 = nt * BN + ((part > 0 && !kpart) ? part * (BN >> q.tail_log2) : 0);
       const int cols = (part < 0 || kpart) ? BN : BN >> q.tail_log2;
       // accumulator row = virtual position vq = strip*Wq + i; columns i >= Wo of a strip are no output
@@ -936,20 +942,20 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
   }
 }
 
-template <int BN>
+template <int BN, bool TAIL>
 __global__ void __launch_bounds__(SHIFT_THREADS, 1)
 conv_f16_nhwc_shift_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
                            const __grid_constant__ CUtensorMap bmap_h, const __grid_constant__ CUtensorMap bmap_q,
                            ShiftViewParams q) {
-  conv_shift_body<BN, false>(amap, bmap, bmap_h, bmap_q, q);
+  conv_shift_body<BN, false, TAIL>(amap, bmap, bmap_h, bmap_q, q);
 }
 
-template <int BN>
+template <int BN, bool TAIL>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(SHIFT_THREADS, 1)
 conv_f16_nhwc_shift_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
                                 const __grid_constant__ CUtensorMap bmap_h, const __grid_constant__ CUtensorMap bmap_q,
                                 ShiftViewParams q) {
-  conv_shift_body<BN, true>(amap, bmap, bmap_h, bmap_q, q);
+  conv_shift_body<BN, true, TAIL>(amap, bmap, bmap_h, bmap_q, q);
 }
 
 // Filter pack (paper Section "Im2win Convolution": height before width; here with the channel below
@@ -1474,7 +1480,8 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
   // two MMA issuers (see the kernel): a resident filter held as whole k2-blocks, and for each issuer
   // activation stages for a whole item (measured: 2-5 % faster then, cfg3 148 -> 142 us, a 3x3 layer
   // with 56x56 images and 64 channels 90 -> 86; with half-item rings a 128-channel layer lost 27 %)
-  q.dual = (q.resident && q.bu == q.Kw && q.sa / 2 >= sp.nkb2 && q.nwork >= 2) ? 1 : 0;
+  // and items of 24 MMAs or more (a 3x3 stem, six MMAs per item and bound by its output stores, lost a third)
+  q.dual = (q.resident && q.bu == q.Kw && q.sa / 2 >= sp.nkb2 && q.nwork >= 2 && sp.nkb2 * q.Kw * (KB / 16) >= 24) ? 1 : 0;
   if (const char* v = debug_getenv("IM2WIN_NHWC_DUAL")) q.dual = (q.dual && v[0] != '0') ? 1 : 0;
   const int smem_bytes = q.sa * (int)sp.a_stage_bytes + q.sb * b_stage + 1024;
   static int cached_clusters[64] = {};
@@ -1486,7 +1493,9 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
   int slots = PAIR ? 74 : 148;
   if (PAIR) {
     if (attr_bytes[dev] < smem_bytes) {
-      cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
+      cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_pair_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
+      if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(conv_f16_nhwc_shift_pair_kernel<BN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
       if (e != cudaSuccess) return report(e, "shared-memory opt-in (shifted view, pairs)");
       attr_bytes[dev] = kSmemMax - 1024;
     }
@@ -1501,7 +1510,7 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
       probe.dynamicSmemBytes = (size_t)(kSmemMax - 1024);   // the worst case: one CTA per SM either way
       probe.attrs = pattr;
       probe.numAttrs = 1;
-      cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_nhwc_shift_pair_kernel<BN>, &probe);
+      cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_nhwc_shift_pair_kernel<BN, true>, &probe);
       if (e != cudaSuccess) return e;
       if (clusters < 1) return cudaErrorInvalidValue;
       cached_clusters[dev] = clusters;
@@ -1563,10 +1572,14 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
     const int clusters = slots < q.nwork ? slots : q.nwork;
     cfg.gridDim = dim3(2 * clusters, 1, 1);
     cfg.numAttrs = 2;
-    return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_pair_kernel<BN>, amap, bmap, bmap_h, bmap_q, q), "pair launch (shifted view)");
+    if (q.tail_log2 > 0)
+      return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_pair_kernel<BN, true>, amap, bmap, bmap_h, bmap_q, q), "pair launch (shifted view, parts)");
+    return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_pair_kernel<BN, false>, amap, bmap, bmap_h, bmap_q, q), "pair launch (shifted view)");
   }
   if (attr_bytes[dev] < smem_bytes) {
-    cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
+    cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(conv_f16_nhwc_shift_kernel<BN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
     if (e != cudaSuccess) return report(e, "shared-memory opt-in (shifted view)");
     attr_bytes[dev] = kSmemMax - 1024;
   }
@@ -1575,7 +1588,9 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cfg.gridDim = dim3((unsigned)(slots < q.nwork ? slots : q.nwork), 1, 1);
-  return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_kernel<BN>, amap, bmap, bmap_h, bmap_q, q), "launch (shifted view)");
+  if (q.tail_log2 > 0)
+    return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_kernel<BN, true>, amap, bmap, bmap_h, bmap_q, q), "launch (shifted view, parts)");
+  return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_kernel<BN, false>, amap, bmap, bmap_h, bmap_q, q), "launch (shifted view)");
 }
 
 cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* y, uint32_t* status, uint32_t* flags,
