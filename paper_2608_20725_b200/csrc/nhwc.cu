@@ -138,10 +138,17 @@ __device__ __forceinline__ void store_chunk(const EpiParams& q, int64_t base, in
 
 // Bias (first K part only), ReLU and store of 32 channels from c0 on of one accumulator row.
 __device__ __forceinline__ void finish_chunk(const EpiParams& e, uint32_t (&v)[32], int c0, int n0, bool first_part,
-                                             bool valid, int64_t base, int64_t cs, bool vec_ok, bool add = false) {
+                                             bool valid, int64_t base, int64_t cs, bool vec_ok, bool add = false,
+                                             const float* bias_regs = nullptr) {
   const int cnt = e.Co - n0 - c0;                // channels left from c0 on
   if (cnt <= 0) return;
-  if (e.bias != nullptr && first_part) {
+  if (bias_regs != nullptr) {
+    // this warp's 32 bias values, loaded once before the first tile (zeros beyond Co)
+    if (first_part) {
+#pragma unroll
+      for (int t = 0; t < 32; ++t) v[t] = __float_as_uint(__uint_as_float(v[t]) + bias_regs[t]);
+    }
+  } else if (e.bias != nullptr && first_part) {
     // every lane adds the same 32 channel values: uniform 16-byte loads (the bias is 16-byte aligned
     // and n0 + c0 a multiple of 32), element by element at the ragged end
     if (cnt >= 32) {
@@ -167,6 +174,19 @@ __device__ __forceinline__ void finish_chunk(const EpiParams& e, uint32_t (&v)[3
   if (valid) store_chunk(e, base + (int64_t)c0 * cs, cs, v, cnt < 32 ? cnt : 32, vec_ok, add);
 }
 
+// Tiles of 64 channels with one channel tile: an epilogue warp stores the same 32 channels for every
+// tile, so it loads their bias once (with the largest shared-memory carve-out a global load per tile is
+// an L2 round trip of 600-800 cycles on warps that bound these layers: measured 143 -> 189 us on a 7x7
+// stem).  Returns whether breg is to be used.
+template <int BN>
+__device__ __forceinline__ bool hoist_bias(const EpiParams& e, int ntn, int warp, float (&breg)[32]) {
+  if (BN != 64 || e.bias == nullptr || ntn != 1) return false;
+  const int c0 = ((warp - WARP_EPI0) >> 2) * 32;
+#pragma unroll
+  for (int t = 0; t < 32; ++t) breg[t] = c0 + t < e.Co ? __ldg(e.bias + c0 + t) : 0.0f;
+  return true;
+}
+
 // One epilogue warp's share of a finished accumulator: tensor-memory lane quadrant warp % 4, the
 // lower (warps 2..5) or upper (warps 6..9) half of the tile's `cols` channels, 32 channels at a time:
 // bias, ReLU, store.  The tensor-memory load of the next 32 channels is in flight while the current
@@ -174,7 +194,7 @@ __device__ __forceinline__ void finish_chunk(const EpiParams& e, uint32_t (&v)[3
 // channel at this lane's position, `cs` the element distance between channels.
 __device__ __forceinline__ void drain_accumulator(const EpiParams& e, int cols, int warp, int lane, uint32_t lane_base,
                                                   bool valid, int64_t base, int64_t cs, int n0, bool first_part, bool vec_ok,
-                                                  bool add = false) {
+                                                  bool add = false, const float* bias_regs = nullptr) {
   const int CH = cols / 2;                       // a multiple of 32
   const int cbeg = ((warp - WARP_EPI0) >> 2) * CH;
   const int cend = cbeg + CH;
@@ -184,7 +204,7 @@ __device__ __forceinline__ void drain_accumulator(const EpiParams& e, int cols, 
   for (int c0 = cbeg; c0 < cend; c0 += 64) {
     tmem_ld_wait_for(va);
     if (c0 + 32 < cend) tmem_ld32_issue(lane_base + (uint32_t)(c0 + 32), vb);
-    finish_chunk(e, va, c0, n0, first_part, valid, base, cs, vec_ok, add);
+    finish_chunk(e, va, c0, n0, first_part, valid, base, cs, vec_ok, add, bias_regs);
     if (c0 + 32 >= cend) break;
     tmem_ld_wait_for(vb);
     if (c0 + 64 < cend) tmem_ld32_issue(lane_base + (uint32_t)(c0 + 64), va);
@@ -368,6 +388,8 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
     const EpiParams& e = q.e;
     const bool vec_ok = e.out16 ? (e.Co % 8 == 0) : (e.Co % 4 == 0);
     wait_for_previous_kernel();                  // before the first store to y
+    float breg[32];
+    const bool hoisted = hoist_bias<BN>(e, q.ntn, warp, breg);
     bool ok = true;
     uint32_t it = 0;
     TIMER_DECL;
@@ -404,7 +426,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(6);     // epilogue: wait for a finished accumulator
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
-      drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok);
+      drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok, false, hoisted ? breg : nullptr);
       // the buffer may be overwritten once all four warps (of both CTAs) have read it
       tc_fence_before();
       __syncwarp();
@@ -866,6 +888,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
     const EpiParams& e = q.e;
     const bool vec_ok = e.out16 ? (e.Co % 8 == 0) : (e.Co % 4 == 0);
     wait_for_previous_kernel();
+    float breg[32];
+    const bool hoisted = hoist_bias<BN>(e, q.ntn, warp, breg);
     bool ok = true;
     uint32_t it = 0;
     TIMER_DECL;
@@ -910,7 +934,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
         ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
         __syncwarp();
       }
-      if (ok) drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, kpart ? part == 0 : ks == 0, vec_ok, adds);
+      if (ok) drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, kpart ? part == 0 : ks == 0, vec_ok, adds,
+                                hoisted ? breg : nullptr);
       if (kpart && part == 0) {
         __threadfence();
         named_barrier_sync(1, EPI_WARPS * 32);          // all eight epilogue warps have stored
