@@ -158,8 +158,10 @@ im2win_status im2win_conv_packed(const void* window, float* y_nchw, void* scratc
  * Words 1 and 2 are testing aids read by the fp16 kernels: a non-zero word 1
  * replaces the number of polls after which a wait gives up (2^24, and never
  * more than about four seconds); the marker 0x0d0a11fe in word 2 makes the
- * one-k-block kernel leave out one barrier arrival, so that a test can watch a
- * wait run out and the kernel return.  Nothing in the library writes them.
+ * one-k-block kernel leave out one barrier arrival, the marker 0x0d0a11ff makes
+ * the NHWC shifted-view kernel keep down the flags its split tiles hand their
+ * partial sums over with, so that a test can watch a wait run out and the
+ * kernel return.  Nothing in the library writes them.
  */
 im2win_status im2win_check_status(const void* scratch, void* cuda_stream);
 

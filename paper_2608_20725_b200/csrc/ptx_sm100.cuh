@@ -18,6 +18,9 @@ constexpr uint64_t SPIN_TIME_NS = 4000000000ull;   // wall-time bound of one wai
 // Word 2 of the status block: this marker makes the one-k-block kernel's copy warp leave out one
 // barrier arrival (the test of the bounded waits; nothing in the library writes it).
 constexpr uint32_t kDebugDropArrive = 0x0d0a11feu;
+// Word 2 again: with this marker the NHWC shifted-view kernel's first K part of a tile does not raise
+// the tile's flag, so that the parts waiting for it run into their limit (same purpose).
+constexpr uint32_t kDebugDropFlag = 0x0d0a11ffu;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);

@@ -191,6 +191,31 @@ def test_conv_nhwc_short_last_round(tail, monkeypatch):
     check_conv(gpu_conv_nhwc(r["x"], r["f"], dims), r["y_pre"], r["a"], "f16", _SHORT_LAST_ROUND.name)
 
 
+def test_conv_nhwc_flag_wait_is_bounded(monkeypatch):
+    """The K parts of a short last round wait for part 0's flag.  With the poll limit lowered (word 1 of
+    the status block) and the flag kept down (marker in word 2) those waits run out: the kernel returns,
+    the status reads IM2WIN_ERR_TIMEOUT, nothing faults or hangs, and the next call on the same buffers
+    (a fresh filter pack clears the block) is exact."""
+    monkeypatch.setenv("IM2WIN_NHWC_KERNEL", "shift")
+    dims = _SHORT_LAST_ROUND.dims()
+    r = _short_last_round_reference()
+    xd, fd = r["xi"].half().cuda(), r["fi"].half().cuda()
+    window, scratch, y = binding.alloc_nhwc_buffers(dims)
+    binding.im2win_transform_nhwc(xd, binding.NCHW, window, dims)
+    binding.im2win_pack_filter_nhwc(fd, scratch, dims)
+    torch.cuda.synchronize()
+    words = scratch[:256].view(torch.int32)
+    words[1] = 4096                       # poll limit of every wait of the next kernel
+    words[2] = 0x0d0a11ff                 # part 0 of every split tile keeps its flag down
+    binding.im2win_conv_packed_nhwc(window, y, scratch, dims)
+    with pytest.raises(binding.Im2winError) as err:
+        binding.im2win_check_status(scratch)          # synchronises: the kernel did return
+    assert err.value.code == 7
+    binding.im2win_conv_f16_nhwc(window, fd, y, scratch, dims)
+    binding.im2win_check_status(scratch)
+    assert np.array_equal(y.cpu().double().numpy().reshape(r["yi"].shape), r["yi"])
+
+
 def test_conv_nhwc_exact_with_integer_bias_relu_and_half_store():
     """Small integers all the way: bias, ReLU and the binary16 store must reproduce the oracle exactly."""
     layer = SMALL[2]
