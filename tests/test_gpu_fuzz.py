@@ -9,7 +9,7 @@ import pytest
 import torch
 
 from paper_2608_20725_b200 import workloads
-from gpu_helpers import check_conv, gpu_conv, gpu_transform, oracle, oracle_inputs
+from gpu_helpers import check_conv, check_fused, gpu_conv, gpu_conv_nhwc, gpu_transform, gpu_transform_nhwc, oracle, oracle_inputs
 
 pytestmark = pytest.mark.gpu
 
@@ -58,3 +58,28 @@ def test_random_layer_all_paths(layer):
     for precision in ("f16", "f16-mat", "f16-shift", "f16-stem", "f16-gather"):
         y, _, _ = gpu_conv(x, f, dims, precision)
         check_conv(y, yr16, ar16, precision, layer.name)
+
+
+@pytest.mark.parametrize("layer", FUZZ, ids=lambda l: l.name)
+def test_random_layer_nhwc_paths(layer, monkeypatch):
+    """The same layers through the channel-innermost (NHWC) form: the transform from both input layouts
+    bit for bit, the convolution through the kernel the library picks and through each of its two
+    kernels forced, and once with the fused epilogue (bias, ReLU, binary16 NHWC store)."""
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    raw = x.half().view(torch.int16)
+    got = gpu_transform_nhwc(raw, dims, "nchw")
+    want = oracle.transform_nhwc(raw.numpy(), dims, "nchw", got.shape[-1])
+    assert np.array_equal(got, want), layer.name
+    assert np.array_equal(gpu_transform_nhwc(raw, dims, "nhwc"), want), layer.name
+    xo, fo = oracle_inputs(x, f, "f16")
+    yr, ar = oracle.conv_direct(xo, fo, dims)
+    for kernel in ("default", "shift", "overlap"):
+        if kernel != "default":
+            monkeypatch.setenv("IM2WIN_NHWC_KERNEL", kernel)
+        check_conv(gpu_conv_nhwc(x, f, dims), yr, ar, "f16", f"{layer.name} {kernel}")
+    monkeypatch.delenv("IM2WIN_NHWC_KERNEL")
+    bias = torch.randn(layer.Co, generator=torch.Generator().manual_seed(layer.seed + 7)).numpy() * 0.5
+    y_pre, a2 = oracle.epilogue(yr, ar, dims, bias=bias, relu=True, out16=False, nhwc=True)
+    y = gpu_conv_nhwc(x, f, dims, bias=bias, relu=True, out16=True, y_nhwc=True)
+    check_fused(y, y_pre, a2, True, f"{layer.name} fused")
