@@ -547,8 +547,11 @@ def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
                "median_ms": median, "back_to_back_ms": b2b, "buffer_sets": sets,
                "kernels": kernel_rooflines(runner, avg, peaks, peak_kind),
                "kernels_back_to_back": kernel_rooflines(runner, b2b, peaks, peak_kind),
-               "conv_kernel": {p: binding.im2win_conv_kernel_name(layer.dims(), binding.F32 if p == "f32" else binding.F16)
-                               for p in layer.precisions},
+               "conv_kernel": dict({p: binding.im2win_conv_kernel_name(layer.dims(), binding.F32 if p == "f32" else binding.F16)
+                                    for p in layer.precisions},
+                                   **({"f16_nhwc": binding.im2win_nhwc_kernel_name(layer.dims()),
+                                       "f16_out16_nhwc": binding.im2win_nhwc_kernel_name(layer.dims(), runner.nhwc["epi16"])}
+                                      if runner.nhwc is not None else {})),
                "memory": runner.memory_report()}
         if with_packed:
             # the convolution kernel without the filter pack (static weights), for reference
@@ -589,7 +592,8 @@ def per_layer_summary(rows):
             e["back_to_back"] = {"ms": round(kb["ms"], 5), "bound": kb["bound"], "frac": round(kb["frac"], 4)}
             if key.startswith("conv"):
                 e["tflops"] = round(row["gflop"] / k["ms"], 2)      # GFLOP per ms = TFLOP/s
-                e["kernel"] = "f16-nhwc-tma" if key.endswith("nhwc") else row["conv_kernel"][key.split("_")[1]]
+                e["kernel"] = row["conv_kernel"]["f16_out16_nhwc" if key == "conv_f16_out16_nhwc" else "f16_nhwc"] \
+                    if key.endswith("nhwc") else row["conv_kernel"][key.split("_")[1]]
                 if "f16" in key:
                     e["frac_of_tensor_peak"] = round(k["frac_of_tensor_peak"], 4)
             entry[key] = e

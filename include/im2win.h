@@ -276,6 +276,17 @@ im2win_status im2win_conv_packed_nhwc(const uint16_t* window, void* y, const im2
                                       void* cuda_stream);
 
 /*
+ * Name of the kernel im2win_conv_f16_nhwc selects for a layer and an epilogue
+ * (NULL: the plain one); host-only, launches nothing, static storage:
+ * "f16-nhwc-shift" (row-shifted MMA views of columns staged once) or
+ * "f16-nhwc-overlap" (a tensor map with overlapping rows), with "+ksplit" when
+ * every tile's reduction is split over several CTAs; "none" for a shape the
+ * NHWC form does not take.  For reports and tests; the choice is an
+ * implementation detail.
+ */
+const char* im2win_nhwc_kernel_name(const im2win_shape* shape, const im2win_epilogue* epilogue);
+
+/*
  * fp32 convolution without a scratch argument, for callers that cannot allocate
  * device memory (the paper has no counterpart; this is a convenience of this
  * library).  Think of code running where cudaMalloc is off limits: a real-time

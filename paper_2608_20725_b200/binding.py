@@ -25,7 +25,7 @@ STATUS_NAMES = {
 EXPORTS = (
     "im2win_status_string", "im2win_workspace_size", "im2win_transform", "im2win_conv_f32", "im2win_conv_f16",
     "im2win_check_status", "im2win_layer_workspace_size", "im2win_layer_forward_host",
-    "im2win_conv_f32_static", "im2win_pack_filter", "im2win_conv_packed", "im2win_conv_kernel_name",
+    "im2win_conv_f32_static", "im2win_pack_filter", "im2win_conv_packed", "im2win_conv_kernel_name", "im2win_nhwc_kernel_name",
     "im2win_nhwc_workspace_size", "im2win_transform_nhwc", "im2win_conv_f16_nhwc", "im2win_pack_filter_nhwc",
     "im2win_conv_packed_nhwc",
 )
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
     for name in EXPORTS[1:]:
         getattr(L, name).restype = ctypes.c_int
     L.im2win_conv_kernel_name.restype = ctypes.c_char_p
+    L.im2win_nhwc_kernel_name.argtypes = [P(Shape), P(Epilogue)]
+    L.im2win_nhwc_kernel_name.restype = ctypes.c_char_p
     _lib = L
     return L
 
@@ -152,6 +154,12 @@ def im2win_conv_kernel_name(shape, dtype: int) -> str:
     """Name of the convolution kernel the library selects for the layer (for reports and tests)."""
     s = as_shape(shape)
     return lib().im2win_conv_kernel_name(ctypes.byref(s), dtype).decode()
+
+
+def im2win_nhwc_kernel_name(shape, epilogue: Optional["Epilogue"] = None) -> str:
+    """Name of the kernel im2win_conv_f16_nhwc selects for the layer and epilogue (for reports and tests)."""
+    s = as_shape(shape)
+    return lib().im2win_nhwc_kernel_name(ctypes.byref(s), None if epilogue is None else ctypes.byref(epilogue)).decode()
 
 
 def im2win_transform(x: torch.Tensor, window: torch.Tensor, shape, stream=None) -> None:

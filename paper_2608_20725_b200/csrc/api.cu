@@ -274,6 +274,13 @@ static im2win_status nhwc_common(const uint16_t* window, const uint16_t* filter,
   return IM2WIN_OK;
 }
 
+const char* im2win_nhwc_kernel_name(const im2win_shape* shape, const im2win_epilogue* epilogue) {
+  Geometry g;
+  EpilogueArgs epi;
+  if (!shape || derive_geometry(shape, &g) != IM2WIN_OK || epilogue_args(epilogue, true, &epi) != IM2WIN_OK) return "none";
+  return nhwc_kernel_name(g, epi);
+}
+
 im2win_status im2win_nhwc_workspace_size(const im2win_shape* shape, size_t* window_bytes, size_t* scratch_bytes,
                                          int32_t* Ho, int32_t* Wo, int32_t* Cp) {
   Geometry g;

@@ -146,6 +146,7 @@ cudaError_t launch_conv_f16_shift(const uint16_t* window, float* y, void* scratc
 
 cudaError_t launch_transform_nhwc(const uint16_t* x, int x_is_nhwc, uint16_t* window, const Geometry& g,
                                   cudaStream_t stream);
+const char* nhwc_kernel_name(const Geometry& g, const EpilogueArgs& epi);
 cudaError_t launch_pack_f16_nhwc(const uint16_t* filter, void* scratch, const Geometry& g, cudaStream_t stream);
 cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch, const Geometry& g,
                                  const EpilogueArgs& epi, cudaStream_t stream);

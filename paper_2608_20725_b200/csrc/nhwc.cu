@@ -1821,14 +1821,21 @@ cudaError_t launch_pack_f16_nhwc(const uint16_t* filter, void* scratch, const Ge
   return cudaGetLastError();
 }
 
-cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch, const Geometry& g,
-                                 const EpilogueArgs& epi, cudaStream_t stream) {
-  NhwcPlan plan = plan_nhwc(g);
-  if (!plan.eligible) return cudaErrorInvalidValue;
-  EncodeTiledFn encode = get_encode_fn();
-  if (!encode) return cudaErrorNotSupported;
-  unsigned char* base = static_cast<unsigned char*>(scratch);
-  uint16_t* fp = reinterpret_cast<uint16_t*>(base + kStatusBytes);
+namespace {
+
+// Everything a convolution call decides before it launches: tile plan, which of the two kernels, and
+// whether every tile's K is split over several CTAs (the output is then cleared first).
+struct NhwcChoice {
+  NhwcPlan plan;
+  ShiftViewPlan sp;
+  bool use_shift, split;
+};
+
+NhwcChoice choose_nhwc(const Geometry& g, const EpilogueArgs& epi) {
+  NhwcChoice c{};
+  NhwcPlan& plan = c.plan;
+  plan = plan_nhwc(g);
+  if (!plan.eligible) return c;
   // testing aids (read only when IM2WIN_DEBUG is set): tile width, pairing and K split
   if (const char* v = debug_getenv("IM2WIN_NHWC_BN")) {
     const int bn = atoi(v);
@@ -1846,7 +1853,8 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   // to keep its MMA warp's barrier traffic low.  Measured: it wins where every column is reused by
   // three kernel columns or more (Kw >= 3s) and two such filter stages fit beside two activation
   // stages; elsewhere the overlapping-row kernel is as fast or faster.
-  const ShiftViewPlan sp = plan_shift_view(g, plan);
+  c.sp = plan_shift_view(g, plan);
+  const ShiftViewPlan& sp = c.sp;
   const int64_t b_bytes = (int64_t)(plan.pair ? plan.bn / 2 : plan.bn) * KB * 2;
   // Kernels no wider than the stride read every column once in either kernel; there the shifted view
   // is taken when its full 128-position tiles need fewer rounds than the overlapping-row kernel's
@@ -1889,6 +1897,31 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
     const double r_split = (double)((it_s * plan.ksplit + slots - 1) / slots) / plan.ksplit + 0.1;
     if (r_tail <= r_split) { split = false; plan.ksplit = 1; }
   }
+  c.use_shift = use_shift;
+  c.split = split;
+  return c;
+}
+
+}  // namespace
+
+const char* nhwc_kernel_name(const Geometry& g, const EpilogueArgs& epi) {
+  const NhwcChoice c = choose_nhwc(g, epi);
+  if (!c.plan.eligible) return "none";
+  if (c.use_shift) return c.split ? "f16-nhwc-shift+ksplit" : "f16-nhwc-shift";
+  return c.split ? "f16-nhwc-overlap+ksplit" : "f16-nhwc-overlap";
+}
+
+cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch, const Geometry& g,
+                                 const EpilogueArgs& epi, cudaStream_t stream) {
+  const NhwcChoice c = choose_nhwc(g, epi);
+  if (!c.plan.eligible) return cudaErrorInvalidValue;
+  const NhwcPlan& plan = c.plan;
+  const ShiftViewPlan& sp = c.sp;
+  const bool use_shift = c.use_shift, split = c.split;
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return cudaErrorNotSupported;
+  unsigned char* base = static_cast<unsigned char*>(scratch);
+  uint16_t* fp = reinterpret_cast<uint16_t*>(base + kStatusBytes);
   if (split) {
     cudaError_t e = cudaMemsetAsync(y, 0, (size_t)g.out_elems * 4, stream);
     if (e != cudaSuccess) return e;
