@@ -107,12 +107,18 @@ struct EpilogueArgs {
   int32_t y_nhwc;          // 1: y is [N][Ho][Wo][Co], 0: [N][Co][Ho][Wo]
 };
 
+// Tile shape of the fp32 kernel for a layer (see conv_f32.cu); the packed filter's K is padded to bk.
+struct F32Plan {
+  int32_t bm, bn, bk;
+};
+F32Plan plan_f32(const Geometry& g);
+
 // Environment switches are testing aids: they are looked at only when IM2WIN_DEBUG is set in the
 // environment (checked once per process), so the default call path reads no environment.
 const char* debug_getenv(const char* name);
 
 constexpr int kStatusBytes = 256;
-constexpr int kF32KBlock = 16;     // k-block of the fp32 kernel
+constexpr int kF32KBlock = 16;     // smallest k-block of the fp32 kernel (see plan_f32)
 constexpr int kF16KBlock = 64;     // k-block of the fp16 kernel (64 halves = one 128-byte swizzle row)
 
 im2win_status derive_geometry(const im2win_shape* s, Geometry* g);

@@ -129,11 +129,13 @@ def test_conv_exact_on_integer_inputs(layer, precision):
 
 
 @pytest.mark.parametrize("layer", [SMALL[1], SMALL[2], L("wide_co", 3, 20, 11, 13, 150, 3, 3, 1, 1, 47)], ids=lambda l: l.name)
-@pytest.mark.parametrize("bm", ["64", "128"])
-def test_conv_f32_both_tile_heights(layer, bm, monkeypatch):
+@pytest.mark.parametrize("bm,bk", [("64", "16"), ("64", "32"), ("128", "16")])
+def test_conv_f32_both_tile_heights(layer, bm, bk, monkeypatch):
     """The fp32 kernel's 64- and 128-position tiles (the library picks by grid size), on 64- and
-    128-channel tiles: exact on integer-valued inputs, within tolerance on the seeded ones."""
+    128-channel tiles, and the 64 x 128 tile with both k-blocks: exact on integer-valued inputs,
+    within tolerance on the seeded ones."""
     monkeypatch.setenv("IM2WIN_F32_BM", bm)
+    monkeypatch.setenv("IM2WIN_F32_BK", bk)
     dims = layer.dims()
     x, f = workloads.make_small_integer_inputs(layer)
     y, _, _ = gpu_conv(x, f, dims, "f32")
