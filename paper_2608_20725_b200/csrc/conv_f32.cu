@@ -232,11 +232,11 @@ F32Plan plan_f32(const Geometry& g) {
     return (double)((tiles + 147) / 148) * bm;
   };
   bool small_m = waves_cost(64) < 0.9 * waves_cost(128);
-  // 128-channel tiles: with four to eight 128-position tiles per SM the partly filled last round of
+  // 128-channel tiles: with four to ten 128-position tiles per SM the partly filled last round of
   // 256-thread CTAs costs more than the 64-position tile's extra filter traffic (measured on 3x3 to
   // 7x7 layers at 28x28 and 10x10: 3-5 % faster; larger grids are 3-4 % faster with 128 positions)
   const int64_t tiles128 = (g.P + 127) / 128 * cot;
-  if (wide && tiles128 >= 4 * 148 && tiles128 < 8 * 148) small_m = true;
+  if (wide && tiles128 >= 4 * 148 && tiles128 < 10 * 148) small_m = true;
   if (const char* v = debug_getenv("IM2WIN_F32_BM")) small_m = atoi(v) == 64;   // testing aid
   p.bm = small_m ? 64 : 128;
   p.bk = (wide && small_m && g.K >= 256) ? 32 : 16;
