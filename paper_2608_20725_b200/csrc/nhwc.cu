@@ -574,7 +574,7 @@ __device__ __forceinline__ void issue_k2_block(uint32_t acc, uint32_t a_stage, u
 // TAIL: the launch has items that are parts of a tile (a short last round, see decode_shift_item); without
 // them every item is a whole tile and the part handling drops out of the code (layers with very short
 // items, a 3x3 stem has six MMAs per item, pay for every instruction in the per-item paths).
-template <int BN, bool PAIR, bool TAIL>
+template <int BN, bool PAIR, bool TAIL, bool HOIST>
 __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const CUtensorMap& bmap, const CUtensorMap& bmap_h,
                                                 const CUtensorMap& bmap_q, const ShiftViewParams& q) {
   constexpr int B_ROWS = PAIR ? BN / 2 : BN;
@@ -888,8 +888,14 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
     const EpiParams& e = q.e;
     const bool vec_ok = e.out16 ? (e.Co % 8 == 0) : (e.Co % 4 == 0);
     wait_for_previous_kernel();
-    float breg[32];
-    const bool hoisted = hoist_bias<BN>(e, q.ntn, warp, breg);
+    // HOIST (64-channel tiles, one channel tile, a bias): the warp's 32 bias values stay in registers.  A
+    // kernel of its own: the same choice taken at run time cost the stems without a bias 8-15 %.
+    float breg[HOIST ? 32 : 1];
+    if (HOIST) {
+      const int c0 = ((warp - WARP_EPI0) >> 2) * 32;
+#pragma unroll
+      for (int t = 0; t < (HOIST ? 32 : 1); ++t) breg[t] = c0 + t < e.Co ? __ldg(e.bias + c0 + t) : 0.0f;
+    }
     bool ok = true;
     uint32_t it = 0;
     TIMER_DECL;
@@ -935,7 +941,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
         __syncwarp();
       }
       if (ok) drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, kpart ? part == 0 : ks == 0, vec_ok, adds,
-                                hoisted ? breg : nullptr);
+                                HOIST ? breg : nullptr);
       if (kpart && part == 0) {
         __threadfence();
         named_barrier_sync(1, EPI_WARPS * 32);          // all eight epilogue warps have stored
@@ -969,20 +975,20 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
   }
 }
 
-template <int BN, bool TAIL>
+template <int BN, bool TAIL, bool HOIST>
 __global__ void __launch_bounds__(SHIFT_THREADS, 1)
 conv_f16_nhwc_shift_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
                            const __grid_constant__ CUtensorMap bmap_h, const __grid_constant__ CUtensorMap bmap_q,
                            ShiftViewParams q) {
-  conv_shift_body<BN, false, TAIL>(amap, bmap, bmap_h, bmap_q, q);
+  conv_shift_body<BN, false, TAIL, HOIST>(amap, bmap, bmap_h, bmap_q, q);
 }
 
-template <int BN, bool TAIL>
+template <int BN, bool TAIL, bool HOIST>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(SHIFT_THREADS, 1)
 conv_f16_nhwc_shift_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap,
                                 const __grid_constant__ CUtensorMap bmap_h, const __grid_constant__ CUtensorMap bmap_q,
                                 ShiftViewParams q) {
-  conv_shift_body<BN, true, TAIL>(amap, bmap, bmap_h, bmap_q, q);
+  conv_shift_body<BN, true, TAIL, HOIST>(amap, bmap, bmap_h, bmap_q, q);
 }
 
 // Filter pack (paper Section "Im2win Convolution": height before width; here with the channel below
@@ -1518,14 +1524,25 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
   // CTAs (pairs) that are resident together: the grid, and what "a round of tiles" means below.  The
   // items of a split last round wait for one another, so every one of them must have a CTA of its own.
   int slots = PAIR ? 74 : 148;
+  // the variants of this tile width: with / without tile parts, with / without the bias in registers
+  // (64-channel tiles with one channel tile only)
+  using Kernel = void (*)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, ShiftViewParams);
+  constexpr bool CAN_HOIST = BN == 64;
+  const Kernel variants[2][2] = {
+      {PAIR ? (Kernel)conv_f16_nhwc_shift_pair_kernel<BN, false, false> : (Kernel)conv_f16_nhwc_shift_kernel<BN, false, false>,
+       PAIR ? (Kernel)conv_f16_nhwc_shift_pair_kernel<BN, false, CAN_HOIST> : (Kernel)conv_f16_nhwc_shift_kernel<BN, false, CAN_HOIST>},
+      {PAIR ? (Kernel)conv_f16_nhwc_shift_pair_kernel<BN, true, false> : (Kernel)conv_f16_nhwc_shift_kernel<BN, true, false>,
+       PAIR ? (Kernel)conv_f16_nhwc_shift_pair_kernel<BN, true, CAN_HOIST> : (Kernel)conv_f16_nhwc_shift_kernel<BN, true, CAN_HOIST>}};
+  const bool hoist = CAN_HOIST && q.e.bias != nullptr && q.ntn == 1;
+  if (attr_bytes[dev] < smem_bytes) {
+    for (int t = 0; t < 2; ++t)
+      for (int h = 0; h < 2; ++h) {
+        const cudaError_t e = cudaFuncSetAttribute((const void*)variants[t][h], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
+        if (e != cudaSuccess) return report(e, "shared-memory opt-in (shifted view)");
+      }
+    attr_bytes[dev] = kSmemMax - 1024;
+  }
   if (PAIR) {
-    if (attr_bytes[dev] < smem_bytes) {
-      cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_pair_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
-      if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(conv_f16_nhwc_shift_pair_kernel<BN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
-      if (e != cudaSuccess) return report(e, "shared-memory opt-in (shifted view, pairs)");
-      attr_bytes[dev] = kSmemMax - 1024;
-    }
     int clusters = cached_clusters[dev];
     if (clusters == 0) {
       cudaLaunchConfig_t probe = {};
@@ -1537,7 +1554,7 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
       probe.dynamicSmemBytes = (size_t)(kSmemMax - 1024);   // the worst case: one CTA per SM either way
       probe.attrs = pattr;
       probe.numAttrs = 1;
-      cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, conv_f16_nhwc_shift_pair_kernel<BN, true>, &probe);
+      cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, (const void*)variants[1][CAN_HOIST ? 1 : 0], &probe);
       if (e != cudaSuccess) return e;
       if (clusters < 1) return cudaErrorInvalidValue;
       cached_clusters[dev] = clusters;
@@ -1599,25 +1616,16 @@ cudaError_t launch_shift_variant(const CUtensorMap& amap, const CUtensorMap& bma
     const int clusters = slots < q.nwork ? slots : q.nwork;
     cfg.gridDim = dim3(2 * clusters, 1, 1);
     cfg.numAttrs = 2;
-    if (q.tail_log2 > 0)
-      return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_pair_kernel<BN, true>, amap, bmap, bmap_h, bmap_q, q), "pair launch (shifted view, parts)");
-    return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_pair_kernel<BN, false>, amap, bmap, bmap_h, bmap_q, q), "pair launch (shifted view)");
-  }
-  if (attr_bytes[dev] < smem_bytes) {
-    cudaError_t e = cudaFuncSetAttribute(conv_f16_nhwc_shift_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(conv_f16_nhwc_shift_kernel<BN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - 1024);
-    if (e != cudaSuccess) return report(e, "shared-memory opt-in (shifted view)");
-    attr_bytes[dev] = kSmemMax - 1024;
+    return report(cudaLaunchKernelEx(&cfg, variants[q.tail_log2 > 0][hoist], amap, bmap, bmap_h, bmap_q, q),
+                  q.tail_log2 > 0 ? "pair launch (shifted view, parts)" : "pair launch (shifted view)");
   }
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cfg.gridDim = dim3((unsigned)(slots < q.nwork ? slots : q.nwork), 1, 1);
-  if (q.tail_log2 > 0)
-    return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_kernel<BN, true>, amap, bmap, bmap_h, bmap_q, q), "launch (shifted view, parts)");
-  return report(cudaLaunchKernelEx(&cfg, conv_f16_nhwc_shift_kernel<BN, false>, amap, bmap, bmap_h, bmap_q, q), "launch (shifted view)");
+  return report(cudaLaunchKernelEx(&cfg, variants[q.tail_log2 > 0][hoist], amap, bmap, bmap_h, bmap_q, q),
+                q.tail_log2 > 0 ? "launch (shifted view, parts)" : "launch (shifted view)");
 }
 
 cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* y, uint32_t* status, uint32_t* flags,
