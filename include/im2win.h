@@ -236,8 +236,10 @@ typedef struct {
 
 /*
  * Buffer sizes of the NHWC form (host-only): window_bytes = N*Ho*(W+2p)*Kh*Cp*2,
- * scratch_bytes for im2win_conv_f16_nhwc (status block + repacked filter), the
- * output size and the stored channel count Cp.  Any output pointer may be NULL.
+ * scratch_bytes for im2win_conv_f16_nhwc (status block + repacked filter + flag
+ * words + for layers of few rounds of tiles 19 MB for partial sums that CTAs
+ * hand to one another), the output size and the stored channel count Cp.  Any
+ * output pointer may be NULL.
  */
 im2win_status im2win_nhwc_workspace_size(const im2win_shape* shape, size_t* window_bytes, size_t* scratch_bytes,
                                          int32_t* Ho, int32_t* Wo, int32_t* Cp);
@@ -261,8 +263,11 @@ im2win_status im2win_transform_nhwc(const uint16_t* x, im2win_layout x_layout, u
  * filter is repacked into `scratch` on every call.  Layers with few position
  * tiles split the reduction over several CTAs, which add their partial sums
  * into a `y` the call clears first (only without ReLU and with binary32
- * output; the summation order then varies from run to run).  Waits are
- * bounded as in im2win_conv_f16 (see im2win_check_status).
+ * output; the summation order then varies from run to run).  A short last
+ * round of tiles may instead be shared between CTAs by runs of the reduction:
+ * the CTA that starts a tile adds the other CTAs' partial sums from `scratch`
+ * in a fixed order and applies the epilogue (any epilogue; deterministic).
+ * Waits are bounded as in im2win_conv_f16 (see im2win_check_status).
  * im2win_pack_filter_nhwc / im2win_conv_packed_nhwc are the two halves for
  * static weights.
  */
@@ -280,7 +285,9 @@ im2win_status im2win_conv_packed_nhwc(const uint16_t* window, void* y, const im2
  * (NULL: the plain one); host-only, launches nothing, static storage:
  * "f16-nhwc-shift" (row-shifted MMA views of columns staged once) or
  * "f16-nhwc-overlap" (a tensor map with overlapping rows), with "+ksplit" when
- * every tile's reduction is split over several CTAs; "none" for a shape the
+ * every tile's reduction is split over several CTAs or "+runs" when the tiles
+ * of a short last round are shared by runs of the reduction (decided for the
+ * nominal 148 SMs; the launch decides for the device); "none" for a shape the
  * NHWC form does not take.  For reports and tests; the choice is an
  * implementation detail.
  */

@@ -95,7 +95,9 @@ struct NhwcPlan {
   int64_t window_elems;    // N*Ho*strip
   int64_t ntm;             // position tiles
   size_t flags_off;        // byte offset of the tail-tile flag words inside the scratch
-  size_t scratch_bytes;    // status block + packed filter + flag words
+  size_t partial_off;      // byte offset and size of the partial-sum area (0 bytes: layer of many rounds of tiles)
+  size_t partial_bytes;
+  size_t scratch_bytes;    // status block + packed filter + flag words + partial sums
 };
 NhwcPlan plan_nhwc(const Geometry& g);
 

@@ -47,6 +47,13 @@ constexpr int A_SLOT_BYTES = TILE_M * KB * 2;  // 16 KB: room for 128 rows even 
 constexpr int kSmemMax = 227 * 1024;
 constexpr int MAX_ACC = 8;                     // accumulator buffers in tensor memory: 512 columns / BN, at most 8
 __host__ __device__ constexpr int acc_buffers(int bn) { return 512 / bn < MAX_ACC ? 512 / bn : MAX_ACC; }
+// Flag words of the hand-offs between CTAs that share a tile of a short last round: two per tile (shifted-view
+// kernel, one per CTA of a pair) or two per CTA pair of the grid (overlapping-row kernel), compared with a
+// value that differs from launch to launch.
+constexpr int kTailFlagBytes = 2048;
+// Partial sums of such tiles (overlapping-row kernel): one accumulator tile of 128 positions x 256 channels
+// of fp32 per CTA of the grid.
+constexpr size_t kPartialBytes = (size_t)148 * TILE_M * 256 * 4;
 
 // What the epilogue needs to know about the output (shared by both kernels of this file).
 struct EpiParams {
@@ -70,6 +77,14 @@ struct NhwcParams {
   int32_t tail_halves;       // host only: the last round's tiles may be handed out as halves
   int32_t n_main;            // work items below this index are whole tiles; each whole tile above it is two
                              // items, one per half of its channels (fills the last, short round of tiles)
+  // ... or, with stream_tiles > 0, the last round's tiles are handed out by reduction length: their
+  // stream_tiles * num_kc chunks in order, stream_u to each of the first stream_ctas CTAs (pairs), so a CTA
+  // holds the end of one tile's reduction and / or the start of the next one's.  The CTA that starts a tile
+  // stores it; the others leave their partial sums in `partial` and raise their flag.
+  int32_t stream_tiles, stream_u, stream_ctas;
+  float* partial;            // kPartialBytes
+  uint32_t* flags;           // two words per CTA (pair) of the grid, compared with `epoch`
+  uint32_t epoch;
 };
 
 // Programmatic dependent launch: the convolution may start while the kernel before it in the stream
@@ -212,6 +227,104 @@ __device__ __forceinline__ void drain_accumulator(const EpiParams& e, int cols, 
   }
 }
 
+// Bounded wait for a flag word to hold `value` (written with release semantics by another CTA).
+__device__ __noinline__ bool wait_flag(const uint32_t* flag, uint32_t value, volatile uint32_t* abort_flag, uint32_t* status) {
+  uint32_t limit = *reinterpret_cast<volatile uint32_t*>(status + 1);
+  if (limit == 0u) limit = SPIN_LIMIT;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t i = 0; i < limit; ++i) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v == value) return true;
+    if ((i & 255u) == 255u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > SPIN_TIME_NS) break;
+    }
+    __nanosleep(64);
+  }
+  *abort_flag = 1u;
+  atomicExch(status, 1u);
+  return false;
+}
+
+__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// CTA `cta`'s two stream items (see NhwcParams): slot 0 is the part of its chunk range that does not start
+// a tile (it ends the tile the CTA before it started), slot 1 the part that starts one.  Every CTA takes
+// slot 0 first, so a partial sum is complete long before the tile's owner, in its slot 1, asks for it, and
+// no item that waits is ever ahead of the item it waits for.  Returns false for an empty slot; else the
+// tile (index among the last round's tiles) and its chunks [kc0, kc1).
+__device__ __forceinline__ bool decode_stream_item(const NhwcParams& q, int cta, int slot, int* tile, int* kc0, int* kc1) {
+  const int n = q.num_kc;
+  const int total = q.stream_tiles * n;
+  const int a = cta * q.stream_u;
+  if (cta >= q.stream_ctas || a >= total) return false;
+  const int b = a + q.stream_u < total ? a + q.stream_u : total;
+  const int t1 = a / n, r = a - t1 * n;
+  const int end1 = b < (t1 + 1) * n ? b - t1 * n : n;        // where the range leaves tile t1 (stream_u <= n)
+  if (slot == 0) {
+    if (r == 0) return false;
+    *tile = t1; *kc0 = r; *kc1 = end1;
+    return true;
+  }
+  if (r == 0) { *tile = t1; *kc0 = 0; *kc1 = end1; return true; }
+  if (b <= (t1 + 1) * n) return false;
+  *tile = t1 + 1; *kc0 = 0; *kc1 = b - (t1 + 1) * n;
+  return true;
+}
+
+// A finished partial accumulator -> this CTA's slot of the partial-sum area, laid out
+// [32-channel chunk][4-channel group][128 rows][4 floats]: the 32 lanes of a warp (32 consecutive rows)
+// write, and the tile's owner later reads, 512 contiguous bytes per instruction.
+__device__ __forceinline__ void dump_partial(int cols, int warp, int lane, uint32_t lane_base, float* slot) {
+  const int CH = cols / 2;
+  const int cbeg = ((warp - WARP_EPI0) >> 2) * CH;
+  const int row = (warp & 3) * 32 + lane;
+#pragma unroll 1
+  for (int c0 = cbeg; c0 < cbeg + CH; c0 += 32) {
+    uint32_t v[32];
+    tmem_ld32_issue(lane_base + (uint32_t)c0, v);
+    tmem_ld_wait_for(v);
+    float4* p = reinterpret_cast<float4*>(slot + (size_t)(c0 >> 5) * (TILE_M * 32)) + row;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      __stcg(p + j * TILE_M, make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                                __uint_as_float(v[4 * j + 3])));
+  }
+}
+
+// The owner's drain of a tile whose reduction other CTAs shared: accumulator + `count` partial tiles
+// (`stride` floats apart from slot0 on), then bias, ReLU and store as for any tile.
+__device__ __forceinline__ void drain_with_partials(const EpiParams& e, int cols, int warp, int lane, uint32_t lane_base,
+                                                    bool valid, int64_t base, int64_t cs, int n0, bool vec_ok,
+                                                    const float* slot0, size_t stride, int count) {
+  const int CH = cols / 2;
+  const int cbeg = ((warp - WARP_EPI0) >> 2) * CH;
+  const int row = (warp & 3) * 32 + lane;
+#pragma unroll 1
+  for (int c0 = cbeg; c0 < cbeg + CH; c0 += 32) {
+    uint32_t v[32];
+    tmem_ld32_issue(lane_base + (uint32_t)c0, v);
+    tmem_ld_wait_for(v);
+    const float* s0 = slot0 + (size_t)(c0 >> 5) * (TILE_M * 32) + row * 4;
+#pragma unroll 1
+    for (int t = 0; t < count; ++t) {
+      const float4* p = reinterpret_cast<const float4*>(s0 + (size_t)t * stride);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float4 a = __ldcg(p + j * TILE_M);
+        v[4 * j] = __float_as_uint(__uint_as_float(v[4 * j]) + a.x);
+        v[4 * j + 1] = __float_as_uint(__uint_as_float(v[4 * j + 1]) + a.y);
+        v[4 * j + 2] = __float_as_uint(__uint_as_float(v[4 * j + 2]) + a.z);
+        v[4 * j + 3] = __float_as_uint(__uint_as_float(v[4 * j + 3]) + a.w);
+      }
+    }
+    finish_chunk(e, v, c0, n0, true, valid, base, cs, vec_ok);
+  }
+}
+
 // Work item w of the overlapping-row kernel -> whole tile index and which part of its channels:
 // half = -1 the whole tile, 0 / 1 its lower / upper half.
 __device__ __forceinline__ void decode_item(const NhwcParams& q, int w, int* whole, int* half) {
@@ -283,8 +396,14 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       uint32_t ph = 0;
       bool ok = true;
       for (int w = w_first; w < q.nwork && ok; w += w_step) {
-        int whole, half;
-        decode_item(q, w, &whole, &half);
+        int whole, half, kc0, kc1;
+        if (BN >= 128 && q.stream_tiles > 0 && w >= q.n_main) {
+          if (!decode_stream_item(q, w_first, (w - q.n_main) / w_step, &whole, &kc0, &kc1)) continue;
+          whole += q.n_main; half = -1;
+        } else {
+          decode_item(q, w, &whole, &half);
+          kc0 = -1;
+        }
         const int mt = whole / per_mt, rem = whole - mt * per_mt;
         const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
         const int mti = PAIR ? 2 * mt + (int)rank : mt;
@@ -294,8 +413,10 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
         const int brow = half < 0 ? nt * BN + (int)rank * B_ROWS : nt * BN + half * (BN / 2) + (int)rank * (B_ROWS / 2);
         const uint32_t b_bytes = half < 0 ? B_BYTES : B_BYTES / 2;
         const CUtensorMap* bm = half < 0 ? &bmap : &bmap_h;
-        const int kc0 = ks * q.kc_per_split;
-        const int kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
+        if (kc0 < 0) {
+          kc0 = ks * q.kc_per_split;
+          kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
+        }
         for (int kc = kc0; kc < kc1; ++kc) {
           ok = mbar_wait(empty0 + 8 * st, ph ^ 1u, &abort_flag, q.status);
           ok = __all_sync(0xffffffffu, ok);
@@ -337,14 +458,18 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       uint32_t ph = 0, it = 0;
       bool ok = true;
       const uint32_t a_lo0 = smem_desc_lo(ring), b_lo0 = smem_desc_lo(ring + (uint32_t)A_SLOT_BYTES);
-      for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
-        int whole, half;
-        decode_item(q, w, &whole, &half);
+      for (int w = w_first; w < q.nwork && ok; w += w_step) {
+        int whole, half, kc0, kc1;
+        if (BN >= 128 && q.stream_tiles > 0 && w >= q.n_main) {
+          if (!decode_stream_item(q, w_first, (w - q.n_main) / w_step, &whole, &kc0, &kc1)) continue;
+          half = -1;
+        } else {
+          decode_item(q, w, &whole, &half);
+          const int ks = (whole % per_mt) % q.ksplit;
+          kc0 = ks * q.kc_per_split;
+          kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
+        }
         const uint32_t idesc = half < 0 ? idesc_whole : idesc_half;
-        const int rem = whole % per_mt;
-        const int ks = rem % q.ksplit;
-        const int kc0 = ks * q.kc_per_split;
-        const int kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
         const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
         ok = mbar_wait(acc_empty0 + 8 * buf, aph ^ 1u, &abort_flag, q.status);
         ok = __all_sync(0xffffffffu, ok);
@@ -380,6 +505,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
           else umma_commit(acc_full0 + 8 * buf);
         }
         __syncwarp();
+        ++it;                                    // (empty stream slots take no accumulator)
       }
     }
   } else if (warp >= WARP_EPI0) {
@@ -393,10 +519,19 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
     bool ok = true;
     uint32_t it = 0;
     TIMER_DECL;
-    for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
+    for (int w = w_first; w < q.nwork && ok; w += w_step) {
       const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
       int whole, half;
-      decode_item(q, w, &whole, &half);
+      // stream items: frag 1 = a partial sum for another CTA's tile, 2 = the start of a tile others complete
+      int frag = 0, fkc1 = 0, ftile = 0;
+      if (BN >= 128 && q.stream_tiles > 0 && w >= q.n_main) {
+        int fkc0;
+        if (!decode_stream_item(q, w_first, (w - q.n_main) / w_step, &ftile, &fkc0, &fkc1)) continue;
+        whole = ftile + q.n_main; half = -1;
+        frag = fkc0 > 0 ? 1 : (fkc1 < q.num_kc ? 2 : 0);
+      } else {
+        decode_item(q, w, &whole, &half);
+      }
       const int mt = whole / per_mt, rem = whole - mt * per_mt;
       const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
       const int mti = PAIR ? 2 * mt + (int)rank : mt;
@@ -426,7 +561,34 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(6);     // epilogue: wait for a finished accumulator
       tc_fence_after();
       const uint32_t lane_base = tmem_acc + buf * (uint32_t)BN + ((uint32_t)(lq * 32) << 16);
-      drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok, false, hoisted ? breg : nullptr);
+      if (BN < 128 || frag == 0) {
+        drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, ks == 0, vec_ok, false, hoisted ? breg : nullptr);
+      } else {
+        constexpr int PER = PAIR ? 2 : 1;                    // slots and flag words per CTA (pair) of the grid
+        constexpr size_t SLOT = (size_t)BN * TILE_M;         // floats of one CTA's partial tile
+        if (frag == 1) {
+          dump_partial(cols, warp, lane, lane_base, q.partial + (size_t)(PER * w_first + (int)rank) * SLOT);
+          __threadfence();
+          named_barrier_sync(1, EPI_WARPS * 32);             // all eight epilogue warps have stored
+          // (testing aid: with the marker in word 2 of the status block the flag stays down)
+          if (threadIdx.x == WARP_EPI0 * 32 && *reinterpret_cast<volatile uint32_t*>(q.status + 2) != kDebugDropFlag)
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(q.flags + PER * w_first + (int)rank), "r"(q.epoch) : "memory");
+        } else {
+          if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(5);
+          // the CTAs after this one whose ranges reach into the tile
+          int last = ((ftile + 1) * q.num_kc - 1) / q.stream_u;
+          if (last > q.stream_ctas - 1) last = q.stream_ctas - 1;
+          const int count = last - w_first;
+          if (lane == 0)
+            for (int t = 1; t <= count && ok; ++t) ok = wait_flag(q.flags + PER * (w_first + t) + (int)rank, q.epoch, &abort_flag, q.status);
+          ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+          __syncwarp();
+          if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(8);   // epilogue: wait for the other CTAs' partial sums
+          if (ok)
+            drain_with_partials(e, cols, warp, lane, lane_base, valid, base, cs, n0, vec_ok,
+                                q.partial + (size_t)(PER * (w_first + 1) + (int)rank) * SLOT, PER * SLOT, count);
+        }
+      }
       // the buffer may be overwritten once all four warps (of both CTAs) have read it
       tc_fence_before();
       __syncwarp();
@@ -434,6 +596,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
         if (PAIR) mbar_arrive_cluster(acc_empty_dst + 8 * buf);
         else mbar_arrive(acc_empty0 + 8 * buf);
       }
+      ++it;
     }
     if (threadIdx.x == WARP_EPI0 * 32 && blockIdx.x == 0) { TIMER_LAP(5); TIMER_FLUSH(); }
   }
@@ -482,7 +645,6 @@ conv_f16_nhwc_pair_kernel(const __grid_constant__ CUtensorMap amap, const __grid
 // fits) stay as they were.  Needs s | Wp.  Of the s column classes only those some kernel column reads
 // (min(s, Kw)) are copied; a 1x1 layer is then a plain product over full 128-position tiles.
 constexpr int MAX_SA = 6, MAX_SB = 12;
-constexpr int kTailFlagBytes = 1024;           // 256 flag words: two per tile of a short last round (at most 37 of them)
 constexpr int MAX_KW = 64;                     // kernel widths the shifted-view kernel takes
 constexpr int WARP_BLOAD = 2 + EPI_WARPS;      // the filter-copy warp of this kernel
 constexpr int SHIFT_THREADS = (NUM_WARPS + 1) * 32;
@@ -520,30 +682,6 @@ __device__ __forceinline__ void item_blocks(const ShiftViewParams& q, int ks, in
   const int first = ((part >= 0 && q.tail_k) ? part : ks) * per;
   *kb0 = first;
   *kb1 = first + per < q.nkb2 ? first + per : q.nkb2;
-}
-
-// Bounded wait for a flag word to hold `value` (written with release semantics by another CTA).
-__device__ __noinline__ bool wait_flag(const uint32_t* flag, uint32_t value, volatile uint32_t* abort_flag, uint32_t* status) {
-  uint32_t limit = *reinterpret_cast<volatile uint32_t*>(status + 1);
-  if (limit == 0u) limit = SPIN_LIMIT;
-  const uint64_t t0 = global_timer_ns();
-  for (uint32_t i = 0; i < limit; ++i) {
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-    if (v == value) return true;
-    if ((i & 255u) == 255u) {
-      if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > SPIN_TIME_NS) break;
-    }
-    __nanosleep(64);
-  }
-  *abort_flag = 1u;
-  atomicExch(status, 1u);
-  return false;
-}
-
-__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 // Work item w of the shifted-view kernel -> whole item index and which part of its channels
@@ -1326,6 +1464,14 @@ cudaError_t report(cudaError_t e, const char* what) {
   return e;
 }
 
+// A value no earlier launch of this process used (flag words are compared with it and need no clearing).
+uint32_t next_epoch() {
+  static std::atomic<uint32_t> launches{0};
+  uint32_t e = ++launches;
+  if (e == 0) e = ++launches;                   // 0 is what cleared flags hold
+  return e;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -1341,6 +1487,46 @@ EncodeTiledFn get_encode_fn() {
     return nullptr;
   fn = reinterpret_cast<EncodeTiledFn>(p);
   return fn;
+}
+
+// Overlapping-row kernel, a short last round of tiles: the reductions of its `tiles` tiles are laid end to
+// end and cut into equal runs of `u` chunks (of ksub k-blocks), one per CTA (pair) for the first `ctas` of
+// them.  The CTA that holds a tile's first chunk adds the others' partial sums (scratch area, one flag per
+// CTA) and stores the tile, so bias, ReLU and the rounding store work as for whole tiles.  At most eight
+// runs per tile (their sums are added one after another) and no run shorter than eight k-blocks.
+// tiles == 0: not worth it; `rounds` is the estimated time of the launch in tile times.
+struct RunPlan {
+  int tiles, u, ctas;
+  double rounds;
+};
+
+RunPlan plan_runs(int64_t nwork, int slots, int num_kc, int ksub, int bn) {
+  RunPlan r{};
+  bool on = bn >= 128;                                      // 64-channel tiles: items too short to share
+  if (const char* v = debug_getenv("IM2WIN_NHWC_STREAM")) on = on && v[0] != '0';
+  const int tail = (int)(nwork % slots);
+  // what the round takes otherwise: a whole tile, or about 0.55 of one as half tiles
+  const double alt = tail == 0 ? 0.0 : ((bn >= 128 && 2 * tail <= slots) ? 0.55 : 1.0);
+  r.rounds = (double)(nwork / slots) + alt;
+  if (!on || tail == 0) return r;
+  const int min_run = (num_kc + 7) / 8 > 8 / ksub ? (num_kc + 7) / 8 : 8 / ksub;
+  const int64_t total = (int64_t)tail * num_kc;
+  int S = slots;
+  if (total / S < min_run) S = (int)(total / min_run);
+  if (S <= tail) return r;
+  const int U = (int)((total + S - 1) / S);
+  S = (int)((total + U - 1) / U);
+  // Worth it when the run, plus the two drains that now follow one another at the end (a partial sum
+  // written, then read by the tile's owner: measured about 24 k-blocks' time together), is clearly
+  // shorter.  (Measured on 3x3 layers of 256 and 512 channels, 36 and 72 k-blocks per tile: 3 to 8 us
+  // slower than half tiles; on 7x7 and 11x11 layers of 256 channels with a ReLU and a binary16 store:
+  // 281 -> 258 us and 717 -> 626 us.)
+  double margin = 24.0 / ((double)num_kc * ksub) + 0.05;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_STREAM_MARGIN")) margin = atof(v);
+  if (U >= num_kc || (double)U / num_kc + margin >= alt) return r;
+  r.tiles = tail; r.u = U; r.ctas = S;
+  r.rounds = (double)(nwork / slots) + (double)U / num_kc + margin;
+  return r;
 }
 
 template <int BN, bool PAIR, int KSUB>
@@ -1403,10 +1589,20 @@ cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, con
     if (e != cudaSuccess) return e;
     attr_done[dev] = true;
   }
-  // The last round of tiles: when it would fill at most half of the CTAs (or pairs), each of its tiles
+  // The last round of tiles, when it is short, handed out as runs of its reduction (plan_runs)
+  q.stream_tiles = 0;
+  if (BN >= 128 && q.partial != nullptr && q.ksplit == 1 && q.tail_halves) {
+    const RunPlan rp = plan_runs(q.nwork, slots, q.num_kc, KSUB, BN);
+    if (rp.tiles > 0) {
+      q.stream_tiles = rp.tiles; q.stream_u = rp.u; q.stream_ctas = rp.ctas;
+      q.n_main = q.nwork - rp.tiles;
+      q.nwork = q.n_main + 2 * slots;            // two stream items per CTA (either may be empty)
+    }
+  }
+  // Else, when that round would fill at most half of the CTAs (or pairs), each of its tiles
   // is handed out as two items of half the channels, so the round takes half as long.  (Not with a K
   // split, whose parts already are the finer grain.)
-  if (BN >= 128 && q.ksplit == 1 && q.tail_halves) {
+  if (q.stream_tiles == 0 && BN >= 128 && q.ksplit == 1 && q.tail_halves) {
     const int tail = q.nwork % slots;
     if (tail > 0 && 2 * tail <= slots) {
       q.n_main = q.nwork - tail;
@@ -1669,13 +1865,8 @@ cudaError_t launch_shift_view(const uint16_t* window, const uint16_t* fp, void* 
   q.nkb2 = sp.nkb2; q.nks_last = sp.nks_last; q.bu = sp.bu;
   q.ksplit = split ? plan.ksplit : 1;
   q.ntn = plan.ntn;
-  {
-    static std::atomic<uint32_t> launches{0};
-    uint32_t e = ++launches;
-    if (e == 0) e = ++launches;                 // 0 is what cleared flags hold
-    q.epoch = e;
-    q.flags = flags;
-  }
+  q.epoch = next_epoch();
+  q.flags = flags;
   if (const char* v = debug_getenv("IM2WIN_NHWC_BU")) { const int bu = atoi(v); if (bu >= 1 && bu <= 8) { q.bu = bu; q.bu_forced = 1; } }
   if (plan.pair) {
     if (plan.bn == 256) return launch_shift_variant<256, true>(amap, bmap, bmap_h, bmap_q, q, plan, sp, stream);
@@ -1741,7 +1932,11 @@ NhwcPlan plan_nhwc(const Geometry& g) {
   // status block, packed filter, then kTailFlagBytes of flag words (hand-off between the CTAs that share
   // a tile of a short last round; cleared by the filter pack)
   p.flags_off = ((size_t)kStatusBytes + (size_t)g.Co * p.K * 2 + 255) / 256 * 256;
-  p.scratch_bytes = p.flags_off + kTailFlagBytes;
+  // ... and, for layers of few rounds of tiles, the partial-sum area of a last round handed out by
+  // reduction length
+  p.partial_off = p.flags_off + kTailFlagBytes;
+  p.partial_bytes = tiles < 8 * slots ? kPartialBytes : 0;
+  p.scratch_bytes = p.partial_off + p.partial_bytes;
   p.eligible = true;
   return p;
 }
@@ -1837,6 +2032,7 @@ struct NhwcChoice {
   NhwcPlan plan;
   ShiftViewPlan sp;
   bool use_shift, split;
+  bool runs;                 // overlapping-row kernel: the last round of tiles goes out as runs of its reduction
 };
 
 NhwcChoice choose_nhwc(const Geometry& g, const EpilogueArgs& epi) {
@@ -1905,6 +2101,21 @@ NhwcChoice choose_nhwc(const Geometry& g, const EpilogueArgs& epi) {
     const double r_split = (double)((it_s * plan.ksplit + slots - 1) / slots) / plan.ksplit + 0.1;
     if (r_tail <= r_split) { split = false; plan.ksplit = 1; }
   }
+  if (!use_shift && plan.partial_bytes > 0) {
+    // Overlapping-row kernel: a short last round handed out as runs of its reduction (plan_runs), against
+    // a K split of every tile (cleared output, atomics; estimated as in the comparison above).  Measured:
+    // 7x7 on 256 channels 250 against 261 us, 11x11 620 against 600.
+    bool tail = true;
+    if (const char* v = debug_getenv("IM2WIN_NHWC_TAIL")) tail = v[0] != '0';
+    const int slots = plan.pair ? 74 : 148;
+    const int64_t it_o = (plan.pair ? (plan.ntm + 1) / 2 : plan.ntm) * plan.ntn;
+    const RunPlan rp = tail ? plan_runs(it_o, slots, plan.num_kb, 1, plan.bn) : RunPlan{};
+    if (split && rp.tiles > 0) {
+      const double r_split = (double)((it_o * plan.ksplit + slots - 1) / slots) / plan.ksplit + 0.1;
+      if (rp.rounds < r_split - 0.03) { split = false; plan.ksplit = 1; }
+    }
+    c.runs = !split && rp.tiles > 0;
+  }
   c.use_shift = use_shift;
   c.split = split;
   return c;
@@ -1916,7 +2127,7 @@ const char* nhwc_kernel_name(const Geometry& g, const EpilogueArgs& epi) {
   const NhwcChoice c = choose_nhwc(g, epi);
   if (!c.plan.eligible) return "none";
   if (c.use_shift) return c.split ? "f16-nhwc-shift+ksplit" : "f16-nhwc-shift";
-  return c.split ? "f16-nhwc-overlap+ksplit" : "f16-nhwc-overlap";
+  return c.split ? "f16-nhwc-overlap+ksplit" : (c.runs ? "f16-nhwc-overlap+runs" : "f16-nhwc-overlap");
 }
 
 cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch, const Geometry& g,
@@ -1980,6 +2191,9 @@ cudaError_t launch_conv_f16_nhwc(const uint16_t* window, void* y, void* scratch,
   if (const char* v = debug_getenv("IM2WIN_NHWC_KSUB")) ksub = atoi(v) == 1 ? 1 : 2;
   q.tail_halves = 1;
   if (const char* v = debug_getenv("IM2WIN_NHWC_TAIL")) q.tail_halves = v[0] != '0';
+  q.flags = reinterpret_cast<uint32_t*>(base + plan.flags_off);
+  q.partial = plan.partial_bytes > 0 ? reinterpret_cast<float*>(base + plan.partial_off) : nullptr;
+  q.epoch = next_epoch();
   if (ksub == 1) return launch_ksub<1>(amap, bmap, bmap_h, q, plan, stream);
   return launch_ksub<2>(amap, bmap, bmap_h, q, plan, stream);
 }

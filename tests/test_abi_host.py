@@ -118,14 +118,17 @@ def test_null_and_misaligned_pointers_rejected_before_launch():
 def test_nhwc_kernel_name_query():
     """Host-only: which NHWC kernel a layer takes (reports and tests use it).  Wide-kernel stride-1
     layers take the shifted views, stride 2 with a 3-wide kernel the overlapping rows; the longest
-    reductions split every tile's K unless the epilogue forbids partial sums."""
+    reductions split every tile's K or, with any epilogue, share the tiles of a short last round by
+    runs of the reduction; short reductions (3x3) do neither."""
     import torch
     name = binding.im2win_nhwc_kernel_name
     assert name(workloads.LAYERS["cfg2"].dims()) == "f16-nhwc-shift"
     assert name(workloads.LAYERS["cfg5k5"].dims()) == "f16-nhwc-shift"
     assert name(workloads.LAYERS["cfg4c"].dims()) == "f16-nhwc-overlap"
-    assert name(workloads.LAYERS["cfg5k11"].dims()) == "f16-nhwc-overlap+ksplit"
     relu16 = binding.make_epilogue(None, True, torch.float16, binding.NCHW)
-    assert name(workloads.LAYERS["cfg5k11"].dims(), relu16) == "f16-nhwc-overlap"
+    assert name(workloads.LAYERS["cfg5k11"].dims()) in ("f16-nhwc-overlap+ksplit", "f16-nhwc-overlap+runs")
+    assert name(workloads.LAYERS["cfg5k11"].dims(), relu16) == "f16-nhwc-overlap+runs"
+    assert name(workloads.LAYERS["cfg5k7"].dims(), relu16) == "f16-nhwc-overlap+runs"
+    assert name(workloads.LAYERS["cfg4a"].dims(), relu16) == "f16-nhwc-overlap"
     huge = dict(workloads.LAYERS["cfg2"].dims(), C=40000)       # beyond the NHWC transform's staging
     assert name(huge) == "none"

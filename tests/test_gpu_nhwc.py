@@ -216,6 +216,57 @@ def test_conv_nhwc_flag_wait_is_bounded(monkeypatch):
     assert np.array_equal(y.cpu().double().numpy().reshape(r["yi"].shape), r["yi"])
 
 
+@pytest.mark.parametrize("tail", ["runs", "halves", "off"])
+def test_conv_nhwc_overlap_short_last_round(tail, monkeypatch):
+    """The same layer through the overlapping-row kernel without a K split of every tile: 78 tile items on
+    74 CTA pairs.  The four tiles of the last round are handed out as runs of their reduction (the CTA that
+    starts a tile adds the other CTAs' partial sums from the scratch area once their flags are up, then
+    applies bias / ReLU and stores), as half tiles, or whole.  Exact on integer-valued inputs, also with a
+    bias and a ReLU (which the runs must pass through unchanged) and on three calls on the same scratch;
+    within tolerance on the seeded inputs."""
+    monkeypatch.setenv("IM2WIN_NHWC_KERNEL", "overlap")
+    monkeypatch.setenv("IM2WIN_NHWC_KSPLIT", "1")
+    if tail == "off":
+        monkeypatch.setenv("IM2WIN_NHWC_TAIL", "0")
+    if tail == "halves":
+        monkeypatch.setenv("IM2WIN_NHWC_STREAM", "0")
+    dims = _SHORT_LAST_ROUND.dims()
+    r = _short_last_round_reference()
+    assert np.array_equal(gpu_conv_nhwc(r["xi"], r["fi"], dims), r["yi"])
+    assert np.array_equal(gpu_conv_nhwc(r["xi"], r["fi"], dims, packed=True, repeat=3), r["yi"])
+    b = (np.arange(_SHORT_LAST_ROUND.Co, dtype=np.float32) % 7) - 3.0
+    want = np.maximum(r["yi"] + b[None, :, None, None], 0)
+    assert np.array_equal(gpu_conv_nhwc(r["xi"], r["fi"], dims, bias=b, relu=True), want)
+    assert np.array_equal(gpu_conv_nhwc(r["xi"], r["fi"], dims, bias=b, relu=True, y_nhwc=True),
+                          want.transpose(0, 2, 3, 1))
+    check_conv(gpu_conv_nhwc(r["x"], r["f"], dims), r["y_pre"], r["a"], "f16", _SHORT_LAST_ROUND.name)
+
+
+def test_conv_nhwc_overlap_flag_wait_is_bounded(monkeypatch):
+    """The CTA that starts a tile of a last round handed out as runs waits for the flags of the CTAs that
+    hold the rest of its reduction.  With the poll limit lowered and the flags kept down those waits run
+    out: the kernel returns, the status reads IM2WIN_ERR_TIMEOUT, and the next call is exact."""
+    monkeypatch.setenv("IM2WIN_NHWC_KERNEL", "overlap")
+    monkeypatch.setenv("IM2WIN_NHWC_KSPLIT", "1")
+    dims = _SHORT_LAST_ROUND.dims()
+    r = _short_last_round_reference()
+    xd, fd = r["xi"].half().cuda(), r["fi"].half().cuda()
+    window, scratch, y = binding.alloc_nhwc_buffers(dims)
+    binding.im2win_transform_nhwc(xd, binding.NCHW, window, dims)
+    binding.im2win_pack_filter_nhwc(fd, scratch, dims)
+    torch.cuda.synchronize()
+    words = scratch[:256].view(torch.int32)
+    words[1] = 4096
+    words[2] = 0x0d0a11ff
+    binding.im2win_conv_packed_nhwc(window, y, scratch, dims)
+    with pytest.raises(binding.Im2winError) as err:
+        binding.im2win_check_status(scratch)
+    assert err.value.code == 7
+    binding.im2win_conv_f16_nhwc(window, fd, y, scratch, dims)
+    binding.im2win_check_status(scratch)
+    assert np.array_equal(y.cpu().double().numpy().reshape(r["yi"].shape), r["yi"])
+
+
 def test_conv_nhwc_exact_with_integer_bias_relu_and_half_store():
     """Small integers all the way: bias, ReLU and the binary16 store must reproduce the oracle exactly."""
     layer = SMALL[2]
@@ -272,6 +323,34 @@ def test_nhwc_full_size_whole_tensors(layer):
         n1 = min(layer.N, n0 + 16)
         yi, ai = oracle.conv_im2win(xo[n0:n1], fo, dict(dims, N=n1 - n0))
         check_conv(y[n0:n1], yi, ai, "f16", f"{layer.name} images {n0}..{n1 - 1}")
+
+
+@pytest.mark.parametrize("name", ["cfg5k7", "cfg5k11"])
+def test_nhwc_full_size_last_round_as_runs_with_fused_epilogue(name):
+    """The two longest reductions at benchmark size with bias, ReLU and the binary16 store: 224 tiles on 74
+    CTA pairs, the two tiles of the last round shared between CTAs as runs of the reduction (partial sums
+    through the scratch area, the epilogue applied once by the CTA that starts the tile).  16 384 sampled
+    outputs from Eq. 1 with the epilogue applied in binary64, and the first and last image whole through
+    the oracle's im2win route and epilogue."""
+    layer = workloads.LAYERS[name]
+    dims = layer.dims()
+    relu16 = binding.make_epilogue(None, True, torch.float16, binding.NCHW)
+    assert binding.im2win_nhwc_kernel_name(dims, relu16) == "f16-nhwc-overlap+runs"
+    x, f = workloads.make_inputs(layer)
+    ho, wo = oracle.out_dims(dims)
+    b = np.linspace(-0.5, 0.5, layer.Co).astype(np.float32)
+    y = gpu_conv_nhwc(x, f, dims, bias=b, relu=True, out16=True)
+    xo, fo = oracle_inputs(x, f, "f16")
+    total = layer.N * layer.Co * ho * wo
+    idx = np.concatenate([np.random.default_rng(layer.seed + 5).integers(0, total, 16384), [0, total - 1]])
+    yr, ar = oracle.conv_direct_points(xo, fo, dims, idx)
+    co = (idx // (ho * wo)) % layer.Co
+    check_fused(y.reshape(-1)[idx], np.maximum(yr + b[co].astype(np.float64), 0.0), ar + np.abs(b[co]), True, name)
+    for n in (0, layer.N - 1):
+        d1 = dict(dims, N=1)
+        yi, ai = oracle.conv_im2win(xo[n:n + 1], fo, d1)
+        yi, ai = oracle.epilogue(yi, ai, d1, bias=b, relu=True, out16=False)
+        check_fused(y[n:n + 1], yi, ai, True, f"{name} image {n}")
 
 
 @pytest.mark.parametrize("name,kernel", [("cfg2", "overlap"), ("cfg4a", "shift"), ("cfg4b", "shift"), ("cfg4c", "shift"),
