@@ -59,7 +59,7 @@ im2win_status derive_geometry(const im2win_shape* s, Geometry* g) {
 im2win_status scratch_layout(const Geometry& g, im2win_dtype dtype, ScratchLayout* l) {
   if (dtype == IM2WIN_F32) {
     l->Kp = round_up(g.K, plan_f32(g).bk);
-    l->Co_pad = g.Co > 64 ? round_up(g.Co, 128) : 64;
+    l->Co_pad = round_up(g.Co, plan_f32(g).bn);
   } else if (dtype == IM2WIN_F16) {
     l->Kp = round_up(g.K, kF16KBlock);
     l->Co_pad = g.Co;

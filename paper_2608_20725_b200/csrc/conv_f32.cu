@@ -57,14 +57,22 @@ __device__ __forceinline__ void split_position(int64_t p, const ConvF32Params& q
   }
 }
 
+// Threads along the channel direction of a BM x BN tile: every thread holds 8 positions x 8 channels, or,
+// for the 96-channel tile (layers of 96, 192, ... output channels, which 64- and 128-channel tiles would
+// pad by a third), 8 x 6: four channels from the tile's first 64 and two from its last 32.
+__host__ __device__ constexpr int f32_tn(int bn) { return bn == 96 ? 16 : bn / 8; }
+
 // BK: the k-block, 16 or 32 (see plan_f32).
 template <int BM, int BN, int BK>
-__global__ void __launch_bounds__((BM / 8) * (BN / 8), ((BM / 8) * (BN / 8) == 256 ? 2 : 3))
+__global__ void __launch_bounds__((BM / 8) * f32_tn(BN), ((BM / 8) * f32_tn(BN) == 256 ? 2 : 3))
 conv_f32_kernel(ConvF32Params q) {
-  constexpr int THREADS = (BM / 8) * (BN / 8);
+  constexpr int THREADS = (BM / 8) * f32_tn(BN);
+  constexpr int NPT = BN / f32_tn(BN);                     // channels per thread: 8 or 6
+  constexpr int NP2 = NPT / 2;                             // ... as pairs
+  constexpr int LO = BN == 96 ? 64 : BN / 2;               // channels of the first group (four per thread)
   constexpr int A_PER_THREAD = BK * BM / THREADS;         // scalar gathers per k-block
   constexpr int A_KK_STEP = THREADS / BM;                 // 2 (256 threads) or 1 (128 threads)
-  constexpr int B_VEC_PER_THREAD = BK * BN / 4 / THREADS; // float4 loads per k-block
+  constexpr int B_VEC_PER_THREAD = (BK * BN / 4 + THREADS - 1) / THREADS; // float4 loads per k-block
   static_assert(THREADS % BM == 0 && A_PER_THREAD * A_KK_STEP == BK, "loader mapping");
 
   constexpr int STAGES = 3;          // shared-memory ring filled by asynchronous copies
@@ -118,6 +126,7 @@ conv_f32_kernel(ConvF32Params q) {
 #pragma unroll
     for (int i = 0; i < B_VEC_PER_THREAD; ++i) {
       const int e = tid + i * THREADS;       // float4 index inside the BK x BN tile
+      if ((BK * BN / 4) % THREADS != 0 && e >= BK * BN / 4) break;
       const int kk = e / (BN / 4);
       const int nn = (e - kk * (BN / 4)) * 4;
       const float* src = q.fk + (int64_t)(k0 + kk) * q.Co_pad + n0 + nn;
@@ -127,11 +136,11 @@ conv_f32_kernel(ConvF32Params q) {
     if (more) load_offsets(kb + 1);
   };
 
-  unsigned long long acc2[8][4];     // acc2[i][jp] = (acc[i][2jp], acc[i][2jp+1])
+  unsigned long long acc2[8][NP2];   // acc2[i][jp] = (acc[i][2jp], acc[i][2jp+1])
 #pragma unroll
   for (int i = 0; i < 8; ++i)
 #pragma unroll
-    for (int jp = 0; jp < 4; ++jp) acc2[i][jp] = 0ull;
+    for (int jp = 0; jp < NP2; ++jp) acc2[i][jp] = 0ull;
 
   const int nkb = q.Kp / BK;
   load_offsets(0);
@@ -157,24 +166,31 @@ conv_f32_kernel(ConvF32Params q) {
       const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][kk][tm * 4]);
       const float4 a1 = *reinterpret_cast<const float4*>(&As[buf][kk][BM / 2 + tm * 4]);
       const ulonglong2 b0 = *reinterpret_cast<const ulonglong2*>(&Bs[buf][kk][tn * 4]);
-      const ulonglong2 b1 = *reinterpret_cast<const ulonglong2*>(&Bs[buf][kk][BN / 2 + tn * 4]);
+      unsigned long long b[4];
+      b[0] = b0.x; b[1] = b0.y;
+      if (NPT == 8) {
+        const ulonglong2 b1 = *reinterpret_cast<const ulonglong2*>(&Bs[buf][kk][LO + tn * 4]);
+        b[2] = b1.x; b[3] = b1.y;
+      } else {
+        b[2] = *reinterpret_cast<const unsigned long long*>(&Bs[buf][kk][LO + tn * 2]);
+        b[3] = 0ull;
+      }
       const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-      const unsigned long long b[4] = {b0.x, b0.y, b1.x, b1.y};
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const unsigned long long ad = dup2(a[i]);
 #pragma unroll
-        for (int jp = 0; jp < 4; ++jp) ffma2(acc2[i][jp], ad, b[jp]);
+        for (int jp = 0; jp < NP2; ++jp) ffma2(acc2[i][jp], ad, b[jp]);
       }
     }
     if (++buf == STAGES) buf = 0;
   }
 
-  float acc[8][8];
+  float acc[8][NPT];
 #pragma unroll
   for (int i = 0; i < 8; ++i)
 #pragma unroll
-    for (int jp = 0; jp < 4; ++jp) {
+    for (int jp = 0; jp < NP2; ++jp) {
       const float2 v = unpack2(acc2[i][jp]);
       acc[i][2 * jp] = v.x;
       acc[i][2 * jp + 1] = v.y;
@@ -199,8 +215,8 @@ conv_f32_kernel(ConvF32Params q) {
       while (rr[i] >= q.HoWo) { rr[i] -= q.HoWo; ++nn[i]; }
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int co = n0 + (j / 4) * (BN / 2) + tn * 4 + (j % 4);
+    for (int j = 0; j < NPT; ++j) {
+      const int co = j < 4 ? n0 + tn * 4 + j : n0 + LO + tn * (NPT - 4) + (j - 4);
       if (co >= q.Co) continue;
       if (vec_ok) {
         float4 v = make_float4(acc[hm * 4 + 0][j], acc[hm * 4 + 1][j], acc[hm * 4 + 2][j], acc[hm * 4 + 3][j]);
@@ -225,8 +241,10 @@ conv_f32_kernel(ConvF32Params q) {
 F32Plan plan_f32(const Geometry& g) {
   F32Plan p;
   const bool wide = g.Co > 64;
-  p.bn = wide ? 128 : 64;
-  const int64_t cot = wide ? (g.Co + 127) / 128 : 1;
+  // 96-channel tiles where they pad the output channels less than 128-channel tiles do (96, 192, 288, ...)
+  const bool bn96 = wide && (g.Co + 95) / 96 * 96 < (g.Co + 127) / 128 * 128;
+  p.bn = wide ? (bn96 ? 96 : 128) : 64;
+  const int64_t cot = wide ? (g.Co + p.bn - 1) / p.bn : 1;
   auto waves_cost = [&](int bm) {
     const int64_t tiles = (g.P + bm - 1) / bm * cot;
     return (double)((tiles + 147) / 148) * bm;
@@ -259,11 +277,14 @@ cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, 
   if (l.Kp % p.bk != 0) return cudaErrorInvalidValue;       // the filter was packed for another k-block
   const int64_t cot = l.Co_pad / p.bn;
   dim3 grid((unsigned)((g.P + p.bm - 1) / p.bm), (unsigned)cot);
-  const int threads = (p.bm / 8) * (p.bn / 8);
+  const int threads = (p.bm / 8) * f32_tn(p.bn);
   const size_t smem = (size_t)3 * p.bk * (p.bm + p.bn) * 4;
   void (*kernel)(ConvF32Params);
   int which;
-  if (p.bn == 128) {
+  if (p.bn == 96) {
+    if (p.bm == 64) { kernel = p.bk == 32 ? conv_f32_kernel<64, 96, 32> : conv_f32_kernel<64, 96, 16>; which = p.bk == 32 ? 5 : 6; }
+    else { kernel = conv_f32_kernel<128, 96, 16>; which = 7; }
+  } else if (p.bn == 128) {
     if (p.bm == 64) { kernel = p.bk == 32 ? conv_f32_kernel<64, 128, 32> : conv_f32_kernel<64, 128, 16>; which = p.bk == 32 ? 0 : 1; }
     else { kernel = conv_f32_kernel<128, 128, 16>; which = 2; }
   } else {
@@ -272,7 +293,7 @@ cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, 
   }
   if (smem > 48 * 1024) {
     // per device and tile shape, once: the opt-in to more than 48 KB of dynamic shared memory
-    static bool attr_done[64][5] = {};
+    static bool attr_done[64][8] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!attr_done[dev][which]) {

@@ -128,12 +128,14 @@ def test_conv_exact_on_integer_inputs(layer, precision):
     assert np.array_equal(y.astype(np.float64), yr)
 
 
-@pytest.mark.parametrize("layer", [SMALL[1], SMALL[2], L("wide_co", 3, 20, 11, 13, 150, 3, 3, 1, 1, 47)], ids=lambda l: l.name)
+@pytest.mark.parametrize("layer", [SMALL[1], SMALL[2], L("wide_co", 3, 20, 11, 13, 150, 3, 3, 1, 1, 47),
+                                   L("co96", 2, 12, 30, 29, 96, 5, 5, 2, 2, 48), L("co200", 1, 9, 14, 15, 200, 3, 3, 1, 1, 49)],
+                         ids=lambda l: l.name)
 @pytest.mark.parametrize("bm,bk", [("64", "16"), ("64", "32"), ("128", "16")])
 def test_conv_f32_both_tile_heights(layer, bm, bk, monkeypatch):
-    """The fp32 kernel's 64- and 128-position tiles (the library picks by grid size), on 64- and
-    128-channel tiles, and the 64 x 128 tile with both k-blocks: exact on integer-valued inputs,
-    within tolerance on the seeded ones."""
+    """The fp32 kernel's 64- and 128-position tiles (the library picks by grid size), on 64-, 96- and
+    128-channel tiles (96 where that pads the output channels least: 96 and 150 here, not 200), and the
+    64-position tiles with both k-blocks: exact on integer-valued inputs, within tolerance on the seeded ones."""
     monkeypatch.setenv("IM2WIN_F32_BM", bm)
     monkeypatch.setenv("IM2WIN_F32_BK", bk)
     dims = layer.dims()
