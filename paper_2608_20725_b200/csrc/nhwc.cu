@@ -2103,16 +2103,18 @@ NhwcChoice choose_nhwc(const Geometry& g, const EpilogueArgs& epi) {
   }
   if (!use_shift && plan.partial_bytes > 0) {
     // Overlapping-row kernel: a short last round handed out as runs of its reduction (plan_runs), against
-    // a K split of every tile (cleared output, atomics; estimated as in the comparison above).  Measured:
-    // 7x7 on 256 channels 250 against 261 us, 11x11 620 against 600.
+    // a K split of every tile (cleared output, atomics).  Measured: 7x7 on 256 channels 250 against 261 us,
+    // 11x11 611-617 against 600.
     bool tail = true;
     if (const char* v = debug_getenv("IM2WIN_NHWC_TAIL")) tail = v[0] != '0';
     const int slots = plan.pair ? 74 : 148;
     const int64_t it_o = (plan.pair ? (plan.ntm + 1) / 2 : plan.ntm) * plan.ntn;
     const RunPlan rp = tail ? plan_runs(it_o, slots, plan.num_kb, 1, plan.bn) : RunPlan{};
     if (split && rp.tiles > 0) {
-      const double r_split = (double)((it_o * plan.ksplit + slots - 1) / slots) / plan.ksplit + 0.1;
-      if (rp.rounds < r_split - 0.03) { split = false; plan.ksplit = 1; }
+      // (the split's parts fill the CTAs almost evenly; its cost is the cleared output and the atomics, a
+      // fixed time that weighs less the longer the tiles are: about 65 k-blocks' worth, measured)
+      const double r_split = (double)it_o / slots + 65.0 / plan.num_kb;
+      if (rp.rounds < r_split) { split = false; plan.ksplit = 1; }
     }
     c.runs = !split && rp.tiles > 0;
   }

@@ -126,7 +126,8 @@ def test_nhwc_kernel_name_query():
     assert name(workloads.LAYERS["cfg5k5"].dims()) == "f16-nhwc-shift"
     assert name(workloads.LAYERS["cfg4c"].dims()) == "f16-nhwc-overlap"
     relu16 = binding.make_epilogue(None, True, torch.float16, binding.NCHW)
-    assert name(workloads.LAYERS["cfg5k11"].dims()) in ("f16-nhwc-overlap+ksplit", "f16-nhwc-overlap+runs")
+    assert name(workloads.LAYERS["cfg5k11"].dims()) == "f16-nhwc-overlap+ksplit"
+    assert name(workloads.LAYERS["cfg5k7"].dims()) == "f16-nhwc-overlap+runs"
     assert name(workloads.LAYERS["cfg5k11"].dims(), relu16) == "f16-nhwc-overlap+runs"
     assert name(workloads.LAYERS["cfg5k7"].dims(), relu16) == "f16-nhwc-overlap+runs"
     assert name(workloads.LAYERS["cfg4a"].dims(), relu16) == "f16-nhwc-overlap"
