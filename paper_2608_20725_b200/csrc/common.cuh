@@ -112,6 +112,7 @@ struct EpilogueArgs {
 // Tile shape of the fp32 kernel for a layer (see conv_f32.cu); the packed filter's K is padded to bk.
 struct F32Plan {
   int32_t bm, bn, bk;
+  bool klanes;             // the window operand is gathered with k along the lanes of a warp
 };
 F32Plan plan_f32(const Geometry& g);
 

@@ -62,8 +62,14 @@ __device__ __forceinline__ void split_position(int64_t p, const ConvF32Params& q
 // pad by a third), 8 x 6: four channels from the tile's first 64 and two from its last 32.
 __host__ __device__ constexpr int f32_tn(int bn) { return bn == 96 ? 16 : bn / 8; }
 
-// BK: the k-block, 16 or 32 (see plan_f32).
-template <int BM, int BN, int BK>
+// BK: the k-block, 16 or 32 (see plan_f32).  KLANES: which way the window operand is gathered.  false: the
+// lanes of a warp are 32 consecutive positions at one k (their elements lie s*Kh apart).  true: the lanes
+// are 8 consecutive k (contiguous in the im2win tensor within a channel) of 4 consecutive positions, so a
+// copy instruction touches about four 32-byte sectors instead of one per lane; shared-memory rows are
+// BM + 4 words apart so that the 32 lanes still write 32 different banks.  Measured: with windows 176
+// bytes apart (11x11, stride 4) 10 % faster; 3 % SLOWER where windows lie 12-56 bytes apart (the sectors
+// of neighbouring positions overlap anyway, and every thread then tracks several positions).
+template <int BM, int BN, int BK, bool KLANES>
 __global__ void __launch_bounds__((BM / 8) * f32_tn(BN), ((BM / 8) * f32_tn(BN) == 256 ? 2 : 3))
 conv_f32_kernel(ConvF32Params q) {
   constexpr int THREADS = (BM / 8) * f32_tn(BN);
@@ -72,13 +78,17 @@ conv_f32_kernel(ConvF32Params q) {
   constexpr int LO = BN == 96 ? 64 : BN / 2;               // channels of the first group (four per thread)
   constexpr int A_PER_THREAD = BK * BM / THREADS;         // scalar gathers per k-block
   constexpr int A_KK_STEP = THREADS / BM;                 // 2 (256 threads) or 1 (128 threads)
+  constexpr int KG = BK / 8;                              // KLANES: groups of eight consecutive k per k-block,
+  constexpr int NPOS = A_PER_THREAD / KG;                 // positions per loader thread,
+  constexpr int APITCH = KLANES ? BM + 4 : BM;            // row pitch of the window operand in shared memory
+  static_assert(!KLANES || (NPOS >= 1 && (THREADS / 32) * NPOS * 4 == BM), "loader mapping (k along lanes)");
   constexpr int B_VEC_PER_THREAD = (BK * BN / 4 + THREADS - 1) / THREADS; // float4 loads per k-block
   static_assert(THREADS % BM == 0 && A_PER_THREAD * A_KK_STEP == BK, "loader mapping");
 
   constexpr int STAGES = 3;          // shared-memory ring filled by asynchronous copies
   extern __shared__ __align__(16) unsigned char smem_f32[];
-  float (*As)[BK][BM] = reinterpret_cast<float (*)[BK][BM]>(smem_f32);
-  float (*Bs)[BK][BN] = reinterpret_cast<float (*)[BK][BN]>(smem_f32 + sizeof(float) * STAGES * BK * BM);
+  float (*As)[BK][APITCH] = reinterpret_cast<float (*)[BK][APITCH]>(smem_f32);
+  float (*Bs)[BK][BN] = reinterpret_cast<float (*)[BK][BN]>(smem_f32 + sizeof(float) * STAGES * BK * APITCH);
 
   const int tid = threadIdx.x;
   const int tm = tid % (BM / 8);     // position direction: fastest across lanes
@@ -86,29 +96,38 @@ conv_f32_kernel(ConvF32Params q) {
   const int64_t m0 = (int64_t)blockIdx.x * BM;
   const int n0 = blockIdx.y * BN;
 
-  // Loader role: one fixed position (row of A) per thread.
-  const int lm = tid % BM;
+  // Loader role: one fixed position (row of A) per thread, or (KLANES) NPOS positions lm + 4 j and
+  // the k's kq + 8 g of every k-block.
+  constexpr int NBASE = KLANES ? NPOS : 1;
+  constexpr int NOFF = KLANES ? KG : A_PER_THREAD;
+  const int kq = tid & 7;
+  const int lm = KLANES ? (tid >> 5) * (NPOS * 4) + ((tid >> 3) & 3) : tid % BM;
   const int lkk0 = tid / BM;
-  const int64_t lp = m0 + lm;
-  const bool lvalid = lp < q.P;
-  const float* abase = q.win;
-  if (lvalid) {
-    int64_t n;
-    int r;
-    split_position(lp, q, n, r);
-    const int ho = r / q.Wo;
-    const int wo = r - ho * q.Wo;
-    abase += n * q.img_stride + ho * q.strip + (int64_t)wo * q.sKh;
+  const float* abase[NBASE];
+  uint32_t lvalid = 0;
+#pragma unroll
+  for (int j = 0; j < NBASE; ++j) {
+    const int64_t lp = m0 + lm + 4 * j;
+    abase[j] = q.win;
+    if (lp < q.P) {
+      int64_t n;
+      int r;
+      split_position(lp, q, n, r);
+      const int ho = r / q.Wo;
+      const int wo = r - ho * q.Wo;
+      abase[j] += n * q.img_stride + ho * q.strip + (int64_t)wo * q.sKh;
+      lvalid |= 1u << j;
+    }
   }
 
-  int offreg[A_PER_THREAD];          // offsets of the next k-block to be issued
+  int offreg[NOFF];                  // offsets of the next k-block to be issued
 
   // The offset table is read one k-block ahead of the copies it addresses, so that issuing
   // the copies never waits for it.
   auto load_offsets = [&](int kb) {
     const int k0 = kb * BK;
 #pragma unroll
-    for (int i = 0; i < A_PER_THREAD; ++i) offreg[i] = __ldg(q.koff + k0 + lkk0 + i * A_KK_STEP);
+    for (int i = 0; i < NOFF; ++i) offreg[i] = __ldg(q.koff + k0 + (KLANES ? i * 8 + kq : lkk0 + i * A_KK_STEP));
   };
   // Asynchronous copies (global -> shared, no registers) of k-block kb into ring slot `buf`:
   // 4-byte gathers of the window operand (zero-filled outside the tensor and in the padded
@@ -116,12 +135,16 @@ conv_f32_kernel(ConvF32Params q) {
   auto issue_copies = [&](int kb, int buf, bool more) {
     const int k0 = kb * BK;
 #pragma unroll
-    for (int i = 0; i < A_PER_THREAD; ++i) {
+    for (int i = 0; i < NOFF; ++i) {
       const int off = offreg[i];
-      const bool ok = lvalid && off >= 0;
-      const float* src = ok ? abase + off : q.win;
-      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&As[buf][lkk0 + i * A_KK_STEP][lm]);
-      asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(ok ? 4 : 0) : "memory");
+#pragma unroll
+      for (int j = 0; j < NBASE; ++j) {
+        const bool ok = ((lvalid >> j) & 1u) && off >= 0;
+        const float* src = ok ? abase[j] + off : q.win;
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(
+            KLANES ? &As[buf][i * 8 + kq][lm + 4 * j] : &As[buf][lkk0 + i * A_KK_STEP][lm]);
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(ok ? 4 : 0) : "memory");
+      }
     }
 #pragma unroll
     for (int i = 0; i < B_VEC_PER_THREAD; ++i) {
@@ -258,6 +281,10 @@ F32Plan plan_f32(const Geometry& g) {
   if (const char* v = debug_getenv("IM2WIN_F32_BM")) small_m = atoi(v) == 64;   // testing aid
   p.bm = small_m ? 64 : 128;
   p.bk = (wide && small_m && g.K >= 256) ? 32 : 16;
+  // k along the lanes of the gather where windows lie 128 bytes or more apart and the reduction is long
+  // enough for the per-thread set-up of several positions not to matter (128-position tiles only)
+  p.klanes = !small_m && g.s * g.Kh >= 32 && g.K >= 256;
+  if (const char* v = debug_getenv("IM2WIN_F32_KLANES")) p.klanes = !small_m && v[0] == '1';   // testing aid
   if (const char* v = debug_getenv("IM2WIN_F32_BK")) { if (wide && small_m) p.bk = atoi(v) == 32 ? 32 : 16; }   // testing aid
   return p;
 }
@@ -278,22 +305,25 @@ cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, 
   const int64_t cot = l.Co_pad / p.bn;
   dim3 grid((unsigned)((g.P + p.bm - 1) / p.bm), (unsigned)cot);
   const int threads = (p.bm / 8) * f32_tn(p.bn);
-  const size_t smem = (size_t)3 * p.bk * (p.bm + p.bn) * 4;
+  const size_t smem = (size_t)3 * p.bk * (p.bm + (p.klanes ? 4 : 0) + p.bn) * 4;
   void (*kernel)(ConvF32Params);
   int which;
   if (p.bn == 96) {
-    if (p.bm == 64) { kernel = p.bk == 32 ? conv_f32_kernel<64, 96, 32> : conv_f32_kernel<64, 96, 16>; which = p.bk == 32 ? 5 : 6; }
-    else { kernel = conv_f32_kernel<128, 96, 16>; which = 7; }
+    if (p.bm == 64) { kernel = p.bk == 32 ? conv_f32_kernel<64, 96, 32, false> : conv_f32_kernel<64, 96, 16, false>; which = p.bk == 32 ? 5 : 6; }
+    else if (p.klanes) { kernel = conv_f32_kernel<128, 96, 16, true>; which = 8; }
+    else { kernel = conv_f32_kernel<128, 96, 16, false>; which = 7; }
   } else if (p.bn == 128) {
-    if (p.bm == 64) { kernel = p.bk == 32 ? conv_f32_kernel<64, 128, 32> : conv_f32_kernel<64, 128, 16>; which = p.bk == 32 ? 0 : 1; }
-    else { kernel = conv_f32_kernel<128, 128, 16>; which = 2; }
+    if (p.bm == 64) { kernel = p.bk == 32 ? conv_f32_kernel<64, 128, 32, false> : conv_f32_kernel<64, 128, 16, false>; which = p.bk == 32 ? 0 : 1; }
+    else if (p.klanes) { kernel = conv_f32_kernel<128, 128, 16, true>; which = 9; }
+    else { kernel = conv_f32_kernel<128, 128, 16, false>; which = 2; }
   } else {
-    if (p.bm == 64) { kernel = conv_f32_kernel<64, 64, 16>; which = 3; }
-    else { kernel = conv_f32_kernel<128, 64, 16>; which = 4; }
+    if (p.bm == 64) { kernel = conv_f32_kernel<64, 64, 16, false>; which = 3; }
+    else if (p.klanes) { kernel = conv_f32_kernel<128, 64, 16, true>; which = 10; }
+    else { kernel = conv_f32_kernel<128, 64, 16, false>; which = 4; }
   }
   if (smem > 48 * 1024) {
     // per device and tile shape, once: the opt-in to more than 48 KB of dynamic shared memory
-    static bool attr_done[64][8] = {};
+    static bool attr_done[64][11] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!attr_done[dev][which]) {

@@ -149,6 +149,25 @@ def test_conv_f32_both_tile_heights(layer, bm, bk, monkeypatch):
     check_conv(y, yr, ar, "f32", layer.name)
 
 
+@pytest.mark.parametrize("layer", [SMALL[1], SMALL[2], SMALL[28], L("wide_co", 3, 20, 11, 13, 150, 3, 3, 1, 1, 47),
+                                   L("co96_s4", 3, 3, 63, 67, 96, 11, 11, 4, 0, 50)], ids=lambda l: l.name)
+def test_conv_f32_gather_with_k_along_lanes(layer, monkeypatch):
+    """The fp32 kernel's second way of gathering the window operand (a warp's copy instruction covers
+    eight consecutive k of four positions; the library takes it for windows 128 bytes or more apart),
+    forced on 128-position tiles of 64, 96 and 128 channels, with ragged position and channel tails."""
+    monkeypatch.setenv("IM2WIN_F32_BM", "128")
+    monkeypatch.setenv("IM2WIN_F32_KLANES", "1")
+    dims = layer.dims()
+    x, f = workloads.make_small_integer_inputs(layer)
+    y, _, _ = gpu_conv(x, f, dims, "f32")
+    yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+    assert np.array_equal(y.astype(np.float64), yr)
+    x, f = workloads.make_inputs(layer)
+    y, _, _ = gpu_conv(x, f, dims, "f32")
+    yr, ar = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+    check_conv(y, yr, ar, "f32", layer.name)
+
+
 def test_f16_inputs_are_the_oracles_rounding():
     """The cast that feeds the fp16 path (torch .half()) and the oracle's rounding agree bit for bit."""
     layer = workloads.LAYERS["cfg5k11"].with_batch(1)
