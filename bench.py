@@ -450,6 +450,9 @@ def time_call(fn, iters, flush):
     total = 0.0
     best = float("inf")
     samples = []
+    for _ in range(2):                 # untimed: the call's own first-use costs stay out of the average
+        fn()
+    torch.cuda.synchronize()
     for _ in range(iters):
         flush.zero_()
         # keep the GPU busy (~0.3 ms) while the host queues the events and the call, so that the
@@ -537,8 +540,8 @@ def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
             # conv_packed_*: the convolution on a filter packed beforehand (static weights), i.e. without
             # the pack kernel that conv_f16_nhwc runs on every call
             for key, fn in (("transform_f16_nhwc", runner.transform_nhwc), ("conv_f16_nhwc", runner.conv_nhwc),
-                            ("conv_f16_out16_nhwc", runner.conv_nhwc_out16),
-                            ("conv_packed_f16_nhwc", runner.conv_nhwc_packed)):
+                            ("conv_packed_f16_nhwc", runner.conv_nhwc_packed),
+                            ("conv_f16_out16_nhwc", runner.conv_nhwc_out16)):
                 avg[key], best[key], median[key] = time_call(fn, iters, flush)
                 b2b[key] = time_back_to_back(lambda i: fn(None, i), sets, iters)
             for d in runner.nhwc_sets:
