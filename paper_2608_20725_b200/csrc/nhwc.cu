@@ -82,6 +82,7 @@ struct NhwcParams {
   // holds the end of one tile's reduction and / or the start of the next one's.  The CTA that starts a tile
   // stores it; the others leave their partial sums in `partial` and raise their flag.
   int32_t stream_tiles, stream_u, stream_ctas;
+  int32_t raster, ntm_eff;   // testing aid: 1 = items in channel-tile-major order (ntm_eff position tiles (pairs) per channel tile)
   float* partial;            // kPartialBytes
   uint32_t* flags;           // two words per CTA (pair) of the grid, compared with `epoch`
   uint32_t epoch;
@@ -325,6 +326,18 @@ __device__ __forceinline__ void drain_with_partials(const EpiParams& e, int cols
   }
 }
 
+// Whole tile index -> (position tile (pair) mt, channel tile nt, K part ks).  Default order: nt and ks
+// fastest, so that the CTAs that share an activation tile run at the same time; the other order (all
+// position tiles of a channel tile, then the next channel tile) exists for the ablation only.
+__device__ __forceinline__ void tile_coords(const NhwcParams& q, int whole, int* mt, int* nt, int* ks) {
+  const int per_mt = q.ntn * q.ksplit;
+  int rem;
+  if (q.raster == 0) { *mt = whole / per_mt; rem = whole - *mt * per_mt; }
+  else { rem = whole / q.ntm_eff; *mt = whole - rem * q.ntm_eff; }
+  *nt = rem / q.ksplit;
+  *ks = rem - *nt * q.ksplit;
+}
+
 // Work item w of the overlapping-row kernel -> whole tile index and which part of its channels:
 // half = -1 the whole tile, 0 / 1 its lower / upper half.
 __device__ __forceinline__ void decode_item(const NhwcParams& q, int w, int* whole, int* half) {
@@ -404,8 +417,8 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
           decode_item(q, w, &whole, &half);
           kc0 = -1;
         }
-        const int mt = whole / per_mt, rem = whole - mt * per_mt;
-        const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
+        int mt, nt, ks;
+        tile_coords(q, whole, &mt, &nt, &ks);
         const int mti = PAIR ? 2 * mt + (int)rank : mt;
         const int rg = mti / q.tw, wt = mti - rg * q.tw;
         const int z = rg * q.G, yc = wt * q.bw;
@@ -465,7 +478,8 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
           half = -1;
         } else {
           decode_item(q, w, &whole, &half);
-          const int ks = (whole % per_mt) % q.ksplit;
+          int mt, nt, ks;
+          tile_coords(q, whole, &mt, &nt, &ks);
           kc0 = ks * q.kc_per_split;
           kc1 = kc0 + q.kc_per_split < q.num_kc ? kc0 + q.kc_per_split : q.num_kc;
         }
@@ -532,8 +546,8 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       } else {
         decode_item(q, w, &whole, &half);
       }
-      const int mt = whole / per_mt, rem = whole - mt * per_mt;
-      const int nt = rem / q.ksplit, ks = rem - nt * q.ksplit;
+      int mt, nt, ks;
+      tile_coords(q, whole, &mt, &nt, &ks);
       const int mti = PAIR ? 2 * mt + (int)rank : mt;
       const int rg = mti / q.tw, wt = mti - rg * q.tw;
       const int n0 = nt * BN + (half > 0 ? BN / 2 : 0);
@@ -1537,6 +1551,7 @@ cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, con
   int stages = (kSmemMax - 2048) / STAGE;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) return cudaErrorInvalidValue;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_STAGES")) { const int n = atoi(v); if (n >= 2 && n < stages) stages = n; }   // ablation: ring depth
   q.stages = stages;
   // K in chunks of KSUB k-blocks; a K split hands out whole chunks
   q.num_kc = (plan.num_kb + KSUB - 1) / KSUB;
@@ -1546,6 +1561,9 @@ cudaError_t launch_variant(const CUtensorMap& amap, const CUtensorMap& bmap, con
   const int64_t ntm_eff = PAIR ? (plan.ntm + 1) / 2 : plan.ntm;
   const int64_t nwork = ntm_eff * q.ntn * q.ksplit;
   if (nwork >= ((int64_t)1 << 30)) return cudaErrorInvalidValue;
+  q.ntm_eff = (int32_t)ntm_eff;
+  q.raster = 0;
+  if (const char* v = debug_getenv("IM2WIN_NHWC_RASTER")) q.raster = v[0] == '1';     // ablation: item order
   q.nwork = (int32_t)nwork;
   q.n_main = q.nwork;
   int slots = PAIR ? 74 : 148;

@@ -137,6 +137,25 @@ def test_conv_nhwc_epilogue_options(layer, out16, y_nhwc, bias, relu, monkeypatc
         assert np.array_equal(y, y.astype(np.float16).astype(np.float64))
 
 
+@pytest.mark.parametrize("raster,stages,bn,ksplit", [("1", "7", "64", "1"), ("1", "2", "128", "2"), ("0", "2", "256", "1"),
+                                                      ("1", "3", "64", "3")])
+def test_conv_nhwc_overlap_item_order_and_ring_depth(raster, stages, bn, ksplit, monkeypatch):
+    """The ablation switches of the overlapping-row kernel (work items in channel-tile-major order, a
+    shallower operand ring) change when a tile is computed, never what: exact on integer-valued inputs on a
+    layer with several position tiles, several channel tiles and a ragged last one."""
+    monkeypatch.setenv("IM2WIN_NHWC_KERNEL", "overlap")
+    monkeypatch.setenv("IM2WIN_NHWC_RASTER", raster)
+    monkeypatch.setenv("IM2WIN_NHWC_STAGES", stages)
+    monkeypatch.setenv("IM2WIN_NHWC_BN", bn)
+    monkeypatch.setenv("IM2WIN_NHWC_KSPLIT", ksplit)
+    layer = L("order_depth", 5, 24, 19, 23, 150, 3, 3, 1, 1, 63)
+    dims = layer.dims()
+    x, f = workloads.make_small_integer_inputs(layer)
+    yr, _ = oracle.conv_direct(x.numpy(), f.numpy(), dims)
+    assert np.array_equal(gpu_conv_nhwc(x, f, dims), yr)
+    assert np.array_equal(gpu_conv_nhwc(x, f, dims, y_nhwc=True), yr.transpose(0, 2, 3, 1))
+
+
 @pytest.mark.parametrize("layer", [L("many_items", 16, 16, 40, 40, 48, 3, 3, 1, 1, 60),
                                    L("many_items_s2", 12, 8, 61, 62, 20, 5, 5, 2, 2, 61)], ids=lambda l: l.name)
 @pytest.mark.parametrize("dual", ["0", "1"])
