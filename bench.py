@@ -168,12 +168,18 @@ class LayerRunner:
                      scratch=scratch, y=y, cp=cp, y16=torch.empty(y.shape, dtype=torch.float16, device="cuda"),
                      bias=torch.zeros(self.layer.Co, dtype=torch.float32, device="cuda"))
             d["epi16"] = b.make_epilogue(d["bias"], True, torch.float16, b.NCHW)
+            d["x_nhwc"] = d["x"].permute(0, 2, 3, 1).contiguous()      # the same input, channel-innermost
             self.nhwc_sets.append(d)
         self.nhwc = self.nhwc_sets[0]
 
     def transform_nhwc(self, prec=None, i=0):
         d = self.nhwc_sets[i]
         self.b.im2win_transform_nhwc(d["x"], self.b.NCHW, d["window"], self.dims)
+
+    def transform_nhwc_from_nhwc(self, prec=None, i=0):
+        """The same window tensor from a channel-innermost input (what a chain of NHWC layers feeds)."""
+        d = self.nhwc_sets[i]
+        self.b.im2win_transform_nhwc(d["x_nhwc"], self.b.NHWC, d["window"], self.dims)
 
     def conv_nhwc(self, prec=None, i=0):
         d = self.nhwc_sets[i]
@@ -539,7 +545,8 @@ def layer_rows(peaks, peak_kind, names=None, iters=20, with_packed=True):
                 runner.conv_nhwc()
             # conv_packed_*: the convolution on a filter packed beforehand (static weights), i.e. without
             # the pack kernel that conv_f16_nhwc runs on every call
-            for key, fn in (("transform_f16_nhwc", runner.transform_nhwc), ("conv_f16_nhwc", runner.conv_nhwc),
+            for key, fn in (("transform_f16_nhwc", runner.transform_nhwc),
+                            ("transform_from_nhwc_f16_nhwc", runner.transform_nhwc_from_nhwc), ("conv_f16_nhwc", runner.conv_nhwc),
                             ("conv_packed_f16_nhwc", runner.conv_nhwc_packed),
                             ("conv_f16_out16_nhwc", runner.conv_nhwc_out16)):
                 avg[key], best[key], median[key] = time_call(fn, iters, flush)
