@@ -177,7 +177,7 @@ __device__ __forceinline__ uint32_t run_pair16(const uint32_t (&r)[KH][NW], int 
 // well under half the instructions of the element-wise form (VB = 0), which is what bounds
 // this kernel.
 template <typename E, int KH, int VB>
-__global__ void __launch_bounds__(kStripThreads)
+__global__ void __launch_bounds__(kStripThreads, KH >= 7 ? 4 : 0)   // (tall kernels: four CTAs per SM; they would otherwise take 76-128 registers and run three)
 transform_strips_kernel(const E* __restrict__ x, E* __restrict__ win, StripParams q) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int ES = (int)sizeof(E);
