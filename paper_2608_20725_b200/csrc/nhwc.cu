@@ -248,8 +248,21 @@ __device__ __noinline__ bool wait_flag(const uint32_t* flag, uint32_t value, vol
   return false;
 }
 
-__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+// The eight epilogue warps have stored their shares of a tile (or of its partial sums); one of them then
+// raises a flag for other CTAs.  Every warp fences its stores and arrives on a CTA-local mbarrier; the first
+// epilogue warp's lane 0 takes the BOUNDED wait for all eight arrivals before it publishes (a bar.sync here
+// could wait for good if one warp had given up on an earlier wait and left the loop).  `phase` is the
+// barrier's parity for this use (all warps count the uses alike).
+__device__ __forceinline__ void publish_when_all_stored(uint32_t epi_bar, uint32_t phase, int warp, int lane, uint32_t* flag,
+                                                        uint32_t epoch, volatile uint32_t* abort_flag, uint32_t* status) {
+  __threadfence();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(epi_bar);
+  if (warp == WARP_EPI0 && lane == 0) {
+    // (testing aid: with the marker in word 2 of the status block the flag stays down)
+    if (mbar_wait(epi_bar, phase, abort_flag, status) && *reinterpret_cast<volatile uint32_t*>(status + 2) != kDebugDropFlag)
+      asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(epoch) : "memory");
+  }
 }
 
 // CTA `cta`'s two stream items (see NhwcParams): slot 0 is the part of its chunk range that does not start
@@ -359,7 +372,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 2 * MAX_ACC];
+  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 2 * MAX_ACC + 1];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile uint32_t abort_flag;
 
@@ -370,6 +383,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
   const uint32_t empty0 = smem_u32(&bars[MAX_STAGES]);
   const uint32_t acc_full0 = smem_u32(&bars[2 * MAX_STAGES]);
   const uint32_t acc_empty0 = smem_u32(&bars[2 * MAX_STAGES + MAX_ACC]);
+  const uint32_t epi_bar = smem_u32(&bars[2 * MAX_STAGES + 2 * MAX_ACC]);   // rendezvous of the epilogue warps (publish_when_all_stored)
 
   if (threadIdx.x == 0) {
     abort_flag = 0u;
@@ -381,6 +395,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
       mbar_init(acc_full0 + 8 * i, 1);
       mbar_init(acc_empty0 + 8 * i, PAIR ? 2 * EPI_WARPS : EPI_WARPS);   // the epilogue warps (of each CTA)
     }
+    mbar_init(epi_bar, EPI_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == WARP_MMA) {
@@ -531,7 +546,7 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
     float breg[32];
     const bool hoisted = hoist_bias<BN>(e, q.ntn, warp, breg);
     bool ok = true;
-    uint32_t it = 0;
+    uint32_t it = 0, epi_phase = 0;
     TIMER_DECL;
     for (int w = w_first; w < q.nwork && ok; w += w_step) {
       const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
@@ -582,11 +597,8 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
         constexpr size_t SLOT = (size_t)BN * TILE_M;         // floats of one CTA's partial tile
         if (frag == 1) {
           dump_partial(cols, warp, lane, lane_base, q.partial + (size_t)(PER * w_first + (int)rank) * SLOT);
-          __threadfence();
-          named_barrier_sync(1, EPI_WARPS * 32);             // all eight epilogue warps have stored
-          // (testing aid: with the marker in word 2 of the status block the flag stays down)
-          if (threadIdx.x == WARP_EPI0 * 32 && *reinterpret_cast<volatile uint32_t*>(q.status + 2) != kDebugDropFlag)
-            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(q.flags + PER * w_first + (int)rank), "r"(q.epoch) : "memory");
+          publish_when_all_stored(epi_bar, epi_phase, warp, lane, q.flags + PER * w_first + (int)rank, q.epoch, &abort_flag, q.status);
+          epi_phase ^= 1u;
         } else {
           if (threadIdx.x == WARP_EPI0 * 32) TIMER_LAP(5);
           // the CTAs after this one whose ranges reach into the tile
@@ -738,7 +750,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
-  __shared__ __align__(8) uint64_t bars[2 * MAX_SA + 2 * MAX_SB + 2 * MAX_ACC];
+  __shared__ __align__(8) uint64_t bars[2 * MAX_SA + 2 * MAX_SB + 2 * MAX_ACC + 1];
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile uint32_t abort_flag;
   __shared__ uint32_t tap16[MAX_KW];           // view of kernel column v inside an activation stage, in 16-byte units
@@ -754,6 +766,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
   const uint32_t b_empty0 = smem_u32(&bars[2 * MAX_SA + MAX_SB]);
   const uint32_t acc_full0 = smem_u32(&bars[2 * MAX_SA + 2 * MAX_SB]);
   const uint32_t acc_empty0 = smem_u32(&bars[2 * MAX_SA + 2 * MAX_SB + MAX_ACC]);
+  const uint32_t epi_bar = smem_u32(&bars[2 * MAX_SA + 2 * MAX_SB + 2 * MAX_ACC]);   // rendezvous of the epilogue warps
 
   if (threadIdx.x == 0) {
     abort_flag = 0u;
@@ -765,6 +778,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       mbar_init(acc_full0 + 8 * i, 1);
       mbar_init(acc_empty0 + 8 * i, PAIR ? 2 * EPI_WARPS : EPI_WARPS);
     }
+    mbar_init(epi_bar, EPI_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == WARP_MMA) {
@@ -1049,7 +1063,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       for (int t = 0; t < (HOIST ? 32 : 1); ++t) breg[t] = c0 + t < e.Co ? __ldg(e.bias + c0 + t) : 0.0f;
     }
     bool ok = true;
-    uint32_t it = 0;
+    uint32_t it = 0, epi_phase = 0;
     TIMER_DECL;
     for (int w = w_first; w < q.nwork && ok; w += w_step, ++it) {
       const uint32_t buf = it % (uint32_t)NACC, aph = (it / (uint32_t)NACC) & 1u;
@@ -1095,11 +1109,8 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       if (ok) drain_accumulator(e, cols, warp, lane, lane_base, valid, base, cs, n0, kpart ? part == 0 : ks == 0, vec_ok, adds,
                                 HOIST ? breg : nullptr);
       if (kpart && part == 0) {
-        __threadfence();
-        named_barrier_sync(1, EPI_WARPS * 32);          // all eight epilogue warps have stored
-        // (testing aid: with the marker in word 2 of the status block the flag stays down)
-        if (threadIdx.x == WARP_EPI0 * 32 && *reinterpret_cast<volatile uint32_t*>(q.status + 2) != kDebugDropFlag)
-          asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(q.epoch) : "memory");
+        publish_when_all_stored(epi_bar, epi_phase, warp, lane, flag, q.epoch, &abort_flag, q.status);
+        epi_phase ^= 1u;
       }
       tc_fence_before();
       __syncwarp();
@@ -1597,6 +1608,7 @@ RunPlan plan_runs(int64_t nwork, int slots, int num_kc, int ksub, int bn) {
   if (!on || tail == 0) return r;
   const int min_run = (num_kc + 7) / 8 > 8 / ksub ? (num_kc + 7) / 8 : 8 / ksub;
   const int64_t total = (int64_t)tail * num_kc;
+  if (total >= ((int64_t)1 << 30)) return r;             // (the kernel indexes the runs with 32-bit integers)
   int S = slots;
   if (total / S < min_run) S = (int)(total / min_run);
   if (S <= tail) return r;
