@@ -410,10 +410,8 @@ __device__ __forceinline__ void conv_nhwc_body(const CUtensorMap& amap, const CU
   const uint32_t full_dst = PAIR ? mapa_shared(full0, 0) : full0;          // the leader's barriers
   const uint32_t acc_empty_dst = PAIR ? mapa_shared(acc_empty0, 0) : acc_empty0;
 
-  // work item w -> (position tile (pair) mt, channel tile nt, k part ks), nt and ks fastest so that
-  // the CTAs that share an activation tile run at the same time.  K is walked in chunks of KSUB
-  // 64-wide k-blocks: one ring stage, one pair of barrier operations per chunk.
-  const int per_mt = q.ntn * q.ksplit;
+  // work item w -> (position tile (pair) mt, channel tile nt, k part ks): tile_coords.  K is walked in
+  // chunks of KSUB 64-wide k-blocks: one ring stage, one pair of barrier operations per chunk.
 
   if (warp == WARP_TMA) {
     // ---------------- copies of both operands ------------------------------------
@@ -910,7 +908,7 @@ __device__ __forceinline__ void conv_shift_body(const CUtensorMap& amap, const C
       uint32_t pha = 0, phb = 0, it = (uint32_t)mid;
       bool ok = true;
       const uint32_t a_lo0 = smem_desc_lo(a_ring), b_lo0 = smem_desc_lo(b_ring);
-      const uint32_t subt16 = q.subt_bytes >> 4, astage16 = q.a_stage_bytes >> 4, bstage16 = b_stage_bytes >> 4;
+      const uint32_t astage16 = q.a_stage_bytes >> 4, bstage16 = b_stage_bytes >> 4;
       uint32_t tapr[7];                          // the first seven view offsets in registers (unrolled issue paths)
 #pragma unroll
       for (int v = 0; v < 7; ++v) tapr[v] = v < q.Kw ? tap16[v] : 0u;
