@@ -113,6 +113,7 @@ struct EpilogueArgs {
 struct F32Plan {
   int32_t bm, bn, bk;
   bool klanes;             // the window operand is gathered with k along the lanes of a warp
+  bool tall;               // 16 positions x 8 channels per thread (position pairs packed)
 };
 F32Plan plan_f32(const Geometry& g);
 

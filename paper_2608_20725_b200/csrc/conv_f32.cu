@@ -15,6 +15,8 @@
 // unchanged -- measured 74 TFLOP/s for both forms -- but the kernel is bound by
 // issue slots, which the packed form halves).  Positions run along the lanes,
 // so stores to the NCHW output are contiguous per output channel.
+// Large layers (128-position tiles) take a second form with a 16 x 8 register tile whose pairs are
+// adjacent POSITIONS (conv_f32_tall_kernel below).
 #include "common.cuh"
 
 namespace im2win {
@@ -255,6 +257,159 @@ conv_f32_kernel(ConvF32Params q) {
   }
 }
 
+
+// Second form of the same kernel: 16 positions x 8 channels per thread, accumulators packed as pairs of
+// adjacent POSITIONS.  The pairs come straight out of the 128-bit loads of the window operand; only the
+// eight filter values of a k are duplicated with moves: per 128 FMAs 64 fma.rn.f32x2 + 8 moves + 6 shared
+// loads against 64 + 16 + 8 in the 8 x 8 form, i.e. 6 % fewer FMA-pipe cycles and 11 % fewer issue slots.
+// (BM/16)*(BN/8) threads: 64 for the 128 x 64 and 64 x 128 tiles, 128 for 128 x 128.  The register cap of 200
+// keeps five 64-thread CTAs on an SM (206 registers uncapped: four CTAs, and 2 % slower than the 8 x 8 form
+// instead of 5 % faster; a cap of 168: spills, 30 % slower).  Every loader thread tracks BM/threads positions;
+// the offsets of the next k-block are prefetched as in the first form.
+template <int BM, int BN, int BK>
+__global__ void __maxnreg__(200)
+conv_f32_tall_kernel(ConvF32Params q) {
+  constexpr int THREADS = (BM / 16) * (BN / 8);
+  constexpr int NPOS = BM / THREADS;                       // positions per loader thread
+  constexpr int B_VEC_PER_THREAD = BK * BN / 4 / THREADS;
+  static_assert(BM % THREADS == 0 && (BK * BN / 4) % THREADS == 0, "loader mapping");
+  constexpr int STAGES = 3;
+  extern __shared__ __align__(16) unsigned char smem_f32[];
+  float (*As)[BK][BM] = reinterpret_cast<float (*)[BK][BM]>(smem_f32);
+  float (*Bs)[BK][BN] = reinterpret_cast<float (*)[BK][BN]>(smem_f32 + sizeof(float) * STAGES * BK * BM);
+
+  const int tid = threadIdx.x;
+  const int tm = tid % (BM / 16);
+  const int tn = tid / (BM / 16);
+  const int64_t m0 = (int64_t)blockIdx.x * BM;
+  const int n0 = blockIdx.y * BN;
+
+  const float* abase[NPOS];
+  uint32_t lvalid = 0;
+#pragma unroll
+  for (int j = 0; j < NPOS; ++j) {
+    const int64_t lp = m0 + tid + j * THREADS;
+    abase[j] = q.win;
+    if (lp < q.P) {
+      int64_t n;
+      int r;
+      split_position(lp, q, n, r);
+      const int ho = r / q.Wo;
+      const int wo = r - ho * q.Wo;
+      abase[j] += n * q.img_stride + ho * q.strip + (int64_t)wo * q.sKh;
+      lvalid |= 1u << j;
+    }
+  }
+  int offreg[BK];
+  auto load_offsets = [&](int kb) {
+#pragma unroll
+    for (int i = 0; i < BK; ++i) offreg[i] = __ldg(q.koff + kb * BK + i);
+  };
+  auto issue_copies = [&](int kb, int buf) {
+    const int k0 = kb * BK;
+#pragma unroll
+    for (int i = 0; i < BK; ++i) {
+      const int off = offreg[i];
+#pragma unroll
+      for (int j = 0; j < NPOS; ++j) {
+        const bool ok = ((lvalid >> j) & 1u) && off >= 0;
+        const float* src = ok ? abase[j] + off : q.win;
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&As[buf][i][tid + j * THREADS]);
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(ok ? 4 : 0) : "memory");
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < B_VEC_PER_THREAD; ++i) {
+      const int e = tid + i * THREADS;
+      const int kk = e / (BN / 4);
+      const int nn = (e - kk * (BN / 4)) * 4;
+      const float* src = q.fk + (int64_t)(k0 + kk) * q.Co_pad + n0 + nn;
+      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&Bs[buf][kk][nn]);
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+    }
+    if (kb + 1 < q.Kp / BK) load_offsets(kb + 1);
+  };
+  load_offsets(0);
+
+  unsigned long long acc2[8][8];     // acc2[ip][j] = (acc[2 ip][j], acc[2 ip + 1][j]): position pairs
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc2[i][j] = 0ull;
+
+  const int nkb = q.Kp / BK;
+#pragma unroll
+  for (int s = 0; s < STAGES - 1; ++s) {
+    if (s < nkb) issue_copies(s, s);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  int buf = 0;
+  for (int kb = 0; kb < nkb; ++kb) {
+    asm volatile("cp.async.wait_group %0;" ::"n"(STAGES - 2) : "memory");
+    __syncthreads();
+    {
+      const int nk = kb + STAGES - 1;
+      int nbuf = buf + STAGES - 1;
+      if (nbuf >= STAGES) nbuf -= STAGES;
+      if (nk < nkb) issue_copies(nk, nbuf);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      unsigned long long a[8];
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(&As[buf][kk][g * (BM / 4) + tm * 4]);
+        a[2 * g] = v.x; a[2 * g + 1] = v.y;
+      }
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][kk][tn * 4]);
+      const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][kk][BN / 2 + tn * 4]);
+      const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const unsigned long long bd = dup2(b[j]);
+#pragma unroll
+        for (int ip = 0; ip < 8; ++ip) ffma2(acc2[ip][j], a[ip], bd);
+      }
+    }
+    if (++buf == STAGES) buf = 0;
+  }
+
+  // positions of pair ip: group g = ip / 2, offset (ip % 2) * 2 .. + 1 inside the group's four
+  const bool vec_ok = (q.HoWo % 4) == 0;
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const int64_t p = m0 + g * (BM / 4) + tm * 4;
+    if (p >= q.P) continue;
+    int64_t n;
+    int r;
+    split_position(p, q, n, r);
+    int64_t nn[4];
+    int rr[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      nn[i] = n; rr[i] = r + i;
+      while (rr[i] >= q.HoWo) { rr[i] -= q.HoWo; ++nn[i]; }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int co = n0 + (j / 4) * (BN / 2) + tn * 4 + (j % 4);
+      if (co >= q.Co) continue;
+      const float2 lo = unpack2(acc2[2 * g][j]), hi = unpack2(acc2[2 * g + 1][j]);
+      const float v[4] = {lo.x, lo.y, hi.x, hi.y};
+      if (vec_ok) {
+        *reinterpret_cast<float4*>(q.y + (n * q.Co + co) * q.HoWo + r) = make_float4(v[0], v[1], v[2], v[3]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (p + i >= q.P) break;
+          q.y[(nn[i] * q.Co + co) * q.HoWo + rr[i]] = v[i];
+        }
+      }
+    }
+  }
+}
+
 }  // namespace
 
 // Tile shape of a layer.  64-channel tiles up to 64 output channels, else 128; 64-position tiles when
@@ -285,6 +440,14 @@ F32Plan plan_f32(const Geometry& g) {
   // enough for the per-thread set-up of several positions not to matter (128-position tiles only)
   p.klanes = !small_m && g.s * g.Kh >= 32 && g.K >= 256;
   if (const char* v = debug_getenv("IM2WIN_F32_KLANES")) p.klanes = !small_m && v[0] == '1';   // testing aid
+  // 16 x 8 outputs per thread on 128-position tiles of 64 or 128 channels (conv_f32_tall_kernel).  Measured
+  // 5-6 % faster there (3x3 on 64 channels at 56x56: 597 -> 567 us; 5x5 on 96 -> 256 channels 0.75 -> 0.79 of
+  // the FFMA peak, 3x3 on 64 -> 128 channels at 112x112 0.77 -> 0.815), 1-4 % slower than the 64-position tile with
+  // k-blocks of 32 where that one is planned, and slower on a reduction of 27 (two k-blocks per tile).
+  const bool tall_ok = !p.klanes && (p.bn == 128 || (p.bn == 64 && p.bm == 128));
+  p.tall = tall_ok && p.bm == 128 && g.K >= 128;
+  if (const char* v = debug_getenv("IM2WIN_F32_TALL")) p.tall = tall_ok && v[0] == '1';   // testing aid
+  if (p.tall) p.bk = 16;
   if (const char* v = debug_getenv("IM2WIN_F32_BK")) { if (wide && small_m) p.bk = atoi(v) == 32 ? 32 : 16; }   // testing aid
   return p;
 }
@@ -331,6 +494,23 @@ cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, 
       if (e != cudaSuccess) return e;
       attr_done[dev][which] = true;
     }
+  }
+  if (p.tall) {
+    void (*tk)(ConvF32Params) = p.bn == 64 ? conv_f32_tall_kernel<128, 64, 16>
+                                           : (p.bm == 64 ? conv_f32_tall_kernel<64, 128, 16> : conv_f32_tall_kernel<128, 128, 16>);
+    const int tw = p.bn == 64 ? 11 : (p.bm == 64 ? 12 : 13);
+    if (smem > 48 * 1024) {
+      static bool tall_attr[64][14] = {};
+      int dev = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+      if (!tall_attr[dev][tw]) {
+        cudaError_t e = cudaFuncSetAttribute(tk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        tall_attr[dev][tw] = true;
+      }
+    }
+    tk<<<grid, (p.bm / 16) * (p.bn / 8), smem, stream>>>(q);
+    return cudaGetLastError();
   }
   kernel<<<grid, threads, smem, stream>>>(q);
   return cudaGetLastError();

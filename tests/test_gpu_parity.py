@@ -131,13 +131,19 @@ def test_conv_exact_on_integer_inputs(layer, precision):
 @pytest.mark.parametrize("layer", [SMALL[1], SMALL[2], L("wide_co", 3, 20, 11, 13, 150, 3, 3, 1, 1, 47),
                                    L("co96", 2, 12, 30, 29, 96, 5, 5, 2, 2, 48), L("co200", 1, 9, 14, 15, 200, 3, 3, 1, 1, 49)],
                          ids=lambda l: l.name)
-@pytest.mark.parametrize("bm,bk", [("64", "16"), ("64", "32"), ("128", "16")])
+@pytest.mark.parametrize("bm,bk", [("64", "16"), ("64", "32"), ("128", "16"), ("128", "tall"), ("64", "tall")])
 def test_conv_f32_both_tile_heights(layer, bm, bk, monkeypatch):
     """The fp32 kernel's 64- and 128-position tiles (the library picks by grid size), on 64-, 96- and
     128-channel tiles (96 where that pads the output channels least: 96 and 150 here, not 200), and the
-    64-position tiles with both k-blocks: exact on integer-valued inputs, within tolerance on the seeded ones."""
+    64-position tiles with both k-blocks, all with the 8 x 8 register tile; then the 16 x 8 register tile
+    (what 128-position tiles of 64 and 128 channels take by default) on 128 x 64, 128 x 128 and 64 x 128
+    tiles: exact on integer-valued inputs, within tolerance on the seeded ones."""
     monkeypatch.setenv("IM2WIN_F32_BM", bm)
-    monkeypatch.setenv("IM2WIN_F32_BK", bk)
+    if bk == "tall":
+        monkeypatch.setenv("IM2WIN_F32_TALL", "1")
+    else:
+        monkeypatch.setenv("IM2WIN_F32_BK", bk)
+        monkeypatch.setenv("IM2WIN_F32_TALL", "0")
     dims = layer.dims()
     x, f = workloads.make_small_integer_inputs(layer)
     y, _, _ = gpu_conv(x, f, dims, "f32")
