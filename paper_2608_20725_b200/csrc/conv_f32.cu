@@ -266,17 +266,23 @@ conv_f32_kernel(ConvF32Params q) {
 // keeps five 64-thread CTAs on an SM (206 registers uncapped: four CTAs, and 2 % slower than the 8 x 8 form
 // instead of 5 % faster; a cap of 168: spills, 30 % slower).  Every loader thread tracks BM/threads positions;
 // the offsets of the next k-block are prefetched as in the first form.
-template <int BM, int BN, int BK>
-__global__ void __maxnreg__(200)
+// 96-channel tiles: 16 x 6 per thread (channels as in the first form); KLANES as in the first form.
+template <int BM, int BN, int BK, bool KLANES>
+__global__ void __maxnreg__(BN == 96 ? 168 : 200)      // (96-channel tiles: 128 threads of 96 accumulators, three CTAs per SM)
 conv_f32_tall_kernel(ConvF32Params q) {
-  constexpr int THREADS = (BM / 16) * (BN / 8);
-  constexpr int NPOS = BM / THREADS;                       // positions per loader thread
+  constexpr int THREADS = (BM / 16) * f32_tn(BN);
+  constexpr int NPT = BN / f32_tn(BN);                     // channels per thread: 8 or 6
+  constexpr int LO = BN == 96 ? 64 : BN / 2;               // channels of the first group (four per thread)
+  constexpr int KG = BK / 8;                               // KLANES: groups of eight consecutive k per k-block
+  constexpr int NPOS = KLANES ? BK * BM / THREADS / KG : BM / THREADS;   // positions per loader thread
+  constexpr int NOFF = KLANES ? KG : BK;                   // offsets per loader thread and k-block
+  constexpr int APITCH = KLANES ? BM + 4 : BM;
   constexpr int B_VEC_PER_THREAD = BK * BN / 4 / THREADS;
-  static_assert(BM % THREADS == 0 && (BK * BN / 4) % THREADS == 0, "loader mapping");
+  static_assert((KLANES ? (THREADS / 32) * NPOS * 4 == BM : BM % THREADS == 0) && (BK * BN / 4) % THREADS == 0, "loader mapping");
   constexpr int STAGES = 3;
   extern __shared__ __align__(16) unsigned char smem_f32[];
-  float (*As)[BK][BM] = reinterpret_cast<float (*)[BK][BM]>(smem_f32);
-  float (*Bs)[BK][BN] = reinterpret_cast<float (*)[BK][BN]>(smem_f32 + sizeof(float) * STAGES * BK * BM);
+  float (*As)[BK][APITCH] = reinterpret_cast<float (*)[BK][APITCH]>(smem_f32);
+  float (*Bs)[BK][BN] = reinterpret_cast<float (*)[BK][BN]>(smem_f32 + sizeof(float) * STAGES * BK * APITCH);
 
   const int tid = threadIdx.x;
   const int tm = tid % (BM / 16);
@@ -284,11 +290,15 @@ conv_f32_tall_kernel(ConvF32Params q) {
   const int64_t m0 = (int64_t)blockIdx.x * BM;
   const int n0 = blockIdx.y * BN;
 
+  // loader: positions lm + lstep*j; (KLANES) the k's kq + 8 g of every k-block, else all of them
+  const int kq = tid & 7;
+  const int lm = KLANES ? (tid >> 5) * (NPOS * 4) + ((tid >> 3) & 3) : tid;
+  constexpr int lstep = KLANES ? 4 : THREADS;
   const float* abase[NPOS];
   uint32_t lvalid = 0;
 #pragma unroll
   for (int j = 0; j < NPOS; ++j) {
-    const int64_t lp = m0 + tid + j * THREADS;
+    const int64_t lp = m0 + lm + j * lstep;
     abase[j] = q.win;
     if (lp < q.P) {
       int64_t n;
@@ -300,21 +310,21 @@ conv_f32_tall_kernel(ConvF32Params q) {
       lvalid |= 1u << j;
     }
   }
-  int offreg[BK];
+  int offreg[NOFF];
   auto load_offsets = [&](int kb) {
 #pragma unroll
-    for (int i = 0; i < BK; ++i) offreg[i] = __ldg(q.koff + kb * BK + i);
+    for (int i = 0; i < NOFF; ++i) offreg[i] = __ldg(q.koff + kb * BK + (KLANES ? i * 8 + kq : i));
   };
   auto issue_copies = [&](int kb, int buf) {
     const int k0 = kb * BK;
 #pragma unroll
-    for (int i = 0; i < BK; ++i) {
+    for (int i = 0; i < NOFF; ++i) {
       const int off = offreg[i];
 #pragma unroll
       for (int j = 0; j < NPOS; ++j) {
         const bool ok = ((lvalid >> j) & 1u) && off >= 0;
         const float* src = ok ? abase[j] + off : q.win;
-        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&As[buf][i][tid + j * THREADS]);
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&As[buf][KLANES ? i * 8 + kq : i][lm + j * lstep]);
         asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(ok ? 4 : 0) : "memory");
       }
     }
@@ -331,11 +341,11 @@ conv_f32_tall_kernel(ConvF32Params q) {
   };
   load_offsets(0);
 
-  unsigned long long acc2[8][8];     // acc2[ip][j] = (acc[2 ip][j], acc[2 ip + 1][j]): position pairs
+  unsigned long long acc2[8][NPT];   // acc2[ip][j] = (acc[2 ip][j], acc[2 ip + 1][j]): position pairs
 #pragma unroll
   for (int i = 0; i < 8; ++i)
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc2[i][j] = 0ull;
+    for (int j = 0; j < NPT; ++j) acc2[i][j] = 0ull;
 
   const int nkb = q.Kp / BK;
 #pragma unroll
@@ -363,10 +373,16 @@ conv_f32_tall_kernel(ConvF32Params q) {
         a[2 * g] = v.x; a[2 * g + 1] = v.y;
       }
       const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][kk][tn * 4]);
-      const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][kk][BN / 2 + tn * 4]);
-      const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+      float b[8] = {b0.x, b0.y, b0.z, b0.w, 0.f, 0.f, 0.f, 0.f};
+      if (NPT == 8) {
+        const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][kk][LO + tn * 4]);
+        b[4] = b1.x; b[5] = b1.y; b[6] = b1.z; b[7] = b1.w;
+      } else {
+        const float2 b1 = *reinterpret_cast<const float2*>(&Bs[buf][kk][LO + tn * 2]);
+        b[4] = b1.x; b[5] = b1.y;
+      }
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < NPT; ++j) {
         const unsigned long long bd = dup2(b[j]);
 #pragma unroll
         for (int ip = 0; ip < 8; ++ip) ffma2(acc2[ip][j], a[ip], bd);
@@ -392,8 +408,8 @@ conv_f32_tall_kernel(ConvF32Params q) {
       while (rr[i] >= q.HoWo) { rr[i] -= q.HoWo; ++nn[i]; }
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int co = n0 + (j / 4) * (BN / 2) + tn * 4 + (j % 4);
+    for (int j = 0; j < NPT; ++j) {
+      const int co = j < 4 ? n0 + tn * 4 + j : n0 + LO + tn * (NPT - 4) + (j - 4);
       if (co >= q.Co) continue;
       const float2 lo = unpack2(acc2[2 * g][j]), hi = unpack2(acc2[2 * g + 1][j]);
       const float v[4] = {lo.x, lo.y, hi.x, hi.y};
@@ -440,15 +456,16 @@ F32Plan plan_f32(const Geometry& g) {
   // enough for the per-thread set-up of several positions not to matter (128-position tiles only)
   p.klanes = !small_m && g.s * g.Kh >= 32 && g.K >= 256;
   if (const char* v = debug_getenv("IM2WIN_F32_KLANES")) p.klanes = !small_m && v[0] == '1';   // testing aid
-  // 16 x 8 outputs per thread on 128-position tiles of 64 or 128 channels (conv_f32_tall_kernel).  Measured
+  // 16 x 8 (96-channel tiles: 16 x 6) outputs per thread on 128-position tiles (conv_f32_tall_kernel).  Measured
   // 5-6 % faster there (3x3 on 64 channels at 56x56: 597 -> 567 us; 5x5 on 96 -> 256 channels 0.75 -> 0.79 of
   // the FFMA peak, 3x3 on 64 -> 128 channels at 112x112 0.77 -> 0.815), 1-4 % slower than the 64-position tile with
-  // k-blocks of 32 where that one is planned, and slower on a reduction of 27 (two k-blocks per tile).
-  const bool tall_ok = !p.klanes && (p.bn == 128 || (p.bn == 64 && p.bm == 128));
+  // k-blocks of 32 where that one is planned, and slower on a reduction of 27 (two k-blocks per tile); the 11x11
+  // stride-4 stems with 96 output channels (k along the lanes, 16 x 6 per thread, three CTAs per SM) 0.60 -> 0.68.
+  const bool tall_ok = p.bm == 128 || (p.bn >= 96 && !p.klanes);
   p.tall = tall_ok && p.bm == 128 && g.K >= 128;
   if (const char* v = debug_getenv("IM2WIN_F32_TALL")) p.tall = tall_ok && v[0] == '1';   // testing aid
-  if (p.tall) p.bk = 16;
   if (const char* v = debug_getenv("IM2WIN_F32_BK")) { if (wide && small_m) p.bk = atoi(v) == 32 ? 32 : 16; }   // testing aid
+  if (p.tall) p.bk = 16;
   return p;
 }
 
@@ -496,9 +513,20 @@ cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, 
     }
   }
   if (p.tall) {
-    void (*tk)(ConvF32Params) = p.bn == 64 ? conv_f32_tall_kernel<128, 64, 16>
-                                           : (p.bm == 64 ? conv_f32_tall_kernel<64, 128, 16> : conv_f32_tall_kernel<128, 128, 16>);
-    const int tw = p.bn == 64 ? 11 : (p.bm == 64 ? 12 : 13);
+    void (*tk)(ConvF32Params);
+    int tw;
+    if (p.klanes) {
+      tk = p.bn == 64 ? conv_f32_tall_kernel<128, 64, 16, true>
+                      : (p.bn == 96 ? conv_f32_tall_kernel<128, 96, 16, true> : conv_f32_tall_kernel<128, 128, 16, true>);
+      tw = p.bn == 64 ? 0 : (p.bn == 96 ? 1 : 2);
+    } else if (p.bn == 96) {
+      tk = p.bm == 64 ? conv_f32_tall_kernel<64, 96, 16, false> : conv_f32_tall_kernel<128, 96, 16, false>;
+      tw = p.bm == 64 ? 3 : 4;
+    } else {
+      tk = p.bn == 64 ? conv_f32_tall_kernel<128, 64, 16, false>
+                      : (p.bm == 64 ? conv_f32_tall_kernel<64, 128, 16, false> : conv_f32_tall_kernel<128, 128, 16, false>);
+      tw = p.bn == 64 ? 11 : (p.bm == 64 ? 12 : 13);
+    }
     if (smem > 48 * 1024) {
       static bool tall_attr[64][14] = {};
       int dev = 0;
@@ -509,7 +537,7 @@ cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, 
         tall_attr[dev][tw] = true;
       }
     }
-    tk<<<grid, (p.bm / 16) * (p.bn / 8), smem, stream>>>(q);
+    tk<<<grid, (p.bm / 16) * f32_tn(p.bn), smem, stream>>>(q);
     return cudaGetLastError();
   }
   kernel<<<grid, threads, smem, stream>>>(q);
