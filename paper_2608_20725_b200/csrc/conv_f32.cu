@@ -267,7 +267,9 @@ conv_f32_kernel(ConvF32Params q) {
 // instead of 5 % faster; a cap of 168: spills, 30 % slower).  Every loader thread tracks BM/threads positions;
 // the offsets of the next k-block are prefetched as in the first form.
 // 96-channel tiles: 16 x 6 per thread (channels as in the first form); KLANES as in the first form.
-template <int BM, int BN, int BK, bool KLANES>
+// STAGED: the epilogue for outputs whose rows do not start on 16-byte boundaries (Ho*Wo no multiple of 4; a
+// kernel of its own, so that the aligned form's registers are not shared with it).
+template <int BM, int BN, int BK, bool KLANES, bool STAGED>
 __global__ void __maxnreg__(BN == 96 ? 168 : 200)      // (96-channel tiles: 128 threads of 96 accumulators, three CTAs per SM)
 conv_f32_tall_kernel(ConvF32Params q) {
   constexpr int THREADS = (BM / 16) * f32_tn(BN);
@@ -392,7 +394,61 @@ conv_f32_tall_kernel(ConvF32Params q) {
   }
 
   // positions of pair ip: group g = ip / 2, offset (ip % 2) * 2 .. + 1 inside the group's four
-  const bool vec_ok = (q.HoWo % 4) == 0;
+  constexpr bool vec_ok = true;        // (STAGED is launched exactly when Ho*Wo is no multiple of 4)
+  if (STAGED) {
+    // Ho*Wo no multiple of 4: a thread's four positions of one channel do not start on a 16-byte boundary.
+    // The tile goes through shared memory (free now) instead, one group of channels at a time, as
+    // Cs[channel][position]; every warp then streams whole rows with consecutive lanes on consecutive
+    // positions: 128 contiguous bytes per store instruction, whatever the alignment (element-wise stores
+    // straight from the registers put 4 bytes at a 16-byte stride: 0.54 against 0.60 of the FFMA peak
+    // on two 7x7 stems that differ only in this).
+    constexpr int CP = BM + 4;                             // row pitch in floats
+    static_assert((size_t)LO * CP <= (size_t)STAGES * BK * (APITCH + BN), "the staged tile fits the operand ring");
+    float* Cs = reinterpret_cast<float*>(smem_f32);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    // this thread's positions while streaming: x = lane + 32 t
+    const int lane = tid & 31, wid = tid >> 5;
+    int64_t obase[BM / 32];
+#pragma unroll
+    for (int t = 0; t < BM / 32; ++t) {
+      const int64_t pp = m0 + lane + 32 * t;
+      obase[t] = -1;
+      if (pp < q.P) {
+        int64_t n;
+        int r;
+        split_position(pp, q, n, r);
+        obase[t] = n * q.Co * q.HoWo + r;
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      constexpr int NJ0 = 4;
+      const int nj = h == 0 ? NJ0 : NPT - 4;               // channels of this thread in the group
+      const int rows = h == 0 ? LO : BN - LO;              // channels of the group
+      __syncthreads();                                     // the ring (or the previous group) has been read
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        if (jj >= nj) break;
+        const int j = h * 4 + jj;
+        const int c = tn * nj + jj;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const float2 lo = unpack2(acc2[2 * g][j]), hi = unpack2(acc2[2 * g + 1][j]);
+          *reinterpret_cast<float4*>(&Cs[c * CP + g * (BM / 4) + tm * 4]) = make_float4(lo.x, lo.y, hi.x, hi.y);
+        }
+      }
+      __syncthreads();
+      const int cbase = n0 + (h == 0 ? 0 : LO);
+      for (int c = wid; c < rows; c += THREADS / 32) {
+        const int co = cbase + c;
+        if (co >= q.Co) break;
+#pragma unroll
+        for (int t = 0; t < BM / 32; ++t)
+          if (obase[t] >= 0) q.y[obase[t] + (int64_t)co * q.HoWo] = Cs[c * CP + lane + 32 * t];
+      }
+    }
+    return;
+  }
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
     const int64_t p = m0 + g * (BM / 4) + tm * 4;
@@ -515,20 +571,22 @@ cudaError_t launch_conv_f32(const float* window, float* y, const void* scratch, 
   if (p.tall) {
     void (*tk)(ConvF32Params);
     int tw;
+    const bool st = (q.HoWo % 4) != 0;
+#define IM2WIN_TALL(BM_, BN_, KL_) (st ? conv_f32_tall_kernel<BM_, BN_, 16, KL_, true> : conv_f32_tall_kernel<BM_, BN_, 16, KL_, false>)
     if (p.klanes) {
-      tk = p.bn == 64 ? conv_f32_tall_kernel<128, 64, 16, true>
-                      : (p.bn == 96 ? conv_f32_tall_kernel<128, 96, 16, true> : conv_f32_tall_kernel<128, 128, 16, true>);
+      tk = p.bn == 64 ? IM2WIN_TALL(128, 64, true) : (p.bn == 96 ? IM2WIN_TALL(128, 96, true) : IM2WIN_TALL(128, 128, true));
       tw = p.bn == 64 ? 0 : (p.bn == 96 ? 1 : 2);
     } else if (p.bn == 96) {
-      tk = p.bm == 64 ? conv_f32_tall_kernel<64, 96, 16, false> : conv_f32_tall_kernel<128, 96, 16, false>;
+      tk = p.bm == 64 ? IM2WIN_TALL(64, 96, false) : IM2WIN_TALL(128, 96, false);
       tw = p.bm == 64 ? 3 : 4;
     } else {
-      tk = p.bn == 64 ? conv_f32_tall_kernel<128, 64, 16, false>
-                      : (p.bm == 64 ? conv_f32_tall_kernel<64, 128, 16, false> : conv_f32_tall_kernel<128, 128, 16, false>);
-      tw = p.bn == 64 ? 11 : (p.bm == 64 ? 12 : 13);
+      tk = p.bn == 64 ? IM2WIN_TALL(128, 64, false) : (p.bm == 64 ? IM2WIN_TALL(64, 128, false) : IM2WIN_TALL(128, 128, false));
+      tw = p.bn == 64 ? 5 : (p.bm == 64 ? 6 : 7);
     }
+#undef IM2WIN_TALL
+    tw = 2 * tw + (st ? 1 : 0);
     if (smem > 48 * 1024) {
-      static bool tall_attr[64][14] = {};
+      static bool tall_attr[64][16] = {};
       int dev = 0;
       if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
       if (!tall_attr[dev][tw]) {
