@@ -61,6 +61,25 @@ def test_random_layer_all_paths(layer):
 
 
 @pytest.mark.parametrize("layer", FUZZ, ids=lambda l: l.name)
+def test_random_layer_f32_tile_forms(layer, monkeypatch):
+    """The fp32 kernel's forms that only large layers take by themselves, forced on the random layers:
+    128-position tiles with the 16-position register tile (and with it the staged epilogue wherever Ho*Wo
+    is no multiple of 4, and 96-channel tiles for Co = 130 and 260), then the same with the window operand
+    gathered with k along the lanes, then 64-position tiles with k-blocks of 32."""
+    dims = layer.dims()
+    x, f = workloads.make_inputs(layer)
+    yr, ar = oracle.conv_direct(*oracle_inputs(x, f, "f32"), dims)
+    for bm, tall, klanes, bk in (("128", "1", "0", None), ("128", "1", "1", None), ("64", "0", "0", "32")):
+        monkeypatch.setenv("IM2WIN_F32_BM", bm)
+        monkeypatch.setenv("IM2WIN_F32_TALL", tall)
+        monkeypatch.setenv("IM2WIN_F32_KLANES", klanes)
+        if bk:
+            monkeypatch.setenv("IM2WIN_F32_BK", bk)
+        y, _, _ = gpu_conv(x, f, dims, "f32")
+        check_conv(y, yr, ar, "f32", f"{layer.name} bm={bm} tall={tall} klanes={klanes}")
+
+
+@pytest.mark.parametrize("layer", FUZZ, ids=lambda l: l.name)
 def test_random_layer_nhwc_paths(layer, monkeypatch):
     """The same layers through the channel-innermost (NHWC) form: the transform from both input layouts
     bit for bit, the convolution through the kernel the library picks and through each of its two
