@@ -1343,12 +1343,19 @@ transform_nhwc_from_nhwc_small_c_kernel(const uint16_t* __restrict__ x, uint4* _
 // fastest), so consecutive threads write consecutive bytes of a column.  Every input element is
 // read once and transposed once; blocks of rows outside the image only write zeros.  Indices are
 // kept in mixed-radix counters (no division per element).
-template <int VEC>
+// SWZ (Cp/8 a power of two): rows of T are Cp halves apart (no padding) and the 16-byte chunk c8 of row r sits at
+// chunk c8 ^ ((r / VEC) & 7): the transposing stores of a warp (lanes on different column groups) still spread
+// over the banks, and phase 2 reads a chunk with ONE 16-byte load and finds (k, chunk) with a shift and a mask
+// (with the odd pitch Cp + 2 a chunk is only 4-byte aligned: four loads, and mixed-radix counters per chunk).
+template <int VEC, bool SWZ>
 __global__ void __launch_bounds__(256)
 transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ win, int C, int Cp, int H, int W,
                                 int Ho, int Wp, int Kh, int s, int p, int kc, int kchunks, int R, int rgroups) {
-  extern __shared__ __align__(16) uint16_t rows_s[];     // T[kc][Cp + 2]
-  const int PC = Cp + 2;
+  extern __shared__ __align__(16) uint16_t rows_s[];     // T[kc][Cp + 2], or (SWZ) T[kc][Cp] with swizzled chunks
+  const int PC = SWZ ? Cp : Cp + 2;
+  const int smask = SWZ ? ((Cp / 8 < 8 ? Cp / 8 : 8) - 1) : 0;
+  // element index of channel c of row r in T
+  auto tidx = [&](int r, int c) { return SWZ ? r * PC + ((((c >> 3) ^ ((r / VEC) & smask)) << 3) | (c & 7)) : r * PC + c; };
   // block -> (image n, group of R consecutive rows of the padded input, column chunk); 32-bit
   // arithmetic (the host keeps the block count below 2^31): the set-up is paid by every thread of
   // every block, and a block's own work is only a few instructions per thread and row
@@ -1392,7 +1399,7 @@ transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __rest
         const int extra = Cp - C;
         for (int i = threadIdx.x; i < nw * extra; i += step) {
           const int r = i / extra, e = i - r * extra;
-          rows_s[r * PC + C + e] = 0;
+          rows_s[tidx(r, C + e)] = 0;
         }
       }
       // phase 1 (W, w0 and nw are multiples of VEC): two VEC*2-byte loads (the second channel's only
@@ -1407,7 +1414,7 @@ transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __rest
           dsts[j] = -1;
           if (i0 + j * step < items) {
             const int c = 2 * cp;
-            dsts[j] = (VEC * col) * PC + c;
+            dsts[j] = tidx(VEC * col, c);            // (rows VEC*col .. + VEC - 1 share the swizzle: + t*PC below)
             const uint16_t* src = xrow + c * cstride + VEC * col;
             r0[j] = __ldg(reinterpret_cast<const V*>(src));
             if (c + 1 < C) r1[j] = __ldg(reinterpret_cast<const V*>(src + cstride));
@@ -1434,6 +1441,16 @@ transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __rest
       const int u = hp - ho * s;
       // chunk (k, oct) of strip (n, ho): ((k*Kh + u)*Cp + 8*oct) halves into the strip
       uint16_t* strip = win + ((n * Ho + ho) * (int64_t)Wp) * Kh * Cp + (int64_t)u * Cp;
+      if (SWZ) {
+        const int lo = 31 - __clz(octs);                  // octs is a power of two
+        for (int j = threadIdx.x; j < chunks; j += step) {
+          const int k = k_lo + (j >> lo), oct = j & (octs - 1);
+          uint4 v = make_uint4(0u, 0u, 0u, 0u);
+          const int r = k - p - w0;
+          if (row_ok && r >= 0 && r < nw) v = *reinterpret_cast<const uint4*>(rows_s + tidx(r, 8 * oct));
+          *reinterpret_cast<uint4*>(strip + (int64_t)k * Kh * Cp + 8 * oct) = v;
+        }
+      } else {
       int k = k_first, oct = oct_first;
       for (int j = threadIdx.x; j < chunks; j += step) {
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -1445,6 +1462,7 @@ transform_nhwc_from_nchw_kernel(const uint16_t* __restrict__ x, uint16_t* __rest
         *reinterpret_cast<uint4*>(strip + (int64_t)k * Kh * Cp + 8 * oct) = v;
         oct += d_o; k += d_k;
         if (oct >= octs) { oct -= octs; ++k; }
+      }
       }
     }
   }
@@ -2092,7 +2110,10 @@ cudaError_t launch_transform_nhwc(const uint16_t* x, int x_is_nhwc, uint16_t* wi
     return cudaGetLastError();
   }
   // columns per block: the whole row when it fits 48 KB of shared memory as T[w][Cp + 2]
-  const int64_t per_col = (int64_t)(plan.Cp + 2) * 2;
+  const int octs = plan.Cp / 8;
+  bool swz = (octs & (octs - 1)) == 0;                     // chunks found by shift and mask, swizzled rows without padding
+  if (const char* v = debug_getenv("IM2WIN_NHWC_TRANSFORM_SWZ")) swz = swz && v[0] != '0';   // testing aid
+  const int64_t per_col = (int64_t)(plan.Cp + (swz ? 0 : 2)) * 2;
   int kc = (int)((48 * 1024) / per_col);
   if (kc < 8) return cudaErrorInvalidValue;
   if (kc > g.W) kc = g.W;
@@ -2111,13 +2132,20 @@ cudaError_t launch_transform_nhwc(const uint16_t* x, int x_is_nhwc, uint16_t* wi
   const int64_t blocks = (int64_t)g.N * rgroups * kchunks;
   if (blocks >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
   const size_t smem = (size_t)(per_col * kc);
-#define IM2WIN_LAUNCH_T(V)                                                                                          \
-  transform_nhwc_from_nchw_kernel<V><<<(unsigned)blocks, 256, smem, stream>>>(x, window, g.C, plan.Cp, g.H, g.W, g.Ho, \
-                                                                            g.Wp, g.Kh, g.s, g.p, kc, kchunks, R, rgroups)
-  if (vec == 8) IM2WIN_LAUNCH_T(8);
-  else if (vec == 4) IM2WIN_LAUNCH_T(4);
-  else if (vec == 2) IM2WIN_LAUNCH_T(2);
-  else IM2WIN_LAUNCH_T(1);
+#define IM2WIN_LAUNCH_T(V, S)                                                                                       \
+  transform_nhwc_from_nchw_kernel<V, S><<<(unsigned)blocks, 256, smem, stream>>>(x, window, g.C, plan.Cp, g.H, g.W, g.Ho, \
+                                                                               g.Wp, g.Kh, g.s, g.p, kc, kchunks, R, rgroups)
+  if (swz) {
+    if (vec == 8) IM2WIN_LAUNCH_T(8, true);
+    else if (vec == 4) IM2WIN_LAUNCH_T(4, true);
+    else if (vec == 2) IM2WIN_LAUNCH_T(2, true);
+    else IM2WIN_LAUNCH_T(1, true);
+  } else {
+    if (vec == 8) IM2WIN_LAUNCH_T(8, false);
+    else if (vec == 4) IM2WIN_LAUNCH_T(4, false);
+    else if (vec == 2) IM2WIN_LAUNCH_T(2, false);
+    else IM2WIN_LAUNCH_T(1, false);
+  }
 #undef IM2WIN_LAUNCH_T
   return cudaGetLastError();
 }

@@ -42,14 +42,17 @@ SMALL = [
 
 
 @pytest.mark.parametrize("layer", SMALL, ids=lambda l: l.name)
-@pytest.mark.parametrize("layout,variant", [("nchw", "default"), ("nchw", "rows"), ("nchw", "rows3"), ("nhwc", "default"),
-                                            ("nhwc", "chunks")])
+@pytest.mark.parametrize("layout,variant", [("nchw", "default"), ("nchw", "rows"), ("nchw", "rows3"), ("nchw", "padded"),
+                                            ("nhwc", "default"), ("nhwc", "chunks")])
 def test_transform_nhwc_bit_exact(layer, layout, variant, monkeypatch):
     """From either input layout; from NCHW through the kernel the library picks (one block per strip
     for up to 8 channels, else blocks of input rows) and through the per-row kernel forced, with
     one and with three rows per block; from NHWC through the kernel the library picks (one block per
     strip when the channel count is a multiple of 8) and through the chunk-per-thread kernel forced."""
-    if variant == "chunks":
+    if variant == "padded":               # the per-row kernel's padded shared-memory rows instead of swizzled ones
+        monkeypatch.setenv("IM2WIN_NHWC_TRANSFORM", "rows")
+        monkeypatch.setenv("IM2WIN_NHWC_TRANSFORM_SWZ", "0")
+    elif variant == "chunks":
         monkeypatch.setenv("IM2WIN_NHWC_TRANSFORM", "chunks")
     elif variant != "default":
         monkeypatch.setenv("IM2WIN_NHWC_TRANSFORM", "rows")
