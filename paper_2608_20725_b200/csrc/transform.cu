@@ -350,7 +350,15 @@ bool plan_strips(const Geometry& g, StripParams* q, size_t* smem_bytes, int* vec
   const int64_t strip_bytes = g.strip * ES;
   const int64_t total_strips = (int64_t)g.N * g.C * g.Ho;
   if (strip_bytes > 64 * 1024 || total_strips >= ((int64_t)1 << 31)) return false;
-  int r = (int)(16384 / strip_bytes);
+  // Staged output per CTA.  A CTA's life is one round of loads, a barrier and one bulk store, so with 16 KB
+  // per CTA the kernel was bound by CTA turnaround, most visibly on short strips of tall kernels (11x11 on
+  // 28x28 images in fp16: 836-byte strips, 24 k CTAs, 123 us; 93 us with 48 KB).  Measured per config: 32 KB
+  // is 1-4 % faster than 16 KB nearly everywhere, 48 KB (just under the default shared-memory limit) wins in
+  // fp16 for kernels 7 and 11 high (cfg3 54 -> 44 us, cfg5k7 79 -> 61) and for large images (3x3 at 112x112:
+  // 339 -> 291 us) and loses 5-7 % on 28x28 images with 5x5 kernels and on 7x7 images.
+  int64_t stage_bytes = (ES == 2 && (g.Kh >= 7 || (int64_t)g.H * g.W >= 2048)) ? 48 * 1024 - 64 : 32 * 1024;
+  if (const char* v = debug_getenv("IM2WIN_TRANSFORM_STAGE")) { const int64_t b = atoll(v); if (b >= 4096 && b <= 160 * 1024) stage_bytes = b; }   // testing aid
+  int r = (int)(stage_bytes / strip_bytes);
   if (r < 1) r = 1;
   q->H = g.H; q->W = g.W; q->Wp = g.Wp; q->Kh = g.Kh; q->s = g.s; q->p = g.p; q->Ho = g.Ho;
   q->L = (int32_t)g.strip;
@@ -418,8 +426,11 @@ cudaError_t launch_typed(const void* x, void* window, const Geometry& g, cudaStr
   TransformParams q;
   q.H = g.H; q.W = g.W; q.Wp = g.Wp; q.Kh = g.Kh; q.s = g.s; q.p = g.p; q.Ho = g.Ho;
   q.total_cols = (int64_t)g.N * g.C * g.Ho * g.Wp;
-  // about 16 KB of staged output per CTA, in whole columns, a multiple of 8 columns
-  int cols = (int)(16384 / (g.Kh * sizeof(E)));
+  // about 32 KB of staged output per CTA (16 KB: 2-9 % slower, CTA turnaround; 48 KB: slower again), in whole
+  // columns, a multiple of 8 columns
+  int64_t stage_bytes = 32768;
+  if (const char* v = debug_getenv("IM2WIN_TRANSFORM_STAGE")) { const int64_t b = atoll(v); if (b >= 4096 && b <= 160 * 1024) stage_bytes = b; }   // testing aid
+  int cols = (int)(stage_bytes / (g.Kh * sizeof(E)));
   cols = cols / 8 * 8;
   if (cols < 8) cols = 8;
   q.cols_per_cta = cols;
